@@ -1,0 +1,194 @@
+"""fp64 CPU oracle for tree-verify attention.  TEST INFRASTRUCTURE ONLY.
+
+Only the tests, the smoke check and the benchmark's CPU-baseline leg may import
+this file; the product (the CUDA library and its binding) never does, and this
+file imports nothing from the product.  It is deliberately plain and slow.
+
+What it computes (every function names the passage of the paper it follows):
+
+* The tree attention mask of Sec. 2 ("Tree Attention", the mask(A) equation): a
+  query node may see key node j exactly when j is one of its ancestors.  As in
+  ordinary causal attention (same paragraph) a token also sees itself, so the
+  visible set of node i is A(i) = {i} + ancestors(i).
+* Parallel verification (Sec. 2, "Speculative Decoding"; App. C: the prompt is
+  part of the attention mask): every tree token is scored by the target model
+  as if its root-to-node path had been decoded after the prefix, i.e. node i
+  attends to all prefix rows and to the tree rows in A(i):
+
+      s_t = scale * <q[i,h,:], k[t,h_kv,:]>,  p = softmax_t over visible t,
+      o[i,h,:] = sum_t p_t * v[t,h_kv,:],     h_kv = h // (H_q / H_kv).
+
+  The method reaches exactly this result (it is not an approximation), so the
+  oracle is this definition written out with a dense boolean mask, in fp64.
+
+Parity status: every function below is pinned by tests/test_oracle_pins.py
+(chain == library causal attention, star == prefix+self, brute force per path
+in pure Python, closed forms, hand-written mask fixture, relabelling
+invariance).  Nothing here is "parity unpinned".
+
+Readings where the paper is silent: scale = 1/sqrt(head_dim); consecutive query
+heads share a KV head; tree K/V rows follow the prefix rows in node order;
+masks are packed LSB-first in uint32 words.
+"""
+from __future__ import annotations
+
+import math
+from typing import List, Sequence
+
+import numpy as np
+
+
+def bf16_bits_to_f64(bits: np.ndarray) -> np.ndarray:
+    """Exact widening: a bf16 value is the top 16 bits of an IEEE fp32."""
+    b = np.ascontiguousarray(bits, dtype=np.uint16).astype(np.uint32) << np.uint32(16)
+    return b.view(np.float32).astype(np.float64)
+
+
+def check_parents(parents: Sequence[int]) -> None:
+    """A valid parent array has parents[i] == -1 (a root) or 0 <= parents[i] < i."""
+    for i, p in enumerate(parents):
+        p = int(p)
+        if p < -1 or p >= i:
+            raise ValueError(f"parents[{i}] = {p} is not in {{-1}} U [0, {i})")
+
+
+def visible_nodes(parents: Sequence[int], i: int) -> List[int]:
+    """A(i): node i followed by its ancestors, found by walking the parent links (Sec. 2, mask(A))."""
+    out = []
+    j = int(i)
+    while j != -1:
+        out.append(j)
+        j = int(parents[j])
+    return out
+
+
+def tree_mask_matrix(parents: Sequence[int]) -> np.ndarray:
+    """Boolean [n][n]; entry [i][j] is True iff query node i may attend to key node j (j in A(i))."""
+    check_parents(parents)
+    n = len(parents)
+    m = np.zeros((n, n), dtype=bool)
+    for i in range(n):
+        for j in visible_nodes(parents, i):
+            m[i, j] = True
+    return m
+
+
+def build_tree_mask(parents: Sequence[int], words_per_row: int):
+    """Packed ancestor bitmasks and depths.
+
+    bits[i][w] has bit b (LSB = bit 0) set iff node 32*w + b is in A(i); unused bits are 0.
+    depth[i] = number of ancestors of i (roots have depth 0).
+    """
+    check_parents(parents)
+    n = len(parents)
+    if 32 * words_per_row < n:
+        raise ValueError("words_per_row too small")
+    bits = np.zeros((n, words_per_row), dtype=np.uint32)
+    depths = np.zeros(n, dtype=np.int32)
+    for i in range(n):
+        vis = visible_nodes(parents, i)
+        for j in vis:
+            bits[i, j // 32] |= np.uint32(1 << (j % 32))
+        depths[i] = len(vis) - 1
+    return bits, depths
+
+
+def tree_attention(q_bits, k_bits, v_bits, prefix_len: int, parents: Sequence[int], scale: float | None = None):
+    """Tree-verify attention for one request, fp64.
+
+    q_bits [n][H_q][D], k_bits / v_bits [prefix_len + n][H_kv][D] (bf16 bit patterns; tree row j
+    sits at row prefix_len + j).  Returns float64 [n][H_q][D].
+    """
+    q = bf16_bits_to_f64(q_bits)
+    k = bf16_bits_to_f64(k_bits)
+    v = bf16_bits_to_f64(v_bits)
+    n, hq, d = q.shape
+    rows, hkv, dk = k.shape
+    L = int(prefix_len)
+    if rows != L + n or dk != d or v.shape != k.shape or hq % hkv != 0 or len(parents) != n:
+        raise ValueError("inconsistent shapes")
+    if scale is None or scale <= 0:
+        scale = 1.0 / math.sqrt(d)
+    g = hq // hkv
+    allowed = np.ones((n, L + n), dtype=bool)           # prefix: always visible
+    allowed[:, L:] = tree_mask_matrix(parents)          # tree block: ancestors and self
+    out = np.zeros((n, hq, d), dtype=np.float64)
+    for h in range(hq):
+        kh = k[:, h // g, :]
+        vh = v[:, h // g, :]
+        s = scale * (q[:, h, :] @ kh.T)                 # [n][L+n]
+        s = np.where(allowed, s, -np.inf)
+        s = s - s.max(axis=1, keepdims=True)
+        p = np.exp(s)
+        p = p / p.sum(axis=1, keepdims=True)
+        out[:, h, :] = p @ vh
+    return out
+
+
+def tree_attention_nodes(q_bits, k_bits, v_bits, prefix_len: int, parents: Sequence[int], nodes: Sequence[int],
+                         scale: float | None = None):
+    """The same definition evaluated only for the query nodes listed in `nodes` -> float64 [len(nodes)][H_q][D].
+
+    Used to check sampled outputs at sizes where all rows would take too long.
+    """
+    check_parents(parents)
+    L = int(prefix_len)
+    nodes = [int(i) for i in nodes]
+    q = bf16_bits_to_f64(np.asarray(q_bits)[nodes])
+    k = bf16_bits_to_f64(k_bits)
+    v = bf16_bits_to_f64(v_bits)
+    m, hq, d = q.shape
+    hkv = k.shape[1]
+    if scale is None or scale <= 0:
+        scale = 1.0 / math.sqrt(d)
+    g = hq // hkv
+    out = np.zeros((m, hq, d), dtype=np.float64)
+    for a, i in enumerate(nodes):
+        rows = list(range(L)) + [L + j for j in sorted(visible_nodes(parents, i))]
+        for h in range(hq):
+            kh = k[rows, h // g, :]
+            vh = v[rows, h // g, :]
+            s = scale * (kh @ q[a, h, :])
+            p = np.exp(s - s.max())
+            out[a, h, :] = (p / p.sum()) @ vh
+    return out
+
+
+def tree_attention_ragged(q_bits, k_bits, v_bits, prefix_len, n_nodes, kv_row_offset, parents_list,
+                          scale: float | None = None):
+    """Ragged batch: requests are independent; request r owns q rows node_offsets[r]..., kv rows
+    kv_row_offset[r] .. + prefix_len[r] + n_nodes[r].  Returns float64 [sum n][H_q][D]."""
+    outs = []
+    qo = 0
+    for r in range(len(prefix_len)):
+        n = int(n_nodes[r])
+        o = int(kv_row_offset[r])
+        rows = int(prefix_len[r]) + n
+        if n:
+            outs.append(tree_attention(q_bits[qo:qo + n], k_bits[o:o + rows], v_bits[o:o + rows],
+                                       int(prefix_len[r]), parents_list[r], scale))
+        qo += n
+    if not outs:
+        return np.zeros((0,) + tuple(q_bits.shape[1:]), dtype=np.float64)
+    return np.concatenate(outs, axis=0)
+
+
+def build_tree_mask_ragged(parents_list, words_per_row: int):
+    """Masks and depths of every request, rows concatenated in request order."""
+    bits, depths = [], []
+    for p in parents_list:
+        b, dpt = build_tree_mask(p, words_per_row)
+        bits.append(b)
+        depths.append(dpt)
+    if not bits:
+        return np.zeros((0, words_per_row), np.uint32), np.zeros(0, np.int32)
+    return np.concatenate(bits, axis=0), np.concatenate(depths)
+
+
+def visible_pair_count(prefix_len, parents_list) -> int:
+    """Sum over nodes of (prefix_len + depth + 1): the number of (query, key) pairs the definition uses."""
+    total = 0
+    for L, p in zip(prefix_len, parents_list):
+        for i in range(len(p)):
+            total += int(L) + len(visible_nodes(p, i))
+    return total

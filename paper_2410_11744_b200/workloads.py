@@ -1,0 +1,185 @@
+"""Seeded synthetic inputs for tree-verify attention.
+
+This module only *draws inputs*: draft-tree topologies, prefix lengths and random
+bf16 Q/K/V tensors shaped like the Llama2-7B / Llama2-70B attention layers the
+paper evaluates (Sec. 5.1; App. C.1 uses 64 heads x head_dim 128).  It holds
+none of the method's arithmetic (no masks, no attention) and is used by the
+tests, the benchmark and the oracle-side scripts alike.  It imports neither the
+CUDA binding nor the oracle.
+
+Tree recipe: a deterministic-score form of the paper's greedy expansion
+(Sec. 4.1-4.2, Algorithm 1; weight model of App. D): node 0 is the root (parent
+-1, score 1).  When a node is created it draws p ~ Dirichlet(alpha * 1_c) and
+pushes its c candidate children with score(node) * p_j on a max-heap; the best
+candidate is popped and becomes the next node, so parent[i] < i, until n nodes
+exist.  Ties: higher score first, then earlier push.
+
+bf16 values are carried as uint16 bit patterns (numpy has no bf16 type).
+"""
+from __future__ import annotations
+
+import heapq
+import math
+from dataclasses import dataclass, field
+from typing import List
+
+import numpy as np
+
+MASTER_SEED = 241011744
+
+
+def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
+    """Round fp32 to bf16 (round-to-nearest-even) and return the uint16 bit patterns.
+
+    Input generation only: the values fed to both implementations are these bits.
+    """
+    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)   # finite inputs: no uint32 overflow below
+    r = (u + np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1))) >> np.uint32(16)
+    return r.astype(np.uint16)
+
+
+def greedy_tree(rng: np.random.Generator, n_nodes: int, n_candidates: int, alpha: float) -> np.ndarray:
+    """Parent array (int32, parents[0] = -1, parents[i] < i) of a greedy best-first tree."""
+    parents = np.full(n_nodes, -1, dtype=np.int32)
+    if n_nodes == 0:
+        return parents
+    heap: list = []
+    push_id = 0
+
+    def expand(node: int, log_score: float) -> None:
+        nonlocal push_id
+        p = rng.dirichlet(np.full(n_candidates, alpha, dtype=np.float64))
+        for j in range(n_candidates):
+            lp = math.log(p[j]) if p[j] > 0.0 else -math.inf
+            heapq.heappush(heap, (-(log_score + lp), push_id, node))
+            push_id += 1
+
+    expand(0, 0.0)
+    for i in range(1, n_nodes):
+        neg_log_score, _, parent = heapq.heappop(heap)
+        parents[i] = parent
+        expand(i, -neg_log_score)
+    return parents
+
+
+def chain_tree(n_nodes: int) -> np.ndarray:
+    return np.arange(-1, n_nodes - 1, dtype=np.int32)
+
+
+def star_forest(n_nodes: int) -> np.ndarray:
+    """Every node is its own root (parent -1)."""
+    return np.full(n_nodes, -1, dtype=np.int32)
+
+
+def random_tree(rng: np.random.Generator, n_nodes: int, p_root: float = 0.0) -> np.ndarray:
+    """Uniform random recursive tree / forest with parents[i] < i."""
+    parents = np.full(n_nodes, -1, dtype=np.int32)
+    for i in range(1, n_nodes):
+        if rng.random() >= p_root:
+            parents[i] = int(rng.integers(0, i))
+    return parents
+
+
+@dataclass
+class Workload:
+    """One ragged batch of verification requests (all arrays host-side numpy)."""
+    name: str
+    n_q_heads: int
+    n_kv_heads: int
+    head_dim: int
+    prefix_len: np.ndarray          # int32 [n_req]
+    n_nodes: np.ndarray             # int32 [n_req]
+    parents: List[np.ndarray]       # per request int32 [n_nodes[r]], request-local indices
+    q: np.ndarray                   # uint16 bf16 bits [sum n_nodes][H_q][D]
+    k: np.ndarray                   # uint16 bf16 bits [total_rows][H_kv][D]
+    v: np.ndarray                   # same layout as k
+    kv_row_offset: np.ndarray       # int64 [n_req]: row of request r's token 0 in k / v
+    meta: dict = field(default_factory=dict)
+
+    @property
+    def n_req(self) -> int:
+        return int(self.prefix_len.shape[0])
+
+    @property
+    def node_offsets(self) -> np.ndarray:
+        return np.concatenate([[0], np.cumsum(self.n_nodes)]).astype(np.int32)
+
+    @property
+    def parents_concat(self) -> np.ndarray:
+        if len(self.parents) == 0:
+            return np.zeros(0, dtype=np.int32)
+        return np.concatenate(self.parents).astype(np.int32)
+
+    @property
+    def total_nodes(self) -> int:
+        return int(self.n_nodes.sum())
+
+    @property
+    def scale(self) -> float:
+        return 1.0 / math.sqrt(self.head_dim)
+
+    def request(self, r: int):
+        """(q, k, v, parents, prefix_len) slices of request r; k/v hold prefix rows then tree rows."""
+        no = self.node_offsets
+        o = int(self.kv_row_offset[r])
+        rows = int(self.prefix_len[r]) + int(self.n_nodes[r])
+        return (self.q[no[r]:no[r + 1]], self.k[o:o + rows], self.v[o:o + rows],
+                self.parents[r], int(self.prefix_len[r]))
+
+
+def _normal_bf16(rng: np.random.Generator, shape) -> np.ndarray:
+    return f32_to_bf16_bits(rng.standard_normal(size=shape, dtype=np.float32))
+
+
+def assemble(name, rng, n_q_heads, n_kv_heads, head_dim, prefix_len, parents_list, meta=None) -> Workload:
+    """Draw Q, K, V ~ N(0,1) (in that order) for given trees and prefix lengths, requests packed back to back."""
+    prefix_len = np.asarray(prefix_len, dtype=np.int32)
+    n_nodes = np.asarray([len(p) for p in parents_list], dtype=np.int32)
+    rows = prefix_len.astype(np.int64) + n_nodes.astype(np.int64)
+    kv_off = np.concatenate([[0], np.cumsum(rows)[:-1]]).astype(np.int64) if len(rows) else np.zeros(0, np.int64)
+    total_rows = int(rows.sum())
+    total_nodes = int(n_nodes.sum())
+    q = _normal_bf16(rng, (total_nodes, n_q_heads, head_dim))
+    k = _normal_bf16(rng, (total_rows, n_kv_heads, head_dim))
+    v = _normal_bf16(rng, (total_rows, n_kv_heads, head_dim))
+    return Workload(name, n_q_heads, n_kv_heads, head_dim, prefix_len, n_nodes,
+                    [np.asarray(p, dtype=np.int32) for p in parents_list], q, k, v, kv_off, meta or {})
+
+
+# Shapes of the five benchmark configurations: (H_q, H_kv, D, prefix_len, n_nodes, candidates, alpha).
+_FIXED = {
+    1: dict(name="c1_tiny_4x4_d64_L128_n16", hq=4, hkv=4, d=64, L=128, n=16, c=4, alpha=0.3),
+    2: dict(name="c2_llama2_7b_L1024_n64", hq=32, hkv=32, d=128, L=1024, n=64, c=8, alpha=0.3),
+    3: dict(name="c3_llama2_7b_L4096_n256", hq=32, hkv=32, d=128, L=4096, n=256, c=8, alpha=0.1),
+    4: dict(name="c4_llama2_70b_L2048_n512", hq=64, hkv=8, d=128, L=2048, n=512, c=8, alpha=0.3),
+}
+
+
+def make_config(index: int, seed: int | None = None) -> Workload:
+    """Config `index` in 1..5 (1 = tiny ... 5 = ragged batch of 8 Llama2-70B-shaped requests)."""
+    if seed is None:
+        seed = MASTER_SEED + index
+    rng = np.random.default_rng(seed)
+    if index in _FIXED:
+        c = _FIXED[index]
+        parents = greedy_tree(rng, c["n"], c["c"], c["alpha"])
+        return assemble(c["name"], rng, c["hq"], c["hkv"], c["d"], [c["L"]], [parents],
+                        dict(config=index, seed=seed, candidates=c["c"], alpha=[c["alpha"]]))
+    if index == 5:
+        n_req = 8
+        Ls, ns, alphas, trees = [], [], [], []
+        for _ in range(n_req):
+            L = int(round(math.exp(rng.uniform(math.log(512.0), math.log(8192.0)))))
+            n = int(rng.integers(32, 769))
+            a = float(rng.uniform(0.05, 1.0))
+            Ls.append(L); ns.append(n); alphas.append(a)
+            trees.append(greedy_tree(rng, n, 8, a))
+        return assemble("c5_ragged8_llama2_70b", rng, 64, 8, 128, Ls, trees,
+                        dict(config=5, seed=seed, candidates=8, alpha=alphas))
+    raise ValueError(f"config index must be 1..5, got {index}")
+
+
+def make_custom(seed: int, n_q_heads: int, n_kv_heads: int, head_dim: int, prefix_len, parents_list,
+                name: str = "custom") -> Workload:
+    return assemble(name, np.random.default_rng(seed), n_q_heads, n_kv_heads, head_dim, prefix_len, parents_list,
+                    dict(seed=seed))
