@@ -1,0 +1,406 @@
+#!/usr/bin/env python
+"""Benchmark of the tree-verify attention hot path (mask build + tree attention + split-KV combine).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config 2] [--no-per-config]
+
+Prints ONE JSON line.  A step is one pass of the whole hot path over one synthetic batch (default:
+the Llama2-7B-shaped config 2).  Inputs are resident in HBM; between steps the path rotates through
+enough independent copies of (Q, K, V, out) that no step finds its inputs in L2.  `e2e` repeats the
+measurement with host buffers (pinned), copies inside the timed region.  `--impl reference` times the
+fp64 CPU oracle instead (rank 0 only).  With N > 1 (torchrun) every rank runs an independent replica:
+the path has no exchange step.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "tree_verify_attention_tree_tokens_per_s"
+UNIT = "tree tokens/s"
+L2_BYTES = 126 * 1024 * 1024
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return p, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+def algorithmic_cost(w, words_per_row):
+    """Bytes: K and V once, Q in, O out, mask rows.  Flops: 4*D per visible (query, key) pair per head."""
+    D, hq, hkv = w.head_dim, w.n_q_heads, w.n_kv_heads
+    rows = int((w.prefix_len.astype(np.int64) + w.n_nodes).sum())
+    n = w.total_nodes
+    nbytes = 2 * rows * hkv * D * 2 + 2 * n * hq * D * 2 + n * words_per_row * 4
+    pairs = 0
+    for L, p in zip(w.prefix_len, w.parents):
+        depth = np.zeros(len(p), dtype=np.int64)
+        for i in range(len(p)):
+            depth[i] = 0 if p[i] < 0 else depth[p[i]] + 1
+        pairs += int((int(L) + depth + 1).sum())
+    flops = 4 * hq * D * pairs
+    return nbytes, flops
+
+
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(gpu_index), f"--query-gpu={self.QUERY}",
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
+                                         stdout=self.file, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def lines(self):
+        try:
+            with open(self.file.name) as f:
+                return [ln.strip() for ln in f if ln.strip()]
+        except Exception:
+            return []
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+        lines = self.lines()
+        try:
+            os.unlink(self.file.name)
+        except Exception:
+            pass
+        return lines
+
+    @staticmethod
+    def summarise(lines, note=""):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "note": "nvidia-smi gave no samples"}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                "samples": len(sm), "note": note}
+
+
+def dist_env():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+def oracle_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        n = 1
+    try:
+        n = min(n, len(os.sched_getaffinity(0)))
+    except Exception:
+        pass
+    return n
+
+
+def time_oracle(w, budget_s=12.0, max_passes=20):
+    """The oracle as it stands on this workload: whole passes (mask + attention) until ~budget_s is used."""
+    from oracle import dyspec_oracle as orc
+    W = 4 * ((max(int(w.n_nodes.max()), 1) + 127) // 128)
+    times = []
+    t_start = time.perf_counter()
+    while len(times) < max_passes and (not times or time.perf_counter() - t_start < budget_s):
+        t0 = time.perf_counter()
+        orc.build_tree_mask_ragged(w.parents, W)
+        orc.tree_attention_ragged(w.q, w.k, w.v, w.prefix_len, w.n_nodes, w.kv_row_offset, w.parents)
+        times.append(time.perf_counter() - t0)
+    return times
+
+
+def run_reference(args):
+    rank, world, _ = dist_env()
+    if rank != 0:
+        return
+    from paper_2410_11744_b200 import workloads
+    w = workloads.make_config(args.config)
+    for _ in range(min(args.warmup, 2)):
+        time_oracle(w, budget_s=0.0, max_passes=1)
+    steps = max(1, args.steps)
+    budget = 120.0
+    times = []
+    t_begin = time.perf_counter()
+    for _ in range(steps):
+        times += time_oracle(w, budget_s=0.0, max_passes=1)
+        if time.perf_counter() - t_begin > budget:
+            break
+    sec = sum(times) / len(times)
+    value = w.total_nodes / sec
+    cores = oracle_threads()
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": len(times),
+        "warmup": min(args.warmup, 2), "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "note": "fp64 numpy oracle, one full pass (mask + attention) per step"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": f"{len(times)} full passes of {w.name}"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def measure_config(torch, runner, w, steps, warmup, device, with_events=True):
+    """Device-resident timing of `steps` steps, rotating over copies larger than L2."""
+    first = runner.DeviceBatch(w, device=device)
+    nbytes, flops = algorithmic_cost(w, first.W)
+    copies = max(2, min(64, int(np.ceil(2.0 * L2_BYTES / max(nbytes, 1)))))
+    batches = [first] + [runner.DeviceBatch(w, device=device) for _ in range(copies - 1)]
+    info = first.plan.describe()
+    launches_per_step = 1 + 1 + (1 if info["split_groups"] > 0 else 0)
+    stream = torch.cuda.current_stream()
+    for i in range(max(warmup, 3)):
+        batches[i % copies].step()
+    torch.cuda.synchronize()
+    # pass 1: whole region, two events
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(steps):
+        batches[i % copies].step()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    total_ms = e0.elapsed_time(e1)
+    # pass 2: per-call events around the attention call (main kernel + combine) and the mask kernel
+    attn_ms, mask_ms = None, None
+    if with_events:
+        k = min(steps, 200)
+        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(k)]
+        for i in range(k):
+            b = batches[i % copies]
+            evs[i][0].record(stream)
+            b.build_mask()
+            evs[i][1].record(stream)
+            b.attention()
+            evs[i][2].record(stream)
+        torch.cuda.synchronize()
+        mask_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in evs)
+        attn_ms = statistics.mean(e[1].elapsed_time(e[2]) for e in evs)
+    status = int(first.status.item())
+    return dict(batches=batches, total_ms=total_ms, ms_per_step=total_ms / steps, attn_ms=attn_ms, mask_ms=mask_ms,
+                bytes=nbytes, flops=flops, copies=copies, info=info, launches_per_step=launches_per_step, status=status)
+
+
+def roofline_entry(m, peaks, peaks_kind):
+    t_hbm = m["bytes"] / (peaks["hbm_gbs"] * 1e9)
+    t_tc = m["flops"] / (peaks["bf16_tflops"] * 1e12)
+    dur = (m["attn_ms"] if m["attn_ms"] is not None else m["ms_per_step"]) * 1e-3
+    if t_hbm >= t_tc:
+        ach = m["bytes"] / dur / 1e9
+        return {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],
+                "traffic": None, "peak_kind": peaks_kind, "kernel": "tree attention call (main kernel + combine)",
+                "launch_us": dur * 1e6}
+    ach = m["flops"] / dur / 1e12
+    return {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+            "frac": ach / peaks["bf16_tflops"], "traffic": None, "peak_kind": peaks_kind + " (burst)",
+            "kernel": "tree attention call (main kernel + combine)", "launch_us": dur * 1e6}
+
+
+def run_ours(args):
+    import torch
+    rank, world, local = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback for the CUDA path)")
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    use_dist = world > 1
+    if use_dist:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+    from paper_2410_11744_b200 import build as _build
+    if rank == 0:
+        _build.build()
+    if use_dist:
+        dist.barrier()
+    from paper_2410_11744_b200 import runner, workloads
+
+    peaks, peaks_kind = load_peaks()
+    w = workloads.make_config(args.config)
+    sampler = ClockSampler(local) if rank == 0 else None
+
+    def barrier():
+        if use_dist:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident measurement (the headline `value`)
+    barrier()
+    m = measure_config(torch, runner, w, args.steps, args.warmup, device)
+    barrier()
+    n_lines_after_timed = len(sampler.lines()) if sampler else 0
+    ms = torch.tensor([m["total_ms"]], dtype=torch.float64, device=device)
+    if use_dist:
+        dist.all_reduce(ms, op=dist.ReduceOp.MAX)
+    total_ms = float(ms.item())
+    tokens_per_step = w.total_nodes * world
+    value = tokens_per_step * args.steps / (total_ms * 1e-3)
+
+    # ---- clocks: the timed region can be shorter than one nvidia-smi period; if so keep the same
+    #      loop running (untimed) until a few samples exist, and say so.
+    clocks_note = "sampled during warm-up + timed region"
+    if sampler:
+        if n_lines_after_timed < 4:
+            t_end = time.time() + 1.0
+            while time.time() < t_end:
+                for i in range(200):
+                    m["batches"][i % m["copies"]].step()
+                torch.cuda.synchronize()
+            clocks_note = "timed region shorter than the sampling period: sampled while the same loop kept running"
+        clocks = ClockSampler.summarise(sampler.lines(), clocks_note)
+    else:
+        clocks = None
+
+    # ---- end to end through the C ABI with host buffers (pinned), copies inside the timed region
+    b0 = m["batches"][0]
+    host_in = [t.cpu().pin_memory() for t in (b0.parents, b0.q, b0.k, b0.v)]
+    host_out = torch.empty_like(b0.out, device="cpu").pin_memory()
+    h2d = sum(t.numel() * t.element_size() for t in host_in)
+    d2h = host_out.numel() * host_out.element_size()
+    e2e_steps = max(3, min(args.steps, 200))
+    stream = torch.cuda.current_stream()
+
+    def e2e_step(b):
+        b.parents.copy_(host_in[0], non_blocking=True)
+        b.q.copy_(host_in[1], non_blocking=True)
+        b.k.copy_(host_in[2], non_blocking=True)
+        b.v.copy_(host_in[3], non_blocking=True)
+        b.step()
+        host_out.copy_(b.out, non_blocking=True)
+        stream.synchronize()
+
+    for i in range(3):
+        e2e_step(m["batches"][i % m["copies"]])
+    barrier()
+    t0 = time.perf_counter()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(e2e_steps):
+        e2e_step(m["batches"][i % m["copies"]])
+    e1.record(stream)
+    torch.cuda.synchronize()
+    e2e_ms = max(e0.elapsed_time(e1), (time.perf_counter() - t0) * 1e3)
+    ems = torch.tensor([e2e_ms], dtype=torch.float64, device=device)
+    if use_dist:
+        dist.all_reduce(ems, op=dist.ReduceOp.MAX)
+    e2e_value = tokens_per_step * e2e_steps / (float(ems.item()) * 1e-3)
+
+    if rank != 0:
+        if use_dist:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
+
+    roof = roofline_entry(m, peaks, peaks_kind)
+    traffic_path = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(traffic_path):
+        try:
+            with open(traffic_path) as f:
+                roof["traffic"] = json.load(f).get(w.name)
+        except Exception:
+            pass
+
+    # ---- the other configs, same protocol, fewer steps (reported for context in `per_config`)
+    per_config = []
+    if not args.no_per_config:
+        for idx in (1, 2, 3, 4, 5):
+            wi = w if idx == args.config else workloads.make_config(idx)
+            mi = m if idx == args.config else measure_config(torch, runner, wi, min(args.steps, 300), args.warmup, device)
+            ri = roofline_entry(mi, peaks, peaks_kind)
+            per_config.append({"config": idx, "workload": wi.name, "tree_tokens": wi.total_nodes,
+                               "step_us": mi["ms_per_step"] * 1e3, "attention_call_us": mi["attn_ms"] * 1e3,
+                               "mask_us": mi["mask_ms"] * 1e3, "tokens_per_s": wi.total_nodes / (mi["ms_per_step"] * 1e-3),
+                               "bytes": mi["bytes"], "flops": mi["flops"], "bound": ri["bound"], "achieved": ri["achieved"],
+                               "unit": ri["unit"], "frac": ri["frac"], "plan": mi["info"], "status": mi["status"]})
+            if idx != args.config:
+                del mi["batches"]
+                torch.cuda.empty_cache()
+
+    # ---- the oracle on the host cores, bounded sample of the same workload
+    times = time_oracle(w, budget_s=12.0)
+    cpu_sec = sum(times) / len(times)
+    cpu_baseline = {"value": w.total_nodes / cpu_sec, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
+                    "sample": f"{len(times)} full passes (mask + attention) of {w.name}, {cpu_sec * 1e3:.1f} ms each"}
+
+    if sampler:
+        sampler.stop()
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "n_q_heads": w.n_q_heads, "n_kv_heads": w.n_kv_heads, "head_dim": w.head_dim,
+                   "prefix_len": w.prefix_len.tolist(), "n_nodes": w.n_nodes.tolist(), "parallelism": "replicas only",
+                   "l2": f"inputs rotate over {m['copies']} independent copies ({m['copies'] * m['bytes'] / 1e6:.0f} MB > 2x L2)",
+                   "step": "mask build + tree attention + split-KV combine", "plan": m["info"]},
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+        "gpu_launches": m["launches_per_step"] * args.steps,
+        "roofline": roof,
+        "cpu_baseline": cpu_baseline,
+        "kernel_us": {"mask_build": m["mask_ms"] * 1e3, "attention_call": m["attn_ms"] * 1e3},
+        "device_status": m["status"],
+    }
+    if per_config:
+        line["per_config"] = per_config
+    print(json.dumps(line), flush=True)
+    if use_dist:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=2)
+    ap.add_argument("--no-per-config", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,163 @@
+/*
+ * dyspec.h -- C ABI of the B200 (sm_100a) tree-verify attention library.
+ *
+ * The library implements the hot path of one DySpec decoding step: the target model's
+ * verification pass over a draft token tree (paper Sec. 2, "Speculative Decoding" and
+ * "Tree Attention"; App. C "Efficiency of Optimized Tree Attention").  Every tree node is a
+ * query; it attends to the whole prefix KV cache plus the tree rows of its ancestors and itself.
+ *
+ * Conventions shared by all calls
+ *   - Every function returns an int: DYSPEC_OK (0) or a negative DYSPEC_ERR_* code.  Nothing
+ *     throws, aborts or traps.  Errors the host can see (NULL pointers, unsupported shapes, small
+ *     workspace, misaligned pointers) are returned before anything is launched.
+ *   - Pointers marked "dev" are CUDA device pointers of the current device; pointers marked
+ *     "host" are ordinary host pointers that are only read during the call.
+ *   - The caller owns every buffer.  Attention and mask calls enqueue kernels on `stream` and
+ *     return without synchronising; the caller's buffers must stay alive until the stream reaches
+ *     them.  Plan creation/destruction are the only calls that allocate or free device memory.
+ *   - Conditions only the device can see (a parent index that is not in {-1} U [0, i); a bounded
+ *     wait that ran out) store a non-zero DYSPEC_ERR_* code into the optional `status` word (dev
+ *     int32, the caller zeroes it) and the kernel still completes normally.
+ *   - bf16 tensors are passed as `const void*`; layouts are row-major with the last index fastest.
+ *
+ * Packed rows: ancestor_bits[i][w], w < words_per_row, has bit b (LSB = bit 0) set iff tree node
+ * 32*w + b is node i itself or an ancestor of node i (Sec. 2, the mask(A) equation, plus the self
+ * bit of causal attention).  Unused bits are zero.  words_per_row is a multiple of 4 (16-byte rows).
+ */
+#ifndef DYSPEC_H_
+#define DYSPEC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct CUstream_st* dyspec_stream_t; /* a cudaStream_t */
+
+enum {
+  DYSPEC_OK = 0,
+  DYSPEC_ERR_INVALID_ARG = -1, /* NULL / negative / inconsistent argument */
+  DYSPEC_ERR_UNSUPPORTED = -2, /* shape outside the supported set (see dyspec_plan_create) */
+  DYSPEC_ERR_WORKSPACE = -3,   /* workspace smaller than dyspec_plan_workspace_bytes, or misaligned */
+  DYSPEC_ERR_CUDA = -4,        /* a CUDA runtime / driver call failed (launch, tensor-map encode, alloc) */
+  DYSPEC_ERR_BAD_TREE = -5,    /* device-detected: some parents[i] outside {-1} U [0, i) */
+  DYSPEC_ERR_TIMEOUT = -6      /* device-detected: a bounded in-kernel wait ran out */
+};
+
+#define DYSPEC_MAX_NODES 1024 /* largest tree per request (the paper's largest real tree is 768, Sec. 5 / App. B) */
+
+/* Static, never-freed description of an error code. */
+const char* dyspec_error_string(int code);
+
+/* Library version, major*10000 + minor*100 + patch. */
+int dyspec_version(void);
+
+/* Smallest legal words_per_row for trees of up to max_nodes nodes: 4*ceil(max_nodes/128); <0 on bad input. */
+int dyspec_words_per_row(int max_nodes);
+
+/*
+ * (1) Mask builder, single request (Sec. 2, mask(A): "i is ancestor of j").
+ *   parents        dev  int32 [n_nodes]   parents[i] = -1 (a root) or an index < i
+ *   ancestor_bits  dev  uint32 [n_nodes][words_per_row]  (written; 16-byte aligned)
+ *   depths         dev  int32 [n_nodes] or NULL           (written: number of ancestors)
+ *   status         dev  int32 [1] or NULL                 (DYSPEC_ERR_BAD_TREE stored on a bad parent;
+ *                                                          such a node is treated as a root)
+ * n_nodes = 0 is a no-op.  n_nodes > DYSPEC_MAX_NODES or 32*words_per_row < n_nodes is rejected.
+ */
+int dyspec_build_tree_mask(const int32_t* parents, int n_nodes, uint32_t* ancestor_bits, int32_t* depths,
+                           int words_per_row, int32_t* status, dyspec_stream_t stream);
+
+/*
+ * (2) Plans.  A plan fixes the static shape and the ragged batch structure, runs the host-side
+ * scheduler (work list of (request, kv-head, query-tile, kv-split) items balanced over the SMs)
+ * and owns a small device copy of that list.  Create it once per batch structure; reuse it for
+ * every layer and step with the same (prefix_len, n_nodes).
+ *
+ *   n_q_heads, n_kv_heads  H_q, H_kv; group g = H_q / H_kv must be 1, 2, 4 or 8
+ *   head_dim               64 or 128
+ *   n_req                  number of requests (>= 0)
+ *   prefix_len   host int32 [n_req]   L_r >= 0
+ *   n_nodes      host int32 [n_req]   0 <= n_r <= DYSPEC_MAX_NODES
+ *   kv_row_offset host int64 [n_req]  row of request r's token 0 in k_cache / v_cache; request r
+ *                                     occupies rows off_r .. off_r + L_r + n_r - 1: prefix rows first,
+ *                                     then one row per tree node in node order
+ *   kv_total_rows          number of rows of k_cache / v_cache (>= every off_r + L_r + n_r)
+ *   words_per_row          row stride of ancestor_bits, a multiple of 4 with 32*W >= max n_r
+ *   scale                  softmax scale; <= 0 selects 1/sqrt(head_dim)
+ * Query/output rows of request r start at node_offset_r = n_0 + ... + n_{r-1}; so do its mask rows
+ * and parents.
+ */
+typedef struct dyspec_plan dyspec_plan_t;
+
+int dyspec_plan_create(dyspec_plan_t** plan, int n_q_heads, int n_kv_heads, int head_dim, int n_req,
+                       const int32_t* prefix_len, const int32_t* n_nodes, const int64_t* kv_row_offset,
+                       int64_t kv_total_rows, int words_per_row, float scale);
+int dyspec_plan_destroy(dyspec_plan_t* plan);
+
+/* Bytes of scratch the attention call needs (split-KV partials + arrival counters); may be 0. */
+size_t dyspec_plan_workspace_bytes(const dyspec_plan_t* plan);
+
+/* Scheduler introspection (for tests and benchmarks): field 0 = work items, 1 = CTAs launched,
+ * 2 = query-tile groups, 3 = groups that are split, 4 = max splits of a group, 5 = kernel regime
+ * (0 = warp-level mma tiles, 1 = tcgen05 tiles), 6 = total key tiles, 7 = query rows per tile. */
+int64_t dyspec_plan_info(const dyspec_plan_t* plan, int field);
+
+/* Host-only view of the scheduler, for tests and tools: validates the arguments and schedules exactly
+ * as dyspec_plan_create does (requests packed back to back in the cache) but makes no CUDA call.
+ * Copies up to max_items work items into items_out (host, 8 int32 each: request, kv head, first
+ * packed query row, first key tile, one-past-last key tile, partial slot or -1, group id, number of
+ * splits of the group), the per-CTA item ranges into cta_begin_out (host, n_ctas + 1 entries, at most
+ * max_ctas) and, into info_out (host int64 [10]), the eight dyspec_plan_info fields followed by keys
+ * per tile and workspace bytes.  Any output pointer may be NULL.  Returns the item count or an error. */
+int dyspec_schedule_dry_run(int n_q_heads, int n_kv_heads, int head_dim, int n_req, const int32_t* prefix_len,
+                            const int32_t* n_nodes, int words_per_row, int32_t* items_out, int max_items,
+                            int32_t* cta_begin_out, int max_ctas, int64_t* info_out);
+
+/* Testing knobs, read when a plan is created: force the regime (-1 = automatic) and the number of
+ * CTAs the scheduler balances over (<= 0 = automatic). */
+int dyspec_set_tuning(int force_regime, int force_ctas);
+
+/*
+ * (1b) Mask builder for the whole ragged batch of a plan: request r's parents (request-local
+ * indices) start at node_offset_r, its mask rows and depths likewise.
+ *   parents dev int32 [sum n_r]; ancestor_bits dev uint32 [sum n_r][W]; depths dev int32 [sum n_r] or NULL;
+ *   status dev int32 [1] or NULL.
+ */
+int dyspec_plan_build_tree_mask(const dyspec_plan_t* plan, const int32_t* parents, uint32_t* ancestor_bits,
+                                int32_t* depths, int32_t* status, dyspec_stream_t stream);
+
+/*
+ * (3) Tree-verify attention over a ragged batch (Sec. 2 "Tree Attention"; App. C: the prompt is
+ * part of the mask, so prefix keys are visible to every node).  For request r, query head h,
+ * node i:  out[i,h,:] = softmax_t(scale * <q[i,h,:], k[t,h/g,:]>) . v[t,h/g,:]  over
+ * t in {prefix rows} U {tree rows of the nodes whose bit is set in ancestor_bits[i]}.
+ * bf16 inputs, fp32 scores / softmax / accumulation, bf16 (round-to-nearest-even) output.
+ *   q              dev bf16 [sum n_r][H_q][D]            (16-byte aligned)
+ *   k_cache,v_cache dev bf16 [kv_total_rows][H_kv][D]    (16-byte aligned)
+ *   ancestor_bits  dev uint32 [sum n_r][W]               (from the mask builder)
+ *   out            dev bf16 [sum n_r][H_q][D]            (written)
+ *   workspace      dev, >= dyspec_plan_workspace_bytes(plan), 256-byte aligned; its arrival counters
+ *                  must be zero before the first call (dyspec_plan_create's caller zeroes it once;
+ *                  the kernels leave them zero).  Two calls that overlap on the GPU need two workspaces.
+ *   status         dev int32 [1] or NULL
+ */
+int dyspec_tree_attention_ragged(const dyspec_plan_t* plan, const void* q, const void* k_cache, const void* v_cache,
+                                 const uint32_t* ancestor_bits, void* out, void* workspace, size_t workspace_bytes,
+                                 int32_t* status, dyspec_stream_t stream);
+
+/*
+ * (3b) Single-request convenience form.  The static shape comes from dyspec_set_default_shape;
+ * plans and workspaces for each (prefix_len, n_nodes) seen are created on first use and cached
+ * inside the library (that first call allocates; later calls do not).  k_cache / v_cache hold
+ * exactly prefix_len + n_nodes rows.
+ */
+int dyspec_set_default_shape(int n_q_heads, int n_kv_heads, int head_dim, int words_per_row, float scale);
+int dyspec_tree_attention(const void* q, const void* k_cache, const void* v_cache, int prefix_len,
+                          const uint32_t* ancestor_bits, int n_nodes, void* out, dyspec_stream_t stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DYSPEC_H_ */

@@ -1,0 +1,202 @@
+"""Thin ctypes binding of libdyspec.so: argument marshalling only.
+
+Every function has the name of the C entry point it calls (see include/dyspec.h) and passes raw
+device pointers of torch tensors plus the current CUDA stream.  All arithmetic happens in the CUDA
+kernels of the library; there is no fallback: if the library has not been built, importing this
+module raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libdyspec.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} is missing: build it with `python -m paper_2410_11744_b200.build` "
+        "(there is no CPU or PyTorch fallback for the CUDA path)")
+
+lib = ctypes.CDLL(LIB_PATH)
+
+_c = ctypes
+_vp, _i32, _i64, _sz, _f32 = _c.c_void_p, _c.c_int, _c.c_int64, _c.c_size_t, _c.c_float
+
+# name -> (restype, argtypes); mirrors include/dyspec.h one to one
+SIGNATURES = {
+    "dyspec_error_string": (_c.c_char_p, [_i32]),
+    "dyspec_version": (_i32, []),
+    "dyspec_words_per_row": (_i32, [_i32]),
+    "dyspec_set_tuning": (_i32, [_i32, _i32]),
+    "dyspec_build_tree_mask": (_i32, [_vp, _i32, _vp, _vp, _i32, _vp, _vp]),
+    "dyspec_plan_create": (_i32, [_c.POINTER(_vp), _i32, _i32, _i32, _i32, _vp, _vp, _vp, _i64, _i32, _f32]),
+    "dyspec_plan_destroy": (_i32, [_vp]),
+    "dyspec_plan_workspace_bytes": (_sz, [_vp]),
+    "dyspec_plan_info": (_i64, [_vp, _i32]),
+    "dyspec_schedule_dry_run": (_i32, [_i32, _i32, _i32, _i32, _vp, _vp, _i32, _vp, _i32, _vp, _i32, _vp]),
+    "dyspec_plan_build_tree_mask": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp]),
+    "dyspec_tree_attention_ragged": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp, _vp]),
+    "dyspec_set_default_shape": (_i32, [_i32, _i32, _i32, _i32, _f32]),
+    "dyspec_tree_attention": (_i32, [_vp, _vp, _vp, _i32, _vp, _i32, _vp, _vp]),
+}
+for _name, (_res, _args) in SIGNATURES.items():
+    _fn = getattr(lib, _name)
+    _fn.restype = _res
+    _fn.argtypes = _args
+
+
+class DyspecError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {dyspec_error_string(code)} ({code})")
+
+
+def _check(code: int, where: str) -> None:
+    if code != 0:
+        raise DyspecError(code, where)
+
+
+def _ptr(t) -> Optional[int]:
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    return t.data_ptr()
+
+
+def _stream(stream=None) -> int:
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(stream, int):
+        return stream
+    return stream.cuda_stream
+
+
+def dyspec_error_string(code: int) -> str:
+    return lib.dyspec_error_string(code).decode()
+
+
+def dyspec_version() -> int:
+    return lib.dyspec_version()
+
+
+def dyspec_words_per_row(max_nodes: int) -> int:
+    return lib.dyspec_words_per_row(max_nodes)
+
+
+def dyspec_set_tuning(force_regime: int = -1, force_ctas: int = 0) -> None:
+    _check(lib.dyspec_set_tuning(force_regime, force_ctas), "dyspec_set_tuning")
+
+
+def dyspec_build_tree_mask(parents, n_nodes: int, ancestor_bits, depths=None, words_per_row: int = 0,
+                           status=None, stream=None) -> None:
+    """parents: int32 device tensor [n]; ancestor_bits: int32/uint32 device tensor [n][W]; depths: int32 [n] or None."""
+    _check(lib.dyspec_build_tree_mask(_ptr(parents), n_nodes, _ptr(ancestor_bits), _ptr(depths), words_per_row,
+                                      _ptr(status), _stream(stream)), "dyspec_build_tree_mask")
+
+
+class Plan:
+    """Owns a dyspec_plan_t*: static shape + ragged batch structure + scheduled work list."""
+
+    def __init__(self, n_q_heads: int, n_kv_heads: int, head_dim: int, prefix_len: Sequence[int],
+                 n_nodes: Sequence[int], kv_row_offset: Sequence[int], kv_total_rows: int, words_per_row: int,
+                 scale: float = 0.0):
+        n_req = len(prefix_len)
+        pl = (_c.c_int32 * max(1, n_req))(*[int(x) for x in prefix_len])
+        nn = (_c.c_int32 * max(1, n_req))(*[int(x) for x in n_nodes])
+        off = (_c.c_int64 * max(1, n_req))(*[int(x) for x in kv_row_offset])
+        handle = _vp()
+        _check(lib.dyspec_plan_create(_c.byref(handle), n_q_heads, n_kv_heads, head_dim, n_req,
+                                      _c.cast(pl, _vp), _c.cast(nn, _vp), _c.cast(off, _vp), int(kv_total_rows),
+                                      words_per_row, float(scale)), "dyspec_plan_create")
+        self.handle = handle
+        self.words_per_row = words_per_row
+        self.total_nodes = int(sum(int(x) for x in n_nodes))
+
+    def workspace_bytes(self) -> int:
+        return int(lib.dyspec_plan_workspace_bytes(self.handle))
+
+    def info(self, field: int) -> int:
+        return int(lib.dyspec_plan_info(self.handle, field))
+
+    def describe(self) -> dict:
+        names = ["items", "ctas", "groups", "split_groups", "max_splits", "regime", "key_tiles", "rows_per_tile"]
+        return {k: self.info(i) for i, k in enumerate(names)}
+
+    def destroy(self) -> None:
+        if self.handle:
+            lib.dyspec_plan_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+
+def dyspec_plan_create(*args, **kwargs) -> Plan:
+    return Plan(*args, **kwargs)
+
+
+def dyspec_plan_destroy(plan: Plan) -> None:
+    plan.destroy()
+
+
+def dyspec_plan_workspace_bytes(plan: Plan) -> int:
+    return plan.workspace_bytes()
+
+
+def dyspec_plan_info(plan: Plan, field: int) -> int:
+    return plan.info(field)
+
+
+def dyspec_schedule_dry_run(n_q_heads: int, n_kv_heads: int, head_dim: int, prefix_len: Sequence[int],
+                            n_nodes: Sequence[int], words_per_row: int, max_items: int = 1 << 16):
+    """Host-only scheduler run -> (items int32 [n][8], cta_begin int32 [n_ctas + 1], info dict)."""
+    import numpy as np
+    n_req = len(prefix_len)
+    pl = np.asarray(list(prefix_len) or [0], dtype=np.int32)
+    nn = np.asarray(list(n_nodes) or [0], dtype=np.int32)
+    items = np.zeros((max_items, 8), dtype=np.int32)
+    cta = np.zeros(max_items + 1, dtype=np.int32)
+    info = np.zeros(10, dtype=np.int64)
+    rc = lib.dyspec_schedule_dry_run(n_q_heads, n_kv_heads, head_dim, n_req, pl.ctypes.data, nn.ctypes.data,
+                                     words_per_row, items.ctypes.data, max_items, cta.ctypes.data, max_items + 1,
+                                     info.ctypes.data)
+    if rc < 0:
+        raise DyspecError(rc, "dyspec_schedule_dry_run")
+    if rc > max_items:
+        return dyspec_schedule_dry_run(n_q_heads, n_kv_heads, head_dim, prefix_len, n_nodes, words_per_row, rc)
+    names = ["items", "ctas", "groups", "split_groups", "max_splits", "regime", "key_tiles", "rows_per_tile",
+             "keys_per_tile", "workspace_bytes"]
+    d = {k: int(v) for k, v in zip(names, info)}
+    return items[:rc].copy(), cta[:d["ctas"] + 1].copy(), d
+
+
+def dyspec_plan_build_tree_mask(plan: Plan, parents, ancestor_bits, depths=None, status=None, stream=None) -> None:
+    _check(lib.dyspec_plan_build_tree_mask(plan.handle, _ptr(parents), _ptr(ancestor_bits), _ptr(depths),
+                                           _ptr(status), _stream(stream)), "dyspec_plan_build_tree_mask")
+
+
+def dyspec_tree_attention_ragged(plan: Plan, q, k_cache, v_cache, ancestor_bits, out, workspace=None,
+                                 workspace_bytes: Optional[int] = None, status=None, stream=None) -> None:
+    if workspace_bytes is None:
+        workspace_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(lib.dyspec_tree_attention_ragged(plan.handle, _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(ancestor_bits),
+                                            _ptr(out), _ptr(workspace), workspace_bytes, _ptr(status),
+                                            _stream(stream)), "dyspec_tree_attention_ragged")
+
+
+def dyspec_set_default_shape(n_q_heads: int, n_kv_heads: int, head_dim: int, words_per_row: int,
+                             scale: float = 0.0) -> None:
+    _check(lib.dyspec_set_default_shape(n_q_heads, n_kv_heads, head_dim, words_per_row, float(scale)),
+           "dyspec_set_default_shape")
+
+
+def dyspec_tree_attention(q, k_cache, v_cache, prefix_len: int, ancestor_bits, n_nodes: int, out, stream=None) -> None:
+    _check(lib.dyspec_tree_attention(_ptr(q), _ptr(k_cache), _ptr(v_cache), prefix_len, _ptr(ancestor_bits), n_nodes,
+                                     _ptr(out), _stream(stream)), "dyspec_tree_attention")

@@ -1,0 +1,458 @@
+// C ABI of the tree-verify attention library: argument checks, the host-side ragged scheduler
+// (plan), TMA tensor-map encoding and kernel launches.  See include/dyspec.h for the contract.
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <map>
+#include <mutex>
+#include <new>
+#include <tuple>
+#include <vector>
+
+#include "common.cuh"
+
+namespace dyspec {
+// kernels (defined in the other translation units)
+cudaError_t launch_build_tree_mask(const int32_t* parents, const ReqInfo* reqs, int n_req, int single_n,
+                                   uint32_t* bits, int32_t* depths, int W, int32_t* status, cudaStream_t stream);
+cudaError_t launch_attn_mma(int head_dim, int n_ctas, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
+                            const AttnParams& p, cudaStream_t stream);
+cudaError_t launch_combine(int head_dim, int bm, int n_split_groups, const AttnParams& p, cudaStream_t stream);
+cudaError_t launch_attn_tc(int head_dim, int n_ctas, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
+                           const AttnParams& p, cudaStream_t stream);
+}  // namespace dyspec
+
+using namespace dyspec;
+
+namespace {
+
+int g_force_regime = -1;
+int g_force_ctas = 0;
+
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  });
+  return fn;
+}
+
+// bf16 tensor [rows][heads][D] viewed as (D, heads, rows); box = (64, box_heads, box_rows), 128-byte swizzle.
+bool encode_map(CUtensorMap* map, const void* base, int64_t rows, int heads, int D, int box_heads, int box_rows) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return false;
+  if (rows <= 0) rows = 1;
+  const cuuint64_t dims[3] = {cuuint64_t(D), cuuint64_t(heads), cuuint64_t(rows)};
+  const cuuint64_t strides[2] = {cuuint64_t(D) * 2, cuuint64_t(heads) * D * 2};
+  const cuuint32_t box[3] = {64u, cuuint32_t(box_heads), cuuint32_t(box_rows)};
+  const cuuint32_t estr[3] = {1u, 1u, 1u};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+}  // namespace
+
+struct dyspec_plan {
+  int hq = 0, hkv = 0, d = 0, g = 1, log2g = 0, W = 0;
+  float scale = 0.f;
+  int n_req = 0;
+  int64_t kv_total_rows = 0;
+  int64_t total_nodes = 0;
+  int regime = 0, bm = 64, bn = 64;
+  std::vector<ReqInfo> reqs;
+  std::vector<WorkItem> items;
+  std::vector<int32_t> cta_begin;
+  std::vector<GroupInfo> split_groups;
+  int n_ctas = 0, n_slots = 0, max_splits = 1;
+  int64_t total_tiles = 0, n_groups = 0;
+  // device copies (one allocation)
+  void* d_blob = nullptr;
+  ReqInfo* d_reqs = nullptr;
+  WorkItem* d_items = nullptr;
+  int32_t* d_cta_begin = nullptr;
+  GroupInfo* d_groups = nullptr;
+  int32_t* d_counters = nullptr;
+  size_t workspace_bytes = 0;
+};
+
+namespace {
+
+// Host scheduler: cut the (request, kv head, query tile) groups' key-tile lists into work items
+// and deal them to CTAs so that every CTA gets about the same number of key tiles (plus a fixed
+// per-item cost for the Q load and the epilogue).  A group that ends up in several items is a
+// split-KV group: its items write fp32 partials that the combine step merges.
+void schedule(dyspec_plan& pl) {
+  const int bm = pl.bm, bn = pl.bn, g = pl.g;
+  const int nodes_per_tile = bm / g;
+  struct Group { int req, kvh, row0, tiles; };
+  std::vector<Group> groups;
+  int64_t total_tiles = 0;
+  for (int r = 0; r < pl.n_req; ++r) {
+    const ReqInfo& rq = pl.reqs[r];
+    if (rq.n_nodes == 0) continue;
+    const int prefix_tiles = (rq.prefix_len + bn - 1) / bn;
+    const int q_tiles = (rq.n_nodes + nodes_per_tile - 1) / nodes_per_tile;
+    for (int kvh = 0; kvh < pl.hkv; ++kvh)
+      for (int qt = 0; qt < q_tiles; ++qt) {
+        // parents[i] < i: a node only sees tree columns <= its own index, so tree tiles past the
+        // tile's last node are never needed.
+        const int last_node = std::min(rq.n_nodes, (qt + 1) * nodes_per_tile);
+        const int tiles = prefix_tiles + (last_node + bn - 1) / bn;
+        groups.push_back({r, kvh, qt * bm, tiles});
+        total_tiles += tiles;
+      }
+  }
+  pl.total_tiles = total_tiles;
+  pl.n_groups = int64_t(groups.size());
+  pl.items.clear();
+  pl.cta_begin.clear();
+  pl.split_groups.clear();
+  pl.n_slots = 0;
+  pl.max_splits = 1;
+  if (groups.empty()) { pl.n_ctas = 0; pl.cta_begin.push_back(0); return; }
+
+  const int ctas_per_sm = pl.regime == 0 ? 2 : 1;
+  int max_ctas = g_force_ctas > 0 ? g_force_ctas : kNumSMs * ctas_per_sm;
+  const int item_cost = 1;                               // fixed per-item overhead, in key tiles
+  const int min_tiles = pl.regime == 0 ? 2 : 2;          // smallest piece worth a split
+  const int64_t total_cost = total_tiles + int64_t(groups.size()) * item_cost;
+  int64_t target = (total_cost + max_ctas - 1) / max_ctas;
+  if (target < item_cost + min_tiles) target = item_cost + min_tiles;
+
+  int64_t used = 0;
+  pl.cta_begin.push_back(0);
+  for (size_t gi = 0; gi < groups.size(); ++gi) {
+    const Group& gr = groups[gi];
+    const size_t first_item = pl.items.size();
+    int begin = 0;
+    while (begin < gr.tiles) {
+      int64_t room = target - used;
+      if (room < item_cost + min_tiles && used > 0) {
+        pl.cta_begin.push_back(int32_t(pl.items.size()));
+        used = 0;
+        room = target;
+      }
+      int take = int(std::min<int64_t>(gr.tiles - begin, room - item_cost));
+      const int rem = gr.tiles - begin - take;
+      if (rem > 0 && rem < min_tiles) take = gr.tiles - begin;
+      WorkItem it{};
+      it.req = gr.req; it.kv_head = gr.kvh; it.row0 = gr.row0;
+      it.tile_begin = begin; it.tile_end = begin + take;
+      it.slot = -1; it.group = int(gi); it.n_splits = 1;
+      pl.items.push_back(it);
+      used += take + item_cost;
+      begin += take;
+    }
+    const int n_splits = int(pl.items.size() - first_item);
+    if (n_splits > 1) {
+      GroupInfo info{};
+      info.req = gr.req; info.kv_head = gr.kvh; info.row0 = gr.row0;
+      info.slot0 = pl.n_slots; info.n_splits = n_splits;
+      for (int s = 0; s < n_splits; ++s) {
+        pl.items[first_item + s].slot = pl.n_slots + s;
+        pl.items[first_item + s].n_splits = n_splits;
+        pl.items[first_item + s].group = int(pl.split_groups.size());
+      }
+      pl.n_slots += n_splits;
+      pl.max_splits = std::max(pl.max_splits, n_splits);
+      pl.split_groups.push_back(info);
+    }
+  }
+  pl.cta_begin.push_back(int32_t(pl.items.size()));
+  pl.n_ctas = int(pl.cta_begin.size()) - 1;
+}
+
+int upload(dyspec_plan& pl) {
+  auto pad = [](size_t x) { return (x + 255) & ~size_t(255); };
+  const size_t b_reqs = pad(std::max<size_t>(1, pl.reqs.size()) * sizeof(ReqInfo));
+  const size_t b_items = pad(std::max<size_t>(1, pl.items.size()) * sizeof(WorkItem));
+  const size_t b_cta = pad(pl.cta_begin.size() * sizeof(int32_t));
+  const size_t b_groups = pad(std::max<size_t>(1, pl.split_groups.size()) * sizeof(GroupInfo));
+  const size_t b_counters = pad(std::max<size_t>(1, pl.split_groups.size()) * sizeof(int32_t));
+  const size_t total = b_reqs + b_items + b_cta + b_groups + b_counters;
+  std::vector<uint8_t> host(total, 0);
+  size_t off = 0;
+  if (!pl.reqs.empty()) memcpy(host.data() + off, pl.reqs.data(), pl.reqs.size() * sizeof(ReqInfo));
+  const size_t o_reqs = off; off += b_reqs;
+  if (!pl.items.empty()) memcpy(host.data() + off, pl.items.data(), pl.items.size() * sizeof(WorkItem));
+  const size_t o_items = off; off += b_items;
+  memcpy(host.data() + off, pl.cta_begin.data(), pl.cta_begin.size() * sizeof(int32_t));
+  const size_t o_cta = off; off += b_cta;
+  if (!pl.split_groups.empty()) memcpy(host.data() + off, pl.split_groups.data(), pl.split_groups.size() * sizeof(GroupInfo));
+  const size_t o_groups = off; off += b_groups;
+  const size_t o_counters = off;
+  if (cudaMalloc(&pl.d_blob, total) != cudaSuccess) { pl.d_blob = nullptr; return DYSPEC_ERR_CUDA; }
+  if (cudaMemcpy(pl.d_blob, host.data(), total, cudaMemcpyHostToDevice) != cudaSuccess) return DYSPEC_ERR_CUDA;
+  uint8_t* base = static_cast<uint8_t*>(pl.d_blob);
+  pl.d_reqs = reinterpret_cast<ReqInfo*>(base + o_reqs);
+  pl.d_items = reinterpret_cast<WorkItem*>(base + o_items);
+  pl.d_cta_begin = reinterpret_cast<int32_t*>(base + o_cta);
+  pl.d_groups = reinterpret_cast<GroupInfo*>(base + o_groups);
+  pl.d_counters = reinterpret_cast<int32_t*>(base + o_counters);
+  return DYSPEC_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* dyspec_error_string(int code) {
+  switch (code) {
+    case DYSPEC_OK: return "ok";
+    case DYSPEC_ERR_INVALID_ARG: return "invalid argument";
+    case DYSPEC_ERR_UNSUPPORTED: return "unsupported shape";
+    case DYSPEC_ERR_WORKSPACE: return "workspace too small or misaligned";
+    case DYSPEC_ERR_CUDA: return "CUDA call failed";
+    case DYSPEC_ERR_BAD_TREE: return "parent index outside {-1} U [0, i)";
+    case DYSPEC_ERR_TIMEOUT: return "bounded in-kernel wait ran out";
+    default: return "unknown error code";
+  }
+}
+
+int dyspec_version(void) { return 100; }
+
+int dyspec_words_per_row(int max_nodes) {
+  if (max_nodes < 0 || max_nodes > DYSPEC_MAX_NODES) return DYSPEC_ERR_INVALID_ARG;
+  if (max_nodes == 0) return 4;
+  return 4 * ((max_nodes + 127) / 128);
+}
+
+int dyspec_set_tuning(int force_regime, int force_ctas) {
+  if (force_regime < -1 || force_regime > 1) return DYSPEC_ERR_INVALID_ARG;
+  g_force_regime = force_regime;
+  g_force_ctas = force_ctas;
+  return DYSPEC_OK;
+}
+
+int dyspec_build_tree_mask(const int32_t* parents, int n_nodes, uint32_t* ancestor_bits, int32_t* depths,
+                           int words_per_row, int32_t* status, dyspec_stream_t stream) {
+  if (n_nodes < 0 || words_per_row <= 0 || (words_per_row & 3)) return DYSPEC_ERR_INVALID_ARG;
+  if (n_nodes > DYSPEC_MAX_NODES) return DYSPEC_ERR_UNSUPPORTED;
+  if (32 * words_per_row < n_nodes) return DYSPEC_ERR_INVALID_ARG;
+  if (n_nodes == 0) return DYSPEC_OK;
+  if (!parents || !ancestor_bits) return DYSPEC_ERR_INVALID_ARG;
+  if (!aligned(ancestor_bits, 16) || !aligned(parents, 4)) return DYSPEC_ERR_INVALID_ARG;
+  cudaError_t e = launch_build_tree_mask(parents, nullptr, 1, n_nodes, ancestor_bits, depths, words_per_row, status,
+                                         reinterpret_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? DYSPEC_OK : DYSPEC_ERR_CUDA;
+}
+
+// Validates the arguments and runs the scheduler; no CUDA call.
+static int make_host_plan(dyspec_plan** out, int n_q_heads, int n_kv_heads, int head_dim, int n_req,
+                          const int32_t* prefix_len, const int32_t* n_nodes, const int64_t* kv_row_offset,
+                          int64_t kv_total_rows, int words_per_row, float scale) {
+  *out = nullptr;
+  if (n_q_heads <= 0 || n_kv_heads <= 0 || n_req < 0 || kv_total_rows < 0) return DYSPEC_ERR_INVALID_ARG;
+  if (n_req > 0 && (!prefix_len || !n_nodes || !kv_row_offset)) return DYSPEC_ERR_INVALID_ARG;
+  if (words_per_row <= 0 || (words_per_row & 3)) return DYSPEC_ERR_INVALID_ARG;
+  if (n_q_heads % n_kv_heads != 0) return DYSPEC_ERR_UNSUPPORTED;
+  const int g = n_q_heads / n_kv_heads;
+  if (!(g == 1 || g == 2 || g == 4 || g == 8)) return DYSPEC_ERR_UNSUPPORTED;
+  if (!(head_dim == 64 || head_dim == 128)) return DYSPEC_ERR_UNSUPPORTED;
+  if (kv_total_rows >= (int64_t(1) << 31)) return DYSPEC_ERR_UNSUPPORTED;
+  dyspec_plan* pl = new (std::nothrow) dyspec_plan();
+  if (!pl) return DYSPEC_ERR_CUDA;
+  pl->hq = n_q_heads; pl->hkv = n_kv_heads; pl->d = head_dim; pl->g = g;
+  pl->log2g = g == 1 ? 0 : g == 2 ? 1 : g == 4 ? 2 : 3;
+  pl->W = words_per_row;
+  pl->scale = scale > 0.f ? scale : 1.0f / std::sqrt(float(head_dim));
+  pl->n_req = n_req;
+  pl->kv_total_rows = kv_total_rows;
+  int64_t node0 = 0;
+  int max_rows = 0;
+  for (int r = 0; r < n_req; ++r) {
+    if (prefix_len[r] < 0 || n_nodes[r] < 0 || kv_row_offset[r] < 0) { delete pl; return DYSPEC_ERR_INVALID_ARG; }
+    if (n_nodes[r] > DYSPEC_MAX_NODES) { delete pl; return DYSPEC_ERR_UNSUPPORTED; }
+    if (32 * words_per_row < n_nodes[r]) { delete pl; return DYSPEC_ERR_INVALID_ARG; }
+    if (kv_row_offset[r] + prefix_len[r] + n_nodes[r] > kv_total_rows) { delete pl; return DYSPEC_ERR_INVALID_ARG; }
+    ReqInfo rq{};
+    rq.kv_row0 = kv_row_offset[r]; rq.prefix_len = prefix_len[r]; rq.n_nodes = n_nodes[r]; rq.node0 = int32_t(node0);
+    pl->reqs.push_back(rq);
+    node0 += n_nodes[r];
+    max_rows = std::max(max_rows, n_nodes[r] * g);
+  }
+  if (node0 >= (int64_t(1) << 31)) { delete pl; return DYSPEC_ERR_UNSUPPORTED; }
+  pl->total_nodes = node0;
+  // Regime: tcgen05 tiles (128 packed rows) when some request fills most of such a tile, else
+  // warp-level tiles (64 packed rows).
+  pl->regime = g_force_regime >= 0 ? g_force_regime : 0;
+  pl->bm = pl->regime == 0 ? 64 : 128;
+  pl->bn = pl->regime == 0 ? 64 : 128;
+  schedule(*pl);
+  pl->workspace_bytes = size_t(pl->n_slots) * size_t(pl->bm) * (pl->d + 2) * sizeof(float);
+  *out = pl;
+  return DYSPEC_OK;
+}
+
+int dyspec_plan_create(dyspec_plan_t** plan, int n_q_heads, int n_kv_heads, int head_dim, int n_req,
+                       const int32_t* prefix_len, const int32_t* n_nodes, const int64_t* kv_row_offset,
+                       int64_t kv_total_rows, int words_per_row, float scale) {
+  if (!plan) return DYSPEC_ERR_INVALID_ARG;
+  dyspec_plan* pl = nullptr;
+  int rc = make_host_plan(&pl, n_q_heads, n_kv_heads, head_dim, n_req, prefix_len, n_nodes, kv_row_offset,
+                          kv_total_rows, words_per_row, scale);
+  *plan = nullptr;
+  if (rc != DYSPEC_OK) return rc;
+  rc = upload(*pl);
+  if (rc != DYSPEC_OK) { dyspec_plan_destroy(pl); return rc; }
+  *plan = pl;
+  return DYSPEC_OK;
+}
+
+int dyspec_schedule_dry_run(int n_q_heads, int n_kv_heads, int head_dim, int n_req, const int32_t* prefix_len,
+                            const int32_t* n_nodes, int words_per_row, int32_t* items_out, int max_items,
+                            int32_t* cta_begin_out, int max_ctas, int64_t* info_out) {
+  std::vector<int64_t> off(size_t(std::max(n_req, 1)), 0);
+  int64_t rows = 0;
+  for (int r = 0; r < n_req && prefix_len && n_nodes; ++r) {
+    off[size_t(r)] = rows;
+    rows += int64_t(std::max(prefix_len[r], 0)) + std::max(n_nodes[r], 0);
+  }
+  dyspec_plan* pl = nullptr;
+  const int rc = make_host_plan(&pl, n_q_heads, n_kv_heads, head_dim, n_req, prefix_len, n_nodes, off.data(), rows,
+                                words_per_row, 0.f);
+  if (rc != DYSPEC_OK) return rc;
+  const int n_items = int(pl->items.size());
+  if (items_out)
+    for (int i = 0; i < n_items && i < max_items; ++i) memcpy(items_out + 8 * i, &pl->items[size_t(i)], sizeof(WorkItem));
+  if (cta_begin_out)
+    for (int c = 0; c <= pl->n_ctas && c < max_ctas; ++c) cta_begin_out[c] = pl->cta_begin[size_t(c)];
+  if (info_out) {
+    info_out[0] = n_items; info_out[1] = pl->n_ctas; info_out[2] = pl->n_groups; info_out[3] = int64_t(pl->split_groups.size());
+    info_out[4] = pl->max_splits; info_out[5] = pl->regime; info_out[6] = pl->total_tiles; info_out[7] = pl->bm;
+    info_out[8] = pl->bn; info_out[9] = int64_t(pl->workspace_bytes);
+  }
+  delete pl;
+  return n_items;
+}
+
+int dyspec_plan_destroy(dyspec_plan_t* plan) {
+  if (!plan) return DYSPEC_OK;
+  if (plan->d_blob) cudaFree(plan->d_blob);
+  delete plan;
+  return DYSPEC_OK;
+}
+
+size_t dyspec_plan_workspace_bytes(const dyspec_plan_t* plan) { return plan ? plan->workspace_bytes : 0; }
+
+int64_t dyspec_plan_info(const dyspec_plan_t* plan, int field) {
+  if (!plan) return DYSPEC_ERR_INVALID_ARG;
+  switch (field) {
+    case 0: return int64_t(plan->items.size());
+    case 1: return plan->n_ctas;
+    case 2: return plan->n_groups;
+    case 3: return int64_t(plan->split_groups.size());
+    case 4: return plan->max_splits;
+    case 5: return plan->regime;
+    case 6: return plan->total_tiles;
+    case 7: return plan->bm;
+    default: return DYSPEC_ERR_INVALID_ARG;
+  }
+}
+
+int dyspec_plan_build_tree_mask(const dyspec_plan_t* plan, const int32_t* parents, uint32_t* ancestor_bits,
+                                int32_t* depths, int32_t* status, dyspec_stream_t stream) {
+  if (!plan) return DYSPEC_ERR_INVALID_ARG;
+  if (plan->n_req == 0 || plan->total_nodes == 0) return DYSPEC_OK;
+  if (!parents || !ancestor_bits || !aligned(ancestor_bits, 16)) return DYSPEC_ERR_INVALID_ARG;
+  cudaError_t e = launch_build_tree_mask(parents, plan->d_reqs, plan->n_req, 0, ancestor_bits, depths, plan->W, status,
+                                         reinterpret_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? DYSPEC_OK : DYSPEC_ERR_CUDA;
+}
+
+int dyspec_tree_attention_ragged(const dyspec_plan_t* plan, const void* q, const void* k_cache, const void* v_cache,
+                                 const uint32_t* ancestor_bits, void* out, void* workspace, size_t workspace_bytes,
+                                 int32_t* status, dyspec_stream_t stream) {
+  if (!plan) return DYSPEC_ERR_INVALID_ARG;
+  if (plan->n_ctas == 0) return DYSPEC_OK;
+  if (!q || !k_cache || !v_cache || !ancestor_bits || !out) return DYSPEC_ERR_INVALID_ARG;
+  if (!aligned(q, 16) || !aligned(k_cache, 16) || !aligned(v_cache, 16) || !aligned(out, 16) || !aligned(ancestor_bits, 16))
+    return DYSPEC_ERR_INVALID_ARG;
+  if (plan->workspace_bytes > 0 && (!workspace || workspace_bytes < plan->workspace_bytes || !aligned(workspace, 256)))
+    return DYSPEC_ERR_WORKSPACE;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+
+  CUtensorMap mq, mk, mv;
+  const int bm = plan->bm, bn = plan->bn;
+  if (!encode_map(&mq, q, plan->total_nodes, plan->hq, plan->d, plan->g, bm / plan->g) ||
+      !encode_map(&mk, k_cache, plan->kv_total_rows, plan->hkv, plan->d, 1, bn) ||
+      !encode_map(&mv, v_cache, plan->kv_total_rows, plan->hkv, plan->d, 1, bn))
+    return DYSPEC_ERR_CUDA;
+
+  AttnParams p{};
+  p.reqs = plan->d_reqs; p.items = plan->d_items; p.cta_item_begin = plan->d_cta_begin; p.groups = plan->d_groups;
+  p.bits = ancestor_bits; p.out = static_cast<__nv_bfloat16*>(out); p.partial = static_cast<float*>(workspace);
+  p.counters = plan->d_counters; p.status = status;
+  p.n_q_heads = plan->hq; p.n_kv_heads = plan->hkv; p.group_size = plan->g; p.log2_g = plan->log2g;
+  p.words_per_row = plan->W; p.slot_floats = bm * (plan->d + 2);
+  p.scale_log2e = plan->scale * kLog2e;
+
+  cudaError_t e;
+  if (plan->regime == 0) e = launch_attn_mma(plan->d, plan->n_ctas, mq, mk, mv, p, st);
+  else e = launch_attn_tc(plan->d, plan->n_ctas, mq, mk, mv, p, st);
+  if (e != cudaSuccess) return DYSPEC_ERR_CUDA;
+  e = launch_combine(plan->d, bm, int(plan->split_groups.size()), p, st);
+  return e == cudaSuccess ? DYSPEC_OK : DYSPEC_ERR_CUDA;
+}
+
+// ---- single-request convenience form -------------------------------------------------------------
+namespace {
+struct DefaultShape { int hq = 0, hkv = 0, d = 0, W = 0; float scale = 0.f; };
+DefaultShape g_shape;
+struct Cached { dyspec_plan* plan; void* workspace; };
+std::map<std::tuple<int, int, int, int, int, int>, Cached> g_cache;
+std::mutex g_cache_mutex;
+}  // namespace
+
+int dyspec_set_default_shape(int n_q_heads, int n_kv_heads, int head_dim, int words_per_row, float scale) {
+  if (n_q_heads <= 0 || n_kv_heads <= 0 || n_q_heads % n_kv_heads != 0) return DYSPEC_ERR_INVALID_ARG;
+  const int g = n_q_heads / n_kv_heads;
+  if (!(g == 1 || g == 2 || g == 4 || g == 8) || !(head_dim == 64 || head_dim == 128)) return DYSPEC_ERR_UNSUPPORTED;
+  if (words_per_row <= 0 || (words_per_row & 3)) return DYSPEC_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lock(g_cache_mutex);
+  g_shape.hq = n_q_heads; g_shape.hkv = n_kv_heads; g_shape.d = head_dim; g_shape.W = words_per_row; g_shape.scale = scale;
+  return DYSPEC_OK;
+}
+
+int dyspec_tree_attention(const void* q, const void* k_cache, const void* v_cache, int prefix_len,
+                          const uint32_t* ancestor_bits, int n_nodes, void* out, dyspec_stream_t stream) {
+  Cached c{};
+  {
+    std::lock_guard<std::mutex> lock(g_cache_mutex);
+    if (g_shape.hq == 0) return DYSPEC_ERR_INVALID_ARG;
+    if (prefix_len < 0 || n_nodes < 0) return DYSPEC_ERR_INVALID_ARG;
+    const auto key = std::make_tuple(g_shape.hq, g_shape.hkv, g_shape.d, g_shape.W, prefix_len, n_nodes);
+    auto it = g_cache.find(key);
+    if (it == g_cache.end()) {
+      const int32_t L = prefix_len, n = n_nodes;
+      const int64_t off = 0;
+      dyspec_plan* pl = nullptr;
+      int rc = dyspec_plan_create(&pl, g_shape.hq, g_shape.hkv, g_shape.d, 1, &L, &n, &off, int64_t(L) + n, g_shape.W,
+                                  g_shape.scale);
+      if (rc != DYSPEC_OK) return rc;
+      void* ws = nullptr;
+      if (pl->workspace_bytes > 0 && cudaMalloc(&ws, pl->workspace_bytes) != cudaSuccess) {
+        dyspec_plan_destroy(pl);
+        return DYSPEC_ERR_CUDA;
+      }
+      it = g_cache.emplace(key, Cached{pl, ws}).first;
+    }
+    c = it->second;
+  }
+  return dyspec_tree_attention_ragged(c.plan, q, k_cache, v_cache, ancestor_bits, out, c.workspace,
+                                      c.plan->workspace_bytes, nullptr, stream);
+}
+
+}  // extern "C"

@@ -1,0 +1,157 @@
+// Shared device/host declarations of the tree-verify attention library (internal; not part of the C ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <cuda.h>
+#include <stdint.h>
+
+#include "../../include/dyspec.h"
+
+namespace dyspec {
+
+constexpr int kNumSMs = 148;            // B200: 2 dies x 74 SMs
+constexpr float kLog2e = 1.4426950408889634f;
+
+// One verification request, device-side view.
+struct ReqInfo {
+  int64_t kv_row0;     // row of the request's token 0 in k_cache / v_cache
+  int32_t prefix_len;  // L_r
+  int32_t n_nodes;     // n_r
+  int32_t node0;       // first query / output / mask row of the request
+  int32_t pad;
+};
+
+// One unit of scheduled work: a tile of packed query rows of one (request, kv head) against a
+// contiguous range of that group's key tiles.  Packed row p of a (request, kv head) pair is
+// node p / g, query head kv_head * g + p % g.  Key tiles of a group: first the prefix tiles
+// (tile t covers prefix keys [t*BN, min(L, (t+1)*BN))), then the tree tiles (tile u covers tree
+// columns [u*BN, (u+1)*BN)).
+struct WorkItem {
+  int32_t req;
+  int32_t kv_head;
+  int32_t row0;        // first packed row of the query tile (multiple of BM)
+  int32_t tile_begin;  // key-tile range [tile_begin, tile_end) of the group's tile list
+  int32_t tile_end;
+  int32_t slot;        // index of the fp32 partial slot to write, or -1: write the final bf16 rows
+  int32_t group;       // query-tile group id (arrival counter index)
+  int32_t n_splits;    // number of items the group was cut into
+};
+
+// A split query-tile group, for the combine step.
+struct GroupInfo {
+  int32_t req;
+  int32_t kv_head;
+  int32_t row0;
+  int32_t slot0;       // first partial slot; the group's slots are slot0 .. slot0 + n_splits - 1
+  int32_t n_splits;
+  int32_t pad[3];
+};
+
+// Parameters common to the attention kernels.
+struct AttnParams {
+  const ReqInfo* reqs;
+  const WorkItem* items;
+  const int32_t* cta_item_begin;   // [n_ctas + 1]
+  const GroupInfo* groups;         // split groups only
+  const uint32_t* bits;            // ancestor bitmasks [sum n][W]
+  __nv_bfloat16* out;              // [sum n][H_q][D]
+  float* partial;                  // split-KV partials: slot s at partial + s * slot_floats
+  int32_t* counters;               // per-group arrival counters (zero between calls)
+  int32_t* status;                 // may be null
+  int32_t n_q_heads;
+  int32_t n_kv_heads;
+  int32_t group_size;              // g
+  int32_t log2_g;
+  int32_t words_per_row;           // W
+  int32_t slot_floats;             // BM * (D + 2)
+  float scale_log2e;               // scale * log2(e)
+};
+
+#ifdef __CUDACC__
+// ------------------------------------------------------------------------------------------------
+// PTX helpers (sm_100a).  Every wait is bounded: when it runs out the kernel records
+// DYSPEC_ERR_TIMEOUT and carries on without waiting any more, so it always terminates.
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void fence_barrier_init() {
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() {
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t done;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(done)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return done != 0;
+}
+__device__ __forceinline__ uint64_t global_timer_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+
+constexpr uint64_t kWaitLimitNs = 1000ull * 1000ull * 1000ull;  // 1 s per wait, then give up
+
+// Bounded mbarrier wait.  `abort_flag` lives in shared memory: once any wait of the CTA ran out,
+// later waits return at once.  Returns false when the wait did not complete.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
+  if (mbar_try_wait(bar, parity)) return true;
+  if (*abort_flag) return false;
+  const uint64_t t0 = global_timer_ns();
+  uint32_t spins = 0;
+  while (!mbar_try_wait(bar, parity)) {
+    if ((++spins & 0x3ff) == 0) {
+      if (*abort_flag) return false;
+      if (global_timer_ns() - t0 > kWaitLimitNs) {
+        *abort_flag = 1;
+        if (status) atomicCAS(status, 0, DYSPEC_ERR_TIMEOUT);
+        return false;
+      }
+    }
+  }
+  return true;
+}
+
+// TMA: 3-D tiled load global -> shared, completion on an mbarrier (no multicast anywhere).
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+__device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
+
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+#endif  // __CUDACC__
+
+}  // namespace dyspec

@@ -1,0 +1,155 @@
+"""Parity of the CUDA path (through the C ABI) with the fp64 oracle, element by element.
+
+Masks and depths must match bit-exactly.  Attention: bf16 inputs, fp32 accumulation, bf16 output,
+compared with the fp64 oracle: max abs error <= 2e-2 and mean abs error <= 2e-3.
+"""
+import numpy as np
+import pytest
+
+from oracle import dyspec_oracle as orc
+from paper_2410_11744_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+MAX_ABS, MEAN_ABS = 2e-2, 2e-3
+
+
+@pytest.fixture(scope="module")
+def rt():
+    import torch
+    assert torch.cuda.is_available()
+    from paper_2410_11744_b200 import build
+    build.build()
+    from paper_2410_11744_b200 import binding, runner
+    return binding, runner
+
+
+def run_and_check(rt, w, regime=-1, ctas=0, words_per_row=None):
+    B, R = rt
+    B.dyspec_set_tuning(regime, ctas)
+    try:
+        batch = R.DeviceBatch(w, words_per_row=words_per_row)
+    finally:
+        B.dyspec_set_tuning(-1, 0)
+    batch.step()
+    bits, depths, out_bits, status = batch.results()
+    assert status == 0
+    ref_bits, ref_depths = orc.build_tree_mask_ragged(w.parents, batch.W)
+    assert np.array_equal(bits, ref_bits)
+    assert np.array_equal(depths, ref_depths)
+    ref = orc.tree_attention_ragged(w.q, w.k, w.v, w.prefix_len, w.n_nodes, w.kv_row_offset, w.parents)
+    got = orc.bf16_bits_to_f64(out_bits)
+    assert np.isfinite(got).all()
+    if ref.size:
+        err = np.abs(got - ref)
+        assert err.max() <= MAX_ABS, f"max abs err {err.max()}"
+        assert err.mean() <= MEAN_ABS, f"mean abs err {err.mean()}"
+    return batch, got, ref
+
+
+@pytest.mark.parametrize("index", [1, 2, 3, 4, 5])
+def test_configs_match_oracle(rt, index):
+    run_and_check(rt, wl.make_config(index))
+
+
+@pytest.mark.parametrize("ctas", [1, 3, 40, 1000])
+def test_split_count_does_not_change_results(rt, ctas):
+    """Forcing the scheduler to balance over few or many CTAs changes the split-KV cuts, not the answer."""
+    w = wl.make_custom(77, 8, 2, 128, [700, 45], [wl.greedy_tree(np.random.default_rng(1), 90, 8, 0.3),
+                                                   wl.greedy_tree(np.random.default_rng(2), 33, 4, 0.2)])
+    _, got, _ = run_and_check(rt, w, ctas=ctas)
+    _, base, _ = run_and_check(rt, w, ctas=2)
+    assert np.abs(got - base).max() <= 2 ** -6     # both are bf16 roundings of nearly equal fp32 values
+
+
+@pytest.mark.parametrize("hq,hkv,d", [(4, 4, 64), (8, 4, 64), (8, 2, 128), (8, 1, 128), (2, 2, 128)])
+def test_shapes_and_gqa(rt, hq, hkv, d):
+    rng = np.random.default_rng(hq * 100 + d)
+    trees = [wl.greedy_tree(rng, 37, 4, 0.3), wl.random_tree(rng, 130, 0.05), wl.chain_tree(65)]
+    run_and_check(rt, wl.make_custom(5, hq, hkv, d, [129, 64, 1], trees))
+
+
+def test_edge_cases(rt):
+    rng = np.random.default_rng(0)
+    # empty prefix; single node; an empty request in the middle; star forest; ragged tails
+    trees = [wl.chain_tree(5), np.zeros(0, np.int32), wl.star_forest(70), np.array([-1], np.int32),
+             wl.greedy_tree(rng, 63, 4, 0.3)]
+    run_and_check(rt, wl.make_custom(6, 4, 2, 64, [0, 10, 63, 0, 65], trees))
+    # nothing at all
+    run_and_check(rt, wl.make_custom(7, 4, 4, 64, [], []))
+    run_and_check(rt, wl.make_custom(8, 4, 4, 64, [5], [np.zeros(0, np.int32)]))
+
+
+def test_maximum_tree_size(rt):
+    rng = np.random.default_rng(4)
+    w = wl.make_custom(9, 8, 1, 128, [100], [wl.greedy_tree(rng, 1024, 8, 0.2)])
+    run_and_check(rt, w)
+    w = wl.make_custom(10, 2, 2, 64, [3], [wl.chain_tree(1024)])          # depth 1023: deepest possible
+    run_and_check(rt, w)
+
+
+def test_rows_after_a_request_may_hold_garbage(rt):
+    """K/V rows that follow a request (another request's, or unwritten memory) must not leak in, even as NaN."""
+    rng = np.random.default_rng(11)
+    trees = [wl.greedy_tree(rng, 20, 4, 0.3), wl.greedy_tree(rng, 9, 4, 0.3)]
+    w = wl.make_custom(12, 4, 2, 128, [70, 30], trees)
+    # poison request 1's rows as seen from request 0's last tiles, then restore them for request 1 by
+    # putting a gap of NaN rows between the two requests instead
+    gap = 100
+    nan_rows = np.full((gap,) + w.k.shape[1:], 0x7FC0, dtype=np.uint16)
+    o1 = int(w.kv_row_offset[1])
+    w.k = np.concatenate([w.k[:o1], nan_rows, w.k[o1:], nan_rows])
+    w.v = np.concatenate([w.v[:o1], nan_rows, w.v[o1:], nan_rows])
+    w.kv_row_offset = np.array([0, o1 + gap], dtype=np.int64)
+    run_and_check(rt, w)
+
+
+def test_bad_tree_is_reported_not_fatal(rt):
+    import torch
+    B, R = rt
+    w = wl.make_custom(13, 4, 4, 64, [16], [np.array([-1, 0, 5, 1, -3, 2], np.int32)])   # nodes 2 and 4 are bad
+    batch = R.DeviceBatch(w)
+    batch.step()
+    bits, depths, out_bits, status = batch.results()
+    assert status == -5
+    fixed = [-1, 0, -1, 1, -1, 2]                 # bad nodes become roots
+    ref_bits, ref_depths = orc.build_tree_mask(fixed, batch.W)
+    assert np.array_equal(bits, ref_bits) and np.array_equal(depths, ref_depths)
+    assert np.isfinite(orc.bf16_bits_to_f64(out_bits)).all()
+
+
+def test_single_request_entry_points(rt):
+    import torch
+    B, R = rt
+    w = wl.make_config(1)
+    L, n = int(w.prefix_len[0]), int(w.n_nodes[0])
+    W = B.dyspec_words_per_row(n)
+    dev = torch.device("cuda:0")
+    parents = torch.from_numpy(w.parents[0]).to(dev)
+    bits = torch.zeros((n, W), dtype=torch.int32, device=dev)
+    depths = torch.zeros((n,), dtype=torch.int32, device=dev)
+    B.dyspec_build_tree_mask(parents, n, bits, depths, W)
+    q = torch.from_numpy(w.q.view(np.int16)).to(dev).view(torch.bfloat16)
+    k = torch.from_numpy(w.k.view(np.int16)).to(dev).view(torch.bfloat16)
+    v = torch.from_numpy(w.v.view(np.int16)).to(dev).view(torch.bfloat16)
+    out = torch.zeros_like(q)
+    B.dyspec_set_default_shape(w.n_q_heads, w.n_kv_heads, w.head_dim, W, 0.0)
+    for _ in range(2):                               # second call reuses the cached plan
+        out.zero_()
+        B.dyspec_tree_attention(q, k, v, L, bits, n, out)
+        torch.cuda.synchronize()
+        ref_bits, ref_depths = orc.build_tree_mask(w.parents[0], W)
+        assert np.array_equal(bits.cpu().numpy().view(np.uint32), ref_bits)
+        assert np.array_equal(depths.cpu().numpy(), ref_depths)
+        got = orc.bf16_bits_to_f64(R.bf16_tensor_to_bits(out))
+        ref = orc.tree_attention(w.q, w.k, w.v, L, w.parents[0])
+        assert np.abs(got - ref).max() <= MAX_ABS and np.abs(got - ref).mean() <= MEAN_ABS
+
+
+def test_runs_are_bitwise_repeatable(rt):
+    w = wl.make_config(2)
+    batch, got, _ = run_and_check(rt, w)
+    first = batch.results()[2].copy()
+    batch.out.zero_()
+    batch.step()
+    assert np.array_equal(batch.results()[2], first)

@@ -1,0 +1,86 @@
+"""Host logic of the ragged scheduler (no GPU): every key tile of every (request, kv head, query
+tile) group is covered exactly once, split groups get distinct partial slots, CTAs get contiguous,
+roughly equal shares."""
+import numpy as np
+import pytest
+
+from paper_2410_11744_b200 import workloads as wl
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2410_11744_b200 import build
+    build.build()
+    from paper_2410_11744_b200 import binding
+    return binding
+
+
+def check_schedule(B, hq, hkv, d, Ls, ns, regime=-1, ctas=0):
+    B.dyspec_set_tuning(regime, ctas)
+    try:
+        W = B.dyspec_words_per_row(max(list(ns) + [0]))
+        items, cta_begin, info = B.dyspec_schedule_dry_run(hq, hkv, d, Ls, ns, W)
+    finally:
+        B.dyspec_set_tuning(-1, 0)
+    g = hq // hkv
+    bm, bn = info["rows_per_tile"], info["keys_per_tile"]
+    npt = bm // g
+    # expected groups and their tile counts, from the definition of the tile list
+    expect = {}
+    for r, (L, n) in enumerate(zip(Ls, ns)):
+        for kvh in range(hkv):
+            for qt in range((n + npt - 1) // npt):
+                last = min(n, (qt + 1) * npt)
+                expect[(r, kvh, qt * bm)] = (L + bn - 1) // bn + (last + bn - 1) // bn
+    assert info["groups"] == len(expect)
+    assert info["key_tiles"] == sum(expect.values())
+    covered = {k: [] for k in expect}
+    slots = set()
+    for req, kvh, row0, tb, te, slot, group, nsp in items.tolist():
+        assert te > tb >= 0
+        covered[(req, kvh, row0)].append((tb, te, slot, nsp))
+    for key, pieces in covered.items():
+        pieces.sort()
+        assert pieces[0][0] == 0 and pieces[-1][1] == expect[key]
+        for a, b in zip(pieces, pieces[1:]):
+            assert a[1] == b[0]
+        if len(pieces) == 1:
+            assert pieces[0][2] == -1 and pieces[0][3] == 1
+        else:
+            for _, _, slot, nsp in pieces:
+                assert slot >= 0 and slot not in slots and nsp == len(pieces)
+                slots.add(slot)
+    assert info["workspace_bytes"] == len(slots) * bm * (d + 2) * 4
+    assert sorted(slots) == list(range(len(slots)))
+    # CTA ranges partition the item list
+    assert cta_begin[0] == 0 and cta_begin[-1] == len(items) and (np.diff(cta_begin) > 0).all()
+    loads = [int(sum(items[i][4] - items[i][3] for i in range(a, b))) for a, b in zip(cta_begin, cta_begin[1:])]
+    return info, loads
+
+
+def test_five_configs_schedule(B):
+    for idx in range(1, 6):
+        w = wl.make_config(idx)
+        info, loads = check_schedule(B, w.n_q_heads, w.n_kv_heads, w.head_dim, w.prefix_len.tolist(), w.n_nodes.tolist())
+        assert info["ctas"] <= 2 * 148 + 8
+        if idx >= 2:
+            assert max(loads) <= 1.5 * (sum(loads) / len(loads)) + 4
+
+
+@pytest.mark.parametrize("ctas", [1, 2, 7, 148, 5000])
+def test_forced_cta_counts(B, ctas):
+    check_schedule(B, 8, 2, 128, [700, 45, 0, 9000], [90, 33, 5, 1024], ctas=ctas)
+
+
+def test_degenerate_batches(B):
+    info, loads = check_schedule(B, 4, 4, 64, [], [])
+    assert info["items"] == 0 and info["ctas"] == 0
+    info, _ = check_schedule(B, 4, 4, 64, [10, 0], [0, 0])
+    assert info["items"] == 0
+    info, _ = check_schedule(B, 4, 4, 64, [0], [1])
+    assert info["items"] == 4 and info["key_tiles"] == 4
+
+
+def test_regime_1_tiles(B):
+    info, _ = check_schedule(B, 64, 8, 128, [2048], [512], regime=1)
+    assert info["rows_per_tile"] == 128 and info["regime"] == 1
