@@ -181,44 +181,56 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
-def measure_config(torch, runner, w, steps, warmup, device, with_events=True):
-    """Device-resident timing of `steps` steps, rotating over copies larger than L2."""
+def _graph_of(torch, fn):
+    """Capture `fn` (which only enqueues library calls on the current stream) into a CUDA graph."""
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        fn()
+    return g
+
+
+def _time_replays(torch, graph, replays, tail=None):
+    stream = torch.cuda.current_stream()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(replays):
+        graph.replay()
+    if tail is not None:
+        tail()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1)
+
+
+def measure_config(torch, runner, w, steps, warmup, device):
+    """Device-resident timing of exactly `steps` steps, rotating over independent copies of the inputs
+    that together exceed 2x L2.  The launch sequence of one rotation is captured in a CUDA graph so
+    that the host's launch overhead (python, ctypes) does not starve the GPU."""
     first = runner.DeviceBatch(w, device=device)
     nbytes, flops = algorithmic_cost(w, first.W)
     copies = max(2, min(64, int(np.ceil(2.0 * L2_BYTES / max(nbytes, 1)))))
-    batches = [first] + [runner.DeviceBatch(w, device=device) for _ in range(copies - 1)]
+    batches = [first] + [runner.DeviceBatch(w, device=device, plan=first.plan) for _ in range(copies - 1)]
     info = first.plan.describe()
     launches_per_step = 1 + 1 + (1 if info["split_groups"] > 0 else 0)
-    stream = torch.cuda.current_stream()
     for i in range(max(warmup, 3)):
         batches[i % copies].step()
     torch.cuda.synchronize()
-    # pass 1: whole region, two events
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for i in range(steps):
-        batches[i % copies].step()
-    e1.record(stream)
+    g_step = _graph_of(torch, lambda: [b.step() for b in batches])
+    g_attn = _graph_of(torch, lambda: [b.attention() for b in batches])
+    g_mask = _graph_of(torch, lambda: [b.build_mask() for b in batches])
+    for g in (g_step, g_attn, g_mask):
+        g.replay()
     torch.cuda.synchronize()
-    total_ms = e0.elapsed_time(e1)
-    # pass 2: per-call events around the attention call (main kernel + combine) and the mask kernel
-    attn_ms, mask_ms = None, None
-    if with_events:
-        k = min(steps, 200)
-        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(k)]
-        for i in range(k):
-            b = batches[i % copies]
-            evs[i][0].record(stream)
-            b.build_mask()
-            evs[i][1].record(stream)
-            b.attention()
-            evs[i][2].record(stream)
-        torch.cuda.synchronize()
-        mask_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in evs)
-        attn_ms = statistics.mean(e[1].elapsed_time(e[2]) for e in evs)
+    replays, rem = divmod(steps, copies)
+    total_ms = _time_replays(torch, g_step, replays, tail=lambda: [batches[i].step() for i in range(rem)])
+    # the dominant kernel alone: attention calls (main kernel + combine) back to back, same rotation
+    r2 = max(1, min(replays, 200))
+    attn_ms = _time_replays(torch, g_attn, r2) / (r2 * copies)
+    mask_ms = _time_replays(torch, g_mask, r2) / (r2 * copies)
     status = int(first.status.item())
     return dict(batches=batches, total_ms=total_ms, ms_per_step=total_ms / steps, attn_ms=attn_ms, mask_ms=mask_ms,
-                bytes=nbytes, flops=flops, copies=copies, info=info, launches_per_step=launches_per_step, status=status)
+                bytes=nbytes, flops=flops, copies=copies, info=info, launches_per_step=launches_per_step, status=status,
+                graph=g_step)
 
 
 def roofline_entry(m, peaks, peaks_kind):
@@ -283,7 +295,7 @@ def run_ours(args):
             t_end = time.time() + 1.0
             while time.time() < t_end:
                 for i in range(200):
-                    m["batches"][i % m["copies"]].step()
+                    m["graph"].replay()
                 torch.cuda.synchronize()
             clocks_note = "timed region shorter than the sampling period: sampled while the same loop kept running"
         clocks = ClockSampler.summarise(sampler.lines(), clocks_note)
@@ -352,7 +364,7 @@ def run_ours(args):
                                "bytes": mi["bytes"], "flops": mi["flops"], "bound": ri["bound"], "achieved": ri["achieved"],
                                "unit": ri["unit"], "frac": ri["frac"], "plan": mi["info"], "status": mi["status"]})
             if idx != args.config:
-                del mi["batches"]
+                del mi["batches"], mi["graph"]
                 torch.cuda.empty_cache()
 
     # ---- the oracle on the host cores, bounded sample of the same workload
@@ -387,6 +399,24 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_profile(args):
+    """A short eager run of the hot path for profilers: no graphs, no timing, no oracle."""
+    import torch
+    from paper_2410_11744_b200 import build as _build
+    _build.build()
+    from paper_2410_11744_b200 import runner, workloads
+    w = workloads.make_config(args.config)
+    first = runner.DeviceBatch(w)
+    nbytes, _ = algorithmic_cost(w, first.W)
+    copies = max(2, min(8, int(np.ceil(1.2 * L2_BYTES / max(nbytes, 1)))))
+    batches = [first] + [runner.DeviceBatch(w, plan=first.plan) for _ in range(copies - 1)]
+    for i in range(args.profile):
+        batches[i % copies].step()
+    torch.cuda.synchronize()
+    print(json.dumps({"profiled_steps": args.profile, "workload": w.name, "copies": copies,
+                      "plan": first.plan.describe(), "status": int(first.status.item())}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -395,7 +425,11 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=2)
     ap.add_argument("--no-per-config", action="store_true")
+    ap.add_argument("--profile", type=int, default=0,
+                    help="run only this many plain (eager) steps of --config and exit: the command to put under ncu")
     args = ap.parse_args()
+    if args.profile > 0:
+        return run_profile(args)
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -285,11 +285,11 @@ static int make_host_plan(dyspec_plan** out, int n_q_heads, int n_kv_heads, int 
   }
   if (node0 >= (int64_t(1) << 31)) { delete pl; return DYSPEC_ERR_UNSUPPORTED; }
   pl->total_nodes = node0;
-  // Regime: tcgen05 tiles (128 packed rows) when some request fills most of such a tile, else
-  // warp-level tiles (64 packed rows).
-  pl->regime = g_force_regime >= 0 ? g_force_regime : 0;
-  pl->bm = pl->regime == 0 ? 64 : 128;
-  pl->bn = pl->regime == 0 ? 64 : 128;
+  // Regime: tcgen05 tiles (2 x 128 packed rows per item) when some request has more packed rows
+  // (nodes x group) than one warp-level tile holds, else warp-level tiles (64 packed rows).
+  pl->regime = g_force_regime >= 0 ? g_force_regime : (max_rows > 64 ? 1 : 0);
+  pl->bm = pl->regime == 0 ? 64 : 256;    // packed query rows per work item (regime 1: two 128-row halves)
+  pl->bn = pl->regime == 0 ? 64 : 128;    // keys per tile
   schedule(*pl);
   pl->workspace_bytes = size_t(pl->n_slots) * size_t(pl->bm) * (pl->d + 2) * sizeof(float);
   *out = pl;
@@ -386,7 +386,8 @@ int dyspec_tree_attention_ragged(const dyspec_plan_t* plan, const void* q, const
 
   CUtensorMap mq, mk, mv;
   const int bm = plan->bm, bn = plan->bn;
-  if (!encode_map(&mq, q, plan->total_nodes, plan->hq, plan->d, plan->g, bm / plan->g) ||
+  const int q_box_rows = plan->regime == 0 ? 64 : 128;   // packed rows per TMA box of Q
+  if (!encode_map(&mq, q, plan->total_nodes, plan->hq, plan->d, plan->g, q_box_rows / plan->g) ||
       !encode_map(&mk, k_cache, plan->kv_total_rows, plan->hkv, plan->d, 1, bn) ||
       !encode_map(&mv, v_cache, plan->kv_total_rows, plan->hkv, plan->d, 1, bn))
     return DYSPEC_ERR_CUDA;

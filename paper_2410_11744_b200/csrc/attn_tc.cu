@@ -1,7 +1,460 @@
-// placeholder until the tcgen05 regime lands
+// Tree-verify attention, tensor-core regime (Sec. 2 "Tree Attention"; App. C: prefix keys are in the mask).
+//
+// Used when tree nodes x GQA group fill 128-row tiles, i.e. when QK^T and PV are real dense
+// contractions.  One CTA per SM, 12 warps:
+//   warp 0        TMA producer: Q tile (2 x 128 packed rows) once per work item, then K and V tiles
+//                 (128 keys) into a 5-slot shared-memory ring, 128-byte swizzled, mbarrier-guarded.
+//   warp 1        tcgen05.mma issuer (one lane).  S = Q K^T: both operands from shared memory,
+//                 accumulator in TMEM.  O += P V: P from TMEM (bf16, written by the softmax warps
+//                 over the S columns), V from shared memory as an MN-major operand.
+//   warp 2        allocates / frees the 512 TMEM columns: S_A, S_B, O_A, O_B (128 fp32 columns each).
+//   warps 4-7     softmax of query half A: one thread per row, S read with tcgen05.ld, fp32 online
+//                 softmax in the exp2 domain, ancestor bitmask on tree tiles, P written back with
+//                 tcgen05.st.  The running output lives in TMEM and is rescaled only when the row
+//                 maximum grows by more than 2^8 (the final normalisation uses the same reference).
+//   warps 8-11    the same for query half B.  The two halves alternate on the tensor pipe, so one
+//                 half's softmax overlaps the other half's MMAs, and each K/V tile is loaded once
+//                 for 256 query rows.
+// Every wait is bounded (see mbar_wait); nothing here uses TMA multicast or clusters.
 #include "common.cuh"
+
 namespace dyspec {
-cudaError_t launch_attn_tc(int, int, const CUtensorMap&, const CUtensorMap&, const CUtensorMap&, const AttnParams&, cudaStream_t) {
-  return cudaErrorNotSupported;
+
+namespace {
+
+constexpr int BMH = 128;          // rows of one UMMA tile (one query half)
+constexpr int BN = 128;           // keys per tile
+constexpr int kThreads = 384;
+constexpr int kSlots = 5;
+constexpr uint32_t kTmemCols = 512;
+constexpr float kRescaleThreshold = 8.0f;   // log2 units
+
+template <int D>
+struct TcLayout {
+  static constexpr int kPanels = D / 64;
+  static constexpr int kPanelBytes = 128 * 128;               // 128 rows x 128 bytes
+  static constexpr int kTileBytes = kPanels * kPanelBytes;    // one K tile, V tile or query half
+  static constexpr int kQBytes = 2 * kTileBytes;
+  static constexpr int kRingOffset = kQBytes;
+  static constexpr int kBarOffset = kRingOffset + kSlots * kTileBytes;
+  static constexpr int kTotal = kBarOffset + 512;
+};
+
+// barrier indices (8 bytes each)
+enum { B_QFULL = 0, B_QFREE = 1, B_SLOT_FULL = 2, B_SLOT_EMPTY = B_SLOT_FULL + kSlots,
+       B_SREADY = B_SLOT_EMPTY + kSlots, B_PREADY = B_SREADY + 2, B_ODONE = B_PREADY + 2, B_OFREE = B_ODONE + 2,
+       B_COUNT = B_OFREE + 2 };
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
+__device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
 }
+__device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle, version 1 (sm_100).  Offsets are in bytes.
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  return uint64_t((saddr >> 4) & 0x3FFFu) | (uint64_t((lbo_bytes >> 4) & 0x3FFFu) << 16) |
+         (uint64_t((sbo_bytes >> 4) & 0x3FFFu) << 32) | (uint64_t(1) << 46) | (uint64_t(2) << 61);
+}
+// Instruction descriptor, kind::f16: bf16 x bf16 -> fp32, A K-major, M = 128.
+__host__ __device__ constexpr uint32_t make_idesc(int n, int b_mn_major) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(b_mn_major) << 16) | (uint32_t(n >> 3) << 17) | (uint32_t(128 >> 4) << 24);
+}
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+        "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+        "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+}  // namespace
+
+template <int D>
+__global__ void __launch_bounds__(kThreads, 1)
+tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                    const __grid_constant__ CUtensorMap map_v, const AttnParams p) {
+  using L = TcLayout<D>;
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const uint32_t s_q = smem_u32(smem);
+  const uint32_t s_ring = s_q + L::kRingOffset;
+  const uint32_t s_bar = s_q + L::kBarOffset;
+  auto bar = [&](int i) { return s_bar + 8u * uint32_t(i); };
+  volatile uint32_t* tmem_holder = reinterpret_cast<volatile uint32_t*>(smem + L::kBarOffset + 8 * B_COUNT);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::kBarOffset + 8 * B_COUNT + 8);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    mbar_init(bar(B_QFULL), 1);
+    mbar_init(bar(B_QFREE), 1);
+    for (int s = 0; s < kSlots; ++s) {
+      mbar_init(bar(B_SLOT_FULL + s), 1);
+      mbar_init(bar(B_SLOT_EMPTY + s), 1);
+    }
+    for (int h = 0; h < 2; ++h) {
+      mbar_init(bar(B_SREADY + h), 1);
+      mbar_init(bar(B_PREADY + h), BMH);
+      mbar_init(bar(B_ODONE + h), 1);
+      mbar_init(bar(B_OFREE + h), BMH);
+    }
+    *abort_flag = 0;
+    fence_barrier_init();
+  }
+  if (warp == 2) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32(const_cast<uint32_t*>(tmem_holder))), "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_holder;
+
+  const int item_begin = p.cta_item_begin[blockIdx.x];
+  const int item_end = p.cta_item_begin[blockIdx.x + 1];
+  const int g = p.group_size;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      prefetch_tensormap(&map_q);
+      prefetch_tensormap(&map_k);
+      prefetch_tensormap(&map_v);
+      uint32_t sc = 0, qit = 0;
+      for (int w = item_begin; w < item_end; ++w, ++qit) {
+        const WorkItem item = p.items[w];
+        const ReqInfo rq = p.reqs[item.req];
+        const int nh = (rq.n_nodes * g - item.row0 > BMH) ? 2 : 1;
+        mbar_wait(bar(B_QFREE), (qit & 1) ^ 1, abort_flag, p.status);
+        mbar_expect_tx(bar(B_QFULL), uint32_t(nh) * L::kTileBytes);
+        for (int h = 0; h < nh; ++h)
+          for (int pn = 0; pn < L::kPanels; ++pn)
+            tma_load_3d(s_q + h * L::kTileBytes + pn * L::kPanelBytes, &map_q, bar(B_QFULL), pn * 64, item.kv_head * g,
+                        rq.node0 + ((item.row0 + h * BMH) >> p.log2_g));
+        const int n_prefix_tiles = (rq.prefix_len + BN - 1) / BN;
+        for (int t = item.tile_begin; t < item.tile_end; ++t) {
+          const int64_t row = rq.kv_row0 + (t < n_prefix_tiles ? int64_t(t) * BN
+                                                               : int64_t(rq.prefix_len) + int64_t(t - n_prefix_tiles) * BN);
+          for (int kv = 0; kv < 2; ++kv, ++sc) {
+            const int slot = sc % kSlots;
+            const uint32_t ph = (sc / kSlots) & 1;
+            mbar_wait(bar(B_SLOT_EMPTY + slot), ph ^ 1, abort_flag, p.status);
+            mbar_expect_tx(bar(B_SLOT_FULL + slot), L::kTileBytes);
+            for (int pn = 0; pn < L::kPanels; ++pn)
+              tma_load_3d(s_ring + slot * L::kTileBytes + pn * L::kPanelBytes, kv == 0 ? &map_k : &map_v,
+                          bar(B_SLOT_FULL + slot), pn * 64, item.kv_head, int(row));
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc_qk = make_idesc(BN, 0);
+      constexpr uint32_t idesc_pv = make_idesc(D, 1);
+      uint32_t sc = 0, qit = 0;
+      uint32_t n_p[2] = {0, 0};      // P-ready phases consumed per half
+      uint32_t n_items_h[2] = {0, 0};
+      auto issue_qk = [&](int h, int slot) {
+        const uint32_t a_base = s_q + h * L::kTileBytes;
+        const uint32_t b_base = s_ring + slot * L::kTileBytes;
+#pragma unroll
+        for (int ks = 0; ks < D / 16; ++ks) {
+          const uint32_t off = uint32_t(ks >> 2) * L::kPanelBytes + uint32_t(ks & 3) * 32u;
+          umma_ss(tmem_base + uint32_t(h) * 128u, make_desc(a_base + off, 16, 1024), make_desc(b_base + off, 16, 1024),
+                  idesc_qk, ks > 0 ? 1u : 0u);
+        }
+        tc_commit(bar(B_SREADY + h));
+      };
+      auto issue_pv = [&](int h, int slot, bool accumulate) {
+        const uint32_t b_base = s_ring + slot * L::kTileBytes;
+#pragma unroll
+        for (int kk = 0; kk < BN / 16; ++kk) {
+          umma_ts(tmem_base + 256u + uint32_t(h) * 128u, tmem_base + uint32_t(h) * 128u + uint32_t(kk) * 8u,
+                  make_desc(b_base + uint32_t(kk) * 2048u, L::kPanelBytes, 1024), idesc_pv, (accumulate || kk > 0) ? 1u : 0u);
+        }
+        tc_commit(bar(B_ODONE + h));
+      };
+      for (int w = item_begin; w < item_end; ++w, ++qit) {
+        const WorkItem item = p.items[w];
+        const ReqInfo rq = p.reqs[item.req];
+        const int nh = (rq.n_nodes * g - item.row0 > BMH) ? 2 : 1;
+        const int T = item.tile_end - item.tile_begin;
+        mbar_wait(bar(B_QFULL), qit & 1, abort_flag, p.status);
+        {
+          const uint32_t kslot = sc++;
+          mbar_wait(bar(B_SLOT_FULL + kslot % kSlots), (kslot / kSlots) & 1, abort_flag, p.status);
+          tc_fence_after();
+          for (int h = 0; h < nh; ++h) issue_qk(h, kslot % kSlots);
+          tc_commit(bar(B_SLOT_EMPTY + kslot % kSlots));
+        }
+        for (int j = 0; j < T; ++j) {
+          const uint32_t vslot = sc++;
+          const bool more = j + 1 < T;
+          const uint32_t kslot = more ? sc++ : 0u;
+          mbar_wait(bar(B_SLOT_FULL + vslot % kSlots), (vslot / kSlots) & 1, abort_flag, p.status);
+          for (int h = 0; h < nh; ++h) {
+            if (j == 0) mbar_wait(bar(B_OFREE + h), (n_items_h[h] & 1) ^ 1, abort_flag, p.status);
+            mbar_wait(bar(B_PREADY + h), n_p[h] & 1, abort_flag, p.status);
+            ++n_p[h];
+            tc_fence_after();
+            issue_pv(h, vslot % kSlots, j > 0);
+            if (more) {
+              if (h == 0) {
+                mbar_wait(bar(B_SLOT_FULL + kslot % kSlots), (kslot / kSlots) & 1, abort_flag, p.status);
+                tc_fence_after();
+              }
+              issue_qk(h, kslot % kSlots);
+            }
+          }
+          tc_commit(bar(B_SLOT_EMPTY + vslot % kSlots));
+          if (more) tc_commit(bar(B_SLOT_EMPTY + kslot % kSlots));
+        }
+        tc_commit(bar(B_QFREE));
+        for (int h = 0; h < nh; ++h) ++n_items_h[h];
+      }
+    }
+  } else if (warp >= 4) {
+    // ------------------------------------------------------------------ softmax + epilogue warps
+    const int h = (warp - 4) >> 2;                       // query half
+    const int r = ((warp & 3) << 5) + lane;              // row of the half == TMEM lane
+    const uint32_t lane_sel = uint32_t((warp & 3) << 5) << 16;
+    const uint32_t t_s = tmem_base + uint32_t(h) * 128u + lane_sel;
+    const uint32_t t_o = tmem_base + 256u + uint32_t(h) * 128u + lane_sel;
+    uint32_t n_s = 0, n_o = 0;                           // S-ready / O-done phases seen by this half
+    uint32_t sc = 0;                                     // ring position (to find V slots)
+
+    for (int w = item_begin; w < item_end; ++w) {
+      const WorkItem item = p.items[w];
+      const ReqInfo rq = p.reqs[item.req];
+      const int n_rows = rq.n_nodes * g;
+      const int nh = (n_rows - item.row0 > BMH) ? 2 : 1;
+      const int T = item.tile_end - item.tile_begin;
+      if (h >= nh) { sc += 2u * uint32_t(T); continue; }
+      const int n_prefix_tiles = (rq.prefix_len + BN - 1) / BN;
+      const int row = item.row0 + h * BMH + r;
+      const bool ok = row < n_rows;
+      const int node = row >> p.log2_g;
+      const uint4* mask_row = reinterpret_cast<const uint4*>(p.bits + size_t(rq.node0 + (ok ? node : 0)) * p.words_per_row);
+
+      float m_used = -INFINITY, l = 0.f;
+      for (int j = 0; j < T; ++j) {
+        const int t = item.tile_begin + j;
+        const uint32_t vslot = sc + 1u;
+        sc += 2u;
+        // visibility of the 128 key columns of this tile for this row
+        uint32_t vis[4];
+        int own;
+        if (t < n_prefix_tiles) {
+          const int valid = min(BN, rq.prefix_len - t * BN);
+          own = min(BN, rq.prefix_len + rq.n_nodes - t * BN);
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4) {
+            const int rem = valid - 32 * q4;
+            vis[q4] = rem >= 32 ? 0xffffffffu : (rem <= 0 ? 0u : ((1u << rem) - 1u));
+          }
+        } else {
+          const int u = t - n_prefix_tiles;
+          own = min(BN, rq.n_nodes - u * BN);
+          uint4 mv = make_uint4(0u, 0u, 0u, 0u);
+          if (ok) mv = __ldg(mask_row + u);
+          vis[0] = mv.x; vis[1] = mv.y; vis[2] = mv.z; vis[3] = mv.w;
+        }
+
+        mbar_wait(bar(B_SREADY + h), n_s & 1, abort_flag, p.status);
+        ++n_s;
+        tc_fence_after();
+
+        // pass 1: row maximum of the visible scaled scores
+        float mx = -INFINITY;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          uint32_t v[32];
+          tmem_ld32(t_s + uint32_t(c) * 32u, v);
+          tmem_wait_ld();
+          const uint32_t bits = vis[c];
+#pragma unroll
+          for (int i = 0; i < 32; ++i)
+            if ((bits >> i) & 1u) mx = fmaxf(mx, __uint_as_float(v[i]));
+        }
+        mx *= p.scale_log2e;    // scale > 0, so the maximum commutes with the scaling
+        const float m_new = fmaxf(m_used, mx);
+        if (j == 0) {
+          m_used = m_new;
+        } else if (__any_sync(0xffffffffu, m_new > m_used + kRescaleThreshold)) {
+          // rescale the running output of this warp's 32 rows: O *= 2^(m_used - m_new)
+          mbar_wait(bar(B_ODONE + h), (n_o + uint32_t(j) - 1u) & 1, abort_flag, p.status);
+          tc_fence_after();
+          const float f = fast_exp2(m_used - (m_new == -INFINITY ? 0.f : m_new));
+#pragma unroll
+          for (int c = 0; c < D / 32; ++c) {
+            uint32_t v[32];
+            tmem_ld32(t_o + uint32_t(c) * 32u, v);
+            tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * f);
+            tmem_st32(t_o + uint32_t(c) * 32u, v);
+          }
+          l *= f;
+          m_used = m_new;
+        }
+        const float ref = m_used == -INFINITY ? 0.f : m_used;
+
+        // pass 2: P = 2^(s - ref) as bf16 pairs, written over the first 64 S columns
+        float sum = 0.f;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          uint32_t v[32];
+          tmem_ld32(t_s + uint32_t(c) * 32u, v);
+          tmem_wait_ld();
+          const uint32_t bits = vis[c];
+          uint32_t pk[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const float p0 = ((bits >> (2 * i)) & 1u) ? fast_exp2(fmaf(__uint_as_float(v[2 * i]), p.scale_log2e, -ref)) : 0.f;
+            const float p1 = ((bits >> (2 * i + 1)) & 1u) ? fast_exp2(fmaf(__uint_as_float(v[2 * i + 1]), p.scale_log2e, -ref)) : 0.f;
+            sum += p0 + p1;
+            pk[i] = pack_bf16x2(p0, p1);
+          }
+          tmem_st16(t_s + uint32_t(c) * 16u, pk);
+        }
+        l += sum;
+
+        // V rows past the end of the request are not ours: zero them (their probabilities are 0, but
+        // 0 * garbage could be NaN).  Half A's warps do it, before P is published to the MMA warp.
+        if (own < BN && h == 0) {
+          mbar_wait(bar(B_SLOT_FULL + vslot % kSlots), (vslot / kSlots) & 1, abort_flag, p.status);
+          uint8_t* v_tile = smem + L::kRingOffset + (vslot % kSlots) * L::kTileBytes;
+          for (int idx = r; idx < (BN - own) * 8 * L::kPanels; idx += BMH) {
+            const int pn = idx / ((BN - own) * 8), rem = idx % ((BN - own) * 8);
+            *reinterpret_cast<uint4*>(v_tile + pn * L::kPanelBytes + (own + rem / 8) * 128 + (rem % 8) * 16) = make_uint4(0u, 0u, 0u, 0u);
+          }
+          fence_proxy_async();
+        }
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(bar(B_PREADY + h));
+      }
+
+      // ---- epilogue: wait for the last PV, read O, normalise (or emit the partial)
+      mbar_wait(bar(B_ODONE + h), (n_o + uint32_t(T) - 1u) & 1, abort_flag, p.status);
+      n_o += uint32_t(T);
+      tc_fence_after();
+      const int head = item.kv_head * g + (row & (g - 1));
+      if (item.slot < 0) {
+        const float inv = l > 0.f ? 1.f / l : 0.f;
+        __nv_bfloat16* out = p.out + (size_t(rq.node0 + node) * p.n_q_heads + head) * D;
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) {
+          uint32_t v[32];
+          tmem_ld32(t_o + uint32_t(c) * 32u, v);
+          tmem_wait_ld();
+          if (ok) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              uint4 o4;
+              o4.x = pack_bf16x2(__uint_as_float(v[8 * i + 0]) * inv, __uint_as_float(v[8 * i + 1]) * inv);
+              o4.y = pack_bf16x2(__uint_as_float(v[8 * i + 2]) * inv, __uint_as_float(v[8 * i + 3]) * inv);
+              o4.z = pack_bf16x2(__uint_as_float(v[8 * i + 4]) * inv, __uint_as_float(v[8 * i + 5]) * inv);
+              o4.w = pack_bf16x2(__uint_as_float(v[8 * i + 6]) * inv, __uint_as_float(v[8 * i + 7]) * inv);
+              *reinterpret_cast<uint4*>(out + c * 32 + i * 8) = o4;
+            }
+          }
+        }
+      } else {
+        // partial slot: O [256][D] fp32, then m [256], then l [256]
+        float* slot = p.partial + size_t(item.slot) * p.slot_floats;
+        const int pr = h * BMH + r;
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) {
+          uint32_t v[32];
+          tmem_ld32(t_o + uint32_t(c) * 32u, v);
+          tmem_wait_ld();
+          if (ok) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+              *reinterpret_cast<uint4*>(slot + pr * D + c * 32 + i * 4) = make_uint4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+          }
+        }
+        if (ok) {
+          slot[2 * BMH * D + pr] = m_used;
+          slot[2 * BMH * D + 2 * BMH + pr] = l;
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(bar(B_OFREE + h));
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 2) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+  }
+}
+
+cudaError_t launch_attn_tc(int head_dim, int n_ctas, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
+                           const AttnParams& p, cudaStream_t stream) {
+  static bool attr_set[2] = {false, false};
+  if (head_dim == 128) {
+    const size_t smem = TcLayout<128>::kTotal + 1024;
+    if (!attr_set[0]) {
+      cudaError_t e = cudaFuncSetAttribute(tree_attn_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+      if (e != cudaSuccess) return e;
+      attr_set[0] = true;
+    }
+    tree_attn_tc_kernel<128><<<n_ctas, kThreads, smem, stream>>>(mq, mk, mv, p);
+  } else {
+    // padded past half of an SM's shared memory: one CTA per SM, since each CTA takes all 512 TMEM columns
+    const size_t smem = 120 * 1024;
+    static_assert(TcLayout<64>::kTotal + 1024 <= 120 * 1024, "smem layout");
+    if (!attr_set[1]) {
+      cudaError_t e = cudaFuncSetAttribute(tree_attn_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+      if (e != cudaSuccess) return e;
+      attr_set[1] = true;
+    }
+    tree_attn_tc_kernel<64><<<n_ctas, kThreads, smem, stream>>>(mq, mk, mv, p);
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace dyspec

@@ -22,15 +22,17 @@ def bf16_tensor_to_bits(t: torch.Tensor) -> np.ndarray:
 class DeviceBatch:
     """Buffers + plan for one Workload.  `step()` = mask build + attention (+ combine) on the current stream."""
 
-    def __init__(self, w: Workload, device="cuda:0", words_per_row: int | None = None, upload: bool = True):
+    def __init__(self, w: Workload, device="cuda:0", words_per_row: int | None = None, upload: bool = True,
+                 plan: "B.Plan | None" = None):
         self.w = w
         self.device = torch.device(device)
         max_n = int(w.n_nodes.max()) if w.n_req else 0
         self.W = words_per_row or B.dyspec_words_per_row(max_n)
         self.total_nodes = w.total_nodes
         self.kv_total_rows = int(w.k.shape[0])
-        self.plan = B.Plan(w.n_q_heads, w.n_kv_heads, w.head_dim, w.prefix_len, w.n_nodes, w.kv_row_offset,
-                           self.kv_total_rows, self.W, 0.0)
+        # a plan depends only on the batch structure, so buffers with the same structure can share one
+        self.plan = plan or B.Plan(w.n_q_heads, w.n_kv_heads, w.head_dim, w.prefix_len, w.n_nodes, w.kv_row_offset,
+                                   self.kv_total_rows, self.W, 0.0)
         dev = self.device
         n = max(1, self.total_nodes)
         self.bits = torch.zeros((n, self.W), dtype=torch.int32, device=dev)

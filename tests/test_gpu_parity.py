@@ -52,6 +52,29 @@ def test_configs_match_oracle(rt, index):
     run_and_check(rt, wl.make_config(index))
 
 
+@pytest.mark.parametrize("case", ["one_tile", "two_halves", "multi_tile", "c3", "c4", "c5"])
+def test_tensor_core_regime(rt, case):
+    """The tcgen05 kernel (regime 1) forced on: single tile first, then both query halves, long key loops, configs."""
+    rng = np.random.default_rng(5)
+    if case == "one_tile":
+        w = wl.make_custom(40, 8, 1, 128, [100], [wl.greedy_tree(rng, 16, 4, 0.3)])        # 128 rows, 2 key tiles
+    elif case == "two_halves":
+        w = wl.make_custom(41, 8, 1, 128, [128], [wl.greedy_tree(rng, 32, 4, 0.3)])        # 256 rows
+    elif case == "multi_tile":
+        w = wl.make_custom(42, 16, 2, 128, [1500, 300], [wl.greedy_tree(rng, 200, 8, 0.2), wl.chain_tree(70)])
+    else:
+        w = wl.make_config(int(case[1]))
+    run_and_check(rt, w, regime=1)
+
+
+@pytest.mark.parametrize("hq,hkv,d", [(8, 1, 64), (4, 4, 64), (4, 4, 128), (4, 2, 128)])
+def test_tensor_core_regime_shapes(rt, hq, hkv, d):
+    rng = np.random.default_rng(hq * 10 + d)
+    trees = [wl.greedy_tree(rng, 300, 8, 0.3), wl.random_tree(rng, 130, 0.05), np.zeros(0, np.int32), wl.chain_tree(129)]
+    for ctas in (0, 5):
+        run_and_check(rt, wl.make_custom(15, hq, hkv, d, [260, 64, 3, 0], trees), regime=1, ctas=ctas)
+
+
 @pytest.mark.parametrize("ctas", [1, 3, 40, 1000])
 def test_split_count_does_not_change_results(rt, ctas):
     """Forcing the scheduler to balance over few or many CTAs changes the split-KV cuts, not the answer."""

@@ -62,7 +62,7 @@ def test_five_configs_schedule(B):
     for idx in range(1, 6):
         w = wl.make_config(idx)
         info, loads = check_schedule(B, w.n_q_heads, w.n_kv_heads, w.head_dim, w.prefix_len.tolist(), w.n_nodes.tolist())
-        assert info["ctas"] <= 2 * 148 + 8
+        assert info["ctas"] <= (2 if info["regime"] == 0 else 1) * 148 + 8
         if idx >= 2:
             assert max(loads) <= 1.5 * (sum(loads) / len(loads)) + 4
 
@@ -83,4 +83,12 @@ def test_degenerate_batches(B):
 
 def test_regime_1_tiles(B):
     info, _ = check_schedule(B, 64, 8, 128, [2048], [512], regime=1)
-    assert info["rows_per_tile"] == 128 and info["regime"] == 1
+    assert info["rows_per_tile"] == 256 and info["keys_per_tile"] == 128 and info["regime"] == 1
+
+
+def test_regime_is_chosen_from_packed_rows(B):
+    # nodes x group <= 64 rows: warp-level tiles; more: tcgen05 tiles
+    assert check_schedule(B, 32, 32, 128, [1024], [64])[0]["regime"] == 0
+    assert check_schedule(B, 64, 8, 128, [1024], [8])[0]["regime"] == 0
+    assert check_schedule(B, 64, 8, 128, [1024], [9])[0]["regime"] == 1
+    assert check_schedule(B, 32, 32, 128, [4096], [256])[0]["regime"] == 1
