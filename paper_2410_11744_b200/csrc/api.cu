@@ -131,6 +131,15 @@ void schedule(dyspec_plan& pl) {
   int64_t target = (total_cost + max_ctas - 1) / max_ctas;
   if (target < item_cost + min_tiles) target = item_cost + min_tiles;
 
+  // Deal the tiles out with a per-CTA budget of `target`; a budget that leaves a CTA too little
+  // room for a useful piece moves on to the next CTA, so the count can overshoot: grow the budget
+  // until the work fits in max_ctas (one wave).
+  for (int attempt = 0; attempt < 64; ++attempt) {
+  pl.items.clear();
+  pl.cta_begin.clear();
+  pl.split_groups.clear();
+  pl.n_slots = 0;
+  pl.max_splits = 1;
   int64_t used = 0;
   pl.cta_begin.push_back(0);
   for (size_t gi = 0; gi < groups.size(); ++gi) {
@@ -172,6 +181,9 @@ void schedule(dyspec_plan& pl) {
   }
   pl.cta_begin.push_back(int32_t(pl.items.size()));
   pl.n_ctas = int(pl.cta_begin.size()) - 1;
+  if (pl.n_ctas <= max_ctas) break;
+  target += std::max<int64_t>(1, target / 16);
+  }
 }
 
 int upload(dyspec_plan& pl) {
