@@ -13,7 +13,7 @@
 
 namespace dyspec {
 // kernels (defined in the other translation units)
-cudaError_t launch_build_tree_mask(const int32_t* parents, const ReqInfo* reqs, int n_req, int single_n,
+cudaError_t launch_build_tree_mask(const int32_t* parents, const ReqInfo* reqs, int n_req, int single_n, int max_n,
                                    uint32_t* bits, int32_t* depths, int W, int32_t* status, cudaStream_t stream);
 cudaError_t launch_attn_mma(int head_dim, int n_ctas, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                             const AttnParams& p, cudaStream_t stream);
@@ -70,6 +70,7 @@ struct dyspec_plan {
   int n_req = 0;
   int64_t kv_total_rows = 0;
   int64_t total_nodes = 0;
+  int max_nodes = 0;
   int regime = 0, bm = 64, bn = 64;
   std::vector<ReqInfo> reqs;
   std::vector<WorkItem> items;
@@ -182,7 +183,7 @@ void schedule(dyspec_plan& pl) {
   pl.cta_begin.push_back(int32_t(pl.items.size()));
   pl.n_ctas = int(pl.cta_begin.size()) - 1;
   if (pl.n_ctas <= max_ctas) break;
-  target += std::max<int64_t>(1, target / 16);
+  target += std::max<int64_t>(1, target / 64);
   }
 }
 
@@ -256,7 +257,7 @@ int dyspec_build_tree_mask(const int32_t* parents, int n_nodes, uint32_t* ancest
   if (n_nodes == 0) return DYSPEC_OK;
   if (!parents || !ancestor_bits) return DYSPEC_ERR_INVALID_ARG;
   if (!aligned(ancestor_bits, 16) || !aligned(parents, 4)) return DYSPEC_ERR_INVALID_ARG;
-  cudaError_t e = launch_build_tree_mask(parents, nullptr, 1, n_nodes, ancestor_bits, depths, words_per_row, status,
+  cudaError_t e = launch_build_tree_mask(parents, nullptr, 1, n_nodes, n_nodes, ancestor_bits, depths, words_per_row, status,
                                          reinterpret_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? DYSPEC_OK : DYSPEC_ERR_CUDA;
 }
@@ -294,6 +295,7 @@ static int make_host_plan(dyspec_plan** out, int n_q_heads, int n_kv_heads, int 
     pl->reqs.push_back(rq);
     node0 += n_nodes[r];
     max_rows = std::max(max_rows, n_nodes[r] * g);
+    pl->max_nodes = std::max(pl->max_nodes, int(n_nodes[r]));
   }
   if (node0 >= (int64_t(1) << 31)) { delete pl; return DYSPEC_ERR_UNSUPPORTED; }
   pl->total_nodes = node0;
@@ -379,7 +381,7 @@ int dyspec_plan_build_tree_mask(const dyspec_plan_t* plan, const int32_t* parent
   if (!plan) return DYSPEC_ERR_INVALID_ARG;
   if (plan->n_req == 0 || plan->total_nodes == 0) return DYSPEC_OK;
   if (!parents || !ancestor_bits || !aligned(ancestor_bits, 16)) return DYSPEC_ERR_INVALID_ARG;
-  cudaError_t e = launch_build_tree_mask(parents, plan->d_reqs, plan->n_req, 0, ancestor_bits, depths, plan->W, status,
+  cudaError_t e = launch_build_tree_mask(parents, plan->d_reqs, plan->n_req, 0, plan->max_nodes, ancestor_bits, depths, plan->W, status,
                                          reinterpret_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? DYSPEC_OK : DYSPEC_ERR_CUDA;
 }
