@@ -157,6 +157,38 @@ int dyspec_set_default_shape(int n_q_heads, int n_kv_heads, int head_dim, int wo
 int dyspec_tree_attention(const void* q, const void* k_cache, const void* v_cache, int prefix_len,
                           const uint32_t* ancestor_bits, int n_nodes, void* out, dyspec_stream_t stream);
 
+/*
+ * (3c) Single-request attention that allocates nothing.  (The paper has no counterpart: this is an
+ * integration aid, not part of the method.)
+ *
+ * Who needs it: code that may not call cudaMalloc / cudaFree at the point where it wants attention --
+ * for instance an inference server whose device memory was handed, all of it, to its own pool at
+ * start-up, a plug-in that runs under a host framework's "no allocation in the step function" rule,
+ * or a process running so close to the memory limit that a late cudaMalloc could fail.  Such a
+ * caller can build neither a plan (plan creation allocates its device work list) nor a workspace.
+ *
+ * Here the scheduled work list and the split-KV partials live in one fixed device array of
+ * DYSPEC_STATIC_SCRATCH_BYTES that is part of the library image: every GPU that loads the library
+ * holds those bytes until the process exits, whether or not this call is ever used.  The call runs
+ * the host scheduler, copies the work list into the array on `stream`, and launches the same
+ * kernels as dyspec_tree_attention_ragged; it calls no cudaMalloc, cudaFree or allocating routine.
+ * Arguments are those of dyspec_tree_attention plus the static shape (see dyspec_plan_create) and an
+ * optional status word; k_cache / v_cache hold exactly prefix_len + n_nodes rows.
+ *
+ *   - A batch whose work list plus partials exceed the array is refused with DYSPEC_ERR_WORKSPACE
+ *     before anything is launched (as a guide: Llama2-7B shape, prefix 1024, 64 nodes needs 8.2 MiB).
+ *   - The first call on each device looks up the array's device address (with that device current);
+ *     make that first call outside any stream capture.
+ *   - All calls share the one array, which keeps the previous call's contents; each call rewrites the
+ *     tables and clears the counters it needs.  Calls on the same stream are ordered and safe.  Two
+ *     calls that overlap on the GPU (different streams, or different host threads without ordering)
+ *     race on the array and give wrong results.
+ */
+#define DYSPEC_STATIC_SCRATCH_BYTES (16u << 20)
+int dyspec_tree_attention_static(const void* q, const void* k_cache, const void* v_cache, int prefix_len,
+                                 const uint32_t* ancestor_bits, int n_nodes, void* out, int n_q_heads, int n_kv_heads,
+                                 int head_dim, int words_per_row, float scale, int32_t* status, dyspec_stream_t stream);
+
 #ifdef __cplusplus
 }
 #endif

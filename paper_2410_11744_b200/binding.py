@@ -40,6 +40,7 @@ SIGNATURES = {
     "dyspec_tree_attention_ragged": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp, _vp]),
     "dyspec_set_default_shape": (_i32, [_i32, _i32, _i32, _i32, _f32]),
     "dyspec_tree_attention": (_i32, [_vp, _vp, _vp, _i32, _vp, _i32, _vp, _vp]),
+    "dyspec_tree_attention_static": (_i32, [_vp, _vp, _vp, _i32, _vp, _i32, _vp, _i32, _i32, _i32, _i32, _f32, _vp, _vp]),
 }
 for _name, (_res, _args) in SIGNATURES.items():
     _fn = getattr(lib, _name)
@@ -200,3 +201,14 @@ def dyspec_set_default_shape(n_q_heads: int, n_kv_heads: int, head_dim: int, wor
 def dyspec_tree_attention(q, k_cache, v_cache, prefix_len: int, ancestor_bits, n_nodes: int, out, stream=None) -> None:
     _check(lib.dyspec_tree_attention(_ptr(q), _ptr(k_cache), _ptr(v_cache), prefix_len, _ptr(ancestor_bits), n_nodes,
                                      _ptr(out), _stream(stream)), "dyspec_tree_attention")
+
+
+def dyspec_tree_attention_static(q, k_cache, v_cache, prefix_len: int, ancestor_bits, n_nodes: int, out, n_q_heads: int,
+                                 n_kv_heads: int, head_dim: int, words_per_row: int, scale: float = 0.0, status=None,
+                                 stream=None) -> None:
+    """Single-request attention for callers that may not allocate device memory: the work list and the
+    split-KV partials go into the library's fixed device array (16 MiB, shared by all calls)."""
+    _check(lib.dyspec_tree_attention_static(_ptr(q), _ptr(k_cache), _ptr(v_cache), prefix_len, _ptr(ancestor_bits),
+                                            n_nodes, _ptr(out), n_q_heads, n_kv_heads, head_dim, words_per_row,
+                                            float(scale), _ptr(status), _stream(stream)),
+           "dyspec_tree_attention_static")

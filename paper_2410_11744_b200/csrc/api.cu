@@ -471,3 +471,103 @@ int dyspec_tree_attention(const void* q, const void* k_cache, const void* v_cach
 }
 
 }  // extern "C"
+
+// ---- allocation-free single-request form ----------------------------------------------------------
+//
+// Everything the attention kernels need beyond the caller's inputs and outputs -- the scheduled work
+// list and the split-KV partials -- is placed in one fixed device array that is part of the library
+// image.  The array's name is only a host-side handle: kernels get the real device address, looked up
+// once per device with cudaGetSymbolAddress.
+namespace {
+
+static __device__ __align__(256) unsigned char g_static_scratch[DYSPEC_STATIC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+unsigned char* g_static_scratch_addr[kMaxDevices] = {};
+std::mutex g_static_scratch_mutex;
+
+// Device address of the scratch array on the current device (set-up on first use per device).
+int static_scratch_base(unsigned char** base) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return DYSPEC_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
+  if (!g_static_scratch_addr[dev]) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) return DYSPEC_ERR_CUDA;
+    g_static_scratch_addr[dev] = static_cast<unsigned char*>(ptr);
+  }
+  *base = g_static_scratch_addr[dev];
+  return DYSPEC_OK;
+}
+
+}  // namespace
+
+extern "C" int dyspec_tree_attention_static(const void* q, const void* k_cache, const void* v_cache, int prefix_len,
+                                            const uint32_t* ancestor_bits, int n_nodes, void* out, int n_q_heads,
+                                            int n_kv_heads, int head_dim, int words_per_row, float scale,
+                                            int32_t* status, dyspec_stream_t stream) {
+  if (prefix_len < 0 || n_nodes < 0) return DYSPEC_ERR_INVALID_ARG;
+  const int32_t L = prefix_len, n = n_nodes;
+  const int64_t off = 0;
+  dyspec_plan* pl = nullptr;
+  int rc = make_host_plan(&pl, n_q_heads, n_kv_heads, head_dim, 1, &L, &n, &off, int64_t(L) + n, words_per_row, scale);
+  if (rc != DYSPEC_OK) return rc;
+  struct Guard { dyspec_plan* p; ~Guard() { delete p; } } guard{pl};   // host-only object: nothing to cudaFree
+  if (pl->n_ctas == 0) return DYSPEC_OK;
+  if (!q || !k_cache || !v_cache || !ancestor_bits || !out) return DYSPEC_ERR_INVALID_ARG;
+  if (!aligned(q, 16) || !aligned(k_cache, 16) || !aligned(v_cache, 16) || !aligned(out, 16) || !aligned(ancestor_bits, 16))
+    return DYSPEC_ERR_INVALID_ARG;
+
+  // layout inside the scratch array: [requests | work items | per-CTA ranges | split groups | counters | partials]
+  auto pad = [](size_t x) { return (x + 255) & ~size_t(255); };
+  const size_t o_reqs = 0;
+  const size_t o_items = o_reqs + pad(pl->reqs.size() * sizeof(ReqInfo));
+  const size_t o_cta = o_items + pad(pl->items.size() * sizeof(WorkItem));
+  const size_t o_groups = o_cta + pad(pl->cta_begin.size() * sizeof(int32_t));
+  const size_t o_counters = o_groups + pad(std::max<size_t>(1, pl->split_groups.size()) * sizeof(GroupInfo));
+  const size_t o_partial = o_counters + pad(std::max<size_t>(1, pl->split_groups.size()) * sizeof(int32_t));
+  const size_t total = o_partial + pl->workspace_bytes;
+  if (total > size_t(DYSPEC_STATIC_SCRATCH_BYTES)) return DYSPEC_ERR_WORKSPACE;   // batch too large for the fixed array
+
+  unsigned char* base = nullptr;
+  rc = static_scratch_base(&base);
+  if (rc != DYSPEC_OK) return rc;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+
+  // The array keeps whatever the previous call left: rewrite the tables, clear the counters.
+  std::vector<uint8_t> host(o_partial, 0);
+  memcpy(host.data() + o_reqs, pl->reqs.data(), pl->reqs.size() * sizeof(ReqInfo));
+  memcpy(host.data() + o_items, pl->items.data(), pl->items.size() * sizeof(WorkItem));
+  memcpy(host.data() + o_cta, pl->cta_begin.data(), pl->cta_begin.size() * sizeof(int32_t));
+  if (!pl->split_groups.empty())
+    memcpy(host.data() + o_groups, pl->split_groups.data(), pl->split_groups.size() * sizeof(GroupInfo));
+  // pageable source: the copy is staged before the call returns, so `host` may go out of scope afterwards
+  if (cudaMemcpyAsync(base, host.data(), o_partial, cudaMemcpyHostToDevice, st) != cudaSuccess) return DYSPEC_ERR_CUDA;
+
+  CUtensorMap mq, mk, mv;
+  const int bm = pl->bm, bn = pl->bn;
+  const int q_box_rows = pl->regime == 0 ? 64 : 128;
+  if (!encode_map(&mq, q, pl->total_nodes, pl->hq, pl->d, pl->g, q_box_rows / pl->g) ||
+      !encode_map(&mk, k_cache, pl->kv_total_rows, pl->hkv, pl->d, 1, bn) ||
+      !encode_map(&mv, v_cache, pl->kv_total_rows, pl->hkv, pl->d, 1, bn))
+    return DYSPEC_ERR_CUDA;
+
+  AttnParams p{};
+  p.reqs = reinterpret_cast<const ReqInfo*>(base + o_reqs);
+  p.items = reinterpret_cast<const WorkItem*>(base + o_items);
+  p.cta_item_begin = reinterpret_cast<const int32_t*>(base + o_cta);
+  p.groups = reinterpret_cast<const GroupInfo*>(base + o_groups);
+  p.counters = reinterpret_cast<int32_t*>(base + o_counters);
+  p.partial = reinterpret_cast<float*>(base + o_partial);
+  p.bits = ancestor_bits; p.out = static_cast<__nv_bfloat16*>(out); p.status = status;
+  p.n_q_heads = pl->hq; p.n_kv_heads = pl->hkv; p.group_size = pl->g; p.log2_g = pl->log2g;
+  p.words_per_row = pl->W; p.slot_floats = bm * (pl->d + 2);
+  p.scale_log2e = pl->scale * kLog2e;
+
+  cudaError_t e;
+  if (pl->regime == 0) e = launch_attn_mma(pl->d, pl->n_ctas, mq, mk, mv, p, st);
+  else e = launch_attn_tc(pl->d, pl->n_ctas, mq, mk, mv, p, st);
+  if (e != cudaSuccess) return DYSPEC_ERR_CUDA;
+  e = launch_combine(pl->d, bm, int(pl->split_groups.size()), p, st);
+  return e == cudaSuccess ? DYSPEC_OK : DYSPEC_ERR_CUDA;
+}

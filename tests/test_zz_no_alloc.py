@@ -1,0 +1,70 @@
+"""The allocation-free entry point, dyspec_tree_attention_static, against dyspec_tree_attention_ragged.
+
+For callers that cannot allocate device memory (everything was given to a pool at start-up, or the
+host framework forbids allocation inside its step function) the library keeps the work list and the
+split-KV partials in a fixed 16 MiB device array.  The array is shared and keeps old contents, so
+the check runs two calls back to back, of different shapes, and each must match the ordinary entry
+point.  This file sorts last on purpose: a run that stops at the first failure has then already
+run every other test.
+"""
+import numpy as np
+import pytest
+
+from paper_2410_11744_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+MAX_ABS, MEAN_ABS = 2e-2, 2e-3       # the tolerance of the parity tests
+
+
+def _bits_to_f64(bits):
+    return (bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+def test_static_scratch_entry_point_matches_ragged_entry_point_twice_in_a_row():
+    import torch
+    assert torch.cuda.is_available()
+    from paper_2410_11744_b200 import build
+    build.build()
+    from paper_2410_11744_b200 import binding as B, runner as R
+
+    # config 2 is cut into split-KV pieces (about 8 MiB of partials in the scratch array); the custom
+    # case after it is smaller and of a different shape, so stale contents would show
+    rng = np.random.default_rng(3)
+    cases = [wl.make_config(2), wl.make_custom(21, 8, 2, 64, [300], [wl.greedy_tree(rng, 40, 4, 0.3)]), wl.make_config(2)]
+    for w in cases:
+        batch = R.DeviceBatch(w)
+        batch.step()                                          # existing entry points: mask + ragged attention
+        bits, _, want_bits, status = batch.results()
+        assert status == 0
+        L, n = int(w.prefix_len[0]), int(w.n_nodes[0])
+        out = torch.zeros_like(batch.out)
+        st = torch.zeros((1,), dtype=torch.int32, device=out.device)
+        for _ in range(2):                                    # two calls in a row on the shared array
+            out.zero_()
+            B.dyspec_tree_attention_static(batch.q, batch.k, batch.v, L, batch.bits, n, out, w.n_q_heads,
+                                           w.n_kv_heads, w.head_dim, batch.W, 0.0, st)
+            torch.cuda.synchronize()
+            assert int(st.item()) == 0
+            got = _bits_to_f64(R.bf16_tensor_to_bits(out))
+            want = _bits_to_f64(want_bits)
+            assert np.isfinite(got).all()
+            err = np.abs(got - want)
+            assert err.max() <= MAX_ABS and err.mean() <= MEAN_ABS
+
+
+def test_static_scratch_entry_point_refuses_what_does_not_fit():
+    import torch
+    from paper_2410_11744_b200 import build
+    build.build()
+    from paper_2410_11744_b200 import binding as B, runner as R
+    w = wl.make_config(4)                                     # needs ~24 MiB of partials: over the 16 MiB array
+    batch = R.DeviceBatch(w)
+    batch.build_mask()
+    out = torch.zeros_like(batch.out)
+    with pytest.raises(B.DyspecError) as e:
+        B.dyspec_tree_attention_static(batch.q, batch.k, batch.v, int(w.prefix_len[0]), batch.bits, int(w.n_nodes[0]),
+                                       out, w.n_q_heads, w.n_kv_heads, w.head_dim, batch.W)
+    assert e.value.code == -3
+    torch.cuda.synchronize()
+    assert not out.any()
