@@ -119,6 +119,13 @@ int dyspec_schedule_dry_run(int n_q_heads, int n_kv_heads, int head_dim, int n_r
  * CTAs the scheduler balances over (<= 0 = automatic). */
 int dyspec_set_tuning(int force_regime, int force_ctas);
 
+/* Developer aid: event trace of the attention kernels.  trace_buffer is a dev uint64 array of
+ * capacity_entries entries that the caller zeroes; while set, CTA 0 of every tensor-core attention
+ * launch writes (tag << 44 | SM clock) entries into three equal regions (MMA issuer, softmax half A,
+ * softmax half B; tags are listed in csrc/attn_tc.cu; zero entries are unused).  Pass (NULL, 0) to
+ * switch it off (the default). */
+int dyspec_set_trace(void* trace_buffer, int capacity_entries);
+
 /*
  * (1b) Mask builder for the whole ragged batch of a plan: request r's parents (request-local
  * indices) start at node_offset_r, its mask rows and depths likewise.

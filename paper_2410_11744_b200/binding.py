@@ -30,6 +30,7 @@ SIGNATURES = {
     "dyspec_version": (_i32, []),
     "dyspec_words_per_row": (_i32, [_i32]),
     "dyspec_set_tuning": (_i32, [_i32, _i32]),
+    "dyspec_set_trace": (_i32, [_vp, _i32]),
     "dyspec_build_tree_mask": (_i32, [_vp, _i32, _vp, _vp, _i32, _vp, _vp]),
     "dyspec_plan_create": (_i32, [_c.POINTER(_vp), _i32, _i32, _i32, _i32, _vp, _vp, _vp, _i64, _i32, _f32]),
     "dyspec_plan_destroy": (_i32, [_vp]),
@@ -90,6 +91,10 @@ def dyspec_words_per_row(max_nodes: int) -> int:
 
 def dyspec_set_tuning(force_regime: int = -1, force_ctas: int = 0) -> None:
     _check(lib.dyspec_set_tuning(force_regime, force_ctas), "dyspec_set_tuning")
+
+
+def dyspec_set_trace(trace_buffer=None, capacity_entries: int = 0) -> None:
+    _check(lib.dyspec_set_trace(_ptr(trace_buffer), capacity_entries), "dyspec_set_trace")
 
 
 def dyspec_build_tree_mask(parents, n_nodes: int, ancestor_bits, depths=None, words_per_row: int = 0,

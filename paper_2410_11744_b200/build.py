@@ -40,6 +40,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     common = ["-O3", "-std=c++17", "-lineinfo", "-Xcompiler", "-fPIC", "--use_fast_math"] + ARCH
     if verbose:
         common += ["-Xptxas", "-v"]
+    common += os.environ.get("DYSPEC_NVCC_FLAGS", "").split()   # developer experiments (-D...)
     procs = []
     for src in SOURCES:
         obj = os.path.join(objdir, src.replace(".cu", ".o"))

@@ -28,6 +28,8 @@ namespace {
 
 int g_force_regime = -1;
 int g_force_ctas = 0;
+unsigned long long* g_trace = nullptr;   // device buffer for the optional kernel event trace
+int g_trace_capacity = 0;
 
 using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -249,6 +251,13 @@ int dyspec_set_tuning(int force_regime, int force_ctas) {
   return DYSPEC_OK;
 }
 
+int dyspec_set_trace(void* trace_buffer, int capacity_entries) {
+  if (capacity_entries < 0 || (trace_buffer == nullptr) != (capacity_entries == 0)) return DYSPEC_ERR_INVALID_ARG;
+  g_trace = static_cast<unsigned long long*>(trace_buffer);
+  g_trace_capacity = capacity_entries;
+  return DYSPEC_OK;
+}
+
 int dyspec_build_tree_mask(const int32_t* parents, int n_nodes, uint32_t* ancestor_bits, int32_t* depths,
                            int words_per_row, int32_t* status, dyspec_stream_t stream) {
   if (n_nodes < 0 || words_per_row <= 0 || (words_per_row & 3)) return DYSPEC_ERR_INVALID_ARG;
@@ -413,6 +422,7 @@ int dyspec_tree_attention_ragged(const dyspec_plan_t* plan, const void* q, const
   p.n_q_heads = plan->hq; p.n_kv_heads = plan->hkv; p.group_size = plan->g; p.log2_g = plan->log2g;
   p.words_per_row = plan->W; p.slot_floats = bm * (plan->d + 2);
   p.scale_log2e = plan->scale * kLog2e;
+  p.trace = g_trace; p.trace_capacity = g_trace_capacity;
 
   cudaError_t e;
   if (plan->regime == 0) e = launch_attn_mma(plan->d, plan->n_ctas, mq, mk, mv, p, st);

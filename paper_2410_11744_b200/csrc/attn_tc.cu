@@ -40,6 +40,13 @@ struct TcLayout {
   static constexpr int kTotal = kBarOffset + 512;
 };
 
+// Trace tags (see dyspec_set_trace): tag = role << 14 | event << 10 | key-tile index j.
+// role 0 = MMA issuer, 1 = softmax half A (row 0), 2 = softmax half B (row 0).
+// MMA events: 1 / 3 P ready seen (half A / B), 5 / 6 PV issued, 2 / 4 next QK issued.  Softmax events: 1 S ready seen, 2 S row loaded,
+// 3 maximum known, 4 P stored (before wait::st), 5 P published, 6 last PV seen, 7 epilogue done.
+// MMA event 9 = role start, 7 = end-of-tile commits issued, 8 = V slot seen.
+#define DYSPEC_TAG(role, event, j) ((uint32_t(role) << 14) | (uint32_t(event) << 10) | (uint32_t(j) & 1023u))
+
 // barrier indices (8 bytes each)
 enum { B_QFULL = 0, B_QFREE = 1, B_SLOT_FULL = 2, B_SLOT_EMPTY = B_SLOT_FULL + kSlots,
        B_SREADY = B_SLOT_EMPTY + kSlots, B_PREADY = B_SREADY + 2, B_ODONE = B_PREADY + 2, B_OFREE = B_ODONE + 2,
@@ -63,6 +70,29 @@ __device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64
       ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
 }
 
+// The same MMAs with the descriptors given as (low word, constant high word): the issuing thread then
+// spends one integer add per instruction instead of rebuilding 64-bit descriptors.
+__device__ __forceinline__ void umma_ss_lohi(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                             uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tsetp.ne.b32 p, %6, 0;\n\t"
+      "mov.b64 da, {%1, %2};\n\tmov.b64 db, {%3, %4};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void umma_ts_lohi(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
+                                             uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+      "mov.b64 db, {%2, %3};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(acc) : "memory");
+}
+// Descriptor words: low = address >> 4 | (leading byte offset >> 4) << 16; high = stride byte offset >> 4 |
+// version 1 (bit 46) | 128-byte swizzle (bits 61-63).
+__host__ __device__ constexpr uint32_t desc_hi(uint32_t sbo_bytes) { return (sbo_bytes >> 4) | (1u << 14) | (2u << 29); }
+__device__ __forceinline__ uint32_t desc_lo(uint32_t saddr, uint32_t lbo_bytes) { return (saddr >> 4) | ((lbo_bytes >> 4) << 16); }
+
 // Shared-memory matrix descriptor, 128-byte swizzle, version 1 (sm_100).  Offsets are in bytes.
 __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
   return uint64_t((saddr >> 4) & 0x3FFFu) | (uint64_t((lbo_bytes >> 4) & 0x3FFFu) << 16) |
@@ -73,7 +103,7 @@ __host__ __device__ constexpr uint32_t make_idesc(int n, int b_mn_major) {
   return (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(b_mn_major) << 16) | (uint32_t(n >> 3) << 17) | (uint32_t(128 >> 4) << 24);
 }
 
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
       "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
@@ -83,7 +113,7 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
         "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr));
 }
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
   asm volatile(
       "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
       "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
@@ -93,7 +123,7 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
         "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
       : "memory");
 }
-__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
   asm volatile(
       "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
       ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
@@ -152,6 +182,9 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   const int item_end = p.cta_item_begin[blockIdx.x + 1];
   const int g = p.group_size;
 
+  // Register budget: the softmax threads hold a whole S row; the control warps need few registers.
+  if (warp < 4) {
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
@@ -177,6 +210,9 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             const int slot = sc % kSlots;
             const uint32_t ph = (sc / kSlots) & 1;
             mbar_wait(bar(B_SLOT_EMPTY + slot), ph ^ 1, abort_flag, p.status);
+#ifdef EXP_SKIP_LOADS
+            if (sc >= kSlots) { mbar_arrive(bar(B_SLOT_FULL + slot)); continue; }
+#endif
             mbar_expect_tx(bar(B_SLOT_FULL + slot), L::kTileBytes);
             for (int pn = 0; pn < L::kPanels; ++pn)
               tma_load_3d(s_ring + slot * L::kTileBytes + pn * L::kPanelBytes, kv == 0 ? &map_k : &map_v,
@@ -188,77 +224,109 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
+      TraceCursor tc_cur = trace_open(p, 0, 3);
+      trace_event(tc_cur, DYSPEC_TAG(0, 9, 0));
       constexpr uint32_t idesc_qk = make_idesc(BN, 0);
       constexpr uint32_t idesc_pv = make_idesc(D, 1);
-      uint32_t sc = 0, qit = 0;
-      uint32_t n_p[2] = {0, 0};      // P-ready phases consumed per half
-      uint32_t n_items_h[2] = {0, 0};
-      auto issue_qk = [&](int h, int slot) {
-        const uint32_t a_base = s_q + h * L::kTileBytes;
-        const uint32_t b_base = s_ring + slot * L::kTileBytes;
+      constexpr uint32_t kHiK = desc_hi(1024);            // K-major operands (Q, K): 8-row groups 1024 B apart
+      constexpr uint32_t kHiV = desc_hi(1024);            // MN-major operand (V): 8-key groups 1024 B apart
+      const uint32_t q_lo0 = desc_lo(s_q, 16);
+      const uint32_t ring_k_lo0 = desc_lo(s_ring, 16);
+      const uint32_t ring_v_lo0 = desc_lo(s_ring, L::kPanelBytes);   // leading offset = next 64-column panel
+      auto issue_qk = [=](int h, uint32_t slot) {
+        const uint32_t a_lo = q_lo0 + uint32_t(h) * (L::kTileBytes >> 4);
+        const uint32_t b_lo = ring_k_lo0 + slot * (L::kTileBytes >> 4);
+        const uint32_t d_tmem = tmem_base + uint32_t(h) * 128u;
 #pragma unroll
         for (int ks = 0; ks < D / 16; ++ks) {
-          const uint32_t off = uint32_t(ks >> 2) * L::kPanelBytes + uint32_t(ks & 3) * 32u;
-          umma_ss(tmem_base + uint32_t(h) * 128u, make_desc(a_base + off, 16, 1024), make_desc(b_base + off, 16, 1024),
-                  idesc_qk, ks > 0 ? 1u : 0u);
+          const uint32_t off = (uint32_t(ks >> 2) * L::kPanelBytes + uint32_t(ks & 3) * 32u) >> 4;
+          umma_ss_lohi(d_tmem, a_lo + off, kHiK, b_lo + off, kHiK, idesc_qk, ks > 0 ? 1u : 0u);
         }
-        tc_commit(bar(B_SREADY + h));
+        tc_commit(s_bar + 8u * uint32_t(B_SREADY + h));
       };
-      auto issue_pv = [&](int h, int slot, bool accumulate) {
-        const uint32_t b_base = s_ring + slot * L::kTileBytes;
+      auto issue_pv = [=](int h, uint32_t slot, bool accumulate) {
+        const uint32_t b_lo = ring_v_lo0 + slot * (L::kTileBytes >> 4);
+        const uint32_t d_tmem = tmem_base + 256u + uint32_t(h) * 128u;
+        const uint32_t a_tmem = tmem_base + uint32_t(h) * 128u;
 #pragma unroll
-        for (int kk = 0; kk < BN / 16; ++kk) {
-          umma_ts(tmem_base + 256u + uint32_t(h) * 128u, tmem_base + uint32_t(h) * 128u + uint32_t(kk) * 8u,
-                  make_desc(b_base + uint32_t(kk) * 2048u, L::kPanelBytes, 1024), idesc_pv, (accumulate || kk > 0) ? 1u : 0u);
-        }
-        tc_commit(bar(B_ODONE + h));
+        for (int kk = 0; kk < BN / 16; ++kk)
+          umma_ts_lohi(d_tmem, a_tmem + uint32_t(kk) * 8u, b_lo + uint32_t(kk) * (2048u >> 4), kHiV, idesc_pv,
+                       (accumulate || kk > 0) ? 1u : 0u);
       };
+      uint32_t sc = 0, qit = 0;
+      uint32_t n_p0 = 0, n_p1 = 0;          // P-ready phases consumed per half
+      uint32_t n_it0 = 0, n_it1 = 0;        // items seen per half (O-free phase)
       for (int w = item_begin; w < item_end; ++w, ++qit) {
         const WorkItem item = p.items[w];
         const ReqInfo rq = p.reqs[item.req];
-        const int nh = (rq.n_nodes * g - item.row0 > BMH) ? 2 : 1;
+        const bool two = rq.n_nodes * g - item.row0 > BMH;        // both query halves live
         const int T = item.tile_end - item.tile_begin;
         mbar_wait(bar(B_QFULL), qit & 1, abort_flag, p.status);
         {
-          const uint32_t kslot = sc++;
-          mbar_wait(bar(B_SLOT_FULL + kslot % kSlots), (kslot / kSlots) & 1, abort_flag, p.status);
+          const uint32_t kslot = sc % kSlots, kph = (sc / kSlots) & 1;
+          ++sc;
+          mbar_wait(bar(B_SLOT_FULL + kslot), kph, abort_flag, p.status);
           tc_fence_after();
-          for (int h = 0; h < nh; ++h) issue_qk(h, kslot % kSlots);
-          tc_commit(bar(B_SLOT_EMPTY + kslot % kSlots));
+          issue_qk(0, kslot);
+          if (two) issue_qk(1, kslot);
+          tc_commit(bar(B_SLOT_EMPTY + kslot));
+          if (T == 1) tc_commit(bar(B_QFREE));            // Q is reusable once the item's last QK^T has run
         }
         for (int j = 0; j < T; ++j) {
-          const uint32_t vslot = sc++;
+          const uint32_t vslot = sc % kSlots, vph = (sc / kSlots) & 1;
+          ++sc;
           const bool more = j + 1 < T;
-          const uint32_t kslot = more ? sc++ : 0u;
-          mbar_wait(bar(B_SLOT_FULL + vslot % kSlots), (vslot / kSlots) & 1, abort_flag, p.status);
-          for (int h = 0; h < nh; ++h) {
-            if (j == 0) mbar_wait(bar(B_OFREE + h), (n_items_h[h] & 1) ^ 1, abort_flag, p.status);
-            mbar_wait(bar(B_PREADY + h), n_p[h] & 1, abort_flag, p.status);
-            ++n_p[h];
-            tc_fence_after();
-            issue_pv(h, vslot % kSlots, j > 0);
-            if (more) {
-              if (h == 0) {
-                mbar_wait(bar(B_SLOT_FULL + kslot % kSlots), (kslot / kSlots) & 1, abort_flag, p.status);
-                tc_fence_after();
-              }
-              issue_qk(h, kslot % kSlots);
-            }
+          const uint32_t kslot = sc % kSlots, kph = (sc / kSlots) & 1;
+          if (more) ++sc;
+          // Slot waits first: an mbarrier wait costs ~180 cycles even when its phase completed long
+          // ago; here that latency hides behind the softmax this thread has to wait for anyway.
+          mbar_wait(bar(B_SLOT_FULL + vslot), vph, abort_flag, p.status);
+          if (more) mbar_wait(bar(B_SLOT_FULL + kslot), kph, abort_flag, p.status);
+          if (j == 0) {
+            mbar_wait(bar(B_OFREE + 0), (n_it0 & 1) ^ 1, abort_flag, p.status);
+            if (two) mbar_wait(bar(B_OFREE + 1), (n_it1 & 1) ^ 1, abort_flag, p.status);
           }
-          tc_commit(bar(B_SLOT_EMPTY + vslot % kSlots));
-          if (more) tc_commit(bar(B_SLOT_EMPTY + kslot % kSlots));
+          // ---- half A: O_A += P_A V, then S_A = Q_A K(j+1)^T
+          mbar_wait(bar(B_PREADY + 0), n_p0 & 1, abort_flag, p.status);
+          ++n_p0;
+          tc_fence_after();
+          trace_event(tc_cur, DYSPEC_TAG(0, 1, j));
+          issue_pv(0, vslot, j > 0);
+          if (!more) tc_commit(bar(B_ODONE + 0));
+          trace_event(tc_cur, DYSPEC_TAG(0, 5, j));
+          if (more) issue_qk(0, kslot);
+          trace_event(tc_cur, DYSPEC_TAG(0, 2, j));
+          // ---- half B
+          if (two) {
+            mbar_wait(bar(B_PREADY + 1), n_p1 & 1, abort_flag, p.status);
+            ++n_p1;
+            tc_fence_after();
+            trace_event(tc_cur, DYSPEC_TAG(0, 3, j));
+            issue_pv(1, vslot, j > 0);
+            if (!more) tc_commit(bar(B_ODONE + 1));
+            trace_event(tc_cur, DYSPEC_TAG(0, 6, j));
+            if (more) issue_qk(1, kslot);
+            trace_event(tc_cur, DYSPEC_TAG(0, 4, j));
+          }
+          tc_commit(bar(B_SLOT_EMPTY + vslot));
+          if (more) tc_commit(bar(B_SLOT_EMPTY + kslot));
+          if (j + 2 == T) tc_commit(bar(B_QFREE));
+          trace_event(tc_cur, DYSPEC_TAG(0, 7, j));
         }
-        tc_commit(bar(B_QFREE));
-        for (int h = 0; h < nh; ++h) ++n_items_h[h];
+        ++n_it0;
+        if (two) ++n_it1;
       }
     }
-  } else if (warp >= 4) {
+  }
+  } else {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");
     // ------------------------------------------------------------------ softmax + epilogue warps
     const int h = (warp - 4) >> 2;                       // query half
     const int r = ((warp & 3) << 5) + lane;              // row of the half == TMEM lane
     const uint32_t lane_sel = uint32_t((warp & 3) << 5) << 16;
     const uint32_t t_s = tmem_base + uint32_t(h) * 128u + lane_sel;
     const uint32_t t_o = tmem_base + 256u + uint32_t(h) * 128u + lane_sel;
+    TraceCursor tc_cur = trace_open(p, 1 + h, 3);
     uint32_t n_s = 0, n_o = 0;                           // S-ready / O-done phases seen by this half
     uint32_t sc = 0;                                     // ring position (to find V slots)
 
@@ -283,8 +351,10 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         // visibility of the 128 key columns of this tile for this row
         uint32_t vis[4];
         int own;
+        bool all_visible = false;                 // CTA-uniform: a full prefix tile needs no mask at all
         if (t < n_prefix_tiles) {
           const int valid = min(BN, rq.prefix_len - t * BN);
+          all_visible = valid == BN;
           own = min(BN, rq.prefix_len + rq.n_nodes - t * BN);
 #pragma unroll
           for (int q4 = 0; q4 < 4; ++q4) {
@@ -302,29 +372,40 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         mbar_wait(bar(B_SREADY + h), n_s & 1, abort_flag, p.status);
         ++n_s;
         tc_fence_after();
+        if (r == 0) trace_event(tc_cur, DYSPEC_TAG(1 + h, 1, j));
 
-        // pass 1: row maximum of the visible scaled scores
-        float mx = -INFINITY;
+#ifdef EXP_SKIP_SOFTMAX
+        if (j >= 0) { tc_fence_before(); mbar_arrive(bar(B_PREADY + h)); continue; }
+#endif
+        // the whole S row (128 fp32) in registers: four loads in flight, one wait
+        uint32_t sv[BN];
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          uint32_t v[32];
-          tmem_ld32(t_s + uint32_t(c) * 32u, v);
-          tmem_wait_ld();
-          const uint32_t bits = vis[c];
+        for (int c = 0; c < 4; ++c) tmem_ld32(t_s + uint32_t(c) * 32u, sv + 32 * c);
+        tmem_wait_ld();
+        if (r == 0) trace_event(tc_cur, DYSPEC_TAG(1 + h, 2, j));
+        if (!all_visible) {
 #pragma unroll
-          for (int i = 0; i < 32; ++i)
-            if ((bits >> i) & 1u) mx = fmaxf(mx, __uint_as_float(v[i]));
+          for (int i = 0; i < BN; ++i)
+            if (!((vis[i >> 5] >> (i & 31)) & 1u)) sv[i] = 0xff800000u;   // -inf
         }
-        mx *= p.scale_log2e;    // scale > 0, so the maximum commutes with the scaling
+        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+        for (int i = 0; i < BN; i += 4) {
+          mx4[0] = fmaxf(mx4[0], __uint_as_float(sv[i]));
+          mx4[1] = fmaxf(mx4[1], __uint_as_float(sv[i + 1]));
+          mx4[2] = fmaxf(mx4[2], __uint_as_float(sv[i + 2]));
+          mx4[3] = fmaxf(mx4[3], __uint_as_float(sv[i + 3]));
+        }
+        const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2e;   // scale > 0
         const float m_new = fmaxf(m_used, mx);
+        if (r == 0) trace_event(tc_cur, DYSPEC_TAG(1 + h, 3, j));
         if (j == 0) {
           m_used = m_new;
         } else if (__any_sync(0xffffffffu, m_new > m_used + kRescaleThreshold)) {
-          // rescale the running output of this warp's 32 rows: O *= 2^(m_used - m_new)
-          mbar_wait(bar(B_ODONE + h), (n_o + uint32_t(j) - 1u) & 1, abort_flag, p.status);
-          tc_fence_after();
+          // rescale the running output of this warp's 32 rows: O *= 2^(m_used - m_new).  The tensor pipe
+          // completes MMAs in issue order, so S(j) being ready already implies that PV(j-1) has finished.
           const float f = fast_exp2(m_used - (m_new == -INFINITY ? 0.f : m_new));
-#pragma unroll
+#pragma unroll 1
           for (int c = 0; c < D / 32; ++c) {
             uint32_t v[32];
             tmem_ld32(t_o + uint32_t(c) * 32u, v);
@@ -336,27 +417,25 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           l *= f;
           m_used = m_new;
         }
-        const float ref = m_used == -INFINITY ? 0.f : m_used;
+        const float neg_ref = m_used == -INFINITY ? 0.f : -m_used;
 
-        // pass 2: P = 2^(s - ref) as bf16 pairs, written over the first 64 S columns
-        float sum = 0.f;
+        // P = 2^(s * scale - ref) as bf16 pairs, written over the first 64 S columns (masked: 2^-inf = 0)
+        float sum4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
-          uint32_t v[32];
-          tmem_ld32(t_s + uint32_t(c) * 32u, v);
-          tmem_wait_ld();
-          const uint32_t bits = vis[c];
           uint32_t pk[16];
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
-            const float p0 = ((bits >> (2 * i)) & 1u) ? fast_exp2(fmaf(__uint_as_float(v[2 * i]), p.scale_log2e, -ref)) : 0.f;
-            const float p1 = ((bits >> (2 * i + 1)) & 1u) ? fast_exp2(fmaf(__uint_as_float(v[2 * i + 1]), p.scale_log2e, -ref)) : 0.f;
-            sum += p0 + p1;
+            const float p0 = fast_exp2(fmaf(__uint_as_float(sv[32 * c + 2 * i]), p.scale_log2e, neg_ref));
+            const float p1 = fast_exp2(fmaf(__uint_as_float(sv[32 * c + 2 * i + 1]), p.scale_log2e, neg_ref));
+            sum4[(2 * i) & 3] += p0;
+            sum4[(2 * i + 1) & 3] += p1;
             pk[i] = pack_bf16x2(p0, p1);
           }
           tmem_st16(t_s + uint32_t(c) * 16u, pk);
         }
-        l += sum;
+        l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+        if (r == 0) trace_event(tc_cur, DYSPEC_TAG(1 + h, 4, j));
 
         // V rows past the end of the request are not ours: zero them (their probabilities are 0, but
         // 0 * garbage could be NaN).  Half A's warps do it, before P is published to the MMA warp.
@@ -372,11 +451,13 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         tmem_wait_st();
         tc_fence_before();
         mbar_arrive(bar(B_PREADY + h));
+        if (r == 0) trace_event(tc_cur, DYSPEC_TAG(1 + h, 5, j));
       }
 
       // ---- epilogue: wait for the last PV, read O, normalise (or emit the partial)
-      mbar_wait(bar(B_ODONE + h), (n_o + uint32_t(T) - 1u) & 1, abort_flag, p.status);
-      n_o += uint32_t(T);
+      mbar_wait(bar(B_ODONE + h), n_o & 1, abort_flag, p.status);
+      ++n_o;
+      if (r == 0) trace_event(tc_cur, DYSPEC_TAG(1 + h, 6, 0));
       tc_fence_after();
       const int head = item.kv_head * g + (row & (g - 1));
       if (item.slot < 0) {
@@ -421,6 +502,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       }
       tc_fence_before();
       mbar_arrive(bar(B_OFREE + h));
+      if (r == 0) trace_event(tc_cur, DYSPEC_TAG(1 + h, 7, 0));
     }
   }
 

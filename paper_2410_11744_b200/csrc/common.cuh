@@ -66,6 +66,8 @@ struct AttnParams {
   int32_t words_per_row;           // W
   int32_t slot_floats;             // BM * (D + 2)
   float scale_log2e;               // scale * log2(e)
+  unsigned long long* trace;       // optional event trace (null in normal use): [0] = count, then entries
+  int32_t trace_capacity;
 };
 
 #ifdef __CUDACC__
@@ -114,11 +116,45 @@ constexpr uint64_t kWaitLimitNs = 1000ull * 1000ull * 1000ull;  // 1 s per wait,
 // Bounded mbarrier wait.  `abort_flag` lives in shared memory: once any wait of the CTA ran out,
 // later waits return at once.  Returns false when the wait did not complete.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
-  if (mbar_try_wait(bar, parity)) return true;
+  // fast path: try_wait itself blocks for a short hardware-defined time, so a few tries cover every
+  // ordinary wait without touching the (slow) global timer
+#pragma unroll 1
+  for (int i = 0; i < 16; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
   if (*abort_flag) return false;
   const uint64_t t0 = global_timer_ns();
   uint32_t spins = 0;
   while (!mbar_try_wait(bar, parity)) {
+    if ((++spins & 0xff) == 0) {
+      if (*abort_flag) return false;
+      if (global_timer_ns() - t0 > kWaitLimitNs) {
+        *abort_flag = 1;
+        if (status) atomicCAS(status, 0, DYSPEC_ERR_TIMEOUT);
+        return false;
+      }
+    }
+  }
+  return true;
+}
+
+// Bounded wait on a monotonically increasing shared-memory counter (release/acquire at CTA scope):
+// a much shorter hand-off than an mbarrier when the waiter only needs "at least `target` arrivals".
+__device__ __forceinline__ uint32_t ld_acquire_shared(uint32_t addr) {
+  uint32_t v;
+  asm volatile("ld.acquire.cta.shared::cta.u32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+  return v;
+}
+__device__ __forceinline__ void red_release_shared_add(uint32_t addr, uint32_t v) {
+  asm volatile("red.release.cta.shared::cta.add.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+}
+__device__ __forceinline__ bool counter_wait(uint32_t addr, uint32_t target, volatile int* abort_flag, int32_t* status) {
+#pragma unroll 1
+  for (int i = 0; i < 64; ++i)
+    if (int32_t(ld_acquire_shared(addr) - target) >= 0) return true;
+  if (*abort_flag) return false;
+  const uint64_t t0 = global_timer_ns();
+  uint32_t spins = 0;
+  while (int32_t(ld_acquire_shared(addr) - target) < 0) {
     if ((++spins & 0x3ff) == 0) {
       if (*abort_flag) return false;
       if (global_timer_ns() - t0 > kWaitLimitNs) {
@@ -140,6 +176,27 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
 }
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
+
+// Optional in-kernel event trace (CTA 0 only).  Each traced thread owns one region of the buffer
+// (region = role) and keeps its own cursor in a register, so an event costs one plain store:
+// entry = tag << 44 | low 44 bits of the SM clock.
+struct TraceCursor {
+  unsigned long long* at;
+  unsigned long long* end;
+};
+__device__ __forceinline__ TraceCursor trace_open(const AttnParams& p, int role, int n_roles) {
+  TraceCursor c{nullptr, nullptr};
+  if (p.trace != nullptr && blockIdx.x == 0) {
+    const int per = p.trace_capacity / n_roles;
+    c.at = p.trace + size_t(role) * per;
+    c.end = c.at + per;
+  }
+  return c;
+}
+__device__ __forceinline__ void trace_event(TraceCursor& c, uint32_t tag) {
+  if (c.at != nullptr && c.at < c.end)
+    *c.at++ = ((unsigned long long)tag << 44) | ((unsigned long long)clock64() & ((1ull << 44) - 1));
 }
 
 __device__ __forceinline__ float fast_exp2(float x) {
