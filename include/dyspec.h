@@ -115,9 +115,10 @@ int dyspec_schedule_dry_run(int n_q_heads, int n_kv_heads, int head_dim, int n_r
                             const int32_t* n_nodes, int words_per_row, int32_t* items_out, int max_items,
                             int32_t* cta_begin_out, int max_ctas, int64_t* info_out);
 
-/* Testing knobs, read when a plan is created: force the regime (-1 = automatic) and the number of
- * CTAs the scheduler balances over (<= 0 = automatic). */
-int dyspec_set_tuning(int force_regime, int force_ctas);
+/* Testing knobs, read when a plan is created: force the regime (-1 = automatic), the number of
+ * CTAs the scheduler balances over (<= 0 = automatic), and whether split-KV partials are merged by the
+ * last work item of a group to finish (1) or by a separate combine kernel (0, the default). */
+int dyspec_set_tuning(int force_regime, int force_ctas, int fuse_combine);
 
 /* Developer aid: event trace of the attention kernels.  trace_buffer is a dev uint64 array of
  * capacity_entries entries that the caller zeroes; while set, CTA 0 of every tensor-core attention

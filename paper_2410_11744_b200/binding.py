@@ -29,7 +29,7 @@ SIGNATURES = {
     "dyspec_error_string": (_c.c_char_p, [_i32]),
     "dyspec_version": (_i32, []),
     "dyspec_words_per_row": (_i32, [_i32]),
-    "dyspec_set_tuning": (_i32, [_i32, _i32]),
+    "dyspec_set_tuning": (_i32, [_i32, _i32, _i32]),
     "dyspec_set_trace": (_i32, [_vp, _i32]),
     "dyspec_build_tree_mask": (_i32, [_vp, _i32, _vp, _vp, _i32, _vp, _vp]),
     "dyspec_plan_create": (_i32, [_c.POINTER(_vp), _i32, _i32, _i32, _i32, _vp, _vp, _vp, _i64, _i32, _f32]),
@@ -89,8 +89,8 @@ def dyspec_words_per_row(max_nodes: int) -> int:
     return lib.dyspec_words_per_row(max_nodes)
 
 
-def dyspec_set_tuning(force_regime: int = -1, force_ctas: int = 0) -> None:
-    _check(lib.dyspec_set_tuning(force_regime, force_ctas), "dyspec_set_tuning")
+def dyspec_set_tuning(force_regime: int = -1, force_ctas: int = 0, fuse_combine: int = 0) -> None:
+    _check(lib.dyspec_set_tuning(force_regime, force_ctas, fuse_combine), "dyspec_set_tuning")
 
 
 def dyspec_set_trace(trace_buffer=None, capacity_entries: int = 0) -> None:

@@ -28,6 +28,7 @@ namespace {
 
 int g_force_regime = -1;
 int g_force_ctas = 0;
+int g_fuse_combine = 0;
 unsigned long long* g_trace = nullptr;   // device buffer for the optional kernel event trace
 int g_trace_capacity = 0;
 
@@ -75,7 +76,10 @@ struct dyspec_plan {
   int max_nodes = 0;
   int regime = 0, bm = 64, bn = 64;
   std::vector<ReqInfo> reqs;
-  std::vector<WorkItem> items;
+  std::vector<WorkItem> items;          // compact list, CTA by CTA
+  std::vector<WorkItem> items_strided;  // device layout: CTA c's items at [c * items_stride, ...)
+  int items_stride = 1;
+  int fuse_combine = 1;
   std::vector<int32_t> cta_begin;
   std::vector<GroupInfo> split_groups;
   int n_ctas = 0, n_slots = 0, max_splits = 1;
@@ -124,9 +128,12 @@ void schedule(dyspec_plan& pl) {
   pl.split_groups.clear();
   pl.n_slots = 0;
   pl.max_splits = 1;
+  pl.items_strided.clear();
+  pl.items_stride = 1;
+  pl.fuse_combine = g_fuse_combine;
   if (groups.empty()) { pl.n_ctas = 0; pl.cta_begin.push_back(0); return; }
 
-  const int ctas_per_sm = pl.regime == 0 ? 2 : 1;
+  const int ctas_per_sm = 1;   // one wave: every CTA is resident from the start and owns its SM's load queue
   int max_ctas = g_force_ctas > 0 ? g_force_ctas : kNumSMs * ctas_per_sm;
   const int item_cost = 1;                               // fixed per-item overhead, in key tiles
   const int min_tiles = pl.regime == 0 ? 2 : 2;          // smallest piece worth a split
@@ -160,6 +167,9 @@ void schedule(dyspec_plan& pl) {
       const int rem = gr.tiles - begin - take;
       if (rem > 0 && rem < min_tiles) take = gr.tiles - begin;
       WorkItem it{};
+      const ReqInfo& rq = pl.reqs[size_t(gr.req)];
+      it.kv_row0 = rq.kv_row0; it.prefix_len = rq.prefix_len; it.n_nodes = rq.n_nodes; it.node0 = rq.node0;
+      it.slot0 = -1; it.n_in_cta = 0;
       it.req = gr.req; it.kv_head = gr.kvh; it.row0 = gr.row0;
       it.tile_begin = begin; it.tile_end = begin + take;
       it.slot = -1; it.group = int(gi); it.n_splits = 1;
@@ -174,6 +184,7 @@ void schedule(dyspec_plan& pl) {
       info.slot0 = pl.n_slots; info.n_splits = n_splits;
       for (int s = 0; s < n_splits; ++s) {
         pl.items[first_item + s].slot = pl.n_slots + s;
+        pl.items[first_item + s].slot0 = pl.n_slots;
         pl.items[first_item + s].n_splits = n_splits;
         pl.items[first_item + s].group = int(pl.split_groups.size());
       }
@@ -187,12 +198,21 @@ void schedule(dyspec_plan& pl) {
   if (pl.n_ctas <= max_ctas) break;
   target += std::max<int64_t>(1, target / 64);
   }
+  // device layout: fixed stride per CTA, count in the CTA's first item
+  pl.items_stride = 1;
+  for (int c = 0; c < pl.n_ctas; ++c) pl.items_stride = std::max(pl.items_stride, pl.cta_begin[size_t(c) + 1] - pl.cta_begin[size_t(c)]);
+  pl.items_strided.assign(size_t(pl.n_ctas) * size_t(pl.items_stride), WorkItem{});
+  for (int c = 0; c < pl.n_ctas; ++c) {
+    const int b = pl.cta_begin[size_t(c)], e = pl.cta_begin[size_t(c) + 1];
+    for (int k = b; k < e; ++k) pl.items_strided[size_t(c) * size_t(pl.items_stride) + size_t(k - b)] = pl.items[size_t(k)];
+    pl.items_strided[size_t(c) * size_t(pl.items_stride)].n_in_cta = e - b;
+  }
 }
 
 int upload(dyspec_plan& pl) {
   auto pad = [](size_t x) { return (x + 255) & ~size_t(255); };
   const size_t b_reqs = pad(std::max<size_t>(1, pl.reqs.size()) * sizeof(ReqInfo));
-  const size_t b_items = pad(std::max<size_t>(1, pl.items.size()) * sizeof(WorkItem));
+  const size_t b_items = pad(std::max<size_t>(1, pl.items_strided.size()) * sizeof(WorkItem));
   const size_t b_cta = pad(pl.cta_begin.size() * sizeof(int32_t));
   const size_t b_groups = pad(std::max<size_t>(1, pl.split_groups.size()) * sizeof(GroupInfo));
   const size_t b_counters = pad(std::max<size_t>(1, pl.split_groups.size()) * sizeof(int32_t));
@@ -201,7 +221,7 @@ int upload(dyspec_plan& pl) {
   size_t off = 0;
   if (!pl.reqs.empty()) memcpy(host.data() + off, pl.reqs.data(), pl.reqs.size() * sizeof(ReqInfo));
   const size_t o_reqs = off; off += b_reqs;
-  if (!pl.items.empty()) memcpy(host.data() + off, pl.items.data(), pl.items.size() * sizeof(WorkItem));
+  if (!pl.items_strided.empty()) memcpy(host.data() + off, pl.items_strided.data(), pl.items_strided.size() * sizeof(WorkItem));
   const size_t o_items = off; off += b_items;
   memcpy(host.data() + off, pl.cta_begin.data(), pl.cta_begin.size() * sizeof(int32_t));
   const size_t o_cta = off; off += b_cta;
@@ -244,10 +264,11 @@ int dyspec_words_per_row(int max_nodes) {
   return 4 * ((max_nodes + 127) / 128);
 }
 
-int dyspec_set_tuning(int force_regime, int force_ctas) {
-  if (force_regime < -1 || force_regime > 1) return DYSPEC_ERR_INVALID_ARG;
+int dyspec_set_tuning(int force_regime, int force_ctas, int fuse_combine) {
+  if (force_regime < -1 || force_regime > 1 || fuse_combine < 0 || fuse_combine > 1) return DYSPEC_ERR_INVALID_ARG;
   g_force_regime = force_regime;
   g_force_ctas = force_ctas;
+  g_fuse_combine = fuse_combine;
   return DYSPEC_OK;
 }
 
@@ -349,7 +370,11 @@ int dyspec_schedule_dry_run(int n_q_heads, int n_kv_heads, int head_dim, int n_r
   if (rc != DYSPEC_OK) return rc;
   const int n_items = int(pl->items.size());
   if (items_out)
-    for (int i = 0; i < n_items && i < max_items; ++i) memcpy(items_out + 8 * i, &pl->items[size_t(i)], sizeof(WorkItem));
+    for (int i = 0; i < n_items && i < max_items; ++i) {
+      const WorkItem& it = pl->items[size_t(i)];
+      const int32_t rec[8] = {it.req, it.kv_head, it.row0, it.tile_begin, it.tile_end, it.slot, it.group, it.n_splits};
+      memcpy(items_out + 8 * i, rec, sizeof(rec));
+    }
   if (cta_begin_out)
     for (int c = 0; c <= pl->n_ctas && c < max_ctas; ++c) cta_begin_out[c] = pl->cta_begin[size_t(c)];
   if (info_out) {
@@ -422,13 +447,15 @@ int dyspec_tree_attention_ragged(const dyspec_plan_t* plan, const void* q, const
   p.n_q_heads = plan->hq; p.n_kv_heads = plan->hkv; p.group_size = plan->g; p.log2_g = plan->log2g;
   p.words_per_row = plan->W; p.slot_floats = bm * (plan->d + 2);
   p.scale_log2e = plan->scale * kLog2e;
+  p.items_stride = plan->items_stride;
+  p.fuse_combine = plan->fuse_combine && plan->regime == 0;
   p.trace = g_trace; p.trace_capacity = g_trace_capacity;
 
   cudaError_t e;
   if (plan->regime == 0) e = launch_attn_mma(plan->d, plan->n_ctas, mq, mk, mv, p, st);
   else e = launch_attn_tc(plan->d, plan->n_ctas, mq, mk, mv, p, st);
   if (e != cudaSuccess) return DYSPEC_ERR_CUDA;
-  e = launch_combine(plan->d, bm, int(plan->split_groups.size()), p, st);
+  if (!p.fuse_combine) e = launch_combine(plan->d, bm, int(plan->split_groups.size()), p, st);
   return e == cudaSuccess ? DYSPEC_OK : DYSPEC_ERR_CUDA;
 }
 
@@ -532,7 +559,7 @@ extern "C" int dyspec_tree_attention_static(const void* q, const void* k_cache, 
   auto pad = [](size_t x) { return (x + 255) & ~size_t(255); };
   const size_t o_reqs = 0;
   const size_t o_items = o_reqs + pad(pl->reqs.size() * sizeof(ReqInfo));
-  const size_t o_cta = o_items + pad(pl->items.size() * sizeof(WorkItem));
+  const size_t o_cta = o_items + pad(pl->items_strided.size() * sizeof(WorkItem));
   const size_t o_groups = o_cta + pad(pl->cta_begin.size() * sizeof(int32_t));
   const size_t o_counters = o_groups + pad(std::max<size_t>(1, pl->split_groups.size()) * sizeof(GroupInfo));
   const size_t o_partial = o_counters + pad(std::max<size_t>(1, pl->split_groups.size()) * sizeof(int32_t));
@@ -547,7 +574,7 @@ extern "C" int dyspec_tree_attention_static(const void* q, const void* k_cache, 
   // The array keeps whatever the previous call left: rewrite the tables, clear the counters.
   std::vector<uint8_t> host(o_partial, 0);
   memcpy(host.data() + o_reqs, pl->reqs.data(), pl->reqs.size() * sizeof(ReqInfo));
-  memcpy(host.data() + o_items, pl->items.data(), pl->items.size() * sizeof(WorkItem));
+  memcpy(host.data() + o_items, pl->items_strided.data(), pl->items_strided.size() * sizeof(WorkItem));
   memcpy(host.data() + o_cta, pl->cta_begin.data(), pl->cta_begin.size() * sizeof(int32_t));
   if (!pl->split_groups.empty())
     memcpy(host.data() + o_groups, pl->split_groups.data(), pl->split_groups.size() * sizeof(GroupInfo));
@@ -573,11 +600,13 @@ extern "C" int dyspec_tree_attention_static(const void* q, const void* k_cache, 
   p.n_q_heads = pl->hq; p.n_kv_heads = pl->hkv; p.group_size = pl->g; p.log2_g = pl->log2g;
   p.words_per_row = pl->W; p.slot_floats = bm * (pl->d + 2);
   p.scale_log2e = pl->scale * kLog2e;
+  p.items_stride = pl->items_stride;
+  p.fuse_combine = pl->fuse_combine && pl->regime == 0;
 
   cudaError_t e;
   if (pl->regime == 0) e = launch_attn_mma(pl->d, pl->n_ctas, mq, mk, mv, p, st);
   else e = launch_attn_tc(pl->d, pl->n_ctas, mq, mk, mv, p, st);
   if (e != cudaSuccess) return DYSPEC_ERR_CUDA;
-  e = launch_combine(pl->d, bm, int(pl->split_groups.size()), p, st);
+  if (!p.fuse_combine) e = launch_combine(pl->d, bm, int(pl->split_groups.size()), p, st);
   return e == cudaSuccess ? DYSPEC_OK : DYSPEC_ERR_CUDA;
 }

@@ -1,7 +1,7 @@
 // Tree-verify attention, warp-level tile regime (Sec. 2 "Tree Attention"; App. C: prefix keys are in the mask).
 //
 // Used when the packed query tile (tree nodes x GQA group) is small, so the work is bound by
-// streaming K/V from HBM rather than by the tensor pipe.  One CTA = 4 compute warps (16 query rows
+// streaming K/V from HBM rather than by the tensor pipe.  One CTA per SM = 4 compute warps (16 query rows
 // each, BM = 64) + 1 producer warp.  The producer streams 64-key K and V tiles through TMA into a
 // 128-byte-swizzled shared-memory ring guarded by mbarriers; compute warps run QK^T and PV with
 // mma.sync.m16n8k16 (bf16 in, fp32 accumulate), an fp32 online softmax in the exp2 domain, and apply
@@ -20,7 +20,7 @@ constexpr int kThreads = (kComputeWarps + 1) * 32;
 
 template <int D>
 struct SmemLayout {
-  static constexpr int kStages = (D == 128) ? 3 : 4;
+  static constexpr int kStages = (D == 128) ? 6 : 8;     // one CTA per SM: keep ~190 KB of K/V loads in flight
   static constexpr int kHalves = D / 64;                 // 64-element (128-byte) column panels per row
   static constexpr int kPanelBytes = BN * 128;           // one panel of a K or V tile: 64 rows x 128 B
   static constexpr int kTileBytes = kPanelBytes * kHalves;
@@ -54,7 +54,7 @@ __device__ __forceinline__ uint32_t swz(int row, int chunk, int panel_bytes) {
 }  // namespace
 
 template <int D>
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __launch_bounds__(kThreads, 1)
 tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                      const __grid_constant__ CUtensorMap map_v, const AttnParams p) {
   using L = SmemLayout<D>;
@@ -71,9 +71,16 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   const uint32_t bar_full = s_bar, bar_empty = s_bar + 8 * kStages;
   const uint32_t bar_qfull = s_bar + 16 * kStages, bar_qempty = bar_qfull + 8;
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::kBarOffset + 16 * kStages + 16);
+  volatile int* last_flag = reinterpret_cast<volatile int*>(smem + L::kBarOffset + 16 * kStages + 20);
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
+  // trace: the last 2048 entries of the buffer hold 8 wall-clock stamps for each of the first 256 CTAs
+  auto stamp = [&](int k) {
+    if (p.trace != nullptr && blockIdx.x < 256 && p.trace_capacity > 4096)
+      p.trace[p.trace_capacity - 2048 + 8 * blockIdx.x + k] = global_timer_ns();
+  };
+  if (threadIdx.x == 0) stamp(0);
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
@@ -87,10 +94,12 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   }
   __syncthreads();
 
-  const int item_begin = p.cta_item_begin[blockIdx.x];
-  const int item_end = p.cta_item_begin[blockIdx.x + 1];
+  const WorkItem* my_items = p.items + size_t(blockIdx.x) * p.items_stride;
+  const int item_begin = 0;
+  const int item_end = my_items[0].n_in_cta;
   const int g = p.group_size;
 
+  trigger_dependents();     // the combine kernel may be scheduled; it waits for this grid before reading partials
   if (warp == kComputeWarps) {
     // ------------------------------------------------------------------ producer warp (one lane issues)
     if (lane == 0) {
@@ -100,8 +109,8 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       uint32_t it = 0;       // running key-tile counter of this CTA (ring position)
       uint32_t qit = 0;      // running item counter (Q buffer phase)
       for (int w = item_begin; w < item_end; ++w, ++qit) {
-        const WorkItem item = p.items[w];
-        const ReqInfo rq = p.reqs[item.req];
+        const WorkItem item = my_items[w];
+        const WorkItem& rq = item;
         // Q tile: box (64 cols, g heads, BM/g nodes) per panel; rows land node-major, head-minor.
         mbar_wait(bar_qempty, (qit & 1) ^ 1, abort_flag, p.status);
         mbar_expect_tx(bar_qfull, L::kQBytes);
@@ -128,14 +137,18 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   }
 
   // -------------------------------------------------------------------- compute warps
+  // Everything read so far (work items, Q/K/V through TMA) is input that no kernel of this stream
+  // writes.  The mask, the partials and the output are: wait for the preceding kernels here, while
+  // the producer warp keeps streaming K/V.
+  grid_dependency_wait();
   const int gid = lane >> 2;      // row within an 8-row slab
   const int tig = lane & 3;       // column pair within an 8-column tile
   const int wrow = warp * 16;
   uint32_t it = 0, qit = 0;
 
   for (int w = item_begin; w < item_end; ++w, ++qit) {
-    const WorkItem item = p.items[w];
-    const ReqInfo rq = p.reqs[item.req];
+    const WorkItem item = my_items[w];
+    const WorkItem& rq = item;
     const int n_prefix_tiles = (rq.prefix_len + BN - 1) / BN;
     const int n_rows = rq.n_nodes * g;                     // packed rows of this (request, kv head)
     const int row_lo = item.row0 + wrow + gid;             // the two packed rows this thread owns
@@ -145,7 +158,9 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
 
     // Q fragments, kept in registers for the whole item.
     uint32_t qf[KS][4];
+    if (threadIdx.x == 0 && w == item_begin) stamp(1);
     mbar_wait(bar_qfull, qit & 1, abort_flag, p.status);
+    if (threadIdx.x == 0 && w == item_begin) stamp(2);
 #pragma unroll
     for (int ks = 0; ks < KS; ++ks) {
       const int row = wrow + (lane & 15);
@@ -166,6 +181,8 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       const uint32_t s_k = s_kv + stage * L::kStageBytes;
       const uint32_t s_v = s_k + L::kTileBytes;
       mbar_wait(bar_full + 8 * stage, ph, abort_flag, p.status);
+      if (threadIdx.x == 0 && w == item_begin && t == item.tile_begin) stamp(3);
+      if (threadIdx.x == 0 && w == item_begin && t == item.tile_end - 1) stamp(4);
 
       // ---- S = Q K^T (16 x 64 per warp)
       float s[BN / 8][4];
@@ -277,6 +294,7 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     }
 
     // ---- epilogue
+    if (threadIdx.x == 0 && w == item_begin) stamp(5);
     l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1);
     l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
     l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1);
@@ -306,8 +324,61 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         if (ok_lo) { slot[BM * D + r_lo] = m_lo; slot[BM * D + BM + r_lo] = l_lo; }
         if (ok_hi) { slot[BM * D + r_hi] = m_hi; slot[BM * D + BM + r_hi] = l_hi; }
       }
+      if (p.fuse_combine) {
+        // Split-KV combine by the last arriver: publish the partial, count this item in, and if every
+        // other item of the group has already been counted, merge all of the group's partials here.
+        __threadfence();
+        asm volatile("bar.sync 1, %0;" ::"n"(kComputeWarps * 32) : "memory");
+        if (threadIdx.x == 0) *last_flag = atomicAdd(p.counters + item.group, 1) == item.n_splits - 1 ? 1 : 0;
+        asm volatile("bar.sync 1, %0;" ::"n"(kComputeWarps * 32) : "memory");
+        if (*last_flag) {
+          __threadfence();
+          if (threadIdx.x == 0) p.counters[item.group] = 0;      // leave the counter ready for the next call
+          const float* base = p.partial + size_t(item.slot0) * p.slot_floats;
+          constexpr int V = D / 32;                              // floats per lane
+          for (int rr = 0; rr < 16; ++rr) {
+            const int r = wrow + rr;
+            const int row = item.row0 + r;
+            if (row >= n_rows) break;
+            float m = -INFINITY;
+            for (int sidx = 0; sidx < item.n_splits; ++sidx)
+              m = fmaxf(m, __ldcg(base + size_t(sidx) * p.slot_floats + BM * D + r));
+            const float ref = m == -INFINITY ? 0.f : m;
+            float acc[V];
+#pragma unroll
+            for (int k = 0; k < V; ++k) acc[k] = 0.f;
+            float lsum = 0.f;
+            for (int sidx = 0; sidx < item.n_splits; ++sidx) {
+              const float* sl = base + size_t(sidx) * p.slot_floats;
+              const float wgt = fast_exp2(__ldcg(sl + BM * D + r) - ref);
+              lsum += wgt * __ldcg(sl + BM * D + BM + r);
+              if constexpr (V == 4) {
+                const float4 v = __ldcg(reinterpret_cast<const float4*>(sl + r * D + lane * 4));
+                acc[0] += wgt * v.x; acc[1] += wgt * v.y; acc[2] += wgt * v.z; acc[3] += wgt * v.w;
+              } else {
+                const float2 v = __ldcg(reinterpret_cast<const float2*>(sl + r * D + lane * 2));
+                acc[0] += wgt * v.x; acc[1] += wgt * v.y;
+              }
+            }
+            const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
+            const int node = row >> p.log2_g;
+            const int head = item.kv_head * g + (row & (g - 1));
+            __nv_bfloat16* out = p.out + (size_t(rq.node0 + node) * p.n_q_heads + head) * D;
+            if constexpr (V == 4) {
+              uint2 o2;
+              o2.x = pack_bf16x2(acc[0] * inv, acc[1] * inv);
+              o2.y = pack_bf16x2(acc[2] * inv, acc[3] * inv);
+              *reinterpret_cast<uint2*>(out + lane * 4) = o2;
+            } else {
+              *reinterpret_cast<uint32_t*>(out + lane * 2) = pack_bf16x2(acc[0] * inv, acc[1] * inv);
+            }
+          }
+        }
+      }
     }
+    if (threadIdx.x == 0 && w == item_begin) stamp(6);
   }
+  if (threadIdx.x == 0) stamp(7);
 }
 
 size_t attn_mma_smem_bytes(int head_dim) {
@@ -319,22 +390,34 @@ cudaError_t launch_attn_mma(int head_dim, int n_ctas, const CUtensorMap& mq, con
                             const AttnParams& p, cudaStream_t stream) {
   const size_t smem = attn_mma_smem_bytes(head_dim);
   static bool attr_set[2] = {false, false};
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(unsigned(n_ctas));
+  cfg.blockDim = dim3(unsigned(kThreads));
+  cfg.stream = stream;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaError_t e = cudaSuccess;
   if (head_dim == 128) {
     if (!attr_set[0]) {
       cudaError_t e = cudaFuncSetAttribute(tree_attn_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
       if (e != cudaSuccess) return e;
       attr_set[0] = true;
     }
-    tree_attn_mma_kernel<128><<<n_ctas, kThreads, smem, stream>>>(mq, mk, mv, p);
+    cfg.dynamicSmemBytes = smem;
+    e = cudaLaunchKernelEx(&cfg, tree_attn_mma_kernel<128>, mq, mk, mv, p);
   } else {
     if (!attr_set[1]) {
       cudaError_t e = cudaFuncSetAttribute(tree_attn_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
       if (e != cudaSuccess) return e;
       attr_set[1] = true;
     }
-    tree_attn_mma_kernel<64><<<n_ctas, kThreads, smem, stream>>>(mq, mk, mv, p);
+    cfg.dynamicSmemBytes = smem;
+    e = cudaLaunchKernelEx(&cfg, tree_attn_mma_kernel<64>, mq, mk, mv, p);
   }
-  return cudaGetLastError();
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace dyspec

@@ -178,11 +178,13 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   tc_fence_after();
   const uint32_t tmem_base = *tmem_holder;
 
-  const int item_begin = p.cta_item_begin[blockIdx.x];
-  const int item_end = p.cta_item_begin[blockIdx.x + 1];
+  const WorkItem* my_items = p.items + size_t(blockIdx.x) * p.items_stride;
+  const int item_begin = 0;
+  const int item_end = my_items[0].n_in_cta;
   const int g = p.group_size;
 
   // Register budget: the softmax threads hold a whole S row; the control warps need few registers.
+  trigger_dependents();     // the combine kernel may be scheduled; it waits for this grid before reading partials
   if (warp < 4) {
   asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
   if (warp == 0) {
@@ -193,8 +195,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       prefetch_tensormap(&map_v);
       uint32_t sc = 0, qit = 0;
       for (int w = item_begin; w < item_end; ++w, ++qit) {
-        const WorkItem item = p.items[w];
-        const ReqInfo rq = p.reqs[item.req];
+        const WorkItem item = my_items[w];
+        const WorkItem& rq = item;
         const int nh = (rq.n_nodes * g - item.row0 > BMH) ? 2 : 1;
         mbar_wait(bar(B_QFREE), (qit & 1) ^ 1, abort_flag, p.status);
         mbar_expect_tx(bar(B_QFULL), uint32_t(nh) * L::kTileBytes);
@@ -257,8 +259,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       uint32_t n_p0 = 0, n_p1 = 0;          // P-ready phases consumed per half
       uint32_t n_it0 = 0, n_it1 = 0;        // items seen per half (O-free phase)
       for (int w = item_begin; w < item_end; ++w, ++qit) {
-        const WorkItem item = p.items[w];
-        const ReqInfo rq = p.reqs[item.req];
+        const WorkItem item = my_items[w];
+        const WorkItem& rq = item;
         const bool two = rq.n_nodes * g - item.row0 > BMH;        // both query halves live
         const int T = item.tile_end - item.tile_begin;
         mbar_wait(bar(B_QFULL), qit & 1, abort_flag, p.status);
@@ -321,6 +323,9 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   } else {
     asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");
     // ------------------------------------------------------------------ softmax + epilogue warps
+    // Q/K/V and the work items are inputs no kernel of this stream writes; the mask, the partials
+    // and the output are: wait for the preceding kernels before touching those.
+    grid_dependency_wait();
     const int h = (warp - 4) >> 2;                       // query half
     const int r = ((warp & 3) << 5) + lane;              // row of the half == TMEM lane
     const uint32_t lane_sel = uint32_t((warp & 3) << 5) << 16;
@@ -331,8 +336,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     uint32_t sc = 0;                                     // ring position (to find V slots)
 
     for (int w = item_begin; w < item_end; ++w) {
-      const WorkItem item = p.items[w];
-      const ReqInfo rq = p.reqs[item.req];
+      const WorkItem item = my_items[w];
+      const WorkItem& rq = item;
       const int n_rows = rq.n_nodes * g;
       const int nh = (n_rows - item.row0 > BMH) ? 2 : 1;
       const int T = item.tile_end - item.tile_begin;
@@ -517,6 +522,16 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
 cudaError_t launch_attn_tc(int head_dim, int n_ctas, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                            const AttnParams& p, cudaStream_t stream) {
   static bool attr_set[2] = {false, false};
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(unsigned(n_ctas));
+  cfg.blockDim = dim3(unsigned(kThreads));
+  cfg.stream = stream;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaError_t le = cudaSuccess;
   if (head_dim == 128) {
     const size_t smem = TcLayout<128>::kTotal + 1024;
     if (!attr_set[0]) {
@@ -524,7 +539,8 @@ cudaError_t launch_attn_tc(int head_dim, int n_ctas, const CUtensorMap& mq, cons
       if (e != cudaSuccess) return e;
       attr_set[0] = true;
     }
-    tree_attn_tc_kernel<128><<<n_ctas, kThreads, smem, stream>>>(mq, mk, mv, p);
+    cfg.dynamicSmemBytes = smem;
+    le = cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<128>, mq, mk, mv, p);
   } else {
     // padded past half of an SM's shared memory: one CTA per SM, since each CTA takes all 512 TMEM columns
     const size_t smem = 120 * 1024;
@@ -534,9 +550,10 @@ cudaError_t launch_attn_tc(int head_dim, int n_ctas, const CUtensorMap& mq, cons
       if (e != cudaSuccess) return e;
       attr_set[1] = true;
     }
-    tree_attn_tc_kernel<64><<<n_ctas, kThreads, smem, stream>>>(mq, mk, mv, p);
+    cfg.dynamicSmemBytes = smem;
+    le = cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<64>, mq, mk, mv, p);
   }
-  return cudaGetLastError();
+  return le != cudaSuccess ? le : cudaGetLastError();
 }
 
 }  // namespace dyspec

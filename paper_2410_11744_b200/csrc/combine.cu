@@ -10,6 +10,7 @@ namespace dyspec {
 template <int D>
 __global__ void __launch_bounds__(256)
 combine_kernel(const AttnParams p, int bm) {
+  grid_dependency_wait();   // launched early (programmatic dependent launch): the partials must be complete
   const int rows_per_block = 8;
   const int blocks_per_group = bm / rows_per_block;
   const GroupInfo gi = p.groups[blockIdx.x / blocks_per_group];
@@ -58,9 +59,19 @@ combine_kernel(const AttnParams p, int bm) {
 cudaError_t launch_combine(int head_dim, int bm, int n_split_groups, const AttnParams& p, cudaStream_t stream) {
   if (n_split_groups <= 0) return cudaSuccess;
   const int blocks = n_split_groups * (bm / 8);
-  if (head_dim == 128) combine_kernel<128><<<blocks, 256, 0, stream>>>(p, bm);
-  else combine_kernel<64><<<blocks, 256, 0, stream>>>(p, bm);
-  return cudaGetLastError();
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(unsigned(blocks));
+  cfg.blockDim = dim3(256u);
+  cfg.stream = stream;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaError_t e;
+  if (head_dim == 128) e = cudaLaunchKernelEx(&cfg, combine_kernel<128>, p, bm);
+  else e = cudaLaunchKernelEx(&cfg, combine_kernel<64>, p, bm);
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace dyspec

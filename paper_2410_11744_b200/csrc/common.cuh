@@ -26,17 +26,27 @@ struct ReqInfo {
 // contiguous range of that group's key tiles.  Packed row p of a (request, kv head) pair is
 // node p / g, query head kv_head * g + p % g.  Key tiles of a group: first the prefix tiles
 // (tile t covers prefix keys [t*BN, min(L, (t+1)*BN))), then the tree tiles (tile u covers tree
-// columns [u*BN, (u+1)*BN)).
+// columns [u*BN, (u+1)*BN)).  The request's shape is repeated inside the item and CTA c's items sit
+// at a fixed stride (items[c * stride + k], k < items[c * stride].n_in_cta), so a CTA reaches its
+// work with one dependent global load instead of three.
 struct WorkItem {
-  int32_t req;
+  int64_t kv_row0;     // row of the request's token 0 in k_cache / v_cache
+  int32_t prefix_len;  // L_r
+  int32_t n_nodes;     // n_r
+  int32_t node0;       // first query / output / mask row of the request
   int32_t kv_head;
   int32_t row0;        // first packed row of the query tile (multiple of BM)
   int32_t tile_begin;  // key-tile range [tile_begin, tile_end) of the group's tile list
   int32_t tile_end;
   int32_t slot;        // index of the fp32 partial slot to write, or -1: write the final bf16 rows
-  int32_t group;       // query-tile group id (arrival counter index)
+  int32_t group;       // split-group id (arrival counter index) when slot >= 0
   int32_t n_splits;    // number of items the group was cut into
+  int32_t slot0;       // first partial slot of the group (slots slot0 .. slot0 + n_splits - 1)
+  int32_t n_in_cta;    // in the first item of a CTA: how many items the CTA owns
+  int32_t req;         // request index
+  int32_t pad;
 };
+static_assert(sizeof(WorkItem) == 64, "WorkItem is one 64-byte record");
 
 // A split query-tile group, for the combine step.
 struct GroupInfo {
@@ -51,8 +61,8 @@ struct GroupInfo {
 // Parameters common to the attention kernels.
 struct AttnParams {
   const ReqInfo* reqs;
-  const WorkItem* items;
-  const int32_t* cta_item_begin;   // [n_ctas + 1]
+  const WorkItem* items;           // [n_ctas * items_stride]
+  const int32_t* cta_item_begin;   // [n_ctas + 1] (host-side view of the same assignment; unused by the kernels)
   const GroupInfo* groups;         // split groups only
   const uint32_t* bits;            // ancestor bitmasks [sum n][W]
   __nv_bfloat16* out;              // [sum n][H_q][D]
@@ -66,6 +76,8 @@ struct AttnParams {
   int32_t words_per_row;           // W
   int32_t slot_floats;             // BM * (D + 2)
   float scale_log2e;               // scale * log2(e)
+  int32_t items_stride;            // items per CTA slot in `items`
+  int32_t fuse_combine;            // 1: the last item of a split group to finish merges the partials itself
   unsigned long long* trace;       // optional event trace (null in normal use): [0] = count, then entries
   int32_t trace_capacity;
 };
@@ -167,6 +179,13 @@ __device__ __forceinline__ bool counter_wait(uint32_t addr, uint32_t target, vol
   return true;
 }
 
+// Programmatic dependent launch: a kernel launched with the programmatic-serialization attribute may
+// start while its predecessor in the stream is still running; it must call grid_dependency_wait()
+// before it reads anything the predecessor writes or writes anything the predecessor (or earlier
+// kernels) may still read.  The predecessor lets dependents start early with trigger_dependents().
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void trigger_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // TMA: 3-D tiled load global -> shared, completion on an mbarrier (no multicast anywhere).
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
   asm volatile(
@@ -188,7 +207,7 @@ struct TraceCursor {
 __device__ __forceinline__ TraceCursor trace_open(const AttnParams& p, int role, int n_roles) {
   TraceCursor c{nullptr, nullptr};
   if (p.trace != nullptr && blockIdx.x == 0) {
-    const int per = p.trace_capacity / n_roles;
+    const int per = (p.trace_capacity > 4096 ? p.trace_capacity - 2048 : p.trace_capacity) / n_roles;
     c.at = p.trace + size_t(role) * per;
     c.end = c.at + per;
   }

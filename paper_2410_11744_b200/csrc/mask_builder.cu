@@ -15,6 +15,7 @@ __global__ void __launch_bounds__(1024, 1)
 build_tree_mask_kernel(const int32_t* __restrict__ parents, const ReqInfo* __restrict__ reqs, int single_n,
                        uint32_t* __restrict__ bits, int32_t* __restrict__ depths, int W, int32_t* status) {
   extern __shared__ __align__(16) uint8_t mask_smem[];
+  trigger_dependents();   // the attention kernel may start streaming K/V now; it waits for us before it reads the mask
   int node0 = 0, n = single_n;
   if (reqs != nullptr) {
     node0 = reqs[blockIdx.x].node0;

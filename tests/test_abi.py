@@ -83,5 +83,5 @@ def test_argument_errors_are_reported_before_any_launch(binding):
     assert create(0, 4, 64) == -1
     assert lib.dyspec_tree_attention_ragged(None, None, None, None, None, None, None, 0, None, None) == -1
     assert lib.dyspec_set_default_shape(4, 4, 96, 4, 0.0) == -2
-    assert lib.dyspec_set_tuning(7, 0) == -1
+    assert lib.dyspec_set_tuning(7, 0, 1) == -1
     assert lib.dyspec_plan_destroy(None) == 0

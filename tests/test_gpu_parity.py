@@ -24,13 +24,13 @@ def rt():
     return binding, runner
 
 
-def run_and_check(rt, w, regime=-1, ctas=0, words_per_row=None):
+def run_and_check(rt, w, regime=-1, ctas=0, words_per_row=None, fuse=0):
     B, R = rt
-    B.dyspec_set_tuning(regime, ctas)
+    B.dyspec_set_tuning(regime, ctas, fuse)
     try:
         batch = R.DeviceBatch(w, words_per_row=words_per_row)
     finally:
-        B.dyspec_set_tuning(-1, 0)
+        B.dyspec_set_tuning(-1, 0, 0)
     batch.step()
     bits, depths, out_bits, status = batch.results()
     assert status == 0
@@ -75,12 +75,13 @@ def test_tensor_core_regime_shapes(rt, hq, hkv, d):
         run_and_check(rt, wl.make_custom(15, hq, hkv, d, [260, 64, 3, 0], trees), regime=1, ctas=ctas)
 
 
+@pytest.mark.parametrize("fuse", [0, 1])
 @pytest.mark.parametrize("ctas", [1, 3, 40, 1000])
-def test_split_count_does_not_change_results(rt, ctas):
+def test_split_count_does_not_change_results(rt, ctas, fuse):
     """Forcing the scheduler to balance over few or many CTAs changes the split-KV cuts, not the answer."""
     w = wl.make_custom(77, 8, 2, 128, [700, 45], [wl.greedy_tree(np.random.default_rng(1), 90, 8, 0.3),
                                                    wl.greedy_tree(np.random.default_rng(2), 33, 4, 0.2)])
-    _, got, _ = run_and_check(rt, w, ctas=ctas)
+    _, got, _ = run_and_check(rt, w, ctas=ctas, fuse=fuse)
     _, base, _ = run_and_check(rt, w, ctas=2)
     assert np.abs(got - base).max() <= 2 ** -6     # both are bf16 roundings of nearly equal fp32 values
 
@@ -170,9 +171,11 @@ def test_single_request_entry_points(rt):
 
 
 def test_runs_are_bitwise_repeatable(rt):
+    """Also checks that the arrival counters of the fused combine are left at zero by every call."""
     w = wl.make_config(2)
     batch, got, _ = run_and_check(rt, w)
     first = batch.results()[2].copy()
-    batch.out.zero_()
-    batch.step()
-    assert np.array_equal(batch.results()[2], first)
+    for _ in range(3):
+        batch.out.zero_()
+        batch.step()
+        assert np.array_equal(batch.results()[2], first)

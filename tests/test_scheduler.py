@@ -15,13 +15,13 @@ def B():
     return binding
 
 
-def check_schedule(B, hq, hkv, d, Ls, ns, regime=-1, ctas=0):
-    B.dyspec_set_tuning(regime, ctas)
+def check_schedule(B, hq, hkv, d, Ls, ns, regime=-1, ctas=0, fuse=0):
+    B.dyspec_set_tuning(regime, ctas, fuse)
     try:
         W = B.dyspec_words_per_row(max(list(ns) + [0]))
         items, cta_begin, info = B.dyspec_schedule_dry_run(hq, hkv, d, Ls, ns, W)
     finally:
-        B.dyspec_set_tuning(-1, 0)
+        B.dyspec_set_tuning(-1, 0, 0)
     g = hq // hkv
     bm, bn = info["rows_per_tile"], info["keys_per_tile"]
     npt = bm // g
