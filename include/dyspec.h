@@ -101,7 +101,8 @@ size_t dyspec_plan_workspace_bytes(const dyspec_plan_t* plan);
 
 /* Scheduler introspection (for tests and benchmarks): field 0 = work items, 1 = CTAs launched,
  * 2 = query-tile groups, 3 = groups that are split, 4 = max splits of a group, 5 = kernel regime
- * (0 = warp-level mma tiles, 1 = tcgen05 tiles), 6 = total key tiles, 7 = query rows per tile. */
+ * (0 = warp-level mma tiles, 1 = tcgen05 tiles), 6 = total key tiles, 7 = query rows per tile,
+ * 8 = thread-block cluster size (1 = no clusters). */
 int64_t dyspec_plan_info(const dyspec_plan_t* plan, int field);
 
 /* Host-only view of the scheduler, for tests and tools: validates the arguments and schedules exactly
@@ -109,15 +110,16 @@ int64_t dyspec_plan_info(const dyspec_plan_t* plan, int field);
  * Copies up to max_items work items into items_out (host, 8 int32 each: request, kv head, first
  * packed query row, first key tile, one-past-last key tile, partial slot or -1, group id, number of
  * splits of the group), the per-CTA item ranges into cta_begin_out (host, n_ctas + 1 entries, at most
- * max_ctas) and, into info_out (host int64 [10]), the eight dyspec_plan_info fields followed by keys
- * per tile and workspace bytes.  Any output pointer may be NULL.  Returns the item count or an error. */
+ * max_ctas) and, into info_out (host int64 [11]), dyspec_plan_info fields 0-7 followed by keys per
+ * tile, workspace bytes and the cluster size.  Any output pointer may be NULL.  Returns the item count or an error. */
 int dyspec_schedule_dry_run(int n_q_heads, int n_kv_heads, int head_dim, int n_req, const int32_t* prefix_len,
                             const int32_t* n_nodes, int words_per_row, int32_t* items_out, int max_items,
                             int32_t* cta_begin_out, int max_ctas, int64_t* info_out);
 
 /* Testing knobs, read when a plan is created: force the regime (-1 = automatic), the number of
- * CTAs the scheduler balances over (<= 0 = automatic), and whether split-KV partials are merged by the
- * last work item of a group to finish (1) or by a separate combine kernel (0, the default). */
+ * CTAs the scheduler balances over (<= 0 = automatic), and how split-KV partials are merged: 0 = by
+ * the separate combine kernel, 2 (default) = inside a thread-block cluster through distributed shared
+ * memory when the plan is uniform enough, else as 0. */
 int dyspec_set_tuning(int force_regime, int force_ctas, int fuse_combine);
 
 /* Developer aid: event trace of the attention kernels.  trace_buffer is a dev uint64 array of

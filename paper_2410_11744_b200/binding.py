@@ -89,7 +89,7 @@ def dyspec_words_per_row(max_nodes: int) -> int:
     return lib.dyspec_words_per_row(max_nodes)
 
 
-def dyspec_set_tuning(force_regime: int = -1, force_ctas: int = 0, fuse_combine: int = 0) -> None:
+def dyspec_set_tuning(force_regime: int = -1, force_ctas: int = 0, fuse_combine: int = 2) -> None:
     _check(lib.dyspec_set_tuning(force_regime, force_ctas, fuse_combine), "dyspec_set_tuning")
 
 
@@ -129,7 +129,8 @@ class Plan:
         return int(lib.dyspec_plan_info(self.handle, field))
 
     def describe(self) -> dict:
-        names = ["items", "ctas", "groups", "split_groups", "max_splits", "regime", "key_tiles", "rows_per_tile"]
+        names = ["items", "ctas", "groups", "split_groups", "max_splits", "regime", "key_tiles", "rows_per_tile",
+                 "cluster"]
         return {k: self.info(i) for i, k in enumerate(names)}
 
     def destroy(self) -> None:
@@ -169,7 +170,7 @@ def dyspec_schedule_dry_run(n_q_heads: int, n_kv_heads: int, head_dim: int, pref
     nn = np.asarray(list(n_nodes) or [0], dtype=np.int32)
     items = np.zeros((max_items, 8), dtype=np.int32)
     cta = np.zeros(max_items + 1, dtype=np.int32)
-    info = np.zeros(10, dtype=np.int64)
+    info = np.zeros(11, dtype=np.int64)
     rc = lib.dyspec_schedule_dry_run(n_q_heads, n_kv_heads, head_dim, n_req, pl.ctypes.data, nn.ctypes.data,
                                      words_per_row, items.ctypes.data, max_items, cta.ctypes.data, max_items + 1,
                                      info.ctypes.data)
@@ -178,7 +179,7 @@ def dyspec_schedule_dry_run(n_q_heads: int, n_kv_heads: int, head_dim: int, pref
     if rc > max_items:
         return dyspec_schedule_dry_run(n_q_heads, n_kv_heads, head_dim, prefix_len, n_nodes, words_per_row, rc)
     names = ["items", "ctas", "groups", "split_groups", "max_splits", "regime", "key_tiles", "rows_per_tile",
-             "keys_per_tile", "workspace_bytes"]
+             "keys_per_tile", "workspace_bytes", "cluster"]
     d = {k: int(v) for k, v in zip(names, info)}
     return items[:rc].copy(), cta[:d["ctas"] + 1].copy(), d
 

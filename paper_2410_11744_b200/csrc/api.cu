@@ -28,7 +28,7 @@ namespace {
 
 int g_force_regime = -1;
 int g_force_ctas = 0;
-int g_fuse_combine = 0;
+int g_fuse_combine = 2;   // 0 separate combine kernel, 2 cluster merge when the plan allows, else as 0
 unsigned long long* g_trace = nullptr;   // device buffer for the optional kernel event trace
 int g_trace_capacity = 0;
 
@@ -80,6 +80,7 @@ struct dyspec_plan {
   std::vector<WorkItem> items_strided;  // device layout: CTA c's items at [c * items_stride, ...)
   int items_stride = 1;
   int fuse_combine = 1;
+  int cluster = 1;                      // > 1: one thread-block cluster of this size per split group
   std::vector<int32_t> cta_begin;
   std::vector<GroupInfo> split_groups;
   int n_ctas = 0, n_slots = 0, max_splits = 1;
@@ -132,6 +133,48 @@ void schedule(dyspec_plan& pl) {
   pl.items_stride = 1;
   pl.fuse_combine = g_fuse_combine;
   if (groups.empty()) { pl.n_ctas = 0; pl.cta_begin.push_back(0); return; }
+
+  // Cluster mode (warp-level regime): when every group can be cut into the same number C of pieces
+  // and all pieces fit in one wave, launch one cluster of C CTAs per group; the pieces are merged
+  // through distributed shared memory instead of a round trip through global memory.
+  pl.cluster = 1;
+  if (pl.regime == 0 && g_fuse_combine == 2 && g_force_ctas <= 0) {
+    int max_tiles = 0;
+    for (const Group& gr : groups) max_tiles = std::max(max_tiles, gr.tiles);
+    const double mean_tiles = double(total_tiles) / double(groups.size());
+    for (int C : {8, 4, 2}) {
+      if (int64_t(groups.size()) * C > kNumSMs) continue;
+      if (mean_tiles / C < 2.0 || double(max_tiles) > 1.3 * mean_tiles) continue;
+      bool ok = true;
+      for (const Group& gr : groups) ok = ok && gr.tiles >= C;
+      if (!ok) continue;
+      pl.cluster = C;
+      break;
+    }
+  }
+  if (pl.cluster > 1) {
+    const int C = pl.cluster;
+    pl.cta_begin.push_back(0);
+    for (size_t gi = 0; gi < groups.size(); ++gi) {
+      const Group& gr = groups[gi];
+      const ReqInfo& rq = pl.reqs[size_t(gr.req)];
+      for (int c = 0; c < C; ++c) {
+        WorkItem it{};
+        it.kv_row0 = rq.kv_row0; it.prefix_len = rq.prefix_len; it.n_nodes = rq.n_nodes; it.node0 = rq.node0;
+        it.req = gr.req; it.kv_head = gr.kvh; it.row0 = gr.row0;
+        it.tile_begin = int(int64_t(gr.tiles) * c / C);
+        it.tile_end = int(int64_t(gr.tiles) * (c + 1) / C);
+        it.slot = -1; it.slot0 = -1; it.group = int(gi); it.n_splits = C; it.n_in_cta = 1;
+        pl.items.push_back(it);
+        pl.cta_begin.push_back(int32_t(pl.items.size()));
+      }
+    }
+    pl.max_splits = C;
+    pl.n_ctas = int(pl.items.size());
+    pl.items_stride = 1;
+    pl.items_strided = pl.items;
+    return;
+  }
 
   const int ctas_per_sm = 1;   // one wave: every CTA is resident from the start and owns its SM's load queue
   int max_ctas = g_force_ctas > 0 ? g_force_ctas : kNumSMs * ctas_per_sm;
@@ -265,7 +308,7 @@ int dyspec_words_per_row(int max_nodes) {
 }
 
 int dyspec_set_tuning(int force_regime, int force_ctas, int fuse_combine) {
-  if (force_regime < -1 || force_regime > 1 || fuse_combine < 0 || fuse_combine > 1) return DYSPEC_ERR_INVALID_ARG;
+  if (force_regime < -1 || force_regime > 1 || (fuse_combine != 0 && fuse_combine != 2)) return DYSPEC_ERR_INVALID_ARG;
   g_force_regime = force_regime;
   g_force_ctas = force_ctas;
   g_fuse_combine = fuse_combine;
@@ -380,7 +423,7 @@ int dyspec_schedule_dry_run(int n_q_heads, int n_kv_heads, int head_dim, int n_r
   if (info_out) {
     info_out[0] = n_items; info_out[1] = pl->n_ctas; info_out[2] = pl->n_groups; info_out[3] = int64_t(pl->split_groups.size());
     info_out[4] = pl->max_splits; info_out[5] = pl->regime; info_out[6] = pl->total_tiles; info_out[7] = pl->bm;
-    info_out[8] = pl->bn; info_out[9] = int64_t(pl->workspace_bytes);
+    info_out[8] = pl->bn; info_out[9] = int64_t(pl->workspace_bytes); info_out[10] = pl->cluster;
   }
   delete pl;
   return n_items;
@@ -406,6 +449,7 @@ int64_t dyspec_plan_info(const dyspec_plan_t* plan, int field) {
     case 5: return plan->regime;
     case 6: return plan->total_tiles;
     case 7: return plan->bm;
+    case 8: return plan->cluster;
     default: return DYSPEC_ERR_INVALID_ARG;
   }
 }
@@ -448,7 +492,8 @@ int dyspec_tree_attention_ragged(const dyspec_plan_t* plan, const void* q, const
   p.words_per_row = plan->W; p.slot_floats = bm * (plan->d + 2);
   p.scale_log2e = plan->scale * kLog2e;
   p.items_stride = plan->items_stride;
-  p.fuse_combine = plan->fuse_combine && plan->regime == 0;
+  p.fuse_combine = 0;
+  p.cluster_size = plan->cluster;
   p.trace = g_trace; p.trace_capacity = g_trace_capacity;
 
   cudaError_t e;
@@ -601,7 +646,8 @@ extern "C" int dyspec_tree_attention_static(const void* q, const void* k_cache, 
   p.words_per_row = pl->W; p.slot_floats = bm * (pl->d + 2);
   p.scale_log2e = pl->scale * kLog2e;
   p.items_stride = pl->items_stride;
-  p.fuse_combine = pl->fuse_combine && pl->regime == 0;
+  p.fuse_combine = 0;
+  p.cluster_size = pl->cluster;
 
   cudaError_t e;
   if (pl->regime == 0) e = launch_attn_mma(pl->d, pl->n_ctas, mq, mk, mv, p, st);

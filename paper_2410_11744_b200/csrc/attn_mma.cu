@@ -6,7 +6,9 @@
 // 128-byte-swizzled shared-memory ring guarded by mbarriers; compute warps run QK^T and PV with
 // mma.sync.m16n8k16 (bf16 in, fp32 accumulate), an fp32 online softmax in the exp2 domain, and apply
 // the ancestor bitmask on tree tiles.  A CTA walks its list of work items; an item either writes
-// final bf16 rows or an fp32 partial (O, m, l) for the split-KV combine.
+// final bf16 rows or an fp32 partial (O, m, l) for the split-KV combine kernel.  In cluster mode
+// (uniform small batches) the splits of a query tile are the CTAs of one thread-block cluster and
+// are merged on chip through distributed shared memory instead.
 #include "common.cuh"
 
 namespace dyspec {
@@ -71,7 +73,6 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   const uint32_t bar_full = s_bar, bar_empty = s_bar + 8 * kStages;
   const uint32_t bar_qfull = s_bar + 16 * kStages, bar_qempty = bar_qfull + 8;
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::kBarOffset + 16 * kStages + 16);
-  volatile int* last_flag = reinterpret_cast<volatile int*>(smem + L::kBarOffset + 16 * kStages + 20);
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -132,6 +133,10 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           }
         }
       }
+    }
+    if (p.cluster_size > 1) {        // every thread of the cluster takes part in the two cluster barriers
+      cluster_sync_all();
+      cluster_sync_all();
     }
     return;
   }
@@ -299,7 +304,92 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
     l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1);
     l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
-    if (item.slot < 0) {
+    if (p.cluster_size > 1) {
+      // ---- split-KV combine inside a thread-block cluster: the CTAs of a cluster hold the splits of
+      // one query tile.  Each parks its partial (O, m, l) in its own shared memory (the K/V ring is
+      // idle by now: a CTA owns exactly one item in this mode), the cluster synchronises, and CTA k
+      // merges rows [k * BM / C, (k + 1) * BM / C) of all C partials through distributed shared memory.
+      const int C = p.cluster_size;                       // 2, 4 or 8
+      const int log2c = C == 2 ? 1 : (C == 4 ? 2 : 3);
+      asm volatile("bar.sync 1, %0;" ::"n"(kComputeWarps * 32) : "memory");     // all warps are done with the ring
+      float* sc_o = reinterpret_cast<float*>(smem + L::kQBytes);                 // [BM][D]
+      float* sc_m = sc_o + BM * D;                                               // [BM]
+      float* sc_l = sc_m + BM;                                                   // [BM]
+      {
+        const int r_lo = wrow + gid, r_hi = r_lo + 8;
+#pragma unroll
+        for (int j = 0; j < DT; ++j) {
+          const int c = j * 8 + tig * 2;
+          *reinterpret_cast<float2*>(sc_o + r_lo * D + c) = make_float2(o[j][0], o[j][1]);
+          *reinterpret_cast<float2*>(sc_o + r_hi * D + c) = make_float2(o[j][2], o[j][3]);
+        }
+        if (tig == 0) { sc_m[r_lo] = m_lo; sc_l[r_lo] = l_lo; sc_m[r_hi] = m_hi; sc_l[r_hi] = l_hi; }
+      }
+      cluster_sync_all();
+      // A warp merges BM / C / 4 rows from C sources: always 16 (row, source) pairs.  All their loads
+      // are issued before the first use, so the merge costs about two remote-load latencies in all.
+      const int rank = int(cluster_ctarank());
+      const int row_base = rank * (BM >> log2c) + warp * ((BM >> log2c) / kComputeWarps);
+      const uint32_t a_o = smem_u32(sc_o), a_m = smem_u32(sc_m), a_l = smem_u32(sc_l);
+      constexpr int V = D / 32;
+      float mm[16], ll[16];
+      float vv[16][V];
+#pragma unroll
+      for (int q = 0; q < 16; ++q) {
+        const int r = row_base + (q >> log2c);
+        const uint32_t src = uint32_t(q & (C - 1));
+        mm[q] = ld_dsmem_f32(map_to_cta(a_m + 4u * uint32_t(r), src));
+        ll[q] = ld_dsmem_f32(map_to_cta(a_l + 4u * uint32_t(r), src));
+        const uint32_t av = map_to_cta(a_o + 4u * uint32_t(r * D + lane * V), src);
+        if constexpr (V == 4) {
+          const float4 v = ld_dsmem_f32x4(av);
+          vv[q][0] = v.x; vv[q][1] = v.y; vv[q][2] = v.z; vv[q][3] = v.w;
+        } else {
+          const float2 v = ld_dsmem_f32x2(av);
+          vv[q][0] = v.x; vv[q][1] = v.y;
+        }
+      }
+      // reduce groups of C consecutive pairs (one row each)
+#pragma unroll
+      for (int q0 = 0; q0 < 16; q0 += 2) {
+        if ((q0 & (C - 1)) != 0) continue;     // q0 starts a row only when it is a multiple of C
+        const int r = row_base + (q0 >> log2c);
+        const int row = item.row0 + r;
+        float m = -INFINITY;
+#pragma unroll
+        for (int c = 0; c < 8; ++c)
+          if (c < C && q0 + c < 16) m = fmaxf(m, mm[q0 + c]);
+        const float ref = m == -INFINITY ? 0.f : m;
+        float acc[V];
+#pragma unroll
+        for (int k = 0; k < V; ++k) acc[k] = 0.f;
+        float lsum = 0.f;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          if (c < C && q0 + c < 16) {
+            const float wgt = fast_exp2(mm[q0 + c] - ref);
+            lsum += wgt * ll[q0 + c];
+#pragma unroll
+            for (int k = 0; k < V; ++k) acc[k] += wgt * vv[q0 + c][k];
+          }
+        }
+        if (row < n_rows) {
+          const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
+          const int node = row >> p.log2_g;
+          const int head = item.kv_head * g + (row & (g - 1));
+          __nv_bfloat16* out = p.out + (size_t(rq.node0 + node) * p.n_q_heads + head) * D;
+          if constexpr (V == 4) {
+            uint2 o2;
+            o2.x = pack_bf16x2(acc[0] * inv, acc[1] * inv);
+            o2.y = pack_bf16x2(acc[2] * inv, acc[3] * inv);
+            *reinterpret_cast<uint2*>(out + lane * 4) = o2;
+          } else {
+            *reinterpret_cast<uint32_t*>(out + lane * 2) = pack_bf16x2(acc[0] * inv, acc[1] * inv);
+          }
+        }
+      }
+      cluster_sync_all();                                 // nobody leaves while a peer still reads its shared memory
+    } else if (item.slot < 0) {
       const float inv_lo = l_lo > 0.f ? 1.f / l_lo : 0.f, inv_hi = l_hi > 0.f ? 1.f / l_hi : 0.f;
       const int head_lo = item.kv_head * g + (row_lo & (g - 1)), head_hi = item.kv_head * g + (row_hi & (g - 1));
       __nv_bfloat16* out_lo = p.out + (size_t(rq.node0 + node_lo) * p.n_q_heads + head_lo) * D;
@@ -324,57 +414,6 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         if (ok_lo) { slot[BM * D + r_lo] = m_lo; slot[BM * D + BM + r_lo] = l_lo; }
         if (ok_hi) { slot[BM * D + r_hi] = m_hi; slot[BM * D + BM + r_hi] = l_hi; }
       }
-      if (p.fuse_combine) {
-        // Split-KV combine by the last arriver: publish the partial, count this item in, and if every
-        // other item of the group has already been counted, merge all of the group's partials here.
-        __threadfence();
-        asm volatile("bar.sync 1, %0;" ::"n"(kComputeWarps * 32) : "memory");
-        if (threadIdx.x == 0) *last_flag = atomicAdd(p.counters + item.group, 1) == item.n_splits - 1 ? 1 : 0;
-        asm volatile("bar.sync 1, %0;" ::"n"(kComputeWarps * 32) : "memory");
-        if (*last_flag) {
-          __threadfence();
-          if (threadIdx.x == 0) p.counters[item.group] = 0;      // leave the counter ready for the next call
-          const float* base = p.partial + size_t(item.slot0) * p.slot_floats;
-          constexpr int V = D / 32;                              // floats per lane
-          for (int rr = 0; rr < 16; ++rr) {
-            const int r = wrow + rr;
-            const int row = item.row0 + r;
-            if (row >= n_rows) break;
-            float m = -INFINITY;
-            for (int sidx = 0; sidx < item.n_splits; ++sidx)
-              m = fmaxf(m, __ldcg(base + size_t(sidx) * p.slot_floats + BM * D + r));
-            const float ref = m == -INFINITY ? 0.f : m;
-            float acc[V];
-#pragma unroll
-            for (int k = 0; k < V; ++k) acc[k] = 0.f;
-            float lsum = 0.f;
-            for (int sidx = 0; sidx < item.n_splits; ++sidx) {
-              const float* sl = base + size_t(sidx) * p.slot_floats;
-              const float wgt = fast_exp2(__ldcg(sl + BM * D + r) - ref);
-              lsum += wgt * __ldcg(sl + BM * D + BM + r);
-              if constexpr (V == 4) {
-                const float4 v = __ldcg(reinterpret_cast<const float4*>(sl + r * D + lane * 4));
-                acc[0] += wgt * v.x; acc[1] += wgt * v.y; acc[2] += wgt * v.z; acc[3] += wgt * v.w;
-              } else {
-                const float2 v = __ldcg(reinterpret_cast<const float2*>(sl + r * D + lane * 2));
-                acc[0] += wgt * v.x; acc[1] += wgt * v.y;
-              }
-            }
-            const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
-            const int node = row >> p.log2_g;
-            const int head = item.kv_head * g + (row & (g - 1));
-            __nv_bfloat16* out = p.out + (size_t(rq.node0 + node) * p.n_q_heads + head) * D;
-            if constexpr (V == 4) {
-              uint2 o2;
-              o2.x = pack_bf16x2(acc[0] * inv, acc[1] * inv);
-              o2.y = pack_bf16x2(acc[2] * inv, acc[3] * inv);
-              *reinterpret_cast<uint2*>(out + lane * 4) = o2;
-            } else {
-              *reinterpret_cast<uint32_t*>(out + lane * 2) = pack_bf16x2(acc[0] * inv, acc[1] * inv);
-            }
-          }
-        }
-      }
     }
     if (threadIdx.x == 0 && w == item_begin) stamp(6);
   }
@@ -390,15 +429,19 @@ cudaError_t launch_attn_mma(int head_dim, int n_ctas, const CUtensorMap& mq, con
                             const AttnParams& p, cudaStream_t stream) {
   const size_t smem = attn_mma_smem_bytes(head_dim);
   static bool attr_set[2] = {false, false};
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[1].id = cudaLaunchAttributeClusterDimension;
+  attr[1].val.clusterDim.x = unsigned(p.cluster_size > 1 ? p.cluster_size : 1);
+  attr[1].val.clusterDim.y = 1;
+  attr[1].val.clusterDim.z = 1;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(unsigned(n_ctas));
   cfg.blockDim = dim3(unsigned(kThreads));
   cfg.stream = stream;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = p.cluster_size > 1 ? 2 : 1;
   cudaError_t e = cudaSuccess;
   if (head_dim == 128) {
     if (!attr_set[0]) {

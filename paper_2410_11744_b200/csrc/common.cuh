@@ -77,7 +77,8 @@ struct AttnParams {
   int32_t slot_floats;             // BM * (D + 2)
   float scale_log2e;               // scale * log2(e)
   int32_t items_stride;            // items per CTA slot in `items`
-  int32_t fuse_combine;            // 1: the last item of a split group to finish merges the partials itself
+  int32_t fuse_combine;            // reserved (0)
+  int32_t cluster_size;            // > 1: one cluster per split group; partials are merged through distributed shared memory
   unsigned long long* trace;       // optional event trace (null in normal use): [0] = count, then entries
   int32_t trace_capacity;
 };
@@ -185,6 +186,36 @@ __device__ __forceinline__ bool counter_wait(uint32_t addr, uint32_t target, vol
 // kernels) may still read.  The predecessor lets dependents start early with trigger_dependents().
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void trigger_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// Thread-block cluster helpers (distributed shared memory; no multicast is used anywhere).
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_smem_addr, uint32_t cta_rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_smem_addr), "r"(cta_rank));
+  return r;
+}
+__device__ __forceinline__ float ld_dsmem_f32(uint32_t addr) {
+  float v;
+  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
+  return v;
+}
+__device__ __forceinline__ float4 ld_dsmem_f32x4(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+  return v;
+}
+__device__ __forceinline__ float2 ld_dsmem_f32x2(uint32_t addr) {
+  float2 v;
+  asm volatile("ld.shared::cluster.v2.f32 {%0,%1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr) : "memory");
+  return v;
+}
 
 // TMA: 3-D tiled load global -> shared, completion on an mbarrier (no multicast anywhere).
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {

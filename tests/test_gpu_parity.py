@@ -24,13 +24,13 @@ def rt():
     return binding, runner
 
 
-def run_and_check(rt, w, regime=-1, ctas=0, words_per_row=None, fuse=0):
+def run_and_check(rt, w, regime=-1, ctas=0, words_per_row=None, fuse=2):
     B, R = rt
     B.dyspec_set_tuning(regime, ctas, fuse)
     try:
         batch = R.DeviceBatch(w, words_per_row=words_per_row)
     finally:
-        B.dyspec_set_tuning(-1, 0, 0)
+        B.dyspec_set_tuning(-1, 0, 2)
     batch.step()
     bits, depths, out_bits, status = batch.results()
     assert status == 0
@@ -75,7 +75,19 @@ def test_tensor_core_regime_shapes(rt, hq, hkv, d):
         run_and_check(rt, wl.make_custom(15, hq, hkv, d, [260, 64, 3, 0], trees), regime=1, ctas=ctas)
 
 
-@pytest.mark.parametrize("fuse", [0, 1])
+@pytest.mark.parametrize("hq,hkv,d,L,n", [(32, 32, 128, 1024, 64), (16, 16, 64, 700, 40), (8, 2, 128, 3000, 16),
+                                          (4, 4, 128, 9000, 33), (64, 8, 128, 600, 8)])
+def test_cluster_combine(rt, hq, hkv, d, L, n):
+    """Uniform small batches: one thread-block cluster per query tile, partials merged through
+    distributed shared memory (cluster sizes 2, 4 and 8, both head dims, ragged last rows)."""
+    B, _ = rt
+    rng = np.random.default_rng(hq + n)
+    w = wl.make_custom(50, hq, hkv, d, [L], [wl.greedy_tree(rng, n, 4, 0.3)])
+    batch, _, _ = run_and_check(rt, w)
+    assert batch.plan.describe()["cluster"] > 1
+
+
+@pytest.mark.parametrize("fuse", [0, 2])
 @pytest.mark.parametrize("ctas", [1, 3, 40, 1000])
 def test_split_count_does_not_change_results(rt, ctas, fuse):
     """Forcing the scheduler to balance over few or many CTAs changes the split-KV cuts, not the answer."""

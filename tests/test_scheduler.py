@@ -15,13 +15,13 @@ def B():
     return binding
 
 
-def check_schedule(B, hq, hkv, d, Ls, ns, regime=-1, ctas=0, fuse=0):
+def check_schedule(B, hq, hkv, d, Ls, ns, regime=-1, ctas=0, fuse=2):
     B.dyspec_set_tuning(regime, ctas, fuse)
     try:
         W = B.dyspec_words_per_row(max(list(ns) + [0]))
         items, cta_begin, info = B.dyspec_schedule_dry_run(hq, hkv, d, Ls, ns, W)
     finally:
-        B.dyspec_set_tuning(-1, 0, 0)
+        B.dyspec_set_tuning(-1, 0, 2)
     g = hq // hkv
     bm, bn = info["rows_per_tile"], info["keys_per_tile"]
     npt = bm // g
@@ -44,7 +44,11 @@ def check_schedule(B, hq, hkv, d, Ls, ns, regime=-1, ctas=0, fuse=0):
         assert pieces[0][0] == 0 and pieces[-1][1] == expect[key]
         for a, b in zip(pieces, pieces[1:]):
             assert a[1] == b[0]
-        if len(pieces) == 1:
+        if info["cluster"] > 1:
+            # cluster mode: every group is cut into `cluster` pieces merged on chip, no global slots
+            assert len(pieces) == info["cluster"]
+            assert all(slot == -1 and nsp == info["cluster"] for _, _, slot, nsp in pieces)
+        elif len(pieces) == 1:
             assert pieces[0][2] == -1 and pieces[0][3] == 1
         else:
             for _, _, slot, nsp in pieces:
@@ -84,6 +88,19 @@ def test_degenerate_batches(B):
 def test_regime_1_tiles(B):
     info, _ = check_schedule(B, 64, 8, 128, [2048], [512], regime=1)
     assert info["rows_per_tile"] == 256 and info["keys_per_tile"] == 128 and info["regime"] == 1
+
+
+def test_cluster_mode_is_used_for_uniform_small_batches(B):
+    # Llama2-7B shape, 64 nodes: 32 groups x 17 tiles -> clusters of 4 (128 CTAs), no workspace
+    info, loads = check_schedule(B, 32, 32, 128, [1024], [64])
+    assert info["cluster"] == 4 and info["ctas"] == 128 and info["workspace_bytes"] == 0
+    assert max(loads) - min(loads) <= 1
+    # forcing a separate combine kernel switches it off
+    info, _ = check_schedule(B, 32, 32, 128, [1024], [64], fuse=0)
+    assert info["cluster"] == 1 and info["workspace_bytes"] > 0
+    # very uneven groups do not qualify
+    info, _ = check_schedule(B, 8, 8, 128, [64, 4096], [16, 16])
+    assert info["cluster"] == 1
 
 
 def test_regime_is_chosen_from_packed_rows(B):
