@@ -30,6 +30,9 @@ if ROOT not in sys.path:
 METRIC = "tree_verify_attention_tree_tokens_per_s"
 UNIT = "tree tokens/s"
 L2_BYTES = 126 * 1024 * 1024
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu
+# captures summarised under profiles/ (tree_attn_mma_c2_*.md, tree_attn_tc_c4_*.md)
+NCU_TRAFFIC_BYTES = {"c2_llama2_7b_L1024_n64": 18407680, "c4_llama2_70b_L2048_n512": 19004928}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -343,13 +346,7 @@ def run_ours(args):
         return
 
     roof = roofline_entry(m, peaks, peaks_kind)
-    traffic_path = os.path.join(ROOT, "profiles", "traffic.json")
-    if os.path.exists(traffic_path):
-        try:
-            with open(traffic_path) as f:
-                roof["traffic"] = json.load(f).get(w.name)
-        except Exception:
-            pass
+    roof["traffic"] = NCU_TRAFFIC_BYTES.get(w.name)
 
     # ---- the other configs, same protocol, fewer steps (reported for context in `per_config`)
     per_config = []
