@@ -118,6 +118,20 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return done != 0;
 }
+// Non-blocking probe.  A try_wait that does not succeed at once suspends the thread for a
+// hardware-defined time slice and is slow to notice the completion (~700 cycles measured on B200);
+// polling with test_wait sees it within one probe latency (~180 cycles).
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+  uint32_t done;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(done)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return done != 0;
+}
 __device__ __forceinline__ uint64_t global_timer_ns() {
   uint64_t t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
@@ -129,11 +143,10 @@ constexpr uint64_t kWaitLimitNs = 1000ull * 1000ull * 1000ull;  // 1 s per wait,
 // Bounded mbarrier wait.  `abort_flag` lives in shared memory: once any wait of the CTA ran out,
 // later waits return at once.  Returns false when the wait did not complete.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
-  // fast path: try_wait itself blocks for a short hardware-defined time, so a few tries cover every
-  // ordinary wait without touching the (slow) global timer
+  // fast path: spin on the non-blocking probe (lowest hand-off latency); ordinary waits end here
 #pragma unroll 1
-  for (int i = 0; i < 16; ++i)
-    if (mbar_try_wait(bar, parity)) return true;
+  for (int i = 0; i < 256; ++i)
+    if (mbar_test_wait(bar, parity)) return true;
   if (*abort_flag) return false;
   const uint64_t t0 = global_timer_ns();
   uint32_t spins = 0;
