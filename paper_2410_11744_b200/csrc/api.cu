@@ -28,6 +28,7 @@ namespace {
 
 int g_force_regime = -1;
 int g_force_ctas = 0;
+int g_item_cost = 0;       // scheduler experiment knob (0 = default)
 int g_fuse_combine = 2;   // 0 separate combine kernel, 2 cluster merge when the plan allows, else as 0
 unsigned long long* g_trace = nullptr;   // device buffer for the optional kernel event trace
 int g_trace_capacity = 0;
@@ -178,7 +179,9 @@ void schedule(dyspec_plan& pl) {
 
   const int ctas_per_sm = 1;   // one wave: every CTA is resident from the start and owns its SM's load queue
   int max_ctas = g_force_ctas > 0 ? g_force_ctas : kNumSMs * ctas_per_sm;
-  const int item_cost = 1;                               // fixed per-item overhead, in key tiles
+  // fixed per-item overhead (Q load, pipeline fill, epilogue), in key tiles: measured ~1 tile of 64 keys in
+  // regime 0 and ~3 tiles of 128 keys in regime 1
+  const int item_cost = g_item_cost > 0 ? g_item_cost : (pl.regime == 0 ? 1 : 3);
   const int min_tiles = pl.regime == 0 ? 2 : 2;          // smallest piece worth a split
   const int64_t total_cost = total_tiles + int64_t(groups.size()) * item_cost;
   int64_t target = (total_cost + max_ctas - 1) / max_ctas;
@@ -310,7 +313,8 @@ int dyspec_words_per_row(int max_nodes) {
 int dyspec_set_tuning(int force_regime, int force_ctas, int fuse_combine) {
   if (force_regime < -1 || force_regime > 1 || (fuse_combine != 0 && fuse_combine != 2)) return DYSPEC_ERR_INVALID_ARG;
   g_force_regime = force_regime;
-  g_force_ctas = force_ctas;
+  g_force_ctas = force_ctas >= 0 ? force_ctas : 0;
+  g_item_cost = force_ctas < 0 ? -force_ctas : 0;   // negative values select the per-item cost instead (experiments)
   g_fuse_combine = fuse_combine;
   return DYSPEC_OK;
 }

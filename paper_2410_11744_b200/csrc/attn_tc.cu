@@ -130,6 +130,12 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
         "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
       : "memory");
 }
+// 256-bit global stores (sm_100): one full 32-byte sector per lane and instruction, which matters when
+// every lane of a warp writes to a different row.
+__device__ __forceinline__ void st_global_v8(void* ptr, const uint32_t* v) {
+  asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+               ::"l"(ptr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]) : "memory");
+}
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -225,8 +231,12 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    // The whole warp walks the loop (addresses, slot indices and barrier waits are warp-uniform);
+    // only the elected lane issues the tcgen05 instructions.
+    {
+      const bool elected = lane == 0;
       TraceCursor tc_cur = trace_open(p, 0, 3);
+      if (!elected) tc_cur.at = nullptr;
       trace_event(tc_cur, DYSPEC_TAG(0, 9, 0));
       constexpr uint32_t idesc_qk = make_idesc(BN, 0);
       constexpr uint32_t idesc_pv = make_idesc(D, 1);
@@ -242,9 +252,9 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
 #pragma unroll
         for (int ks = 0; ks < D / 16; ++ks) {
           const uint32_t off = (uint32_t(ks >> 2) * L::kPanelBytes + uint32_t(ks & 3) * 32u) >> 4;
-          umma_ss_lohi(d_tmem, a_lo + off, kHiK, b_lo + off, kHiK, idesc_qk, ks > 0 ? 1u : 0u);
+          if (elected) umma_ss_lohi(d_tmem, a_lo + off, kHiK, b_lo + off, kHiK, idesc_qk, ks > 0 ? 1u : 0u);
         }
-        tc_commit(s_bar + 8u * uint32_t(B_SREADY + h));
+        if (elected) tc_commit(s_bar + 8u * uint32_t(B_SREADY + h));
       };
       auto issue_pv = [=](int h, uint32_t slot, bool accumulate) {
         const uint32_t b_lo = ring_v_lo0 + slot * (L::kTileBytes >> 4);
@@ -252,7 +262,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         const uint32_t a_tmem = tmem_base + uint32_t(h) * 128u;
 #pragma unroll
         for (int kk = 0; kk < BN / 16; ++kk)
-          umma_ts_lohi(d_tmem, a_tmem + uint32_t(kk) * 8u, b_lo + uint32_t(kk) * (2048u >> 4), kHiV, idesc_pv,
+          if (elected) umma_ts_lohi(d_tmem, a_tmem + uint32_t(kk) * 8u, b_lo + uint32_t(kk) * (2048u >> 4), kHiV, idesc_pv,
                        (accumulate || kk > 0) ? 1u : 0u);
       };
       uint32_t sc = 0, qit = 0;
@@ -271,8 +281,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           tc_fence_after();
           issue_qk(0, kslot);
           if (two) issue_qk(1, kslot);
-          tc_commit(bar(B_SLOT_EMPTY + kslot));
-          if (T == 1) tc_commit(bar(B_QFREE));            // Q is reusable once the item's last QK^T has run
+          if (elected) tc_commit(bar(B_SLOT_EMPTY + kslot));
+          if (T == 1) if (elected) tc_commit(bar(B_QFREE));            // Q is reusable once the item's last QK^T has run
         }
         for (int j = 0; j < T; ++j) {
           const uint32_t vslot = sc % kSlots, vph = (sc / kSlots) & 1;
@@ -282,8 +292,10 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           if (more) ++sc;
           // Slot waits first: an mbarrier wait costs ~180 cycles even when its phase completed long
           // ago; here that latency hides behind the softmax this thread has to wait for anyway.
+#ifndef EXP_NO_SLOT_WAIT
           mbar_wait(bar(B_SLOT_FULL + vslot), vph, abort_flag, p.status);
           if (more) mbar_wait(bar(B_SLOT_FULL + kslot), kph, abort_flag, p.status);
+#endif
           if (j == 0) {
             mbar_wait(bar(B_OFREE + 0), (n_it0 & 1) ^ 1, abort_flag, p.status);
             if (two) mbar_wait(bar(B_OFREE + 1), (n_it1 & 1) ^ 1, abort_flag, p.status);
@@ -294,7 +306,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           tc_fence_after();
           trace_event(tc_cur, DYSPEC_TAG(0, 1, j));
           issue_pv(0, vslot, j > 0);
-          if (!more) tc_commit(bar(B_ODONE + 0));
+          if (!more) if (elected) tc_commit(bar(B_ODONE + 0));
           trace_event(tc_cur, DYSPEC_TAG(0, 5, j));
           if (more) issue_qk(0, kslot);
           trace_event(tc_cur, DYSPEC_TAG(0, 2, j));
@@ -305,14 +317,14 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             tc_fence_after();
             trace_event(tc_cur, DYSPEC_TAG(0, 3, j));
             issue_pv(1, vslot, j > 0);
-            if (!more) tc_commit(bar(B_ODONE + 1));
+            if (!more) if (elected) tc_commit(bar(B_ODONE + 1));
             trace_event(tc_cur, DYSPEC_TAG(0, 6, j));
             if (more) issue_qk(1, kslot);
             trace_event(tc_cur, DYSPEC_TAG(0, 4, j));
           }
-          tc_commit(bar(B_SLOT_EMPTY + vslot));
-          if (more) tc_commit(bar(B_SLOT_EMPTY + kslot));
-          if (j + 2 == T) tc_commit(bar(B_QFREE));
+          if (elected) tc_commit(bar(B_SLOT_EMPTY + vslot));
+          if (more) if (elected) tc_commit(bar(B_SLOT_EMPTY + kslot));
+          if (j + 2 == T) if (elected) tc_commit(bar(B_QFREE));
           trace_event(tc_cur, DYSPEC_TAG(0, 7, j));
         }
         ++n_it0;
@@ -379,6 +391,9 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         tc_fence_after();
         if (r == 0) trace_event(tc_cur, DYSPEC_TAG(1 + h, 1, j));
 
+#ifdef EXP_SKIP_SOFTMAX
+        if (j >= 0) { tc_fence_before(); mbar_arrive(bar(B_PREADY + h)); continue; }
+#endif
 #ifdef EXP_SKIP_SOFTMAX
         if (j >= 0) { tc_fence_before(); mbar_arrive(bar(B_PREADY + h)); continue; }
 #endif
@@ -468,20 +483,24 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       if (item.slot < 0) {
         const float inv = l > 0.f ? 1.f / l : 0.f;
         __nv_bfloat16* out = p.out + (size_t(rq.node0 + node) * p.n_q_heads + head) * D;
+        const bool out_aligned32 = (reinterpret_cast<uintptr_t>(p.out) & 31) == 0;   // rows are multiples of 128 bytes
 #pragma unroll
         for (int c = 0; c < D / 32; ++c) {
           uint32_t v[32];
           tmem_ld32(t_o + uint32_t(c) * 32u, v);
           tmem_wait_ld();
           if (ok) {
+            uint32_t pk[16];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              uint4 o4;
-              o4.x = pack_bf16x2(__uint_as_float(v[8 * i + 0]) * inv, __uint_as_float(v[8 * i + 1]) * inv);
-              o4.y = pack_bf16x2(__uint_as_float(v[8 * i + 2]) * inv, __uint_as_float(v[8 * i + 3]) * inv);
-              o4.z = pack_bf16x2(__uint_as_float(v[8 * i + 4]) * inv, __uint_as_float(v[8 * i + 5]) * inv);
-              o4.w = pack_bf16x2(__uint_as_float(v[8 * i + 6]) * inv, __uint_as_float(v[8 * i + 7]) * inv);
-              *reinterpret_cast<uint4*>(out + c * 32 + i * 8) = o4;
+            for (int i = 0; i < 16; ++i)
+              pk[i] = pack_bf16x2(__uint_as_float(v[2 * i]) * inv, __uint_as_float(v[2 * i + 1]) * inv);
+            if (out_aligned32) {
+              st_global_v8(out + c * 32, pk);
+              st_global_v8(out + c * 32 + 16, pk + 8);
+            } else {
+#pragma unroll
+              for (int i = 0; i < 4; ++i)
+                *reinterpret_cast<uint4*>(out + c * 32 + i * 8) = make_uint4(pk[4 * i], pk[4 * i + 1], pk[4 * i + 2], pk[4 * i + 3]);
             }
           }
         }
@@ -494,10 +513,9 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           uint32_t v[32];
           tmem_ld32(t_o + uint32_t(c) * 32u, v);
           tmem_wait_ld();
-          if (ok) {
+          if (ok) {   // the workspace is 256-byte aligned and slots / rows are multiples of 32 bytes
 #pragma unroll
-            for (int i = 0; i < 8; ++i)
-              *reinterpret_cast<uint4*>(slot + pr * D + c * 32 + i * 4) = make_uint4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+            for (int i = 0; i < 4; ++i) st_global_v8(slot + pr * D + c * 32 + i * 8, v + 8 * i);
           }
         }
         if (ok) {
