@@ -186,7 +186,8 @@ int dyspec_tree_attention(const void* q, const void* k_cache, const void* v_cach
  * optional status word; k_cache / v_cache hold exactly prefix_len + n_nodes rows.
  *
  *   - A batch whose work list plus partials exceed the array is refused with DYSPEC_ERR_WORKSPACE
- *     before anything is launched (as a guide: Llama2-7B shape, prefix 1024, 64 nodes needs 8.2 MiB).
+ *     before anything is launched (as a guide: Llama2-70B shape, prefix 1500, 40 nodes needs 12.2 MiB;
+ *     small uniform batches that merge their splits on chip need only a few KiB).
  *   - The first call on each device looks up the array's device address (with that device current);
  *     make that first call outside any stream capture.
  *   - All calls share the one array, which keeps the previous call's contents; each call rewrites the

@@ -28,10 +28,12 @@ def test_static_scratch_entry_point_matches_ragged_entry_point_twice_in_a_row():
     build.build()
     from paper_2410_11744_b200 import binding as B, runner as R
 
-    # config 2 is cut into split-KV pieces (about 8 MiB of partials in the scratch array); the custom
-    # case after it is smaller and of a different shape, so stale contents would show
+    # the first case is cut into split-KV pieces (about 12 MiB of partials in the scratch array); the
+    # cases after it are smaller and of other shapes (config 2 merges its splits on chip and only
+    # needs the work list), so stale contents would show; then the first shape again
     rng = np.random.default_rng(3)
-    cases = [wl.make_config(2), wl.make_custom(21, 8, 2, 64, [300], [wl.greedy_tree(rng, 40, 4, 0.3)]), wl.make_config(2)]
+    big = wl.make_custom(20, 64, 8, 128, [1500], [wl.greedy_tree(rng, 40, 8, 0.3)])
+    cases = [big, wl.make_custom(21, 8, 2, 64, [300], [wl.greedy_tree(rng, 40, 4, 0.3)]), wl.make_config(2), big]
     for w in cases:
         batch = R.DeviceBatch(w)
         batch.step()                                          # existing entry points: mask + ragged attention
@@ -58,7 +60,7 @@ def test_static_scratch_entry_point_refuses_what_does_not_fit():
     from paper_2410_11744_b200 import build
     build.build()
     from paper_2410_11744_b200 import binding as B, runner as R
-    w = wl.make_config(4)                                     # needs ~24 MiB of partials: over the 16 MiB array
+    w = wl.make_config(3)                                     # 32 heads x 5 splits: ~21 MiB of partials, over the 16 MiB array
     batch = R.DeviceBatch(w)
     batch.build_mask()
     out = torch.zeros_like(batch.out)
