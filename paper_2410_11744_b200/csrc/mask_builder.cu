@@ -27,12 +27,13 @@ build_tree_mask_kernel(const int32_t* __restrict__ parents, const ReqInfo* __res
   int* s_anc = reinterpret_cast<int*>(mask_smem + size_t(n) * W * 4);      // [n]
   int* s_dist = s_anc + n;                                                 // [n]
   const int tid = threadIdx.x, nthr = blockDim.x;
+  bool bad = false;
 
   for (int i = tid; i < n; i += nthr) {
     int parent = parents[node0 + i];
     if (parent < -1 || parent >= i) {
       parent = -1;
-      if (status) atomicCAS(status, 0, DYSPEC_ERR_BAD_TREE);
+      bad = true;
     }
     s_anc[i] = parent;
     s_dist[i] = parent >= 0 ? 1 : 0;
@@ -73,6 +74,11 @@ build_tree_mask_kernel(const int32_t* __restrict__ parents, const ReqInfo* __res
     __syncthreads();
   }
 
+  // Launched with programmatic dependent launch: everything above only read `parents` and worked in
+  // shared memory, so it may overlap the tail of the kernel before it in the stream.  The outputs may
+  // still be in use by that kernel (the mask of the previous call): wait for it before writing.
+  grid_dependency_wait();
+  if (bad && status) atomicCAS(status, 0, DYSPEC_ERR_BAD_TREE);
   for (int i = tid; i < n; i += nthr)
     if (depths) depths[node0 + i] = s_dist[i];
   uint4* out = reinterpret_cast<uint4*>(bits) + size_t(node0) * W4;
@@ -91,8 +97,18 @@ cudaError_t launch_build_tree_mask(const int32_t* parents, const ReqInfo* reqs, 
   }
   int threads = ((max_n + 31) / 32) * 32;
   if (threads < 256) threads = 256;
-  build_tree_mask_kernel<<<n_req, threads, smem, stream>>>(parents, reqs, single_n, bits, depths, W, status);
-  return cudaGetLastError();
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(unsigned(n_req));
+  cfg.blockDim = dim3(unsigned(threads));
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, build_tree_mask_kernel, parents, reqs, single_n, bits, depths, W, status);
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace dyspec
