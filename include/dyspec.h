@@ -117,10 +117,11 @@ int dyspec_schedule_dry_run(int n_q_heads, int n_kv_heads, int head_dim, int n_r
                             int32_t* cta_begin_out, int max_ctas, int64_t* info_out);
 
 /* Testing knobs, read when a plan is created: force the regime (-1 = automatic), the number of
- * CTAs the scheduler balances over (<= 0 = automatic), and how split-KV partials are merged: 0 = by
+ * CTAs the scheduler balances over (0 = automatic; a negative value -c instead sets the scheduler's
+ * per-item cost to c key tiles), and how split-KV partials are merged: 0 = by
  * the separate combine kernel, 2 (default) = inside a thread-block cluster through distributed shared
  * memory when the plan is uniform enough, else as 0. */
-int dyspec_set_tuning(int force_regime, int force_ctas, int fuse_combine);
+int dyspec_set_tuning(int force_regime, int force_ctas, int combine_mode);
 
 /* Developer aid: event trace of the attention kernels.  trace_buffer is a dev uint64 array of
  * capacity_entries entries that the caller zeroes; while set, CTA 0 of every tensor-core attention

@@ -89,8 +89,8 @@ def dyspec_words_per_row(max_nodes: int) -> int:
     return lib.dyspec_words_per_row(max_nodes)
 
 
-def dyspec_set_tuning(force_regime: int = -1, force_ctas: int = 0, fuse_combine: int = 2) -> None:
-    _check(lib.dyspec_set_tuning(force_regime, force_ctas, fuse_combine), "dyspec_set_tuning")
+def dyspec_set_tuning(force_regime: int = -1, force_ctas: int = 0, combine_mode: int = 2) -> None:
+    _check(lib.dyspec_set_tuning(force_regime, force_ctas, combine_mode), "dyspec_set_tuning")
 
 
 def dyspec_set_trace(trace_buffer=None, capacity_entries: int = 0) -> None:

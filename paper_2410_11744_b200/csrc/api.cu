@@ -29,7 +29,7 @@ namespace {
 int g_force_regime = -1;
 int g_force_ctas = 0;
 int g_item_cost = 0;       // scheduler experiment knob (0 = default)
-int g_fuse_combine = 2;   // 0 separate combine kernel, 2 cluster merge when the plan allows, else as 0
+int g_combine_mode = 2;   // 0 separate combine kernel, 2 cluster merge when the plan allows, else as 0
 unsigned long long* g_trace = nullptr;   // device buffer for the optional kernel event trace
 int g_trace_capacity = 0;
 
@@ -80,7 +80,6 @@ struct dyspec_plan {
   std::vector<WorkItem> items;          // compact list, CTA by CTA
   std::vector<WorkItem> items_strided;  // device layout: CTA c's items at [c * items_stride, ...)
   int items_stride = 1;
-  int fuse_combine = 1;
   int cluster = 1;                      // > 1: one thread-block cluster of this size per split group
   std::vector<int32_t> cta_begin;
   std::vector<GroupInfo> split_groups;
@@ -90,7 +89,6 @@ struct dyspec_plan {
   void* d_blob = nullptr;
   ReqInfo* d_reqs = nullptr;
   WorkItem* d_items = nullptr;
-  int32_t* d_cta_begin = nullptr;
   GroupInfo* d_groups = nullptr;
   int32_t* d_counters = nullptr;
   size_t workspace_bytes = 0;
@@ -132,14 +130,13 @@ void schedule(dyspec_plan& pl) {
   pl.max_splits = 1;
   pl.items_strided.clear();
   pl.items_stride = 1;
-  pl.fuse_combine = g_fuse_combine;
   if (groups.empty()) { pl.n_ctas = 0; pl.cta_begin.push_back(0); return; }
 
   // Cluster mode (warp-level regime): when every group can be cut into the same number C of pieces
   // and all pieces fit in one wave, launch one cluster of C CTAs per group; the pieces are merged
   // through distributed shared memory instead of a round trip through global memory.
   pl.cluster = 1;
-  if (pl.regime == 0 && g_fuse_combine == 2 && g_force_ctas <= 0) {
+  if (pl.regime == 0 && g_combine_mode == 2 && g_force_ctas <= 0) {
     int max_tiles = 0;
     for (const Group& gr : groups) max_tiles = std::max(max_tiles, gr.tiles);
     const double mean_tiles = double(total_tiles) / double(groups.size());
@@ -259,18 +256,15 @@ int upload(dyspec_plan& pl) {
   auto pad = [](size_t x) { return (x + 255) & ~size_t(255); };
   const size_t b_reqs = pad(std::max<size_t>(1, pl.reqs.size()) * sizeof(ReqInfo));
   const size_t b_items = pad(std::max<size_t>(1, pl.items_strided.size()) * sizeof(WorkItem));
-  const size_t b_cta = pad(pl.cta_begin.size() * sizeof(int32_t));
   const size_t b_groups = pad(std::max<size_t>(1, pl.split_groups.size()) * sizeof(GroupInfo));
   const size_t b_counters = pad(std::max<size_t>(1, pl.split_groups.size()) * sizeof(int32_t));
-  const size_t total = b_reqs + b_items + b_cta + b_groups + b_counters;
+  const size_t total = b_reqs + b_items + b_groups + b_counters;
   std::vector<uint8_t> host(total, 0);
   size_t off = 0;
   if (!pl.reqs.empty()) memcpy(host.data() + off, pl.reqs.data(), pl.reqs.size() * sizeof(ReqInfo));
   const size_t o_reqs = off; off += b_reqs;
   if (!pl.items_strided.empty()) memcpy(host.data() + off, pl.items_strided.data(), pl.items_strided.size() * sizeof(WorkItem));
   const size_t o_items = off; off += b_items;
-  memcpy(host.data() + off, pl.cta_begin.data(), pl.cta_begin.size() * sizeof(int32_t));
-  const size_t o_cta = off; off += b_cta;
   if (!pl.split_groups.empty()) memcpy(host.data() + off, pl.split_groups.data(), pl.split_groups.size() * sizeof(GroupInfo));
   const size_t o_groups = off; off += b_groups;
   const size_t o_counters = off;
@@ -279,7 +273,6 @@ int upload(dyspec_plan& pl) {
   uint8_t* base = static_cast<uint8_t*>(pl.d_blob);
   pl.d_reqs = reinterpret_cast<ReqInfo*>(base + o_reqs);
   pl.d_items = reinterpret_cast<WorkItem*>(base + o_items);
-  pl.d_cta_begin = reinterpret_cast<int32_t*>(base + o_cta);
   pl.d_groups = reinterpret_cast<GroupInfo*>(base + o_groups);
   pl.d_counters = reinterpret_cast<int32_t*>(base + o_counters);
   return DYSPEC_OK;
@@ -310,12 +303,12 @@ int dyspec_words_per_row(int max_nodes) {
   return 4 * ((max_nodes + 127) / 128);
 }
 
-int dyspec_set_tuning(int force_regime, int force_ctas, int fuse_combine) {
-  if (force_regime < -1 || force_regime > 1 || (fuse_combine != 0 && fuse_combine != 2)) return DYSPEC_ERR_INVALID_ARG;
+int dyspec_set_tuning(int force_regime, int force_ctas, int combine_mode) {
+  if (force_regime < -1 || force_regime > 1 || (combine_mode != 0 && combine_mode != 2)) return DYSPEC_ERR_INVALID_ARG;
   g_force_regime = force_regime;
   g_force_ctas = force_ctas >= 0 ? force_ctas : 0;
   g_item_cost = force_ctas < 0 ? -force_ctas : 0;   // negative values select the per-item cost instead (experiments)
-  g_fuse_combine = fuse_combine;
+  g_combine_mode = combine_mode;
   return DYSPEC_OK;
 }
 
@@ -489,14 +482,13 @@ int dyspec_tree_attention_ragged(const dyspec_plan_t* plan, const void* q, const
     return DYSPEC_ERR_CUDA;
 
   AttnParams p{};
-  p.reqs = plan->d_reqs; p.items = plan->d_items; p.cta_item_begin = plan->d_cta_begin; p.groups = plan->d_groups;
+  p.reqs = plan->d_reqs; p.items = plan->d_items; p.groups = plan->d_groups;
   p.bits = ancestor_bits; p.out = static_cast<__nv_bfloat16*>(out); p.partial = static_cast<float*>(workspace);
   p.counters = plan->d_counters; p.status = status;
   p.n_q_heads = plan->hq; p.n_kv_heads = plan->hkv; p.group_size = plan->g; p.log2_g = plan->log2g;
   p.words_per_row = plan->W; p.slot_floats = bm * (plan->d + 2);
   p.scale_log2e = plan->scale * kLog2e;
   p.items_stride = plan->items_stride;
-  p.fuse_combine = 0;
   p.cluster_size = plan->cluster;
   p.trace = g_trace; p.trace_capacity = g_trace_capacity;
 
@@ -504,7 +496,7 @@ int dyspec_tree_attention_ragged(const dyspec_plan_t* plan, const void* q, const
   if (plan->regime == 0) e = launch_attn_mma(plan->d, plan->n_ctas, mq, mk, mv, p, st);
   else e = launch_attn_tc(plan->d, plan->n_ctas, mq, mk, mv, p, st);
   if (e != cudaSuccess) return DYSPEC_ERR_CUDA;
-  if (!p.fuse_combine) e = launch_combine(plan->d, bm, int(plan->split_groups.size()), p, st);
+  e = launch_combine(plan->d, bm, int(plan->split_groups.size()), p, st);
   return e == cudaSuccess ? DYSPEC_OK : DYSPEC_ERR_CUDA;
 }
 
@@ -604,12 +596,11 @@ extern "C" int dyspec_tree_attention_static(const void* q, const void* k_cache, 
   if (!aligned(q, 16) || !aligned(k_cache, 16) || !aligned(v_cache, 16) || !aligned(out, 16) || !aligned(ancestor_bits, 16))
     return DYSPEC_ERR_INVALID_ARG;
 
-  // layout inside the scratch array: [requests | work items | per-CTA ranges | split groups | counters | partials]
+  // layout inside the scratch array: [requests | work items | split groups | counters | partials]
   auto pad = [](size_t x) { return (x + 255) & ~size_t(255); };
   const size_t o_reqs = 0;
   const size_t o_items = o_reqs + pad(pl->reqs.size() * sizeof(ReqInfo));
-  const size_t o_cta = o_items + pad(pl->items_strided.size() * sizeof(WorkItem));
-  const size_t o_groups = o_cta + pad(pl->cta_begin.size() * sizeof(int32_t));
+  const size_t o_groups = o_items + pad(pl->items_strided.size() * sizeof(WorkItem));
   const size_t o_counters = o_groups + pad(std::max<size_t>(1, pl->split_groups.size()) * sizeof(GroupInfo));
   const size_t o_partial = o_counters + pad(std::max<size_t>(1, pl->split_groups.size()) * sizeof(int32_t));
   const size_t total = o_partial + pl->workspace_bytes;
@@ -624,7 +615,6 @@ extern "C" int dyspec_tree_attention_static(const void* q, const void* k_cache, 
   std::vector<uint8_t> host(o_partial, 0);
   memcpy(host.data() + o_reqs, pl->reqs.data(), pl->reqs.size() * sizeof(ReqInfo));
   memcpy(host.data() + o_items, pl->items_strided.data(), pl->items_strided.size() * sizeof(WorkItem));
-  memcpy(host.data() + o_cta, pl->cta_begin.data(), pl->cta_begin.size() * sizeof(int32_t));
   if (!pl->split_groups.empty())
     memcpy(host.data() + o_groups, pl->split_groups.data(), pl->split_groups.size() * sizeof(GroupInfo));
   // pageable source: the copy is staged before the call returns, so `host` may go out of scope afterwards
@@ -641,7 +631,6 @@ extern "C" int dyspec_tree_attention_static(const void* q, const void* k_cache, 
   AttnParams p{};
   p.reqs = reinterpret_cast<const ReqInfo*>(base + o_reqs);
   p.items = reinterpret_cast<const WorkItem*>(base + o_items);
-  p.cta_item_begin = reinterpret_cast<const int32_t*>(base + o_cta);
   p.groups = reinterpret_cast<const GroupInfo*>(base + o_groups);
   p.counters = reinterpret_cast<int32_t*>(base + o_counters);
   p.partial = reinterpret_cast<float*>(base + o_partial);
@@ -650,13 +639,12 @@ extern "C" int dyspec_tree_attention_static(const void* q, const void* k_cache, 
   p.words_per_row = pl->W; p.slot_floats = bm * (pl->d + 2);
   p.scale_log2e = pl->scale * kLog2e;
   p.items_stride = pl->items_stride;
-  p.fuse_combine = 0;
   p.cluster_size = pl->cluster;
 
   cudaError_t e;
   if (pl->regime == 0) e = launch_attn_mma(pl->d, pl->n_ctas, mq, mk, mv, p, st);
   else e = launch_attn_tc(pl->d, pl->n_ctas, mq, mk, mv, p, st);
   if (e != cudaSuccess) return DYSPEC_ERR_CUDA;
-  if (!p.fuse_combine) e = launch_combine(pl->d, bm, int(pl->split_groups.size()), p, st);
+  e = launch_combine(pl->d, bm, int(pl->split_groups.size()), p, st);
   return e == cudaSuccess ? DYSPEC_OK : DYSPEC_ERR_CUDA;
 }

@@ -62,7 +62,6 @@ struct GroupInfo {
 struct AttnParams {
   const ReqInfo* reqs;
   const WorkItem* items;           // [n_ctas * items_stride]
-  const int32_t* cta_item_begin;   // [n_ctas + 1] (host-side view of the same assignment; unused by the kernels)
   const GroupInfo* groups;         // split groups only
   const uint32_t* bits;            // ancestor bitmasks [sum n][W]
   __nv_bfloat16* out;              // [sum n][H_q][D]
@@ -77,7 +76,6 @@ struct AttnParams {
   int32_t slot_floats;             // BM * (D + 2)
   float scale_log2e;               // scale * log2(e)
   int32_t items_stride;            // items per CTA slot in `items`
-  int32_t fuse_combine;            // reserved (0)
   int32_t cluster_size;            // > 1: one cluster per split group; partials are merged through distributed shared memory
   unsigned long long* trace;       // optional event trace (null in normal use): [0] = count, then entries
   int32_t trace_capacity;
