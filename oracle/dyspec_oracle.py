@@ -24,11 +24,15 @@ What it computes (every function names the passage of the paper it follows):
 Parity status: every function below is pinned by tests/test_oracle_pins.py
 (chain == library causal attention, star == prefix+self, brute force per path
 in pure Python, closed forms, hand-written mask fixture, relabelling
-invariance).  Nothing here is "parity unpinned".
+invariance); the token-reorder functions at the end (App. C) are pinned by
+tests/test_reorder_pins.py (the block counts the paper prints in Table 5,
+closed forms, a hand example, subtree contiguity, attention invariance).
+Nothing here is "parity unpinned".
 
 Readings where the paper is silent: scale = 1/sqrt(head_dim); consecutive query
 heads share a KV head; tree K/V rows follow the prefix rows in node order;
-masks are packed LSB-first in uint32 words.
+masks are packed LSB-first in uint32 words; the DFS renumbering visits roots
+and children in increasing index (the order that reproduces Table 5).
 """
 from __future__ import annotations
 
@@ -192,3 +196,66 @@ def visible_pair_count(prefix_len, parents_list) -> int:
         for i in range(len(p)):
             total += int(L) + len(visible_nodes(p, i))
     return total
+
+
+# ----------------------------------------------------------------------------------------------------
+# Block-sparsity friendly token order (App. C): depth-first renumbering and the non-zero block count.
+# ----------------------------------------------------------------------------------------------------
+def dfs_order(parents: Sequence[int]) -> List[int]:
+    """Depth-first (pre-order) visiting sequence of the forest: order[k] = old index of the node that
+    gets new index k.  Roots, and the children of a node, are visited in increasing old index (App. C:
+    DySpec renumbers nodes in DFS order because it approximates heavy-path order)."""
+    check_parents(parents)
+    n = len(parents)
+    children: List[List[int]] = [[] for _ in range(n)]
+    roots: List[int] = []
+    for i in range(n):
+        p = int(parents[i])
+        if p < 0:
+            roots.append(i)
+        else:
+            children[p].append(i)
+    order: List[int] = []
+
+    def visit(u: int) -> None:
+        order.append(u)
+        for c in children[u]:
+            visit(c)
+
+    import sys
+    limit = sys.getrecursionlimit()
+    sys.setrecursionlimit(max(limit, n + 100))
+    try:
+        for r in roots:
+            visit(r)
+    finally:
+        sys.setrecursionlimit(limit)
+    return order
+
+
+def relabel_tree(parents: Sequence[int], order: Sequence[int]):
+    """Parent array after renumbering: new node k is old node order[k].  Returns (new_parents int32 [n],
+    new_of_old int32 [n]).  For a DFS order the result again satisfies new_parents[k] < k."""
+    n = len(parents)
+    new_of_old = np.full(n, -1, dtype=np.int32)
+    for k, old in enumerate(order):
+        new_of_old[int(old)] = k
+    new_parents = np.full(n, -1, dtype=np.int32)
+    for k, old in enumerate(order):
+        p = int(parents[int(old)])
+        new_parents[k] = -1 if p < 0 else int(new_of_old[p])
+    return new_parents, new_of_old
+
+
+def mask_block_count(parents: Sequence[int], block: int = 32) -> int:
+    """Number of block x block tiles of the tree attention mask (ancestors and self) that hold at
+    least one visible entry: the workload measure of App. C.1, Table 5."""
+    m = tree_mask_matrix(parents)
+    n = m.shape[0]
+    t = (n + block - 1) // block
+    count = 0
+    for a in range(t):
+        for b in range(t):
+            if m[a * block:(a + 1) * block, b * block:(b + 1) * block].any():
+                count += 1
+    return count
