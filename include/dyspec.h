@@ -19,6 +19,14 @@
  *     wait that ran out) store a non-zero DYSPEC_ERR_* code into the optional `status` word (dev
  *     int32, the caller zeroes it) and the kernel still completes normally.
  *   - bf16 tensors are passed as `const void*`; layouts are row-major with the last index fastest.
+ *   - Stream order.  Kernels are launched with programmatic stream serialisation: a kernel may start
+ *     while the kernel before it in the stream is finishing, and it reads its pure inputs (parents,
+ *     q, k_cache, v_cache) before it waits for that kernel; everything it writes, and the mask it
+ *     reads, it touches only after the wait.  Inputs written by ordinary kernels or copies earlier in
+ *     the stream are safe (without an early-launch signal the stream serialises fully, as always),
+ *     and so is every sequence of this library's own calls.  The one thing to avoid is producing
+ *     those inputs with a foreign kernel that itself signals early launch of its dependents
+ *     (griddepcontrol.launch_dependents) directly before a call of this library.
  *
  * Packed rows: ancestor_bits[i][w], w < words_per_row, has bit b (LSB = bit 0) set iff tree node
  * 32*w + b is node i itself or an ancestor of node i (Sec. 2, the mask(A) equation, plus the self
@@ -46,7 +54,8 @@ enum {
   DYSPEC_ERR_TIMEOUT = -6      /* device-detected: a bounded in-kernel wait ran out */
 };
 
-#define DYSPEC_MAX_NODES 1024 /* largest tree per request (the paper's largest real tree is 768, Sec. 5 / App. B) */
+#define DYSPEC_MAX_NODES 2048 /* largest tree per request (the paper's largest real tree is 768, Sec. 5 / App. B;
+                                 its random-tree experiment goes up to 2048, App. C.1, Table 5) */
 
 /* Static, never-freed description of an error code. */
 const char* dyspec_error_string(int code);
@@ -84,7 +93,8 @@ int dyspec_build_tree_mask(const int32_t* parents, int n_nodes, uint32_t* ancest
  *                                     occupies rows off_r .. off_r + L_r + n_r - 1: prefix rows first,
  *                                     then one row per tree node in node order
  *   kv_total_rows          number of rows of k_cache / v_cache (>= every off_r + L_r + n_r)
- *   words_per_row          row stride of ancestor_bits, a multiple of 4 with 32*W >= max n_r
+ *   words_per_row          row stride of ancestor_bits, a multiple of 4 with 32*W >= max n_r and
+ *                          W <= DYSPEC_MAX_NODES / 32
  *   scale                  softmax scale; <= 0 selects 1/sqrt(head_dim)
  * Query/output rows of request r start at node_offset_r = n_0 + ... + n_{r-1}; so do its mask rows
  * and parents.
@@ -200,6 +210,51 @@ int dyspec_tree_attention(const void* q, const void* k_cache, const void* v_cach
 int dyspec_tree_attention_static(const void* q, const void* k_cache, const void* v_cache, int prefix_len,
                                  const uint32_t* ancestor_bits, int n_nodes, void* out, int n_q_heads, int n_kv_heads,
                                  int head_dim, int words_per_row, float scale, int32_t* status, dyspec_stream_t stream);
+
+/*
+ * (4) Block-sparsity friendly token order (App. C; Table 5).  The paper renumbers the tree tokens in
+ * depth-first order (an approximation of heavy-path order) so that the tree part of the attention
+ * mask touches few b x b blocks, and lets the attention kernel skip the empty blocks.
+ *
+ * dyspec_dfs_reorder / dyspec_plan_dfs_reorder: pre-order numbering that visits roots, and the
+ * children of every node, in increasing old index.
+ *   parents      dev int32 [n]          as for the mask builder (ragged form: all requests, node order)
+ *   order        dev int32 [n] or NULL  (written) order[k] = old index of the node whose new index is k
+ *   new_of_old   dev int32 [n] or NULL  (written) inverse permutation
+ *   new_parents  dev int32 [n] or NULL  (written) parent array in the new numbering; again
+ *                                        new_parents[k] < k.  Must not alias parents.
+ *   status       dev int32 [1] or NULL  DYSPEC_ERR_BAD_TREE on a bad parent (node treated as a root)
+ * Indices are local to the request; request r's entries start at node_offset_r in every array.
+ * The caller feeds the tree tokens to the model in the new order (token k = old token order[k]), so
+ * Q rows and tree K/V rows arrive in that order, and builds the mask from new_parents.
+ *
+ * dyspec_build_tree_mask_tiles / dyspec_plan_build_tree_mask_tiles: the mask builder, which also
+ * writes for every node which 64-column tiles of the tree its row touches:
+ *   node_tiles   dev uint32 [n]  (written) bit t set iff the node or one of its ancestors has an
+ *                                 index in [64 t, 64 t + 64)
+ * dyspec_tree_attention_ragged_sparse: dyspec_tree_attention_ragged that skips the tree key tiles no
+ * row of a query tile touches (node_tiles must come from the same parents as ancestor_bits; NULL
+ * gives dyspec_tree_attention_ragged).  Results are those of the dense call up to the order of the
+ * fp32 additions.  Only the tcgen05 regime skips tiles; the small-tree regime, whose tree part is one
+ * or two key tiles, ignores node_tiles.
+ */
+int dyspec_dfs_reorder(const int32_t* parents, int n_nodes, int32_t* order, int32_t* new_of_old, int32_t* new_parents,
+                       int32_t* status, dyspec_stream_t stream);
+int dyspec_plan_dfs_reorder(const dyspec_plan_t* plan, const int32_t* parents, int32_t* order, int32_t* new_of_old,
+                            int32_t* new_parents, int32_t* status, dyspec_stream_t stream);
+int dyspec_build_tree_mask_tiles(const int32_t* parents, int n_nodes, uint32_t* ancestor_bits, int32_t* depths,
+                                 uint32_t* node_tiles, int words_per_row, int32_t* status, dyspec_stream_t stream);
+int dyspec_plan_build_tree_mask_tiles(const dyspec_plan_t* plan, const int32_t* parents, uint32_t* ancestor_bits,
+                                      int32_t* depths, uint32_t* node_tiles, int32_t* status, dyspec_stream_t stream);
+/* The paper's workload measure for this optimisation (App. C.1, Table 5, "Block Count"): the number of
+ * block x block tiles of one request's packed mask that hold a visible pair.  block = 32, 64 or 128;
+ * count: dev uint64 [1] (written; cleared first, on `stream`). */
+int dyspec_mask_block_count(const uint32_t* ancestor_bits, int n_nodes, int words_per_row, int block, uint64_t* count,
+                            dyspec_stream_t stream);
+int dyspec_tree_attention_ragged_sparse(const dyspec_plan_t* plan, const void* q, const void* k_cache,
+                                        const void* v_cache, const uint32_t* ancestor_bits, const uint32_t* node_tiles,
+                                        void* out, void* workspace, size_t workspace_bytes, int32_t* status,
+                                        dyspec_stream_t stream);
 
 #ifdef __cplusplus
 }

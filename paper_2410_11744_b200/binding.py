@@ -41,6 +41,12 @@ SIGNATURES = {
     "dyspec_tree_attention_ragged": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp, _vp]),
     "dyspec_set_default_shape": (_i32, [_i32, _i32, _i32, _i32, _f32]),
     "dyspec_tree_attention": (_i32, [_vp, _vp, _vp, _i32, _vp, _i32, _vp, _vp]),
+    "dyspec_dfs_reorder": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _vp]),
+    "dyspec_plan_dfs_reorder": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "dyspec_build_tree_mask_tiles": (_i32, [_vp, _i32, _vp, _vp, _vp, _i32, _vp, _vp]),
+    "dyspec_plan_build_tree_mask_tiles": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "dyspec_mask_block_count": (_i32, [_vp, _i32, _i32, _i32, _vp, _vp]),
+    "dyspec_tree_attention_ragged_sparse": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp, _vp]),
     "dyspec_tree_attention_static": (_i32, [_vp, _vp, _vp, _i32, _vp, _i32, _vp, _i32, _i32, _i32, _i32, _f32, _vp, _vp]),
 }
 for _name, (_res, _args) in SIGNATURES.items():
@@ -218,3 +224,46 @@ def dyspec_tree_attention_static(q, k_cache, v_cache, prefix_len: int, ancestor_
                                             n_nodes, _ptr(out), n_q_heads, n_kv_heads, head_dim, words_per_row,
                                             float(scale), _ptr(status), _stream(stream)),
            "dyspec_tree_attention_static")
+
+
+def dyspec_dfs_reorder(parents, n_nodes: int, order=None, new_of_old=None, new_parents=None, status=None,
+                       stream=None) -> None:
+    """Depth-first renumbering of one tree; all arrays are int32 device tensors [n] (outputs may be None)."""
+    _check(lib.dyspec_dfs_reorder(_ptr(parents), n_nodes, _ptr(order), _ptr(new_of_old), _ptr(new_parents),
+                                  _ptr(status), _stream(stream)), "dyspec_dfs_reorder")
+
+
+def dyspec_plan_dfs_reorder(plan: Plan, parents, order=None, new_of_old=None, new_parents=None, status=None,
+                            stream=None) -> None:
+    _check(lib.dyspec_plan_dfs_reorder(plan.handle, _ptr(parents), _ptr(order), _ptr(new_of_old), _ptr(new_parents),
+                                       _ptr(status), _stream(stream)), "dyspec_plan_dfs_reorder")
+
+
+def dyspec_build_tree_mask_tiles(parents, n_nodes: int, ancestor_bits, depths, node_tiles, words_per_row: int,
+                                 status=None, stream=None) -> None:
+    _check(lib.dyspec_build_tree_mask_tiles(_ptr(parents), n_nodes, _ptr(ancestor_bits), _ptr(depths), _ptr(node_tiles),
+                                            words_per_row, _ptr(status), _stream(stream)),
+           "dyspec_build_tree_mask_tiles")
+
+
+def dyspec_plan_build_tree_mask_tiles(plan: Plan, parents, ancestor_bits, depths, node_tiles, status=None,
+                                      stream=None) -> None:
+    _check(lib.dyspec_plan_build_tree_mask_tiles(plan.handle, _ptr(parents), _ptr(ancestor_bits), _ptr(depths),
+                                                 _ptr(node_tiles), _ptr(status), _stream(stream)),
+           "dyspec_plan_build_tree_mask_tiles")
+
+
+def dyspec_mask_block_count(ancestor_bits, n_nodes: int, words_per_row: int, block: int, count, stream=None) -> None:
+    """count: int64 device tensor [1] (written)."""
+    _check(lib.dyspec_mask_block_count(_ptr(ancestor_bits), n_nodes, words_per_row, block, _ptr(count),
+                                       _stream(stream)), "dyspec_mask_block_count")
+
+
+def dyspec_tree_attention_ragged_sparse(plan: Plan, q, k_cache, v_cache, ancestor_bits, node_tiles, out, workspace=None,
+                                        workspace_bytes: Optional[int] = None, status=None, stream=None) -> None:
+    if workspace_bytes is None:
+        workspace_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(lib.dyspec_tree_attention_ragged_sparse(plan.handle, _ptr(q), _ptr(k_cache), _ptr(v_cache),
+                                                   _ptr(ancestor_bits), _ptr(node_tiles), _ptr(out), _ptr(workspace),
+                                                   workspace_bytes, _ptr(status), _stream(stream)),
+           "dyspec_tree_attention_ragged_sparse")

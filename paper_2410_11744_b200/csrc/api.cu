@@ -14,7 +14,13 @@
 namespace dyspec {
 // kernels (defined in the other translation units)
 cudaError_t launch_build_tree_mask(const int32_t* parents, const ReqInfo* reqs, int n_req, int single_n, int max_n,
-                                   uint32_t* bits, int32_t* depths, int W, int32_t* status, cudaStream_t stream);
+                                   uint32_t* bits, int32_t* depths, uint32_t* node_tiles, int W, int32_t* status,
+                                   cudaStream_t stream);
+cudaError_t launch_dfs_reorder(const int32_t* parents, const ReqInfo* reqs, int n_req, int single_n, int max_n,
+                               int32_t* order, int32_t* new_of_old, int32_t* new_parents, int32_t* status,
+                               cudaStream_t stream);
+cudaError_t launch_mask_block_count(const uint32_t* bits, int n, int W, int block, unsigned long long* count,
+                                    cudaStream_t stream);
 cudaError_t launch_attn_mma(int head_dim, int n_ctas, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                             const AttnParams& p, cudaStream_t stream);
 cudaError_t launch_combine(int head_dim, int bm, int n_split_groups, const AttnParams& p, cudaStream_t stream);
@@ -319,16 +325,51 @@ int dyspec_set_trace(void* trace_buffer, int capacity_entries) {
   return DYSPEC_OK;
 }
 
-int dyspec_build_tree_mask(const int32_t* parents, int n_nodes, uint32_t* ancestor_bits, int32_t* depths,
-                           int words_per_row, int32_t* status, dyspec_stream_t stream) {
+static int build_tree_mask_checked(const int32_t* parents, int n_nodes, uint32_t* ancestor_bits, int32_t* depths,
+                                   uint32_t* node_tiles, int words_per_row, int32_t* status, dyspec_stream_t stream) {
   if (n_nodes < 0 || words_per_row <= 0 || (words_per_row & 3)) return DYSPEC_ERR_INVALID_ARG;
-  if (n_nodes > DYSPEC_MAX_NODES) return DYSPEC_ERR_UNSUPPORTED;
+  if (n_nodes > DYSPEC_MAX_NODES || words_per_row > DYSPEC_MAX_NODES / 32) return DYSPEC_ERR_UNSUPPORTED;
   if (32 * words_per_row < n_nodes) return DYSPEC_ERR_INVALID_ARG;
   if (n_nodes == 0) return DYSPEC_OK;
   if (!parents || !ancestor_bits) return DYSPEC_ERR_INVALID_ARG;
-  if (!aligned(ancestor_bits, 16) || !aligned(parents, 4)) return DYSPEC_ERR_INVALID_ARG;
-  cudaError_t e = launch_build_tree_mask(parents, nullptr, 1, n_nodes, n_nodes, ancestor_bits, depths, words_per_row, status,
-                                         reinterpret_cast<cudaStream_t>(stream));
+  if (!aligned(ancestor_bits, 16) || !aligned(parents, 4) || !aligned(node_tiles, 4)) return DYSPEC_ERR_INVALID_ARG;
+  cudaError_t e = launch_build_tree_mask(parents, nullptr, 1, n_nodes, n_nodes, ancestor_bits, depths, node_tiles,
+                                         words_per_row, status, reinterpret_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? DYSPEC_OK : DYSPEC_ERR_CUDA;
+}
+
+int dyspec_build_tree_mask(const int32_t* parents, int n_nodes, uint32_t* ancestor_bits, int32_t* depths,
+                           int words_per_row, int32_t* status, dyspec_stream_t stream) {
+  return build_tree_mask_checked(parents, n_nodes, ancestor_bits, depths, nullptr, words_per_row, status, stream);
+}
+
+int dyspec_build_tree_mask_tiles(const int32_t* parents, int n_nodes, uint32_t* ancestor_bits, int32_t* depths,
+                                 uint32_t* node_tiles, int words_per_row, int32_t* status, dyspec_stream_t stream) {
+  if (n_nodes > 0 && !node_tiles) return DYSPEC_ERR_INVALID_ARG;
+  return build_tree_mask_checked(parents, n_nodes, ancestor_bits, depths, node_tiles, words_per_row, status, stream);
+}
+
+int dyspec_dfs_reorder(const int32_t* parents, int n_nodes, int32_t* order, int32_t* new_of_old, int32_t* new_parents,
+                       int32_t* status, dyspec_stream_t stream) {
+  if (n_nodes < 0) return DYSPEC_ERR_INVALID_ARG;
+  if (n_nodes > DYSPEC_MAX_NODES) return DYSPEC_ERR_UNSUPPORTED;
+  if (n_nodes == 0) return DYSPEC_OK;
+  if (!parents || !aligned(parents, 4) || !aligned(order, 4) || !aligned(new_of_old, 4) || !aligned(new_parents, 4))
+    return DYSPEC_ERR_INVALID_ARG;
+  if (new_parents == parents) return DYSPEC_ERR_INVALID_ARG;      // not in place: other requests' CTAs may still read
+  cudaError_t e = launch_dfs_reorder(parents, nullptr, 1, n_nodes, n_nodes, order, new_of_old, new_parents, status,
+                                     reinterpret_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? DYSPEC_OK : DYSPEC_ERR_CUDA;
+}
+
+int dyspec_mask_block_count(const uint32_t* ancestor_bits, int n_nodes, int words_per_row, int block, uint64_t* count,
+                            dyspec_stream_t stream) {
+  if (n_nodes < 0 || words_per_row <= 0 || (words_per_row & 3) || 32 * words_per_row < n_nodes) return DYSPEC_ERR_INVALID_ARG;
+  if (!(block == 32 || block == 64 || block == 128)) return DYSPEC_ERR_UNSUPPORTED;
+  if (n_nodes > DYSPEC_MAX_NODES) return DYSPEC_ERR_UNSUPPORTED;
+  if (!count || !aligned(count, 8) || (n_nodes > 0 && (!ancestor_bits || !aligned(ancestor_bits, 16)))) return DYSPEC_ERR_INVALID_ARG;
+  cudaError_t e = launch_mask_block_count(ancestor_bits, n_nodes, words_per_row, block,
+                                          reinterpret_cast<unsigned long long*>(count), reinterpret_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? DYSPEC_OK : DYSPEC_ERR_CUDA;
 }
 
@@ -340,6 +381,7 @@ static int make_host_plan(dyspec_plan** out, int n_q_heads, int n_kv_heads, int 
   if (n_q_heads <= 0 || n_kv_heads <= 0 || n_req < 0 || kv_total_rows < 0) return DYSPEC_ERR_INVALID_ARG;
   if (n_req > 0 && (!prefix_len || !n_nodes || !kv_row_offset)) return DYSPEC_ERR_INVALID_ARG;
   if (words_per_row <= 0 || (words_per_row & 3)) return DYSPEC_ERR_INVALID_ARG;
+  if (words_per_row > DYSPEC_MAX_NODES / 32) return DYSPEC_ERR_UNSUPPORTED;
   if (n_q_heads % n_kv_heads != 0) return DYSPEC_ERR_UNSUPPORTED;
   const int g = n_q_heads / n_kv_heads;
   if (!(g == 1 || g == 2 || g == 4 || g == 8)) return DYSPEC_ERR_UNSUPPORTED;
@@ -451,20 +493,52 @@ int64_t dyspec_plan_info(const dyspec_plan_t* plan, int field) {
   }
 }
 
-int dyspec_plan_build_tree_mask(const dyspec_plan_t* plan, const int32_t* parents, uint32_t* ancestor_bits,
-                                int32_t* depths, int32_t* status, dyspec_stream_t stream) {
+static int plan_build_tree_mask_checked(const dyspec_plan_t* plan, const int32_t* parents, uint32_t* ancestor_bits,
+                                        int32_t* depths, uint32_t* node_tiles, int32_t* status, dyspec_stream_t stream) {
   if (!plan) return DYSPEC_ERR_INVALID_ARG;
   if (plan->n_req == 0 || plan->total_nodes == 0) return DYSPEC_OK;
-  if (!parents || !ancestor_bits || !aligned(ancestor_bits, 16)) return DYSPEC_ERR_INVALID_ARG;
-  cudaError_t e = launch_build_tree_mask(parents, plan->d_reqs, plan->n_req, 0, plan->max_nodes, ancestor_bits, depths, plan->W, status,
-                                         reinterpret_cast<cudaStream_t>(stream));
+  if (!parents || !ancestor_bits || !aligned(ancestor_bits, 16) || !aligned(node_tiles, 4)) return DYSPEC_ERR_INVALID_ARG;
+  cudaError_t e = launch_build_tree_mask(parents, plan->d_reqs, plan->n_req, 0, plan->max_nodes, ancestor_bits, depths,
+                                         node_tiles, plan->W, status, reinterpret_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? DYSPEC_OK : DYSPEC_ERR_CUDA;
+}
+
+int dyspec_plan_build_tree_mask(const dyspec_plan_t* plan, const int32_t* parents, uint32_t* ancestor_bits,
+                                int32_t* depths, int32_t* status, dyspec_stream_t stream) {
+  return plan_build_tree_mask_checked(plan, parents, ancestor_bits, depths, nullptr, status, stream);
+}
+
+int dyspec_plan_build_tree_mask_tiles(const dyspec_plan_t* plan, const int32_t* parents, uint32_t* ancestor_bits,
+                                      int32_t* depths, uint32_t* node_tiles, int32_t* status, dyspec_stream_t stream) {
+  if (plan && plan->total_nodes > 0 && !node_tiles) return DYSPEC_ERR_INVALID_ARG;
+  return plan_build_tree_mask_checked(plan, parents, ancestor_bits, depths, node_tiles, status, stream);
+}
+
+int dyspec_plan_dfs_reorder(const dyspec_plan_t* plan, const int32_t* parents, int32_t* order, int32_t* new_of_old,
+                            int32_t* new_parents, int32_t* status, dyspec_stream_t stream) {
+  if (!plan) return DYSPEC_ERR_INVALID_ARG;
+  if (plan->n_req == 0 || plan->total_nodes == 0) return DYSPEC_OK;
+  if (!parents || !aligned(parents, 4) || !aligned(order, 4) || !aligned(new_of_old, 4) || !aligned(new_parents, 4))
+    return DYSPEC_ERR_INVALID_ARG;
+  if (new_parents == parents) return DYSPEC_ERR_INVALID_ARG;
+  cudaError_t e = launch_dfs_reorder(parents, plan->d_reqs, plan->n_req, 0, plan->max_nodes, order, new_of_old,
+                                     new_parents, status, reinterpret_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? DYSPEC_OK : DYSPEC_ERR_CUDA;
 }
 
 int dyspec_tree_attention_ragged(const dyspec_plan_t* plan, const void* q, const void* k_cache, const void* v_cache,
                                  const uint32_t* ancestor_bits, void* out, void* workspace, size_t workspace_bytes,
                                  int32_t* status, dyspec_stream_t stream) {
+  return dyspec_tree_attention_ragged_sparse(plan, q, k_cache, v_cache, ancestor_bits, nullptr, out, workspace,
+                                             workspace_bytes, status, stream);
+}
+
+int dyspec_tree_attention_ragged_sparse(const dyspec_plan_t* plan, const void* q, const void* k_cache,
+                                        const void* v_cache, const uint32_t* ancestor_bits, const uint32_t* node_tiles,
+                                        void* out, void* workspace, size_t workspace_bytes, int32_t* status,
+                                        dyspec_stream_t stream) {
   if (!plan) return DYSPEC_ERR_INVALID_ARG;
+  if (!aligned(node_tiles, 4)) return DYSPEC_ERR_INVALID_ARG;
   if (plan->n_ctas == 0) return DYSPEC_OK;
   if (!q || !k_cache || !v_cache || !ancestor_bits || !out) return DYSPEC_ERR_INVALID_ARG;
   if (!aligned(q, 16) || !aligned(k_cache, 16) || !aligned(v_cache, 16) || !aligned(out, 16) || !aligned(ancestor_bits, 16))
@@ -483,7 +557,8 @@ int dyspec_tree_attention_ragged(const dyspec_plan_t* plan, const void* q, const
 
   AttnParams p{};
   p.reqs = plan->d_reqs; p.items = plan->d_items; p.groups = plan->d_groups;
-  p.bits = ancestor_bits; p.out = static_cast<__nv_bfloat16*>(out); p.partial = static_cast<float*>(workspace);
+  p.bits = ancestor_bits; p.node_tiles = node_tiles; p.out = static_cast<__nv_bfloat16*>(out);
+  p.partial = static_cast<float*>(workspace);
   p.counters = plan->d_counters; p.status = status;
   p.n_q_heads = plan->hq; p.n_kv_heads = plan->hkv; p.group_size = plan->g; p.log2_g = plan->log2g;
   p.words_per_row = plan->W; p.slot_floats = bm * (plan->d + 2);

@@ -139,6 +139,45 @@ __device__ __forceinline__ void st_global_v8(void* ptr, const uint32_t* v) {
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
+// Which key tiles of an item's range are processed.  The prefix tiles always are; of the tree tiles
+// only those that some row of the query tile can see (App. C: empty blocks of the tree mask are
+// skipped), when the caller passed the per-node tile sets; all of them otherwise.  Every role of the
+// CTA derives the same walk from the same inputs.
+struct TileWalk {
+  int P;            // prefix tiles in the range: tiles tile_begin .. tile_begin + P - 1
+  int T;            // tiles processed in all
+  uint32_t need;    // tree tiles processed: bit u = tree columns [u * BN, (u + 1) * BN)
+};
+__device__ __forceinline__ TileWalk walk_dense(const WorkItem& item, int n_prefix_tiles) {
+  TileWalk wk;
+  wk.P = max(0, min(item.tile_end, n_prefix_tiles) - item.tile_begin);
+  const int u0 = max(item.tile_begin, n_prefix_tiles) - n_prefix_tiles, u1 = item.tile_end - n_prefix_tiles;
+  wk.need = u1 > u0 ? (((1u << u1) - 1u) & ~((1u << u0) - 1u)) : 0u;
+  wk.T = wk.P + __popc(wk.need);
+  return wk;
+}
+// Whole warp.  The mask kernel must have completed (grid_dependency_wait) before this reads node_tiles.
+__device__ __forceinline__ TileWalk walk_sparse(const AttnParams& p, const WorkItem& item, int n_prefix_tiles, int lane) {
+  TileWalk wk = walk_dense(item, n_prefix_tiles);
+  if (p.node_tiles == nullptr || wk.need == 0u) return wk;
+  const int node_lo = item.row0 >> p.log2_g;
+  const int node_hi = min(item.n_nodes, ((item.row0 + 2 * BMH - 1) >> p.log2_g) + 1);
+  uint32_t occ = 0u;
+  for (int node = node_lo + lane; node < node_hi; node += 32) occ |= __ldg(p.node_tiles + item.node0 + node);
+  occ = __reduce_or_sync(0xffffffffu, occ);
+  // node_tiles counts 64-column tiles; a key tile here is BN = 128 columns: OR the bit pairs together
+  uint32_t x = (occ | (occ >> 1)) & 0x55555555u;
+  x = (x | (x >> 1)) & 0x33333333u;
+  x = (x | (x >> 2)) & 0x0f0f0f0fu;
+  x = (x | (x >> 4)) & 0x00ff00ffu;
+  x = (x | (x >> 8)) & 0x0000ffffu;
+  const uint32_t first = wk.need & (0u - wk.need);
+  wk.need &= x;
+  if (wk.P == 0 && wk.need == 0u) wk.need = first;     // an item always runs at least one (fully masked) tile
+  wk.T = wk.P + __popc(wk.need);
+  return wk;
+}
+
 }  // namespace
 
 template <int D>
@@ -195,36 +234,58 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
-    if (lane == 0) {
-      prefetch_tensormap(&map_q);
-      prefetch_tensormap(&map_k);
-      prefetch_tensormap(&map_v);
+    // The whole warp walks the loop (the tile walk is a warp-wide computation); one lane issues.
+    {
+      const bool elected = lane == 0;
+      if (elected) {
+        prefetch_tensormap(&map_q);
+        prefetch_tensormap(&map_k);
+        prefetch_tensormap(&map_v);
+      }
       uint32_t sc = 0, qit = 0;
       for (int w = item_begin; w < item_end; ++w, ++qit) {
         const WorkItem item = my_items[w];
         const WorkItem& rq = item;
         const int nh = (rq.n_nodes * g - item.row0 > BMH) ? 2 : 1;
         mbar_wait(bar(B_QFREE), (qit & 1) ^ 1, abort_flag, p.status);
-        mbar_expect_tx(bar(B_QFULL), uint32_t(nh) * L::kTileBytes);
-        for (int h = 0; h < nh; ++h)
-          for (int pn = 0; pn < L::kPanels; ++pn)
-            tma_load_3d(s_q + h * L::kTileBytes + pn * L::kPanelBytes, &map_q, bar(B_QFULL), pn * 64, item.kv_head * g,
-                        rq.node0 + ((item.row0 + h * BMH) >> p.log2_g));
+        if (elected) {
+          mbar_expect_tx(bar(B_QFULL), uint32_t(nh) * L::kTileBytes);
+          for (int h = 0; h < nh; ++h)
+            for (int pn = 0; pn < L::kPanels; ++pn)
+              tma_load_3d(s_q + h * L::kTileBytes + pn * L::kPanelBytes, &map_q, bar(B_QFULL), pn * 64, item.kv_head * g,
+                          rq.node0 + ((item.row0 + h * BMH) >> p.log2_g));
+        }
         const int n_prefix_tiles = (rq.prefix_len + BN - 1) / BN;
-        for (int t = item.tile_begin; t < item.tile_end; ++t) {
+        // Prefix tiles stream at once; the set of tree tiles may depend on the mask kernel's output,
+        // so it is settled (after waiting for that kernel) only when the walk reaches the tree.
+        TileWalk wk = walk_dense(item, n_prefix_tiles);
+        bool exact = p.node_tiles == nullptr || wk.need == 0u;
+        uint32_t rem = wk.need;
+        for (int j = 0;; ++j) {
+          if (!exact && j >= wk.P) {
+            grid_dependency_wait();
+            wk = walk_sparse(p, item, n_prefix_tiles, lane);
+            rem = wk.need;
+            exact = true;
+          }
+          if (j >= wk.T) break;
+          int t = item.tile_begin + j;
+          if (j >= wk.P) {
+            t = n_prefix_tiles + __ffs(rem) - 1;
+            rem &= rem - 1u;
+          }
           const int64_t row = rq.kv_row0 + (t < n_prefix_tiles ? int64_t(t) * BN
                                                                : int64_t(rq.prefix_len) + int64_t(t - n_prefix_tiles) * BN);
           for (int kv = 0; kv < 2; ++kv, ++sc) {
             const int slot = sc % kSlots;
             const uint32_t ph = (sc / kSlots) & 1;
             mbar_wait(bar(B_SLOT_EMPTY + slot), ph ^ 1, abort_flag, p.status);
-#ifdef EXP_SKIP_LOADS
-            if (sc >= kSlots) { mbar_arrive(bar(B_SLOT_FULL + slot)); continue; }
-#endif
-            mbar_expect_tx(bar(B_SLOT_FULL + slot), L::kTileBytes);
-            for (int pn = 0; pn < L::kPanels; ++pn)
-              tma_load_3d(s_ring + slot * L::kTileBytes + pn * L::kPanelBytes, kv == 0 ? &map_k : &map_v,
-                          bar(B_SLOT_FULL + slot), pn * 64, item.kv_head, int(row));
+            if (elected) {
+              mbar_expect_tx(bar(B_SLOT_FULL + slot), L::kTileBytes);
+              for (int pn = 0; pn < L::kPanels; ++pn)
+                tma_load_3d(s_ring + slot * L::kTileBytes + pn * L::kPanelBytes, kv == 0 ? &map_k : &map_v,
+                            bar(B_SLOT_FULL + slot), pn * 64, item.kv_head, int(row));
+            }
           }
         }
       }
@@ -272,7 +333,22 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         const WorkItem item = my_items[w];
         const WorkItem& rq = item;
         const bool two = rq.n_nodes * g - item.row0 > BMH;        // both query halves live
-        const int T = item.tile_end - item.tile_begin;
+        // Number of tiles of the item.  With per-node tile sets it depends on the mask kernel's
+        // output; it is settled two tiles before the prefix part ends (until then "more tiles
+        // follow" is all this loop needs to know), so the prefix still overlaps that kernel.
+        const int n_prefix_tiles = (rq.prefix_len + BN - 1) / BN;
+        TileWalk wk = walk_dense(item, n_prefix_tiles);
+        bool exact = p.node_tiles == nullptr || wk.need == 0u;
+        int T = exact ? wk.T : 0x7fffffff;
+        auto settle = [&](int j) {
+          if (!exact && j + 2 >= wk.P) {
+            grid_dependency_wait();
+            wk = walk_sparse(p, item, n_prefix_tiles, lane);
+            T = wk.T;
+            exact = true;
+          }
+        };
+        settle(-1);
         mbar_wait(bar(B_QFULL), qit & 1, abort_flag, p.status);
         {
           const uint32_t kslot = sc % kSlots, kph = (sc / kSlots) & 1;
@@ -284,7 +360,9 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           if (elected) tc_commit(bar(B_SLOT_EMPTY + kslot));
           if (T == 1) if (elected) tc_commit(bar(B_QFREE));            // Q is reusable once the item's last QK^T has run
         }
-        for (int j = 0; j < T; ++j) {
+        for (int j = 0;; ++j) {
+          settle(j);
+          if (j >= T) break;
           const uint32_t vslot = sc % kSlots, vph = (sc / kSlots) & 1;
           ++sc;
           const bool more = j + 1 < T;
@@ -352,9 +430,11 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       const WorkItem& rq = item;
       const int n_rows = rq.n_nodes * g;
       const int nh = (n_rows - item.row0 > BMH) ? 2 : 1;
-      const int T = item.tile_end - item.tile_begin;
-      if (h >= nh) { sc += 2u * uint32_t(T); continue; }
       const int n_prefix_tiles = (rq.prefix_len + BN - 1) / BN;
+      const TileWalk wk = walk_sparse(p, item, n_prefix_tiles, lane);
+      const int T = wk.T;
+      if (h >= nh) { sc += 2u * uint32_t(T); continue; }
+      uint32_t rem = wk.need;
       const int row = item.row0 + h * BMH + r;
       const bool ok = row < n_rows;
       const int node = row >> p.log2_g;
@@ -362,7 +442,11 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
 
       float m_used = -INFINITY, l = 0.f;
       for (int j = 0; j < T; ++j) {
-        const int t = item.tile_begin + j;
+        int t = item.tile_begin + j;
+        if (j >= wk.P) {
+          t = n_prefix_tiles + __ffs(rem) - 1;
+          rem &= rem - 1u;
+        }
         const uint32_t vslot = sc + 1u;
         sc += 2u;
         // visibility of the 128 key columns of this tile for this row
@@ -391,12 +475,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         tc_fence_after();
         if (r == 0) trace_event(tc_cur, DYSPEC_TAG(1 + h, 1, j));
 
-#ifdef EXP_SKIP_SOFTMAX
-        if (j >= 0) { tc_fence_before(); mbar_arrive(bar(B_PREADY + h)); continue; }
-#endif
-#ifdef EXP_SKIP_SOFTMAX
-        if (j >= 0) { tc_fence_before(); mbar_arrive(bar(B_PREADY + h)); continue; }
-#endif
         // the whole S row (128 fp32) in registers: four loads in flight, one wait
         uint32_t sv[BN];
 #pragma unroll

@@ -64,6 +64,7 @@ struct AttnParams {
   const WorkItem* items;           // [n_ctas * items_stride]
   const GroupInfo* groups;         // split groups only
   const uint32_t* bits;            // ancestor bitmasks [sum n][W]
+  const uint32_t* node_tiles;      // optional [sum n]: bit t = the node's row touches tree columns [64 t, 64 t + 64)
   __nv_bfloat16* out;              // [sum n][H_q][D]
   float* partial;                  // split-KV partials: slot s at partial + s * slot_floats
   int32_t* counters;               // per-group arrival counters (zero between calls)

@@ -23,8 +23,9 @@ class DeviceBatch:
     """Buffers + plan for one Workload.  `step()` = mask build + attention (+ combine) on the current stream."""
 
     def __init__(self, w: Workload, device="cuda:0", words_per_row: int | None = None, upload: bool = True,
-                 plan: "B.Plan | None" = None):
+                 plan: "B.Plan | None" = None, sparse: bool = False):
         self.w = w
+        self.sparse = sparse            # also emit per-node tile sets and let the attention skip empty tree tiles
         self.device = torch.device(device)
         max_n = int(w.n_nodes.max()) if w.n_req else 0
         self.W = words_per_row or B.dyspec_words_per_row(max_n)
@@ -37,6 +38,7 @@ class DeviceBatch:
         n = max(1, self.total_nodes)
         self.bits = torch.zeros((n, self.W), dtype=torch.int32, device=dev)
         self.depths = torch.zeros((n,), dtype=torch.int32, device=dev)
+        self.node_tiles = torch.zeros((n,), dtype=torch.int32, device=dev) if sparse else None
         self.status = torch.zeros((1,), dtype=torch.int32, device=dev)
         self.out = torch.zeros((n, w.n_q_heads, w.head_dim), dtype=torch.bfloat16, device=dev)
         ws = self.plan.workspace_bytes()
@@ -54,11 +56,30 @@ class DeviceBatch:
         self.v = _bits_to_bf16(w.v if self.kv_total_rows else np.zeros(kv_shape, np.uint16), dev)
 
     def build_mask(self):
-        B.dyspec_plan_build_tree_mask(self.plan, self.parents, self.bits, self.depths, self.status)
+        if self.sparse:
+            B.dyspec_plan_build_tree_mask_tiles(self.plan, self.parents, self.bits, self.depths, self.node_tiles,
+                                                self.status)
+        else:
+            B.dyspec_plan_build_tree_mask(self.plan, self.parents, self.bits, self.depths, self.status)
 
     def attention(self):
-        B.dyspec_tree_attention_ragged(self.plan, self.q, self.k, self.v, self.bits, self.out, self.workspace,
-                                       self.workspace_bytes, self.status)
+        if self.sparse:
+            B.dyspec_tree_attention_ragged_sparse(self.plan, self.q, self.k, self.v, self.bits, self.node_tiles,
+                                                  self.out, self.workspace, self.workspace_bytes, self.status)
+        else:
+            B.dyspec_tree_attention_ragged(self.plan, self.q, self.k, self.v, self.bits, self.out, self.workspace,
+                                           self.workspace_bytes, self.status)
+
+    def dfs_reorder(self):
+        """Runs the reorder kernel on the batch's parents -> (order, new_of_old, new_parents) int32 numpy [sum n]."""
+        n = max(1, self.total_nodes)
+        order = torch.full((n,), -7, dtype=torch.int32, device=self.device)
+        new_of_old = torch.full((n,), -7, dtype=torch.int32, device=self.device)
+        new_parents = torch.full((n,), -7, dtype=torch.int32, device=self.device)
+        B.dyspec_plan_dfs_reorder(self.plan, self.parents, order, new_of_old, new_parents, self.status)
+        torch.cuda.synchronize(self.device)
+        m = self.total_nodes
+        return order[:m].cpu().numpy(), new_of_old[:m].cpu().numpy(), new_parents[:m].cpu().numpy()
 
     def step(self):
         self.build_mask()

@@ -183,3 +183,32 @@ def make_custom(seed: int, n_q_heads: int, n_kv_heads: int, head_dim: int, prefi
                 name: str = "custom") -> Workload:
     return assemble(name, np.random.default_rng(seed), n_q_heads, n_kv_heads, head_dim, prefix_len, parents_list,
                     dict(seed=seed))
+
+
+def make_random_tree_case(n_nodes: int, seed: int | None = None, n_heads: int = 64, head_dim: int = 128,
+                          prefix_len: int = 0) -> Workload:
+    """The random-tree attention experiment of App. C.1 (Table 5): one request, 64 heads of dimension
+    128, no prefix, a uniform random recursive tree of n_nodes tokens in creation order."""
+    if seed is None:
+        seed = MASTER_SEED + 5000 + n_nodes
+    rng = np.random.default_rng(seed)
+    parents = random_tree(rng, n_nodes)
+    return assemble(f"random_tree_n{n_nodes}_h{n_heads}_d{head_dim}_L{prefix_len}", rng, n_heads, n_heads, head_dim,
+                    [prefix_len], [parents], dict(seed=seed, experiment="random_tree"))
+
+
+def permute_tree_tokens(w: Workload, orders: List[np.ndarray], new_parents: List[np.ndarray]) -> Workload:
+    """The same requests with their tree tokens renumbered: new token k of request r is old token
+    orders[r][k] (its Q row and its K/V row move with it); new_parents[r] is the parent array in the
+    new numbering (computed by whoever chose the order; this function only moves rows)."""
+    q, k, v = w.q.copy(), w.k.copy(), w.v.copy()
+    no = w.node_offsets
+    for r in range(w.n_req):
+        order = np.asarray(orders[r], dtype=np.int64)
+        base = int(w.kv_row_offset[r]) + int(w.prefix_len[r])
+        q[no[r]:no[r + 1]] = w.q[no[r] + order]
+        k[base:base + len(order)] = w.k[base + order]
+        v[base:base + len(order)] = w.v[base + order]
+    return Workload(w.name + "_reordered", w.n_q_heads, w.n_kv_heads, w.head_dim, w.prefix_len.copy(), w.n_nodes.copy(),
+                    [np.asarray(p, dtype=np.int32) for p in new_parents], q, k, v, w.kv_row_offset.copy(),
+                    dict(w.meta, reordered=True))

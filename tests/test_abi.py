@@ -47,7 +47,8 @@ def test_host_only_entry_points(binding):
     assert B.dyspec_words_per_row(129) == 8
     assert B.dyspec_words_per_row(768) == 24
     assert B.dyspec_words_per_row(1024) == 32
-    assert B.dyspec_words_per_row(1025) < 0
+    assert B.dyspec_words_per_row(2048) == 64
+    assert B.dyspec_words_per_row(2049) < 0
     assert B.dyspec_error_string(0) == "ok"
     for code in range(-6, 0):
         assert B.dyspec_error_string(code) not in ("ok", "unknown error code")
@@ -60,7 +61,7 @@ def test_argument_errors_are_reported_before_any_launch(binding):
     # mask builder: bad sizes are rejected on the host (no device pointer is touched)
     assert lib.dyspec_build_tree_mask(None, -1, None, None, 4, None, None) == -1
     assert lib.dyspec_build_tree_mask(None, 5, None, None, 3, None, None) == -1          # W not a multiple of 4
-    assert lib.dyspec_build_tree_mask(None, 2000, None, None, 64, None, None) == -2       # > DYSPEC_MAX_NODES
+    assert lib.dyspec_build_tree_mask(None, 3000, None, None, 96, None, None) == -2       # > DYSPEC_MAX_NODES
     assert lib.dyspec_build_tree_mask(None, 200, None, None, 4, None, None) == -1         # 32*W < n
     assert lib.dyspec_build_tree_mask(None, 0, None, None, 4, None, None) == 0            # empty tree: no-op
     assert lib.dyspec_build_tree_mask(None, 5, None, None, 4, None, None) == -1           # NULL pointers
@@ -77,7 +78,7 @@ def test_argument_errors_are_reported_before_any_launch(binding):
     assert create(48, 4, 64) == -2           # g = 12
     assert create(4, 4, 96) == -2            # head_dim
     assert create(4, 4, 64, W=6) == -1
-    assert create(4, 4, 64, n=1025, W=64) == -2
+    assert create(4, 4, 64, n=2049, W=68) == -2
     assert create(4, 4, 64, n=200, W=4) == -1
     assert create(4, 4, 64, total=10) == -1  # request does not fit in the cache
     assert create(0, 4, 64) == -1
