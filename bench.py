@@ -205,14 +205,14 @@ def _time_replays(torch, graph, replays, tail=None):
     return e0.elapsed_time(e1)
 
 
-def measure_config(torch, runner, w, steps, warmup, device):
+def measure_config(torch, runner, w, steps, warmup, device, sparse=False):
     """Device-resident timing of exactly `steps` steps, rotating over independent copies of the inputs
     that together exceed 2x L2.  The launch sequence of one rotation is captured in a CUDA graph so
     that the host's launch overhead (python, ctypes) does not starve the GPU."""
-    first = runner.DeviceBatch(w, device=device)
+    first = runner.DeviceBatch(w, device=device, sparse=sparse)
     nbytes, flops = algorithmic_cost(w, first.W)
     copies = max(2, min(64, int(np.ceil(2.0 * L2_BYTES / max(nbytes, 1)))))
-    batches = [first] + [runner.DeviceBatch(w, device=device, plan=first.plan) for _ in range(copies - 1)]
+    batches = [first] + [runner.DeviceBatch(w, device=device, plan=first.plan, sparse=sparse) for _ in range(copies - 1)]
     info = first.plan.describe()
     launches_per_step = 1 + 1 + (1 if info["split_groups"] > 0 else 0)
     for i in range(max(warmup, 3)):
@@ -234,6 +234,48 @@ def measure_config(torch, runner, w, steps, warmup, device):
     return dict(batches=batches, total_ms=total_ms, ms_per_step=total_ms / steps, attn_ms=attn_ms, mask_ms=mask_ms,
                 bytes=nbytes, flops=flops, copies=copies, info=info, launches_per_step=launches_per_step, status=status,
                 graph=g_step)
+
+
+def random_tree_experiment(torch, runner, workloads, B, peaks, device, sizes=(256, 512, 1024, 2048), steps=200):
+    """The paper's random-tree attention experiment (App. C.1, Table 5: one request, 64 heads x 128,
+    no prefix, uniform random recursive trees): block counts and attention time in creation order
+    (dense call) and after the GPU's DFS renumbering with empty tree tiles skipped."""
+    rows = []
+    for n in sizes:
+        w = workloads.make_random_tree_case(n)
+        probe = runner.DeviceBatch(w, device=device)
+        order, _, new_parents = probe.dfs_reorder()
+        w2 = workloads.permute_tree_tokens(w, [order], [new_parents])
+        count = torch.zeros(1, dtype=torch.int64, device=device)
+        blocks = []
+        for batch in (probe, runner.DeviceBatch(w2, device=device, plan=probe.plan)):
+            batch.build_mask()
+            B.dyspec_mask_block_count(batch.bits, n, batch.W, 32, count)
+            torch.cuda.synchronize()
+            blocks.append(int(count.item()))
+        # the reorder kernel alone, from resident parents
+        order_d = torch.empty(n, dtype=torch.int32, device=device)
+        newp_d = torch.empty(n, dtype=torch.int32, device=device)
+        g_re = _graph_of(torch, lambda: [B.dyspec_plan_dfs_reorder(probe.plan, probe.parents, order_d, None, newp_d, None)
+                                         for _ in range(20)])
+        g_re.replay()
+        torch.cuda.synchronize()
+        reorder_us = _time_replays(torch, g_re, 10) / 200 * 1e3
+        del probe
+        m1 = measure_config(torch, runner, w, steps, 3, device)
+        m2 = measure_config(torch, runner, w2, steps, 3, device, sparse=True)
+        t_hbm_us = m1["bytes"] / (peaks["hbm_gbs"] * 1e9) * 1e6
+        rows.append({"tree_size": n, "workload": w.name, "blocks32": {"creation_order": blocks[0], "dfs_order": blocks[1]},
+                     "attention_call_us": {"creation_order_dense": m1["attn_ms"] * 1e3,
+                                           "dfs_order_skipping": m2["attn_ms"] * 1e3},
+                     "mask_us": {"plain": m1["mask_ms"] * 1e3, "with_tile_sets": m2["mask_ms"] * 1e3},
+                     "reorder_us": reorder_us, "bytes": m1["bytes"], "hbm_floor_us": t_hbm_us,
+                     "frac_of_hbm_floor": {"creation_order_dense": t_hbm_us / (m1["attn_ms"] * 1e3),
+                                           "dfs_order_skipping": t_hbm_us / (m2["attn_ms"] * 1e3)},
+                     "plan": m1["info"], "status": [m1["status"], m2["status"]]})
+        del m1, m2
+        torch.cuda.empty_cache()
+    return rows
 
 
 def roofline_entry(m, peaks, peaks_kind):
@@ -364,6 +406,11 @@ def run_ours(args):
                 del mi["batches"], mi["graph"]
                 torch.cuda.empty_cache()
 
+    random_tree = None
+    if not args.no_per_config and world == 1:
+        from paper_2410_11744_b200 import binding
+        random_tree = random_tree_experiment(torch, runner, workloads, binding, peaks, device)
+
     # ---- the oracle on the host cores, bounded sample of the same workload
     times = time_oracle(w, budget_s=12.0)
     cpu_sec = sum(times) / len(times)
@@ -390,6 +437,8 @@ def run_ours(args):
     }
     if per_config:
         line["per_config"] = per_config
+    if random_tree:
+        line["random_tree_experiment"] = random_tree
     print(json.dumps(line), flush=True)
     if use_dist:
         dist.barrier()

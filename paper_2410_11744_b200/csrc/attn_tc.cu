@@ -139,6 +139,33 @@ __device__ __forceinline__ void st_global_v8(void* ptr, const uint32_t* v) {
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
+// Packed fp32 pairs (sm_100: one instruction works on two floats held in a 64-bit register pair)
+// and the three-input maximum: the softmax threads are bound by instruction issue, and these halve
+// the count of the scale, sum and max instructions.
+__device__ __forceinline__ uint64_t pack_f32x2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack_f32x2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ float max3_f32(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+
 // Which key tiles of an item's range are processed.  The prefix tiles always are; of the tree tiles
 // only those that some row of the query tile can see (App. C: empty blocks of the tree mask are
 // skipped), when the caller passed the per-node tile sets; all of them otherwise.  Every role of the
@@ -488,11 +515,11 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         }
         float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-        for (int i = 0; i < BN; i += 4) {
-          mx4[0] = fmaxf(mx4[0], __uint_as_float(sv[i]));
-          mx4[1] = fmaxf(mx4[1], __uint_as_float(sv[i + 1]));
-          mx4[2] = fmaxf(mx4[2], __uint_as_float(sv[i + 2]));
-          mx4[3] = fmaxf(mx4[3], __uint_as_float(sv[i + 3]));
+        for (int i = 0; i < BN; i += 8) {
+          mx4[0] = max3_f32(mx4[0], __uint_as_float(sv[i]), __uint_as_float(sv[i + 1]));
+          mx4[1] = max3_f32(mx4[1], __uint_as_float(sv[i + 2]), __uint_as_float(sv[i + 3]));
+          mx4[2] = max3_f32(mx4[2], __uint_as_float(sv[i + 4]), __uint_as_float(sv[i + 5]));
+          mx4[3] = max3_f32(mx4[3], __uint_as_float(sv[i + 6]), __uint_as_float(sv[i + 7]));
         }
         const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2e;   // scale > 0
         const float m_new = fmaxf(m_used, mx);
@@ -518,21 +545,29 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         const float neg_ref = m_used == -INFINITY ? 0.f : -m_used;
 
         // P = 2^(s * scale - ref) as bf16 pairs, written over the first 64 S columns (masked: 2^-inf = 0)
-        float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+        const uint64_t scale2 = pack_f32x2(p.scale_log2e, p.scale_log2e), ref2 = pack_f32x2(neg_ref, neg_ref);
+        uint64_t sum2[2] = {0ull, 0ull};
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
           uint32_t pk[16];
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
-            const float p0 = fast_exp2(fmaf(__uint_as_float(sv[32 * c + 2 * i]), p.scale_log2e, neg_ref));
-            const float p1 = fast_exp2(fmaf(__uint_as_float(sv[32 * c + 2 * i + 1]), p.scale_log2e, neg_ref));
-            sum4[(2 * i) & 3] += p0;
-            sum4[(2 * i + 1) & 3] += p1;
+            const uint64_t x = fma_f32x2(pack_f32x2(__uint_as_float(sv[32 * c + 2 * i]), __uint_as_float(sv[32 * c + 2 * i + 1])),
+                                         scale2, ref2);
+            float x0, x1;
+            unpack_f32x2(x, x0, x1);
+            const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
+            sum2[i & 1] = add_f32x2(sum2[i & 1], pack_f32x2(p0, p1));
             pk[i] = pack_bf16x2(p0, p1);
           }
           tmem_st16(t_s + uint32_t(c) * 16u, pk);
         }
-        l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+        {
+          float a0, a1, b0, b1;
+          unpack_f32x2(sum2[0], a0, a1);
+          unpack_f32x2(sum2[1], b0, b1);
+          l += (a0 + a1) + (b0 + b1);
+        }
         if (r == 0) trace_event(tc_cur, DYSPEC_TAG(1 + h, 4, j));
 
         // V rows past the end of the request are not ours: zero them (their probabilities are 0, but
