@@ -1,6 +1,7 @@
 // C ABI of the tree-verify attention library: argument checks, the host-side ragged scheduler
 // (plan), TMA tensor-map encoding and kernel launches.  See include/dyspec.h for the contract.
 #include <cmath>
+#include <cstdio>
 #include <cstdlib>
 #include <cstring>
 #include <map>
@@ -68,6 +69,12 @@ bool encode_map(CUtensorMap* map, const void* base, int64_t rows, int heads, int
   return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// DYSPEC_ERR_CUDA, with the runtime's own message on stderr when DYSPEC_DEBUG is set in the environment.
+int cuda_failed(cudaError_t e, const char* where) {
+  if (std::getenv("DYSPEC_DEBUG")) std::fprintf(stderr, "dyspec: %s: %s\n", where, cudaGetErrorString(e));
+  return DYSPEC_ERR_CUDA;
 }
 
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
@@ -162,6 +169,27 @@ void schedule(dyspec_plan& pl) {
     for (size_t gi = 0; gi < groups.size(); ++gi) {
       const Group& gr = groups[gi];
       const ReqInfo& rq = pl.reqs[size_t(gr.req)];
+      // Who merges: with equal pieces every CTA takes BM / C rows.  With unequal pieces the CTAs with
+      // the larger pieces finish last; they only hand their partial rows over, and the C / 2 CTAs with
+      // the smallest pieces (lowest ranks on ties) share the rows, so the merge work is done -- all
+      // but folding in the last arrival -- before the slowest CTA gets there.
+      int owners = (1 << C) - 1;
+      {
+        int lo = gr.tiles, hi = 0;
+        for (int c = 0; c < C; ++c) {
+          const int sz = int(int64_t(gr.tiles) * (c + 1) / C) - int(int64_t(gr.tiles) * c / C);
+          lo = std::min(lo, sz); hi = std::max(hi, sz);
+        }
+        if (hi != lo) {
+          owners = 0;
+          int taken = 0;
+          for (int want = lo; want <= hi && taken < C / 2; ++want)
+            for (int c = 0; c < C && taken < C / 2; ++c) {
+              const int sz = int(int64_t(gr.tiles) * (c + 1) / C) - int(int64_t(gr.tiles) * c / C);
+              if (sz == want) { owners |= 1 << c; ++taken; }
+            }
+        }
+      }
       for (int c = 0; c < C; ++c) {
         WorkItem it{};
         it.kv_row0 = rq.kv_row0; it.prefix_len = rq.prefix_len; it.n_nodes = rq.n_nodes; it.node0 = rq.node0;
@@ -169,6 +197,7 @@ void schedule(dyspec_plan& pl) {
         it.tile_begin = int(int64_t(gr.tiles) * c / C);
         it.tile_end = int(int64_t(gr.tiles) * (c + 1) / C);
         it.slot = -1; it.slot0 = -1; it.group = int(gi); it.n_splits = C; it.n_in_cta = 1;
+        it.merge_owners = owners;
         pl.items.push_back(it);
         pl.cta_begin.push_back(int32_t(pl.items.size()));
       }
@@ -570,9 +599,9 @@ int dyspec_tree_attention_ragged_sparse(const dyspec_plan_t* plan, const void* q
   cudaError_t e;
   if (plan->regime == 0) e = launch_attn_mma(plan->d, plan->n_ctas, mq, mk, mv, p, st);
   else e = launch_attn_tc(plan->d, plan->n_ctas, mq, mk, mv, p, st);
-  if (e != cudaSuccess) return DYSPEC_ERR_CUDA;
+  if (e != cudaSuccess) return cuda_failed(e, "attention launch");
   e = launch_combine(plan->d, bm, int(plan->split_groups.size()), p, st);
-  return e == cudaSuccess ? DYSPEC_OK : DYSPEC_ERR_CUDA;
+  return e == cudaSuccess ? DYSPEC_OK : cuda_failed(e, "combine launch");
 }
 
 // ---- single-request convenience form -------------------------------------------------------------

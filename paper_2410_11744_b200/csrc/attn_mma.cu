@@ -69,10 +69,13 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   const uint32_t s_q = smem_u32(smem);
   const uint32_t s_kv = s_q + L::kQBytes;
   const uint32_t s_bar = s_q + L::kBarOffset;
-  // barriers: full[kStages], empty[kStages], q_full, q_empty
+  // barriers: full[kStages], empty[kStages], q_full, q_empty, src[8] (one per cluster peer)
   const uint32_t bar_full = s_bar, bar_empty = s_bar + 8 * kStages;
-  const uint32_t bar_qfull = s_bar + 16 * kStages, bar_qempty = bar_qfull + 8;
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::kBarOffset + 16 * kStages + 16);
+  const uint32_t bar_qfull = s_bar + 16 * kStages, bar_qempty = bar_qfull + 8, bar_src = bar_qempty + 8;
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::kBarOffset + 16 * kStages + 16 + 64);
+  // In cluster mode the last two ring stages are not part of the ring: peers push their partial rows
+  // into them (see the epilogue), possibly while this CTA is still streaming K/V through the others.
+  const int n_stages = p.cluster_size > 1 ? kStages - 2 : kStages;
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -90,10 +93,12 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     }
     mbar_init(bar_qfull, 1);
     mbar_init(bar_qempty, kComputeWarps);
+    for (int k = 0; k < 8; ++k) mbar_init(bar_src + 8 * k, 1);
     *abort_flag = 0;
     fence_barrier_init();
   }
   __syncthreads();
+  if (p.cluster_size > 1) cluster_arrive();     // "my barriers exist"; peers wait for this only just before they push
 
   const WorkItem* my_items = p.items + size_t(blockIdx.x) * p.items_stride;
   const int item_begin = 0;
@@ -107,7 +112,8 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       prefetch_tensormap(&map_q);
       prefetch_tensormap(&map_k);
       prefetch_tensormap(&map_v);
-      uint32_t it = 0;       // running key-tile counter of this CTA (ring position)
+      int ring_stage = 0;    // ring position of the next key tile of this CTA
+      uint32_t ring_phase = 0;
       uint32_t qit = 0;      // running item counter (Q buffer phase)
       for (int w = item_begin; w < item_end; ++w, ++qit) {
         const WorkItem item = my_items[w];
@@ -119,9 +125,10 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           tma_load_3d(s_q + h * (BM * 128), &map_q, bar_qfull, h * 64, item.kv_head * g,
                       rq.node0 + (item.row0 >> p.log2_g));
         const int n_prefix_tiles = (rq.prefix_len + BN - 1) / BN;
-        for (int t = item.tile_begin; t < item.tile_end; ++t, ++it) {
-          const int stage = it % kStages;
-          const uint32_t ph = (it / kStages) & 1;
+        for (int t = item.tile_begin; t < item.tile_end; ++t) {
+          const int stage = ring_stage;
+          const uint32_t ph = ring_phase;
+          if (++ring_stage == n_stages) { ring_stage = 0; ring_phase ^= 1u; }
           mbar_wait(bar_empty + 8 * stage, ph ^ 1, abort_flag, p.status);
           const int64_t row = rq.kv_row0 + (t < n_prefix_tiles ? int64_t(t) * BN
                                                                : int64_t(rq.prefix_len) + int64_t(t - n_prefix_tiles) * BN);
@@ -134,10 +141,7 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         }
       }
     }
-    if (p.cluster_size > 1) {        // every thread of the cluster takes part in the two cluster barriers
-      cluster_sync_all();
-      cluster_sync_all();
-    }
+    if (p.cluster_size > 1) cluster_wait();      // pairs with the arrive above (all threads of the cluster take part)
     return;
   }
 
@@ -149,7 +153,8 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   const int gid = lane >> 2;      // row within an 8-row slab
   const int tig = lane & 3;       // column pair within an 8-column tile
   const int wrow = warp * 16;
-  uint32_t it = 0, qit = 0;
+  int ring_stage = 0;
+  uint32_t ring_phase = 0, qit = 0;
 
   for (int w = item_begin; w < item_end; ++w, ++qit) {
     const WorkItem item = my_items[w];
@@ -180,9 +185,10 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     for (int j = 0; j < DT; ++j) { o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f; }
     float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;
 
-    for (int t = item.tile_begin; t < item.tile_end; ++t, ++it) {
-      const int stage = it % kStages;
-      const uint32_t ph = (it / kStages) & 1;
+    for (int t = item.tile_begin; t < item.tile_end; ++t) {
+      const int stage = ring_stage;
+      const uint32_t ph = ring_phase;
+      if (++ring_stage == n_stages) { ring_stage = 0; ring_phase ^= 1u; }
       const uint32_t s_k = s_kv + stage * L::kStageBytes;
       const uint32_t s_v = s_k + L::kTileBytes;
       mbar_wait(bar_full + 8 * stage, ph, abort_flag, p.status);
@@ -306,89 +312,144 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
     if (p.cluster_size > 1) {
       // ---- split-KV combine inside a thread-block cluster: the CTAs of a cluster hold the splits of
-      // one query tile.  Each parks its partial (O, m, l) in its own shared memory (the K/V ring is
-      // idle by now: a CTA owns exactly one item in this mode), the cluster synchronises, and CTA k
-      // merges rows [k * BM / C, (k + 1) * BM / C) of all C partials through distributed shared memory.
+      // one query tile (a CTA owns exactly one item in this mode).  The scheduler names the owners
+      // (item.merge_owners): n_own of the C CTAs, each responsible for R = BM / n_own rows.  Every
+      // CTA parks its partial (O, m, l) in its own shared memory (the K/V ring is idle by now),
+      // grouped by owner, and PUSHES each group into its owner's receive buffer with one asynchronous
+      // shared-to-shared bulk copy that signals a barrier of the owner.  An owner folds the groups
+      // into its own, one source at a time as they arrive (owners first, then the CTAs with the
+      // larger pieces), with loops kept rolled: this code runs once per CTA, so its cost is mostly
+      // instruction fetch, and only the fold of the last arrival is on the critical path.  No remote
+      // loads; the only cluster barrier is split around the whole kernel body.
       const int C = p.cluster_size;                       // 2, 4 or 8
-      const int log2c = C == 2 ? 1 : (C == 4 ? 2 : 3);
+      const uint32_t owners = uint32_t(item.merge_owners);
+      const int n_own = __popc(owners);                   // 1, 2, 4 or 8
+      const int log2r = 6 - (31 - __clz(n_own));
+      const int R = 1 << log2r;                           // rows per owner
+      const int chunk_floats = R * (D + 2);               // R rows of O, then R maxima, then R sums
+      const uint32_t chunk_bytes = uint32_t(chunk_floats) * 4u;
+      const int rank = int(cluster_ctarank());
+      const bool own = (owners >> rank) & 1u;
+      const int my_oi = __popc(owners & ((1u << rank) - 1u));                                        // which group is mine
+      float* send = reinterpret_cast<float*>(smem + L::kQBytes);                                    // [n_own][chunk]
+      float* recv = reinterpret_cast<float*>(smem + L::kQBytes + (kStages - 2) * L::kStageBytes);   // [C - 1][chunk]
+      if (own && threadIdx.x == 0)
+        for (int s_ = 0; s_ < C; ++s_)
+          if (s_ != rank) mbar_expect_tx(bar_src + 8 * s_, chunk_bytes);
       asm volatile("bar.sync 1, %0;" ::"n"(kComputeWarps * 32) : "memory");     // all warps are done with the ring
-      float* sc_o = reinterpret_cast<float*>(smem + L::kQBytes);                 // [BM][D]
-      float* sc_m = sc_o + BM * D;                                               // [BM]
-      float* sc_l = sc_m + BM;                                                   // [BM]
       {
+        // columns are XOR-swizzled by the row so that the 8 rows a warp stores at once hit different banks
         const int r_lo = wrow + gid, r_hi = r_lo + 8;
+        float* c_lo = send + (r_lo >> log2r) * chunk_floats;
+        float* c_hi = send + (r_hi >> log2r) * chunk_floats;
+        const int rr_lo = r_lo & (R - 1), rr_hi = r_hi & (R - 1);
 #pragma unroll
         for (int j = 0; j < DT; ++j) {
           const int c = j * 8 + tig * 2;
-          *reinterpret_cast<float2*>(sc_o + r_lo * D + c) = make_float2(o[j][0], o[j][1]);
-          *reinterpret_cast<float2*>(sc_o + r_hi * D + c) = make_float2(o[j][2], o[j][3]);
+          *reinterpret_cast<float2*>(c_lo + rr_lo * D + (c ^ ((rr_lo & 7) << 3))) = make_float2(o[j][0], o[j][1]);
+          *reinterpret_cast<float2*>(c_hi + rr_hi * D + (c ^ ((rr_hi & 7) << 3))) = make_float2(o[j][2], o[j][3]);
         }
-        if (tig == 0) { sc_m[r_lo] = m_lo; sc_l[r_lo] = l_lo; sc_m[r_hi] = m_hi; sc_l[r_hi] = l_hi; }
-      }
-      cluster_sync_all();
-      // A warp merges BM / C / 4 rows from C sources: always 16 (row, source) pairs.  All their loads
-      // are issued before the first use, so the merge costs about two remote-load latencies in all.
-      const int rank = int(cluster_ctarank());
-      const int row_base = rank * (BM >> log2c) + warp * ((BM >> log2c) / kComputeWarps);
-      const uint32_t a_o = smem_u32(sc_o), a_m = smem_u32(sc_m), a_l = smem_u32(sc_l);
-      constexpr int V = D / 32;
-      float mm[16], ll[16];
-      float vv[16][V];
-#pragma unroll
-      for (int q = 0; q < 16; ++q) {
-        const int r = row_base + (q >> log2c);
-        const uint32_t src = uint32_t(q & (C - 1));
-        mm[q] = ld_dsmem_f32(map_to_cta(a_m + 4u * uint32_t(r), src));
-        ll[q] = ld_dsmem_f32(map_to_cta(a_l + 4u * uint32_t(r), src));
-        const uint32_t av = map_to_cta(a_o + 4u * uint32_t(r * D + lane * V), src);
-        if constexpr (V == 4) {
-          const float4 v = ld_dsmem_f32x4(av);
-          vv[q][0] = v.x; vv[q][1] = v.y; vv[q][2] = v.z; vv[q][3] = v.w;
-        } else {
-          const float2 v = ld_dsmem_f32x2(av);
-          vv[q][0] = v.x; vv[q][1] = v.y;
+        if (tig == 0) {
+          c_lo[R * D + rr_lo] = m_lo; c_lo[R * D + R + rr_lo] = l_lo;
+          c_hi[R * D + rr_hi] = m_hi; c_hi[R * D + R + rr_hi] = l_hi;
         }
       }
-      // reduce groups of C consecutive pairs (one row each)
+      fence_proxy_async();                                 // the bulk copies below read what was just stored
+      cluster_wait();                                      // every peer has initialised its barriers (arrived long ago)
+      asm volatile("bar.sync 1, %0;" ::"n"(kComputeWarps * 32) : "memory");
+      const bool pusher = warp == 0 && lane < C && lane != rank && ((owners >> lane) & 1u);
+      if (pusher) {
+        const uint32_t slot = uint32_t(rank < lane ? rank : rank - 1);          // where owner `lane` keeps source `rank`
+        const uint32_t oi = uint32_t(__popc(owners & ((1u << lane) - 1u)));     // the group that owner is responsible for
+        dsmem_push(map_to_cta(smem_u32(recv) + slot * chunk_bytes, uint32_t(lane)),
+                   smem_u32(send) + oi * chunk_bytes, chunk_bytes, map_to_cta(bar_src + 8 * rank, uint32_t(lane)));
+      }
+      if (own) {
+        float* acc_o = send + my_oi * chunk_floats;        // the running merge lives in this CTA's own group
+        float* acc_m = acc_o + R * D;
+        float* acc_l = acc_m + R;
+        const int tid = threadIdx.x;                       // compute warps are threads 0 .. 127
+        const int n_vec = (R * D) >> 2;                    // float4 elements of a group
+        constexpr int kB = 4;
+        // sources in the order they are expected: the other owners (small pieces), then the rest
+#pragma unroll 1
+        for (int pass = 0; pass < 2; ++pass) {
+#pragma unroll 1
+          for (int s_ = 0; s_ < C; ++s_) {
+            if (s_ == rank || int((owners >> s_) & 1u) == pass) continue;
+            mbar_wait(bar_src + 8 * s_, 0, abort_flag, p.status);
+            const float* src_o = recv + (s_ < rank ? s_ : s_ - 1) * chunk_floats;
+            const float* src_m = src_o + R * D;
+            const float* src_l = src_m + R;
+            // batches of kB independent elements per thread: all loads first, then the math, then the
+            // stores (a rolled element-by-element loop is a chain of shared-memory latencies)
+#pragma unroll 1
+            for (int base = tid; base < n_vec; base += kB * kComputeWarps * 32) {
+              float4 a[kB], b_[kB];
+              float ma[kB], ms[kB];
 #pragma unroll
-      for (int q0 = 0; q0 < 16; q0 += 2) {
-        if ((q0 & (C - 1)) != 0) continue;     // q0 starts a row only when it is a multiple of C
-        const int r = row_base + (q0 >> log2c);
-        const int row = item.row0 + r;
-        float m = -INFINITY;
+              for (int k = 0; k < kB; ++k) {
+                const int idx = min(base + k * kComputeWarps * 32, n_vec - 1);
+                const int rr = idx / (D / 4);
+                ma[k] = acc_m[rr]; ms[k] = src_m[rr];
+                a[k] = reinterpret_cast<const float4*>(acc_o)[idx];
+                b_[k] = reinterpret_cast<const float4*>(src_o)[idx];
+              }
 #pragma unroll
-        for (int c = 0; c < 8; ++c)
-          if (c < C && q0 + c < 16) m = fmaxf(m, mm[q0 + c]);
-        const float ref = m == -INFINITY ? 0.f : m;
-        float acc[V];
+              for (int k = 0; k < kB; ++k) {
+                const float mn = fmaxf(ma[k], ms[k]);
+                const float ref = mn == -INFINITY ? 0.f : mn;
+                const float keep = fast_exp2(ma[k] - ref), wgt = fast_exp2(ms[k] - ref);
+                a[k].x = a[k].x * keep + b_[k].x * wgt; a[k].y = a[k].y * keep + b_[k].y * wgt;
+                a[k].z = a[k].z * keep + b_[k].z * wgt; a[k].w = a[k].w * keep + b_[k].w * wgt;
+              }
 #pragma unroll
-        for (int k = 0; k < V; ++k) acc[k] = 0.f;
-        float lsum = 0.f;
-#pragma unroll
-        for (int c = 0; c < 8; ++c) {
-          if (c < C && q0 + c < 16) {
-            const float wgt = fast_exp2(mm[q0 + c] - ref);
-            lsum += wgt * ll[q0 + c];
-#pragma unroll
-            for (int k = 0; k < V; ++k) acc[k] += wgt * vv[q0 + c][k];
+              for (int k = 0; k < kB; ++k) {
+                const int idx = base + k * kComputeWarps * 32;
+                if (idx < n_vec) reinterpret_cast<float4*>(acc_o)[idx] = a[k];
+              }
+            }
+            asm volatile("bar.sync 1, %0;" ::"n"(kComputeWarps * 32) : "memory");   // every row's old maximum has been used
+            if (tid < R) {
+              const float ma = acc_m[tid], ms = src_m[tid];
+              const float mn = fmaxf(ma, ms);
+              const float ref = mn == -INFINITY ? 0.f : mn;
+              acc_l[tid] = acc_l[tid] * fast_exp2(ma - ref) + src_l[tid] * fast_exp2(ms - ref);
+              acc_m[tid] = mn;
+            }
+            asm volatile("bar.sync 1, %0;" ::"n"(kComputeWarps * 32) : "memory");
           }
         }
-        if (row < n_rows) {
-          const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
-          const int node = row >> p.log2_g;
-          const int head = item.kv_head * g + (row & (g - 1));
-          __nv_bfloat16* out = p.out + (size_t(rq.node0 + node) * p.n_q_heads + head) * D;
-          if constexpr (V == 4) {
-            uint2 o2;
-            o2.x = pack_bf16x2(acc[0] * inv, acc[1] * inv);
-            o2.y = pack_bf16x2(acc[2] * inv, acc[3] * inv);
-            *reinterpret_cast<uint2*>(out + lane * 4) = o2;
-          } else {
-            *reinterpret_cast<uint32_t*>(out + lane * 2) = pack_bf16x2(acc[0] * inv, acc[1] * inv);
+        // normalise and write the R rows (element idx sits at swizzled column cs of row rr)
+#pragma unroll 1
+        for (int base = tid; base < n_vec; base += kB * kComputeWarps * 32) {
+          float4 a[kB];
+          float lsum[kB];
+#pragma unroll
+          for (int k = 0; k < kB; ++k) {
+            const int idx = min(base + k * kComputeWarps * 32, n_vec - 1);
+            lsum[k] = acc_l[idx / (D / 4)];
+            a[k] = reinterpret_cast<const float4*>(acc_o)[idx];
+          }
+#pragma unroll
+          for (int k = 0; k < kB; ++k) {
+            const int idx = base + k * kComputeWarps * 32;
+            const int rr = idx / (D / 4);
+            const int c = ((idx - rr * (D / 4)) * 4) ^ ((rr & 7) << 3);
+            const int row = item.row0 + my_oi * R + rr;
+            if (idx < n_vec && row < n_rows) {
+              const float inv = lsum[k] > 0.f ? 1.f / lsum[k] : 0.f;
+              const int node = row >> p.log2_g;
+              const int head = item.kv_head * g + (row & (g - 1));
+              uint2 o2;
+              o2.x = pack_bf16x2(a[k].x * inv, a[k].y * inv);
+              o2.y = pack_bf16x2(a[k].z * inv, a[k].w * inv);
+              *reinterpret_cast<uint2*>(p.out + (size_t(rq.node0 + node) * p.n_q_heads + head) * D + c) = o2;
+            }
           }
         }
       }
-      cluster_sync_all();                                 // nobody leaves while a peer still reads its shared memory
+      if (pusher) dsmem_push_wait_source_read();          // the parked rows must outlive the copies that read them
     } else if (item.slot < 0) {
       const float inv_lo = l_lo > 0.f ? 1.f / l_lo : 0.f, inv_hi = l_hi > 0.f ? 1.f / l_hi : 0.f;
       const int head_lo = item.kv_head * g + (row_lo & (g - 1)), head_hi = item.kv_head * g + (row_hi & (g - 1));

@@ -44,7 +44,7 @@ struct WorkItem {
   int32_t slot0;       // first partial slot of the group (slots slot0 .. slot0 + n_splits - 1)
   int32_t n_in_cta;    // in the first item of a CTA: how many items the CTA owns
   int32_t req;         // request index
-  int32_t pad;
+  int32_t merge_owners;  // cluster mode: bit k set = CTA k of the cluster merges a share of the rows (see attn_mma.cu)
 };
 static_assert(sizeof(WorkItem) == 64, "WorkItem is one 64-byte record");
 
@@ -207,6 +207,23 @@ __device__ __forceinline__ uint32_t cluster_ctarank() {
 }
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// The two halves of the cluster barrier, for a hand-shake whose latency should stay hidden: every
+// thread arrives early and waits only when it needs the peers to have arrived.
+// (relaxed: what the peers must see -- the initialised mbarriers -- was published by fence.mbarrier_init)
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+// Asynchronous copy of `bytes` (a multiple of 16; both addresses 16-byte aligned) from this CTA's
+// shared memory into a peer CTA's; the peer's mbarrier receives the byte count when the data has
+// landed.  dst and bar are shared::cluster addresses (see map_to_cta).  Not a multicast.
+__device__ __forceinline__ void dsmem_push(uint32_t dst_cluster_addr, uint32_t src_local_addr, uint32_t bytes,
+                                           uint32_t bar_cluster_addr) {
+  asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst_cluster_addr), "r"(src_local_addr), "r"(bytes), "r"(bar_cluster_addr) : "memory");
+}
+// Until this returns, the source of this thread's dsmem_push calls must stay intact.
+__device__ __forceinline__ void dsmem_push_wait_source_read() {
+  asm volatile("cp.async.bulk.commit_group;\n\tcp.async.bulk.wait_group.read 0;" ::: "memory");
 }
 __device__ __forceinline__ uint32_t map_to_cta(uint32_t local_smem_addr, uint32_t cta_rank) {
   uint32_t r;
