@@ -395,18 +395,22 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           const bool more = j + 1 < T;
           const uint32_t kslot = sc % kSlots, kph = (sc / kSlots) & 1;
           if (more) ++sc;
-          // Slot waits first: an mbarrier wait costs ~180 cycles even when its phase completed long
-          // ago; here that latency hides behind the softmax this thread has to wait for anyway.
-#ifndef EXP_NO_SLOT_WAIT
-          mbar_wait(bar(B_SLOT_FULL + vslot), vph, abort_flag, p.status);
-          if (more) mbar_wait(bar(B_SLOT_FULL + kslot), kph, abort_flag, p.status);
-#endif
-          if (j == 0) {
-            mbar_wait(bar(B_OFREE + 0), (n_it0 & 1) ^ 1, abort_flag, p.status);
-            if (two) mbar_wait(bar(B_OFREE + 1), (n_it1 & 1) ^ 1, abort_flag, p.status);
+          // An mbarrier probe takes ~180 cycles to answer even when the phase completed long ago.  The
+          // three barriers this tile starts with (V slot, next K slot, P of half A) are probed in one
+          // go, so their round trips overlap; only what is really not there yet is then waited for.
+          {
+            const uint32_t got = __reduce_and_sync(0xffffffffu,
+                mbar_test_wait3(bar(B_SLOT_FULL + vslot), vph, bar(B_SLOT_FULL + (more ? kslot : vslot)), more ? kph : vph,
+                                bar(B_PREADY + 0), n_p0 & 1));
+            if (!(got & 1u)) mbar_wait(bar(B_SLOT_FULL + vslot), vph, abort_flag, p.status);
+            if (more && !(got & 2u)) mbar_wait(bar(B_SLOT_FULL + kslot), kph, abort_flag, p.status);
+            if (j == 0) {
+              mbar_wait(bar(B_OFREE + 0), (n_it0 & 1) ^ 1, abort_flag, p.status);
+              if (two) mbar_wait(bar(B_OFREE + 1), (n_it1 & 1) ^ 1, abort_flag, p.status);
+            }
+            // ---- half A: O_A += P_A V, then S_A = Q_A K(j+1)^T
+            if (!(got & 4u)) mbar_wait(bar(B_PREADY + 0), n_p0 & 1, abort_flag, p.status);
           }
-          // ---- half A: O_A += P_A V, then S_A = Q_A K(j+1)^T
-          mbar_wait(bar(B_PREADY + 0), n_p0 & 1, abort_flag, p.status);
           ++n_p0;
           tc_fence_after();
           trace_event(tc_cur, DYSPEC_TAG(0, 1, j));

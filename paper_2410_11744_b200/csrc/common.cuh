@@ -131,6 +131,24 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return done != 0;
 }
+// Three probes whose round trips overlap: the answers come back together, about one probe latency
+// after the first was issued (three mbar_test_wait calls in a row would take three latencies, since
+// each consumes its predicate before the next is issued).  Bit k of the result = barrier k's phase done.
+__device__ __forceinline__ uint32_t mbar_test_wait3(uint32_t bar0, uint32_t parity0, uint32_t bar1, uint32_t parity1,
+                                                    uint32_t bar2, uint32_t parity2) {
+  uint32_t done;
+  asm volatile(
+      "{\n\t.reg .pred p0, p1, p2;\n\t.reg .u32 r0, r1, r2;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p0, [%1], %2;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p1, [%3], %4;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p2, [%5], %6;\n\t"
+      "selp.u32 r0, 1, 0, p0;\n\tselp.u32 r1, 2, 0, p1;\n\tselp.u32 r2, 4, 0, p2;\n\t"
+      "or.b32 r0, r0, r1;\n\tor.b32 %0, r0, r2;\n\t}"
+      : "=r"(done)
+      : "r"(bar0), "r"(parity0), "r"(bar1), "r"(parity1), "r"(bar2), "r"(parity2)
+      : "memory");
+  return done;
+}
 __device__ __forceinline__ uint64_t global_timer_ns() {
   uint64_t t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
