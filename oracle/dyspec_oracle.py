@@ -26,13 +26,19 @@ Parity status: every function below is pinned by tests/test_oracle_pins.py
 in pure Python, closed forms, hand-written mask fixture, relabelling
 invariance); the token-reorder functions at the end (App. C) are pinned by
 tests/test_reorder_pins.py (the block counts the paper prints in Table 5,
-closed forms, a hand example, subtree contiguity, attention invariance).
+closed forms, a hand example, subtree contiguity, attention invariance);
+verify_tree (Algorithm 3) by tests/test_verify_pins.py (the output distribution
+equals the target's, Draft == Target accepts every first branch, closed-form
+acceptance rates, forced rejections, the all-zero early exit).
 Nothing here is "parity unpinned".
 
 Readings where the paper is silent: scale = 1/sqrt(head_dim); consecutive query
 heads share a KV head; tree K/V rows follow the prefix rows in node order;
 masks are packed LSB-first in uint32 words; the DFS renumbering visits roots
-and children in increasing index (the order that reproduces Table 5).
+and children in increasing index (the order that reproduces Table 5);
+Algorithm 3 draws its acceptance number from U(0,1) (printed as N(0,1)), the
+branches of a node are its children in increasing index, and the final token
+is drawn from the residual by inverse CDF in token order.
 """
 from __future__ import annotations
 
@@ -259,3 +265,80 @@ def mask_block_count(parents: Sequence[int], block: int = 32) -> int:
             if m[a * block:(a + 1) * block, b * block:(b + 1) * block].any():
                 count += 1
     return count
+
+
+# ----------------------------------------------------------------------------------------------------
+# Verification of the token tree against the target model (App. "Verification", Algorithm 3).
+# ----------------------------------------------------------------------------------------------------
+def verify_tree(parents: Sequence[int], tokens: Sequence[int], draft_probs, target_probs, accept_u, sample_u,
+                bonus_at_leaf: bool = False):
+    """Algorithm 3 (multi-branch rejection sampling along the tree), in fp64.
+
+    parents[i], tokens[i]  the tree and the token each node carries (the root's token is not used);
+                           the branches of a node are its children in increasing index
+    draft_probs[i][v]      Draft(node i, v): the distribution node i's children were drawn from
+    target_probs[i][v]     Target(node i, v)
+    accept_u[i]            the number drawn when child i is tried; the paper prints c ~ N(0,1), which
+                           cannot be meant for an accept-with-probability-R[y]/D[y] test: read U(0,1)
+    sample_u[i]            the U(0,1) number used if the walk ends at node i and a token is drawn from
+                           the residual R there (inverse CDF: the first v with cumsum(R)[v] > u * sum(R))
+    Roots other than node 0 are ignored (the walk starts at node 0).  As printed, the loop runs while
+    the current node has branches, so a walk that reaches a leaf ends there without a further token;
+    bonus_at_leaf=True adds the usual extra token drawn from Target(leaf, .) instead.
+
+    Returns (accepted_tokens, accepted_nodes, margins): the token sequence A, the nodes that were
+    accepted (the final, sampled token has no node), and for every decision taken the distance of the
+    deciding number from its threshold (so that a lower-precision implementation can be excused where
+    the decision was a coin toss).
+    """
+    check_parents(parents)
+    n = len(parents)
+    D_all = np.asarray(draft_probs, dtype=np.float64)
+    T_all = np.asarray(target_probs, dtype=np.float64)
+    children: List[List[int]] = [[] for _ in range(n)]
+    for i in range(1, n):
+        if int(parents[i]) >= 0:
+            children[int(parents[i])].append(i)
+    accepted_tokens: List[int] = []
+    accepted_nodes: List[int] = []
+    margins: List[float] = []
+    cur = 0
+    while True:
+        if not children[cur] and not bonus_at_leaf:
+            break
+        R = T_all[cur].copy()
+        moved = False
+        if children[cur]:
+            D = D_all[cur].copy()
+            for child in children[cur]:
+                y = int(tokens[child])
+                c = float(accept_u[child])
+                ratio = R[y] / D[y] if D[y] > 0 else (np.inf if R[y] > 0 else 0.0)
+                margins.append(abs(c - ratio))
+                if c <= ratio:
+                    accepted_tokens.append(y)
+                    accepted_nodes.append(child)
+                    cur = child
+                    moved = True
+                    break
+                R = np.maximum(R - D, 0.0)
+                if R.sum() > 0:
+                    R = R / R.sum()
+                D[y] = 0.0
+                if not (D > 0).any():
+                    break
+                D = D / D.sum()
+        if not moved:
+            total = R.sum()
+            if total <= 0:              # nothing left to sample from (cannot happen when Draft != Target on the support)
+                R = T_all[cur].copy()
+                total = R.sum()
+            cdf = np.cumsum(R)
+            target = float(sample_u[cur]) * total
+            y = int(np.searchsorted(cdf, target, side="right"))
+            y = min(y, len(R) - 1)
+            lo = cdf[y - 1] if y > 0 else 0.0
+            margins.append(min(abs(target - lo), abs(cdf[y] - target)) / total)
+            accepted_tokens.append(y)
+            break
+    return accepted_tokens, accepted_nodes, margins
