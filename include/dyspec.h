@@ -256,6 +256,40 @@ int dyspec_tree_attention_ragged_sparse(const dyspec_plan_t* plan, const void* q
                                         void* out, void* workspace, size_t workspace_bytes, int32_t* status,
                                         dyspec_stream_t stream);
 
+/*
+ * (5) Verification of the token tree (Algorithm 3: multi-branch rejection sampling along the tree), the
+ * step that follows the tree attention.  For each request the walk starts at node 0; at a node it tries
+ * the node's children in increasing index: child with token y is accepted when u <= R[y] / D[y]
+ * (R starts as the target distribution at the node, D as the draft distribution there); after a
+ * rejection R <- norm(max(R - D, 0)), D[y] <- 0, and the node is given up when D has become all zero,
+ * else D <- norm(D).  When no child is accepted a token is drawn from R and the walk ends.  As the
+ * paper prints it, a walk that reaches a leaf ends without a further token; bonus_at_leaf != 0 draws
+ * the usual extra token from the target distribution at the leaf.  The paper prints the acceptance
+ * number as N(0,1); it is read as U(0,1).  Random numbers are inputs.
+ *
+ *   parents, tokens   dev int32 [N]        N = node_offsets[n_req]; token carried by each node (root's unused)
+ *   draft_probs       dev float [N][vocab] Draft(node, .): what the node's children were drawn from
+ *   target_probs      dev float [N][vocab] Target(node, .)          (rows 16-byte aligned: vocab % 4 == 0)
+ *   accept_u          dev float [N]        U(0,1) number used when that node is tried
+ *   sample_u          dev float [N]        U(0,1) number used when a token is drawn at that node (inverse
+ *                                          CDF in token order: first v with cumsum(R)[v] > u * sum(R))
+ *   node_offsets      dev int32 [n_req+1]  request r owns nodes node_offsets[r] .. node_offsets[r+1]-1
+ *   max_nodes         upper bound of the requests' node counts (<= DYSPEC_MAX_NODES)
+ *   vocab             <= DYSPEC_MAX_VOCAB
+ *   accepted_tokens   dev int32 [n_req][max_out]  (written) the emitted tokens, in order
+ *   accepted_nodes    dev int32 [n_req][max_out]  (written) the accepted node of each, -1 for a drawn token
+ *   n_accepted        dev int32 [n_req]           (written) how many (entries past max_out are dropped)
+ *   status            DYSPEC_ERR_BAD_TREE on a bad parent, DYSPEC_ERR_INVALID_ARG on a token outside the vocabulary
+ * Probabilities are fp32; decisions are taken in fp32 with sums in a different order from a
+ * sequential implementation, so a decision whose deciding number lies within rounding of its
+ * threshold may differ from another implementation's.
+ */
+#define DYSPEC_MAX_VOCAB 32768
+int dyspec_verify_tree(const int32_t* parents, const int32_t* tokens, const float* draft_probs, const float* target_probs,
+                       const float* accept_u, const float* sample_u, const int32_t* node_offsets, int n_req,
+                       int max_nodes, int vocab, int bonus_at_leaf, int32_t* accepted_tokens, int32_t* accepted_nodes,
+                       int32_t* n_accepted, int max_out, int32_t* status, dyspec_stream_t stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -287,9 +287,10 @@ def verify_tree(parents: Sequence[int], tokens: Sequence[int], draft_probs, targ
     bonus_at_leaf=True adds the usual extra token drawn from Target(leaf, .) instead.
 
     Returns (accepted_tokens, accepted_nodes, margins): the token sequence A, the nodes that were
-    accepted (the final, sampled token has no node), and for every decision taken the distance of the
-    deciding number from its threshold (so that a lower-precision implementation can be excused where
-    the decision was a coin toss).
+    accepted (the final, sampled token has no node), and for every decision taken a pair (kind,
+    distance of the deciding number from its threshold): ("accept", |c - R[y]/D[y]|) or ("sample",
+    distance of u from the nearer edge of the drawn token's CDF interval), so that a lower-precision
+    implementation can be excused where the decision was a coin toss.
     """
     check_parents(parents)
     n = len(parents)
@@ -301,7 +302,9 @@ def verify_tree(parents: Sequence[int], tokens: Sequence[int], draft_probs, targ
             children[int(parents[i])].append(i)
     accepted_tokens: List[int] = []
     accepted_nodes: List[int] = []
-    margins: List[float] = []
+    margins: List[tuple] = []
+    if n == 0:
+        return accepted_tokens, accepted_nodes, margins
     cur = 0
     while True:
         if not children[cur] and not bonus_at_leaf:
@@ -314,7 +317,7 @@ def verify_tree(parents: Sequence[int], tokens: Sequence[int], draft_probs, targ
                 y = int(tokens[child])
                 c = float(accept_u[child])
                 ratio = R[y] / D[y] if D[y] > 0 else (np.inf if R[y] > 0 else 0.0)
-                margins.append(abs(c - ratio))
+                margins.append(("accept", abs(c - ratio)))
                 if c <= ratio:
                     accepted_tokens.append(y)
                     accepted_nodes.append(child)
@@ -338,7 +341,7 @@ def verify_tree(parents: Sequence[int], tokens: Sequence[int], draft_probs, targ
             y = int(np.searchsorted(cdf, target, side="right"))
             y = min(y, len(R) - 1)
             lo = cdf[y - 1] if y > 0 else 0.0
-            margins.append(min(abs(target - lo), abs(cdf[y] - target)) / total)
+            margins.append(("sample", min(abs(target - lo), abs(cdf[y] - target)) / total))
             accepted_tokens.append(y)
             break
     return accepted_tokens, accepted_nodes, margins

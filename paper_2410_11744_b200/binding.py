@@ -47,6 +47,7 @@ SIGNATURES = {
     "dyspec_plan_build_tree_mask_tiles": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "dyspec_mask_block_count": (_i32, [_vp, _i32, _i32, _i32, _vp, _vp]),
     "dyspec_tree_attention_ragged_sparse": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp, _vp]),
+    "dyspec_verify_tree": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _i32, _vp, _vp]),
     "dyspec_tree_attention_static": (_i32, [_vp, _vp, _vp, _i32, _vp, _i32, _vp, _i32, _i32, _i32, _i32, _f32, _vp, _vp]),
 }
 for _name, (_res, _args) in SIGNATURES.items():
@@ -267,3 +268,13 @@ def dyspec_tree_attention_ragged_sparse(plan: Plan, q, k_cache, v_cache, ancesto
                                                    _ptr(ancestor_bits), _ptr(node_tiles), _ptr(out), _ptr(workspace),
                                                    workspace_bytes, _ptr(status), _stream(stream)),
            "dyspec_tree_attention_ragged_sparse")
+
+
+def dyspec_verify_tree(parents, tokens, draft_probs, target_probs, accept_u, sample_u, node_offsets, n_req: int,
+                       max_nodes: int, vocab: int, accepted_tokens, accepted_nodes, n_accepted, max_out: int,
+                       bonus_at_leaf: bool = False, status=None, stream=None) -> None:
+    """Tree verification (Algorithm 3) for n_req requests; all arrays are device tensors (see include/dyspec.h)."""
+    _check(lib.dyspec_verify_tree(_ptr(parents), _ptr(tokens), _ptr(draft_probs), _ptr(target_probs), _ptr(accept_u),
+                                  _ptr(sample_u), _ptr(node_offsets), n_req, max_nodes, vocab, int(bool(bonus_at_leaf)),
+                                  _ptr(accepted_tokens), _ptr(accepted_nodes), _ptr(n_accepted), max_out, _ptr(status),
+                                  _stream(stream)), "dyspec_verify_tree")

@@ -22,6 +22,11 @@ cudaError_t launch_dfs_reorder(const int32_t* parents, const ReqInfo* reqs, int 
                                cudaStream_t stream);
 cudaError_t launch_mask_block_count(const uint32_t* bits, int n, int W, int block, unsigned long long* count,
                                     cudaStream_t stream);
+cudaError_t launch_verify_tree(const int32_t* parents, const int32_t* tokens, const float* draft_probs,
+                               const float* target_probs, const float* accept_u, const float* sample_u,
+                               const int32_t* node_offsets, int n_req, int max_nodes, int vocab, int bonus_at_leaf,
+                               int32_t* out_tokens, int32_t* out_nodes, int32_t* out_count, int max_out, int32_t* status,
+                               cudaStream_t stream);
 cudaError_t launch_attn_mma(int head_dim, int n_ctas, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                             const AttnParams& p, cudaStream_t stream);
 cudaError_t launch_combine(int head_dim, int bm, int n_split_groups, const AttnParams& p, cudaStream_t stream);
@@ -400,6 +405,23 @@ int dyspec_mask_block_count(const uint32_t* ancestor_bits, int n_nodes, int word
   cudaError_t e = launch_mask_block_count(ancestor_bits, n_nodes, words_per_row, block,
                                           reinterpret_cast<unsigned long long*>(count), reinterpret_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? DYSPEC_OK : DYSPEC_ERR_CUDA;
+}
+
+int dyspec_verify_tree(const int32_t* parents, const int32_t* tokens, const float* draft_probs, const float* target_probs,
+                       const float* accept_u, const float* sample_u, const int32_t* node_offsets, int n_req,
+                       int max_nodes, int vocab, int bonus_at_leaf, int32_t* accepted_tokens, int32_t* accepted_nodes,
+                       int32_t* n_accepted, int max_out, int32_t* status, dyspec_stream_t stream) {
+  if (n_req < 0 || max_nodes < 0 || vocab <= 0 || (vocab & 3) || max_out <= 0) return DYSPEC_ERR_INVALID_ARG;
+  if (max_nodes > DYSPEC_MAX_NODES || vocab > DYSPEC_MAX_VOCAB) return DYSPEC_ERR_UNSUPPORTED;
+  if (n_req == 0) return DYSPEC_OK;
+  if (!parents || !tokens || !draft_probs || !target_probs || !accept_u || !sample_u || !node_offsets ||
+      !accepted_tokens || !accepted_nodes || !n_accepted)
+    return DYSPEC_ERR_INVALID_ARG;
+  if (!aligned(draft_probs, 16) || !aligned(target_probs, 16)) return DYSPEC_ERR_INVALID_ARG;
+  cudaError_t e = launch_verify_tree(parents, tokens, draft_probs, target_probs, accept_u, sample_u, node_offsets, n_req,
+                                     max_nodes, vocab, bonus_at_leaf, accepted_tokens, accepted_nodes, n_accepted, max_out,
+                                     status, reinterpret_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? DYSPEC_OK : cuda_failed(e, "verify launch");
 }
 
 // Validates the arguments and runs the scheduler; no CUDA call.

@@ -212,3 +212,59 @@ def permute_tree_tokens(w: Workload, orders: List[np.ndarray], new_parents: List
     return Workload(w.name + "_reordered", w.n_q_heads, w.n_kv_heads, w.head_dim, w.prefix_len.copy(), w.n_nodes.copy(),
                     [np.asarray(p, dtype=np.int32) for p in new_parents], q, k, v, w.kv_row_offset.copy(),
                     dict(w.meta, reordered=True))
+
+
+@dataclass
+class VerifyCase:
+    """Inputs of the tree verification (Algorithm 3) for a ragged batch: all arrays host-side numpy."""
+    name: str
+    vocab: int
+    node_offsets: np.ndarray        # int32 [n_req + 1]
+    parents: List[np.ndarray]       # per request int32 [n]
+    tokens: List[np.ndarray]        # per request int32 [n]: token carried by each node (root: 0)
+    draft_probs: np.ndarray         # float32 [N][vocab]
+    target_probs: np.ndarray        # float32 [N][vocab]
+    accept_u: np.ndarray            # float32 [N]
+    sample_u: np.ndarray            # float32 [N]
+
+
+def _softmax_rows(x: np.ndarray) -> np.ndarray:
+    x = x - x.max(axis=1, keepdims=True)
+    e = np.exp(x)
+    return (e / e.sum(axis=1, keepdims=True)).astype(np.float32)
+
+
+def make_verify_case(seed: int, vocab: int, parents_list, sharpness: float = 4.0, disagreement: float = 1.0,
+                     same: bool = False, name: str = "verify") -> VerifyCase:
+    """Draft rows = softmax(sharpness * N(0,1) logits); target rows = softmax of the same logits plus
+    disagreement * N(0,1) noise (same=True: identical rows).  The children of a node carry tokens drawn
+    from the node's draft row without replacement, in child order, which is how a draft tree comes
+    about (Sec. 4.1); when the row runs out of mass the remaining children get unused tokens."""
+    rng = np.random.default_rng(seed)
+    offs = np.concatenate([[0], np.cumsum([len(p) for p in parents_list])]).astype(np.int32)
+    N = int(offs[-1])
+    logits = rng.standard_normal((N, vocab)).astype(np.float32) * np.float32(sharpness)
+    draft = _softmax_rows(logits)
+    target = draft.copy() if same else _softmax_rows(logits + np.float32(disagreement) * rng.standard_normal((N, vocab)).astype(np.float32))
+    tokens = []
+    for r, parents in enumerate(parents_list):
+        n = len(parents)
+        tok = np.zeros(n, dtype=np.int32)
+        children = [[] for _ in range(n)]
+        for i in range(1, n):
+            if parents[i] >= 0:
+                children[int(parents[i])].append(i)
+        for u in range(n):
+            if not children[u]:
+                continue
+            d = draft[offs[r] + u].astype(np.float64).copy()
+            for c in children[u]:
+                if d.sum() > 0:
+                    y = int(rng.choice(vocab, p=d / d.sum()))
+                else:
+                    y = int(np.flatnonzero(draft[offs[r] + u] == 0)[0]) if (draft[offs[r] + u] == 0).any() else 0
+                tok[c] = y
+                d[y] = 0.0
+        tokens.append(tok)
+    return VerifyCase(name, vocab, offs, [np.asarray(p, np.int32) for p in parents_list], tokens, draft, target,
+                      rng.random(N, dtype=np.float32), rng.random(N, dtype=np.float32))

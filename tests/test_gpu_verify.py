@@ -1,0 +1,118 @@
+"""GPU parity of the tree verification kernel (Algorithm 3) with the oracle.  Accepted nodes and
+emitted tokens must match exactly; a request is excused only where the oracle reports that a deciding
+number lay within rounding of its threshold (1e-4 for an acceptance ratio, 3e-6 of the total mass for
+the inverse CDF): fp32 sums in another order may then fall the other way."""
+import numpy as np
+import pytest
+
+from oracle import dyspec_oracle as orc
+from paper_2410_11744_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+EPS = {"accept": 1e-4, "sample": 3e-6}      # ratios are O(1); the CDF is a sum of <= 32768 fp32 terms of total 1
+
+
+@pytest.fixture(scope="module")
+def B():
+    import torch
+    assert torch.cuda.is_available()
+    from paper_2410_11744_b200 import build
+    build.build()
+    from paper_2410_11744_b200 import binding
+    return binding
+
+
+def run_gpu(B, case, bonus=False, max_out=64):
+    import torch
+    dev = "cuda:0"
+    t = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(dev)
+    n_req = len(case.parents)
+    parents = t(np.concatenate(case.parents) if n_req else np.zeros(0, np.int32))
+    tokens = t(np.concatenate(case.tokens) if n_req else np.zeros(0, np.int32))
+    out_t = torch.full((max(1, n_req), max_out), -9, dtype=torch.int32, device=dev)
+    out_n = torch.full((max(1, n_req), max_out), -9, dtype=torch.int32, device=dev)
+    cnt = torch.full((max(1, n_req),), -9, dtype=torch.int32, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    max_nodes = max([len(p) for p in case.parents] + [0])
+    B.dyspec_verify_tree(parents, tokens, t(case.draft_probs), t(case.target_probs), t(case.accept_u), t(case.sample_u),
+                         t(case.node_offsets), n_req, max_nodes, case.vocab, out_t, out_n, cnt, max_out,
+                         bonus_at_leaf=bonus, status=status)
+    torch.cuda.synchronize()
+    return out_t.cpu().numpy(), out_n.cpu().numpy(), cnt.cpu().numpy(), int(status.item())
+
+
+def check(B, case, bonus=False, max_excused=0.25):
+    out_t, out_n, cnt, status = run_gpu(B, case, bonus)
+    assert status == 0
+    excused = 0
+    offs = case.node_offsets
+    for r in range(len(case.parents)):
+        sl = slice(offs[r], offs[r + 1])
+        A, nodes, margins = orc.verify_tree(case.parents[r], case.tokens[r], case.draft_probs[sl], case.target_probs[sl],
+                                            case.accept_u[sl], case.sample_u[sl], bonus_at_leaf=bonus)
+        if any(m < EPS[kind] for kind, m in margins):
+            excused += 1
+            continue
+        k = int(cnt[r])
+        assert k == len(A), (r, k, A)
+        assert out_t[r, :k].tolist() == A
+        want_nodes = nodes + [-1] * (len(A) - len(nodes))
+        assert out_n[r, :k].tolist() == want_nodes
+    assert excused <= max_excused * max(1, len(case.parents))
+    return excused
+
+
+@pytest.mark.parametrize("vocab,disagreement", [(32000, 1.0), (32000, 0.3), (32768, 2.0), (1000, 1.0), (4096, 0.5), (8, 1.0)])
+def test_verify_matches_oracle(B, vocab, disagreement):
+    rng = np.random.default_rng(vocab + int(disagreement * 10))
+    trees = [wl.greedy_tree(rng, 64, 8, 0.3), wl.greedy_tree(rng, 40, 4, 0.5), wl.chain_tree(12), wl.random_tree(rng, 33)]
+    if vocab == 8:
+        trees = [wl.greedy_tree(rng, 20, 3, 0.5), wl.chain_tree(5), wl.random_tree(rng, 9)]
+    case = wl.make_verify_case(7 + vocab, vocab, trees, sharpness=3.0 if vocab > 100 else 1.0, disagreement=disagreement)
+    for bonus in (False, True):
+        check(B, case, bonus)
+
+
+def test_verify_many_requests_and_rejections(B):
+    """Flat draft rows and a target that disagrees: long runs of rejections, some down to the all-zero exit."""
+    rng = np.random.default_rng(3)
+    trees = [wl.greedy_tree(rng, int(rng.integers(2, 60)), 6, 1.0) for _ in range(40)]
+    trees.append(np.concatenate([[-1], np.zeros(15, np.int32)]).astype(np.int32))      # 15 branches at the root
+    case = wl.make_verify_case(5, 16, trees, sharpness=0.5, disagreement=3.0)
+    check(B, case, bonus=False, max_excused=0.3)
+    check(B, case, bonus=True, max_excused=0.3)
+
+
+def test_verify_draft_equal_to_target_walks_first_branches(B):
+    rng = np.random.default_rng(9)
+    trees = [wl.greedy_tree(rng, 64, 8, 0.3), wl.chain_tree(30)]
+    case = wl.make_verify_case(2, 32000, trees, same=True)
+    out_t, out_n, cnt, status = run_gpu(B, case, bonus=True)
+    assert status == 0
+    for r, parents in enumerate(case.parents):
+        node, path = 0, []
+        while True:
+            ch = [i for i in range(1, len(parents)) if parents[i] == node]
+            if not ch:
+                break
+            node = ch[0]
+            path.append(node)
+        k = int(cnt[r])
+        assert out_n[r, :k].tolist() == path + [-1]
+        assert out_t[r, :k - 1].tolist() == [int(case.tokens[r][i]) for i in path]
+
+
+def test_verify_large_tree_small_vocab_and_empty_request(B):
+    rng = np.random.default_rng(4)
+    trees = [wl.random_tree(rng, 2048), np.zeros(0, np.int32), np.array([-1], np.int32), wl.greedy_tree(rng, 768, 8, 0.05)]
+    case = wl.make_verify_case(11, 64, trees, sharpness=1.0, disagreement=0.5)
+    check(B, case, bonus=False)
+    check(B, case, bonus=True)
+
+
+def test_verify_reports_bad_token(B):
+    rng = np.random.default_rng(1)
+    case = wl.make_verify_case(3, 16, [wl.chain_tree(4)])
+    case.tokens[0][1] = 99
+    _, _, _, status = run_gpu(B, case)
+    assert status == -1
