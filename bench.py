@@ -278,6 +278,52 @@ def random_tree_experiment(torch, runner, workloads, B, peaks, device, sizes=(25
     return rows
 
 
+def verification_experiment(torch, workloads, B, peaks, device):
+    """Tree verification (Algorithm 3) on the device: Llama2 vocabulary (32000), the 64-node tree shape of
+    config 2 for one request (the paper's batch size) and a batch of 8 requests with 256-node trees.
+    Inputs rotate over copies that exceed 2x L2; algorithmic bytes = the draft and target rows of the
+    visited nodes."""
+    rows = []
+    rng = np.random.default_rng(workloads.MASTER_SEED + 7000)
+    for label, trees in (("1 request, 64 nodes", [workloads.greedy_tree(rng, 64, 8, 0.3)]),
+                         ("8 requests, 256 nodes", [workloads.greedy_tree(rng, 256, 8, 0.1) for _ in range(8)])):
+        case = workloads.make_verify_case(workloads.MASTER_SEED + 7001, 32000, trees, sharpness=3.0, disagreement=1.0)
+        n_req = len(trees)
+        N = int(case.node_offsets[-1])
+        row_bytes = 2 * N * case.vocab * 4
+        copies = max(2, min(32, int(np.ceil(2.0 * L2_BYTES / row_bytes))))
+        t = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(device)
+        parents, tokens = t(np.concatenate(case.parents)), t(np.concatenate(case.tokens))
+        offs, au, su = t(case.node_offsets), t(case.accept_u), t(case.sample_u)
+        bufs = [(t(case.draft_probs), t(case.target_probs)) for _ in range(copies)]
+        out_t = torch.zeros((n_req, 64), dtype=torch.int32, device=device)
+        out_n = torch.zeros((n_req, 64), dtype=torch.int32, device=device)
+        cnt = torch.zeros((n_req,), dtype=torch.int32, device=device)
+        status = torch.zeros(1, dtype=torch.int32, device=device)
+        max_nodes = max(len(p) for p in trees)
+
+        def call(d, tg):
+            B.dyspec_verify_tree(parents, tokens, d, tg, au, su, offs, n_req, max_nodes, case.vocab, out_t, out_n, cnt, 64,
+                                 bonus_at_leaf=True, status=status)
+        for d, tg in bufs:
+            call(d, tg)
+        torch.cuda.synchronize()
+        g = _graph_of(torch, lambda: [call(d, tg) for d, tg in bufs])
+        g.replay()
+        torch.cuda.synchronize()
+        us = _time_replays(torch, g, 20) / (20 * copies) * 1e3
+        emitted = cnt.cpu().numpy()
+        visited = int(emitted.sum())                       # nodes whose rows were read: accepted ones + the start node - ... = tokens emitted
+        nbytes = visited * 2 * case.vocab * 4
+        rows.append({"case": label, "vocab": case.vocab, "call_us": us, "tokens_emitted": emitted.tolist(),
+                     "rows_read": visited, "bytes": nbytes, "achieved_gbs": nbytes / (us * 1e-6) / 1e9,
+                     "frac_of_hbm": nbytes / (us * 1e-6) / 1e9 / peaks["hbm_gbs"], "copies": copies,
+                     "status": int(status.item())})
+        del bufs
+        torch.cuda.empty_cache()
+    return rows
+
+
 def roofline_entry(m, peaks, peaks_kind):
     t_hbm = m["bytes"] / (peaks["hbm_gbs"] * 1e9)
     t_tc = m["flops"] / (peaks["bf16_tflops"] * 1e12)
@@ -411,6 +457,10 @@ def run_ours(args):
         from paper_2410_11744_b200 import binding
         random_tree = random_tree_experiment(torch, runner, workloads, binding, peaks, device)
 
+    verification = None
+    if not args.no_per_config and world == 1:
+        verification = verification_experiment(torch, workloads, binding, peaks, device)
+
     # ---- the oracle on the host cores, bounded sample of the same workload
     times = time_oracle(w, budget_s=12.0)
     cpu_sec = sum(times) / len(times)
@@ -439,6 +489,8 @@ def run_ours(args):
         line["per_config"] = per_config
     if random_tree:
         line["random_tree_experiment"] = random_tree
+    if verification:
+        line["verification_experiment"] = verification
     print(json.dumps(line), flush=True)
     if use_dist:
         dist.barrier()
