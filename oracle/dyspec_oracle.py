@@ -29,7 +29,11 @@ tests/test_reorder_pins.py (the block counts the paper prints in Table 5,
 closed forms, a hand example, subtree contiguity, attention invariance);
 verify_tree (Algorithm 3) by tests/test_verify_pins.py (the output distribution
 equals the target's, Draft == Target accepts every first branch, closed-form
-acceptance rates, forced rejections, the all-zero early exit).
+acceptance rates, forced rejections, the all-zero early exit); the tree
+construction (Algorithms 1 and 2) by tests/test_construct_pins.py (values
+decrease, the closed form of the estimated acceptance rate in raw draft
+probabilities, Algorithm 2 at the last value == Algorithm 1, guesses at a
+position are draws without replacement).
 Nothing here is "parity unpinned".
 
 Readings where the paper is silent: scale = 1/sqrt(head_dim); consecutive query
@@ -38,7 +42,9 @@ masks are packed LSB-first in uint32 words; the DFS renumbering visits roots
 and children in increasing index (the order that reproduces Table 5);
 Algorithm 3 draws its acceptance number from U(0,1) (printed as N(0,1)), the
 branches of a node are its children in increasing index, and the final token
-is drawn from the residual by inverse CDF in token order.
+is drawn from the residual by inverse CDF in token order; Algorithm 1 samples
+the token before it adds the node, Algorithm 2 expands while v >= t, the draft
+model is a table lookup keyed by tree position (see build_tree_greedy).
 """
 from __future__ import annotations
 
@@ -345,3 +351,115 @@ def verify_tree(parents: Sequence[int], tokens: Sequence[int], draft_probs, targ
             accepted_tokens.append(y)
             break
     return accepted_tokens, accepted_nodes, margins
+
+
+# ----------------------------------------------------------------------------------------------------
+# Construction of the draft token tree (Sec. 4.1-4.3, Algorithm 1; App. B, Algorithm 2).
+#
+# The draft model is abstracted as a table: the distribution that follows a tree position is a row of
+# `rows`, chosen by a fixed integer function of the position (row of the parent, token), and the
+# uniform number used by the j-th sampling at a position is an entry of `uniforms` chosen the same way.
+# Both algorithms therefore see the same distribution and draw the same token for the same (position,
+# attempt), which is what makes the paper's statement "with the threshold set to the value of the last
+# node, Algorithm 2 gives exactly the tree of Algorithm 1" checkable.
+# ----------------------------------------------------------------------------------------------------
+def draft_row_of_child(parent_row: int, token: int, n_rows: int) -> int:
+    return ((parent_row * 2654435761 + (token + 1) * 40503) % (1 << 32)) % n_rows
+
+
+def draft_uniform_index(row: int, attempt: int, n_uniforms: int) -> int:
+    return ((row * 7919 + attempt * 104729 + 17) % (1 << 32)) % n_uniforms
+
+
+def _sample_residual(raw_row: np.ndarray, taken: List[int], u: float):
+    """Draws from norm(raw_row with the `taken` tokens zeroed) by inverse CDF in token order.
+    Returns (token, its probability under that residual, margin of u from the CDF interval's edges)."""
+    res = raw_row.astype(np.float64).copy()
+    res[taken] = 0.0
+    total = res.sum()
+    cdf = np.cumsum(res)
+    target = float(u) * total
+    y = int(np.searchsorted(cdf, target, side="right"))
+    y = min(y, len(res) - 1)
+    lo = cdf[y - 1] if y > 0 else 0.0
+    margin = min(abs(target - lo), abs(cdf[y] - target)) / total if total > 0 else 0.0
+    return y, (res[y] / total if total > 0 else 0.0), margin
+
+
+def build_tree_greedy(rows, uniforms, m: int):
+    """Algorithm 1: the tree of the m guesses with the largest estimated acceptance rate.
+
+    A slot (v, position, attempt) stands for "the next sampling at this position"; the slot with the
+    largest v is taken (ties: the one pushed first), a token is sampled from the position's residual
+    distribution (the printed listing adds the node one line before it samples the token: read in the
+    order that makes sense), the node is created, and two slots are pushed: the next sampling at the
+    same position with v (1 - R[y]) and the first sampling under the new node with v R[y].
+
+    Returns dict(parents, tokens, values, child_values, rows, margins): node 0 is the root (the last
+    prompt token; value 1); values[k] is the slot value node k was created from, child_values[k] the
+    value of the first sampling under it; margins as in verify_tree, plus ("order", gap between the
+    best and the second best slot value, relative)."""
+    rows = np.asarray(rows)
+    T, Tu = rows.shape[0], len(uniforms)
+    parents, tokens, values, child_values, node_rows = [-1], [0], [1.0], [1.0], [0]
+    taken: List[List[int]] = [[]]
+    slots = [(1.0, 0, 0)]                      # (v, position, attempt), in push order
+    margins: List[tuple] = []
+    while len(parents) - 1 < m and slots:
+        best = max(range(len(slots)), key=lambda i: (slots[i][0], -i))
+        if len(slots) > 1:
+            second = max(s[0] for i, s in enumerate(slots) if i != best)
+            margins.append(("order", (slots[best][0] - second) / max(slots[best][0], 1e-300)))
+        v, pos, attempt = slots.pop(best)
+        u = uniforms[draft_uniform_index(node_rows[pos], attempt, Tu)]
+        y, r, mg = _sample_residual(rows[node_rows[pos]], taken[pos], u)
+        margins.append(("sample", mg))
+        k = len(parents)
+        parents.append(pos); tokens.append(y); values.append(v); child_values.append(v * r)
+        node_rows.append(draft_row_of_child(node_rows[pos], y, T))
+        taken.append([])
+        taken[pos].append(y)
+        if 1.0 - r > 0.0:
+            slots.append((v * (1.0 - r), pos, attempt + 1))
+        slots.append((v * r, k, 0))
+    return dict(parents=np.asarray(parents, np.int32), tokens=np.asarray(tokens, np.int32),
+                values=np.asarray(values), child_values=np.asarray(child_values),
+                rows=np.asarray(node_rows, np.int32), margins=margins)
+
+
+def build_tree_threshold(rows, uniforms, threshold: float, max_nodes: int):
+    """Algorithm 2: layer by layer, every position keeps sampling while its estimated acceptance rate
+    is at least `threshold` (the printed loop condition `v < t` would expand exactly the guesses the
+    text says to drop: read `v >= t`).  Stops early when max_nodes guesses exist.  Same return value as
+    build_tree_greedy (node order: by layer, then by parent, then by sampling order)."""
+    rows = np.asarray(rows)
+    T, Tu = rows.shape[0], len(uniforms)
+    parents, tokens, values, child_values, node_rows = [-1], [0], [1.0], [1.0], [0]
+    margins: List[tuple] = []
+    leaves = [0]
+    while leaves and len(parents) - 1 < max_nodes:
+        new_leaves = []
+        for node in leaves:
+            v = child_values[node]
+            taken: List[int] = []
+            attempt = 0
+            while v >= threshold and len(parents) - 1 < max_nodes:
+                margins.append(("threshold", abs(v - threshold) / max(threshold, 1e-300)))
+                u = uniforms[draft_uniform_index(node_rows[node], attempt, Tu)]
+                y, r, mg = _sample_residual(rows[node_rows[node]], taken, u)
+                margins.append(("sample", mg))
+                k = len(parents)
+                parents.append(node); tokens.append(y); values.append(v); child_values.append(v * r)
+                node_rows.append(draft_row_of_child(node_rows[node], y, T))
+                new_leaves.append(k)
+                taken.append(y)
+                v = v * (1.0 - r)
+                attempt += 1
+                if not (1.0 - r > 0.0):
+                    break
+            if v < threshold:
+                margins.append(("threshold", abs(v - threshold) / max(threshold, 1e-300)))
+        leaves = new_leaves
+    return dict(parents=np.asarray(parents, np.int32), tokens=np.asarray(tokens, np.int32),
+                values=np.asarray(values), child_values=np.asarray(child_values),
+                rows=np.asarray(node_rows, np.int32), margins=margins)
