@@ -290,6 +290,42 @@ int dyspec_verify_tree(const int32_t* parents, const int32_t* tokens, const floa
                        int max_nodes, int vocab, int bonus_at_leaf, int32_t* accepted_tokens, int32_t* accepted_nodes,
                        int32_t* n_accepted, int max_out, int32_t* status, dyspec_stream_t stream);
 
+/*
+ * (6) Construction of the draft token tree (Sec. 4.1-4.3, Algorithm 1; App. B, Algorithm 2), the step
+ * before the tree attention.  The paper runs it on the CPU between draft-model calls; here the draft
+ * model is represented by a table so that the whole loop runs in one launch: the distribution that
+ * follows a tree position is row  (row(parent) * 2654435761 + (token + 1) * 40503  mod 2^32) mod n_rows
+ * of draft_table (the root's row is root_row[r]), and the uniform number of the j-th sampling at a
+ * position is uniforms[(row * 7919 + j * 104729 + 17  mod 2^32) mod n_uniforms].  A real draft model
+ * replaces the table by its own calls; the arithmetic per node is the same.
+ *
+ * greedy (Algorithm 1): repeat m times: take the expandable slot with the largest estimated
+ * acceptance rate v (ties: the one opened first), draw a token y from the residual distribution R at
+ * that position (inverse CDF in token order), add the node, open the slots (v (1 - R[y]), same
+ * position, next attempt) and (v R[y], first sampling under the new node).  (The printed listing
+ * adds the node one line before it samples the token: read in the order that makes sense.)
+ * threshold (Algorithm 2): layer by layer, every position keeps drawing while v >= threshold (the
+ * listing prints `v < t`; the text says the guesses above the threshold are the ones kept), until
+ * max_nodes guesses exist.  With threshold = values[m] of the greedy tree it builds the same tree.
+ *
+ *   draft_table   dev float [n_rows][vocab]   (rows 16-byte aligned: vocab % 4 == 0, vocab <= DYSPEC_MAX_VOCAB)
+ *   uniforms      dev float [n_uniforms]      U(0,1) numbers
+ *   root_row      dev int32 [n_req]
+ *   outputs, stride S = m + 1 (greedy) or max_nodes + 1 (threshold) per request, node 0 = the root:
+ *   parents, tokens, rows  dev int32 [n_req][S];  values, child_values  dev float [n_req][S]
+ *                 values[k] = the estimated acceptance rate node k was created with, child_values[k] =
+ *                 that of the first sampling under it;  n_nodes dev int32 [n_req] = nodes incl. the root
+ * m, max_nodes <= DYSPEC_MAX_NODES - 1.  Values are fp32; as for dyspec_verify_tree, a choice between
+ * numbers closer than rounding may fall differently from another implementation's.
+ */
+int dyspec_build_tree_greedy(const float* draft_table, int n_rows, int vocab, const float* uniforms, int n_uniforms,
+                             const int32_t* root_row, int n_req, int m, int32_t* parents, int32_t* tokens, float* values,
+                             float* child_values, int32_t* rows, int32_t* n_nodes, dyspec_stream_t stream);
+int dyspec_build_tree_threshold(const float* draft_table, int n_rows, int vocab, const float* uniforms, int n_uniforms,
+                                const int32_t* root_row, int n_req, float threshold, int max_nodes, int32_t* parents,
+                                int32_t* tokens, float* values, float* child_values, int32_t* rows, int32_t* n_nodes,
+                                dyspec_stream_t stream);
+
 #ifdef __cplusplus
 }
 #endif

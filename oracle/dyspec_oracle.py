@@ -386,7 +386,7 @@ def _sample_residual(raw_row: np.ndarray, taken: List[int], u: float):
     return y, (res[y] / total if total > 0 else 0.0), margin
 
 
-def build_tree_greedy(rows, uniforms, m: int):
+def build_tree_greedy(rows, uniforms, m: int, root_row: int = 0):
     """Algorithm 1: the tree of the m guesses with the largest estimated acceptance rate.
 
     A slot (v, position, attempt) stands for "the next sampling at this position"; the slot with the
@@ -401,7 +401,7 @@ def build_tree_greedy(rows, uniforms, m: int):
     best and the second best slot value, relative)."""
     rows = np.asarray(rows)
     T, Tu = rows.shape[0], len(uniforms)
-    parents, tokens, values, child_values, node_rows = [-1], [0], [1.0], [1.0], [0]
+    parents, tokens, values, child_values, node_rows = [-1], [0], [1.0], [1.0], [int(root_row) % rows.shape[0]]
     taken: List[List[int]] = [[]]
     slots = [(1.0, 0, 0)]                      # (v, position, attempt), in push order
     margins: List[tuple] = []
@@ -427,14 +427,14 @@ def build_tree_greedy(rows, uniforms, m: int):
                 rows=np.asarray(node_rows, np.int32), margins=margins)
 
 
-def build_tree_threshold(rows, uniforms, threshold: float, max_nodes: int):
+def build_tree_threshold(rows, uniforms, threshold: float, max_nodes: int, root_row: int = 0):
     """Algorithm 2: layer by layer, every position keeps sampling while its estimated acceptance rate
     is at least `threshold` (the printed loop condition `v < t` would expand exactly the guesses the
     text says to drop: read `v >= t`).  Stops early when max_nodes guesses exist.  Same return value as
     build_tree_greedy (node order: by layer, then by parent, then by sampling order)."""
     rows = np.asarray(rows)
     T, Tu = rows.shape[0], len(uniforms)
-    parents, tokens, values, child_values, node_rows = [-1], [0], [1.0], [1.0], [0]
+    parents, tokens, values, child_values, node_rows = [-1], [0], [1.0], [1.0], [int(root_row) % rows.shape[0]]
     margins: List[tuple] = []
     leaves = [0]
     while leaves and len(parents) - 1 < max_nodes:

@@ -48,6 +48,8 @@ SIGNATURES = {
     "dyspec_mask_block_count": (_i32, [_vp, _i32, _i32, _i32, _vp, _vp]),
     "dyspec_tree_attention_ragged_sparse": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp, _vp]),
     "dyspec_verify_tree": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _i32, _vp, _vp]),
+    "dyspec_build_tree_greedy": (_i32, [_vp, _i32, _i32, _vp, _i32, _vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "dyspec_build_tree_threshold": (_i32, [_vp, _i32, _i32, _vp, _i32, _vp, _i32, _f32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "dyspec_tree_attention_static": (_i32, [_vp, _vp, _vp, _i32, _vp, _i32, _vp, _i32, _i32, _i32, _i32, _f32, _vp, _vp]),
 }
 for _name, (_res, _args) in SIGNATURES.items():
@@ -278,3 +280,21 @@ def dyspec_verify_tree(parents, tokens, draft_probs, target_probs, accept_u, sam
                                   _ptr(sample_u), _ptr(node_offsets), n_req, max_nodes, vocab, int(bool(bonus_at_leaf)),
                                   _ptr(accepted_tokens), _ptr(accepted_nodes), _ptr(n_accepted), max_out, _ptr(status),
                                   _stream(stream)), "dyspec_verify_tree")
+
+
+def dyspec_build_tree_greedy(draft_table, n_rows: int, vocab: int, uniforms, n_uniforms: int, root_row, n_req: int, m: int,
+                             parents, tokens, values, child_values, rows, n_nodes, stream=None) -> None:
+    """Algorithm 1 over a table-lookup draft model; outputs are device tensors [n_req][m + 1] (see include/dyspec.h)."""
+    _check(lib.dyspec_build_tree_greedy(_ptr(draft_table), n_rows, vocab, _ptr(uniforms), n_uniforms, _ptr(root_row), n_req,
+                                        m, _ptr(parents), _ptr(tokens), _ptr(values), _ptr(child_values), _ptr(rows),
+                                        _ptr(n_nodes), _stream(stream)), "dyspec_build_tree_greedy")
+
+
+def dyspec_build_tree_threshold(draft_table, n_rows: int, vocab: int, uniforms, n_uniforms: int, root_row, n_req: int,
+                                threshold: float, max_nodes: int, parents, tokens, values, child_values, rows, n_nodes,
+                                stream=None) -> None:
+    """Algorithm 2 over a table-lookup draft model; outputs are device tensors [n_req][max_nodes + 1]."""
+    _check(lib.dyspec_build_tree_threshold(_ptr(draft_table), n_rows, vocab, _ptr(uniforms), n_uniforms, _ptr(root_row),
+                                           n_req, float(threshold), max_nodes, _ptr(parents), _ptr(tokens), _ptr(values),
+                                           _ptr(child_values), _ptr(rows), _ptr(n_nodes), _stream(stream)),
+           "dyspec_build_tree_threshold")

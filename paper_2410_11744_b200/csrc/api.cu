@@ -27,6 +27,14 @@ cudaError_t launch_verify_tree(const int32_t* parents, const int32_t* tokens, co
                                const int32_t* node_offsets, int n_req, int max_nodes, int vocab, int bonus_at_leaf,
                                int32_t* out_tokens, int32_t* out_nodes, int32_t* out_count, int max_out, int32_t* status,
                                cudaStream_t stream);
+cudaError_t launch_build_tree_greedy(const float* draft_table, int n_rows, int vocab, const float* uniforms, int n_uniforms,
+                                     const int32_t* root_row, int n_req, int m, int32_t* parents, int32_t* tokens,
+                                     float* values, float* child_values, int32_t* rows, int32_t* n_nodes,
+                                     cudaStream_t stream);
+cudaError_t launch_build_tree_threshold(const float* draft_table, int n_rows, int vocab, const float* uniforms,
+                                        int n_uniforms, const int32_t* root_row, int n_req, float threshold, int max_nodes,
+                                        int32_t* parents, int32_t* tokens, float* values, float* child_values, int32_t* rows,
+                                        int32_t* n_nodes, cudaStream_t stream);
 cudaError_t launch_attn_mma(int head_dim, int n_ctas, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                             const AttnParams& p, cudaStream_t stream);
 cudaError_t launch_combine(int head_dim, int bm, int n_split_groups, const AttnParams& p, cudaStream_t stream);
@@ -422,6 +430,43 @@ int dyspec_verify_tree(const int32_t* parents, const int32_t* tokens, const floa
                                      max_nodes, vocab, bonus_at_leaf, accepted_tokens, accepted_nodes, n_accepted, max_out,
                                      status, reinterpret_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? DYSPEC_OK : cuda_failed(e, "verify launch");
+}
+
+static int check_tree_build_args(const float* draft_table, int n_rows, int vocab, const float* uniforms, int n_uniforms,
+                                 const int32_t* root_row, int n_req, int nodes, const void* parents, const void* tokens,
+                                 const void* values, const void* child_values, const void* rows, const void* n_nodes) {
+  if (n_rows <= 0 || vocab <= 0 || (vocab & 3) || n_uniforms <= 0 || n_req < 0 || nodes < 0) return DYSPEC_ERR_INVALID_ARG;
+  if (vocab > DYSPEC_MAX_VOCAB || nodes > DYSPEC_MAX_NODES - 1) return DYSPEC_ERR_UNSUPPORTED;
+  if (n_req == 0) return DYSPEC_OK;
+  if (!draft_table || !uniforms || !root_row || !parents || !tokens || !values || !child_values || !rows || !n_nodes)
+    return DYSPEC_ERR_INVALID_ARG;
+  if (!aligned(draft_table, 16)) return DYSPEC_ERR_INVALID_ARG;
+  return DYSPEC_OK;
+}
+
+int dyspec_build_tree_greedy(const float* draft_table, int n_rows, int vocab, const float* uniforms, int n_uniforms,
+                             const int32_t* root_row, int n_req, int m, int32_t* parents, int32_t* tokens, float* values,
+                             float* child_values, int32_t* rows, int32_t* n_nodes, dyspec_stream_t stream) {
+  const int rc = check_tree_build_args(draft_table, n_rows, vocab, uniforms, n_uniforms, root_row, n_req, m, parents, tokens,
+                                       values, child_values, rows, n_nodes);
+  if (rc != DYSPEC_OK || n_req == 0) return rc;
+  cudaError_t e = launch_build_tree_greedy(draft_table, n_rows, vocab, uniforms, n_uniforms, root_row, n_req, m, parents,
+                                           tokens, values, child_values, rows, n_nodes, reinterpret_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? DYSPEC_OK : cuda_failed(e, "greedy tree launch");
+}
+
+int dyspec_build_tree_threshold(const float* draft_table, int n_rows, int vocab, const float* uniforms, int n_uniforms,
+                                const int32_t* root_row, int n_req, float threshold, int max_nodes, int32_t* parents,
+                                int32_t* tokens, float* values, float* child_values, int32_t* rows, int32_t* n_nodes,
+                                dyspec_stream_t stream) {
+  const int rc = check_tree_build_args(draft_table, n_rows, vocab, uniforms, n_uniforms, root_row, n_req, max_nodes, parents,
+                                       tokens, values, child_values, rows, n_nodes);
+  if (rc != DYSPEC_OK || n_req == 0) return rc;
+  if (!(threshold > 0.f)) return DYSPEC_ERR_INVALID_ARG;
+  cudaError_t e = launch_build_tree_threshold(draft_table, n_rows, vocab, uniforms, n_uniforms, root_row, n_req, threshold,
+                                              max_nodes, parents, tokens, values, child_values, rows, n_nodes,
+                                              reinterpret_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? DYSPEC_OK : cuda_failed(e, "threshold tree launch");
 }
 
 // Validates the arguments and runs the scheduler; no CUDA call.

@@ -15,38 +15,9 @@
 //
 // The branches of a node are its children in increasing index; they are gathered per visited node with
 // warp ballots (no precomputed child lists).
-#include "common.cuh"
+#include "vocab_ops.cuh"
 
 namespace dyspec {
-
-namespace {
-
-constexpr int kVThreads = 1024;
-constexpr int kMaxChunks = 8;                 // float4 chunks per thread: vocabulary <= 8 * 1024 * 4 = 32768
-
-__device__ __forceinline__ float warp_sum(float v) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-  return v;
-}
-
-// Sum over the block; every thread gets the result.  `scratch` holds 33 floats.
-__device__ __forceinline__ float block_sum(float v, float* scratch) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  v = warp_sum(v);
-  __syncthreads();                            // scratch may still be read from the previous use
-  if (lane == 0) scratch[warp] = v;
-  __syncthreads();
-  if (warp == 0) {
-    float t = scratch[lane];
-    t = warp_sum(t);
-    if (lane == 0) scratch[32] = t;
-  }
-  __syncthreads();
-  return scratch[32];
-}
-
-}  // namespace
 
 __global__ void __launch_bounds__(kVThreads, 1)
 verify_tree_kernel(const int32_t* __restrict__ parents, const int32_t* __restrict__ tokens,
@@ -59,11 +30,9 @@ verify_tree_kernel(const int32_t* __restrict__ parents, const int32_t* __restric
   float4* s_d = reinterpret_cast<float4*>(vsm);                                   // draft row, [chunk][thread]
   int32_t* s_par = reinterpret_cast<int32_t*>(vsm + size_t(kMaxChunks) * kVThreads * 16);   // [n] parents of the request
   // small scalars
-  __shared__ float s_red[33];
-  __shared__ float s_rows[kMaxChunks][32];
-  __shared__ float s_rowtot[kMaxChunks];
+  __shared__ VocabScratch s_vs;
   __shared__ int s_cnt[64];
-  __shared__ int s_nchild, s_pick;
+  __shared__ int s_nchild;
   __shared__ float s_ry, s_dy;
   __shared__ int16_t s_child[2048];
 
@@ -141,7 +110,7 @@ verify_tree_kernel(const int32_t* __restrict__ parents, const int32_t* __restric
       }
     }
     float sR = 1.f, sD = 1.f;
-    int nnz = n_child > 0 ? int(block_sum(nnz_f, s_red) + 0.5f) : 0;
+    int nnz = n_child > 0 ? int(block_sum(nnz_f, s_vs) + 0.5f) : 0;
     bool moved = false;
     for (int b = 0; b < n_child; ++b) {
       const int child = s_child[b];
@@ -185,7 +154,7 @@ verify_tree_kernel(const int32_t* __restrict__ parents, const int32_t* __restric
           part += (R[k].x + R[k].y) + (R[k].z + R[k].w);
         }
       }
-      const float tot = block_sum(part, s_red);                  // (its barriers also order the reads of s_d above)
+      const float tot = block_sum(part, s_vs);                  // (its barriers also order the reads of s_d above)
       sR = tot > 0.f ? 1.f / tot : 1.f;
       if (tid == yt) {
         float* dv = reinterpret_cast<float*>(&s_d[yk * kVThreads + yt]);
@@ -200,93 +169,13 @@ verify_tree_kernel(const int32_t* __restrict__ parents, const int32_t* __restric
 
     // ---- no branch accepted (or a leaf with the bonus token): draw the token from R by inverse CDF
     {
-      float rowp[kMaxChunks];
       float part = 0.f;
 #pragma unroll
-      for (int k = 0; k < kMaxChunks; ++k) {
-        rowp[k] = (R[k].x + R[k].y) + (R[k].z + R[k].w);
-        part += rowp[k];
-      }
-      float total = block_sum(part, s_red);
-      if (!(total > 0.f)) {                                      // nothing left (Draft covers Target): fall back to Target
-#pragma unroll
-        for (int k = 0; k < kMaxChunks; ++k) {
-          const int v4 = k * kVThreads + tid;
-          R[k] = (k < n_chunks && v4 < n_vec) ? __ldg(t_row + v4) : make_float4(0.f, 0.f, 0.f, 0.f);
-          rowp[k] = (R[k].x + R[k].y) + (R[k].z + R[k].w);
-        }
-        part = 0.f;
-#pragma unroll
-        for (int k = 0; k < kMaxChunks; ++k) part += rowp[k];
-        total = block_sum(part, s_red);
-      }
-      const float target = sample_u[node0 + cur] * total;
-      // row totals: row k = tokens [4096 k, 4096 k + 4096)
-#pragma unroll
-      for (int k = 0; k < kMaxChunks; ++k) {
-        const float w_ = warp_sum(rowp[k]);
-        if (lane == 0) s_rows[k][warp] = w_;
-      }
-      __syncthreads();
-      if (warp < kMaxChunks) {
-        const float w_ = warp_sum(s_rows[warp][lane]);
-        if (lane == 0) s_rowtot[warp] = w_;
-      }
-      if (tid == 0) s_pick = 0x7fffffff;
-      __syncthreads();
-      // the row that holds the crossing, and the mass before it
-      int krow = n_chunks - 1;
-      float before = 0.f;
-      {
-        float acc = 0.f;
-        bool found = false;
-#pragma unroll
-        for (int k = 0; k < kMaxChunks; ++k) {
-          if (k < n_chunks && !found) {
-            if (acc + s_rowtot[k] > target) { krow = k; before = acc; found = true; }
-            else acc += s_rowtot[k];
-          }
-        }
-        if (!found) before = acc - s_rowtot[n_chunks - 1];
-      }
-      // exclusive scan, inside that row, of the threads' 4-token sums
-      float mine = 0.f;
-      float4 rv = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-      for (int k = 0; k < kMaxChunks; ++k)
-        if (k == krow) { mine = rowp[k]; rv = R[k]; }
-      float incl = mine;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const float t = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += t;
-      }
-      __syncthreads();
-      if (lane == 31) s_red[warp] = incl;
-      __syncthreads();
-      if (warp == 0) {
-        const float w_ = s_red[lane];
-        float x = w_;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-          const float t = __shfl_up_sync(0xffffffffu, x, o);
-          if (lane >= o) x += t;
-        }
-        s_red[lane] = x - w_;                                    // mass of the warps before this one
-      }
-      __syncthreads();
-      float cum = before + s_red[warp] + (incl - mine);          // mass before this thread's 4 tokens
-      const int v0 = (krow * kVThreads + tid) * 4;
-      int pick = 0x7fffffff;
-      const float e4[4] = {rv.x, rv.y, rv.z, rv.w};
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        cum += e4[e];
-        if (pick == 0x7fffffff && v0 + e < vocab && cum > target) pick = v0 + e;
-      }
-      if (pick != 0x7fffffff) atomicMin(&s_pick, pick);
-      __syncthreads();
-      const int y = min(s_pick, vocab - 1);
+      for (int k = 0; k < kMaxChunks; ++k) part += (R[k].x + R[k].y) + (R[k].z + R[k].w);
+      const float left = block_sum(part, s_vs);
+      if (!(left > 0.f)) load_row(R, target_probs + size_t(node0 + cur) * vocab, vocab);    // nothing left: fall back to Target
+      double total;
+      const int y = sample_inverse_cdf(R, vocab, sample_u[node0 + cur], total, s_vs);
       if (tid == 0 && n_out < max_out) { out_tokens[size_t(r) * max_out + n_out] = y; out_nodes[size_t(r) * max_out + n_out] = -1; }
       ++n_out;
     }

@@ -268,3 +268,11 @@ def make_verify_case(seed: int, vocab: int, parents_list, sharpness: float = 4.0
         tokens.append(tok)
     return VerifyCase(name, vocab, offs, [np.asarray(p, np.int32) for p in parents_list], tokens, draft, target,
                       rng.random(N, dtype=np.float32), rng.random(N, dtype=np.float32))
+
+
+def make_draft_table(seed: int, n_rows: int, vocab: int, sharpness: float = 3.0, n_uniforms: int = 4099):
+    """The table-lookup draft model of the tree-construction kernels: n_rows distributions over the
+    vocabulary (softmax of sharpness * N(0,1) logits, fp32) and a table of U(0,1) numbers."""
+    rng = np.random.default_rng(seed)
+    rows = _softmax_rows(rng.standard_normal((n_rows, vocab)).astype(np.float32) * np.float32(sharpness))
+    return rows, rng.random(n_uniforms, dtype=np.float32)

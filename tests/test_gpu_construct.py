@@ -1,0 +1,129 @@
+"""GPU parity of the tree-construction kernels (Algorithms 1 and 2) with the oracle.  Structure, tokens
+and row ids must match exactly, values to fp32 rounding (they are stored as fp32).  The kernels take
+their decisions (order of slot values, CDF search, v against t) in fp64 like the oracle, so a request
+would be excused only where the oracle reports a decision within 1e-12 of its threshold."""
+import numpy as np
+import pytest
+
+from oracle import dyspec_oracle as orc
+from paper_2410_11744_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+EPS = {"order": 1e-12, "sample": 1e-12, "threshold": 1e-12}     # the kernels carry these sums and values in fp64
+
+
+@pytest.fixture(scope="module")
+def B():
+    import torch
+    assert torch.cuda.is_available()
+    from paper_2410_11744_b200 import build
+    build.build()
+    from paper_2410_11744_b200 import binding
+    return binding
+
+
+def run_gpu(B, rows, uni, roots, m=None, threshold=None, max_nodes=None):
+    import torch
+    dev = "cuda:0"
+    t = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(dev)
+    n_req = len(roots)
+    S = (m if threshold is None else max_nodes) + 1
+    parents = torch.full((n_req, S), -9, dtype=torch.int32, device=dev)
+    tokens = torch.full((n_req, S), -9, dtype=torch.int32, device=dev)
+    nrows = torch.full((n_req, S), -9, dtype=torch.int32, device=dev)
+    values = torch.zeros((n_req, S), dtype=torch.float32, device=dev)
+    cvalues = torch.zeros((n_req, S), dtype=torch.float32, device=dev)
+    n_nodes = torch.zeros((n_req,), dtype=torch.int32, device=dev)
+    args = (t(rows), rows.shape[0], rows.shape[1], t(uni), len(uni), t(np.asarray(roots, np.int32)), n_req)
+    if threshold is None:
+        B.dyspec_build_tree_greedy(*args, m, parents, tokens, values, cvalues, nrows, n_nodes)
+    else:
+        B.dyspec_build_tree_threshold(*args, threshold, max_nodes, parents, tokens, values, cvalues, nrows, n_nodes)
+    torch.cuda.synchronize()
+    return [x.cpu().numpy() for x in (parents, tokens, values, cvalues, nrows, n_nodes)]
+
+
+def compare(got, r, ref):
+    parents, tokens, values, cvalues, nrows, n_nodes = got
+    n = len(ref["parents"])
+    assert int(n_nodes[r]) == n
+    assert np.array_equal(parents[r, :n], ref["parents"])
+    assert np.array_equal(tokens[r, :n], ref["tokens"])
+    assert np.array_equal(nrows[r, :n], ref["rows"])
+    assert np.allclose(values[r, :n], ref["values"], rtol=2e-5, atol=0)
+    assert np.allclose(cvalues[r, :n], ref["child_values"], rtol=2e-5, atol=1e-30)
+
+
+def excused(ref):
+    return any(mg < EPS[kind] for kind, mg in ref["margins"])
+
+
+@pytest.mark.parametrize("vocab,n_rows,m,sharp", [(32000, 24, 64, 3.0), (32768, 8, 40, 2.0), (1000, 64, 200, 2.0), (64, 16, 60, 1.0)])
+def test_greedy_tree_matches_oracle(B, vocab, n_rows, m, sharp):
+    rows, uni = wl.make_draft_table(100 + vocab, n_rows, vocab, sharp)
+    roots = [0, 3, 5, 7]
+    got = run_gpu(B, rows, uni, roots, m=m)
+    skipped = 0
+    for r, root in enumerate(roots):
+        ref = orc.build_tree_greedy(rows, uni, m, root_row=root)
+        if excused(ref):
+            skipped += 1
+            continue
+        compare(got, r, ref)
+    assert skipped == 0
+
+
+@pytest.mark.parametrize("vocab,n_rows,threshold,cap,sharp", [(32000, 24, 0.02, 300, 3.0), (1000, 64, 0.004, 600, 2.0),
+                                                              (64, 16, 0.01, 50, 1.0), (32000, 8, 0.5, 10, 3.0)])
+def test_threshold_tree_matches_oracle(B, vocab, n_rows, threshold, cap, sharp):
+    rows, uni = wl.make_draft_table(200 + vocab, n_rows, vocab, sharp)
+    roots = [1, 2, 6]
+    got = run_gpu(B, rows, uni, roots, threshold=threshold, max_nodes=cap)
+    skipped = 0
+    for r, root in enumerate(roots):
+        ref = orc.build_tree_threshold(rows, uni, threshold, cap, root_row=root)
+        if excused(ref):
+            skipped += 1
+            continue
+        compare(got, r, ref)
+    assert skipped == 0
+
+
+def test_gpu_threshold_at_last_greedy_value_builds_the_same_tree(B):
+    """The paper's statement (App. B), on the GPU alone: same set of root-to-node token paths."""
+    rows, uni = wl.make_draft_table(9, 32, 4096, 3.0)
+    m = 80
+    g = run_gpu(B, rows, uni, [4], m=m)
+    t = float(g[2][0, m])
+    h = run_gpu(B, rows, uni, [4], threshold=t, max_nodes=4 * m)
+
+    def paths(parents, tokens, n):
+        out = set()
+        for k in range(1, n):
+            p, j = [], k
+            while j > 0:
+                p.append(int(tokens[j]))
+                j = int(parents[j])
+            out.add(tuple(reversed(p)))
+        return out
+    assert paths(g[0][0], g[1][0], int(g[5][0])) == paths(h[0][0], h[1][0], int(h[5][0]))
+
+
+def test_constructed_tree_feeds_the_mask_builder(B):
+    """The greedy tree's parent array is a legal input of the attention path (parents[i] < i)."""
+    import torch
+    rows, uni = wl.make_draft_table(3, 16, 2048, 2.5)
+    m = 255
+    got = run_gpu(B, rows, uni, [0], m=m)
+    parents = np.ascontiguousarray(got[0][0])
+    n = m + 1
+    W = B.dyspec_words_per_row(n)
+    bits = torch.zeros((n, W), dtype=torch.int32, device="cuda:0")
+    depths = torch.zeros((n,), dtype=torch.int32, device="cuda:0")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda:0")
+    B.dyspec_build_tree_mask(torch.from_numpy(parents).to("cuda:0"), n, bits, depths, W, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    ref_bits, ref_depths = orc.build_tree_mask(parents, W)
+    assert np.array_equal(bits.cpu().numpy().view(np.uint32), ref_bits)
+    assert np.array_equal(depths.cpu().numpy(), ref_depths)
