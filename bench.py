@@ -324,6 +324,60 @@ def verification_experiment(torch, workloads, B, peaks, device):
     return rows
 
 
+def construction_experiment(torch, workloads, B, peaks, device):
+    """Tree construction (Algorithms 1 and 2) on the device over the table-lookup draft model: vocabulary
+    32000, 64 language-model-like (Zipf) table rows; the paper's two tree sizes (64 and 768 guesses) for one request, and the
+    threshold form at the value of the greedy tree's last node.  Algorithmic bytes = one draft row
+    (vocab * 4) per guess (greedy) or per expanded position (threshold)."""
+    rows_np, uni_np = workloads.make_draft_table(workloads.MASTER_SEED + 8000, 64, 32000, zipf=True)
+    t = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(device)
+    rows, uni = t(rows_np), t(uni_np)
+    root = torch.zeros(1, dtype=torch.int32, device=device)
+    out = []
+    for m in (64, 768):
+        S = m + 1
+        bufs = [torch.zeros((1, S), dtype=torch.int32, device=device) for _ in range(3)]
+        vals = [torch.zeros((1, S), dtype=torch.float32, device=device) for _ in range(2)]
+        cnt = torch.zeros(1, dtype=torch.int32, device=device)
+        greedy = lambda: B.dyspec_build_tree_greedy(rows, 64, 32000, uni, len(uni_np), root, 1, m, bufs[0], bufs[1], vals[0],
+                                                    vals[1], bufs[2], cnt)
+        greedy()
+        torch.cuda.synchronize()
+        thr = float(vals[0][0, m].item())
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(5):
+            greedy()
+        e1.record()
+        torch.cuda.synchronize()
+        g_us = e0.elapsed_time(e1) / 5 * 1e3
+        parents = bufs[0][0].cpu().numpy()
+        cap = 4 * m if 4 * m < 2047 else 2047
+        tb = [torch.zeros((1, cap + 1), dtype=torch.int32, device=device) for _ in range(3)]
+        tv = [torch.zeros((1, cap + 1), dtype=torch.float32, device=device) for _ in range(2)]
+        layered = lambda: B.dyspec_build_tree_threshold(rows, 64, 32000, uni, len(uni_np), root, 1, thr, cap, tb[0], tb[1],
+                                                        tv[0], tv[1], tb[2], cnt)
+        layered()
+        torch.cuda.synchronize()
+        n_thr = int(cnt.item()) - 1
+        e0.record()
+        for _ in range(5):
+            layered()
+        e1.record()
+        torch.cuda.synchronize()
+        t_us = e0.elapsed_time(e1) / 5 * 1e3
+        tp = tb[0][0, :n_thr + 1].cpu().numpy()
+        positions = len(set(int(x) for x in tp[1:]))
+        depth = np.zeros(m + 1, int)
+        for k in range(1, m + 1):
+            depth[k] = depth[parents[k]] + 1
+        out.append({"guesses": m, "vocab": 32000, "greedy_us": g_us, "greedy_us_per_guess": g_us / m,
+                    "greedy_gbs": m * 32000 * 4 / (g_us * 1e-6) / 1e9, "depth": int(depth.max()),
+                    "threshold": thr, "threshold_guesses": n_thr, "threshold_positions": positions, "threshold_us": t_us,
+                    "threshold_gbs": positions * 32000 * 4 / (t_us * 1e-6) / 1e9})
+    return out
+
+
 def roofline_entry(m, peaks, peaks_kind):
     t_hbm = m["bytes"] / (peaks["hbm_gbs"] * 1e9)
     t_tc = m["flops"] / (peaks["bf16_tflops"] * 1e12)
@@ -461,6 +515,10 @@ def run_ours(args):
     if not args.no_per_config and world == 1:
         verification = verification_experiment(torch, workloads, binding, peaks, device)
 
+    construction = None
+    if not args.no_per_config and world == 1:
+        construction = construction_experiment(torch, workloads, binding, peaks, device)
+
     # ---- the oracle on the host cores, bounded sample of the same workload
     times = time_oracle(w, budget_s=12.0)
     cpu_sec = sum(times) / len(times)
@@ -491,6 +549,8 @@ def run_ours(args):
         line["random_tree_experiment"] = random_tree
     if verification:
         line["verification_experiment"] = verification
+    if construction:
+        line["construction_experiment"] = construction
     print(json.dumps(line), flush=True)
     if use_dist:
         dist.barrier()

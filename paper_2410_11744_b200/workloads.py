@@ -270,9 +270,19 @@ def make_verify_case(seed: int, vocab: int, parents_list, sharpness: float = 4.0
                       rng.random(N, dtype=np.float32), rng.random(N, dtype=np.float32))
 
 
-def make_draft_table(seed: int, n_rows: int, vocab: int, sharpness: float = 3.0, n_uniforms: int = 4099):
+def make_draft_table(seed: int, n_rows: int, vocab: int, sharpness: float = 3.0, n_uniforms: int = 4099,
+                     zipf: bool = False):
     """The table-lookup draft model of the tree-construction kernels: n_rows distributions over the
-    vocabulary (softmax of sharpness * N(0,1) logits, fp32) and a table of U(0,1) numbers."""
+    vocabulary and a table of U(0,1) numbers.  Rows are softmax(sharpness * N(0,1) logits), or with
+    zipf=True language-model-like: p ~ rank^-a with a ~ U(1.1, 2.2) per row over a random permutation
+    of the tokens (top token 0.2 - 0.7), fp32."""
     rng = np.random.default_rng(seed)
-    rows = _softmax_rows(rng.standard_normal((n_rows, vocab)).astype(np.float32) * np.float32(sharpness))
+    if zipf:
+        rows = np.empty((n_rows, vocab), dtype=np.float32)
+        ranks = np.arange(1, vocab + 1, dtype=np.float64)
+        for i in range(n_rows):
+            p = ranks ** (-rng.uniform(1.1, 2.2))
+            rows[i, rng.permutation(vocab)] = (p / p.sum()).astype(np.float32)
+    else:
+        rows = _softmax_rows(rng.standard_normal((n_rows, vocab)).astype(np.float32) * np.float32(sharpness))
     return rows, rng.random(n_uniforms, dtype=np.float32)

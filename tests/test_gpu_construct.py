@@ -89,6 +89,23 @@ def test_threshold_tree_matches_oracle(B, vocab, n_rows, threshold, cap, sharp):
     assert skipped == 0
 
 
+def test_zipf_rows_give_deep_trees_and_match_oracle(B):
+    rows, uni = wl.make_draft_table(77, 48, 32000, zipf=True)
+    m = 96
+    roots = list(range(8))
+    got = run_gpu(B, rows, uni, roots, m=m)
+    deepest = 0
+    for r, root in enumerate(roots):
+        ref = orc.build_tree_greedy(rows, uni, m, root_row=root)
+        assert not excused(ref)
+        compare(got, r, ref)
+        depth = np.zeros(m + 1, int)
+        for k in range(1, m + 1):
+            depth[k] = depth[ref["parents"][k]] + 1
+        deepest = max(deepest, int(depth.max()))
+    assert deepest >= 3            # peaked rows give chains, flat rows give stars: both shapes are exercised
+
+
 def test_gpu_threshold_at_last_greedy_value_builds_the_same_tree(B):
     """The paper's statement (App. B), on the GPU alone: same set of root-to-node token paths."""
     rows, uni = wl.make_draft_table(9, 32, 4096, 3.0)
