@@ -33,7 +33,9 @@ acceptance rates, forced rejections, the all-zero early exit); the tree
 construction (Algorithms 1 and 2) by tests/test_construct_pins.py (values
 decrease, the closed form of the estimated acceptance rate in raw draft
 probabilities, Algorithm 2 at the last value == Algorithm 1, guesses at a
-position are draws without replacement).
+position are draws without replacement); compact_kv by
+tests/test_compact_pins.py (hand example, no-op on a chain prefix, attention
+over the compacted cache == attention along the accepted path).
 Nothing here is "parity unpinned".
 
 Readings where the paper is silent: scale = 1/sqrt(head_dim); consecutive query
@@ -463,3 +465,20 @@ def build_tree_threshold(rows, uniforms, threshold: float, max_nodes: int, root_
     return dict(parents=np.asarray(parents, np.int32), tokens=np.asarray(tokens, np.int32),
                 values=np.asarray(values), child_values=np.asarray(child_values),
                 rows=np.asarray(node_rows, np.int32), margins=margins)
+
+
+# ----------------------------------------------------------------------------------------------------
+# Keeping the accepted path in the KV cache (the step after verification; the paper only says that the
+# accepted tokens extend the prefix, Sec. 2 / Algorithm 3).
+# ----------------------------------------------------------------------------------------------------
+def compact_kv(cache: np.ndarray, kv_row0: int, prefix_len: int, accepted_nodes: Sequence[int]) -> int:
+    """After a verification step the cache of a request holds prefix_len prefix rows followed by one row
+    per tree node (node j at row kv_row0 + prefix_len + j).  The accepted nodes a_0 < a_1 < ... become
+    part of the prefix: row kv_row0 + prefix_len + i takes the content of node a_i's row, in place.
+    Entries < 0 (an emitted token that has no tree node) are skipped.  Returns the new prefix length."""
+    nodes = [int(a) for a in accepted_nodes if int(a) >= 0]
+    base = int(kv_row0) + int(prefix_len)
+    gathered = [cache[base + a].copy() for a in nodes]       # all reads first: the definition is a gather
+    for i, row in enumerate(gathered):
+        cache[base + i] = row
+    return int(prefix_len) + len(nodes)
