@@ -378,6 +378,34 @@ def construction_experiment(torch, workloads, B, peaks, device):
     return out
 
 
+def compaction_experiment(torch, B, peaks, device):
+    """Accepted-path KV compaction: 8 accepted nodes per request, Llama2-7B rows (32 x 128 bf16 = 8 KB) for
+    1 request and Llama2-70B rows (8 x 128 = 2 KB) for a batch of 64; algorithmic bytes = rows moved x 2
+    (read + write) x 2 (K and V)."""
+    out = []
+    for label, n_req, hkv in (("1 request, 32 kv heads", 1, 32), ("64 requests, 8 kv heads", 64, 8)):
+        d, L, n, max_out = 128, 1024, 64, 16
+        rows = n_req * (L + n)
+        k = torch.zeros((rows, hkv, d), dtype=torch.bfloat16, device=device)
+        v = torch.zeros((rows, hkv, d), dtype=torch.bfloat16, device=device)
+        offs = torch.arange(n_req, dtype=torch.int64, device=device) * (L + n)
+        Ls = torch.full((n_req,), L, dtype=torch.int32, device=device)
+        acc = torch.tensor([[1, 4, 9, 17, 22, 30, 41, 55, -1] + [0] * (max_out - 9)] * n_req, dtype=torch.int32, device=device)
+        cnt = torch.full((n_req,), 9, dtype=torch.int32, device=device)
+        newL = torch.zeros(n_req, dtype=torch.int32, device=device)
+        call = lambda: B.dyspec_compact_kv(k, v, offs, Ls, acc, cnt, n_req, max_out, hkv, d, newL)
+        call()
+        torch.cuda.synchronize()
+        g = _graph_of(torch, lambda: [call() for _ in range(20)])
+        g.replay()
+        torch.cuda.synchronize()
+        us = _time_replays(torch, g, 20) / 400 * 1e3
+        nbytes = n_req * 8 * hkv * d * 2 * 2 * 2
+        out.append({"case": label, "call_us": us, "bytes": nbytes, "achieved_gbs": nbytes / (us * 1e-6) / 1e9,
+                    "frac_of_hbm": nbytes / (us * 1e-6) / 1e9 / peaks["hbm_gbs"]})
+    return out
+
+
 def roofline_entry(m, peaks, peaks_kind):
     t_hbm = m["bytes"] / (peaks["hbm_gbs"] * 1e9)
     t_tc = m["flops"] / (peaks["bf16_tflops"] * 1e12)
@@ -519,6 +547,10 @@ def run_ours(args):
     if not args.no_per_config and world == 1:
         construction = construction_experiment(torch, workloads, binding, peaks, device)
 
+    compaction = None
+    if not args.no_per_config and world == 1:
+        compaction = compaction_experiment(torch, binding, peaks, device)
+
     # ---- the oracle on the host cores, bounded sample of the same workload
     times = time_oracle(w, budget_s=12.0)
     cpu_sec = sum(times) / len(times)
@@ -551,6 +583,8 @@ def run_ours(args):
         line["verification_experiment"] = verification
     if construction:
         line["construction_experiment"] = construction
+    if compaction:
+        line["compaction_experiment"] = compaction
     print(json.dumps(line), flush=True)
     if use_dist:
         dist.barrier()

@@ -326,6 +326,21 @@ int dyspec_build_tree_threshold(const float* draft_table, int n_rows, int vocab,
                                 int32_t* tokens, float* values, float* child_values, int32_t* rows, int32_t* n_nodes,
                                 dyspec_stream_t stream);
 
+/*
+ * (7) Keeping the accepted path in the KV cache (after dyspec_verify_tree; the paper only says that the
+ * accepted tokens extend the prefix).  For request r with accepted nodes a_0 < a_1 < ... (entries < 0,
+ * i.e. emitted tokens without a tree node, are skipped) row off_r + L_r + i of k_cache and v_cache
+ * takes the content of row off_r + L_r + a_i, in place, and new_prefix_len[r] = L_r + their number.
+ * Rows past the new prefix keep their old content.  One call per layer (per pair of caches).
+ *   k_cache, v_cache  dev bf16 [rows][n_kv_heads][head_dim] (16-byte aligned; row bytes a multiple of 16)
+ *   kv_row_offset     dev int64 [n_req];  prefix_len  dev int32 [n_req]
+ *   accepted_nodes    dev int32 [n_req][max_out], n_accepted dev int32 [n_req]  (as written by dyspec_verify_tree)
+ *   new_prefix_len    dev int32 [n_req] or NULL (written)
+ */
+int dyspec_compact_kv(void* k_cache, void* v_cache, const int64_t* kv_row_offset, const int32_t* prefix_len,
+                      const int32_t* accepted_nodes, const int32_t* n_accepted, int n_req, int max_out, int n_kv_heads,
+                      int head_dim, int32_t* new_prefix_len, dyspec_stream_t stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -50,6 +50,7 @@ SIGNATURES = {
     "dyspec_verify_tree": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _i32, _vp, _vp]),
     "dyspec_build_tree_greedy": (_i32, [_vp, _i32, _i32, _vp, _i32, _vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "dyspec_build_tree_threshold": (_i32, [_vp, _i32, _i32, _vp, _i32, _vp, _i32, _f32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "dyspec_compact_kv": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _i32, _i32, _i32, _i32, _vp, _vp]),
     "dyspec_tree_attention_static": (_i32, [_vp, _vp, _vp, _i32, _vp, _i32, _vp, _i32, _i32, _i32, _i32, _f32, _vp, _vp]),
 }
 for _name, (_res, _args) in SIGNATURES.items():
@@ -298,3 +299,11 @@ def dyspec_build_tree_threshold(draft_table, n_rows: int, vocab: int, uniforms, 
                                            n_req, float(threshold), max_nodes, _ptr(parents), _ptr(tokens), _ptr(values),
                                            _ptr(child_values), _ptr(rows), _ptr(n_nodes), _stream(stream)),
            "dyspec_build_tree_threshold")
+
+
+def dyspec_compact_kv(k_cache, v_cache, kv_row_offset, prefix_len, accepted_nodes, n_accepted, n_req: int, max_out: int,
+                      n_kv_heads: int, head_dim: int, new_prefix_len=None, stream=None) -> None:
+    """Moves the accepted nodes' K/V rows behind the prefix, in place (see include/dyspec.h)."""
+    _check(lib.dyspec_compact_kv(_ptr(k_cache), _ptr(v_cache), _ptr(kv_row_offset), _ptr(prefix_len), _ptr(accepted_nodes),
+                                 _ptr(n_accepted), n_req, max_out, n_kv_heads, head_dim, _ptr(new_prefix_len),
+                                 _stream(stream)), "dyspec_compact_kv")

@@ -35,6 +35,9 @@ cudaError_t launch_build_tree_threshold(const float* draft_table, int n_rows, in
                                         int n_uniforms, const int32_t* root_row, int n_req, float threshold, int max_nodes,
                                         int32_t* parents, int32_t* tokens, float* values, float* child_values, int32_t* rows,
                                         int32_t* n_nodes, cudaStream_t stream);
+cudaError_t launch_compact_kv(void* k_cache, void* v_cache, const int64_t* kv_row_offset, const int32_t* prefix_len,
+                              const int32_t* accepted_nodes, const int32_t* n_accepted, int n_req, int max_out,
+                              int row_bytes, int32_t* new_prefix_len, cudaStream_t stream);
 cudaError_t launch_attn_mma(int head_dim, int n_ctas, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                             const AttnParams& p, cudaStream_t stream);
 cudaError_t launch_combine(int head_dim, int bm, int n_split_groups, const AttnParams& p, cudaStream_t stream);
@@ -467,6 +470,20 @@ int dyspec_build_tree_threshold(const float* draft_table, int n_rows, int vocab,
                                               max_nodes, parents, tokens, values, child_values, rows, n_nodes,
                                               reinterpret_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? DYSPEC_OK : cuda_failed(e, "threshold tree launch");
+}
+
+int dyspec_compact_kv(void* k_cache, void* v_cache, const int64_t* kv_row_offset, const int32_t* prefix_len,
+                      const int32_t* accepted_nodes, const int32_t* n_accepted, int n_req, int max_out, int n_kv_heads,
+                      int head_dim, int32_t* new_prefix_len, dyspec_stream_t stream) {
+  if (n_req < 0 || max_out <= 0 || n_kv_heads <= 0 || head_dim <= 0) return DYSPEC_ERR_INVALID_ARG;
+  const int64_t row_bytes = int64_t(n_kv_heads) * head_dim * 2;
+  if (row_bytes % 16 != 0 || row_bytes > (1 << 24)) return DYSPEC_ERR_UNSUPPORTED;
+  if (n_req == 0) return DYSPEC_OK;
+  if (!k_cache || !v_cache || !kv_row_offset || !prefix_len || !accepted_nodes || !n_accepted) return DYSPEC_ERR_INVALID_ARG;
+  if (!aligned(k_cache, 16) || !aligned(v_cache, 16)) return DYSPEC_ERR_INVALID_ARG;
+  cudaError_t e = launch_compact_kv(k_cache, v_cache, kv_row_offset, prefix_len, accepted_nodes, n_accepted, n_req, max_out,
+                                    int(row_bytes), new_prefix_len, reinterpret_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? DYSPEC_OK : cuda_failed(e, "compact launch");
 }
 
 // Validates the arguments and runs the scheduler; no CUDA call.

@@ -1,0 +1,47 @@
+// Keeping the accepted path in the KV cache after verification: for each request, the tree rows of the
+// accepted nodes a_0 < a_1 < ... move to the rows right after the prefix (row L + i <- row L + a_i), in
+// place, for K and V, and the prefix length grows by their number.
+//
+// a_i >= i, so a destination never lies behind its own source, but it can be an EARLIER step's
+// source (path 1, 2, 3: slot 1 receives node 2 after it has given node 1 away).  A thread owns fixed
+// 16-byte columns of a row and walks the steps in order, so for any byte the read of step i precedes
+// the write of step i + 1 in program order, and no two threads ever touch the same byte: no barriers.
+// grid = (requests, column chunks, 2 for K / V); the copy is a few hundred KB at most, i.e. bound by
+// launch latency.
+#include "common.cuh"
+
+namespace dyspec {
+
+__global__ void __launch_bounds__(256)
+compact_kv_kernel(uint4* __restrict__ k_cache, uint4* __restrict__ v_cache, const int64_t* __restrict__ kv_row_offset,
+                  const int32_t* __restrict__ prefix_len, const int32_t* __restrict__ accepted_nodes,
+                  const int32_t* __restrict__ n_accepted, int max_out, int row_vecs, int32_t* __restrict__ new_prefix_len) {
+  const int r = blockIdx.x;
+  uint4* cache = blockIdx.z == 0 ? k_cache : v_cache;
+  const int L = prefix_len[r];
+  const int64_t base = (kv_row_offset[r] + L) * int64_t(row_vecs);
+  const int n = min(n_accepted[r], max_out);
+  const int32_t* acc = accepted_nodes + size_t(r) * max_out;
+  const int col = blockIdx.y * blockDim.x + threadIdx.x;
+  int kept = 0;
+  for (int i = 0; i < n; ++i) {
+    const int a = acc[i];
+    if (a < 0) continue;                       // an emitted token without a tree node
+    if (col < row_vecs && a != kept) cache[base + int64_t(kept) * row_vecs + col] = cache[base + int64_t(a) * row_vecs + col];
+    ++kept;
+  }
+  if (new_prefix_len && blockIdx.y == 0 && blockIdx.z == 0 && threadIdx.x == 0) new_prefix_len[r] = L + kept;
+}
+
+cudaError_t launch_compact_kv(void* k_cache, void* v_cache, const int64_t* kv_row_offset, const int32_t* prefix_len,
+                              const int32_t* accepted_nodes, const int32_t* n_accepted, int n_req, int max_out,
+                              int row_bytes, int32_t* new_prefix_len, cudaStream_t stream) {
+  if (n_req <= 0) return cudaSuccess;
+  const int row_vecs = row_bytes / 16;
+  const dim3 grid(unsigned(n_req), unsigned((row_vecs + 255) / 256), 2u);
+  compact_kv_kernel<<<grid, 256, 0, stream>>>(static_cast<uint4*>(k_cache), static_cast<uint4*>(v_cache), kv_row_offset,
+                                              prefix_len, accepted_nodes, n_accepted, max_out, row_vecs, new_prefix_len);
+  return cudaGetLastError();
+}
+
+}  // namespace dyspec
