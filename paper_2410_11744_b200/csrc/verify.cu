@@ -100,14 +100,15 @@ verify_tree_kernel(const int32_t* __restrict__ parents, const int32_t* __restric
     for (int k = 0; k < kMaxChunks; ++k) {
       const int v4 = k * kVThreads + tid;
       R[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+      float4 d = make_float4(0.f, 0.f, 0.f, 0.f);
       if (k < n_chunks && v4 < n_vec) {
         R[k] = __ldg(t_row + v4);
         if (n_child > 0) {
-          const float4 d = __ldg(d_row + v4);
-          s_d[k * kVThreads + tid] = d;
+          d = __ldg(d_row + v4);
           nnz_f += (d.x > 0.f) + (d.y > 0.f) + (d.z > 0.f) + (d.w > 0.f);
         }
       }
+      if (n_child > 0) s_d[k * kVThreads + tid] = d;          // the ragged tail of the last chunk must read as zero
     }
     float sR = 1.f, sD = 1.f;
     int nnz = n_child > 0 ? int(block_sum(nnz_f, s_vs) + 0.5f) : 0;
