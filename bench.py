@@ -592,21 +592,69 @@ def run_ours(args):
 
 
 def run_profile(args):
-    """A short eager run of the hot path for profilers: no graphs, no timing, no oracle."""
+    """A short eager run for profilers: no graphs, no timing, no oracle.  --profile-op step (default):
+    mask build + attention of --config; sparse: DFS reorder + mask with tile sets + tile-skipping
+    attention on the 2048-token random tree; verify / construct: those kernels on small cases."""
     import torch
     from paper_2410_11744_b200 import build as _build
     _build.build()
-    from paper_2410_11744_b200 import runner, workloads
-    w = workloads.make_config(args.config)
-    first = runner.DeviceBatch(w)
-    nbytes, _ = algorithmic_cost(w, first.W)
-    copies = max(2, min(8, int(np.ceil(1.2 * L2_BYTES / max(nbytes, 1)))))
-    batches = [first] + [runner.DeviceBatch(w, plan=first.plan) for _ in range(copies - 1)]
-    for i in range(args.profile):
-        batches[i % copies].step()
-    torch.cuda.synchronize()
-    print(json.dumps({"profiled_steps": args.profile, "workload": w.name, "copies": copies,
-                      "plan": first.plan.describe(), "status": int(first.status.item())}))
+    from paper_2410_11744_b200 import binding as B, runner, workloads
+    dev = torch.device("cuda", 0)
+    t = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(dev)
+    if args.profile_op == "step":
+        w = workloads.make_config(args.config)
+        first = runner.DeviceBatch(w)
+        nbytes, _ = algorithmic_cost(w, first.W)
+        copies = max(2, min(8, int(np.ceil(1.2 * L2_BYTES / max(nbytes, 1)))))
+        batches = [first] + [runner.DeviceBatch(w, plan=first.plan) for _ in range(copies - 1)]
+        for i in range(args.profile):
+            batches[i % copies].step()
+        torch.cuda.synchronize()
+        info = {"workload": w.name, "copies": copies, "plan": first.plan.describe(), "status": int(first.status.item())}
+    elif args.profile_op == "sparse":
+        w = workloads.make_random_tree_case(2048)
+        probe = runner.DeviceBatch(w)
+        order, _, new_parents = probe.dfs_reorder()
+        w2 = workloads.permute_tree_tokens(w, [order], [new_parents])
+        batches = [runner.DeviceBatch(w2, plan=probe.plan, sparse=True) for _ in range(2)]     # 2 x 134 MB > L2
+        order_d = torch.empty(2048, dtype=torch.int32, device=dev)
+        newp_d = torch.empty(2048, dtype=torch.int32, device=dev)
+        for i in range(args.profile):
+            B.dyspec_plan_dfs_reorder(probe.plan, probe.parents, order_d, None, newp_d, None)
+            batches[i % 2].step()
+        torch.cuda.synchronize()
+        info = {"workload": w2.name, "copies": 2, "plan": probe.plan.describe(), "status": int(batches[0].status.item())}
+    elif args.profile_op == "verify":
+        rng = np.random.default_rng(workloads.MASTER_SEED + 7000)
+        trees = [workloads.greedy_tree(rng, 256, 8, 0.1) for _ in range(8)]
+        case = workloads.make_verify_case(workloads.MASTER_SEED + 7001, 32000, trees, sharpness=3.0, disagreement=1.0)
+        d, tg = t(case.draft_probs), t(case.target_probs)
+        out_t = torch.zeros((8, 64), dtype=torch.int32, device=dev)
+        out_n = torch.zeros((8, 64), dtype=torch.int32, device=dev)
+        cnt = torch.zeros(8, dtype=torch.int32, device=dev)
+        args_ = (t(np.concatenate(case.parents)), t(np.concatenate(case.tokens)), d, tg, t(case.accept_u), t(case.sample_u),
+                 t(case.node_offsets), 8, 256, 32000, out_t, out_n, cnt, 64)
+        for _ in range(args.profile):
+            B.dyspec_verify_tree(*args_, bonus_at_leaf=True)
+        torch.cuda.synchronize()
+        info = {"workload": "verify 8 requests x 256 nodes, vocab 32000", "emitted": cnt.cpu().numpy().tolist()}
+    else:
+        rows_np, uni_np = workloads.make_draft_table(workloads.MASTER_SEED + 8000, 64, 32000, zipf=True)
+        rows, uni = t(rows_np), t(uni_np)
+        root = torch.arange(8, dtype=torch.int32, device=dev)
+        m = 64
+        bufs = [torch.zeros((8, m + 1), dtype=torch.int32, device=dev) for _ in range(3)]
+        vals = [torch.zeros((8, m + 1), dtype=torch.float32, device=dev) for _ in range(2)]
+        cnt = torch.zeros(8, dtype=torch.int32, device=dev)
+        for _ in range(args.profile):
+            B.dyspec_build_tree_greedy(rows, 64, 32000, uni, len(uni_np), root, 8, m, bufs[0], bufs[1], vals[0], vals[1],
+                                       bufs[2], cnt)
+            B.dyspec_build_tree_threshold(rows, 64, 32000, uni, len(uni_np), root, 8, 0.05, 200, *[
+                torch.zeros((8, 201), dtype=(torch.float32 if i in (2, 3) else torch.int32), device=dev) for i in range(5)], cnt)
+        torch.cuda.synchronize()
+        info = {"workload": "construct 8 requests, 64 guesses, vocab 32000"}
+    info.update({"profiled_steps": args.profile, "op": args.profile_op})
+    print(json.dumps(info))
 
 
 def main():
@@ -619,6 +667,7 @@ def main():
     ap.add_argument("--no-per-config", action="store_true")
     ap.add_argument("--profile", type=int, default=0,
                     help="run only this many plain (eager) steps of --config and exit: the command to put under ncu")
+    ap.add_argument("--profile-op", default="step", choices=["step", "sparse", "verify", "construct"])
     args = ap.parse_args()
     if args.profile > 0:
         return run_profile(args)
