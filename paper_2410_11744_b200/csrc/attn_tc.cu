@@ -52,6 +52,18 @@ enum { B_QFULL = 0, B_QFREE = 1, B_SLOT_FULL = 2, B_SLOT_EMPTY = B_SLOT_FULL + k
        B_SREADY = B_SLOT_EMPTY + kSlots, B_PREADY = B_SREADY + 2, B_ODONE = B_PREADY + 2, B_OFREE = B_ODONE + 2,
        B_COUNT = B_OFREE + 2 };
 
+// Hardware named barriers for thread-to-thread hand-offs inside the CTA (P ready: 128 softmax threads
+// -> the MMA-issuing warp): an order of magnitude quicker to notice than an mbarrier in shared memory
+// (tens of cycles against 180-300), which is what the issuing warp's time goes into.  mbarriers stay
+// where an asynchronous unit signals (TMA bytes, tcgen05.commit).  The arriving side never runs a
+// phase ahead: it cannot produce P(j+1) before the issuing warp, having consumed P(j), has issued the
+// scores it is computed from.  Every participant reaches its arrive / sync unconditionally (bounded
+// mbarrier waits that run out just fall through), so these cannot wait for ever.
+__device__ __forceinline__ void named_arrive(int id, int count) { asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(count) : "memory"); }
+__device__ __forceinline__ void named_sync(int id, int count) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory"); }
+constexpr int kBarPReady = 1;               // named barriers 1, 2: P of half A, B is in TMEM
+constexpr int kPReadyCount = BMH + 32;      // the half's softmax threads + the issuing warp
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
@@ -396,12 +408,12 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           const uint32_t kslot = sc % kSlots, kph = (sc / kSlots) & 1;
           if (more) ++sc;
           // An mbarrier probe takes ~180 cycles to answer even when the phase completed long ago.  The
-          // three barriers this tile starts with (V slot, next K slot, P of half A) are probed in one
-          // go, so their round trips overlap; only what is really not there yet is then waited for.
+          // two slot barriers this tile starts with (V slot, next K slot) are probed in one go, so
+          // their round trips overlap; only what is really not there yet is then waited for.
           {
             const uint32_t got = __reduce_and_sync(0xffffffffu,
                 mbar_test_wait3(bar(B_SLOT_FULL + vslot), vph, bar(B_SLOT_FULL + (more ? kslot : vslot)), more ? kph : vph,
-                                bar(B_PREADY + 0), n_p0 & 1));
+                                bar(B_SLOT_FULL + vslot), vph));
             if (!(got & 1u)) mbar_wait(bar(B_SLOT_FULL + vslot), vph, abort_flag, p.status);
             if (more && !(got & 2u)) mbar_wait(bar(B_SLOT_FULL + kslot), kph, abort_flag, p.status);
             if (j == 0) {
@@ -409,7 +421,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
               if (two) mbar_wait(bar(B_OFREE + 1), (n_it1 & 1) ^ 1, abort_flag, p.status);
             }
             // ---- half A: O_A += P_A V, then S_A = Q_A K(j+1)^T
-            if (!(got & 4u)) mbar_wait(bar(B_PREADY + 0), n_p0 & 1, abort_flag, p.status);
+            named_sync(kBarPReady + 0, kPReadyCount);
           }
           ++n_p0;
           tc_fence_after();
@@ -421,7 +433,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           trace_event(tc_cur, DYSPEC_TAG(0, 2, j));
           // ---- half B
           if (two) {
-            mbar_wait(bar(B_PREADY + 1), n_p1 & 1, abort_flag, p.status);
+            named_sync(kBarPReady + 1, kPReadyCount);
             ++n_p1;
             tc_fence_after();
             trace_event(tc_cur, DYSPEC_TAG(0, 3, j));
@@ -587,7 +599,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         }
         tmem_wait_st();
         tc_fence_before();
-        mbar_arrive(bar(B_PREADY + h));
+        named_arrive(kBarPReady + h, kPReadyCount);
         if (r == 0) trace_event(tc_cur, DYSPEC_TAG(1 + h, 5, j));
       }
 
