@@ -35,7 +35,11 @@ decrease, the closed form of the estimated acceptance rate in raw draft
 probabilities, Algorithm 2 at the last value == Algorithm 1, guesses at a
 position are draws without replacement); compact_kv by
 tests/test_compact_pins.py (hand example, no-op on a chain prefix, attention
-over the compacted cache == attention along the accepted path).
+over the compacted cache == attention along the accepted path); the paged
+forms by tests/test_paged_pins.py (a hand-written page table, the identity
+table == the contiguous layout, any scattering of the pages leaves the
+attention bit-identical, compaction == the contiguous one read back through
+the table).
 Nothing here is "parity unpinned".
 
 Readings where the paper is silent: scale = 1/sqrt(head_dim); consecutive query
@@ -46,7 +50,8 @@ Algorithm 3 draws its acceptance number from U(0,1) (printed as N(0,1)), the
 branches of a node are its children in increasing index, and the final token
 is drawn from the residual by inverse CDF in token order; Algorithm 1 samples
 the token before it adds the node, Algorithm 2 expands while v >= t, the draft
-model is a table lookup keyed by tree position (see build_tree_greedy).
+model is a table lookup keyed by tree position (see build_tree_greedy); in
+the paged layout the tree rows are a contiguous run outside the prefix pages.
 """
 from __future__ import annotations
 
@@ -482,3 +487,44 @@ def compact_kv(cache: np.ndarray, kv_row0: int, prefix_len: int, accepted_nodes:
     for i, row in enumerate(gathered):
         cache[base + i] = row
     return int(prefix_len) + len(nodes)
+
+
+# ----------------------------------------------------------------------------------------------------
+# Paged KV cache (the paper is silent on the cache's memory layout; this is the layout a serving stack
+# keeps its caches in).  The cache is a pool of pages of page_size rows.  Prefix token t of a request
+# lies in the request's page number t // page_size, at row t % page_size of that page; the request's
+# tree rows (one per node, in node order) are a contiguous run of pool rows of their own.
+# ----------------------------------------------------------------------------------------------------
+def paged_prefix_rows(page_table_row: Sequence[int], page_size: int, length: int) -> List[int]:
+    """Pool row of each of the first `length` tokens of a request whose pages are page_table_row."""
+    return [int(page_table_row[t // page_size]) * page_size + t % page_size for t in range(int(length))]
+
+
+def tree_attention_paged(q_bits, k_pool, v_pool, page_table, page_size: int, prefix_len, n_nodes, tree_row_offset,
+                         parents_list, scale: float | None = None):
+    """Tree-verify attention (same definition as tree_attention) with the prefix keys read through the
+    page table and the tree keys from rows tree_row_offset[r] ..  Returns float64 [sum n][H_q][D]."""
+    outs = []
+    qo = 0
+    for r in range(len(prefix_len)):
+        n, L = int(n_nodes[r]), int(prefix_len[r])
+        if n:
+            rows = paged_prefix_rows(page_table[r], page_size, L) + [int(tree_row_offset[r]) + j for j in range(n)]
+            outs.append(tree_attention(q_bits[qo:qo + n], k_pool[rows], v_pool[rows], L, parents_list[r], scale))
+        qo += n
+    if not outs:
+        return np.zeros((0,) + tuple(q_bits.shape[1:]), dtype=np.float64)
+    return np.concatenate(outs, axis=0)
+
+
+def compact_kv_paged(pool: np.ndarray, page_table_row: Sequence[int], page_size: int, tree_row0: int, prefix_len: int,
+                     accepted_nodes: Sequence[int]) -> int:
+    """The accepted nodes a_0 < a_1 < ... become prefix tokens L, L + 1, ...: the pool row of token
+    L + i (through the page table) takes the content of tree row tree_row0 + a_i.  Entries < 0 are
+    skipped.  Returns the new prefix length."""
+    nodes = [int(a) for a in accepted_nodes if int(a) >= 0]
+    L = int(prefix_len)
+    dst = paged_prefix_rows(page_table_row, page_size, L + len(nodes))[L:]
+    for d, a in zip(dst, nodes):
+        pool[d] = pool[int(tree_row0) + a]
+    return L + len(nodes)

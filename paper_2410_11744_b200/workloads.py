@@ -286,3 +286,65 @@ def make_draft_table(seed: int, n_rows: int, vocab: int, sharpness: float = 3.0,
     else:
         rows = _softmax_rows(rng.standard_normal((n_rows, vocab)).astype(np.float32) * np.float32(sharpness))
     return rows, rng.random(n_uniforms, dtype=np.float32)
+
+
+@dataclass
+class PagedWorkload:
+    """A Workload whose KV cache is a pool of pages: prefix token t of request r lies at pool row
+    page_table[r, t // page_size] * page_size + t % page_size; the tree rows of request r are the
+    contiguous pool rows tree_row_offset[r] .. + n_nodes[r]."""
+    base: Workload                  # q, parents, prefix_len, n_nodes as in the contiguous layout
+    page_size: int
+    page_table: np.ndarray          # int32 [n_req][pages_per_req], -1 = no page
+    tree_row_offset: np.ndarray     # int64 [n_req]
+    k: np.ndarray                   # uint16 bf16 bits [pool_rows][H_kv][D]
+    v: np.ndarray
+
+    @property
+    def pages_per_req(self) -> int:
+        return int(self.page_table.shape[1])
+
+    @property
+    def pool_rows(self) -> int:
+        return int(self.k.shape[0])
+
+
+def to_paged(w: Workload, page_size: int, seed: int = 0, room_for_accepted: bool = True) -> PagedWorkload:
+    """Scatters w's contiguous cache into a paged pool.  Every request gets enough pages for its prefix
+    (plus its tree size when room_for_accepted, so that accepted tokens have somewhere to go), the page
+    numbers of all requests are shuffled together, rows of a page past the prefix hold finite filler
+    (large values, so that a key that leaks through a mask shows), and the tree rows follow the pages
+    with odd gaps between requests."""
+    rng = np.random.default_rng(seed + 99173)
+    n_req = w.n_req
+    need = [-(-(int(w.prefix_len[r]) + (int(w.n_nodes[r]) if room_for_accepted else 0)) // page_size) for r in range(n_req)]
+    pages_per_req = max(need + [1])
+    n_pages = sum(need) + 2                                   # two pages nobody owns
+    ids = rng.permutation(n_pages)
+    page_table = np.full((n_req, pages_per_req), -1, dtype=np.int32)
+    at = 0
+    for r in range(n_req):
+        page_table[r, :need[r]] = ids[at:at + need[r]]
+        at += need[r]
+    tree_row_offset = np.zeros(n_req, dtype=np.int64)
+    row = n_pages * page_size
+    for r in range(n_req):
+        row += 3 + 2 * r
+        tree_row_offset[r] = row
+        row += int(w.n_nodes[r])
+    pool_rows = row + 5
+    shape = (pool_rows,) + tuple(w.k.shape[1:])
+    filler = np.array([0x4248, 0xC248, 0x4170, 0xC170], dtype=np.uint16)     # bf16 50, -50, 15, -15
+    k = filler[rng.integers(0, 4, size=shape)]
+    v = filler[rng.integers(0, 4, size=shape)]
+    for r in range(n_req):
+        o, L, n = int(w.kv_row_offset[r]), int(w.prefix_len[r]), int(w.n_nodes[r])
+        for t0 in range(0, L, page_size):
+            cnt = min(page_size, L - t0)
+            dst = int(page_table[r, t0 // page_size]) * page_size
+            k[dst:dst + cnt] = w.k[o + t0:o + t0 + cnt]
+            v[dst:dst + cnt] = w.v[o + t0:o + t0 + cnt]
+        t = int(tree_row_offset[r])
+        k[t:t + n] = w.k[o + L:o + L + n]
+        v[t:t + n] = w.v[o + L:o + L + n]
+    return PagedWorkload(w, int(page_size), page_table, tree_row_offset, k, v)
