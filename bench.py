@@ -205,14 +205,15 @@ def _time_replays(torch, graph, replays, tail=None):
     return e0.elapsed_time(e1)
 
 
-def measure_config(torch, runner, w, steps, warmup, device, sparse=False):
+def measure_config(torch, runner, w, steps, warmup, device, sparse=False, paged=None):
     """Device-resident timing of exactly `steps` steps, rotating over independent copies of the inputs
     that together exceed 2x L2.  The launch sequence of one rotation is captured in a CUDA graph so
     that the host's launch overhead (python, ctypes) does not starve the GPU."""
-    first = runner.DeviceBatch(w, device=device, sparse=sparse)
+    first = runner.DeviceBatch(w, device=device, sparse=sparse, paged=paged)
     nbytes, flops = algorithmic_cost(w, first.W)
     copies = max(2, min(64, int(np.ceil(2.0 * L2_BYTES / max(nbytes, 1)))))
-    batches = [first] + [runner.DeviceBatch(w, device=device, plan=first.plan, sparse=sparse) for _ in range(copies - 1)]
+    batches = [first] + [runner.DeviceBatch(w, device=device, plan=first.plan, sparse=sparse, paged=paged)
+                         for _ in range(copies - 1)]
     info = first.plan.describe()
     launches_per_step = 1 + 1 + (1 if info["split_groups"] > 0 else 0)
     for i in range(max(warmup, 3)):
@@ -406,6 +407,49 @@ def compaction_experiment(torch, B, peaks, device):
     return out
 
 
+def paged_experiment(torch, runner, workloads, B, peaks, device, configs=(2, 3, 4), page_size=256, steps=400):
+    """The same step with the cache in shuffled pages of page_size rows (prefix through a page table,
+    tree rows in a run of their own) beside the contiguous layout: same algorithmic bytes, so the two
+    times should agree.  After it, the paged accepted-path compaction (8 accepted nodes, 64 requests)."""
+    out = {"page_size": page_size, "configs": []}
+    for idx in configs:
+        w = workloads.make_config(idx)
+        mc = measure_config(torch, runner, w, steps, 3, device)
+        t_c = (mc["ms_per_step"], mc["attn_ms"])
+        del mc
+        torch.cuda.empty_cache()
+        mp = measure_config(torch, runner, w, steps, 3, device, paged=workloads.to_paged(w, page_size, idx))
+        out["configs"].append({"config": idx, "workload": w.name, "contiguous_step_us": t_c[0] * 1e3,
+                               "contiguous_attention_us": t_c[1] * 1e3, "paged_step_us": mp["ms_per_step"] * 1e3,
+                               "paged_attention_us": mp["attn_ms"] * 1e3, "bytes": mp["bytes"], "status": mp["status"]})
+        del mp
+        torch.cuda.empty_cache()
+    n_req, hkv, d, L, n, max_out = 64, 8, 128, 1024, 64, 16
+    pages_per_req = (L + n + page_size - 1) // page_size
+    n_pages = n_req * pages_per_req
+    rows = n_pages * page_size + n_req * n
+    k = torch.zeros((rows, hkv, d), dtype=torch.bfloat16, device=device)
+    v = torch.zeros((rows, hkv, d), dtype=torch.bfloat16, device=device)
+    table = torch.randperm(n_pages, device=device).to(torch.int32).reshape(n_req, pages_per_req).contiguous()
+    tree0 = n_pages * page_size + torch.arange(n_req, dtype=torch.int64, device=device) * n
+    Ls = torch.full((n_req,), L, dtype=torch.int32, device=device)
+    acc = torch.tensor([[1, 4, 9, 17, 22, 30, 41, 55, -1] + [0] * (max_out - 9)] * n_req, dtype=torch.int32, device=device)
+    cnt = torch.full((n_req,), 9, dtype=torch.int32, device=device)
+    newL = torch.zeros(n_req, dtype=torch.int32, device=device)
+    call = lambda: B.dyspec_compact_kv_paged(k, v, tree0, table, pages_per_req, page_size, Ls, acc, cnt, n_req, max_out,
+                                             hkv, d, newL)
+    call()
+    torch.cuda.synchronize()
+    g = _graph_of(torch, lambda: [call() for _ in range(20)])
+    g.replay()
+    torch.cuda.synchronize()
+    us = _time_replays(torch, g, 20) / 400 * 1e3
+    nbytes = n_req * 8 * hkv * d * 2 * 2 * 2
+    out["compaction"] = {"case": "64 requests, 8 kv heads, 8 accepted nodes", "call_us": us, "bytes": nbytes,
+                         "achieved_gbs": nbytes / (us * 1e-6) / 1e9}
+    return out
+
+
 def roofline_entry(m, peaks, peaks_kind):
     t_hbm = m["bytes"] / (peaks["hbm_gbs"] * 1e9)
     t_tc = m["flops"] / (peaks["bf16_tflops"] * 1e12)
@@ -551,6 +595,10 @@ def run_ours(args):
     if not args.no_per_config and world == 1:
         compaction = compaction_experiment(torch, binding, peaks, device)
 
+    paged = None
+    if not args.no_per_config and world == 1:
+        paged = paged_experiment(torch, runner, workloads, binding, peaks, device)
+
     # ---- the oracle on the host cores, bounded sample of the same workload
     times = time_oracle(w, budget_s=12.0)
     cpu_sec = sum(times) / len(times)
@@ -585,6 +633,8 @@ def run_ours(args):
         line["construction_experiment"] = construction
     if compaction:
         line["compaction_experiment"] = compaction
+    if paged:
+        line["paged_cache_experiment"] = paged
     print(json.dumps(line), flush=True)
     if use_dist:
         dist.barrier()

@@ -341,6 +341,49 @@ int dyspec_compact_kv(void* k_cache, void* v_cache, const int64_t* kv_row_offset
                       const int32_t* accepted_nodes, const int32_t* n_accepted, int n_req, int max_out, int n_kv_heads,
                       int head_dim, int32_t* new_prefix_len, dyspec_stream_t stream);
 
+/*
+ * (8) Paged KV cache (the paper does not fix the cache's memory layout; this is the layout of a serving
+ * stack).  k_cache / v_cache are a pool of pages of page_size rows (a power of two, >= 128, so that no
+ * key tile straddles two pages).  Prefix token t of request r lies at pool row
+ *     page_table[r * pages_per_req + t / page_size] * page_size + t % page_size
+ * and the request's tree rows (one per node, in node order) are the contiguous pool rows
+ * tree_row_offset[r] .. tree_row_offset[r] + n_r - 1, outside the prefix pages (scratch rows of the
+ * speculation step; dyspec_compact_kv_paged moves the accepted ones into the prefix pages).
+ * Rows of a mapped page past the prefix are read and masked: they must hold finite values (zero a page
+ * when it is allocated).  A page number that is negative or beyond the pool reads as zeros, it does not
+ * fault; the result for that request is then meaningless.
+ *
+ * dyspec_plan_create_paged: as dyspec_plan_create, with tree_row_offset (host int64 [n_req]) in place of
+ * kv_row_offset, kv_total_rows = rows of the pool, and the page size.  The plan works with
+ * dyspec_tree_attention_paged only (the contiguous calls return DYSPEC_ERR_INVALID_ARG for it, and this
+ * call for a contiguous plan); the mask builder and reorder calls take either kind.
+ *   page_table   dev int32 [n_req][pages_per_req]; entries past a request's last prefix page are not read.
+ *                Like q and the caches it is read before the preceding kernel of the stream is known to
+ *                have finished, so it must not be written by the kernel launched just before this call.
+ *   node_tiles   as in dyspec_tree_attention_ragged_sparse, or NULL
+ * Everything else as in dyspec_tree_attention_ragged.
+ */
+int dyspec_plan_create_paged(dyspec_plan_t** plan, int n_q_heads, int n_kv_heads, int head_dim, int n_req,
+                             const int32_t* prefix_len, const int32_t* n_nodes, const int64_t* tree_row_offset,
+                             int64_t kv_total_rows, int page_size, int words_per_row, float scale);
+int dyspec_tree_attention_paged(const dyspec_plan_t* plan, const void* q, const void* k_cache, const void* v_cache,
+                                const int32_t* page_table, int pages_per_req, const uint32_t* ancestor_bits,
+                                const uint32_t* node_tiles, void* out, void* workspace, size_t workspace_bytes,
+                                int32_t* status, dyspec_stream_t stream);
+
+/*
+ * (8b) Accepted-path compaction for the paged cache: for request r with accepted nodes a_0 < a_1 < ...
+ * (entries < 0 skipped) the pool row of prefix token L_r + i takes the content of tree row
+ * tree_row_offset[r] + a_i, for K and V, and new_prefix_len[r] = L_r + their number.  The page table must
+ * already hold a page for every new token; a token without one (entry < 0 or past pages_per_req) stops
+ * that request's copy there, new_prefix_len[r] counts what was kept, and *status = DYSPEC_ERR_INVALID_ARG.
+ * page_size: a power of two (any).  Other arguments as in dyspec_compact_kv; all arrays dev.
+ */
+int dyspec_compact_kv_paged(void* k_cache, void* v_cache, const int64_t* tree_row_offset, const int32_t* page_table,
+                            int pages_per_req, int page_size, const int32_t* prefix_len, const int32_t* accepted_nodes,
+                            const int32_t* n_accepted, int n_req, int max_out, int n_kv_heads, int head_dim,
+                            int32_t* new_prefix_len, int32_t* status, dyspec_stream_t stream);
+
 #ifdef __cplusplus
 }
 #endif

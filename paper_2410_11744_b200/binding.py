@@ -51,6 +51,9 @@ SIGNATURES = {
     "dyspec_build_tree_greedy": (_i32, [_vp, _i32, _i32, _vp, _i32, _vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "dyspec_build_tree_threshold": (_i32, [_vp, _i32, _i32, _vp, _i32, _vp, _i32, _f32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "dyspec_compact_kv": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _i32, _i32, _i32, _i32, _vp, _vp]),
+    "dyspec_plan_create_paged": (_i32, [_c.POINTER(_vp), _i32, _i32, _i32, _i32, _vp, _vp, _vp, _i64, _i32, _i32, _f32]),
+    "dyspec_tree_attention_paged": (_i32, [_vp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp, _vp, _sz, _vp, _vp]),
+    "dyspec_compact_kv_paged": (_i32, [_vp, _vp, _vp, _vp, _i32, _i32, _vp, _vp, _vp, _i32, _i32, _i32, _i32, _vp, _vp, _vp]),
     "dyspec_tree_attention_static": (_i32, [_vp, _vp, _vp, _i32, _vp, _i32, _vp, _i32, _i32, _i32, _i32, _f32, _vp, _vp]),
 }
 for _name, (_res, _args) in SIGNATURES.items():
@@ -119,16 +122,24 @@ class Plan:
 
     def __init__(self, n_q_heads: int, n_kv_heads: int, head_dim: int, prefix_len: Sequence[int],
                  n_nodes: Sequence[int], kv_row_offset: Sequence[int], kv_total_rows: int, words_per_row: int,
-                 scale: float = 0.0):
+                 scale: float = 0.0, page_size: Optional[int] = None):
+        """A page_size makes a plan for the paged cache: kv_row_offset is then the first tree row of each
+        request and kv_total_rows the rows of the pool (dyspec_plan_create_paged)."""
         n_req = len(prefix_len)
         pl = (_c.c_int32 * max(1, n_req))(*[int(x) for x in prefix_len])
         nn = (_c.c_int32 * max(1, n_req))(*[int(x) for x in n_nodes])
         off = (_c.c_int64 * max(1, n_req))(*[int(x) for x in kv_row_offset])
         handle = _vp()
-        _check(lib.dyspec_plan_create(_c.byref(handle), n_q_heads, n_kv_heads, head_dim, n_req,
-                                      _c.cast(pl, _vp), _c.cast(nn, _vp), _c.cast(off, _vp), int(kv_total_rows),
-                                      words_per_row, float(scale)), "dyspec_plan_create")
+        if page_size is not None:
+            _check(lib.dyspec_plan_create_paged(_c.byref(handle), n_q_heads, n_kv_heads, head_dim, n_req,
+                                                _c.cast(pl, _vp), _c.cast(nn, _vp), _c.cast(off, _vp), int(kv_total_rows),
+                                                int(page_size), words_per_row, float(scale)), "dyspec_plan_create_paged")
+        else:
+            _check(lib.dyspec_plan_create(_c.byref(handle), n_q_heads, n_kv_heads, head_dim, n_req,
+                                          _c.cast(pl, _vp), _c.cast(nn, _vp), _c.cast(off, _vp), int(kv_total_rows),
+                                          words_per_row, float(scale)), "dyspec_plan_create")
         self.handle = handle
+        self.page_size = int(page_size or 0)
         self.words_per_row = words_per_row
         self.total_nodes = int(sum(int(x) for x in n_nodes))
 
@@ -157,6 +168,13 @@ class Plan:
 
 def dyspec_plan_create(*args, **kwargs) -> Plan:
     return Plan(*args, **kwargs)
+
+
+def dyspec_plan_create_paged(n_q_heads: int, n_kv_heads: int, head_dim: int, prefix_len: Sequence[int],
+                             n_nodes: Sequence[int], tree_row_offset: Sequence[int], kv_total_rows: int, page_size: int,
+                             words_per_row: int, scale: float = 0.0) -> Plan:
+    return Plan(n_q_heads, n_kv_heads, head_dim, prefix_len, n_nodes, tree_row_offset, kv_total_rows, words_per_row,
+                scale, page_size=page_size)
 
 
 def dyspec_plan_destroy(plan: Plan) -> None:
@@ -307,3 +325,23 @@ def dyspec_compact_kv(k_cache, v_cache, kv_row_offset, prefix_len, accepted_node
     _check(lib.dyspec_compact_kv(_ptr(k_cache), _ptr(v_cache), _ptr(kv_row_offset), _ptr(prefix_len), _ptr(accepted_nodes),
                                  _ptr(n_accepted), n_req, max_out, n_kv_heads, head_dim, _ptr(new_prefix_len),
                                  _stream(stream)), "dyspec_compact_kv")
+
+
+def dyspec_tree_attention_paged(plan: Plan, q, k_cache, v_cache, page_table, pages_per_req: int, ancestor_bits,
+                                node_tiles, out, workspace=None, status=None, stream=None) -> None:
+    """Tree attention over a paged cache (see include/dyspec.h); node_tiles may be None."""
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(lib.dyspec_tree_attention_paged(plan.handle, _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(page_table),
+                                           int(pages_per_req), _ptr(ancestor_bits), _ptr(node_tiles), _ptr(out),
+                                           _ptr(workspace), ws_bytes, _ptr(status), _stream(stream)),
+           "dyspec_tree_attention_paged")
+
+
+def dyspec_compact_kv_paged(k_cache, v_cache, tree_row_offset, page_table, pages_per_req: int, page_size: int, prefix_len,
+                            accepted_nodes, n_accepted, n_req: int, max_out: int, n_kv_heads: int, head_dim: int,
+                            new_prefix_len=None, status=None, stream=None) -> None:
+    """Moves the accepted nodes' K/V rows from the tree rows into the prefix pages (see include/dyspec.h)."""
+    _check(lib.dyspec_compact_kv_paged(_ptr(k_cache), _ptr(v_cache), _ptr(tree_row_offset), _ptr(page_table),
+                                       int(pages_per_req), int(page_size), _ptr(prefix_len), _ptr(accepted_nodes),
+                                       _ptr(n_accepted), n_req, max_out, n_kv_heads, head_dim, _ptr(new_prefix_len),
+                                       _ptr(status), _stream(stream)), "dyspec_compact_kv_paged")

@@ -35,6 +35,10 @@ cudaError_t launch_build_tree_threshold(const float* draft_table, int n_rows, in
                                         int n_uniforms, const int32_t* root_row, int n_req, float threshold, int max_nodes,
                                         int32_t* parents, int32_t* tokens, float* values, float* child_values, int32_t* rows,
                                         int32_t* n_nodes, cudaStream_t stream);
+cudaError_t launch_compact_kv_paged(void* k_cache, void* v_cache, const int64_t* tree_row_offset, const int32_t* page_table,
+                                    int pages_per_req, int page_shift, const int32_t* prefix_len,
+                                    const int32_t* accepted_nodes, const int32_t* n_accepted, int n_req, int max_out,
+                                    int row_bytes, int32_t* new_prefix_len, int32_t* status, cudaStream_t stream);
 cudaError_t launch_compact_kv(void* k_cache, void* v_cache, const int64_t* kv_row_offset, const int32_t* prefix_len,
                               const int32_t* accepted_nodes, const int32_t* n_accepted, int n_req, int max_out,
                               int row_bytes, int32_t* new_prefix_len, cudaStream_t stream);
@@ -102,6 +106,7 @@ struct dyspec_plan {
   float scale = 0.f;
   int n_req = 0;
   int64_t kv_total_rows = 0;
+  int page_size = 0;                    // > 0: paged cache (prefix through a page table, kv_row0 = first tree row)
   int64_t total_nodes = 0;
   int max_nodes = 0;
   int regime = 0, bm = 64, bn = 64;
@@ -486,12 +491,34 @@ int dyspec_compact_kv(void* k_cache, void* v_cache, const int64_t* kv_row_offset
   return e == cudaSuccess ? DYSPEC_OK : cuda_failed(e, "compact launch");
 }
 
+int dyspec_compact_kv_paged(void* k_cache, void* v_cache, const int64_t* tree_row_offset, const int32_t* page_table,
+                            int pages_per_req, int page_size, const int32_t* prefix_len, const int32_t* accepted_nodes,
+                            const int32_t* n_accepted, int n_req, int max_out, int n_kv_heads, int head_dim,
+                            int32_t* new_prefix_len, int32_t* status, dyspec_stream_t stream) {
+  if (n_req < 0 || max_out <= 0 || n_kv_heads <= 0 || head_dim <= 0 || pages_per_req <= 0) return DYSPEC_ERR_INVALID_ARG;
+  if (page_size <= 0 || (page_size & (page_size - 1))) return DYSPEC_ERR_INVALID_ARG;
+  const int64_t row_bytes = int64_t(n_kv_heads) * head_dim * 2;
+  if (row_bytes % 16 != 0 || row_bytes > (1 << 24)) return DYSPEC_ERR_UNSUPPORTED;
+  if (n_req == 0) return DYSPEC_OK;
+  if (!k_cache || !v_cache || !tree_row_offset || !page_table || !prefix_len || !accepted_nodes || !n_accepted)
+    return DYSPEC_ERR_INVALID_ARG;
+  if (!aligned(k_cache, 16) || !aligned(v_cache, 16)) return DYSPEC_ERR_INVALID_ARG;
+  int shift = 0;
+  while ((1 << shift) < page_size) ++shift;
+  cudaError_t e = launch_compact_kv_paged(k_cache, v_cache, tree_row_offset, page_table, pages_per_req, shift, prefix_len,
+                                          accepted_nodes, n_accepted, n_req, max_out, int(row_bytes), new_prefix_len,
+                                          status, reinterpret_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? DYSPEC_OK : cuda_failed(e, "paged compact launch");
+}
+
 // Validates the arguments and runs the scheduler; no CUDA call.
 static int make_host_plan(dyspec_plan** out, int n_q_heads, int n_kv_heads, int head_dim, int n_req,
                           const int32_t* prefix_len, const int32_t* n_nodes, const int64_t* kv_row_offset,
-                          int64_t kv_total_rows, int words_per_row, float scale) {
+                          int64_t kv_total_rows, int words_per_row, float scale, int page_size = 0) {
   *out = nullptr;
   if (n_q_heads <= 0 || n_kv_heads <= 0 || n_req < 0 || kv_total_rows < 0) return DYSPEC_ERR_INVALID_ARG;
+  if (page_size < 0 || (page_size & (page_size - 1))) return DYSPEC_ERR_INVALID_ARG;
+  if (page_size != 0 && (page_size < 128 || page_size > (1 << 20))) return DYSPEC_ERR_UNSUPPORTED;
   if (n_req > 0 && (!prefix_len || !n_nodes || !kv_row_offset)) return DYSPEC_ERR_INVALID_ARG;
   if (words_per_row <= 0 || (words_per_row & 3)) return DYSPEC_ERR_INVALID_ARG;
   if (words_per_row > DYSPEC_MAX_NODES / 32) return DYSPEC_ERR_UNSUPPORTED;
@@ -508,13 +535,14 @@ static int make_host_plan(dyspec_plan** out, int n_q_heads, int n_kv_heads, int 
   pl->scale = scale > 0.f ? scale : 1.0f / std::sqrt(float(head_dim));
   pl->n_req = n_req;
   pl->kv_total_rows = kv_total_rows;
+  pl->page_size = page_size;
   int64_t node0 = 0;
   int max_rows = 0;
   for (int r = 0; r < n_req; ++r) {
     if (prefix_len[r] < 0 || n_nodes[r] < 0 || kv_row_offset[r] < 0) { delete pl; return DYSPEC_ERR_INVALID_ARG; }
     if (n_nodes[r] > DYSPEC_MAX_NODES) { delete pl; return DYSPEC_ERR_UNSUPPORTED; }
     if (32 * words_per_row < n_nodes[r]) { delete pl; return DYSPEC_ERR_INVALID_ARG; }
-    if (kv_row_offset[r] + prefix_len[r] + n_nodes[r] > kv_total_rows) { delete pl; return DYSPEC_ERR_INVALID_ARG; }
+    if (kv_row_offset[r] + (page_size ? 0 : prefix_len[r]) + n_nodes[r] > kv_total_rows) { delete pl; return DYSPEC_ERR_INVALID_ARG; }
     ReqInfo rq{};
     rq.kv_row0 = kv_row_offset[r]; rq.prefix_len = prefix_len[r]; rq.n_nodes = n_nodes[r]; rq.node0 = int32_t(node0);
     pl->reqs.push_back(rq);
@@ -543,6 +571,22 @@ int dyspec_plan_create(dyspec_plan_t** plan, int n_q_heads, int n_kv_heads, int 
   int rc = make_host_plan(&pl, n_q_heads, n_kv_heads, head_dim, n_req, prefix_len, n_nodes, kv_row_offset,
                           kv_total_rows, words_per_row, scale);
   *plan = nullptr;
+  if (rc != DYSPEC_OK) return rc;
+  rc = upload(*pl);
+  if (rc != DYSPEC_OK) { dyspec_plan_destroy(pl); return rc; }
+  *plan = pl;
+  return DYSPEC_OK;
+}
+
+int dyspec_plan_create_paged(dyspec_plan_t** plan, int n_q_heads, int n_kv_heads, int head_dim, int n_req,
+                             const int32_t* prefix_len, const int32_t* n_nodes, const int64_t* tree_row_offset,
+                             int64_t kv_total_rows, int page_size, int words_per_row, float scale) {
+  if (!plan) return DYSPEC_ERR_INVALID_ARG;
+  *plan = nullptr;
+  if (page_size <= 0) return DYSPEC_ERR_INVALID_ARG;
+  dyspec_plan* pl = nullptr;
+  int rc = make_host_plan(&pl, n_q_heads, n_kv_heads, head_dim, n_req, prefix_len, n_nodes, tree_row_offset,
+                          kv_total_rows, words_per_row, scale, page_size);
   if (rc != DYSPEC_OK) return rc;
   rc = upload(*pl);
   if (rc != DYSPEC_OK) { dyspec_plan_destroy(pl); return rc; }
@@ -646,10 +690,37 @@ int dyspec_tree_attention_ragged(const dyspec_plan_t* plan, const void* q, const
                                              workspace_bytes, status, stream);
 }
 
+static int run_attention(const dyspec_plan_t* plan, const void* q, const void* k_cache, const void* v_cache,
+                         const int32_t* page_table, int pages_per_req, const uint32_t* ancestor_bits,
+                         const uint32_t* node_tiles, void* out, void* workspace, size_t workspace_bytes, int32_t* status,
+                         dyspec_stream_t stream);
+
 int dyspec_tree_attention_ragged_sparse(const dyspec_plan_t* plan, const void* q, const void* k_cache,
                                         const void* v_cache, const uint32_t* ancestor_bits, const uint32_t* node_tiles,
                                         void* out, void* workspace, size_t workspace_bytes, int32_t* status,
                                         dyspec_stream_t stream) {
+  if (plan && plan->page_size != 0) return DYSPEC_ERR_INVALID_ARG;      // a paged plan needs its page table
+  return run_attention(plan, q, k_cache, v_cache, nullptr, 0, ancestor_bits, node_tiles, out, workspace, workspace_bytes,
+                       status, stream);
+}
+
+int dyspec_tree_attention_paged(const dyspec_plan_t* plan, const void* q, const void* k_cache, const void* v_cache,
+                                const int32_t* page_table, int pages_per_req, const uint32_t* ancestor_bits,
+                                const uint32_t* node_tiles, void* out, void* workspace, size_t workspace_bytes,
+                                int32_t* status, dyspec_stream_t stream) {
+  if (!plan || plan->page_size == 0) return DYSPEC_ERR_INVALID_ARG;
+  if (plan->n_ctas == 0) return DYSPEC_OK;
+  if (!page_table || !aligned(page_table, 4) || pages_per_req <= 0) return DYSPEC_ERR_INVALID_ARG;
+  for (const ReqInfo& rq : plan->reqs)                                   // every prefix token has a table entry
+    if ((int64_t(rq.prefix_len) + plan->page_size - 1) / plan->page_size > pages_per_req) return DYSPEC_ERR_INVALID_ARG;
+  return run_attention(plan, q, k_cache, v_cache, page_table, pages_per_req, ancestor_bits, node_tiles, out, workspace,
+                       workspace_bytes, status, stream);
+}
+
+static int run_attention(const dyspec_plan_t* plan, const void* q, const void* k_cache, const void* v_cache,
+                         const int32_t* page_table, int pages_per_req, const uint32_t* ancestor_bits,
+                         const uint32_t* node_tiles, void* out, void* workspace, size_t workspace_bytes, int32_t* status,
+                         dyspec_stream_t stream) {
   if (!plan) return DYSPEC_ERR_INVALID_ARG;
   if (!aligned(node_tiles, 4)) return DYSPEC_ERR_INVALID_ARG;
   if (plan->n_ctas == 0) return DYSPEC_OK;
@@ -679,6 +750,8 @@ int dyspec_tree_attention_ragged_sparse(const dyspec_plan_t* plan, const void* q
   p.items_stride = plan->items_stride;
   p.cluster_size = plan->cluster;
   p.trace = g_trace; p.trace_capacity = g_trace_capacity;
+  p.page_table = page_table; p.pages_per_req = pages_per_req;
+  for (p.page_shift = 0; page_table && (1 << p.page_shift) < plan->page_size; ++p.page_shift) {}
 
   cudaError_t e;
   if (plan->regime == 0) e = launch_attn_mma(plan->d, plan->n_ctas, mq, mk, mv, p, st);

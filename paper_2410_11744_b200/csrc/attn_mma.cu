@@ -130,8 +130,7 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           const uint32_t ph = ring_phase;
           if (++ring_stage == n_stages) { ring_stage = 0; ring_phase ^= 1u; }
           mbar_wait(bar_empty + 8 * stage, ph ^ 1, abort_flag, p.status);
-          const int64_t row = rq.kv_row0 + (t < n_prefix_tiles ? int64_t(t) * BN
-                                                               : int64_t(rq.prefix_len) + int64_t(t - n_prefix_tiles) * BN);
+          const int64_t row = kv_tile_row(p, item, t, n_prefix_tiles, BN);
           const uint32_t dst = s_kv + stage * L::kStageBytes;
           mbar_expect_tx(bar_full + 8 * stage, L::kStageBytes);
           for (int h = 0; h < L::kHalves; ++h) {

@@ -313,8 +313,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             t = n_prefix_tiles + __ffs(rem) - 1;
             rem &= rem - 1u;
           }
-          const int64_t row = rq.kv_row0 + (t < n_prefix_tiles ? int64_t(t) * BN
-                                                               : int64_t(rq.prefix_len) + int64_t(t - n_prefix_tiles) * BN);
+          const int64_t row = kv_tile_row(p, item, t, n_prefix_tiles, BN);
           for (int kv = 0; kv < 2; ++kv, ++sc) {
             const int slot = sc % kSlots;
             const uint32_t ph = (sc / kSlots) & 1;

@@ -80,9 +80,26 @@ struct AttnParams {
   int32_t cluster_size;            // > 1: one cluster per split group; partials are merged through distributed shared memory
   unsigned long long* trace;       // optional event trace (null in normal use): [0] = count, then entries
   int32_t trace_capacity;
+  // Paged cache (null page_table = contiguous layout): prefix token t of request r lies at cache row
+  // (page_table[r * pages_per_req + (t >> page_shift)] << page_shift) + (t & (page_size - 1)); the
+  // request's tree rows start at its kv_row0.  The page size is a multiple of every key-tile size,
+  // so a prefix tile never straddles two pages.
+  const int32_t* page_table;
+  int32_t pages_per_req;
+  int32_t page_shift;
 };
 
 #ifdef __CUDACC__
+// First cache row of key tile t of a work item's group (tiles of BN keys: prefix tiles, then tree tiles).
+__device__ __forceinline__ int64_t kv_tile_row(const AttnParams& p, const WorkItem& it, int t, int n_prefix_tiles, int BN) {
+  if (t >= n_prefix_tiles)
+    return it.kv_row0 + (p.page_table ? 0 : int64_t(it.prefix_len)) + int64_t(t - n_prefix_tiles) * BN;
+  const int64_t s = int64_t(t) * BN;
+  if (!p.page_table) return it.kv_row0 + s;
+  const int32_t page = __ldg(p.page_table + int64_t(it.req) * p.pages_per_req + (s >> p.page_shift));
+  return (int64_t(page) << p.page_shift) + (s & ((int64_t(1) << p.page_shift) - 1));
+}
+
 // ------------------------------------------------------------------------------------------------
 // PTX helpers (sm_100a).  Every wait is bounded: when it runs out the kernel records
 // DYSPEC_ERR_TIMEOUT and carries on without waiting any more, so it always terminates.

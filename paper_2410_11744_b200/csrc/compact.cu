@@ -33,6 +33,57 @@ compact_kv_kernel(uint4* __restrict__ k_cache, uint4* __restrict__ v_cache, cons
   if (new_prefix_len && blockIdx.y == 0 && blockIdx.z == 0 && threadIdx.x == 0) new_prefix_len[r] = L + kept;
 }
 
+// Paged cache: the accepted nodes' rows leave the request's tree rows (tree_row_offset[r] + a_i) for the
+// pages of the prefix: token L + i lies in page (L + i) / page_size of the request, at row (L + i) %
+// page_size of it.  Source and destination never overlap (the tree rows are outside the prefix pages),
+// so the steps are independent.
+__global__ void __launch_bounds__(256)
+compact_kv_paged_kernel(uint4* __restrict__ k_cache, uint4* __restrict__ v_cache, const int64_t* __restrict__ tree_row_offset,
+                        const int32_t* __restrict__ page_table, int pages_per_req, int page_shift,
+                        const int32_t* __restrict__ prefix_len, const int32_t* __restrict__ accepted_nodes,
+                        const int32_t* __restrict__ n_accepted, int max_out, int row_vecs,
+                        int32_t* __restrict__ new_prefix_len, int32_t* __restrict__ status) {
+  const int r = blockIdx.x;
+  uint4* cache = blockIdx.z == 0 ? k_cache : v_cache;
+  const int L = prefix_len[r];
+  const int64_t src0 = tree_row_offset[r];
+  const int n = min(n_accepted[r], max_out);
+  const int32_t* acc = accepted_nodes + size_t(r) * max_out;
+  const int32_t* pages = page_table + size_t(r) * pages_per_req;
+  const int col = blockIdx.y * blockDim.x + threadIdx.x;
+  int kept = 0;
+  for (int i = 0; i < n; ++i) {
+    const int a = acc[i];
+    if (a < 0) continue;                       // an emitted token without a tree node
+    const int t = L + kept;
+    const int pi = t >> page_shift;
+    const int page = pi < pages_per_req ? pages[pi] : -1;
+    if (page < 0) {                            // no page for this token: report it, keep what fits
+      if (status && col == 0 && blockIdx.z == 0) atomicCAS(status, 0, DYSPEC_ERR_INVALID_ARG);
+      break;
+    }
+    if (col < row_vecs) {
+      const int64_t dst = (int64_t(page) << page_shift) + (t & ((1 << page_shift) - 1));
+      cache[dst * row_vecs + col] = cache[(src0 + a) * int64_t(row_vecs) + col];
+    }
+    ++kept;
+  }
+  if (new_prefix_len && blockIdx.y == 0 && blockIdx.z == 0 && threadIdx.x == 0) new_prefix_len[r] = L + kept;
+}
+
+cudaError_t launch_compact_kv_paged(void* k_cache, void* v_cache, const int64_t* tree_row_offset, const int32_t* page_table,
+                                    int pages_per_req, int page_shift, const int32_t* prefix_len,
+                                    const int32_t* accepted_nodes, const int32_t* n_accepted, int n_req, int max_out,
+                                    int row_bytes, int32_t* new_prefix_len, int32_t* status, cudaStream_t stream) {
+  if (n_req <= 0) return cudaSuccess;
+  const int row_vecs = row_bytes / 16;
+  const dim3 grid(unsigned(n_req), unsigned((row_vecs + 255) / 256), 2u);
+  compact_kv_paged_kernel<<<grid, 256, 0, stream>>>(static_cast<uint4*>(k_cache), static_cast<uint4*>(v_cache),
+                                                    tree_row_offset, page_table, pages_per_req, page_shift, prefix_len,
+                                                    accepted_nodes, n_accepted, max_out, row_vecs, new_prefix_len, status);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_compact_kv(void* k_cache, void* v_cache, const int64_t* kv_row_offset, const int32_t* prefix_len,
                               const int32_t* accepted_nodes, const int32_t* n_accepted, int n_req, int max_out,
                               int row_bytes, int32_t* new_prefix_len, cudaStream_t stream) {

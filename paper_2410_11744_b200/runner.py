@@ -23,15 +23,21 @@ class DeviceBatch:
     """Buffers + plan for one Workload.  `step()` = mask build + attention (+ combine) on the current stream."""
 
     def __init__(self, w: Workload, device="cuda:0", words_per_row: int | None = None, upload: bool = True,
-                 plan: "B.Plan | None" = None, sparse: bool = False):
+                 plan: "B.Plan | None" = None, sparse: bool = False, paged=None):
+        """paged: a workloads.PagedWorkload of w; the cache buffers are then its pool and the attention
+        reads the prefix through its page table."""
         self.w = w
+        self.paged = paged
         self.sparse = sparse            # also emit per-node tile sets and let the attention skip empty tree tiles
         self.device = torch.device(device)
         max_n = int(w.n_nodes.max()) if w.n_req else 0
         self.W = words_per_row or B.dyspec_words_per_row(max_n)
         self.total_nodes = w.total_nodes
-        self.kv_total_rows = int(w.k.shape[0])
+        self.kv_total_rows = int(w.k.shape[0]) if paged is None else paged.pool_rows
         # a plan depends only on the batch structure, so buffers with the same structure can share one
+        if plan is None and paged is not None:
+            plan = B.Plan(w.n_q_heads, w.n_kv_heads, w.head_dim, w.prefix_len, w.n_nodes, paged.tree_row_offset,
+                          self.kv_total_rows, self.W, 0.0, page_size=paged.page_size)
         self.plan = plan or B.Plan(w.n_q_heads, w.n_kv_heads, w.head_dim, w.prefix_len, w.n_nodes, w.kv_row_offset,
                                    self.kv_total_rows, self.W, 0.0)
         dev = self.device
@@ -52,8 +58,11 @@ class DeviceBatch:
         self.parents = torch.from_numpy(w.parents_concat if self.total_nodes else np.zeros(1, np.int32)).to(dev)
         self.q = _bits_to_bf16(w.q if self.total_nodes else np.zeros((1, w.n_q_heads, w.head_dim), np.uint16), dev)
         kv_shape = (max(1, self.kv_total_rows), w.n_kv_heads, w.head_dim)
-        self.k = _bits_to_bf16(w.k if self.kv_total_rows else np.zeros(kv_shape, np.uint16), dev)
-        self.v = _bits_to_bf16(w.v if self.kv_total_rows else np.zeros(kv_shape, np.uint16), dev)
+        src = w if self.paged is None else self.paged
+        self.k = _bits_to_bf16(src.k if self.kv_total_rows else np.zeros(kv_shape, np.uint16), dev)
+        self.v = _bits_to_bf16(src.v if self.kv_total_rows else np.zeros(kv_shape, np.uint16), dev)
+        if self.paged is not None:
+            self.page_table = torch.from_numpy(np.ascontiguousarray(self.paged.page_table)).to(dev)
 
     def build_mask(self):
         if self.sparse:
@@ -63,7 +72,11 @@ class DeviceBatch:
             B.dyspec_plan_build_tree_mask(self.plan, self.parents, self.bits, self.depths, self.status)
 
     def attention(self):
-        if self.sparse:
+        if self.paged is not None:
+            B.dyspec_tree_attention_paged(self.plan, self.q, self.k, self.v, self.page_table, self.paged.pages_per_req,
+                                          self.bits, self.node_tiles if self.sparse else None, self.out,
+                                          self.workspace, self.status)
+        elif self.sparse:
             B.dyspec_tree_attention_ragged_sparse(self.plan, self.q, self.k, self.v, self.bits, self.node_tiles,
                                                   self.out, self.workspace, self.workspace_bytes, self.status)
         else:
