@@ -1,14 +1,24 @@
-// Tree-verify attention, warp-level tile regime (Sec. 2 "Tree Attention"; App. C: prefix keys are in the mask).
+// Tree-verify attention, small-tile regime (Sec. 2 "Tree Attention"; App. C: prefix keys are in the mask).
 //
 // Used when the packed query tile (tree nodes x GQA group) is small, so the work is bound by
-// streaming K/V from HBM rather than by the tensor pipe.  One CTA per SM = 4 compute warps (16 query rows
-// each, BM = 64) + 1 producer warp.  The producer streams 64-key K and V tiles through TMA into a
-// 128-byte-swizzled shared-memory ring guarded by mbarriers; compute warps run QK^T and PV with
-// mma.sync.m16n8k16 (bf16 in, fp32 accumulate), an fp32 online softmax in the exp2 domain, and apply
-// the ancestor bitmask on tree tiles.  A CTA walks its list of work items; an item either writes
-// final bf16 rows or an fp32 partial (O, m, l) for the split-KV combine kernel.  In cluster mode
-// (uniform small batches) the splits of a query tile are the CTAs of one thread-block cluster and
-// are merged on chip through distributed shared memory instead.
+// streaming K/V from HBM rather than by the tensor pipe.  One CTA per SM, BM = 64 query rows:
+//   warp 8     producer: streams 64-key K and V tiles through TMA into a 128-byte-swizzled
+//              shared-memory ring guarded by mbarriers;
+//   warp 9     issues S = Q K^T on the tensor cores (tcgen05.mma, M = 64, N = 64, both operands from
+//              shared memory) as soon as a stage's K tile has landed; every ring stage has a score
+//              buffer of its own in tensor memory, so the scores run ahead of the softmax;
+//   warps 0-7  two sets of four compute warps (16 query rows per warp).  The sets take alternate key
+//              tiles: a warp reads its 16 x 64 scores with tcgen05.ld (the 16x256b shape returns them
+//              laid out like an mma.sync accumulator), applies the ancestor bitmask on tree tiles,
+//              runs the fp32 online softmax in the exp2 domain and accumulates O += P V with
+//              mma.sync.m16n8k16 (P stays in registers, V through ldmatrix.trans).  The per-tile code
+//              is a chain of dependent instructions, so one warp per scheduler leaves the SM mostly
+//              idle; two interleaved tiles per scheduler double the rate.  At the end of an item set 1
+//              hands its (O, m, l) to set 0 through shared memory, thread to thread.
+// A CTA walks its list of work items; an item either writes final bf16 rows or an fp32 partial
+// (O, m, l) for the split-KV combine kernel.  In cluster mode (uniform small batches) the splits of
+// a query tile are the CTAs of one thread-block cluster and are merged on chip through distributed
+// shared memory instead.
 #include "common.cuh"
 
 namespace dyspec {
@@ -17,8 +27,12 @@ namespace {
 
 constexpr int BM = 64;       // packed query rows per tile
 constexpr int BN = 64;       // keys per tile
-constexpr int kComputeWarps = 4;
-constexpr int kThreads = (kComputeWarps + 1) * 32;
+constexpr int kComputeWarps = 4;                            // per warp set: 16 query rows each
+constexpr int kSets = 2;                                    // two sets take alternate key tiles
+constexpr int kProducerWarp = kSets * kComputeWarps;        // TMA
+constexpr int kMmaWarp = kProducerWarp + 1;                 // tcgen05.mma issuer for S = Q K^T
+constexpr int kThreads = (kSets * kComputeWarps + 2) * 32;
+constexpr int kBarExchFull = 2, kBarExchFree = 3, kBarRingIdle = 4;   // named barriers between the two warp sets
 
 template <int D>
 struct SmemLayout {
@@ -29,13 +43,11 @@ struct SmemLayout {
   static constexpr int kQBytes = BM * 128 * kHalves;
   static constexpr int kStageBytes = 2 * kTileBytes;     // K then V
   static constexpr int kBarOffset = kQBytes + kStages * kStageBytes;
-  static constexpr int kTotal = kBarOffset + 256;
+  static constexpr int kExchMlOffset = kBarOffset + 512;  // set 1 -> set 0: (m, l) of every thread's two rows
+  static constexpr int kTotal = kExchMlOffset + kComputeWarps * 32 * 16;
+  static constexpr int kTmemCols = 512;                  // one 64-column score buffer per ring stage (power of two)
 };
 
-__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
-}
 __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
                : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
@@ -51,6 +63,49 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1
 // panels with the 128-byte TMA swizzle (chunk index XOR row mod 8 inside each 128-byte row).
 __device__ __forceinline__ uint32_t swz(int row, int chunk, int panel_bytes) {
   return static_cast<uint32_t>((chunk >> 3) * panel_bytes + row * 128 + (((chunk & 7) ^ (row & 7)) << 4));
+}
+
+// ---- tcgen05 pieces for S = Q K^T (M = 64 query rows, N = 64 keys, fp32 scores in tensor memory)
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// Both operands from shared memory; descriptors as (low word, constant high word).
+__device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+      "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(acc) : "memory");
+}
+// Shared-memory matrix descriptor of a K-major operand stored as 128-byte rows with the 128-byte swizzle
+// (8-row groups 1024 bytes apart): low word = address >> 4 | (16 >> 4) << 16; high word = 1024 >> 4 |
+// version 1 | swizzle mode 2.
+constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
+__device__ __forceinline__ uint32_t desc_lo(uint32_t saddr) { return (saddr >> 4) | (1u << 16); }
+// Instruction descriptor, kind::f16: bf16 x bf16 -> fp32, both operands K-major, M = 64, N = 64.
+constexpr uint32_t kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(BN >> 3) << 17) | (uint32_t(BM >> 4) << 24);
+// With M = 64 the accumulator row r lives in TMEM lane 32 (r / 16) + r % 16, so warp w reads rows
+// 16 w .. 16 w + 15 from its own lane quarter, and the 16x256b load shape hands them out exactly as
+// mma.sync hands out a 16 x 8 accumulator tile: registers 4j .. 4j+3 of lane (gid, tig) are
+// (row gid, columns 8j + 2 tig, +1) and (row gid + 8, same columns).
+__device__ __forceinline__ void tmem_ld_scores(uint32_t taddr, float (&s)[BN / 8][4]) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.16x256b.x8.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int j = 0; j < BN / 8; ++j) {
+    s[j][0] = __uint_as_float(r[4 * j]); s[j][1] = __uint_as_float(r[4 * j + 1]);
+    s[j][2] = __uint_as_float(r[4 * j + 2]); s[j][3] = __uint_as_float(r[4 * j + 3]);
+  }
 }
 
 }  // namespace
@@ -69,49 +124,70 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   const uint32_t s_q = smem_u32(smem);
   const uint32_t s_kv = s_q + L::kQBytes;
   const uint32_t s_bar = s_q + L::kBarOffset;
-  // barriers: full[kStages], empty[kStages], q_full, q_empty, src[8] (one per cluster peer)
+  // barriers: full[kStages], empty[kStages], q_full, q_empty, src[8] (one per cluster peer), s_full[kStages]
   const uint32_t bar_full = s_bar, bar_empty = s_bar + 8 * kStages;
   const uint32_t bar_qfull = s_bar + 16 * kStages, bar_qempty = bar_qfull + 8, bar_src = bar_qempty + 8;
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::kBarOffset + 16 * kStages + 16 + 64);
-  // In cluster mode the last two ring stages are not part of the ring: peers push their partial rows
-  // into them (see the epilogue), possibly while this CTA is still streaming K/V through the others.
-  const int n_stages = p.cluster_size > 1 ? kStages - 2 : kStages;
+  const uint32_t bar_sfull = bar_src + 64;
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::kBarOffset + 24 * kStages + 16 + 64);
+  volatile uint32_t* tmem_holder = reinterpret_cast<volatile uint32_t*>(smem + L::kBarOffset + 24 * kStages + 16 + 64 + 4);
+  float4* exch_ml = reinterpret_cast<float4*>(smem + L::kExchMlOffset);
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  // trace: the last 2048 entries of the buffer hold 8 wall-clock stamps for each of the first 256 CTAs
+  // trace: the last 2048 entries of the buffer hold 8 wall-clock stamps for each of the first 256 CTAs, all
+  // taken by thread 0 for the CTA's first item: 0 entry, 3 first scores read, 5 key loop done, 1 set 1's
+  // partial folded in, 6 partial parked, 2 pushes issued, 4 (owners) last fold done, 7 exit
   auto stamp = [&](int k) {
     if (p.trace != nullptr && blockIdx.x < 256 && p.trace_capacity > 4096)
       p.trace[p.trace_capacity - 2048 + 8 * blockIdx.x + k] = global_timer_ns();
   };
   if (threadIdx.x == 0) stamp(0);
+  if (threadIdx.x == kProducerWarp * 32) {      // the descriptors' fetch overlaps the set-up below
+    prefetch_tensormap(&map_q);
+    prefetch_tensormap(&map_k);
+    prefetch_tensormap(&map_v);
+  }
+  const WorkItem* my_items = p.items + size_t(blockIdx.x) * p.items_stride;
+  const int item_begin = 0;
+  const int item_end = my_items[0].n_in_cta;    // issued before the barrier below, used after it
+  // Ring depth.  The last stage is where warp set 1 hands its partial output to set 0 (without clusters
+  // the ring is busy with the next item's tiles by then).  In cluster mode a CTA that merges (an owner)
+  // keeps the last TWO stages free for the partial rows its peers push into them, possibly while it
+  // is still streaming K/V itself, and hands over through a ring stage once the ring is idle; a CTA
+  // that does not merge receives nothing (it is the one with the most tiles).
+  const bool merge_owner = p.cluster_size > 1 && ((uint32_t(my_items[0].merge_owners) >> cluster_ctarank()) & 1u);
+  float4* exch_o = reinterpret_cast<float4*>(smem + L::kQBytes + (merge_owner ? 2 : kStages - 1) * L::kStageBytes);
+  const int n_stages = merge_owner ? kStages - 2 : kStages - 1;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
       mbar_init(bar_full + 8 * s, 1);
       mbar_init(bar_empty + 8 * s, kComputeWarps);
+      mbar_init(bar_sfull + 8 * s, 1);
     }
     mbar_init(bar_qfull, 1);
-    mbar_init(bar_qempty, kComputeWarps);
+    mbar_init(bar_qempty, 1);                    // arrived on by the commit behind an item's last Q K^T
     for (int k = 0; k < 8; ++k) mbar_init(bar_src + 8 * k, 1);
     *abort_flag = 0;
     fence_barrier_init();
   }
+  if (warp == kMmaWarp) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32(const_cast<uint32_t*>(tmem_holder))), "r"(uint32_t(L::kTmemCols)) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
   __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_holder;
   if (p.cluster_size > 1) cluster_arrive();     // "my barriers exist"; peers wait for this only just before they push
 
-  const WorkItem* my_items = p.items + size_t(blockIdx.x) * p.items_stride;
-  const int item_begin = 0;
-  const int item_end = my_items[0].n_in_cta;
   const int g = p.group_size;
 
   trigger_dependents();     // the combine kernel may be scheduled; it waits for this grid before reading partials
-  if (warp == kComputeWarps) {
+  if (warp == kProducerWarp) {
     // ------------------------------------------------------------------ producer warp (one lane issues)
     if (lane == 0) {
-      prefetch_tensormap(&map_q);
-      prefetch_tensormap(&map_k);
-      prefetch_tensormap(&map_v);
       int ring_stage = 0;    // ring position of the next key tile of this CTA
       uint32_t ring_phase = 0;
       uint32_t qit = 0;      // running item counter (Q buffer phase)
@@ -141,17 +217,53 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       }
     }
     if (p.cluster_size > 1) cluster_wait();      // pairs with the arrive above (all threads of the cluster take part)
-    return;
-  }
-
+  } else if (warp == kMmaWarp) {
+    // ------------------------------------------------------------------ S = Q K^T on the tensor cores (one lane issues)
+    // Ring stage s has a score buffer of its own (TMEM columns 64 s ..): as soon as the stage's K tile
+    // has landed its scores are computed, so they run ahead of the softmax by the depth of the ring.
+    // The buffer is free again when the stage is (the compute warps release the stage after they have
+    // read the scores and used V), so no barrier of its own guards it.
+    if (lane == 0) {
+      int ring_stage = 0;
+      uint32_t ring_phase = 0;
+      uint32_t qit = 0;
+      const uint32_t q_lo = desc_lo(s_q);
+      for (int w = item_begin; w < item_end; ++w, ++qit) {
+        const WorkItem item = my_items[w];
+        mbar_wait(bar_qfull, qit & 1, abort_flag, p.status);
+        for (int t = item.tile_begin; t < item.tile_end; ++t) {
+          const int stage = ring_stage;
+          const uint32_t ph = ring_phase;
+          if (++ring_stage == n_stages) { ring_stage = 0; ring_phase ^= 1u; }
+          mbar_wait(bar_full + 8 * stage, ph, abort_flag, p.status);
+          tc_fence_after();
+          const uint32_t k_lo = desc_lo(s_kv + stage * L::kStageBytes);
+#pragma unroll
+          for (int ks = 0; ks < KS; ++ks) {
+            const uint32_t off = uint32_t((ks >> 2) * L::kPanelBytes + (ks & 3) * 32) >> 4;   // Q and K panels have the same size
+            umma_ss(tmem_base + uint32_t(stage) * BN, q_lo + off, k_lo + off, kDescHi, kIdescQK, ks > 0 ? 1u : 0u);
+          }
+          tc_commit(bar_sfull + 8 * stage);
+        }
+        tc_commit(bar_qempty);                    // the Q tile may be replaced once these products are done
+      }
+    }
+    if (p.cluster_size > 1) cluster_wait();
+  } else {
   // -------------------------------------------------------------------- compute warps
   // Everything read so far (work items, Q/K/V through TMA) is input that no kernel of this stream
   // writes.  The mask, the partials and the output are: wait for the preceding kernels here, while
   // the producer warp keeps streaming K/V.
   grid_dependency_wait();
+  // "Every peer has initialised its barriers": the peers arrived right after their set-up, long before
+  // the first K/V tile can be here, so waiting now costs nothing and the merge does not have to.
+  if (p.cluster_size > 1) cluster_wait();
   const int gid = lane >> 2;      // row within an 8-row slab
   const int tig = lane & 3;       // column pair within an 8-column tile
-  const int wrow = warp * 16;
+  const int set = warp >> 2;      // warp set: takes the item's key tiles of this parity
+  const int cw = warp & 3;        // row block inside the set
+  const int wrow = cw * 16;
+  const int ctid = cw * 32 + lane;   // thread index inside the set
   int ring_stage = 0;
   uint32_t ring_phase = 0, qit = 0;
 
@@ -165,19 +277,14 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     const int node_lo = row_lo >> p.log2_g, node_hi = row_hi >> p.log2_g;
     const bool ok_lo = row_lo < n_rows, ok_hi = row_hi < n_rows;
 
-    // Q fragments, kept in registers for the whole item.
-    uint32_t qf[KS][4];
-    if (threadIdx.x == 0 && w == item_begin) stamp(1);
-    mbar_wait(bar_qfull, qit & 1, abort_flag, p.status);
-    if (threadIdx.x == 0 && w == item_begin) stamp(2);
-#pragma unroll
-    for (int ks = 0; ks < KS; ++ks) {
-      const int row = wrow + (lane & 15);
-      const int chunk = ks * 2 + (lane >> 4);
-      ldmatrix_x4(s_q + swz(row, chunk, BM * 128), qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3]);
+
+    // The mask words of the first tree tile are fetched now: the tree tiles come last in an item, and a
+    // global load in front of the last tile's softmax would sit on the critical path of the CTA.
+    uint2 pre_lo = make_uint2(0u, 0u), pre_hi = make_uint2(0u, 0u);
+    if (item.tile_end > n_prefix_tiles) {
+      if (ok_lo) pre_lo = __ldg(reinterpret_cast<const uint2*>(p.bits + size_t(rq.node0 + node_lo) * p.words_per_row));
+      if (ok_hi) pre_hi = __ldg(reinterpret_cast<const uint2*>(p.bits + size_t(rq.node0 + node_hi) * p.words_per_row));
     }
-    __syncwarp();
-    if (lane == 0) mbar_arrive(bar_qempty);
 
     float o[DT][4];
 #pragma unroll
@@ -188,29 +295,18 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       const int stage = ring_stage;
       const uint32_t ph = ring_phase;
       if (++ring_stage == n_stages) { ring_stage = 0; ring_phase ^= 1u; }
+      if (((t - item.tile_begin) & 1) != set) continue;     // the other set's tile
       const uint32_t s_k = s_kv + stage * L::kStageBytes;
       const uint32_t s_v = s_k + L::kTileBytes;
+      // ---- S = Q K^T (16 x 64 per warp) from the stage's score buffer.  The stage's own barrier is
+      //      complete by then (the products were issued behind it); waiting on it as well costs one
+      //      probe and makes the TMA-written V tile visible to this thread.
+      mbar_wait(bar_sfull + 8 * stage, ph, abort_flag, p.status);
       mbar_wait(bar_full + 8 * stage, ph, abort_flag, p.status);
+      tc_fence_after();
       if (threadIdx.x == 0 && w == item_begin && t == item.tile_begin) stamp(3);
-      if (threadIdx.x == 0 && w == item_begin && t == item.tile_end - 1) stamp(4);
-
-      // ---- S = Q K^T (16 x 64 per warp)
       float s[BN / 8][4];
-#pragma unroll
-      for (int j = 0; j < BN / 8; ++j) { s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f; }
-#pragma unroll
-      for (int ks = 0; ks < KS; ++ks) {
-#pragma unroll
-        for (int jp = 0; jp < BN / 16; ++jp) {
-          const int mi = lane >> 3;
-          const int row = jp * 16 + (lane & 7) + ((mi >> 1) << 3);
-          const int chunk = ks * 2 + (mi & 1);
-          uint32_t b0, b1, b2, b3;
-          ldmatrix_x4(s_k + swz(row, chunk, L::kPanelBytes), b0, b1, b2, b3);
-          mma_bf16(s[2 * jp], qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3], b0, b1);
-          mma_bf16(s[2 * jp + 1], qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3], b2, b3);
-        }
-      }
+      tmem_ld_scores(tmem_base + (uint32_t(cw * 32) << 16) + uint32_t(stage) * BN, s);
 
       // ---- visibility of the 64 key columns for this thread's two rows
       uint64_t vis_lo, vis_hi;
@@ -223,15 +319,14 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       } else {
         const int u = t - n_prefix_tiles;
         own = min(BN, rq.n_nodes - u * BN);
-        vis_lo = vis_hi = 0ull;
-        if (ok_lo) {
-          const uint2 wv = __ldg(reinterpret_cast<const uint2*>(p.bits + size_t(rq.node0 + node_lo) * p.words_per_row) + u);
-          vis_lo = (uint64_t(wv.y) << 32) | wv.x;
+        uint2 w_lo = pre_lo, w_hi = pre_hi;
+        if (u > 0) {
+          w_lo = w_hi = make_uint2(0u, 0u);
+          if (ok_lo) w_lo = __ldg(reinterpret_cast<const uint2*>(p.bits + size_t(rq.node0 + node_lo) * p.words_per_row) + u);
+          if (ok_hi) w_hi = __ldg(reinterpret_cast<const uint2*>(p.bits + size_t(rq.node0 + node_hi) * p.words_per_row) + u);
         }
-        if (ok_hi) {
-          const uint2 wv = __ldg(reinterpret_cast<const uint2*>(p.bits + size_t(rq.node0 + node_hi) * p.words_per_row) + u);
-          vis_hi = (uint64_t(wv.y) << 32) | wv.x;
-        }
+        vis_lo = (uint64_t(w_lo.y) << 32) | w_lo.x;
+        vis_hi = (uint64_t(w_hi.y) << 32) | w_hi.x;
       }
 
       // ---- online softmax (exp2 domain)
@@ -309,6 +404,40 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
     l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1);
     l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
+
+    // ---- the two warp sets took alternate tiles: set 1 hands its (O, m, l) to set 0, thread to thread
+    //      (thread ctid of either set owns the same rows and columns), and set 0 alone runs the epilogue.
+    if (merge_owner)              // the hand-over buffer is a ring stage here: both sets must be done with the ring
+      asm volatile("bar.sync %0, %1;" ::"n"(kBarRingIdle), "n"(kSets * kComputeWarps * 32) : "memory");
+    if (set == 1) {
+      if (w != item_begin)        // set 0 has read the previous item's values
+        asm volatile("bar.sync %0, %1;" ::"n"(kBarExchFree), "n"(kSets * kComputeWarps * 32) : "memory");
+#pragma unroll
+      for (int j = 0; j < DT; ++j) exch_o[j * (kComputeWarps * 32) + ctid] = make_float4(o[j][0], o[j][1], o[j][2], o[j][3]);
+      exch_ml[ctid] = make_float4(m_lo, m_hi, l_lo, l_hi);
+      asm volatile("bar.arrive %0, %1;" ::"n"(kBarExchFull), "n"(kSets * kComputeWarps * 32) : "memory");
+      if (p.cluster_size <= 1) continue;         // in cluster mode the set lends its threads to the merge below
+    } else {
+    asm volatile("bar.sync %0, %1;" ::"n"(kBarExchFull), "n"(kSets * kComputeWarps * 32) : "memory");
+    {
+      const float4 ml = exch_ml[ctid];
+      const float mn_lo = fmaxf(m_lo, ml.x), mn_hi = fmaxf(m_hi, ml.y);
+      const float ref_lo = mn_lo == -INFINITY ? 0.f : mn_lo, ref_hi = mn_hi == -INFINITY ? 0.f : mn_hi;
+      const float ka_lo = fast_exp2(m_lo - ref_lo), kb_lo = fast_exp2(ml.x - ref_lo);
+      const float ka_hi = fast_exp2(m_hi - ref_hi), kb_hi = fast_exp2(ml.y - ref_hi);
+#pragma unroll
+      for (int j = 0; j < DT; ++j) {
+        const float4 ob = exch_o[j * (kComputeWarps * 32) + ctid];
+        o[j][0] = o[j][0] * ka_lo + ob.x * kb_lo; o[j][1] = o[j][1] * ka_lo + ob.y * kb_lo;
+        o[j][2] = o[j][2] * ka_hi + ob.z * kb_hi; o[j][3] = o[j][3] * ka_hi + ob.w * kb_hi;
+      }
+      l_lo = l_lo * ka_lo + ml.z * kb_lo; l_hi = l_hi * ka_hi + ml.w * kb_hi;
+      m_lo = mn_lo; m_hi = mn_hi;
+    }
+    if (threadIdx.x == 0 && w == item_begin) stamp(1);
+    if (w + 1 < item_end)
+      asm volatile("bar.arrive %0, %1;" ::"n"(kBarExchFree), "n"(kSets * kComputeWarps * 32) : "memory");
+    }
     if (p.cluster_size > 1) {
       // ---- split-KV combine inside a thread-block cluster: the CTAs of a cluster hold the splits of
       // one query tile (a CTA owns exactly one item in this mode).  The scheduler names the owners
@@ -335,8 +464,8 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       if (own && threadIdx.x == 0)
         for (int s_ = 0; s_ < C; ++s_)
           if (s_ != rank) mbar_expect_tx(bar_src + 8 * s_, chunk_bytes);
-      asm volatile("bar.sync 1, %0;" ::"n"(kComputeWarps * 32) : "memory");     // all warps are done with the ring
-      {
+      // (every warp is done with the ring: set 0's warps met at the hand-over barrier, which set 1 arrived on)
+      if (set == 0) {
         // columns are XOR-swizzled by the row so that the 8 rows a warp stores at once hit different banks
         const int r_lo = wrow + gid, r_hi = r_lo + 8;
         float* c_lo = send + (r_lo >> log2r) * chunk_floats;
@@ -353,21 +482,25 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           c_hi[R * D + rr_hi] = m_hi; c_hi[R * D + R + rr_hi] = l_hi;
         }
       }
+      if (threadIdx.x == 0) stamp(6);
       fence_proxy_async();                                 // the bulk copies below read what was just stored
-      cluster_wait();                                      // every peer has initialised its barriers (arrived long ago)
-      asm volatile("bar.sync 1, %0;" ::"n"(kComputeWarps * 32) : "memory");
-      const bool pusher = warp == 0 && lane < C && lane != rank && ((owners >> lane) & 1u);
+      asm volatile("bar.sync 1, %0;" ::"n"(kSets * kComputeWarps * 32) : "memory");
+      // one copy per (owner, quarter of the group): four lanes of warp 0 per owner, so that the copies overlap
+      const int tgt = lane & 7, piece = lane >> 3;
+      const bool pusher = warp == 0 && tgt < C && tgt != rank && ((owners >> tgt) & 1u);
       if (pusher) {
-        const uint32_t slot = uint32_t(rank < lane ? rank : rank - 1);          // where owner `lane` keeps source `rank`
-        const uint32_t oi = uint32_t(__popc(owners & ((1u << lane) - 1u)));     // the group that owner is responsible for
-        dsmem_push(map_to_cta(smem_u32(recv) + slot * chunk_bytes, uint32_t(lane)),
-                   smem_u32(send) + oi * chunk_bytes, chunk_bytes, map_to_cta(bar_src + 8 * rank, uint32_t(lane)));
+        const uint32_t slot = uint32_t(rank < tgt ? rank : rank - 1);           // where owner `tgt` keeps source `rank`
+        const uint32_t oi = uint32_t(__popc(owners & ((1u << tgt) - 1u)));      // the group that owner is responsible for
+        const uint32_t part = chunk_bytes >> 2, at = uint32_t(piece) * part;    // a multiple of 16 bytes for every R and D
+        dsmem_push(map_to_cta(smem_u32(recv) + slot * chunk_bytes + at, uint32_t(tgt)),
+                   smem_u32(send) + oi * chunk_bytes + at, part, map_to_cta(bar_src + 8 * rank, uint32_t(tgt)));
       }
+      if (threadIdx.x == 0) stamp(2);
       if (own) {
         float* acc_o = send + my_oi * chunk_floats;        // the running merge lives in this CTA's own group
         float* acc_m = acc_o + R * D;
         float* acc_l = acc_m + R;
-        const int tid = threadIdx.x;                       // compute warps are threads 0 .. 127
+        const int tid = threadIdx.x;                       // compute warps (both sets) are threads 0 .. 255
         const int n_vec = (R * D) >> 2;                    // float4 elements of a group
         constexpr int kB = 4;
         // sources in the order they are expected: the other owners (small pieces), then the rest
@@ -383,12 +516,12 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             // batches of kB independent elements per thread: all loads first, then the math, then the
             // stores (a rolled element-by-element loop is a chain of shared-memory latencies)
 #pragma unroll 1
-            for (int base = tid; base < n_vec; base += kB * kComputeWarps * 32) {
+            for (int base = tid; base < n_vec; base += kB * kSets * kComputeWarps * 32) {
               float4 a[kB], b_[kB];
               float ma[kB], ms[kB];
 #pragma unroll
               for (int k = 0; k < kB; ++k) {
-                const int idx = min(base + k * kComputeWarps * 32, n_vec - 1);
+                const int idx = min(base + k * kSets * kComputeWarps * 32, n_vec - 1);
                 const int rr = idx / (D / 4);
                 ma[k] = acc_m[rr]; ms[k] = src_m[rr];
                 a[k] = reinterpret_cast<const float4*>(acc_o)[idx];
@@ -404,11 +537,11 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
               }
 #pragma unroll
               for (int k = 0; k < kB; ++k) {
-                const int idx = base + k * kComputeWarps * 32;
+                const int idx = base + k * kSets * kComputeWarps * 32;
                 if (idx < n_vec) reinterpret_cast<float4*>(acc_o)[idx] = a[k];
               }
             }
-            asm volatile("bar.sync 1, %0;" ::"n"(kComputeWarps * 32) : "memory");   // every row's old maximum has been used
+            asm volatile("bar.sync 1, %0;" ::"n"(kSets * kComputeWarps * 32) : "memory");   // every row's old maximum has been used
             if (tid < R) {
               const float ma = acc_m[tid], ms = src_m[tid];
               const float mn = fmaxf(ma, ms);
@@ -416,23 +549,24 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
               acc_l[tid] = acc_l[tid] * fast_exp2(ma - ref) + src_l[tid] * fast_exp2(ms - ref);
               acc_m[tid] = mn;
             }
-            asm volatile("bar.sync 1, %0;" ::"n"(kComputeWarps * 32) : "memory");
+            asm volatile("bar.sync 1, %0;" ::"n"(kSets * kComputeWarps * 32) : "memory");
           }
         }
+        if (threadIdx.x == 0) stamp(4);
         // normalise and write the R rows (element idx sits at swizzled column cs of row rr)
 #pragma unroll 1
-        for (int base = tid; base < n_vec; base += kB * kComputeWarps * 32) {
+        for (int base = tid; base < n_vec; base += kB * kSets * kComputeWarps * 32) {
           float4 a[kB];
           float lsum[kB];
 #pragma unroll
           for (int k = 0; k < kB; ++k) {
-            const int idx = min(base + k * kComputeWarps * 32, n_vec - 1);
+            const int idx = min(base + k * kSets * kComputeWarps * 32, n_vec - 1);
             lsum[k] = acc_l[idx / (D / 4)];
             a[k] = reinterpret_cast<const float4*>(acc_o)[idx];
           }
 #pragma unroll
           for (int k = 0; k < kB; ++k) {
-            const int idx = base + k * kComputeWarps * 32;
+            const int idx = base + k * kSets * kComputeWarps * 32;
             const int rr = idx / (D / 4);
             const int c = ((idx - rr * (D / 4)) * 4) ^ ((rr & 7) << 3);
             const int row = item.row0 + my_oi * R + rr;
@@ -475,9 +609,16 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         if (ok_hi) { slot[BM * D + r_hi] = m_hi; slot[BM * D + BM + r_hi] = l_hi; }
       }
     }
-    if (threadIdx.x == 0 && w == item_begin) stamp(6);
   }
   if (threadIdx.x == 0) stamp(7);
+  }  // compute warps
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == kMmaWarp) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(uint32_t(L::kTmemCols)) : "memory");
+  }
 }
 
 size_t attn_mma_smem_bytes(int head_dim) {
