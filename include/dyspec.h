@@ -128,9 +128,11 @@ int dyspec_schedule_dry_run(int n_q_heads, int n_kv_heads, int head_dim, int n_r
 
 /* Testing knobs, read when a plan is created: force the regime (-1 = automatic), the number of
  * CTAs the scheduler balances over (0 = automatic; a negative value -c instead sets the scheduler's
- * per-item cost to c key tiles), and how split-KV partials are merged: 0 = by
- * the separate combine kernel, 2 (default) = inside a thread-block cluster through distributed shared
- * memory when the plan is uniform enough, else as 0. */
+ * per-item cost to c key tiles), and combine_mode = m + 16 k.  m says how split-KV partials are merged:
+ * 0 = by the separate combine kernel, 2 (default) = inside a thread-block cluster through distributed
+ * shared memory when the plan is uniform enough, else as 0.  k says whether the scheduler may deal whole
+ * (unsplit) groups to the CTAs instead of cutting them to equal budgets: 0 (default) = when its cost
+ * model says that is quicker (and force_ctas is 0), 1 = never, 2 = always. */
 int dyspec_set_tuning(int force_regime, int force_ctas, int combine_mode);
 
 /* Developer aid: event trace of the attention kernels.  trace_buffer is a dev uint64 array of

@@ -1,5 +1,6 @@
 // C ABI of the tree-verify attention library: argument checks, the host-side ragged scheduler
 // (plan), TMA tensor-map encoding and kernel launches.  See include/dyspec.h for the contract.
+#include <algorithm>
 #include <cmath>
 #include <cstdio>
 #include <cstdlib>
@@ -57,6 +58,7 @@ int g_force_regime = -1;
 int g_force_ctas = 0;
 int g_item_cost = 0;       // scheduler experiment knob (0 = default)
 int g_combine_mode = 2;   // 0 separate combine kernel, 2 cluster merge when the plan allows, else as 0
+int g_whole_groups = 0;   // 0: the scheduler's cost model chooses; 1: never deal whole groups; 2: always
 unsigned long long* g_trace = nullptr;   // device buffer for the optional kernel event trace
 int g_trace_capacity = 0;
 
@@ -297,6 +299,63 @@ void schedule(dyspec_plan& pl) {
   if (pl.n_ctas <= max_ctas) break;
   target += std::max<int64_t>(1, target / 64);
   }
+  // The alternative without any split: whole groups dealt to the CTAs, largest first, each to the CTA
+  // with the least work so far.  No partials and no combine launch, but the longest group bounds the
+  // makespan.  Costs in key tiles: every item item_cost; an item that writes a partial one more tile
+  // (fp32 rows instead of bf16); the combine launch behind the main kernel three (regime 1: 128-key
+  // tiles of ~2 us) or four (regime 0) -- measured on the Llama2-70B shape, where the budgeted plan
+  // (136 CTAs, 32 split groups) took 53.5 us and whole groups on 128 CTAs 48.1 us.
+  if (g_whole_groups != 1 && (g_force_ctas <= 0 || g_whole_groups == 2)) {
+    const int partial_cost = 1, combine_cost = pl.regime == 0 ? 4 : 3;
+    int64_t cost_split = 0;
+    for (int c = 0; c < pl.n_ctas; ++c) {
+      int64_t load = 0;
+      for (int k = pl.cta_begin[size_t(c)]; k < pl.cta_begin[size_t(c) + 1]; ++k) {
+        const WorkItem& it = pl.items[size_t(k)];
+        load += (it.tile_end - it.tile_begin) + item_cost + (it.slot >= 0 ? partial_cost : 0);
+      }
+      cost_split = std::max(cost_split, load);
+    }
+    if (!pl.split_groups.empty()) cost_split += combine_cost;
+    const int n_bins = int(std::min<int64_t>(int64_t(groups.size()), max_ctas));
+    std::vector<size_t> order(groups.size());
+    for (size_t i = 0; i < order.size(); ++i) order[i] = i;
+    std::stable_sort(order.begin(), order.end(), [&](size_t a, size_t b) { return groups[a].tiles > groups[b].tiles; });
+    std::vector<int64_t> load(size_t(n_bins), 0);
+    std::vector<std::vector<size_t>> bins{size_t(n_bins)};
+    for (size_t gi : order) {
+      size_t best = 0;
+      for (size_t b = 1; b < load.size(); ++b)
+        if (load[b] < load[best]) best = b;
+      load[best] += groups[gi].tiles + item_cost;
+      bins[best].push_back(gi);
+    }
+    const int64_t cost_whole = *std::max_element(load.begin(), load.end());
+    if (!pl.split_groups.empty() && (cost_whole <= cost_split || g_whole_groups == 2)) {
+      pl.items.clear();
+      pl.cta_begin.clear();
+      pl.split_groups.clear();
+      pl.n_slots = 0;
+      pl.max_splits = 1;
+      pl.cta_begin.push_back(0);
+      for (const std::vector<size_t>& bin : bins) {
+        for (size_t gi : bin) {
+          const Group& gr = groups[gi];
+          const ReqInfo& rq = pl.reqs[size_t(gr.req)];
+          WorkItem it{};
+          it.kv_row0 = rq.kv_row0; it.prefix_len = rq.prefix_len; it.n_nodes = rq.n_nodes; it.node0 = rq.node0;
+          it.slot0 = -1; it.n_in_cta = 0;
+          it.req = gr.req; it.kv_head = gr.kvh; it.row0 = gr.row0;
+          it.tile_begin = 0; it.tile_end = gr.tiles;
+          it.slot = -1; it.group = int(gi); it.n_splits = 1;
+          pl.items.push_back(it);
+        }
+        pl.cta_begin.push_back(int32_t(pl.items.size()));
+      }
+      pl.n_ctas = n_bins;
+    }
+  }
+
   // device layout: fixed stride per CTA, count in the CTA's first item
   pl.items_stride = 1;
   for (int c = 0; c < pl.n_ctas; ++c) pl.items_stride = std::max(pl.items_stride, pl.cta_begin[size_t(c) + 1] - pl.cta_begin[size_t(c)]);
@@ -360,7 +419,11 @@ int dyspec_words_per_row(int max_nodes) {
 }
 
 int dyspec_set_tuning(int force_regime, int force_ctas, int combine_mode) {
-  if (force_regime < -1 || force_regime > 1 || (combine_mode != 0 && combine_mode != 2)) return DYSPEC_ERR_INVALID_ARG;
+  if (combine_mode < 0) return DYSPEC_ERR_INVALID_ARG;
+  const int whole = combine_mode >> 4;
+  combine_mode &= 15;
+  if (force_regime < -1 || force_regime > 1 || (combine_mode != 0 && combine_mode != 2) || whole > 2) return DYSPEC_ERR_INVALID_ARG;
+  g_whole_groups = whole;
   g_force_regime = force_regime;
   g_force_ctas = force_ctas >= 0 ? force_ctas : 0;
   g_item_cost = force_ctas < 0 ? -force_ctas : 0;   // negative values select the per-item cost instead (experiments)

@@ -109,3 +109,32 @@ def test_regime_is_chosen_from_packed_rows(B):
     assert check_schedule(B, 64, 8, 128, [1024], [8])[0]["regime"] == 0
     assert check_schedule(B, 64, 8, 128, [1024], [9])[0]["regime"] == 1
     assert check_schedule(B, 32, 32, 128, [4096], [256])[0]["regime"] == 1
+
+
+def test_whole_group_plan_is_chosen_when_cheaper(B):
+    """Many groups of similar length (Llama2-70B shape, 512-node tree: 128 groups of 17 - 20 key tiles):
+    dealing whole groups needs no partials and no combine launch, and the cost model prefers it; a few
+    long groups (Llama2-7B, 4096-token prefix: 32 groups of 34 tiles) must still be split."""
+    w = wl.make_config(4)
+    args = (w.n_q_heads, w.n_kv_heads, w.head_dim, w.prefix_len.tolist(), w.n_nodes.tolist())
+    info, loads = check_schedule(B, *args)
+    assert info["split_groups"] == 0 and info["ctas"] == 128 and max(loads) == 20
+    info_never, _ = check_schedule(B, *args, fuse=2 + 16)          # whole groups switched off
+    assert info_never["split_groups"] > 0
+    w3 = wl.make_config(3)
+    args3 = (w3.n_q_heads, w3.n_kv_heads, w3.head_dim, w3.prefix_len.tolist(), w3.n_nodes.tolist())
+    info3, _ = check_schedule(B, *args3)
+    assert info3["split_groups"] == 32
+    info3_always, loads3 = check_schedule(B, *args3, fuse=2 + 32)   # forced: 32 CTAs with 34 tiles each
+    assert info3_always["split_groups"] == 0 and info3_always["ctas"] == 32 and set(loads3) == {34}
+
+
+def test_whole_group_plan_balances_a_ragged_batch(B):
+    """Ragged batch: groups sorted by length and dealt to the least loaded CTA; no CTA ends up with more
+    than the mean plus the longest group."""
+    w = wl.make_config(5)
+    info, loads = check_schedule(B, w.n_q_heads, w.n_kv_heads, w.head_dim, w.prefix_len.tolist(), w.n_nodes.tolist(),
+                                 fuse=2 + 32)
+    assert info["split_groups"] == 0 and info["ctas"] == 148
+    longest = max(-(-int(L) // 128) + -(-int(n) // 128) for L, n in zip(w.prefix_len, w.n_nodes))
+    assert max(loads) <= sum(loads) / len(loads) + longest
