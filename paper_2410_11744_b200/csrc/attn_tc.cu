@@ -4,14 +4,19 @@
 // contractions.  One CTA per SM, 12 warps:
 //   warp 0        TMA producer: Q tile (2 x 128 packed rows) once per work item, then K and V tiles
 //                 (128 keys) into a 5-slot shared-memory ring, 128-byte swizzled, mbarrier-guarded.
-//   warp 1        tcgen05.mma issuer (one lane).  S = Q K^T: both operands from shared memory,
-//                 accumulator in TMEM.  O += P V: P from TMEM (bf16, written by the softmax warps
-//                 over the S columns), V from shared memory as an MN-major operand.
-//   warp 2        allocates / frees the 512 TMEM columns: S_A, S_B, O_A, O_B (128 fp32 columns each).
-//   warps 4-7     softmax of query half A: one thread per row, S read with tcgen05.ld, fp32 online
-//                 softmax in the exp2 domain, ancestor bitmask on tree tiles, P written back with
-//                 tcgen05.st.  The running output lives in TMEM and is rescaled only when the row
-//                 maximum grows by more than 2^8 (the final normalisation uses the same reference).
+//   warps 1, 3    tcgen05.mma issuers, one per query half (one lane each).  S = Q K^T: both operands
+//                 from shared memory, accumulator in TMEM.  O += P V: P from TMEM (bf16, written by the
+//                 softmax warps), V from shared memory as an MN-major operand.  Issuing a tcgen05.mma
+//                 holds the thread until the pipe has taken it, so with one issuer the pipe idles
+//                 during every barrier probe and commit; with two, one warp's hand-offs overlap the
+//                 other's batch.
+//   warp 2        allocates / frees the 512 TMEM columns: one S buffer (128 fp32 columns) that the halves
+//                 use in turn, P_A and P_B (64 columns of bf16 pairs each), O_A, O_B (128 each).
+//   warps 4-7     softmax of query half A: one thread per row, S read with tcgen05.ld (after which the
+//                 buffer is handed to the other half), fp32 online softmax in the exp2 domain, ancestor
+//                 bitmask on tree tiles, P written with tcgen05.st.  The running output lives in TMEM and
+//                 is rescaled only when the row maximum grows by more than 2^8 (the final normalisation
+//                 uses the same reference).
 //   warps 8-11    the same for query half B.  The two halves alternate on the tensor pipe, so one
 //                 half's softmax overlaps the other half's MMAs, and each K/V tile is loaded once
 //                 for 256 query rows.
@@ -50,7 +55,7 @@ struct TcLayout {
 // barrier indices (8 bytes each)
 enum { B_QFULL = 0, B_QFREE = 1, B_SLOT_FULL = 2, B_SLOT_EMPTY = B_SLOT_FULL + kSlots,
        B_SREADY = B_SLOT_EMPTY + kSlots, B_PREADY = B_SREADY + 2, B_ODONE = B_PREADY + 2, B_OFREE = B_ODONE + 2,
-       B_COUNT = B_OFREE + 2 };
+       B_PVDONE = B_OFREE + 2, B_COUNT = B_PVDONE + 2 };
 
 // Hardware named barriers for thread-to-thread hand-offs inside the CTA (P ready: 128 softmax threads
 // -> the MMA-issuing warp): an order of magnitude quicker to notice than an mbarrier in shared memory
@@ -62,7 +67,8 @@ enum { B_QFULL = 0, B_QFREE = 1, B_SLOT_FULL = 2, B_SLOT_EMPTY = B_SLOT_FULL + k
 __device__ __forceinline__ void named_arrive(int id, int count) { asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(count) : "memory"); }
 __device__ __forceinline__ void named_sync(int id, int count) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory"); }
 constexpr int kBarPReady = 1;               // named barriers 1, 2: P of half A, B is in TMEM
-constexpr int kPReadyCount = BMH + 32;      // the half's softmax threads + the issuing warp
+constexpr int kBarSFree = 3;                // named barrier 3: the S buffer has been read out
+constexpr int kPReadyCount = BMH + 32;      // a half's softmax threads + the issuing warp
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -232,24 +238,31 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   auto bar = [&](int i) { return s_bar + 8u * uint32_t(i); };
   volatile uint32_t* tmem_holder = reinterpret_cast<volatile uint32_t*>(smem + L::kBarOffset + 8 * B_COUNT);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::kBarOffset + 8 * B_COUNT + 8);
+  // "S read out" counters, one per half: its four softmax warps each add 1 after loading a score tile.
+  // A monotonic counter, not a phase barrier: the waiting issuer may not have looked at this half's
+  // counter for many uses (items with one half in between), which a parity wait would misread.
+  const uint32_t s_free_ctr = s_bar + 8u * uint32_t(B_COUNT) + 16u;
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
     mbar_init(bar(B_QFULL), 1);
-    mbar_init(bar(B_QFREE), 1);
+    mbar_init(bar(B_QFREE), 2);
     for (int s = 0; s < kSlots; ++s) {
       mbar_init(bar(B_SLOT_FULL + s), 1);
-      mbar_init(bar(B_SLOT_EMPTY + s), 1);
+      mbar_init(bar(B_SLOT_EMPTY + s), 2);
     }
     for (int h = 0; h < 2; ++h) {
       mbar_init(bar(B_SREADY + h), 1);
       mbar_init(bar(B_PREADY + h), BMH);
       mbar_init(bar(B_ODONE + h), 1);
       mbar_init(bar(B_OFREE + h), BMH);
+      mbar_init(bar(B_PVDONE + h), 1);
     }
     *abort_flag = 0;
+    *reinterpret_cast<volatile uint32_t*>(smem + L::kBarOffset + 8 * B_COUNT + 16) = 0u;
+    *reinterpret_cast<volatile uint32_t*>(smem + L::kBarOffset + 8 * B_COUNT + 20) = 0u;
     fence_barrier_init();
   }
   if (warp == 2) {
@@ -328,52 +341,61 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         }
       }
     }
-  } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
-    // The whole warp walks the loop (addresses, slot indices and barrier waits are warp-uniform);
-    // only the elected lane issues the tcgen05 instructions.
+  } else if (warp == 1 || warp == 3) {
+    // ------------------------------------------------------------------ MMA issuers: warp 1 for query half A, warp 3 for B
+    // Issuing a tcgen05.mma holds the thread until the tensor pipe has taken it, so nothing queues up
+    // behind a batch and the pipe idles while its issuer probes barriers, commits or waits.  With one
+    // issuer per half, one warp's hand-offs overlap the other's batch.  The halves share the S buffer
+    // and the K/V slots: S is handed from use to use in the fixed order A(0) B(0) A(1) B(1) ... (an
+    // item with one half: A only) through the "S read out" barrier of the half that used it last, and a
+    // slot or the Q tile is released by two commits (both from warp 1 when the item has no half B).
+    // The whole warp walks the loop; only the elected lane issues the tcgen05 instructions.
     {
+      const int h = warp == 1 ? 0 : 1;
       const bool elected = lane == 0;
       TraceCursor tc_cur = trace_open(p, 0, 3);
-      if (!elected) tc_cur.at = nullptr;
+      if (!elected || h != 0) tc_cur.at = nullptr;
       trace_event(tc_cur, DYSPEC_TAG(0, 9, 0));
       constexpr uint32_t idesc_qk = make_idesc(BN, 0);
       constexpr uint32_t idesc_pv = make_idesc(D, 1);
       constexpr uint32_t kHiK = desc_hi(1024);            // K-major operands (Q, K): 8-row groups 1024 B apart
       constexpr uint32_t kHiV = desc_hi(1024);            // MN-major operand (V): 8-key groups 1024 B apart
-      const uint32_t q_lo0 = desc_lo(s_q, 16);
+      const uint32_t q_lo0 = desc_lo(s_q, 16) + uint32_t(h) * (L::kTileBytes >> 4);
       const uint32_t ring_k_lo0 = desc_lo(s_ring, 16);
       const uint32_t ring_v_lo0 = desc_lo(s_ring, L::kPanelBytes);   // leading offset = next 64-column panel
-      auto issue_qk = [=](int h, uint32_t slot) {
-        const uint32_t a_lo = q_lo0 + uint32_t(h) * (L::kTileBytes >> 4);
+      auto issue_qk = [=](uint32_t slot) {
         const uint32_t b_lo = ring_k_lo0 + slot * (L::kTileBytes >> 4);
-        const uint32_t d_tmem = tmem_base + uint32_t(h) * 128u;
 #pragma unroll
         for (int ks = 0; ks < D / 16; ++ks) {
           const uint32_t off = (uint32_t(ks >> 2) * L::kPanelBytes + uint32_t(ks & 3) * 32u) >> 4;
-          if (elected) umma_ss_lohi(d_tmem, a_lo + off, kHiK, b_lo + off, kHiK, idesc_qk, ks > 0 ? 1u : 0u);
+          if (elected) umma_ss_lohi(tmem_base, q_lo0 + off, kHiK, b_lo + off, kHiK, idesc_qk, ks > 0 ? 1u : 0u);
         }
         if (elected) tc_commit(s_bar + 8u * uint32_t(B_SREADY + h));
       };
-      auto issue_pv = [=](int h, uint32_t slot, bool accumulate) {
+      auto issue_pv = [=](uint32_t slot, bool accumulate) {
         const uint32_t b_lo = ring_v_lo0 + slot * (L::kTileBytes >> 4);
         const uint32_t d_tmem = tmem_base + 256u + uint32_t(h) * 128u;
-        const uint32_t a_tmem = tmem_base + uint32_t(h) * 128u;
+        const uint32_t a_tmem = tmem_base + 128u + uint32_t(h) * 64u;
 #pragma unroll
         for (int kk = 0; kk < BN / 16; ++kk)
           if (elected) umma_ts_lohi(d_tmem, a_tmem + uint32_t(kk) * 8u, b_lo + uint32_t(kk) * (2048u >> 4), kHiV, idesc_pv,
                        (accumulate || kk > 0) ? 1u : 0u);
       };
       uint32_t sc = 0, qit = 0;
-      uint32_t n_p0 = 0, n_p1 = 0;          // P-ready phases consumed per half
-      uint32_t n_it0 = 0, n_it1 = 0;        // items seen per half (O-free phase)
+      uint32_t n_use[2] = {0, 0};           // S uses (QK^T products) issued so far by half A / B, both counted by both warps
+      int last_user = -1;                   // which half used the S buffer last (-1: nobody yet)
+      uint32_t n_it = 0;                    // items this half took part in (O-free phase)
+      // Before S use: the half that used the buffer last must have read its scores out.
+      auto wait_s_free = [&]() {
+        if (last_user >= 0) {
+          counter_wait(s_free_ctr + 4u * uint32_t(last_user), 4u * n_use[last_user], abort_flag, p.status);
+          tc_fence_after();
+        }
+      };
       for (int w = item_begin; w < item_end; ++w, ++qit) {
         const WorkItem item = my_items[w];
         const WorkItem& rq = item;
         const bool two = rq.n_nodes * g - item.row0 > BMH;        // both query halves live
-        // Number of tiles of the item.  With per-node tile sets it depends on the mask kernel's
-        // output; it is settled two tiles before the prefix part ends (until then "more tiles
-        // follow" is all this loop needs to know), so the prefix still overlaps that kernel.
         const int n_prefix_tiles = (rq.prefix_len + BN - 1) / BN;
         TileWalk wk = walk_dense(item, n_prefix_tiles);
         bool exact = p.node_tiles == nullptr || wk.need == 0u;
@@ -387,16 +409,32 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           }
         };
         settle(-1);
-        mbar_wait(bar(B_QFULL), qit & 1, abort_flag, p.status);
+        // S uses of this item, in order: tile 0: A (B), tile 1: A (B), ...  Each warp issues its own and
+        // only counts the other's.
+        auto release = [&](int b) {                               // one of the two commits that free a slot / the Q tile
+          if (elected) tc_commit(bar(b));
+          if (!two && elected) tc_commit(bar(b));                 // no half B in this item: warp 1 gives both
+        };
+        const bool mine = h == 0 || two;
+        if (mine) mbar_wait(bar(B_QFULL), qit & 1, abort_flag, p.status);
         {
           const uint32_t kslot = sc % kSlots, kph = (sc / kSlots) & 1;
           ++sc;
-          mbar_wait(bar(B_SLOT_FULL + kslot), kph, abort_flag, p.status);
-          tc_fence_after();
-          issue_qk(0, kslot);
-          if (two) issue_qk(1, kslot);
-          if (elected) tc_commit(bar(B_SLOT_EMPTY + kslot));
-          if (T == 1) if (elected) tc_commit(bar(B_QFREE));            // Q is reusable once the item's last QK^T has run
+          if (mine) {
+            mbar_wait(bar(B_SLOT_FULL + kslot), kph, abort_flag, p.status);
+            tc_fence_after();
+          }
+          // use A(0)
+          if (h == 0) { wait_s_free(); issue_qk(kslot); }
+          ++n_use[0]; last_user = 0;
+          if (two) {                                              // use B(0)
+            if (h == 1) { wait_s_free(); issue_qk(kslot); }
+            ++n_use[1]; last_user = 1;
+          }
+          if (mine) {
+            release(B_SLOT_EMPTY + kslot);
+            if (T == 1) release(B_QFREE);                         // Q is reusable once the item's last QK^T has run
+          }
         }
         for (int j = 0;; ++j) {
           settle(j);
@@ -406,49 +444,39 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           const bool more = j + 1 < T;
           const uint32_t kslot = sc % kSlots, kph = (sc / kSlots) & 1;
           if (more) ++sc;
-          // An mbarrier probe takes ~180 cycles to answer even when the phase completed long ago.  The
-          // two slot barriers this tile starts with (V slot, next K slot) are probed in one go, so
-          // their round trips overlap; only what is really not there yet is then waited for.
-          {
+          if (mine) {
             const uint32_t got = __reduce_and_sync(0xffffffffu,
                 mbar_test_wait3(bar(B_SLOT_FULL + vslot), vph, bar(B_SLOT_FULL + (more ? kslot : vslot)), more ? kph : vph,
                                 bar(B_SLOT_FULL + vslot), vph));
             if (!(got & 1u)) mbar_wait(bar(B_SLOT_FULL + vslot), vph, abort_flag, p.status);
             if (more && !(got & 2u)) mbar_wait(bar(B_SLOT_FULL + kslot), kph, abort_flag, p.status);
-            if (j == 0) {
-              mbar_wait(bar(B_OFREE + 0), (n_it0 & 1) ^ 1, abort_flag, p.status);
-              if (two) mbar_wait(bar(B_OFREE + 1), (n_it1 & 1) ^ 1, abort_flag, p.status);
+            if (j == 0) mbar_wait(bar(B_OFREE + h), (n_it & 1) ^ 1, abort_flag, p.status);
+          }
+          // S = Q K(j+1)^T as soon as the S buffer has been read out: issued BEFORE this tile's PV, it does
+          // not depend on P, so the tensor work is off the softmax threads' chain.
+          if (more) {
+            if (h == 0) { wait_s_free(); issue_qk(kslot); }
+            ++n_use[0]; last_user = 0;
+            if (two) {
+              if (h == 1) { wait_s_free(); issue_qk(kslot); }
+              ++n_use[1]; last_user = 1;
             }
-            // ---- half A: O_A += P_A V, then S_A = Q_A K(j+1)^T
-            named_sync(kBarPReady + 0, kPReadyCount);
           }
-          ++n_p0;
-          tc_fence_after();
-          trace_event(tc_cur, DYSPEC_TAG(0, 1, j));
-          issue_pv(0, vslot, j > 0);
-          if (!more) if (elected) tc_commit(bar(B_ODONE + 0));
-          trace_event(tc_cur, DYSPEC_TAG(0, 5, j));
-          if (more) issue_qk(0, kslot);
-          trace_event(tc_cur, DYSPEC_TAG(0, 2, j));
-          // ---- half B
-          if (two) {
-            named_sync(kBarPReady + 1, kPReadyCount);
-            ++n_p1;
+          if (mine) {
+            trace_event(tc_cur, DYSPEC_TAG(0, 2, j));
+            named_sync(kBarPReady + h, kPReadyCount);
             tc_fence_after();
-            trace_event(tc_cur, DYSPEC_TAG(0, 3, j));
-            issue_pv(1, vslot, j > 0);
-            if (!more) if (elected) tc_commit(bar(B_ODONE + 1));
-            trace_event(tc_cur, DYSPEC_TAG(0, 6, j));
-            if (more) issue_qk(1, kslot);
-            trace_event(tc_cur, DYSPEC_TAG(0, 4, j));
+            trace_event(tc_cur, DYSPEC_TAG(0, 1, j));
+            issue_pv(vslot, j > 0);
+            if (elected) tc_commit(bar((more ? B_PVDONE : B_ODONE) + h));
+            trace_event(tc_cur, DYSPEC_TAG(0, 5, j));
+            release(B_SLOT_EMPTY + vslot);
+            if (more) release(B_SLOT_EMPTY + kslot);
+            if (j + 2 == T) release(B_QFREE);
+            trace_event(tc_cur, DYSPEC_TAG(0, 7, j));
           }
-          if (elected) tc_commit(bar(B_SLOT_EMPTY + vslot));
-          if (more) if (elected) tc_commit(bar(B_SLOT_EMPTY + kslot));
-          if (j + 2 == T) if (elected) tc_commit(bar(B_QFREE));
-          trace_event(tc_cur, DYSPEC_TAG(0, 7, j));
         }
-        ++n_it0;
-        if (two) ++n_it1;
+        if (mine) ++n_it;
       }
     }
   }
@@ -461,10 +489,12 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     const int h = (warp - 4) >> 2;                       // query half
     const int r = ((warp & 3) << 5) + lane;              // row of the half == TMEM lane
     const uint32_t lane_sel = uint32_t((warp & 3) << 5) << 16;
-    const uint32_t t_s = tmem_base + uint32_t(h) * 128u + lane_sel;
+    const uint32_t t_s = tmem_base + lane_sel;                                  // scores (one buffer, the halves take turns)
+    const uint32_t t_p = tmem_base + 128u + uint32_t(h) * 64u + lane_sel;       // this half's probabilities (bf16 pairs)
     const uint32_t t_o = tmem_base + 256u + uint32_t(h) * 128u + lane_sel;
     TraceCursor tc_cur = trace_open(p, 1 + h, 3);
     uint32_t n_s = 0, n_o = 0;                           // S-ready / O-done phases seen by this half
+    uint32_t n_pv = 0;                                   // PV-done phases seen by this half
     uint32_t sc = 0;                                     // ring position (to find V slots)
 
     for (int w = item_begin; w < item_end; ++w) {
@@ -522,6 +552,9 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
 #pragma unroll
         for (int c = 0; c < 4; ++c) tmem_ld32(t_s + uint32_t(c) * 32u, sv + 32 * c);
         tmem_wait_ld();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) red_release_shared_add(s_free_ctr + 4u * uint32_t(h), 1u);   // this warp's rows are in registers: 4 of these and S may be overwritten
         if (r == 0) trace_event(tc_cur, DYSPEC_TAG(1 + h, 2, j));
         if (!all_visible) {
 #pragma unroll
@@ -539,11 +572,16 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2e;   // scale > 0
         const float m_new = fmaxf(m_used, mx);
         if (r == 0) trace_event(tc_cur, DYSPEC_TAG(1 + h, 3, j));
+        if (j > 0) {
+          // P(j-1) is still being read, and O still being written, until PV(j-1) has completed
+          mbar_wait(bar(B_PVDONE + h), n_pv & 1, abort_flag, p.status);
+          ++n_pv;
+          tc_fence_after();
+        }
         if (j == 0) {
           m_used = m_new;
         } else if (__any_sync(0xffffffffu, m_new > m_used + kRescaleThreshold)) {
-          // rescale the running output of this warp's 32 rows: O *= 2^(m_used - m_new).  The tensor pipe
-          // completes MMAs in issue order, so S(j) being ready already implies that PV(j-1) has finished.
+          // rescale the running output of this warp's 32 rows: O *= 2^(m_used - m_new)
           const float f = fast_exp2(m_used - (m_new == -INFINITY ? 0.f : m_new));
 #pragma unroll 1
           for (int c = 0; c < D / 32; ++c) {
@@ -575,7 +613,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             sum2[i & 1] = add_f32x2(sum2[i & 1], pack_f32x2(p0, p1));
             pk[i] = pack_bf16x2(p0, p1);
           }
-          tmem_st16(t_s + uint32_t(c) * 16u, pk);
+          tmem_st16(t_p + uint32_t(c) * 16u, pk);
         }
         {
           float a0, a1, b0, b1;
