@@ -138,8 +138,10 @@ int dyspec_set_tuning(int force_regime, int force_ctas, int combine_mode);
 /* Developer aid: event trace of the attention kernels.  trace_buffer is a dev uint64 array of
  * capacity_entries entries that the caller zeroes; while set, CTA 0 of every tensor-core attention
  * launch writes (tag << 44 | SM clock) entries into three equal regions (MMA issuer, softmax half A,
- * softmax half B; tags are listed in csrc/attn_tc.cu; zero entries are unused).  Pass (NULL, 0) to
- * switch it off (the default). */
+ * softmax half B; tags are listed in csrc/attn_tc.cu; zero entries are unused).  When capacity_entries
+ * > 4096 the last 2048 entries are not part of those regions: there each of the first 256 CTAs of an
+ * attention launch (either kernel) leaves 8 wall-clock stamps (globaltimer, ns) of its phases, listed
+ * where the kernels take them.  Pass (NULL, 0) to switch it off (the default). */
 int dyspec_set_trace(void* trace_buffer, int capacity_entries);
 
 /*

@@ -493,6 +493,13 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     const uint32_t t_p = tmem_base + 128u + uint32_t(h) * 64u + lane_sel;       // this half's probabilities (bf16 pairs)
     const uint32_t t_o = tmem_base + 256u + uint32_t(h) * 128u + lane_sel;
     TraceCursor tc_cur = trace_open(p, 1 + h, 3);
+    // wall-clock stamps of every CTA (last 2048 entries of the trace buffer, 8 per CTA, first 256 CTAs), by
+    // row 0 of half A: 0 start, 1 first scores seen, 2 .. 6 end of the CTA's items 0 .. 4, 7 exit
+    auto stamp = [&](int k) {
+      if (p.trace != nullptr && h == 0 && r == 0 && blockIdx.x < 256 && p.trace_capacity > 4096)
+        p.trace[p.trace_capacity - 2048 + 8 * blockIdx.x + k] = global_timer_ns();
+    };
+    stamp(0);
     uint32_t n_s = 0, n_o = 0;                           // S-ready / O-done phases seen by this half
     uint32_t n_pv = 0;                                   // PV-done phases seen by this half
     uint32_t sc = 0;                                     // ring position (to find V slots)
@@ -543,6 +550,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         }
 
         mbar_wait(bar(B_SREADY + h), n_s & 1, abort_flag, p.status);
+        if (n_s == 0) stamp(1);
         ++n_s;
         tc_fence_after();
         if (r == 0) trace_event(tc_cur, DYSPEC_TAG(1 + h, 1, j));
@@ -692,7 +700,9 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       tc_fence_before();
       mbar_arrive(bar(B_OFREE + h));
       if (r == 0) trace_event(tc_cur, DYSPEC_TAG(1 + h, 7, 0));
+      if (w - item_begin < 5) stamp(2 + (w - item_begin));
     }
+    stamp(7);
   }
 
   tc_fence_before();
