@@ -111,7 +111,7 @@ size_t dyspec_plan_workspace_bytes(const dyspec_plan_t* plan);
 
 /* Scheduler introspection (for tests and benchmarks): field 0 = work items, 1 = CTAs launched,
  * 2 = query-tile groups, 3 = groups that are split, 4 = max splits of a group, 5 = kernel regime
- * (0 = warp-level mma tiles, 1 = tcgen05 tiles), 6 = total key tiles, 7 = query rows per tile,
+ * (0 = 64-row tiles for small trees, 1 = 2 x 128-row tcgen05 tiles), 6 = total key tiles, 7 = query rows per tile,
  * 8 = thread-block cluster size (1 = no clusters). */
 int64_t dyspec_plan_info(const dyspec_plan_t* plan, int field);
 
