@@ -112,7 +112,8 @@ size_t dyspec_plan_workspace_bytes(const dyspec_plan_t* plan);
 /* Scheduler introspection (for tests and benchmarks): field 0 = work items, 1 = CTAs launched,
  * 2 = query-tile groups, 3 = groups that are split, 4 = max splits of a group, 5 = kernel regime
  * (0 = 64-row tiles for small trees, 1 = 2 x 128-row tcgen05 tiles), 6 = total key tiles, 7 = query rows per tile,
- * 8 = thread-block cluster size (1 = no clusters). */
+ * 8 = thread-block cluster size (1 = no clusters), 9 = 1 when the CTAs take whole groups from a shared
+ * queue on the device instead of fixed lists (the item list then shows the nominal assignment). */
 int64_t dyspec_plan_info(const dyspec_plan_t* plan, int field);
 
 /* Host-only view of the scheduler, for tests and tools: validates the arguments and schedules exactly
@@ -140,8 +141,10 @@ int dyspec_set_tuning(int force_regime, int force_ctas, int combine_mode);
  * launch writes (tag << 44 | SM clock) entries into three equal regions (MMA issuer, softmax half A,
  * softmax half B; tags are listed in csrc/attn_tc.cu; zero entries are unused).  When capacity_entries
  * > 4096 the last 2048 entries are not part of those regions: there each of the first 256 CTAs of an
- * attention launch (either kernel) leaves 8 wall-clock stamps (globaltimer, ns) of its phases, listed
- * where the kernels take them.  Pass (NULL, 0) to switch it off (the default). */
+ * attention launch leaves 8 wall-clock stamps (globaltimer, ns) of its phases, listed where the kernels
+ * take them (the tensor-core kernel only in a library built with -DDYSPEC_CTA_STAMPS: its softmax threads
+ * sit at the register limit and the stamps cost it ~2 us per launch).  Pass (NULL, 0) to switch it off
+ * (the default). */
 int dyspec_set_trace(void* trace_buffer, int capacity_entries);
 
 /*
@@ -165,7 +168,10 @@ int dyspec_plan_build_tree_mask(const dyspec_plan_t* plan, const int32_t* parent
  *   out            dev bf16 [sum n_r][H_q][D]            (written)
  *   workspace      dev, >= dyspec_plan_workspace_bytes(plan), 256-byte aligned; its arrival counters
  *                  must be zero before the first call (dyspec_plan_create's caller zeroes it once;
- *                  the kernels leave them zero).  Two calls that overlap on the GPU need two workspaces.
+ *                  the kernels leave them zero).  Two calls that overlap on the GPU need two workspaces
+ *                  AND two plans (a plan owns device words that a launch uses and clears: arrival
+ *                  counters of split groups, the head of the shared work queue); calls that follow
+ *                  each other on one stream may share both.
  *   status         dev int32 [1] or NULL
  */
 int dyspec_tree_attention_ragged(const dyspec_plan_t* plan, const void* q, const void* k_cache, const void* v_cache,

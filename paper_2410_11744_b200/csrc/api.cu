@@ -127,6 +127,9 @@ struct dyspec_plan {
   WorkItem* d_items = nullptr;
   GroupInfo* d_groups = nullptr;
   int32_t* d_counters = nullptr;
+  int32_t* d_queue = nullptr;           // dynamic plans: [0] next item of the shared queue, [1] CTAs that have drained it
+  bool dynamic = false;                 // whole groups taken from a shared queue (longest first) instead of fixed lists
+  std::vector<WorkItem> items_queue;    // dynamic plans: all items in queue order
   size_t workspace_bytes = 0;
 };
 
@@ -166,6 +169,8 @@ void schedule(dyspec_plan& pl) {
   pl.max_splits = 1;
   pl.items_strided.clear();
   pl.items_stride = 1;
+  pl.dynamic = false;
+  pl.items_queue.clear();
   if (groups.empty()) { pl.n_ctas = 0; pl.cta_begin.push_back(0); return; }
 
   // Cluster mode (warp-level regime): when every group can be cut into the same number C of pieces
@@ -353,9 +358,32 @@ void schedule(dyspec_plan& pl) {
         pl.cta_begin.push_back(int32_t(pl.items.size()));
       }
       pl.n_ctas = n_bins;
+      // More groups than CTAs (tensor-core regime): the fixed lists above are only the nominal plan.
+      // On the device the CTAs take the groups from one queue, longest first (CTA c starts with the
+      // c-th longest), so that what the cost model cannot see -- tree tiles skipped by the tile sets,
+      // cache misses of one request's long prefix -- does not leave some CTAs working while others idle.
+      if (pl.regime == 1 && int64_t(groups.size()) > n_bins) {
+        pl.dynamic = true;
+        for (size_t gi : order) {
+          const Group& gr = groups[gi];
+          const ReqInfo& rq = pl.reqs[size_t(gr.req)];
+          WorkItem it{};
+          it.kv_row0 = rq.kv_row0; it.prefix_len = rq.prefix_len; it.n_nodes = rq.n_nodes; it.node0 = rq.node0;
+          it.slot0 = -1; it.n_in_cta = 1;
+          it.req = gr.req; it.kv_head = gr.kvh; it.row0 = gr.row0;
+          it.tile_begin = 0; it.tile_end = gr.tiles;
+          it.slot = -1; it.group = int(gi); it.n_splits = 1;
+          pl.items_queue.push_back(it);
+        }
+      }
     }
   }
 
+  if (pl.dynamic) {                     // device layout: the queue itself
+    pl.items_stride = 1;
+    pl.items_strided = pl.items_queue;
+    return;
+  }
   // device layout: fixed stride per CTA, count in the CTA's first item
   pl.items_stride = 1;
   for (int c = 0; c < pl.n_ctas; ++c) pl.items_stride = std::max(pl.items_stride, pl.cta_begin[size_t(c) + 1] - pl.cta_begin[size_t(c)]);
@@ -372,7 +400,7 @@ int upload(dyspec_plan& pl) {
   const size_t b_reqs = pad(std::max<size_t>(1, pl.reqs.size()) * sizeof(ReqInfo));
   const size_t b_items = pad(std::max<size_t>(1, pl.items_strided.size()) * sizeof(WorkItem));
   const size_t b_groups = pad(std::max<size_t>(1, pl.split_groups.size()) * sizeof(GroupInfo));
-  const size_t b_counters = pad(std::max<size_t>(1, pl.split_groups.size()) * sizeof(int32_t));
+  const size_t b_counters = pad(std::max<size_t>(1, pl.split_groups.size()) * sizeof(int32_t)) + 256;   // + the queue words
   const size_t total = b_reqs + b_items + b_groups + b_counters;
   std::vector<uint8_t> host(total, 0);
   size_t off = 0;
@@ -390,6 +418,7 @@ int upload(dyspec_plan& pl) {
   pl.d_items = reinterpret_cast<WorkItem*>(base + o_items);
   pl.d_groups = reinterpret_cast<GroupInfo*>(base + o_groups);
   pl.d_counters = reinterpret_cast<int32_t*>(base + o_counters);
+  pl.d_queue = reinterpret_cast<int32_t*>(base + o_counters + b_counters - 256);
   return DYSPEC_OK;
 }
 
@@ -709,6 +738,7 @@ int64_t dyspec_plan_info(const dyspec_plan_t* plan, int field) {
     case 6: return plan->total_tiles;
     case 7: return plan->bm;
     case 8: return plan->cluster;
+    case 9: return plan->dynamic ? 1 : 0;
     default: return DYSPEC_ERR_INVALID_ARG;
   }
 }
@@ -807,6 +837,8 @@ static int run_attention(const dyspec_plan_t* plan, const void* q, const void* k
   p.bits = ancestor_bits; p.node_tiles = node_tiles; p.out = static_cast<__nv_bfloat16*>(out);
   p.partial = static_cast<float*>(workspace);
   p.counters = plan->d_counters; p.status = status;
+  p.queue = plan->dynamic ? plan->d_queue : nullptr;
+  p.n_items_total = int32_t(plan->items_strided.size());
   p.n_q_heads = plan->hq; p.n_kv_heads = plan->hkv; p.group_size = plan->g; p.log2_g = plan->log2g;
   p.words_per_row = plan->W; p.slot_floats = bm * (plan->d + 2);
   p.scale_log2e = plan->scale * kLog2e;

@@ -225,7 +225,10 @@ __device__ __forceinline__ TileWalk walk_sparse(const AttnParams& p, const WorkI
 
 }  // namespace
 
-template <int D>
+// kDyn: the CTAs take their items from the shared queue (AttnParams::queue) instead of fixed lists.  A
+// template parameter, not a run-time flag: the softmax threads sit right at the register limit and the
+// fixed-list kernel should compile exactly as it would without the queue.
+template <int D, bool kDyn>
 __global__ void __launch_bounds__(kThreads, 1)
 tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                     const __grid_constant__ CUtensorMap map_v, const AttnParams p) {
@@ -242,6 +245,11 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   // A monotonic counter, not a phase barrier: the waiting issuer may not have looked at this half's
   // counter for many uses (items with one half in between), which a parity wait would misread.
   const uint32_t s_free_ctr = s_bar + 8u * uint32_t(B_COUNT) + 16u;
+  // Shared work queue (see AttnParams::queue): the producer warp takes the CTA's next item and passes
+  // its index on to the other roles through an 8-entry ring (a full barrier per entry; the roles are
+  // never more than two items apart, since there is one Q buffer, so entries need no "empty" barrier).
+  const uint32_t q_full = s_bar + 8u * uint32_t(B_COUNT) + 32u;
+  volatile int32_t* q_idx = reinterpret_cast<volatile int32_t*>(smem + L::kBarOffset + 8 * B_COUNT + 96);
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -260,6 +268,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       mbar_init(bar(B_OFREE + h), BMH);
       mbar_init(bar(B_PVDONE + h), 1);
     }
+    for (int e = 0; e < 8; ++e) mbar_init(q_full + 8u * uint32_t(e), 1);
     *abort_flag = 0;
     *reinterpret_cast<volatile uint32_t*>(smem + L::kBarOffset + 8 * B_COUNT + 16) = 0u;
     *reinterpret_cast<volatile uint32_t*>(smem + L::kBarOffset + 8 * B_COUNT + 20) = 0u;
@@ -275,9 +284,35 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   tc_fence_after();
   const uint32_t tmem_base = *tmem_holder;
 
-  const WorkItem* my_items = p.items + size_t(blockIdx.x) * p.items_stride;
-  const int item_begin = 0;
-  const int item_end = my_items[0].n_in_cta;
+  // Fixed lists: CTA c's items are my_items[0 .. item_end).  Queue: my_items is the whole queue, the
+  // CTA's k-th item is my_items[index], the index -1 ends the CTA's work.
+  const WorkItem* my_items = p.items + (kDyn ? size_t(0) : size_t(blockIdx.x) * p.items_stride);
+  const int item_end = kDyn ? 0x7fffffff : my_items[0].n_in_cta;
+  // for the producer warp (all lanes call it): takes the next item off the queue and publishes it
+  auto take_index = [&](int k) -> int {
+    if (k == 0) return int(blockIdx.x);
+    int idx = 0;
+    if (lane == 0) {
+      // The queue words were cleared by the last CTA of the previous launch that used this plan; that
+      // launch is complete once the kernels this one depends on are.
+      if (k == 1) grid_dependency_wait();
+      const int t = atomicAdd(p.queue, 1) + int(gridDim.x);
+      idx = t < p.n_items_total ? t : -1;
+      q_idx[(k - 1) & 7] = idx;
+      mbar_arrive(q_full + 8u * uint32_t((k - 1) & 7));
+      if (idx < 0 && atomicAdd(p.queue + 1, 1) == int(gridDim.x) - 1) {   // every CTA has drained the queue
+        p.queue[0] = 0;
+        p.queue[1] = 0;
+      }
+    }
+    return __shfl_sync(0xffffffffu, idx, 0);
+  };
+  // for every other role
+  auto next_index = [&](int k) -> int {
+    if (k == 0) return int(blockIdx.x);
+    mbar_wait(q_full + 8u * uint32_t((k - 1) & 7), uint32_t((k - 1) >> 3) & 1u, abort_flag, p.status);
+    return q_idx[(k - 1) & 7];
+  };
   const int g = p.group_size;
 
   // Register budget: the softmax threads hold a whole S row; the control warps need few registers.
@@ -295,8 +330,13 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         prefetch_tensormap(&map_v);
       }
       uint32_t sc = 0, qit = 0;
-      for (int w = item_begin; w < item_end; ++w, ++qit) {
-        const WorkItem item = my_items[w];
+      for (int w = 0; w < item_end; ++w, ++qit) {
+        int item_at = w;
+        if constexpr (kDyn) {
+          item_at = take_index(w);
+          if (item_at < 0) break;
+        }
+        const WorkItem item = my_items[item_at];
         const WorkItem& rq = item;
         const int nh = (rq.n_nodes * g - item.row0 > BMH) ? 2 : 1;
         mbar_wait(bar(B_QFREE), (qit & 1) ^ 1, abort_flag, p.status);
@@ -392,8 +432,13 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           tc_fence_after();
         }
       };
-      for (int w = item_begin; w < item_end; ++w, ++qit) {
-        const WorkItem item = my_items[w];
+      for (int w = 0; w < item_end; ++w, ++qit) {
+        int item_at = w;
+        if constexpr (kDyn) {
+          item_at = next_index(w);
+          if (item_at < 0) break;
+        }
+        const WorkItem item = my_items[item_at];
         const WorkItem& rq = item;
         const bool two = rq.n_nodes * g - item.row0 > BMH;        // both query halves live
         const int n_prefix_tiles = (rq.prefix_len + BN - 1) / BN;
@@ -496,16 +541,25 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     // wall-clock stamps of every CTA (last 2048 entries of the trace buffer, 8 per CTA, first 256 CTAs), by
     // row 0 of half A: 0 start, 1 first scores seen, 2 .. 6 end of the CTA's items 0 .. 4, 7 exit
     auto stamp = [&](int k) {
+#ifdef DYSPEC_CTA_STAMPS
       if (p.trace != nullptr && h == 0 && r == 0 && blockIdx.x < 256 && p.trace_capacity > 4096)
         p.trace[p.trace_capacity - 2048 + 8 * blockIdx.x + k] = global_timer_ns();
+#else
+      (void)k;
+#endif
     };
     stamp(0);
     uint32_t n_s = 0, n_o = 0;                           // S-ready / O-done phases seen by this half
     uint32_t n_pv = 0;                                   // PV-done phases seen by this half
     uint32_t sc = 0;                                     // ring position (to find V slots)
 
-    for (int w = item_begin; w < item_end; ++w) {
-      const WorkItem item = my_items[w];
+    for (int w = 0; w < item_end; ++w) {
+      int item_at = w;
+      if constexpr (kDyn) {
+        item_at = next_index(w);
+        if (item_at < 0) break;
+      }
+      const WorkItem item = my_items[item_at];
       const WorkItem& rq = item;
       const int n_rows = rq.n_nodes * g;
       const int nh = (n_rows - item.row0 > BMH) ? 2 : 1;
@@ -700,7 +754,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       tc_fence_before();
       mbar_arrive(bar(B_OFREE + h));
       if (r == 0) trace_event(tc_cur, DYSPEC_TAG(1 + h, 7, 0));
-      if (w - item_begin < 5) stamp(2 + (w - item_begin));
+      if (w < 5) stamp(2 + w);
     }
     stamp(7);
   }
@@ -713,9 +767,23 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   }
 }
 
+namespace {
+template <int D, bool kDyn>
+cudaError_t launch_one(cudaLaunchConfig_t& cfg, size_t smem, const CUtensorMap& mq, const CUtensorMap& mk,
+                       const CUtensorMap& mv, const AttnParams& p) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(tree_attn_tc_kernel<D, kDyn>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  cfg.dynamicSmemBytes = smem;
+  return cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<D, kDyn>, mq, mk, mv, p);
+}
+}  // namespace
+
 cudaError_t launch_attn_tc(int head_dim, int n_ctas, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                            const AttnParams& p, cudaStream_t stream) {
-  static bool attr_set[2] = {false, false};
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
@@ -725,27 +793,16 @@ cudaError_t launch_attn_tc(int head_dim, int n_ctas, const CUtensorMap& mq, cons
   cfg.stream = stream;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
+  const bool dyn = p.queue != nullptr;
   cudaError_t le = cudaSuccess;
   if (head_dim == 128) {
     const size_t smem = TcLayout<128>::kTotal + 1024;
-    if (!attr_set[0]) {
-      cudaError_t e = cudaFuncSetAttribute(tree_attn_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
-      if (e != cudaSuccess) return e;
-      attr_set[0] = true;
-    }
-    cfg.dynamicSmemBytes = smem;
-    le = cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<128>, mq, mk, mv, p);
+    le = dyn ? launch_one<128, true>(cfg, smem, mq, mk, mv, p) : launch_one<128, false>(cfg, smem, mq, mk, mv, p);
   } else {
     // padded past half of an SM's shared memory: one CTA per SM, since each CTA takes all 512 TMEM columns
     const size_t smem = 120 * 1024;
     static_assert(TcLayout<64>::kTotal + 1024 <= 120 * 1024, "smem layout");
-    if (!attr_set[1]) {
-      cudaError_t e = cudaFuncSetAttribute(tree_attn_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
-      if (e != cudaSuccess) return e;
-      attr_set[1] = true;
-    }
-    cfg.dynamicSmemBytes = smem;
-    le = cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<64>, mq, mk, mv, p);
+    le = dyn ? launch_one<64, true>(cfg, smem, mq, mk, mv, p) : launch_one<64, false>(cfg, smem, mq, mk, mv, p);
   }
   return le != cudaSuccess ? le : cudaGetLastError();
 }

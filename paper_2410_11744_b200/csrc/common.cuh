@@ -87,6 +87,11 @@ struct AttnParams {
   const int32_t* page_table;
   int32_t pages_per_req;
   int32_t page_shift;
+  // Shared work queue (null = every CTA has a fixed list): `items` then holds all n_items_total items in
+  // queue order, CTA c starts with item c and takes further ones with an atomic add on queue[0];
+  // queue[1] counts the CTAs that found the queue empty, and the last of them clears both words.
+  int32_t* queue;
+  int32_t n_items_total;
 };
 
 #ifdef __CUDACC__

@@ -191,3 +191,38 @@ def test_runs_are_bitwise_repeatable(rt):
         batch.out.zero_()
         batch.step()
         assert np.array_equal(batch.results()[2], first)
+
+
+def test_shared_queue_plan_is_repeatable_and_leaves_the_queue_empty(rt):
+    """More groups than CTAs in the tensor-core regime: the CTAs take whole groups from a shared queue.
+    Every launch must see the queue as the previous one left it (cleared), back to back and through
+    two buffer sets that share the plan, and the result cannot depend on which CTA took which group."""
+    B, R = rt
+    rng = np.random.default_rng(31)
+    trees = [wl.greedy_tree(rng, n, 8, 0.3) for n in (300, 700, 130, 520)]
+    w = wl.make_custom(33, 16, 2, 128, [600, 90, 2000, 0], trees)      # 8 rows per node: 52 query tiles x 2 kv heads... x 4 requests
+    w_big = wl.make_custom(34, 64, 8, 128, [1500, 300, 40, 700, 2500, 0], [wl.greedy_tree(rng, n, 8, 0.3) for n in (400, 640, 96, 512, 333, 768)])
+    for wk in (w, w_big):
+        batch, got, _ = run_and_check(rt, wk, regime=1)
+        info = batch.plan.describe()
+        if wk is w_big:
+            assert info["dynamic"] == 1 and info["split_groups"] == 0 and info["groups"] > info["ctas"]
+        first = batch.results()[2].copy()
+        twin = R.DeviceBatch(wk, plan=batch.plan)
+        for _ in range(3):
+            batch.out.zero_()
+            batch.step()
+            twin.step()
+            assert np.array_equal(batch.results()[2], first)
+            assert np.array_equal(twin.results()[2], first)
+    # the budgeted split plan (fixed lists, partials merged by the combine kernel) agrees up to the
+    # rounding of a different summation order
+    B.dyspec_set_tuning(1, 0, 2 + 16)
+    try:
+        fixed = R.DeviceBatch(w_big)
+    finally:
+        B.dyspec_set_tuning(-1, 0, 2)
+    assert fixed.plan.describe()["dynamic"] == 0
+    fixed.step()
+    diff = np.abs(orc.bf16_bits_to_f64(fixed.results()[2]) - orc.bf16_bits_to_f64(first))
+    assert diff.max() <= MAX_ABS
