@@ -450,6 +450,30 @@ def paged_experiment(torch, runner, workloads, B, peaks, device, configs=(2, 3, 
     return out
 
 
+def small_tree_batch_experiment(torch, runner, workloads, peaks, device, steps=100):
+    """The small-tree regime at a size where its rate, not its latency, shows: 8 requests of the Llama2-7B
+    shape (32 heads x 128, 64-node greedy trees as in config 2) over 4096-token prefixes, and a ragged batch
+    of 16 requests (prefix 200 - 3000, 32-node trees).  HBM-bound: achieved bytes/s against the measured copy peak."""
+    rng = np.random.default_rng(workloads.MASTER_SEED + 77)
+    cases = [
+        ("8 requests, 32 heads, prefix 4096, 64-node trees",
+         workloads.make_custom(1, 32, 32, 128, [4096] * 8, [workloads.greedy_tree(rng, 64, 8, 0.3) for _ in range(8)])),
+        ("16 requests, 32 heads, prefix 200-3000, 32-node trees",
+         workloads.make_custom(3, 32, 32, 128, [int(x) for x in rng.integers(200, 3000, 16)],
+                               [workloads.greedy_tree(rng, 32, 8, 0.3) for _ in range(16)])),
+    ]
+    out = []
+    for label, w in cases:
+        m = measure_config(torch, runner, w, steps, 3, device)
+        gbs = m["bytes"] / (m["attn_ms"] * 1e-3) / 1e9
+        out.append({"case": label, "tree_tokens": w.total_nodes, "attention_call_us": m["attn_ms"] * 1e3,
+                    "step_us": m["ms_per_step"] * 1e3, "bytes": m["bytes"], "achieved_gbs": gbs,
+                    "frac_of_hbm": gbs / peaks["hbm_gbs"], "plan": m["info"], "status": m["status"]})
+        del m
+        torch.cuda.empty_cache()
+    return out
+
+
 def roofline_entry(m, peaks, peaks_kind):
     t_hbm = m["bytes"] / (peaks["hbm_gbs"] * 1e9)
     t_tc = m["flops"] / (peaks["bf16_tflops"] * 1e12)
@@ -599,6 +623,10 @@ def run_ours(args):
     if not args.no_per_config and world == 1:
         paged = paged_experiment(torch, runner, workloads, binding, peaks, device)
 
+    small_batch = None
+    if not args.no_per_config and world == 1:
+        small_batch = small_tree_batch_experiment(torch, runner, workloads, peaks, device)
+
     # ---- the oracle on the host cores, bounded sample of the same workload
     times = time_oracle(w, budget_s=12.0)
     cpu_sec = sum(times) / len(times)
@@ -635,6 +663,8 @@ def run_ours(args):
         line["compaction_experiment"] = compaction
     if paged:
         line["paged_cache_experiment"] = paged
+    if small_batch:
+        line["small_tree_batch_experiment"] = small_batch
     print(json.dumps(line), flush=True)
     if use_dist:
         dist.barrier()
