@@ -13,8 +13,9 @@
 //              runs the fp32 online softmax in the exp2 domain and accumulates O += P V with
 //              mma.sync.m16n8k16 (P stays in registers, V through ldmatrix.trans).  The per-tile code
 //              is a chain of dependent instructions, so one warp per scheduler leaves the SM mostly
-//              idle; two interleaved tiles per scheduler double the rate.  At the end of an item set 1
-//              hands its (O, m, l) to set 0 through shared memory, thread to thread.
+//              idle; two interleaved tiles per scheduler double the rate.  At the end of an item the
+//              sets swap column halves of their (O, m, l) through shared memory, thread to thread, and
+//              each finishes one half of the columns.
 // A CTA walks its list of work items; an item either writes final bf16 rows or an fp32 partial
 // (O, m, l) for the split-KV combine kernel.  In cluster mode (uniform small batches) the splits of
 // a query tile are the CTAs of one thread-block cluster and are merged on chip through distributed
@@ -44,7 +45,7 @@ struct SmemLayout {
   static constexpr int kStageBytes = 2 * kTileBytes;     // K then V
   static constexpr int kBarOffset = kQBytes + kStages * kStageBytes;
   static constexpr int kExchMlOffset = kBarOffset + 512;  // set 1 -> set 0: (m, l) of every thread's two rows
-  static constexpr int kTotal = kExchMlOffset + kComputeWarps * 32 * 16;
+  static constexpr int kTotal = kExchMlOffset + kSets * kComputeWarps * 32 * 16;
   static constexpr int kTmemCols = 512;                  // one 64-column score buffer per ring stage (power of two)
 };
 
@@ -405,39 +406,47 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1);
     l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
 
-    // ---- the two warp sets took alternate tiles: set 1 hands its (O, m, l) to set 0, thread to thread
-    //      (thread ctid of either set owns the same rows and columns), and set 0 alone runs the epilogue.
+    // ---- the two warp sets took alternate tiles and thread ctid of either set owns the same rows and
+    //      column pairs.  They swap halves: set 0 gives away its right half of the columns (D/2 ..) and
+    //      receives set 1's left half, and the other way round, so that afterwards each set holds the
+    //      merged values of ONE half (moved to o[0 .. DT/2)) and both run every later step (parking,
+    //      storing) on half the columns each.  (m, l) are merged identically on both sides.
+    constexpr int HT = DT / 2;                    // 8-column tiles per half
+    constexpr int kAll = kSets * kComputeWarps * 32;
     if (merge_owner)              // the hand-over buffer is a ring stage here: both sets must be done with the ring
-      asm volatile("bar.sync %0, %1;" ::"n"(kBarRingIdle), "n"(kSets * kComputeWarps * 32) : "memory");
-    if (set == 1) {
-      if (w != item_begin)        // set 0 has read the previous item's values
-        asm volatile("bar.sync %0, %1;" ::"n"(kBarExchFree), "n"(kSets * kComputeWarps * 32) : "memory");
-#pragma unroll
-      for (int j = 0; j < DT; ++j) exch_o[j * (kComputeWarps * 32) + ctid] = make_float4(o[j][0], o[j][1], o[j][2], o[j][3]);
-      exch_ml[ctid] = make_float4(m_lo, m_hi, l_lo, l_hi);
-      asm volatile("bar.arrive %0, %1;" ::"n"(kBarExchFull), "n"(kSets * kComputeWarps * 32) : "memory");
-      if (p.cluster_size <= 1) continue;         // in cluster mode the set lends its threads to the merge below
-    } else {
-    asm volatile("bar.sync %0, %1;" ::"n"(kBarExchFull), "n"(kSets * kComputeWarps * 32) : "memory");
+      asm volatile("bar.sync %0, %1;" ::"n"(kBarRingIdle), "n"(kAll) : "memory");
+    if (w != item_begin)          // both sets have read the previous item's values
+      asm volatile("bar.sync %0, %1;" ::"n"(kBarExchFree), "n"(kAll) : "memory");
     {
-      const float4 ml = exch_ml[ctid];
+      float4* give = exch_o + set * (HT * kComputeWarps * 32);
+      const float4* take = exch_o + (1 - set) * (HT * kComputeWarps * 32);
+      if (set == 0) {
+#pragma unroll
+        for (int j = 0; j < HT; ++j) give[j * (kComputeWarps * 32) + ctid] = make_float4(o[HT + j][0], o[HT + j][1], o[HT + j][2], o[HT + j][3]);
+      } else {
+#pragma unroll
+        for (int j = 0; j < HT; ++j) give[j * (kComputeWarps * 32) + ctid] = make_float4(o[j][0], o[j][1], o[j][2], o[j][3]);
+#pragma unroll
+        for (int j = 0; j < HT; ++j) { o[j][0] = o[HT + j][0]; o[j][1] = o[HT + j][1]; o[j][2] = o[HT + j][2]; o[j][3] = o[HT + j][3]; }
+      }
+      exch_ml[set * (kComputeWarps * 32) + ctid] = make_float4(m_lo, m_hi, l_lo, l_hi);
+      asm volatile("bar.sync %0, %1;" ::"n"(kBarExchFull), "n"(kAll) : "memory");
+      const float4 ml = exch_ml[(1 - set) * (kComputeWarps * 32) + ctid];
       const float mn_lo = fmaxf(m_lo, ml.x), mn_hi = fmaxf(m_hi, ml.y);
       const float ref_lo = mn_lo == -INFINITY ? 0.f : mn_lo, ref_hi = mn_hi == -INFINITY ? 0.f : mn_hi;
       const float ka_lo = fast_exp2(m_lo - ref_lo), kb_lo = fast_exp2(ml.x - ref_lo);
       const float ka_hi = fast_exp2(m_hi - ref_hi), kb_hi = fast_exp2(ml.y - ref_hi);
 #pragma unroll
-      for (int j = 0; j < DT; ++j) {
-        const float4 ob = exch_o[j * (kComputeWarps * 32) + ctid];
+      for (int j = 0; j < HT; ++j) {
+        const float4 ob = take[j * (kComputeWarps * 32) + ctid];
         o[j][0] = o[j][0] * ka_lo + ob.x * kb_lo; o[j][1] = o[j][1] * ka_lo + ob.y * kb_lo;
         o[j][2] = o[j][2] * ka_hi + ob.z * kb_hi; o[j][3] = o[j][3] * ka_hi + ob.w * kb_hi;
       }
       l_lo = l_lo * ka_lo + ml.z * kb_lo; l_hi = l_hi * ka_hi + ml.w * kb_hi;
       m_lo = mn_lo; m_hi = mn_hi;
     }
+    const int cbase = set * (D / 2);              // first column of this set's half
     if (threadIdx.x == 0 && w == item_begin) stamp(1);
-    if (w + 1 < item_end)
-      asm volatile("bar.arrive %0, %1;" ::"n"(kBarExchFree), "n"(kSets * kComputeWarps * 32) : "memory");
-    }
     if (p.cluster_size > 1) {
       // ---- split-KV combine inside a thread-block cluster: the CTAs of a cluster hold the splits of
       // one query tile (a CTA owns exactly one item in this mode).  The scheduler names the owners
@@ -464,20 +473,20 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       if (own && threadIdx.x == 0)
         for (int s_ = 0; s_ < C; ++s_)
           if (s_ != rank) mbar_expect_tx(bar_src + 8 * s_, chunk_bytes);
-      // (every warp is done with the ring: set 0's warps met at the hand-over barrier, which set 1 arrived on)
-      if (set == 0) {
+      // (every warp is done with the ring: all of them met at the hand-over barrier)
+      {
         // columns are XOR-swizzled by the row so that the 8 rows a warp stores at once hit different banks
         const int r_lo = wrow + gid, r_hi = r_lo + 8;
         float* c_lo = send + (r_lo >> log2r) * chunk_floats;
         float* c_hi = send + (r_hi >> log2r) * chunk_floats;
         const int rr_lo = r_lo & (R - 1), rr_hi = r_hi & (R - 1);
 #pragma unroll
-        for (int j = 0; j < DT; ++j) {
-          const int c = j * 8 + tig * 2;
+        for (int j = 0; j < HT; ++j) {
+          const int c = cbase + j * 8 + tig * 2;
           *reinterpret_cast<float2*>(c_lo + rr_lo * D + (c ^ ((rr_lo & 7) << 3))) = make_float2(o[j][0], o[j][1]);
           *reinterpret_cast<float2*>(c_hi + rr_hi * D + (c ^ ((rr_hi & 7) << 3))) = make_float2(o[j][2], o[j][3]);
         }
-        if (tig == 0) {
+        if (tig == 0 && set == 0) {
           c_lo[R * D + rr_lo] = m_lo; c_lo[R * D + R + rr_lo] = l_lo;
           c_hi[R * D + rr_hi] = m_hi; c_hi[R * D + R + rr_hi] = l_hi;
         }
@@ -589,8 +598,8 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       __nv_bfloat16* out_lo = p.out + (size_t(rq.node0 + node_lo) * p.n_q_heads + head_lo) * D;
       __nv_bfloat16* out_hi = p.out + (size_t(rq.node0 + node_hi) * p.n_q_heads + head_hi) * D;
 #pragma unroll
-      for (int j = 0; j < DT; ++j) {
-        const int c = j * 8 + tig * 2;
+      for (int j = 0; j < HT; ++j) {
+        const int c = cbase + j * 8 + tig * 2;
         if (ok_lo) *reinterpret_cast<uint32_t*>(out_lo + c) = pack_bf16x2(o[j][0] * inv_lo, o[j][1] * inv_lo);
         if (ok_hi) *reinterpret_cast<uint32_t*>(out_hi + c) = pack_bf16x2(o[j][2] * inv_hi, o[j][3] * inv_hi);
       }
@@ -599,12 +608,12 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       float* slot = p.partial + size_t(item.slot) * p.slot_floats;
       const int r_lo = wrow + gid, r_hi = r_lo + 8;
 #pragma unroll
-      for (int j = 0; j < DT; ++j) {
-        const int c = j * 8 + tig * 2;
+      for (int j = 0; j < HT; ++j) {
+        const int c = cbase + j * 8 + tig * 2;
         if (ok_lo) *reinterpret_cast<float2*>(slot + r_lo * D + c) = make_float2(o[j][0], o[j][1]);
         if (ok_hi) *reinterpret_cast<float2*>(slot + r_hi * D + c) = make_float2(o[j][2], o[j][3]);
       }
-      if (tig == 0) {
+      if (tig == 0 && set == 0) {
         if (ok_lo) { slot[BM * D + r_lo] = m_lo; slot[BM * D + BM + r_lo] = l_lo; }
         if (ok_hi) { slot[BM * D + r_hi] = m_hi; slot[BM * D + BM + r_hi] = l_hi; }
       }
