@@ -202,10 +202,11 @@ def test_shared_queue_plan_is_repeatable_and_leaves_the_queue_empty(rt):
     trees = [wl.greedy_tree(rng, n, 8, 0.3) for n in (300, 700, 130, 520)]
     w = wl.make_custom(33, 16, 2, 128, [600, 90, 2000, 0], trees)      # 8 rows per node: 52 query tiles x 2 kv heads... x 4 requests
     w_big = wl.make_custom(34, 64, 8, 128, [1500, 300, 40, 700, 2500, 0], [wl.greedy_tree(rng, n, 8, 0.3) for n in (400, 640, 96, 512, 333, 768)])
-    for wk in (w, w_big):
+    w_d64 = wl.make_custom(35, 32, 8, 64, [900, 64, 0, 1300, 257], [wl.greedy_tree(rng, n, 8, 0.3) for n in (700, 512, 90, 640, 333)])
+    for wk in (w, w_big, w_d64):
         batch, got, _ = run_and_check(rt, wk, regime=1)
         info = batch.plan.describe()
-        if wk is w_big:
+        if wk is not w:
             assert info["dynamic"] == 1 and info["split_groups"] == 0 and info["groups"] > info["ctas"]
         first = batch.results()[2].copy()
         twin = R.DeviceBatch(wk, plan=batch.plan)
@@ -224,5 +225,8 @@ def test_shared_queue_plan_is_repeatable_and_leaves_the_queue_empty(rt):
         B.dyspec_set_tuning(-1, 0, 2)
     assert fixed.plan.describe()["dynamic"] == 0
     fixed.step()
+    first = R.DeviceBatch(w_big)
+    first.step()
+    first = first.results()[2]
     diff = np.abs(orc.bf16_bits_to_f64(fixed.results()[2]) - orc.bf16_bits_to_f64(first))
     assert diff.max() <= MAX_ABS
