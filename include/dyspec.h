@@ -79,6 +79,16 @@ int dyspec_build_tree_mask(const int32_t* parents, int n_nodes, uint32_t* ancest
                            int words_per_row, int32_t* status, dyspec_stream_t stream);
 
 /*
+ * (1a) The same for a ragged batch without a plan: node_offsets is a HOST array [n_req + 1] (prefix sums
+ * of the tree sizes), parents are request-local indices, concatenated; request r's mask rows and depths
+ * start at node_offsets[r]; every row uses the same words_per_row.  status: dev int32 [n_req] or NULL (one
+ * word per request).  Runs one launch per request; dyspec_plan_build_tree_mask (1b) does a batch in one.
+ */
+int dyspec_build_tree_mask_batched(const int32_t* parents, const int32_t* node_offsets_host, int n_req,
+                                   uint32_t* ancestor_bits, int32_t* depths, int words_per_row, int32_t* status,
+                                   dyspec_stream_t stream);
+
+/*
  * (2) Plans.  A plan fixes the static shape and the ragged batch structure, runs the host-side
  * scheduler (work list of (request, kv-head, query-tile, kv-split) items balanced over the SMs)
  * and owns a small device copy of that list.  Create it once per batch structure; reuse it for
@@ -106,7 +116,8 @@ int dyspec_plan_create(dyspec_plan_t** plan, int n_q_heads, int n_kv_heads, int 
                        int64_t kv_total_rows, int words_per_row, float scale);
 int dyspec_plan_destroy(dyspec_plan_t* plan);
 
-/* Bytes of scratch the attention call needs (split-KV partials + arrival counters); may be 0. */
+/* Bytes of scratch the attention call needs (split-KV partials, the words of the shared work queue); may
+ * be 0.  The caller zeroes the workspace once, before its first use. */
 size_t dyspec_plan_workspace_bytes(const dyspec_plan_t* plan);
 
 /* Scheduler introspection (for tests and benchmarks): field 0 = work items, 1 = CTAs launched,
@@ -169,9 +180,9 @@ int dyspec_plan_build_tree_mask(const dyspec_plan_t* plan, const int32_t* parent
  *   workspace      dev, >= dyspec_plan_workspace_bytes(plan), 256-byte aligned; its arrival counters
  *                  must be zero before the first call (dyspec_plan_create's caller zeroes it once;
  *                  the kernels leave them zero).  Two calls that overlap on the GPU need two workspaces
- *                  AND two plans (a plan owns device words that a launch uses and clears: arrival
- *                  counters of split groups, the head of the shared work queue); calls that follow
- *                  each other on one stream may share both.
+ *                  (a workspace holds words that a launch uses and clears: the head of the plan's
+ *                  shared work queue); calls that follow each other on one stream may share one, and a
+ *                  plan may be shared by any number of calls.
  *   status         dev int32 [1] or NULL
  */
 int dyspec_tree_attention_ragged(const dyspec_plan_t* plan, const void* q, const void* k_cache, const void* v_cache,

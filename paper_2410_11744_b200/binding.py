@@ -32,6 +32,7 @@ SIGNATURES = {
     "dyspec_set_tuning": (_i32, [_i32, _i32, _i32]),
     "dyspec_set_trace": (_i32, [_vp, _i32]),
     "dyspec_build_tree_mask": (_i32, [_vp, _i32, _vp, _vp, _i32, _vp, _vp]),
+    "dyspec_build_tree_mask_batched": (_i32, [_vp, _vp, _i32, _vp, _vp, _i32, _vp, _vp]),
     "dyspec_plan_create": (_i32, [_c.POINTER(_vp), _i32, _i32, _i32, _i32, _vp, _vp, _vp, _i64, _i32, _f32]),
     "dyspec_plan_destroy": (_i32, [_vp]),
     "dyspec_plan_workspace_bytes": (_sz, [_vp]),
@@ -345,3 +346,12 @@ def dyspec_compact_kv_paged(k_cache, v_cache, tree_row_offset, page_table, pages
                                        int(pages_per_req), int(page_size), _ptr(prefix_len), _ptr(accepted_nodes),
                                        _ptr(n_accepted), n_req, max_out, n_kv_heads, head_dim, _ptr(new_prefix_len),
                                        _ptr(status), _stream(stream)), "dyspec_compact_kv_paged")
+
+
+def dyspec_build_tree_mask_batched(parents, node_offsets: Sequence[int], ancestor_bits, depths, words_per_row: int,
+                                   status=None, stream=None) -> None:
+    """Ragged batch without a plan: node_offsets is a host sequence [n_req + 1] (see include/dyspec.h)."""
+    n_req = len(node_offsets) - 1
+    offs = (_c.c_int32 * (n_req + 1))(*[int(x) for x in node_offsets])
+    _check(lib.dyspec_build_tree_mask_batched(_ptr(parents), _c.cast(offs, _vp), n_req, _ptr(ancestor_bits), _ptr(depths),
+                                              words_per_row, _ptr(status), _stream(stream)), "dyspec_build_tree_mask_batched")

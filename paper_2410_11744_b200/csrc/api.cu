@@ -127,8 +127,9 @@ struct dyspec_plan {
   WorkItem* d_items = nullptr;
   GroupInfo* d_groups = nullptr;
   int32_t* d_counters = nullptr;
-  int32_t* d_queue = nullptr;           // dynamic plans: [0] next item of the shared queue, [1] CTAs that have drained it
   bool dynamic = false;                 // whole groups taken from a shared queue (longest first) instead of fixed lists
+  bool allow_queue = true;              // false: fixed lists only (callers that cannot provide zeroed queue words)
+  size_t queue_offset = 0;              // dynamic plans: byte offset of the two queue words inside the caller's workspace
   std::vector<WorkItem> items_queue;    // dynamic plans: all items in queue order
   size_t workspace_bytes = 0;
 };
@@ -362,7 +363,7 @@ void schedule(dyspec_plan& pl) {
       // On the device the CTAs take the groups from one queue, longest first (CTA c starts with the
       // c-th longest), so that what the cost model cannot see -- tree tiles skipped by the tile sets,
       // cache misses of one request's long prefix -- does not leave some CTAs working while others idle.
-      if (pl.regime == 1 && int64_t(groups.size()) > n_bins) {
+      if (pl.allow_queue && pl.regime == 1 && int64_t(groups.size()) > n_bins) {
         pl.dynamic = true;
         for (size_t gi : order) {
           const Group& gr = groups[gi];
@@ -400,7 +401,7 @@ int upload(dyspec_plan& pl) {
   const size_t b_reqs = pad(std::max<size_t>(1, pl.reqs.size()) * sizeof(ReqInfo));
   const size_t b_items = pad(std::max<size_t>(1, pl.items_strided.size()) * sizeof(WorkItem));
   const size_t b_groups = pad(std::max<size_t>(1, pl.split_groups.size()) * sizeof(GroupInfo));
-  const size_t b_counters = pad(std::max<size_t>(1, pl.split_groups.size()) * sizeof(int32_t)) + 256;   // + the queue words
+  const size_t b_counters = pad(std::max<size_t>(1, pl.split_groups.size()) * sizeof(int32_t));
   const size_t total = b_reqs + b_items + b_groups + b_counters;
   std::vector<uint8_t> host(total, 0);
   size_t off = 0;
@@ -418,7 +419,6 @@ int upload(dyspec_plan& pl) {
   pl.d_items = reinterpret_cast<WorkItem*>(base + o_items);
   pl.d_groups = reinterpret_cast<GroupInfo*>(base + o_groups);
   pl.d_counters = reinterpret_cast<int32_t*>(base + o_counters);
-  pl.d_queue = reinterpret_cast<int32_t*>(base + o_counters + b_counters - 256);
   return DYSPEC_OK;
 }
 
@@ -483,6 +483,26 @@ static int build_tree_mask_checked(const int32_t* parents, int n_nodes, uint32_t
 int dyspec_build_tree_mask(const int32_t* parents, int n_nodes, uint32_t* ancestor_bits, int32_t* depths,
                            int words_per_row, int32_t* status, dyspec_stream_t stream) {
   return build_tree_mask_checked(parents, n_nodes, ancestor_bits, depths, nullptr, words_per_row, status, stream);
+}
+
+int dyspec_build_tree_mask_batched(const int32_t* parents, const int32_t* node_offsets_host, int n_req,
+                                   uint32_t* ancestor_bits, int32_t* depths, int words_per_row, int32_t* status,
+                                   dyspec_stream_t stream) {
+  if (n_req < 0 || (n_req > 0 && !node_offsets_host)) return DYSPEC_ERR_INVALID_ARG;
+  for (int r = 0; r < n_req; ++r)
+    if (node_offsets_host[r] < 0 || node_offsets_host[r + 1] < node_offsets_host[r]) return DYSPEC_ERR_INVALID_ARG;
+  // Without a plan there is no device copy of the request list: one launch per request (the kernel of
+  // the single-request call), each on the request's slice of the arrays.  dyspec_plan_build_tree_mask
+  // does the whole batch in one launch.
+  for (int r = 0; r < n_req; ++r) {
+    const int64_t at = node_offsets_host[r];
+    const int n = node_offsets_host[r + 1] - node_offsets_host[r];
+    const int rc = build_tree_mask_checked(parents ? parents + at : nullptr, n, ancestor_bits ? ancestor_bits + at * words_per_row : nullptr,
+                                           depths ? depths + at : nullptr, nullptr, words_per_row, status ? status + r : nullptr,
+                                           stream);
+    if (rc != DYSPEC_OK) return rc;
+  }
+  return DYSPEC_OK;
 }
 
 int dyspec_build_tree_mask_tiles(const int32_t* parents, int n_nodes, uint32_t* ancestor_bits, int32_t* depths,
@@ -606,7 +626,8 @@ int dyspec_compact_kv_paged(void* k_cache, void* v_cache, const int64_t* tree_ro
 // Validates the arguments and runs the scheduler; no CUDA call.
 static int make_host_plan(dyspec_plan** out, int n_q_heads, int n_kv_heads, int head_dim, int n_req,
                           const int32_t* prefix_len, const int32_t* n_nodes, const int64_t* kv_row_offset,
-                          int64_t kv_total_rows, int words_per_row, float scale, int page_size = 0) {
+                          int64_t kv_total_rows, int words_per_row, float scale, int page_size = 0,
+                          bool allow_queue = true) {
   *out = nullptr;
   if (n_q_heads <= 0 || n_kv_heads <= 0 || n_req < 0 || kv_total_rows < 0) return DYSPEC_ERR_INVALID_ARG;
   if (page_size < 0 || (page_size & (page_size - 1))) return DYSPEC_ERR_INVALID_ARG;
@@ -628,6 +649,7 @@ static int make_host_plan(dyspec_plan** out, int n_q_heads, int n_kv_heads, int 
   pl->n_req = n_req;
   pl->kv_total_rows = kv_total_rows;
   pl->page_size = page_size;
+  pl->allow_queue = allow_queue;
   int64_t node0 = 0;
   int max_rows = 0;
   for (int r = 0; r < n_req; ++r) {
@@ -651,6 +673,10 @@ static int make_host_plan(dyspec_plan** out, int n_q_heads, int n_kv_heads, int 
   pl->bn = pl->regime == 0 ? 64 : 128;    // keys per tile
   schedule(*pl);
   pl->workspace_bytes = size_t(pl->n_slots) * size_t(pl->bm) * (pl->d + 2) * sizeof(float);
+  if (pl->dynamic) {                    // the queue words follow the partials (there are none in such a plan today)
+    pl->queue_offset = (pl->workspace_bytes + 255) & ~size_t(255);
+    pl->workspace_bytes = pl->queue_offset + 256;
+  }
   *out = pl;
   return DYSPEC_OK;
 }
@@ -837,7 +863,7 @@ static int run_attention(const dyspec_plan_t* plan, const void* q, const void* k
   p.bits = ancestor_bits; p.node_tiles = node_tiles; p.out = static_cast<__nv_bfloat16*>(out);
   p.partial = static_cast<float*>(workspace);
   p.counters = plan->d_counters; p.status = status;
-  p.queue = plan->dynamic ? plan->d_queue : nullptr;
+  p.queue = plan->dynamic ? reinterpret_cast<int32_t*>(static_cast<unsigned char*>(workspace) + plan->queue_offset) : nullptr;
   p.n_items_total = int32_t(plan->items_strided.size());
   p.n_q_heads = plan->hq; p.n_kv_heads = plan->hkv; p.group_size = plan->g; p.log2_g = plan->log2g;
   p.words_per_row = plan->W; p.slot_floats = bm * (plan->d + 2);
@@ -892,7 +918,9 @@ int dyspec_tree_attention(const void* q, const void* k_cache, const void* v_cach
                                   g_shape.scale);
       if (rc != DYSPEC_OK) return rc;
       void* ws = nullptr;
-      if (pl->workspace_bytes > 0 && cudaMalloc(&ws, pl->workspace_bytes) != cudaSuccess) {
+      if (pl->workspace_bytes > 0 &&
+          (cudaMalloc(&ws, pl->workspace_bytes) != cudaSuccess || cudaMemset(ws, 0, pl->workspace_bytes) != cudaSuccess)) {
+        if (ws) cudaFree(ws);
         dyspec_plan_destroy(pl);
         return DYSPEC_ERR_CUDA;
       }
@@ -944,7 +972,9 @@ extern "C" int dyspec_tree_attention_static(const void* q, const void* k_cache, 
   const int32_t L = prefix_len, n = n_nodes;
   const int64_t off = 0;
   dyspec_plan* pl = nullptr;
-  int rc = make_host_plan(&pl, n_q_heads, n_kv_heads, head_dim, 1, &L, &n, &off, int64_t(L) + n, words_per_row, scale);
+  // fixed work lists only: the scratch array is rewritten by every call, there is no zeroed queue to share
+  int rc = make_host_plan(&pl, n_q_heads, n_kv_heads, head_dim, 1, &L, &n, &off, int64_t(L) + n, words_per_row, scale,
+                          0, false);
   if (rc != DYSPEC_OK) return rc;
   struct Guard { dyspec_plan* p; ~Guard() { delete p; } } guard{pl};   // host-only object: nothing to cudaFree
   if (pl->n_ctas == 0) return DYSPEC_OK;

@@ -48,7 +48,7 @@ class DeviceBatch:
         self.status = torch.zeros((1,), dtype=torch.int32, device=dev)
         self.out = torch.zeros((n, w.n_q_heads, w.head_dim), dtype=torch.bfloat16, device=dev)
         ws = self.plan.workspace_bytes()
-        self.workspace = torch.empty((max(ws, 256),), dtype=torch.uint8, device=dev)
+        self.workspace = torch.zeros((max(ws, 256),), dtype=torch.uint8, device=dev)   # zeroed once: queue words live in it
         self.workspace_bytes = ws
         if upload:
             self.upload()

@@ -230,3 +230,31 @@ def test_shared_queue_plan_is_repeatable_and_leaves_the_queue_empty(rt):
     first = first.results()[2]
     diff = np.abs(orc.bf16_bits_to_f64(fixed.results()[2]) - orc.bf16_bits_to_f64(first))
     assert diff.max() <= MAX_ABS
+
+
+def test_mask_builder_batched_without_a_plan(rt):
+    """dyspec_build_tree_mask_batched (host node offsets, no plan) == the oracle, request by request,
+    including an empty request and a bad parent that must be reported for its own request only."""
+    import torch
+    B, _ = rt
+    rng = np.random.default_rng(41)
+    trees = [wl.greedy_tree(rng, 70, 6, 0.3), np.zeros(0, np.int32), wl.chain_tree(5), wl.random_tree(rng, 300),
+             np.array([-1, 0, 7, 1], np.int32)]                       # entry 2 of the last tree is invalid
+    offs = np.concatenate([[0], np.cumsum([len(t) for t in trees])]).astype(np.int32)
+    n = int(offs[-1])
+    W = B.dyspec_words_per_row(max(len(t) for t in trees))
+    dev = "cuda:0"
+    parents = torch.from_numpy(np.concatenate(trees).astype(np.int32)).to(dev)
+    bits = torch.full((n, W), -1, dtype=torch.int32, device=dev)
+    depths = torch.full((n,), -1, dtype=torch.int32, device=dev)
+    status = torch.zeros(len(trees), dtype=torch.int32, device=dev)
+    B.dyspec_build_tree_mask_batched(parents, offs.tolist(), bits, depths, W, status)
+    torch.cuda.synchronize()
+    assert status.cpu().numpy().tolist() == [0, 0, 0, 0, -5]
+    fixed = [t.copy() for t in trees]
+    fixed[-1][2] = -1                                                   # an invalid parent is treated as "no parent"
+    ref_bits, ref_depths = orc.build_tree_mask_ragged(fixed, W)
+    assert np.array_equal(bits.cpu().numpy().view(np.uint32), ref_bits)
+    assert np.array_equal(depths.cpu().numpy(), ref_depths)
+    with pytest.raises(B.DyspecError):
+        B.dyspec_build_tree_mask_batched(parents, [0, 5, 3], bits, depths, W, None)     # offsets must not decrease

@@ -33,12 +33,16 @@ def test_static_scratch_entry_point_matches_ragged_entry_point_twice_in_a_row():
     # needs the work list), so stale contents would show; then the first shape again
     rng = np.random.default_rng(3)
     big = wl.make_custom(20, 64, 8, 128, [1500], [wl.greedy_tree(rng, 40, 8, 0.3)])
-    cases = [big, wl.make_custom(21, 8, 2, 64, [300], [wl.greedy_tree(rng, 40, 4, 0.3)]), wl.make_config(2), big]
+    # ... and one request with more (kv head, query tile) groups than CTAs: through a plan it runs from
+    # the shared queue in the caller's workspace, here (no workspace) from fixed lists
+    many = wl.make_custom(22, 64, 8, 128, [200], [wl.greedy_tree(rng, 1024, 8, 0.3)])
+    cases = [big, wl.make_custom(21, 8, 2, 64, [300], [wl.greedy_tree(rng, 40, 4, 0.3)]), wl.make_config(2), many, big]
     for w in cases:
         batch = R.DeviceBatch(w)
         batch.step()                                          # existing entry points: mask + ragged attention
         bits, _, want_bits, status = batch.results()
         assert status == 0
+        assert batch.plan.describe()["dynamic"] == (1 if w is many else 0)
         L, n = int(w.prefix_len[0]), int(w.n_nodes[0])
         out = torch.zeros_like(batch.out)
         st = torch.zeros((1,), dtype=torch.int32, device=out.device)
