@@ -33,6 +33,7 @@ L2_BYTES = 126 * 1024 * 1024
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu
 # captures summarised under profiles/ (tree_attn_mma_c2_*.md, tree_attn_tc_c4_*.md)
 NCU_TRAFFIC_BYTES = {"c2_llama2_7b_L1024_n64": 18413312, "c4_llama2_70b_L2048_n512": 18991872}
+NOMINAL_HBM_GBS, NOMINAL_BF16_TFLOPS = 8000.0, 2250.0
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -478,15 +479,18 @@ def roofline_entry(m, peaks, peaks_kind):
     t_hbm = m["bytes"] / (peaks["hbm_gbs"] * 1e9)
     t_tc = m["flops"] / (peaks["bf16_tflops"] * 1e12)
     dur = (m["attn_ms"] if m["attn_ms"] is not None else m["ms_per_step"]) * 1e-3
+    # nominal figures (HGX B200: 8 TB/s HBM3e as the workload definition quotes it, 2.25 PFLOP/s dense bf16): context only
     if t_hbm >= t_tc:
         ach = m["bytes"] / dur / 1e9
         return {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],
                 "traffic": None, "peak_kind": peaks_kind, "kernel": "tree attention call (main kernel + combine)",
-                "launch_us": dur * 1e6}
+                "launch_us": dur * 1e6, "frac_of_nominal": ach / NOMINAL_HBM_GBS, "nominal_peak": NOMINAL_HBM_GBS}
     ach = m["flops"] / dur / 1e12
     return {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
             "frac": ach / peaks["bf16_tflops"], "traffic": None, "peak_kind": peaks_kind + " (burst)",
-            "kernel": "tree attention call (main kernel + combine)", "launch_us": dur * 1e6}
+            "kernel": "tree attention call (main kernel + combine)", "launch_us": dur * 1e6,
+            "frac_of_sustained": ach / peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]),
+            "frac_of_nominal": ach / NOMINAL_BF16_TFLOPS, "nominal_peak": NOMINAL_BF16_TFLOPS}
 
 
 def run_ours(args):
@@ -585,6 +589,13 @@ def run_ours(args):
 
     roof = roofline_entry(m, peaks, peaks_kind)
     roof["traffic"] = NCU_TRAFFIC_BYTES.get(w.name)
+    # the same call on ONE buffer set over and over: inputs stay in L2 (not the graded number)
+    b_warm = m["batches"][0]
+    g_warm = _graph_of(torch, lambda: [b_warm.attention() for _ in range(20)])
+    g_warm.replay()
+    torch.cuda.synchronize()
+    warm_us = _time_replays(torch, g_warm, 20) / 400 * 1e3
+    del g_warm
 
     # ---- the other configs, same protocol, fewer steps (reported for context in `per_config`)
     per_config = []
@@ -648,7 +659,8 @@ def run_ours(args):
         "gpu_launches": m["launches_per_step"] * args.steps,
         "roofline": roof,
         "cpu_baseline": cpu_baseline,
-        "kernel_us": {"mask_build": m["mask_ms"] * 1e3, "attention_call": m["attn_ms"] * 1e3},
+        "kernel_us": {"mask_build": m["mask_ms"] * 1e3, "attention_call": m["attn_ms"] * 1e3,
+                      "attention_call_L2_resident": warm_us},
         "device_status": m["status"],
     }
     if per_config:
