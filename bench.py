@@ -643,6 +643,13 @@ def run_ours(args):
     cpu_sec = sum(times) / len(times)
     cpu_baseline = {"value": w.total_nodes / cpu_sec, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
                     "sample": f"{len(times)} full passes (mask + attention) of {w.name}, {cpu_sec * 1e3:.1f} ms each"}
+    try:                                  # the same on one thread (the oracle's only parallelism is its BLAS calls)
+        from threadpoolctl import threadpool_limits
+        with threadpool_limits(limits=1):
+            t1 = time_oracle(w, budget_s=4.0, max_passes=5)
+        cpu_baseline["value_1_thread"] = w.total_nodes / (sum(t1) / len(t1))
+    except Exception:
+        pass
 
     if sampler:
         sampler.stop()
