@@ -310,8 +310,10 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   // for every other role
   auto next_index = [&](int k) -> int {
     if (k == 0) return int(blockIdx.x);
-    mbar_wait(q_full + 8u * uint32_t((k - 1) & 7), uint32_t((k - 1) >> 3) & 1u, abort_flag, p.status);
-    return q_idx[(k - 1) & 7];
+    // a wait that ran out (the CTA is in its error state) ends the CTA's work: never index with a stale entry
+    if (!mbar_wait(q_full + 8u * uint32_t((k - 1) & 7), uint32_t((k - 1) >> 3) & 1u, abort_flag, p.status)) return -1;
+    const int idx = q_idx[(k - 1) & 7];
+    return idx < p.n_items_total ? idx : -1;
   };
   const int g = p.group_size;
 
