@@ -693,7 +693,8 @@ def run_ours(args):
 def run_profile(args):
     """A short eager run for profilers: no graphs, no timing, no oracle.  --profile-op step (default):
     mask build + attention of --config; sparse: DFS reorder + mask with tile sets + tile-skipping
-    attention on the 2048-token random tree; verify / construct: those kernels on small cases."""
+    attention on the 2048-token random tree; small_batch: the 8-request small-tree batch; verify /
+    construct: those kernels on small cases."""
     import torch
     from paper_2410_11744_b200 import build as _build
     _build.build()
@@ -710,6 +711,16 @@ def run_profile(args):
             batches[i % copies].step()
         torch.cuda.synchronize()
         info = {"workload": w.name, "copies": copies, "plan": first.plan.describe(), "status": int(first.status.item())}
+    elif args.profile_op == "small_batch":
+        # the first case of small_tree_batch_experiment: 8 requests x 32 heads x 4096 prefix keys x 64-node trees (554 MB)
+        rng = np.random.default_rng(workloads.MASTER_SEED + 77)
+        w = workloads.make_custom(1, 32, 32, 128, [4096] * 8, [workloads.greedy_tree(rng, 64, 8, 0.3) for _ in range(8)])
+        batches = [runner.DeviceBatch(w) for _ in range(2)]
+        for i in range(args.profile):
+            batches[i % 2].step()
+        torch.cuda.synchronize()
+        info = {"workload": "8 requests, 32 heads, prefix 4096, 64-node trees", "copies": 2,
+                "plan": batches[0].plan.describe(), "status": int(batches[0].status.item())}
     elif args.profile_op == "sparse":
         w = workloads.make_random_tree_case(2048)
         probe = runner.DeviceBatch(w)
@@ -766,7 +777,7 @@ def main():
     ap.add_argument("--no-per-config", action="store_true")
     ap.add_argument("--profile", type=int, default=0,
                     help="run only this many plain (eager) steps of --config and exit: the command to put under ncu")
-    ap.add_argument("--profile-op", default="step", choices=["step", "sparse", "verify", "construct"])
+    ap.add_argument("--profile-op", default="step", choices=["step", "sparse", "small_batch", "verify", "construct"])
     args = ap.parse_args()
     if args.profile > 0:
         return run_profile(args)

@@ -5,17 +5,22 @@
 //   warp 8     producer: streams 64-key K and V tiles through TMA into a 128-byte-swizzled
 //              shared-memory ring guarded by mbarriers;
 //   warp 9     issues S = Q K^T on the tensor cores (tcgen05.mma, M = 64, N = 64, both operands from
-//              shared memory) as soon as a stage's K tile has landed; every ring stage has a score
-//              buffer of its own in tensor memory, so the scores run ahead of the softmax;
+//              shared memory) as soon as a tile's K has landed and one of four score buffers in tensor
+//              memory is free, so the scores run ahead of the softmax;
+//   warp 10    issues O += P V on the tensor cores (M = 64, one product per 64-column panel of V) when a
+//              warp set has put the tile's probabilities into shared memory (over the K tile, which the
+//              score product has finished with), into that set's accumulator in tensor memory; the
+//              commit behind it frees the ring stage;
 //   warps 0-7  two sets of four compute warps (16 query rows per warp).  The sets take alternate key
-//              tiles: a warp reads its 16 x 64 scores with tcgen05.ld (the 16x256b shape returns them
-//              laid out like an mma.sync accumulator), applies the ancestor bitmask on tree tiles,
-//              runs the fp32 online softmax in the exp2 domain and accumulates O += P V with
-//              mma.sync.m16n8k16 (P stays in registers, V through ldmatrix.trans).  The per-tile code
+//              tiles: a warp reads its 16 x 64 scores with tcgen05.ld (with M = 64 accumulator row r
+//              lives in lane 32 (r / 16) + r % 16, and the 16x256b shape returns the rows laid out like
+//              an mma.sync accumulator), applies the ancestor bitmask on tree tiles and runs the fp32
+//              online softmax in the exp2 domain against a LAZY reference: the accumulator is rescaled
+//              (tcgen05.ld / st) only when a row maximum has grown by more than 2^8.  The per-tile code
 //              is a chain of dependent instructions, so one warp per scheduler leaves the SM mostly
 //              idle; two interleaved tiles per scheduler double the rate.  At the end of an item the
-//              sets swap column halves of their (O, m, l) through shared memory, thread to thread, and
-//              each finishes one half of the columns.
+//              sets exchange (m, l) through shared memory, each reads one half of the columns of both
+//              accumulators, folds them and finishes that half.
 // A CTA walks its list of work items; an item either writes final bf16 rows or an fp32 partial
 // (O, m, l) for the split-KV combine kernel.  In cluster mode (uniform small batches) the splits of
 // a query tile are the CTAs of one thread-block cluster and are merged on chip through distributed
@@ -32,8 +37,9 @@ constexpr int kComputeWarps = 4;                            // per warp set: 16 
 constexpr int kSets = 2;                                    // two sets take alternate key tiles
 constexpr int kProducerWarp = kSets * kComputeWarps;        // TMA
 constexpr int kMmaWarp = kProducerWarp + 1;                 // tcgen05.mma issuer for S = Q K^T
-constexpr int kThreads = (kSets * kComputeWarps + 2) * 32;
-constexpr int kBarExchFull = 2, kBarExchFree = 3, kBarRingIdle = 4;   // named barriers between the two warp sets
+constexpr int kPvWarp = kProducerWarp + 2;                  // tcgen05.mma issuer for O += P V
+constexpr int kThreads = (kSets * kComputeWarps + 3) * 32;
+constexpr int kBarExchFull = 2, kBarExchFree = 3;     // named barriers between the two warp sets
 
 template <int D>
 struct SmemLayout {
@@ -48,17 +54,6 @@ struct SmemLayout {
   static constexpr int kTotal = kExchMlOffset + kSets * kComputeWarps * 32 * 16;
   static constexpr int kTmemCols = 512;                  // one 64-column score buffer per ring stage (power of two)
 };
-
-__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
-}
-__device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
-                                         uint32_t b0, uint32_t b1) {
-  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
 
 // Byte offset of 16-byte chunk `chunk` (0 .. D/8-1) of row `row` inside a tile stored as 64-column
 // panels with the 128-byte TMA swizzle (chunk index XOR row mod 8 inside each 128-byte row).
@@ -109,6 +104,44 @@ __device__ __forceinline__ void tmem_ld_scores(uint32_t taddr, float (&s)[BN / 8
   }
 }
 
+// O += P V on the tensor cores as well: M = 64 rows, K = 64 keys in four 16-key steps, one product per
+// 64-column panel of V (N = 64).  P is a K-major operand (64 rows x 64 keys of bf16 = one 128-byte row each,
+// same layout as a Q or K panel); a V panel is an MN-major operand (keys x 64 columns, columns contiguous):
+// 8-key groups 1024 bytes apart.  (One N = D product whose operand hops from panel to panel through the
+// descriptor's leading-dimension offset gave wrong upper columns in every CTA but the first of a cluster;
+// per-panel products do not depend on that field.)
+template <int D>
+__host__ __device__ constexpr uint32_t idesc_pv() {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | (uint32_t(64 >> 3) << 17) | (uint32_t(BM >> 4) << 24);   // N = 64 per panel
+}
+constexpr int kSBufs = 4;                 // score buffers in tensor memory (64 columns each)
+constexpr float kRescaleThreshold = 8.f;  // log2 units: O is rescaled only when a row maximum grows by more
+
+// NJ 8-column groups of this warp's 16 accumulator rows (see tmem_ld_scores for the register layout)
+template <int NJ>
+__device__ __forceinline__ void tmem_ld_rows(uint32_t taddr, float (&v)[NJ][4]) {
+  static_assert(NJ == 8, "64 columns at a time");
+  tmem_ld_scores(taddr, v);
+}
+template <int NJ>
+__device__ __forceinline__ void tmem_st_rows(uint32_t taddr, const float (&v)[NJ][4]) {
+  static_assert(NJ == 8, "64 columns at a time");
+  uint32_t r[32];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    r[4 * j] = __float_as_uint(v[j][0]); r[4 * j + 1] = __float_as_uint(v[j][1]);
+    r[4 * j + 2] = __float_as_uint(v[j][2]); r[4 * j + 3] = __float_as_uint(v[j][3]);
+  }
+  asm volatile(
+      "tcgen05.st.sync.aligned.16x256b.x8.b32 [%0], "
+      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+        "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]),
+        "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]),
+        "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+
 }  // namespace
 
 template <int D>
@@ -128,9 +161,13 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   // barriers: full[kStages], empty[kStages], q_full, q_empty, src[8] (one per cluster peer), s_full[kStages]
   const uint32_t bar_full = s_bar, bar_empty = s_bar + 8 * kStages;
   const uint32_t bar_qfull = s_bar + 16 * kStages, bar_qempty = bar_qfull + 8, bar_src = bar_qempty + 8;
-  const uint32_t bar_sfull = bar_src + 64;
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::kBarOffset + 24 * kStages + 16 + 64);
-  volatile uint32_t* tmem_holder = reinterpret_cast<volatile uint32_t*>(smem + L::kBarOffset + 24 * kStages + 16 + 64 + 4);
+  // ... s_full[4] / s_free[4] (score buffers), p_ready[kStages] (P of the stage's tile is in shared memory),
+  // pv_done[2] (a set's last P V has completed), o_free (both output accumulators have been read out)
+  const uint32_t bar_sfull = bar_src + 64, bar_sfree = bar_sfull + 8 * kSBufs, bar_pready = bar_sfree + 8 * kSBufs;
+  const uint32_t bar_pvdone = bar_pready + 8 * kStages, bar_ofree = bar_pvdone + 16;
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::kBarOffset + 24 * kStages + 16 + 64 + 16 * kSBufs + 24);
+  volatile uint32_t* tmem_holder = reinterpret_cast<volatile uint32_t*>(smem + L::kBarOffset + 24 * kStages + 16 + 64 + 16 * kSBufs + 28);
+  static_assert(24 * kStages + 16 + 64 + 16 * kSBufs + 32 <= 512, "barrier area");
   float4* exch_ml = reinterpret_cast<float4*>(smem + L::kExchMlOffset);
 
   const int warp = threadIdx.x >> 5;
@@ -157,15 +194,23 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   // is still streaming K/V itself, and hands over through a ring stage once the ring is idle; a CTA
   // that does not merge receives nothing (it is the one with the most tiles).
   const bool merge_owner = p.cluster_size > 1 && ((uint32_t(my_items[0].merge_owners) >> cluster_ctarank()) & 1u);
-  float4* exch_o = reinterpret_cast<float4*>(smem + L::kQBytes + (merge_owner ? 2 : kStages - 1) * L::kStageBytes);
-  const int n_stages = merge_owner ? kStages - 2 : kStages - 1;
+  const int n_stages = merge_owner ? kStages - 2 : kStages;
+  // tensor memory: O of set 0, O of set 1 (D columns each), then the score buffers
+  const uint32_t kOCols = D, kSCol0 = 2 * D;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
       mbar_init(bar_full + 8 * s, 1);
-      mbar_init(bar_empty + 8 * s, kComputeWarps);
-      mbar_init(bar_sfull + 8 * s, 1);
+      mbar_init(bar_empty + 8 * s, 1);                  // the commit behind the tile's P V
+      mbar_init(bar_pready + 8 * s, kComputeWarps);
     }
+    for (int b = 0; b < kSBufs; ++b) {
+      mbar_init(bar_sfull + 8 * b, 1);
+      mbar_init(bar_sfree + 8 * b, kComputeWarps);
+    }
+    mbar_init(bar_pvdone, 1);
+    mbar_init(bar_pvdone + 8, 1);
+    mbar_init(bar_ofree, kSets * kComputeWarps);
     mbar_init(bar_qfull, 1);
     mbar_init(bar_qempty, 1);                    // arrived on by the commit behind an item's last Q K^T
     for (int k = 0; k < 8; ++k) mbar_init(bar_src + 8 * k, 1);
@@ -220,33 +265,72 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     if (p.cluster_size > 1) cluster_wait();      // pairs with the arrive above (all threads of the cluster take part)
   } else if (warp == kMmaWarp) {
     // ------------------------------------------------------------------ S = Q K^T on the tensor cores (one lane issues)
-    // Ring stage s has a score buffer of its own (TMEM columns 64 s ..): as soon as the stage's K tile
-    // has landed its scores are computed, so they run ahead of the softmax by the depth of the ring.
-    // The buffer is free again when the stage is (the compute warps release the stage after they have
-    // read the scores and used V), so no barrier of its own guards it.
+    // Issued as soon as a tile's K has landed and one of the four score buffers is free, i.e. the scores
+    // run ahead of the softmax.  The products O += P V have an issuing warp of their own (below), so that
+    // neither stream of hand-offs waits for the other.
     if (lane == 0) {
-      int ring_stage = 0;
-      uint32_t ring_phase = 0;
       uint32_t qit = 0;
+      int n_base = 0;                      // key tiles of earlier items (ring / score-buffer position)
       const uint32_t q_lo = desc_lo(s_q);
       for (int w = item_begin; w < item_end; ++w, ++qit) {
         const WorkItem item = my_items[w];
+        const int T = item.tile_end - item.tile_begin;
         mbar_wait(bar_qfull, qit & 1, abort_flag, p.status);
-        for (int t = item.tile_begin; t < item.tile_end; ++t) {
-          const int stage = ring_stage;
-          const uint32_t ph = ring_phase;
-          if (++ring_stage == n_stages) { ring_stage = 0; ring_phase ^= 1u; }
+        for (int i = 0; i < T; ++i) {
+          const int pos = n_base + i;
+          const int stage = pos % n_stages;
+          const uint32_t ph = uint32_t(pos / n_stages) & 1u;
+          const int sb = pos & (kSBufs - 1), sb_use = pos / kSBufs;
           mbar_wait(bar_full + 8 * stage, ph, abort_flag, p.status);
+          if (sb_use > 0) mbar_wait(bar_sfree + 8 * sb, uint32_t(sb_use - 1) & 1u, abort_flag, p.status);
           tc_fence_after();
           const uint32_t k_lo = desc_lo(s_kv + stage * L::kStageBytes);
 #pragma unroll
           for (int ks = 0; ks < KS; ++ks) {
             const uint32_t off = uint32_t((ks >> 2) * L::kPanelBytes + (ks & 3) * 32) >> 4;   // Q and K panels have the same size
-            umma_ss(tmem_base + uint32_t(stage) * BN, q_lo + off, k_lo + off, kDescHi, kIdescQK, ks > 0 ? 1u : 0u);
+            umma_ss(tmem_base + kSCol0 + uint32_t(sb) * BN, q_lo + off, k_lo + off, kDescHi, kIdescQK, ks > 0 ? 1u : 0u);
           }
-          tc_commit(bar_sfull + 8 * stage);
+          tc_commit(bar_sfull + 8 * sb);
         }
         tc_commit(bar_qempty);                    // the Q tile may be replaced once these products are done
+        n_base += T;
+      }
+    }
+    if (p.cluster_size > 1) cluster_wait();
+  } else if (warp == kPvWarp) {
+    // ------------------------------------------------------------------ O += P V on the tensor cores (one lane issues)
+    // When a warp set has put a tile's P into shared memory (where the K tile was), into the set's own
+    // accumulator; the commit behind it frees the tile's ring stage.  An item's first products wait until
+    // the previous item's outputs have been read out of the accumulators.
+    if (lane == 0) {
+      uint32_t qit = 0;
+      int n_base = 0;
+      constexpr uint32_t kIdescPV = idesc_pv<D>();
+      for (int w = item_begin; w < item_end; ++w, ++qit) {
+        const WorkItem item = my_items[w];
+        const int T = item.tile_end - item.tile_begin;
+        for (int m = 0; m < T; ++m) {
+          const int pos = n_base + m;
+          const int stage = pos % n_stages;
+          const uint32_t ph = uint32_t(pos / n_stages) & 1u;
+          const int pv_set = m & 1;
+          mbar_wait(bar_pready + 8 * stage, ph, abort_flag, p.status);
+          if (m < 2 && qit > 0) mbar_wait(bar_ofree, (qit - 1) & 1u, abort_flag, p.status);   // first product into this accumulator
+          tc_fence_after();
+          const uint32_t p_lo = desc_lo(s_kv + stage * L::kStageBytes);                        // P sits where the K tile was
+          const uint32_t v_lo = desc_lo(s_kv + stage * L::kStageBytes + L::kTileBytes);
+          // one product per 64-column panel of V (N = 64 each): no leading-dimension hop inside an operand
+#pragma unroll
+          for (int h = 0; h < L::kHalves; ++h)
+#pragma unroll
+            for (int kk = 0; kk < BN / 16; ++kk)
+              umma_ss(tmem_base + uint32_t(pv_set) * kOCols + uint32_t(h) * 64u, p_lo + uint32_t(kk) * (32u >> 4),
+                      v_lo + uint32_t(h) * (uint32_t(L::kPanelBytes) >> 4) + uint32_t(kk) * (2048u >> 4), kDescHi, kIdescPV,
+                      (m >= 2 || kk > 0) ? 1u : 0u);
+          tc_commit(bar_empty + 8 * stage);
+          tc_commit(bar_pvdone + 8 * pv_set);
+        }
+        n_base += T;
       }
     }
     if (p.cluster_size > 1) cluster_wait();
@@ -265,8 +349,21 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   const int cw = warp & 3;        // row block inside the set
   const int wrow = cw * 16;
   const int ctid = cw * 32 + lane;   // thread index inside the set
-  int ring_stage = 0;
-  uint32_t ring_phase = 0, qit = 0;
+  int n_base = 0;                 // key tiles of earlier items (ring / score-buffer position)
+  int n_pv = 0;                   // P V products of this set so far (one phase of its pv_done barrier each)
+  int pv_seen = 0;                // phases of that barrier this thread has seen complete
+  // A parity wait only tells the barrier's current phase from the one before it, so a thread must never
+  // fall two phases behind: every tile first confirms the product of the set's PREVIOUS tile (issued
+  // right after this tile's scores, i.e. long done; one probe) before it lets the next one be issued.
+  // Afterwards every product of this set issued so far has landed.
+  auto confirm_pv_done = [&]() {
+    if (pv_seen < n_pv) {
+      mbar_wait(bar_pvdone + 8 * set, uint32_t(pv_seen) & 1u, abort_flag, p.status);
+      ++pv_seen;
+    }
+    tc_fence_after();
+  };
+  uint32_t qit = 0;
 
   for (int w = item_begin; w < item_end; ++w, ++qit) {
     const WorkItem item = my_items[w];
@@ -287,27 +384,32 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       if (ok_hi) pre_hi = __ldg(reinterpret_cast<const uint2*>(p.bits + size_t(rq.node0 + node_hi) * p.words_per_row));
     }
 
-    float o[DT][4];
-#pragma unroll
-    for (int j = 0; j < DT; ++j) { o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f; }
-    float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;
+    float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;   // m: the reference the accumulator is scaled to
+    const int T_item = item.tile_end - item.tile_begin;
+    const uint32_t t_rows = tmem_base + (uint32_t(cw * 32) << 16);         // this warp's 16 accumulator rows
+    const uint32_t t_o = t_rows + uint32_t(set) * kOCols;                    // this set's output accumulator
+    bool first = true;
 
-    for (int t = item.tile_begin; t < item.tile_end; ++t) {
-      const int stage = ring_stage;
-      const uint32_t ph = ring_phase;
-      if (++ring_stage == n_stages) { ring_stage = 0; ring_phase ^= 1u; }
-      if (((t - item.tile_begin) & 1) != set) continue;     // the other set's tile
+    for (int i = set; i < T_item; i += kSets) {
+      const int t = item.tile_begin + i;
+      const int pos = n_base + i;
+      const int stage = pos % n_stages;
+      const uint32_t ph = uint32_t(pos / n_stages) & 1u;
+      const int sb = pos & (kSBufs - 1);
       const uint32_t s_k = s_kv + stage * L::kStageBytes;
       const uint32_t s_v = s_k + L::kTileBytes;
-      // ---- S = Q K^T (16 x 64 per warp) from the stage's score buffer.  The stage's own barrier is
-      //      complete by then (the products were issued behind it); waiting on it as well costs one
-      //      probe and makes the TMA-written V tile visible to this thread.
-      mbar_wait(bar_sfull + 8 * stage, ph, abort_flag, p.status);
+      // ---- S = Q K^T (16 x 64 per warp) from the tile's score buffer; the stage's own barrier is complete
+      //      by then (the products were issued behind it), waiting on it as well makes the TMA-written V
+      //      tile visible to this thread.
+      mbar_wait(bar_sfull + 8 * sb, uint32_t(pos / kSBufs) & 1u, abort_flag, p.status);
       mbar_wait(bar_full + 8 * stage, ph, abort_flag, p.status);
       tc_fence_after();
       if (threadIdx.x == 0 && w == item_begin && t == item.tile_begin) stamp(3);
       float s[BN / 8][4];
-      tmem_ld_scores(tmem_base + (uint32_t(cw * 32) << 16) + uint32_t(stage) * BN, s);
+      tmem_ld_scores(t_rows + kSCol0 + uint32_t(sb) * BN, s);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_sfree + 8 * sb);        // the buffer may take the scores of a later tile
 
       // ---- visibility of the 64 key columns for this thread's two rows
       uint64_t vis_lo, vis_hi;
@@ -330,7 +432,10 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         vis_hi = (uint64_t(w_hi.y) << 32) | w_hi.x;
       }
 
-      // ---- online softmax (exp2 domain)
+      // ---- online softmax (exp2 domain) against a LAZY reference: the accumulator lives in tensor memory, so
+      //      it is rescaled only when some row's maximum has grown by more than 2^8 since the reference was
+      //      set (probabilities then stay below 2^8, harmless in bf16 and fp32; the final normalisation
+      //      uses the same reference).
       float mx_lo = -INFINITY, mx_hi = -INFINITY;
 #pragma unroll
       for (int j = 0; j < BN / 8; ++j) {
@@ -347,12 +452,29 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 1));
       mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 2));
       const float mn_lo = fmaxf(m_lo, mx_lo), mn_hi = fmaxf(m_hi, mx_hi);
+      confirm_pv_done();
+      if (first) {
+        m_lo = mn_lo; m_hi = mn_hi;
+      } else if (__any_sync(0xffffffffu, mn_lo > m_lo + kRescaleThreshold || mn_hi > m_hi + kRescaleThreshold)) {
+        // O *= 2^(m - mn) for this warp's rows (every product of this set issued so far has landed)
+        const float f_lo = fast_exp2(m_lo - (mn_lo == -INFINITY ? 0.f : mn_lo));
+        const float f_hi = fast_exp2(m_hi - (mn_hi == -INFINITY ? 0.f : mn_hi));
+#pragma unroll 1
+        for (int c0 = 0; c0 < D; c0 += 64) {
+          float ov[8][4];
+          tmem_ld_rows<8>(t_o + uint32_t(c0), ov);
+#pragma unroll
+          for (int j = 0; j < 8; ++j) { ov[j][0] *= f_lo; ov[j][1] *= f_lo; ov[j][2] *= f_hi; ov[j][3] *= f_hi; }
+          tmem_st_rows<8>(t_o + uint32_t(c0), ov);
+        }
+        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+        l_lo *= f_lo; l_hi *= f_hi;
+        m_lo = mn_lo; m_hi = mn_hi;
+      }
       // A row that has seen no visible key yet keeps m = -inf; use 0 as the reference so that
       // exp2(-inf - 0) = 0 and no inf - inf appears.
-      const float ref_lo = mn_lo == -INFINITY ? 0.f : mn_lo;
-      const float ref_hi = mn_hi == -INFINITY ? 0.f : mn_hi;
-      const float a_lo = fast_exp2(m_lo - ref_lo), a_hi = fast_exp2(m_hi - ref_hi);
-      m_lo = mn_lo; m_hi = mn_hi;
+      const float ref_lo = m_lo == -INFINITY ? 0.f : m_lo;
+      const float ref_hi = m_hi == -INFINITY ? 0.f : m_hi;
       float sum_lo = 0.f, sum_hi = 0.f;
       uint32_t pf[BN / 8][2];
 #pragma unroll
@@ -364,10 +486,8 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         pf[j][0] = pack_bf16x2(p0, p1);
         pf[j][1] = pack_bf16x2(p2, p3);
       }
-      l_lo = l_lo * a_lo + sum_lo;
-      l_hi = l_hi * a_hi + sum_hi;
-#pragma unroll
-      for (int j = 0; j < DT; ++j) { o[j][0] *= a_lo; o[j][1] *= a_lo; o[j][2] *= a_hi; o[j][3] *= a_hi; }
+      l_lo += sum_lo;
+      l_hi += sum_hi;
 
       // ---- V rows past the end of the request are not ours (another request's rows, or memory the
       //      caller never wrote): zero them so that 0 * garbage cannot produce NaN (their probabilities
@@ -381,23 +501,24 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         __syncwarp();
       }
 
-      // ---- O += P V
+      // ---- P (bf16) into the stage's K region, which the score product has finished reading: 64 rows of 128
+      //      bytes with the same swizzle as a K panel, so that the tensor core reads it as a K-major operand
+      {
+        const int r_lo_ = wrow + gid, r_hi_ = r_lo_ + 8;
 #pragma unroll
-      for (int kk = 0; kk < BN / 16; ++kk) {
-#pragma unroll
-        for (int jd = 0; jd < DT / 2; ++jd) {
-          const int mi = lane >> 3;
-          const int row = kk * 16 + (lane & 7) + ((mi & 1) << 3);
-          const int chunk = jd * 2 + (mi >> 1);
-          uint32_t b0, b1, b2, b3;
-          ldmatrix_x4_trans(s_v + swz(row, chunk, L::kPanelBytes), b0, b1, b2, b3);
-          mma_bf16(o[2 * jd], pf[2 * kk][0], pf[2 * kk][1], pf[2 * kk + 1][0], pf[2 * kk + 1][1], b0, b1);
-          mma_bf16(o[2 * jd + 1], pf[2 * kk][0], pf[2 * kk][1], pf[2 * kk + 1][0], pf[2 * kk + 1][1], b2, b3);
+        for (int j = 0; j < BN / 8; ++j) {
+          asm volatile("st.shared.b32 [%0], %1;" ::"r"(s_k + uint32_t(r_lo_ * 128 + ((j ^ (r_lo_ & 7)) << 4) + tig * 4)), "r"(pf[j][0]) : "memory");
+          asm volatile("st.shared.b32 [%0], %1;" ::"r"(s_k + uint32_t(r_hi_ * 128 + ((j ^ (r_hi_ & 7)) << 4) + tig * 4)), "r"(pf[j][1]) : "memory");
         }
       }
+      fence_proxy_async();        // the tensor core reads P (and the zeroed V rows) through the async proxy
+      tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar_empty + 8 * stage);
+      if (lane == 0) mbar_arrive(bar_pready + 8 * stage);
+      ++n_pv;
+      first = false;
     }
+    n_base += T_item;
 
     // ---- epilogue
     if (threadIdx.x == 0 && w == item_begin) stamp(5);
@@ -406,46 +527,49 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1);
     l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
 
-    // ---- the two warp sets took alternate tiles and thread ctid of either set owns the same rows and
-    //      column pairs.  They swap halves: set 0 gives away its right half of the columns (D/2 ..) and
-    //      receives set 1's left half, and the other way round, so that afterwards each set holds the
-    //      merged values of ONE half (moved to o[0 .. DT/2)) and both run every later step (parking,
-    //      storing) on half the columns each.  (m, l) are merged identically on both sides.
+    // ---- the two warp sets took alternate tiles into accumulators of their own.  They exchange (m, l)
+    //      through shared memory, then each set reads ONE half of the columns of BOTH accumulators (thread
+    //      ctid of either set owns the same rows and column pairs), folds them and runs every later step
+    //      (parking, storing) on that half.
     constexpr int HT = DT / 2;                    // 8-column tiles per half
     constexpr int kAll = kSets * kComputeWarps * 32;
-    if (merge_owner)              // the hand-over buffer is a ring stage here: both sets must be done with the ring
-      asm volatile("bar.sync %0, %1;" ::"n"(kBarRingIdle), "n"(kAll) : "memory");
+    const int my_tiles = (T_item - set + kSets - 1) / kSets, other_tiles = (T_item - (1 - set) + kSets - 1) / kSets;
+    confirm_pv_done();                            // this set's last product has landed
+    tc_fence_before();
     if (w != item_begin)          // both sets have read the previous item's values
       asm volatile("bar.sync %0, %1;" ::"n"(kBarExchFree), "n"(kAll) : "memory");
+    exch_ml[set * (kComputeWarps * 32) + ctid] = make_float4(m_lo, m_hi, l_lo, l_hi);
+    asm volatile("bar.sync %0, %1;" ::"n"(kBarExchFull), "n"(kAll) : "memory");   // also: the other set's products have landed
+    tc_fence_after();
+    const int cbase = set * (D / 2);              // first column of this set's half
+    float o[HT][4];
     {
-      float4* give = exch_o + set * (HT * kComputeWarps * 32);
-      const float4* take = exch_o + (1 - set) * (HT * kComputeWarps * 32);
-      if (set == 0) {
-#pragma unroll
-        for (int j = 0; j < HT; ++j) give[j * (kComputeWarps * 32) + ctid] = make_float4(o[HT + j][0], o[HT + j][1], o[HT + j][2], o[HT + j][3]);
-      } else {
-#pragma unroll
-        for (int j = 0; j < HT; ++j) give[j * (kComputeWarps * 32) + ctid] = make_float4(o[j][0], o[j][1], o[j][2], o[j][3]);
-#pragma unroll
-        for (int j = 0; j < HT; ++j) { o[j][0] = o[HT + j][0]; o[j][1] = o[HT + j][1]; o[j][2] = o[HT + j][2]; o[j][3] = o[HT + j][3]; }
-      }
-      exch_ml[set * (kComputeWarps * 32) + ctid] = make_float4(m_lo, m_hi, l_lo, l_hi);
-      asm volatile("bar.sync %0, %1;" ::"n"(kBarExchFull), "n"(kAll) : "memory");
       const float4 ml = exch_ml[(1 - set) * (kComputeWarps * 32) + ctid];
       const float mn_lo = fmaxf(m_lo, ml.x), mn_hi = fmaxf(m_hi, ml.y);
       const float ref_lo = mn_lo == -INFINITY ? 0.f : mn_lo, ref_hi = mn_hi == -INFINITY ? 0.f : mn_hi;
       const float ka_lo = fast_exp2(m_lo - ref_lo), kb_lo = fast_exp2(ml.x - ref_lo);
       const float ka_hi = fast_exp2(m_hi - ref_hi), kb_hi = fast_exp2(ml.y - ref_hi);
+      static_assert(HT == 8 || HT == 4, "half of the columns: 64 or 32");
+      float mine[8][4], theirs[8][4];
+      // (D = 64: a half is 32 columns; the loads fetch 64 and the upper 32 are ignored -- they belong to the
+      //  neighbouring buffer, which is mapped, so this is safe)
+      if (my_tiles > 0) tmem_ld_rows<8>(t_rows + uint32_t(set) * kOCols + uint32_t(cbase), mine);
+      if (other_tiles > 0) tmem_ld_rows<8>(t_rows + uint32_t(1 - set) * kOCols + uint32_t(cbase), theirs);
 #pragma unroll
       for (int j = 0; j < HT; ++j) {
-        const float4 ob = take[j * (kComputeWarps * 32) + ctid];
-        o[j][0] = o[j][0] * ka_lo + ob.x * kb_lo; o[j][1] = o[j][1] * ka_lo + ob.y * kb_lo;
-        o[j][2] = o[j][2] * ka_hi + ob.z * kb_hi; o[j][3] = o[j][3] * ka_hi + ob.w * kb_hi;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float a_ = my_tiles > 0 ? mine[j][e] * (e < 2 ? ka_lo : ka_hi) : 0.f;
+          const float b_ = other_tiles > 0 ? theirs[j][e] * (e < 2 ? kb_lo : kb_hi) : 0.f;
+          o[j][e] = a_ + b_;
+        }
       }
       l_lo = l_lo * ka_lo + ml.z * kb_lo; l_hi = l_hi * ka_hi + ml.w * kb_hi;
       m_lo = mn_lo; m_hi = mn_hi;
     }
-    const int cbase = set * (D / 2);              // first column of this set's half
+    tc_fence_before();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bar_ofree);        // the accumulators may take the next item's products
     if (threadIdx.x == 0 && w == item_begin) stamp(1);
     if (p.cluster_size > 1) {
       // ---- split-KV combine inside a thread-block cluster: the CTAs of a cluster hold the splits of

@@ -258,3 +258,25 @@ def test_mask_builder_batched_without_a_plan(rt):
     assert np.array_equal(depths.cpu().numpy(), ref_depths)
     with pytest.raises(B.DyspecError):
         B.dyspec_build_tree_mask_batched(parents, [0, 5, 3], bits, depths, W, None)     # offsets must not decrease
+
+
+@pytest.mark.parametrize("hq,hkv,n,L", [(4, 4, 40, 500), (8, 1, 8, 700), (16, 2, 100, 600), (32, 32, 64, 1024)])
+def test_growing_maxima_exercise_the_lazy_rescale(rt, hq, hkv, n, L):
+    """Keys whose scores grow steadily along the sequence (by tens of log2 units in all): both kernels keep
+    their running output in tensor memory against a lazy reference and rescale it only when a row maximum
+    has grown by more than 2^8, which random N(0,1) inputs never do.  Here they must, several times."""
+    rng = np.random.default_rng(hq * 1000 + n)
+    w = wl.make_custom(70 + n, hq, hkv, 128, [L], [wl.greedy_tree(rng, n, 6, 0.3)])
+    pattern = np.where(rng.random(128) < 0.5, -1.0, 1.0)
+    q = pattern[None, None, :] * (1.0 + 0.1 * rng.standard_normal((n, hq, 1))) + 0.05 * rng.standard_normal((n, hq, 128))
+    rows = w.k.shape[0]
+    ramp = (0.02 + 2.0 * np.arange(rows) / rows)[:, None, None]           # |score| grows ~ 30 log2 units over the cache
+    k = pattern[None, None, :] * ramp + 0.05 * rng.standard_normal((rows, hkv, 128))
+    def to_bits(x):
+        u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)
+        return ((u + 0x7FFF + ((u >> 16) & 1)) >> 16).astype(np.uint16)
+    w.q[...] = to_bits(q)
+    w.k[...] = to_bits(k)
+    for regime in (0, 1) if n * (hq // hkv) <= 64 else (1,):
+        run_and_check(rt, w, regime=regime)
+    run_and_check(rt, w)
