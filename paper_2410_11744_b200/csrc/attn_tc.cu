@@ -20,7 +20,7 @@
 //   warps 8-11    the same for query half B.  The two halves alternate on the tensor pipe, so one
 //                 half's softmax overlaps the other half's MMAs, and each K/V tile is loaded once
 //                 for 256 query rows.
-// Every wait is bounded (see mbar_wait); nothing here uses TMA multicast or clusters.
+// Every wait is bounded (see mbar_wait); every TMA load goes to this CTA alone, and the kernel is never launched in clusters.
 #include "common.cuh"
 
 namespace dyspec {

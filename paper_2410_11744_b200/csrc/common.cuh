@@ -239,7 +239,7 @@ __device__ __forceinline__ bool counter_wait(uint32_t addr, uint32_t target, vol
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void trigger_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
-// Thread-block cluster helpers (distributed shared memory; no multicast is used anywhere).
+// Thread-block cluster helpers (distributed shared memory; every copy has exactly one destination CTA).
 __device__ __forceinline__ uint32_t cluster_ctarank() {
   uint32_t r;
   asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
@@ -255,7 +255,7 @@ __device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster
 __device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
 // Asynchronous copy of `bytes` (a multiple of 16; both addresses 16-byte aligned) from this CTA's
 // shared memory into a peer CTA's; the peer's mbarrier receives the byte count when the data has
-// landed.  dst and bar are shared::cluster addresses (see map_to_cta).  Not a multicast.
+// landed.  dst and bar are shared::cluster addresses (see map_to_cta).  One destination CTA.
 __device__ __forceinline__ void dsmem_push(uint32_t dst_cluster_addr, uint32_t src_local_addr, uint32_t bytes,
                                            uint32_t bar_cluster_addr) {
   asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
@@ -286,7 +286,7 @@ __device__ __forceinline__ float2 ld_dsmem_f32x2(uint32_t addr) {
   return v;
 }
 
-// TMA: 3-D tiled load global -> shared, completion on an mbarrier (no multicast anywhere).
+// TMA: 3-D tiled load global -> shared, completion on an mbarrier (destination: this CTA only).
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
   asm volatile(
       "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
