@@ -1,0 +1,75 @@
+"""GPU parity on randomly drawn small batches: head grouping, head size, prefix lengths around the tile
+boundaries, tree shapes and sizes on both sides of the regime boundary, empty requests, forced CTA counts
+and both ways of merging split-KV partials; every case runs twice on the same buffers and is compared
+with the oracle element by element."""
+import numpy as np
+import pytest
+
+from oracle import dyspec_oracle as orc
+from paper_2410_11744_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+MAX_ABS, MEAN_ABS = 2e-2, 2e-3
+
+
+@pytest.fixture(scope="module")
+def rt():
+    import torch
+    assert torch.cuda.is_available()
+    from paper_2410_11744_b200 import build
+    build.build()
+    from paper_2410_11744_b200 import binding, runner
+    return binding, runner
+
+
+def _draw(rng, index):
+    g = int(rng.choice([1, 2, 4, 8]))
+    hkv = int(rng.choice([1, 2, 4]))
+    d = int(rng.choice([64, 128]))
+    n_req = int(rng.integers(1, 6))
+    Ls = [int(x) for x in rng.choice([0, 1, 5, 63, 64, 65, 127, 128, 129, 200, 500, 900], n_req)]
+    max_n = 64 // g if rng.random() < 0.6 else 300
+    trees = []
+    for _ in range(n_req):
+        n = int(rng.integers(0, max_n + 1))
+        kind = int(rng.integers(0, 4))
+        if n == 0:
+            trees.append(np.zeros(0, np.int32))
+        elif kind == 0:
+            trees.append(wl.chain_tree(n))
+        elif kind == 1:
+            trees.append(wl.star_forest(n))
+        elif kind == 2:
+            trees.append(wl.random_tree(rng, n))
+        else:
+            trees.append(wl.greedy_tree(rng, n, 4, 0.3))
+    w = wl.make_custom(9000 + index, hkv * g, hkv, d, Ls, trees)
+    return w, int(rng.choice([0, 0, 0, 1, 3, 7, 148])), int(rng.choice([2, 2, 0]))
+
+
+@pytest.mark.parametrize("seed", [11, 12, 13])
+def test_random_small_batches(rt, seed):
+    B, R = rt
+    rng = np.random.default_rng(seed)
+    for index in range(24):
+        w, ctas, combine = _draw(rng, 100 * seed + index)
+        B.dyspec_set_tuning(-1, ctas, combine)
+        try:
+            batch = R.DeviceBatch(w)
+        finally:
+            B.dyspec_set_tuning(-1, 0, 2)
+        for _ in range(2):
+            batch.step()
+        bits, depths, out_bits, status = batch.results()
+        what = dict(heads=(w.n_q_heads, w.n_kv_heads), d=w.head_dim, L=w.prefix_len.tolist(), n=w.n_nodes.tolist(),
+                    ctas=ctas, combine=combine, plan=batch.plan.describe())
+        assert status == 0, what
+        ref_bits, ref_depths = orc.build_tree_mask_ragged(w.parents, batch.W)
+        assert np.array_equal(bits, ref_bits) and np.array_equal(depths, ref_depths), what
+        ref = orc.tree_attention_ragged(w.q, w.k, w.v, w.prefix_len, w.n_nodes, w.kv_row_offset, w.parents)
+        if ref.size:
+            got = orc.bf16_bits_to_f64(out_bits)
+            assert np.isfinite(got).all(), what
+            err = np.abs(got - ref)
+            assert err.max() <= MAX_ABS and err.mean() <= MEAN_ABS, (what, err.max(), err.mean())
