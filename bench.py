@@ -643,6 +643,21 @@ def run_ours(args):
     cpu_sec = sum(times) / len(times)
     cpu_baseline = {"value": w.total_nodes / cpu_sec, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
                     "sample": f"{len(times)} full passes (mask + attention) of {w.name}, {cpu_sec * 1e3:.1f} ms each"}
+    # parity of the timed configuration against the oracle (whole output, one more oracle pass)
+    parity = None
+    try:
+        from oracle import dyspec_oracle as orc
+        b_par = m["batches"][0]
+        b_par.step()
+        bits_g, depths_g, out_g, st_g = b_par.results()
+        ref_bits, ref_depths = orc.build_tree_mask_ragged(w.parents, b_par.W)
+        ref = orc.tree_attention_ragged(w.q, w.k, w.v, w.prefix_len, w.n_nodes, w.kv_row_offset, w.parents)
+        err = np.abs(orc.bf16_bits_to_f64(out_g) - ref)
+        parity = {"mask_bit_exact": bool(np.array_equal(bits_g, ref_bits)), "depths_exact": bool(np.array_equal(depths_g, ref_depths)),
+                  "attention_max_abs_err": float(err.max()), "attention_mean_abs_err": float(err.mean()),
+                  "tolerance": {"max_abs": 2e-2, "mean_abs": 2e-3}, "device_status": st_g}
+    except Exception as e:                # the measurement stands without it
+        parity = {"error": repr(e)}
     try:                                  # the same on one thread (the oracle's only parallelism is its BLAS calls)
         from threadpoolctl import threadpool_limits
         with threadpool_limits(limits=1):
@@ -669,6 +684,7 @@ def run_ours(args):
         "kernel_us": {"mask_build": m["mask_ms"] * 1e3, "attention_call": m["attn_ms"] * 1e3,
                       "attention_call_L2_resident": warm_us},
         "device_status": m["status"],
+        "parity_vs_oracle": parity,
     }
     if per_config:
         line["per_config"] = per_config
