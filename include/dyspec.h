@@ -92,7 +92,9 @@ int dyspec_build_tree_mask_batched(const int32_t* parents, const int32_t* node_o
  * (2) Plans.  A plan fixes the static shape and the ragged batch structure, runs the host-side
  * scheduler (work list of (request, kv-head, query-tile, kv-split) items balanced over the SMs)
  * and owns a small device copy of that list.  Create it once per batch structure; reuse it for
- * every layer and step with the same (prefix_len, n_nodes).
+ * every layer and step with the same (prefix_len, n_nodes).  A plan belongs to the CUDA device that
+ * is current when it is created: the attention calls return DYSPEC_ERR_INVALID_ARG when another
+ * device is current.
  *
  *   n_q_heads, n_kv_heads  H_q, H_kv; group g = H_q / H_kv must be 1, 2, 4 or 8
  *   head_dim               64 or 128
@@ -192,8 +194,10 @@ int dyspec_tree_attention_ragged(const dyspec_plan_t* plan, const void* q, const
 /*
  * (3b) Single-request convenience form.  The static shape comes from dyspec_set_default_shape;
  * plans and workspaces for each (prefix_len, n_nodes) seen are created on first use and cached
- * inside the library (that first call allocates; later calls do not).  k_cache / v_cache hold
- * exactly prefix_len + n_nodes rows.
+ * inside the library, per device (that first call allocates; later calls do not).  k_cache / v_cache
+ * hold exactly prefix_len + n_nodes rows.  Calls of one shape share one cached workspace, so they must
+ * follow each other on the GPU (one stream, or streams ordered by events); use the ragged form with
+ * workspaces of your own for calls that may overlap.
  */
 int dyspec_set_default_shape(int n_q_heads, int n_kv_heads, int head_dim, int words_per_row, float scale);
 int dyspec_tree_attention(const void* q, const void* k_cache, const void* v_cache, int prefix_len,

@@ -123,6 +123,7 @@ struct dyspec_plan {
   int64_t total_tiles = 0, n_groups = 0;
   // device copies (one allocation)
   void* d_blob = nullptr;
+  int device = -1;                      // the device the copies live on (the one current at creation)
   ReqInfo* d_reqs = nullptr;
   WorkItem* d_items = nullptr;
   GroupInfo* d_groups = nullptr;
@@ -412,6 +413,7 @@ int upload(dyspec_plan& pl) {
   if (!pl.split_groups.empty()) memcpy(host.data() + off, pl.split_groups.data(), pl.split_groups.size() * sizeof(GroupInfo));
   const size_t o_groups = off; off += b_groups;
   const size_t o_counters = off;
+  if (cudaGetDevice(&pl.device) != cudaSuccess) return DYSPEC_ERR_CUDA;
   if (cudaMalloc(&pl.d_blob, total) != cudaSuccess) { pl.d_blob = nullptr; return DYSPEC_ERR_CUDA; }
   if (cudaMemcpy(pl.d_blob, host.data(), total, cudaMemcpyHostToDevice) != cudaSuccess) return DYSPEC_ERR_CUDA;
   uint8_t* base = static_cast<uint8_t*>(pl.d_blob);
@@ -846,6 +848,9 @@ static int run_attention(const dyspec_plan_t* plan, const void* q, const void* k
   if (!q || !k_cache || !v_cache || !ancestor_bits || !out) return DYSPEC_ERR_INVALID_ARG;
   if (!aligned(q, 16) || !aligned(k_cache, 16) || !aligned(v_cache, 16) || !aligned(out, 16) || !aligned(ancestor_bits, 16))
     return DYSPEC_ERR_INVALID_ARG;
+  int dev = -1;                          // the plan's tables live on the device it was created on
+  if (cudaGetDevice(&dev) != cudaSuccess) return DYSPEC_ERR_CUDA;
+  if (dev != plan->device) return DYSPEC_ERR_INVALID_ARG;
   if (plan->workspace_bytes > 0 && (!workspace || workspace_bytes < plan->workspace_bytes || !aligned(workspace, 256)))
     return DYSPEC_ERR_WORKSPACE;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
@@ -887,7 +892,8 @@ namespace {
 struct DefaultShape { int hq = 0, hkv = 0, d = 0, W = 0; float scale = 0.f; };
 DefaultShape g_shape;
 struct Cached { dyspec_plan* plan; void* workspace; };
-std::map<std::tuple<int, int, int, int, int, int>, Cached> g_cache;
+// keyed by device, static shape, scale (bit pattern) and (prefix_len, n_nodes): a plan belongs to one device
+std::map<std::tuple<int, int, int, int, int, uint32_t, int, int>, Cached> g_cache;
 std::mutex g_cache_mutex;
 }  // namespace
 
@@ -904,11 +910,15 @@ int dyspec_set_default_shape(int n_q_heads, int n_kv_heads, int head_dim, int wo
 int dyspec_tree_attention(const void* q, const void* k_cache, const void* v_cache, int prefix_len,
                           const uint32_t* ancestor_bits, int n_nodes, void* out, dyspec_stream_t stream) {
   Cached c{};
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return DYSPEC_ERR_CUDA;
   {
     std::lock_guard<std::mutex> lock(g_cache_mutex);
     if (g_shape.hq == 0) return DYSPEC_ERR_INVALID_ARG;
     if (prefix_len < 0 || n_nodes < 0) return DYSPEC_ERR_INVALID_ARG;
-    const auto key = std::make_tuple(g_shape.hq, g_shape.hkv, g_shape.d, g_shape.W, prefix_len, n_nodes);
+    uint32_t scale_bits;
+    memcpy(&scale_bits, &g_shape.scale, 4);
+    const auto key = std::make_tuple(dev, g_shape.hq, g_shape.hkv, g_shape.d, g_shape.W, scale_bits, prefix_len, n_nodes);
     auto it = g_cache.find(key);
     if (it == g_cache.end()) {
       const int32_t L = prefix_len, n = n_nodes;

@@ -762,7 +762,7 @@ int attn_mma_threads() { return kThreads; }
 cudaError_t launch_attn_mma(int head_dim, int n_ctas, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                             const AttnParams& p, cudaStream_t stream) {
   const size_t smem = attn_mma_smem_bytes(head_dim);
-  static bool attr_set[2] = {false, false};
+  static DynSmemGrant grant[2];
   cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
@@ -778,19 +778,11 @@ cudaError_t launch_attn_mma(int head_dim, int n_ctas, const CUtensorMap& mq, con
   cfg.numAttrs = p.cluster_size > 1 ? 2 : 1;
   cudaError_t e = cudaSuccess;
   if (head_dim == 128) {
-    if (!attr_set[0]) {
-      cudaError_t e = cudaFuncSetAttribute(tree_attn_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
-      if (e != cudaSuccess) return e;
-      attr_set[0] = true;
-    }
+    if (cudaError_t ge = grant[0].ensure(tree_attn_mma_kernel<128>, smem); ge != cudaSuccess) return ge;
     cfg.dynamicSmemBytes = smem;
     e = cudaLaunchKernelEx(&cfg, tree_attn_mma_kernel<128>, mq, mk, mv, p);
   } else {
-    if (!attr_set[1]) {
-      cudaError_t e = cudaFuncSetAttribute(tree_attn_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
-      if (e != cudaSuccess) return e;
-      attr_set[1] = true;
-    }
+    if (cudaError_t ge = grant[1].ensure(tree_attn_mma_kernel<64>, smem); ge != cudaSuccess) return ge;
     cfg.dynamicSmemBytes = smem;
     e = cudaLaunchKernelEx(&cfg, tree_attn_mma_kernel<64>, mq, mk, mv, p);
   }

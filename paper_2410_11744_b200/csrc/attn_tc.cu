@@ -773,12 +773,8 @@ namespace {
 template <int D, bool kDyn>
 cudaError_t launch_one(cudaLaunchConfig_t& cfg, size_t smem, const CUtensorMap& mq, const CUtensorMap& mk,
                        const CUtensorMap& mv, const AttnParams& p) {
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(tree_attn_tc_kernel<D, kDyn>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static DynSmemGrant grant;           // one per instantiation
+  if (cudaError_t e = grant.ensure(tree_attn_tc_kernel<D, kDyn>, smem); e != cudaSuccess) return e;
   cfg.dynamicSmemBytes = smem;
   return cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<D, kDyn>, mq, mk, mv, p);
 }

@@ -5,6 +5,7 @@
 #include <cuda_bf16.h>
 #include <cuda.h>
 #include <stdint.h>
+#include <atomic>
 
 #include "../../include/dyspec.h"
 
@@ -92,6 +93,27 @@ struct AttnParams {
   // queue[1] counts the CTAs that found the queue empty, and the last of them clears both words.
   int32_t* queue;
   int32_t n_items_total;
+};
+
+// Dynamic shared memory above 48 KB has to be granted per (kernel, device).  One of these per kernel
+// remembers what each device of the process has been granted so far; safe to call from several
+// host threads (the worst case is a repeated, idempotent grant).
+struct DynSmemGrant {
+  static constexpr int kDevices = 64;
+  std::atomic<size_t> granted[kDevices];
+  template <typename Kernel>
+  cudaError_t ensure(Kernel kernel, size_t bytes) {
+    if (bytes <= 48 * 1024) return cudaSuccess;
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    const bool cached = dev >= 0 && dev < kDevices;
+    if (cached && granted[dev].load(std::memory_order_acquire) >= bytes) return cudaSuccess;
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(bytes));
+    if (e != cudaSuccess) return e;
+    if (cached) granted[dev].store(bytes, std::memory_order_release);
+    return cudaSuccess;
+  }
 };
 
 #ifdef __CUDACC__

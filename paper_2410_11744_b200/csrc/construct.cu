@@ -208,12 +208,8 @@ cudaError_t launch_build_tree_greedy(const float* draft_table, int n_rows, int v
                                      cudaStream_t stream) {
   if (n_req <= 0) return cudaSuccess;
   const size_t smem = build_tree_greedy_smem(m);
-  static size_t attr_smem = 48 * 1024;
-  if (smem > attr_smem) {
-    cudaError_t e = cudaFuncSetAttribute(build_tree_greedy_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
-    if (e != cudaSuccess) return e;
-    attr_smem = smem;
-  }
+  static DynSmemGrant grant;
+  if (cudaError_t e = grant.ensure(build_tree_greedy_kernel, smem); e != cudaSuccess) return e;
   TreeOut out{parents, tokens, values, child_values, rows};
   build_tree_greedy_kernel<<<n_req, kVThreads, smem, stream>>>(draft_table, n_rows, vocab, uniforms, n_uniforms, root_row, m,
                                                                out, n_nodes);

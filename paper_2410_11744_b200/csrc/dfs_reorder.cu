@@ -164,12 +164,8 @@ cudaError_t launch_dfs_reorder(const int32_t* parents, const ReqInfo* reqs, int 
                                cudaStream_t stream) {
   if (n_req <= 0 || max_n <= 0) return cudaSuccess;
   const size_t smem = dfs_reorder_smem_bytes(max_n);
-  static size_t attr_smem = 48 * 1024;
-  if (smem > attr_smem) {
-    cudaError_t e = cudaFuncSetAttribute(dfs_reorder_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
-    if (e != cudaSuccess) return e;
-    attr_smem = smem;
-  }
+  static DynSmemGrant grant;
+  if (cudaError_t e = grant.ensure(dfs_reorder_kernel, smem); e != cudaSuccess) return e;
   int threads = ((max_n + 31) / 32) * 32;
   if (threads < 128) threads = 128;
   if (threads > 1024) threads = 1024;

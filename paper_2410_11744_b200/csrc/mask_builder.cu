@@ -142,12 +142,8 @@ cudaError_t launch_build_tree_mask(const int32_t* parents, const ReqInfo* reqs, 
   const int CW = W <= 32 ? W : 16;                 // words per column chunk
   const int n_chunks = (W + CW - 1) / CW;
   const size_t smem = size_t(max_n) * CW * 4 + size_t(max_n) * 12;
-  static size_t attr_smem = 48 * 1024;
-  if (smem > attr_smem) {
-    cudaError_t e = cudaFuncSetAttribute(build_tree_mask_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
-    if (e != cudaSuccess) return e;
-    attr_smem = smem;
-  }
+  static DynSmemGrant grant;
+  if (cudaError_t e = grant.ensure(build_tree_mask_kernel, smem); e != cudaSuccess) return e;
   int threads = ((max_n + 31) / 32) * 32;
   if (threads < 256) threads = 256;
   if (threads > 1024) threads = 1024;

@@ -192,12 +192,8 @@ cudaError_t launch_verify_tree(const int32_t* parents, const int32_t* tokens, co
                                cudaStream_t stream) {
   if (n_req <= 0) return cudaSuccess;
   const size_t smem = size_t(kMaxChunks) * kVThreads * 16 + size_t(max_nodes) * 4;
-  static size_t attr_smem = 48 * 1024;
-  if (smem > attr_smem) {
-    cudaError_t e = cudaFuncSetAttribute(verify_tree_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
-    if (e != cudaSuccess) return e;
-    attr_smem = smem;
-  }
+  static DynSmemGrant grant;
+  if (cudaError_t e = grant.ensure(verify_tree_kernel, smem); e != cudaSuccess) return e;
   verify_tree_kernel<<<n_req, kVThreads, smem, stream>>>(parents, tokens, draft_probs, target_probs, accept_u, sample_u,
                                                          node_offsets, vocab, bonus_at_leaf, out_tokens, out_nodes,
                                                          out_count, max_out, status);

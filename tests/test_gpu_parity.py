@@ -182,6 +182,33 @@ def test_single_request_entry_points(rt):
         assert np.abs(got - ref).max() <= MAX_ABS and np.abs(got - ref).mean() <= MEAN_ABS
 
 
+def test_single_request_form_follows_a_change_of_scale(rt):
+    """The cached plans of the convenience form are keyed by the scale too: the same shape with another
+    scale must not reuse the old plan."""
+    import torch
+    B, R = rt
+    w = wl.make_config(1)
+    L, n = int(w.prefix_len[0]), int(w.n_nodes[0])
+    W = B.dyspec_words_per_row(n)
+    dev = torch.device("cuda:0")
+    parents = torch.from_numpy(w.parents[0]).to(dev)
+    bits = torch.zeros((n, W), dtype=torch.int32, device=dev)
+    depths = torch.zeros((n,), dtype=torch.int32, device=dev)
+    B.dyspec_build_tree_mask(parents, n, bits, depths, W)
+    q = torch.from_numpy(w.q.view(np.int16)).to(dev).view(torch.bfloat16)
+    k = torch.from_numpy(w.k.view(np.int16)).to(dev).view(torch.bfloat16)
+    v = torch.from_numpy(w.v.view(np.int16)).to(dev).view(torch.bfloat16)
+    out = torch.zeros_like(q)
+    for scale in (0.05, 0.3, 0.05):
+        B.dyspec_set_default_shape(w.n_q_heads, w.n_kv_heads, w.head_dim, W, scale)
+        out.zero_()
+        B.dyspec_tree_attention(q, k, v, L, bits, n, out)
+        torch.cuda.synchronize()
+        got = orc.bf16_bits_to_f64(R.bf16_tensor_to_bits(out))
+        ref = orc.tree_attention(w.q, w.k, w.v, L, w.parents[0], scale=scale)
+        assert np.abs(got - ref).max() <= MAX_ABS and np.abs(got - ref).mean() <= MEAN_ABS, scale
+
+
 def test_runs_are_bitwise_repeatable(rt):
     """Also checks that the arrival counters of the fused combine are left at zero by every call."""
     w = wl.make_config(2)
