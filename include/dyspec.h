@@ -299,7 +299,8 @@ int dyspec_tree_attention_ragged_sparse(const dyspec_plan_t* plan, const void* q
  *   sample_u          dev float [N]        U(0,1) number used when a token is drawn at that node (inverse
  *                                          CDF in token order: first v with cumsum(R)[v] > u * sum(R))
  *   node_offsets      dev int32 [n_req+1]  request r owns nodes node_offsets[r] .. node_offsets[r+1]-1
- *   max_nodes         upper bound of the requests' node counts (<= DYSPEC_MAX_NODES)
+ *   max_nodes         upper bound of the requests' node counts (<= DYSPEC_MAX_NODES); a request with more
+ *                     nodes emits nothing (n_accepted = 0) and sets status DYSPEC_ERR_INVALID_ARG
  *   vocab             <= DYSPEC_MAX_VOCAB
  *   accepted_tokens   dev int32 [n_req][max_out]  (written) the emitted tokens, in order
  *   accepted_nodes    dev int32 [n_req][max_out]  (written) the accepted node of each, -1 for a drawn token

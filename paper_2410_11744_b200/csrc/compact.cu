@@ -26,7 +26,7 @@ compact_kv_kernel(uint4* __restrict__ k_cache, uint4* __restrict__ v_cache, cons
   int kept = 0;
   for (int i = 0; i < n; ++i) {
     const int a = acc[i];
-    if (a < 0) continue;                       // an emitted token without a tree node
+    if (a < 0 || a >= DYSPEC_MAX_NODES) continue;   // an emitted token without a tree node (or not a node index at all)
     if (col < row_vecs && a != kept) cache[base + int64_t(kept) * row_vecs + col] = cache[base + int64_t(a) * row_vecs + col];
     ++kept;
   }
@@ -54,7 +54,7 @@ compact_kv_paged_kernel(uint4* __restrict__ k_cache, uint4* __restrict__ v_cache
   int kept = 0;
   for (int i = 0; i < n; ++i) {
     const int a = acc[i];
-    if (a < 0) continue;                       // an emitted token without a tree node
+    if (a < 0 || a >= DYSPEC_MAX_NODES) continue;   // an emitted token without a tree node (or not a node index at all)
     const int t = L + kept;
     const int pi = t >> page_shift;
     const int page = pi < pages_per_req ? pages[pi] : -1;

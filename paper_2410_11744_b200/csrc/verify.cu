@@ -23,7 +23,7 @@ __global__ void __launch_bounds__(kVThreads, 1)
 verify_tree_kernel(const int32_t* __restrict__ parents, const int32_t* __restrict__ tokens,
                    const float* __restrict__ draft_probs, const float* __restrict__ target_probs,
                    const float* __restrict__ accept_u, const float* __restrict__ sample_u,
-                   const int32_t* __restrict__ node_offsets, int vocab, int bonus_at_leaf,
+                   const int32_t* __restrict__ node_offsets, int max_nodes, int vocab, int bonus_at_leaf,
                    int32_t* __restrict__ out_tokens, int32_t* __restrict__ out_nodes, int32_t* __restrict__ out_count,
                    int max_out, int32_t* status) {
   extern __shared__ __align__(16) uint8_t vsm[];
@@ -42,8 +42,11 @@ verify_tree_kernel(const int32_t* __restrict__ parents, const int32_t* __restric
   const int n_vec = vocab >> 2;                                  // float4 chunks in a row
   const int n_chunks = (n_vec + kVThreads - 1) / kVThreads;      // per thread, <= kMaxChunks
   int n_out = 0;
-  if (n <= 0) {
-    if (tid == 0) out_count[r] = 0;
+  if (n <= 0 || n > max_nodes) {            // max_nodes sized the shared arrays: a larger request is refused
+    if (tid == 0) {
+      out_count[r] = 0;
+      if (n > max_nodes && status) atomicCAS(status, 0, DYSPEC_ERR_INVALID_ARG);
+    }
     return;
   }
   bool bad = false;
@@ -195,7 +198,7 @@ cudaError_t launch_verify_tree(const int32_t* parents, const int32_t* tokens, co
   static DynSmemGrant grant;
   if (cudaError_t e = grant.ensure(verify_tree_kernel, smem); e != cudaSuccess) return e;
   verify_tree_kernel<<<n_req, kVThreads, smem, stream>>>(parents, tokens, draft_probs, target_probs, accept_u, sample_u,
-                                                         node_offsets, vocab, bonus_at_leaf, out_tokens, out_nodes,
+                                                         node_offsets, max_nodes, vocab, bonus_at_leaf, out_tokens, out_nodes,
                                                          out_count, max_out, status);
   return cudaGetLastError();
 }

@@ -22,7 +22,7 @@ def B():
     return binding
 
 
-def run_gpu(B, case, bonus=False, max_out=64):
+def run_gpu(B, case, bonus=False, max_out=64, max_nodes=None):
     import torch
     dev = "cuda:0"
     t = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(dev)
@@ -33,7 +33,8 @@ def run_gpu(B, case, bonus=False, max_out=64):
     out_n = torch.full((max(1, n_req), max_out), -9, dtype=torch.int32, device=dev)
     cnt = torch.full((max(1, n_req),), -9, dtype=torch.int32, device=dev)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
-    max_nodes = max([len(p) for p in case.parents] + [0])
+    if max_nodes is None:
+        max_nodes = max([len(p) for p in case.parents] + [0])
     B.dyspec_verify_tree(parents, tokens, t(case.draft_probs), t(case.target_probs), t(case.accept_u), t(case.sample_u),
                          t(case.node_offsets), n_req, max_nodes, case.vocab, out_t, out_n, cnt, max_out,
                          bonus_at_leaf=bonus, status=status)
@@ -116,3 +117,17 @@ def test_verify_reports_bad_token(B):
     case.tokens[0][1] = 99
     _, _, _, status = run_gpu(B, case)
     assert status == -1
+
+
+def test_verify_refuses_a_request_larger_than_max_nodes(B):
+    """max_nodes sizes the kernel's shared arrays: a request with more nodes emits nothing and is
+    reported; the other requests of the batch are verified as usual."""
+    rng = np.random.default_rng(2)
+    case = wl.make_verify_case(5, 64, [wl.chain_tree(6), wl.chain_tree(40), wl.chain_tree(5)])
+    out_t, out_n, cnt, status = run_gpu(B, case, max_nodes=8)
+    assert status == -1 and int(cnt[1]) == 0
+    ref_t, ref_n, ref_cnt, ref_status = run_gpu(B, case)
+    assert ref_status == 0 and int(ref_cnt[1]) > 0
+    for r in (0, 2):
+        k = int(cnt[r])
+        assert k == int(ref_cnt[r]) and out_t[r, :k].tolist() == ref_t[r, :k].tolist() and out_n[r, :k].tolist() == ref_n[r, :k].tolist()
