@@ -336,7 +336,7 @@ int dyspec_verify_tree(const int32_t* parents, const int32_t* tokens, const floa
  *
  *   draft_table   dev float [n_rows][vocab]   (rows 16-byte aligned: vocab % 4 == 0, vocab <= DYSPEC_MAX_VOCAB)
  *   uniforms      dev float [n_uniforms]      U(0,1) numbers
- *   root_row      dev int32 [n_req]
+ *   root_row      dev int32 [n_req]           (taken modulo n_rows, non-negative remainder)
  *   outputs, stride S = m + 1 (greedy) or max_nodes + 1 (threshold) per request, node 0 = the root:
  *   parents, tokens, rows  dev int32 [n_req][S];  values, child_values  dev float [n_req][S]
  *                 values[k] = the estimated acceptance rate node k was created with, child_values[k] =

@@ -61,7 +61,7 @@ build_tree_greedy_kernel(const float* __restrict__ draft_table, int n_rows, int 
   const size_t base = size_t(r) * (m + 1);
   for (int i = tid; i <= m; i += kVThreads) { s_first[i] = -1; s_next[i] = -1; s_last[i] = -1; }
   if (tid == 0) {
-    s_row[0] = root_row[r] % n_rows;
+    s_row[0] = ((root_row[r] % n_rows) + n_rows) % n_rows;        // non-negative remainder: any int32 maps to a row
     s_tok[0] = 0;
     s_v[0] = 1.0; s_pos[0] = 0; s_att[0] = 0;
     write_node(out, base, 0, -1, 0, 1.f, 1.f, s_row[0]);
@@ -157,7 +157,7 @@ build_tree_threshold_kernel(const float* __restrict__ draft_table, int n_rows, i
   const int r = blockIdx.x, tid = threadIdx.x;
   const size_t base = size_t(r) * (max_nodes + 1);
   if (tid == 0) {
-    s_row[0] = root_row[r] % n_rows;
+    s_row[0] = ((root_row[r] % n_rows) + n_rows) % n_rows;        // non-negative remainder: any int32 maps to a row
     s_cv[0] = 1.0;
     write_node(out, base, 0, -1, 0, 1.f, 1.f, s_row[0]);
   }
@@ -198,8 +198,8 @@ build_tree_threshold_kernel(const float* __restrict__ draft_table, int n_rows, i
 }
 
 size_t build_tree_greedy_smem(int m) {
-  const size_t max_slots = 2 * size_t(m) + 2;          // value (4 bytes) + position and attempt (2 + 2) per slot
-  return 12 * max_slots + 14 * size_t(m + 1) + 64;     // (value 8 bytes) row and token (4 + 4) + three 2-byte links per node
+  const size_t max_slots = 2 * size_t(m) + 2;          // value (8 bytes) + position and attempt (2 + 2) per slot
+  return 12 * max_slots + 14 * size_t(m + 1) + 64;     // row and token (4 + 4) + three 2-byte links per node
 }
 
 cudaError_t launch_build_tree_greedy(const float* draft_table, int n_rows, int vocab, const float* uniforms, int n_uniforms,
