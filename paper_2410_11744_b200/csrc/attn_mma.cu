@@ -636,44 +636,71 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         const int tid = threadIdx.x;                       // compute warps (both sets) are threads 0 .. 255
         const int n_vec = (R * D) >> 2;                    // float4 elements of a group
         constexpr int kB = 4;
-        // sources in the order they are expected: the other owners (small pieces), then the rest
+        // Sources in the order they are expected: the other owners (small pieces), then the rest.  The
+        // LAST source is folded, normalised and stored to global memory in one pass (no write-back of
+        // the merged rows, no barriers behind it): it is the only fold on the critical path.
+        uint32_t pool_a = owners & ~(1u << rank), pool_b = ((1u << C) - 1u) & ~owners;
 #pragma unroll 1
-        for (int pass = 0; pass < 2; ++pass) {
+        for (int k_src = 0; k_src < C - 1; ++k_src) {
+          int s_;
+          if (pool_a) { s_ = __ffs(pool_a) - 1; pool_a &= pool_a - 1u; }
+          else { s_ = __ffs(pool_b) - 1; pool_b &= pool_b - 1u; }
+          const bool last = k_src == C - 2;
+          mbar_wait(bar_src + 8 * s_, 0, abort_flag, p.status);
+          const float* src_o = recv + (s_ < rank ? s_ : s_ - 1) * chunk_floats;
+          const float* src_m = src_o + R * D;
+          const float* src_l = src_m + R;
+          // batches of kB independent elements per thread: all loads first, then the math, then the
+          // stores (a rolled element-by-element loop is a chain of shared-memory latencies)
 #pragma unroll 1
-          for (int s_ = 0; s_ < C; ++s_) {
-            if (s_ == rank || int((owners >> s_) & 1u) == pass) continue;
-            mbar_wait(bar_src + 8 * s_, 0, abort_flag, p.status);
-            const float* src_o = recv + (s_ < rank ? s_ : s_ - 1) * chunk_floats;
-            const float* src_m = src_o + R * D;
-            const float* src_l = src_m + R;
-            // batches of kB independent elements per thread: all loads first, then the math, then the
-            // stores (a rolled element-by-element loop is a chain of shared-memory latencies)
-#pragma unroll 1
-            for (int base = tid; base < n_vec; base += kB * kSets * kComputeWarps * 32) {
-              float4 a[kB], b_[kB];
-              float ma[kB], ms[kB];
+          for (int base = tid; base < n_vec; base += kB * kSets * kComputeWarps * 32) {
+            float4 a[kB], b_[kB];
+            float ma[kB], ms[kB], la[kB], ls[kB];
 #pragma unroll
-              for (int k = 0; k < kB; ++k) {
-                const int idx = min(base + k * kSets * kComputeWarps * 32, n_vec - 1);
-                const int rr = idx / (D / 4);
-                ma[k] = acc_m[rr]; ms[k] = src_m[rr];
-                a[k] = reinterpret_cast<const float4*>(acc_o)[idx];
-                b_[k] = reinterpret_cast<const float4*>(src_o)[idx];
-              }
+            for (int k = 0; k < kB; ++k) {
+              const int idx = min(base + k * kSets * kComputeWarps * 32, n_vec - 1);
+              const int rr = idx / (D / 4);
+              ma[k] = acc_m[rr]; ms[k] = src_m[rr];
+              la[k] = acc_l[rr]; ls[k] = src_l[rr];
+              a[k] = reinterpret_cast<const float4*>(acc_o)[idx];
+              b_[k] = reinterpret_cast<const float4*>(src_o)[idx];
+            }
 #pragma unroll
-              for (int k = 0; k < kB; ++k) {
-                const float mn = fmaxf(ma[k], ms[k]);
-                const float ref = mn == -INFINITY ? 0.f : mn;
-                const float keep = fast_exp2(ma[k] - ref), wgt = fast_exp2(ms[k] - ref);
-                a[k].x = a[k].x * keep + b_[k].x * wgt; a[k].y = a[k].y * keep + b_[k].y * wgt;
-                a[k].z = a[k].z * keep + b_[k].z * wgt; a[k].w = a[k].w * keep + b_[k].w * wgt;
-              }
+            for (int k = 0; k < kB; ++k) {
+              const float mn = fmaxf(ma[k], ms[k]);
+              const float ref = mn == -INFINITY ? 0.f : mn;
+              const float keep = fast_exp2(ma[k] - ref), wgt = fast_exp2(ms[k] - ref);
+              a[k].x = a[k].x * keep + b_[k].x * wgt; a[k].y = a[k].y * keep + b_[k].y * wgt;
+              a[k].z = a[k].z * keep + b_[k].z * wgt; a[k].w = a[k].w * keep + b_[k].w * wgt;
+              la[k] = la[k] * keep + ls[k] * wgt;
+            }
+            if (!last) {
 #pragma unroll
               for (int k = 0; k < kB; ++k) {
                 const int idx = base + k * kSets * kComputeWarps * 32;
                 if (idx < n_vec) reinterpret_cast<float4*>(acc_o)[idx] = a[k];
               }
+            } else {
+              // normalise and write the rows (element idx sits at swizzled column c of row rr)
+#pragma unroll
+              for (int k = 0; k < kB; ++k) {
+                const int idx = base + k * kSets * kComputeWarps * 32;
+                const int rr = idx / (D / 4);
+                const int c = ((idx - rr * (D / 4)) * 4) ^ ((rr & 7) << 3);
+                const int row = item.row0 + my_oi * R + rr;
+                if (idx < n_vec && row < n_rows) {
+                  const float inv = la[k] > 0.f ? 1.f / la[k] : 0.f;
+                  const int node = row >> p.log2_g;
+                  const int head = item.kv_head * g + (row & (g - 1));
+                  uint2 o2;
+                  o2.x = pack_bf16x2(a[k].x * inv, a[k].y * inv);
+                  o2.y = pack_bf16x2(a[k].z * inv, a[k].w * inv);
+                  *reinterpret_cast<uint2*>(p.out + (size_t(rq.node0 + node) * p.n_q_heads + head) * D + c) = o2;
+                }
+              }
             }
+          }
+          if (!last) {
             asm volatile("bar.sync 1, %0;" ::"n"(kSets * kComputeWarps * 32) : "memory");   // every row's old maximum has been used
             if (tid < R) {
               const float ma = acc_m[tid], ms = src_m[tid];
@@ -686,34 +713,6 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           }
         }
         if (threadIdx.x == 0) stamp(4);
-        // normalise and write the R rows (element idx sits at swizzled column cs of row rr)
-#pragma unroll 1
-        for (int base = tid; base < n_vec; base += kB * kSets * kComputeWarps * 32) {
-          float4 a[kB];
-          float lsum[kB];
-#pragma unroll
-          for (int k = 0; k < kB; ++k) {
-            const int idx = min(base + k * kSets * kComputeWarps * 32, n_vec - 1);
-            lsum[k] = acc_l[idx / (D / 4)];
-            a[k] = reinterpret_cast<const float4*>(acc_o)[idx];
-          }
-#pragma unroll
-          for (int k = 0; k < kB; ++k) {
-            const int idx = base + k * kSets * kComputeWarps * 32;
-            const int rr = idx / (D / 4);
-            const int c = ((idx - rr * (D / 4)) * 4) ^ ((rr & 7) << 3);
-            const int row = item.row0 + my_oi * R + rr;
-            if (idx < n_vec && row < n_rows) {
-              const float inv = lsum[k] > 0.f ? 1.f / lsum[k] : 0.f;
-              const int node = row >> p.log2_g;
-              const int head = item.kv_head * g + (row & (g - 1));
-              uint2 o2;
-              o2.x = pack_bf16x2(a[k].x * inv, a[k].y * inv);
-              o2.y = pack_bf16x2(a[k].z * inv, a[k].w * inv);
-              *reinterpret_cast<uint2*>(p.out + (size_t(rq.node0 + node) * p.n_q_heads + head) * D + c) = o2;
-            }
-          }
-        }
       }
       if (pusher) dsmem_push_wait_source_read();          // the parked rows must outlive the copies that read them
     } else if (item.slot < 0) {
