@@ -119,6 +119,17 @@ class ClockSampler:
                 "samples": len(sm), "note": note}
 
 
+def whole_job_throughput(local_ms, units_per_step_per_rank, steps, world, dist=None, device="cpu"):
+    """Replicas: every rank runs the same workload; the job's time is the slowest rank's, its work the
+    sum over ranks.  `dist` = torch.distributed (initialised) when world > 1.  Returns (value, max_ms)."""
+    import torch
+    ms = torch.tensor([float(local_ms)], dtype=torch.float64, device=device)
+    if dist is not None and world > 1:
+        dist.all_reduce(ms, op=dist.ReduceOp.MAX)
+    max_ms = float(ms.item())
+    return units_per_step_per_rank * world * steps / (max_ms * 1e-3), max_ms
+
+
 def dist_env():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -525,12 +536,8 @@ def run_ours(args):
     m = measure_config(torch, runner, w, args.steps, args.warmup, device)
     barrier()
     n_lines_after_timed = len(sampler.lines()) if sampler else 0
-    ms = torch.tensor([m["total_ms"]], dtype=torch.float64, device=device)
-    if use_dist:
-        dist.all_reduce(ms, op=dist.ReduceOp.MAX)
-    total_ms = float(ms.item())
+    value, total_ms = whole_job_throughput(m["total_ms"], w.total_nodes, args.steps, world, dist if use_dist else None, device)
     tokens_per_step = w.total_nodes * world
-    value = tokens_per_step * args.steps / (total_ms * 1e-3)
 
     # ---- clocks: the timed region can be shorter than one nvidia-smi period; if so keep the same
     #      loop running (untimed) until a few samples exist, and say so.
@@ -576,10 +583,7 @@ def run_ours(args):
     e1.record(stream)
     torch.cuda.synchronize()
     e2e_ms = max(e0.elapsed_time(e1), (time.perf_counter() - t0) * 1e3)
-    ems = torch.tensor([e2e_ms], dtype=torch.float64, device=device)
-    if use_dist:
-        dist.all_reduce(ems, op=dist.ReduceOp.MAX)
-    e2e_value = tokens_per_step * e2e_steps / (float(ems.item()) * 1e-3)
+    e2e_value, _ = whole_job_throughput(e2e_ms, w.total_nodes, e2e_steps, world, dist if use_dist else None, device)
 
     if rank != 0:
         if use_dist:

@@ -72,3 +72,35 @@ def test_reference_arm_under_torchrun_two_ranks():
     assert r.returncode == 0, r.stderr[-2000:]
     lines = _json_lines(r.stdout)
     assert len(lines) == 1 and lines[0]["impl"] == "reference" and lines[0]["n_gpus"] == 2
+
+
+def _throughput_rank(rank, world, port, q):
+    import torch.distributed as dist
+    sys.path.insert(0, ROOT)
+    import bench
+    dist.init_process_group("gloo", init_method=f"tcp://127.0.0.1:{port}", rank=rank, world_size=world)
+    local_ms = 10.0 if rank == 0 else 25.0                      # rank 1 is the slow one
+    value, max_ms = bench.whole_job_throughput(local_ms, 64, 100, world, dist, "cpu")
+    q.put((rank, value, max_ms))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_whole_job_throughput_is_all_units_over_the_slowest_rank():
+    """N > 1 (replicas, gloo, two CPU ranks): the units of all ranks divided by the maximum over ranks of the time."""
+    import torch.multiprocessing as mp
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    procs = [ctx.Process(target=_throughput_rank, args=(r, 2, 29741, q)) for r in range(2)]
+    for p_ in procs:
+        p_.start()
+    got = sorted(q.get(timeout=300) for _ in procs)
+    for p_ in procs:
+        p_.join(timeout=60)
+        assert p_.exitcode == 0
+    for rank, value, max_ms in got:
+        assert max_ms == 25.0 and abs(value - 2 * 64 * 100 / 25e-3) < 1e-6
+    sys.path.insert(0, ROOT)
+    import bench
+    value, max_ms = bench.whole_job_throughput(10.0, 64, 100, 1)
+    assert max_ms == 10.0 and abs(value - 64 * 100 / 10e-3) < 1e-6
