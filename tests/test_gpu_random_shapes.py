@@ -73,3 +73,57 @@ def test_random_small_batches(rt, seed):
             assert np.isfinite(got).all(), what
             err = np.abs(got - ref)
             assert err.max() <= MAX_ABS and err.mean() <= MEAN_ABS, (what, err.max(), err.mean())
+
+
+def _draw_large(rng, index):
+    g = int(rng.choice([1, 2, 4, 8]))
+    hkv = int(rng.choice([1, 2, 4, 8]))
+    d = int(rng.choice([64, 128]))
+    n_req = int(rng.integers(1, 10))
+    Ls = [int(np.exp(rng.uniform(0.0, np.log(6000.0)))) for _ in range(n_req)]
+    trees = []
+    for _ in range(n_req):
+        n = int(rng.choice([1, 17, 64, 65, 128, 129, 255, 256, 257, 511, 700, 1024, 1500, 2048]))
+        kind = int(rng.integers(0, 3))
+        if kind == 0 and n <= 300:
+            trees.append(wl.chain_tree(n))
+        elif kind <= 1:
+            trees.append(wl.random_tree(rng, n))
+        else:
+            trees.append(wl.greedy_tree(rng, n, 8, 0.2))
+    w = wl.make_custom(20000 + index, hkv * g, hkv, d, Ls, trees)
+    return w, bool(rng.integers(0, 2)), int(rng.choice([0, 0, 1, 2]))
+
+
+@pytest.mark.parametrize("seed", [21, 22])
+def test_random_large_ragged_batches_on_sampled_rows(rt, seed):
+    """Trees up to 2048 nodes, prefixes up to 6000 keys, up to 9 requests: split plans, whole-group plans and
+    the shared queue, with and without tile skipping.  Masks and depths are compared in full, the attention
+    on sampled query nodes of every request (the oracle evaluates those one by one)."""
+    B, R = rt
+    rng = np.random.default_rng(seed)
+    for index in range(8):
+        w, sparse, whole = _draw_large(rng, 100 * seed + index)
+        B.dyspec_set_tuning(-1, 0, 2 + 16 * whole)
+        try:
+            batch = R.DeviceBatch(w, sparse=sparse)
+        finally:
+            B.dyspec_set_tuning(-1, 0, 2)
+        for _ in range(2):
+            batch.step()
+        bits, depths, out_bits, status = batch.results()
+        what = dict(heads=(w.n_q_heads, w.n_kv_heads), d=w.head_dim, L=w.prefix_len.tolist(), n=w.n_nodes.tolist(),
+                    sparse=sparse, whole=whole, plan=batch.plan.describe())
+        assert status == 0, what
+        ref_bits, ref_depths = orc.build_tree_mask_ragged(w.parents, batch.W)
+        assert np.array_equal(bits, ref_bits) and np.array_equal(depths, ref_depths), what
+        got = orc.bf16_bits_to_f64(out_bits)
+        assert np.isfinite(got).all(), what
+        qo = 0
+        for r in range(w.n_req):
+            n, o, L = int(w.n_nodes[r]), int(w.kv_row_offset[r]), int(w.prefix_len[r])
+            nodes = sorted(set(rng.integers(0, n, size=min(n, 24)).tolist() + [0, n - 1]))
+            ref = orc.tree_attention_nodes(w.q[qo:qo + n], w.k[o:o + L + n], w.v[o:o + L + n], L, w.parents[r], nodes)
+            err = np.abs(got[qo:qo + n][nodes] - ref)
+            assert err.max() <= MAX_ABS and err.mean() <= MEAN_ABS, (what, r, err.max(), err.mean())
+            qo += n
