@@ -44,7 +44,7 @@ cudaError_t launch_compact_kv(void* k_cache, void* v_cache, const int64_t* kv_ro
                               const int32_t* accepted_nodes, const int32_t* n_accepted, int n_req, int max_out,
                               int row_bytes, int32_t* new_prefix_len, cudaStream_t stream);
 cudaError_t launch_attn_mma(int head_dim, int n_ctas, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
-                            const AttnParams& p, cudaStream_t stream);
+                            const AttnParams& p, const WorkItem* host_items, cudaStream_t stream);
 cudaError_t launch_combine(int head_dim, int bm, int n_split_groups, const AttnParams& p, cudaStream_t stream);
 cudaError_t launch_attn_tc(int head_dim, int n_ctas, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                            const AttnParams& p, cudaStream_t stream);
@@ -880,7 +880,7 @@ static int run_attention(const dyspec_plan_t* plan, const void* q, const void* k
   for (p.page_shift = 0; page_table && (1 << p.page_shift) < plan->page_size; ++p.page_shift) {}
 
   cudaError_t e;
-  if (plan->regime == 0) e = launch_attn_mma(plan->d, plan->n_ctas, mq, mk, mv, p, st);
+  if (plan->regime == 0) e = launch_attn_mma(plan->d, plan->n_ctas, mq, mk, mv, p, plan->items_strided.data(), st);
   else e = launch_attn_tc(plan->d, plan->n_ctas, mq, mk, mv, p, st);
   if (e != cudaSuccess) return cuda_failed(e, "attention launch");
   e = launch_combine(plan->d, bm, int(plan->split_groups.size()), p, st);
@@ -1038,7 +1038,7 @@ extern "C" int dyspec_tree_attention_static(const void* q, const void* k_cache, 
   p.cluster_size = pl->cluster;
 
   cudaError_t e;
-  if (pl->regime == 0) e = launch_attn_mma(pl->d, pl->n_ctas, mq, mk, mv, p, st);
+  if (pl->regime == 0) e = launch_attn_mma(pl->d, pl->n_ctas, mq, mk, mv, p, pl->items_strided.data(), st);
   else e = launch_attn_tc(pl->d, pl->n_ctas, mq, mk, mv, p, st);
   if (e != cudaSuccess) return DYSPEC_ERR_CUDA;
   e = launch_combine(pl->d, bm, int(pl->split_groups.size()), p, st);

@@ -147,7 +147,8 @@ __device__ __forceinline__ void tmem_st_rows(uint32_t taddr, const float (&v)[NJ
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                     const __grid_constant__ CUtensorMap map_v, const AttnParams p) {
+                     const __grid_constant__ CUtensorMap map_v, const AttnParams p,
+                     const __grid_constant__ FirstItems first) {
   using L = SmemLayout<D>;
   constexpr int kStages = L::kStages;
   constexpr int KS = D / 16;        // k-steps of QK^T
@@ -186,14 +187,17 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     prefetch_tensormap(&map_v);
   }
   const WorkItem* my_items = p.items + size_t(blockIdx.x) * p.items_stride;
+  // the CTA's w-th item: the first one comes with the kernel parameters, the others from global memory
+  const bool first_here = blockIdx.x < kFirstItems;
+  auto item_of = [&](int w) -> WorkItem { return (w == 0 && first_here) ? first.item[blockIdx.x] : my_items[w]; };
   const int item_begin = 0;
-  const int item_end = my_items[0].n_in_cta;    // issued before the barrier below, used after it
+  const int item_end = first_here ? first.item[blockIdx.x].n_in_cta : my_items[0].n_in_cta;
   // Ring depth.  The last stage is where warp set 1 hands its partial output to set 0 (without clusters
   // the ring is busy with the next item's tiles by then).  In cluster mode a CTA that merges (an owner)
   // keeps the last TWO stages free for the partial rows its peers push into them, possibly while it
   // is still streaming K/V itself, and hands over through a ring stage once the ring is idle; a CTA
   // that does not merge receives nothing (it is the one with the most tiles).
-  const bool merge_owner = p.cluster_size > 1 && ((uint32_t(my_items[0].merge_owners) >> cluster_ctarank()) & 1u);
+  const bool merge_owner = p.cluster_size > 1 && ((uint32_t(first_here ? first.item[blockIdx.x].merge_owners : my_items[0].merge_owners) >> cluster_ctarank()) & 1u);
   const int n_stages = merge_owner ? kStages - 2 : kStages;
   // tensor memory: O of set 0, O of set 1 (D columns each), then the score buffers
   const uint32_t kOCols = D, kSCol0 = 2 * D;
@@ -238,7 +242,7 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       uint32_t ring_phase = 0;
       uint32_t qit = 0;      // running item counter (Q buffer phase)
       for (int w = item_begin; w < item_end; ++w, ++qit) {
-        const WorkItem item = my_items[w];
+        const WorkItem item = item_of(w);
         const WorkItem& rq = item;
         // Q tile: box (64 cols, g heads, BM/g nodes) per panel; rows land node-major, head-minor.
         mbar_wait(bar_qempty, (qit & 1) ^ 1, abort_flag, p.status);
@@ -273,7 +277,7 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       int n_base = 0;                      // key tiles of earlier items (ring / score-buffer position)
       const uint32_t q_lo = desc_lo(s_q);
       for (int w = item_begin; w < item_end; ++w, ++qit) {
-        const WorkItem item = my_items[w];
+        const WorkItem item = item_of(w);
         const int T = item.tile_end - item.tile_begin;
         mbar_wait(bar_qfull, qit & 1, abort_flag, p.status);
         for (int i = 0; i < T; ++i) {
@@ -307,7 +311,7 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       int n_base = 0;
       constexpr uint32_t kIdescPV = idesc_pv<D>();
       for (int w = item_begin; w < item_end; ++w, ++qit) {
-        const WorkItem item = my_items[w];
+        const WorkItem item = item_of(w);
         const int T = item.tile_end - item.tile_begin;
         for (int m = 0; m < T; ++m) {
           const int pos = n_base + m;
@@ -366,7 +370,7 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   uint32_t qit = 0;
 
   for (int w = item_begin; w < item_end; ++w, ++qit) {
-    const WorkItem item = my_items[w];
+    const WorkItem item = item_of(w);
     const WorkItem& rq = item;
     const int n_prefix_tiles = (rq.prefix_len + BN - 1) / BN;
     const int n_rows = rq.n_nodes * g;                     // packed rows of this (request, kv head)
@@ -759,7 +763,11 @@ size_t attn_mma_smem_bytes(int head_dim) {
 int attn_mma_threads() { return kThreads; }
 
 cudaError_t launch_attn_mma(int head_dim, int n_ctas, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
-                            const AttnParams& p, cudaStream_t stream) {
+                            const AttnParams& p, const WorkItem* host_items, cudaStream_t stream) {
+  // host_items: the host copy of p.items (same stride); each CTA's first item travels as a kernel parameter
+  FirstItems first;
+  for (int c = 0; c < kFirstItems; ++c)
+    first.item[c] = c < n_ctas ? host_items[size_t(c) * p.items_stride] : WorkItem{};
   const size_t smem = attn_mma_smem_bytes(head_dim);
   static DynSmemGrant grant[2];
   cudaLaunchAttribute attr[2];
@@ -779,11 +787,11 @@ cudaError_t launch_attn_mma(int head_dim, int n_ctas, const CUtensorMap& mq, con
   if (head_dim == 128) {
     if (cudaError_t ge = grant[0].ensure(tree_attn_mma_kernel<128>, smem); ge != cudaSuccess) return ge;
     cfg.dynamicSmemBytes = smem;
-    e = cudaLaunchKernelEx(&cfg, tree_attn_mma_kernel<128>, mq, mk, mv, p);
+    e = cudaLaunchKernelEx(&cfg, tree_attn_mma_kernel<128>, mq, mk, mv, p, first);
   } else {
     if (cudaError_t ge = grant[1].ensure(tree_attn_mma_kernel<64>, smem); ge != cudaSuccess) return ge;
     cfg.dynamicSmemBytes = smem;
-    e = cudaLaunchKernelEx(&cfg, tree_attn_mma_kernel<64>, mq, mk, mv, p);
+    e = cudaLaunchKernelEx(&cfg, tree_attn_mma_kernel<64>, mq, mk, mv, p, first);
   }
   return e != cudaSuccess ? e : cudaGetLastError();
 }

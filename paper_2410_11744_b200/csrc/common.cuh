@@ -49,6 +49,11 @@ struct WorkItem {
 };
 static_assert(sizeof(WorkItem) == 64, "WorkItem is one 64-byte record");
 
+// The first work item of every CTA, passed to the small-tile kernel by value (kernel parameter space):
+// a CTA then knows its first item without a global-memory round trip in front of its first loads.
+constexpr int kFirstItems = 148;
+struct FirstItems { WorkItem item[kFirstItems]; };
+
 // A split query-tile group, for the combine step.
 struct GroupInfo {
   int32_t req;
