@@ -340,10 +340,17 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     if (p.cluster_size > 1) cluster_wait();
   } else {
   // -------------------------------------------------------------------- compute warps
-  // Everything read so far (work items, Q/K/V through TMA) is input that no kernel of this stream
-  // writes.  The mask, the partials and the output are: wait for the preceding kernels here, while
-  // the producer warp keeps streaming K/V.
-  grid_dependency_wait();
+  // Work items and Q/K/V (through TMA) are inputs that no kernel launched with early start writes: the
+  // prefix tiles need nothing else, so they are processed while the preceding kernels of the stream may
+  // still be running.  The mask, the partials and the output do depend on them: every thread waits
+  // for the preceding kernels right before it first reads mask words or writes to global memory.
+  bool dep_ok = false;
+  auto need_dep = [&]() {
+    if (!dep_ok) {
+      grid_dependency_wait();
+      dep_ok = true;
+    }
+  };
   // "Every peer has initialised its barriers": the peers arrived right after their set-up, long before
   // the first K/V tile can be here, so waiting now costs nothing and the merge does not have to.
   if (p.cluster_size > 1) cluster_wait();
@@ -380,13 +387,6 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     const bool ok_lo = row_lo < n_rows, ok_hi = row_hi < n_rows;
 
 
-    // The mask words of the first tree tile are fetched now: the tree tiles come last in an item, and a
-    // global load in front of the last tile's softmax would sit on the critical path of the CTA.
-    uint2 pre_lo = make_uint2(0u, 0u), pre_hi = make_uint2(0u, 0u);
-    if (item.tile_end > n_prefix_tiles) {
-      if (ok_lo) pre_lo = __ldg(reinterpret_cast<const uint2*>(p.bits + size_t(rq.node0 + node_lo) * p.words_per_row));
-      if (ok_hi) pre_hi = __ldg(reinterpret_cast<const uint2*>(p.bits + size_t(rq.node0 + node_hi) * p.words_per_row));
-    }
 
     float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;   // m: the reference the accumulator is scaled to
     const int T_item = item.tile_end - item.tile_begin;
@@ -405,6 +405,15 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       // ---- S = Q K^T (16 x 64 per warp) from the tile's score buffer; the stage's own barrier is complete
       //      by then (the products were issued behind it), waiting on it as well makes the TMA-written V
       //      tile visible to this thread.
+      // A tree tile's mask words are fetched first (after the preceding kernels are known to be done:
+      // the mask builder is one of them), so that the loads are in flight during the waits below.
+      uint2 w_lo = make_uint2(0u, 0u), w_hi = make_uint2(0u, 0u);
+      if (t >= n_prefix_tiles) {
+        need_dep();
+        const int u = t - n_prefix_tiles;
+        if (ok_lo) w_lo = __ldg(reinterpret_cast<const uint2*>(p.bits + size_t(rq.node0 + node_lo) * p.words_per_row) + u);
+        if (ok_hi) w_hi = __ldg(reinterpret_cast<const uint2*>(p.bits + size_t(rq.node0 + node_hi) * p.words_per_row) + u);
+      }
       mbar_wait(bar_sfull + 8 * sb, uint32_t(pos / kSBufs) & 1u, abort_flag, p.status);
       mbar_wait(bar_full + 8 * stage, ph, abort_flag, p.status);
       tc_fence_after();
@@ -426,12 +435,6 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       } else {
         const int u = t - n_prefix_tiles;
         own = min(BN, rq.n_nodes - u * BN);
-        uint2 w_lo = pre_lo, w_hi = pre_hi;
-        if (u > 0) {
-          w_lo = w_hi = make_uint2(0u, 0u);
-          if (ok_lo) w_lo = __ldg(reinterpret_cast<const uint2*>(p.bits + size_t(rq.node0 + node_lo) * p.words_per_row) + u);
-          if (ok_hi) w_hi = __ldg(reinterpret_cast<const uint2*>(p.bits + size_t(rq.node0 + node_hi) * p.words_per_row) + u);
-        }
         vis_lo = (uint64_t(w_lo.y) << 32) | w_lo.x;
         vis_hi = (uint64_t(w_hi.y) << 32) | w_hi.x;
       }
@@ -634,6 +637,7 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       }
       if (threadIdx.x == 0) stamp(2);
       if (own) {
+        need_dep();                                        // the merged rows go to global memory
         float* acc_o = send + my_oi * chunk_floats;        // the running merge lives in this CTA's own group
         float* acc_m = acc_o + R * D;
         float* acc_l = acc_m + R;
@@ -720,6 +724,7 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       }
       if (pusher) dsmem_push_wait_source_read();          // the parked rows must outlive the copies that read them
     } else if (item.slot < 0) {
+      need_dep();
       const float inv_lo = l_lo > 0.f ? 1.f / l_lo : 0.f, inv_hi = l_hi > 0.f ? 1.f / l_hi : 0.f;
       const int head_lo = item.kv_head * g + (row_lo & (g - 1)), head_hi = item.kv_head * g + (row_hi & (g - 1));
       __nv_bfloat16* out_lo = p.out + (size_t(rq.node0 + node_lo) * p.n_q_heads + head_lo) * D;
@@ -732,6 +737,7 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       }
     } else {
       // partial slot: O [BM][D] fp32, then m [BM], then l [BM]
+      need_dep();                                          // (the previous launch's combine may still be reading the slots)
       float* slot = p.partial + size_t(item.slot) * p.slot_floats;
       const int r_lo = wrow + gid, r_hi = r_lo + 8;
 #pragma unroll
