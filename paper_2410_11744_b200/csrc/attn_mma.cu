@@ -411,8 +411,8 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       if (t >= n_prefix_tiles) {
         need_dep();
         const int u = t - n_prefix_tiles;
-        if (ok_lo) w_lo = __ldg(reinterpret_cast<const uint2*>(p.bits + size_t(rq.node0 + node_lo) * p.words_per_row) + u);
-        if (ok_hi) w_hi = __ldg(reinterpret_cast<const uint2*>(p.bits + size_t(rq.node0 + node_hi) * p.words_per_row) + u);
+        if (ok_lo) w_lo = ld_after_dependency_v2(reinterpret_cast<const uint2*>(p.bits + size_t(rq.node0 + node_lo) * p.words_per_row) + u);
+        if (ok_hi) w_hi = ld_after_dependency_v2(reinterpret_cast<const uint2*>(p.bits + size_t(rq.node0 + node_hi) * p.words_per_row) + u);
       }
       mbar_wait(bar_sfull + 8 * sb, uint32_t(pos / kSBufs) & 1u, abort_flag, p.status);
       mbar_wait(bar_full + 8 * stage, ph, abort_flag, p.status);

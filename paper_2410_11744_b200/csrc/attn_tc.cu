@@ -190,7 +190,7 @@ __device__ __forceinline__ TileWalk walk_sparse(const AttnParams& p, const WorkI
   const int node_lo = item.row0 >> p.log2_g;
   const int node_hi = min(item.n_nodes, ((item.row0 + 2 * BMH - 1) >> p.log2_g) + 1);
   uint32_t occ = 0u;
-  for (int node = node_lo + lane; node < node_hi; node += 32) occ |= __ldg(p.node_tiles + item.node0 + node);
+  for (int node = node_lo + lane; node < node_hi; node += 32) occ |= ld_after_dependency_u32(p.node_tiles + item.node0 + node);
   occ = __reduce_or_sync(0xffffffffu, occ);
   // node_tiles counts 64-column tiles; a key tile here is BN = 128 columns: OR the bit pairs together
   uint32_t x = (occ | (occ >> 1)) & 0x55555555u;
@@ -512,9 +512,17 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   } else {
     asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");
     // ------------------------------------------------------------------ softmax + epilogue warps
-    // Q/K/V and the work items are inputs no kernel of this stream writes; the mask, the partials
-    // and the output are: wait for the preceding kernels before touching those.
-    grid_dependency_wait();
+    // Q/K/V and the work items are inputs no kernel launched with early start writes, and full prefix
+    // tiles need nothing else: they are processed while the preceding kernels of the stream may still be
+    // running.  The mask, the tile sets, the partials and the output do depend on those kernels: the
+    // thread waits for them right before it first touches any of these.
+    bool dep_ok = false;
+    auto need_dep = [&]() {
+      if (!dep_ok) {
+        grid_dependency_wait();
+        dep_ok = true;
+      }
+    };
     const int h = (warp - 4) >> 2;                       // query half
     const int r = ((warp & 3) << 5) + lane;              // row of the half == TMEM lane
     const uint32_t lane_sel = uint32_t((warp & 3) << 5) << 16;
@@ -548,6 +556,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       const int n_rows = rq.n_nodes * g;
       const int nh = (n_rows - item.row0 > BMH) ? 2 : 1;
       const int n_prefix_tiles = (rq.prefix_len + BN - 1) / BN;
+      if (p.node_tiles != nullptr) need_dep();           // the tile walk reads the per-node tile sets
       const TileWalk wk = walk_sparse(p, item, n_prefix_tiles, lane);
       const int T = wk.T;
       if (h >= nh) { sc += 2u * uint32_t(T); continue; }
@@ -583,7 +592,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           const int u = t - n_prefix_tiles;
           own = min(BN, rq.n_nodes - u * BN);
           uint4 mv = make_uint4(0u, 0u, 0u, 0u);
-          if (ok) mv = __ldg(mask_row + u);
+          need_dep();
+          if (ok) mv = ld_after_dependency_v4(mask_row + u);
           vis[0] = mv.x; vis[1] = mv.y; vis[2] = mv.z; vis[3] = mv.w;
         }
 
@@ -691,6 +701,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       ++n_o;
       if (r == 0) trace_event(tc_cur, DYSPEC_TAG(1 + h, 6, 0));
       tc_fence_after();
+      need_dep();                                          // global writes from here on
       const int head = item.kv_head * g + (row & (g - 1));
       if (item.slot < 0) {
         const float inv = l > 0.f ? 1.f / l : 0.f;

@@ -263,6 +263,24 @@ __device__ __forceinline__ bool counter_wait(uint32_t addr, uint32_t target, vol
 // start while its predecessor in the stream is still running; it must call grid_dependency_wait()
 // before it reads anything the predecessor writes or writes anything the predecessor (or earlier
 // kernels) may still read.  The predecessor lets dependents start early with trigger_dependents().
+// Loads of data that a preceding kernel of the stream wrote (mask words, tile sets), for use after
+// grid_dependency_wait(): ordinary coherent loads that the compiler may not move (a read-only __ldg
+// could legally be hoisted above the wait and would then see the buffer's old contents).
+__device__ __forceinline__ uint4 ld_after_dependency_v4(const void* ptr) {
+  uint4 v;
+  asm volatile("ld.global.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(ptr) : "memory");
+  return v;
+}
+__device__ __forceinline__ uint2 ld_after_dependency_v2(const void* ptr) {
+  uint2 v;
+  asm volatile("ld.global.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(ptr) : "memory");
+  return v;
+}
+__device__ __forceinline__ uint32_t ld_after_dependency_u32(const void* ptr) {
+  uint32_t v;
+  asm volatile("ld.global.u32 %0, [%1];" : "=r"(v) : "l"(ptr) : "memory");
+  return v;
+}
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void trigger_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 

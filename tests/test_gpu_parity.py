@@ -307,3 +307,28 @@ def test_growing_maxima_exercise_the_lazy_rescale(rt, hq, hkv, n, L):
     for regime in (0, 1) if n * (hq // hkv) <= 64 else (1,):
         run_and_check(rt, w, regime=regime)
     run_and_check(rt, w)
+
+
+@pytest.mark.parametrize("n_nodes,heads", [(64, (8, 8)), (48, (32, 4)), (1024, (2, 2))])
+def test_mask_of_this_step_is_the_one_used_when_the_tree_changes(rt, n_nodes, heads):
+    """The attention kernels start on the prefix tiles before the mask builder of the same step has
+    finished and wait for it only in front of the tree tiles.  Same buffers, same shape, the tree
+    changes from step to step (chain, star, random): a mask word read too early would be the previous
+    step's."""
+    import torch
+    B, R = rt
+    rng = np.random.default_rng(n_nodes)
+    trees = [wl.chain_tree(n_nodes), wl.star_forest(n_nodes), wl.random_tree(rng, n_nodes), wl.chain_tree(n_nodes)]
+    ws = [wl.make_custom(77, heads[0], heads[1], 64, [200], [t]) for t in trees]      # same seed: same Q, K, V
+    batch = R.DeviceBatch(ws[0])
+    refs = [orc.tree_attention_ragged(w.q, w.k, w.v, w.prefix_len, w.n_nodes, w.kv_row_offset, w.parents) for w in ws]
+    for it in range(12):
+        k = it % len(ws)
+        batch.parents.copy_(torch.from_numpy(ws[k].parents_concat).to(batch.parents.device))
+        batch.step()
+        bits, depths, out_bits, status = batch.results()
+        assert status == 0
+        ref_bits, _ = orc.build_tree_mask_ragged(ws[k].parents, batch.W)
+        assert np.array_equal(bits, ref_bits)
+        err = np.abs(orc.bf16_bits_to_f64(out_bits) - refs[k])
+        assert err.max() <= MAX_ABS and err.mean() <= MEAN_ABS, (it, k, err.max())
