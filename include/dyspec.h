@@ -20,9 +20,10 @@
  *     int32, the caller zeroes it) and the kernel still completes normally.
  *   - bf16 tensors are passed as `const void*`; layouts are row-major with the last index fastest.
  *   - Stream order.  Kernels are launched with programmatic stream serialisation: a kernel may start
- *     while the kernel before it in the stream is finishing, and it reads its pure inputs (parents,
- *     q, k_cache, v_cache) before it waits for that kernel; everything it writes, and the mask it
- *     reads, it touches only after the wait.  Inputs written by ordinary kernels or copies earlier in
+ *     while the kernel before it in the stream is finishing, and it reads and processes its pure
+ *     inputs (parents, q, k_cache, v_cache, page_table: the attention kernels work through the prefix
+ *     keys) before it waits for that kernel; everything it writes, and the mask and tile sets it reads,
+ *     it touches only after the wait.  Inputs written by ordinary kernels or copies earlier in
  *     the stream are safe (without an early-launch signal the stream serialises fully, as always),
  *     and so is every sequence of this library's own calls.  The one thing to avoid is producing
  *     those inputs with a foreign kernel that itself signals early launch of its dependents
