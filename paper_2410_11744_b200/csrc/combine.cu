@@ -10,7 +10,10 @@ namespace dyspec {
 template <int D>
 __global__ void __launch_bounds__(256)
 combine_kernel(const AttnParams p, int bm) {
-  grid_dependency_wait();   // launched early (programmatic dependent launch): the partials must be complete
+  // Launched early (programmatic dependent launch), and lets its own successor start early too: the next
+  // call's kernels wait for this grid's completion themselves before they touch anything it reads or writes.
+  trigger_dependents();
+  grid_dependency_wait();   // the partials must be complete
   const int rows_per_block = 8;
   const int blocks_per_group = bm / rows_per_block;
   const GroupInfo gi = p.groups[blockIdx.x / blocks_per_group];
