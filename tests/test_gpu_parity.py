@@ -332,3 +332,37 @@ def test_mask_of_this_step_is_the_one_used_when_the_tree_changes(rt, n_nodes, he
         assert np.array_equal(bits, ref_bits)
         err = np.abs(orc.bf16_bits_to_f64(out_bits) - refs[k])
         assert err.max() <= MAX_ABS and err.mean() <= MEAN_ABS, (it, k, err.max())
+
+
+@pytest.mark.parametrize("shape", ["split_small_tiles", "split_tensor_core"])
+def test_calls_that_follow_each_other_may_share_a_workspace(rt, shape):
+    """Split-KV plans (partials + combine launch): two batches with different inputs share ONE plan and
+    ONE workspace and are stepped alternately without any synchronisation in between.  The kernels of
+    consecutive calls overlap on the GPU (early start), so a call that wrote its partials before the
+    previous call's combine had read its own would corrupt the previous output."""
+    B, R = rt
+    if shape == "split_small_tiles":
+        mk = lambda seed: wl.make_custom(seed, 8, 8, 128, [3000, 700], [wl.greedy_tree(np.random.default_rng(5), 48, 4, 0.3),
+                                                                      wl.chain_tree(17)])
+        tuning = (-1, 0, 0)          # separate combine kernel instead of the cluster merge
+    else:
+        mk = lambda seed: wl.make_custom(seed, 4, 4, 128, [2500], [wl.random_tree(np.random.default_rng(6), 256)])
+        tuning = (-1, 0, 2)
+    wa, wb = mk(301), mk(302)
+    B.dyspec_set_tuning(*tuning)
+    try:
+        ba = R.DeviceBatch(wa)
+        bb = R.DeviceBatch(wb, plan=ba.plan)
+    finally:
+        B.dyspec_set_tuning(-1, 0, 2)
+    assert ba.plan.describe()["split_groups"] > 0
+    bb.workspace, bb.workspace_bytes = ba.workspace, ba.workspace_bytes
+    for _ in range(6):
+        ba.step()
+        bb.step()
+    for batch, w in ((ba, wa), (bb, wb)):
+        bits, depths, out_bits, status = batch.results()
+        assert status == 0
+        ref = orc.tree_attention_ragged(w.q, w.k, w.v, w.prefix_len, w.n_nodes, w.kv_row_offset, w.parents)
+        err = np.abs(orc.bf16_bits_to_f64(out_bits) - ref)
+        assert err.max() <= MAX_ABS and err.mean() <= MEAN_ABS, (shape, err.max())
