@@ -600,6 +600,15 @@ def run_ours(args):
     torch.cuda.synchronize()
     warm_us = _time_replays(torch, g_warm, 20) / 400 * 1e3
     del g_warm
+    # one call at a time on an idle GPU, cold inputs (rotating buffer sets): what a single call costs when
+    # nothing of a neighbouring call overlaps it (includes the launch gap; not the graded number)
+    iso = []
+    g_iso = [_graph_of(torch, (lambda b=b: b.attention())) for b in m["batches"][:4]]
+    for i in range(24):
+        torch.cuda.synchronize()
+        iso.append(_time_replays(torch, g_iso[i % len(g_iso)], 1) * 1e3)
+    iso_us = float(np.median(iso[4:]))
+    del g_iso
 
     # ---- the other configs, same protocol, fewer steps (reported for context in `per_config`)
     per_config = []
@@ -686,7 +695,7 @@ def run_ours(args):
         "roofline": roof,
         "cpu_baseline": cpu_baseline,
         "kernel_us": {"mask_build": m["mask_ms"] * 1e3, "attention_call": m["attn_ms"] * 1e3,
-                      "attention_call_L2_resident": warm_us},
+                      "attention_call_L2_resident": warm_us, "attention_call_isolated": iso_us},
         "device_status": m["status"],
         "parity_vs_oracle": parity,
     }
