@@ -386,6 +386,21 @@ void schedule(dyspec_plan& pl) {
     pl.items_strided = pl.items_queue;
     return;
   }
+  // Order of a CTA's items.  Items are independent, and a kernel waits for the preceding kernels of the
+  // stream only in front of an item's first tree tile or, for a piece without tree tiles, in front of its
+  // partial write.  So the items that can run longest without that wait go first: in a chain of calls a
+  // CTA then starts on work that does not depend on the previous call while that call is still draining.
+  {
+    const int bn = pl.bn;
+    auto ungated_tiles = [&](const WorkItem& it) {
+      const int npt = (it.prefix_len + bn - 1) / bn;
+      const int prefix_part = std::max(0, std::min(int(it.tile_end), npt) - int(it.tile_begin));
+      return it.tile_end > npt ? prefix_part : int(it.tile_end - it.tile_begin);
+    };
+    for (int c = 0; c < pl.n_ctas; ++c)
+      std::stable_sort(pl.items.begin() + pl.cta_begin[size_t(c)], pl.items.begin() + pl.cta_begin[size_t(c) + 1],
+                       [&](const WorkItem& a, const WorkItem& b) { return ungated_tiles(a) > ungated_tiles(b); });
+  }
   // device layout: fixed stride per CTA, count in the CTA's first item
   pl.items_stride = 1;
   for (int c = 0; c < pl.n_ctas; ++c) pl.items_stride = std::max(pl.items_stride, pl.cta_begin[size_t(c) + 1] - pl.cta_begin[size_t(c)]);
