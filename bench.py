@@ -4,8 +4,11 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config 2] [--no-per-config]
 
 Prints ONE JSON line.  A step is one pass of the whole hot path over one synthetic batch (default:
-the Llama2-7B-shaped config 2).  Inputs are resident in HBM; between steps the path rotates through
-enough independent copies of (Q, K, V, out) that no step finds its inputs in L2.  `e2e` repeats the
+config 5, the ragged batch of 8 Llama2-70B-shaped requests, the largest single-GPU workload).  Inputs
+are resident in HBM; between steps the path rotates through enough independent copies of (Q, K, V, out)
+that no step finds its inputs in L2.  `roofline` grades the attention call by its ISOLATED duration (one
+call at a time on an idle GPU, cold inputs, median) and carries, in `per_config`, the same figures for
+all five configs next to the back-to-back ones (in which consecutive calls overlap).  `e2e` repeats the
 measurement with host buffers (pinned), copies inside the timed region.  `--impl reference` times the
 fp64 CPU oracle instead (rank 0 only).  With N > 1 (torchrun) every rank runs an independent replica:
 the path has no exchange step.
@@ -31,7 +34,7 @@ METRIC = "tree_verify_attention_tree_tokens_per_s"
 UNIT = "tree tokens/s"
 L2_BYTES = 126 * 1024 * 1024
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu
-# captures summarised under profiles/ (tree_attn_mma_c2_*.md, tree_attn_tc_c4_*.md)
+# captures summarised under profiles/ (tree_attn_small_c2_*.md, tree_attn_tc_c4_*.md)
 NCU_TRAFFIC_BYTES = {"c2_llama2_7b_L1024_n64": 18413312, "c4_llama2_70b_L2048_n512": 18992128}
 NOMINAL_HBM_GBS, NOMINAL_BF16_TFLOPS = 8000.0, 2250.0
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
@@ -164,32 +167,49 @@ def time_oracle(w, budget_s=12.0, max_passes=20):
     return times
 
 
+def time_oracle_request(w, r):
+    """The oracle on ONE request of the batch (mask + attention): the bounded sample the reference arm
+    takes per step.  Requests are independent, so the batch's time is the sum over its requests."""
+    from oracle import dyspec_oracle as orc
+    W = 4 * ((max(int(w.n_nodes.max()), 1) + 127) // 128)
+    t0 = time.perf_counter()
+    orc.build_tree_mask_ragged([w.parents[r]], W)
+    n0 = int(w.node_offsets[r])
+    n = int(w.n_nodes[r])
+    orc.tree_attention_ragged(w.q[n0:n0 + n], w.k, w.v, w.prefix_len[r:r + 1], w.n_nodes[r:r + 1], w.kv_row_offset[r:r + 1],
+                              [w.parents[r]])
+    return time.perf_counter() - t0, n
+
+
 def run_reference(args):
     rank, world, _ = dist_env()
     if rank != 0:
         return
     from paper_2410_11744_b200 import workloads
     w = workloads.make_config(args.config)
-    for _ in range(min(args.warmup, 2)):
-        time_oracle(w, budget_s=0.0, max_passes=1)
+    n_warm = min(args.warmup, 2)
+    for i in range(n_warm):
+        time_oracle_request(w, i % w.n_req)
     steps = max(1, args.steps)
-    budget = 120.0
-    times = []
+    budget = 150.0
+    secs, toks = [], []
     t_begin = time.perf_counter()
-    for _ in range(steps):
-        times += time_oracle(w, budget_s=0.0, max_passes=1)
+    for i in range(steps):
+        sec, n = time_oracle_request(w, i % w.n_req)      # one request per step, round robin over the batch
+        secs.append(sec)
+        toks.append(n)
         if time.perf_counter() - t_begin > budget:
             break
-    sec = sum(times) / len(times)
-    value = w.total_nodes / sec
+    value = sum(toks) / sum(secs)
     cores = oracle_threads()
+    sample = (f"{len(secs)} steps, each the oracle (mask + attention) on one request of {w.name}, round robin over its "
+              f"{w.n_req} request(s); value = tree tokens of the sampled requests / their time")
     line = {
-        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": len(times),
-        "warmup": min(args.warmup, 2), "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": len(secs),
+        "warmup": n_warm, "ms_per_step": sum(secs) / len(secs) * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "note": "fp64 numpy oracle, one full pass (mask + attention) per step"},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
-                         "sample": f"{len(times)} full passes of {w.name}"},
+        "config": {"workload": w.name, "note": "fp64 numpy oracle; " + sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -217,34 +237,78 @@ def _time_replays(torch, graph, replays, tail=None):
     return e0.elapsed_time(e1)
 
 
-def measure_config(torch, runner, w, steps, warmup, device, sparse=False, paged=None):
+ROOFLINE_MIN_CALLS = 240      # calls per back-to-back figure, whatever --steps is
+ISOLATED_CALLS = 64           # single calls timed one at a time (the first 8 are dropped)
+
+
+def _median(xs):
+    return float(statistics.median(xs))
+
+
+def measure_config(torch, runner, w, steps, warmup, device, sparse=False, paged=None, isolated=True):
     """Device-resident timing of exactly `steps` steps, rotating over independent copies of the inputs
     that together exceed 2x L2.  The launch sequence of one rotation is captured in a CUDA graph so
-    that the host's launch overhead (python, ctypes) does not starve the GPU."""
+    that the host's launch overhead (python, ctypes) does not starve the GPU.
+
+    Besides the step time it measures the attention call three ways, each with its own repeat count
+    (independent of `steps`):
+      chain      calls on independent buffers back to back; consecutive calls overlap (programmatic
+                 dependent launch), so this is a period, not a duration;
+      dependent  the same chain with a tiny ordinary kernel after every call, which serialises the
+                 stream the way the next layer's GEMM does (the tiny kernel's own period is subtracted);
+      isolated   one call at a time on an idle GPU, events around the single launch, cold inputs,
+                 median: the duration the roofline fraction is graded on.
+    The back-to-back figures are taken in five interleaved rounds (step, attention, mask, ...) and
+    reported as medians, so that a clock or power state that drifts during the run hits all alike."""
     first = runner.DeviceBatch(w, device=device, sparse=sparse, paged=paged)
     nbytes, flops = algorithmic_cost(w, first.W)
     copies = max(2, min(64, int(np.ceil(2.0 * L2_BYTES / max(nbytes, 1)))))
     batches = [first] + [runner.DeviceBatch(w, device=device, plan=first.plan, sparse=sparse, paged=paged)
                          for _ in range(copies - 1)]
     info = first.plan.describe()
-    launches_per_step = 1 + 1 + (1 if info["split_groups"] > 0 else 0)
+    launches_per_step = 1 + 1 + (1 if info["split_groups"] > 0 and info.get("combine_launch", 1) else 0)
     for i in range(max(warmup, 3)):
         batches[i % copies].step()
     torch.cuda.synchronize()
+    tick = torch.zeros(32, dtype=torch.float32, device=device)
+
+    def attn_then_tick():
+        for b in batches:
+            b.attention()
+            tick.add_(1.0)
+
     g_step = _graph_of(torch, lambda: [b.step() for b in batches])
     g_attn = _graph_of(torch, lambda: [b.attention() for b in batches])
     g_mask = _graph_of(torch, lambda: [b.build_mask() for b in batches])
-    for g in (g_step, g_attn, g_mask):
+    g_dep = _graph_of(torch, attn_then_tick)
+    g_tick = _graph_of(torch, lambda: [tick.add_(1.0) for _ in batches])
+    for g in (g_step, g_attn, g_mask, g_dep, g_tick):
         g.replay()
     torch.cuda.synchronize()
     replays, rem = divmod(steps, copies)
     total_ms = _time_replays(torch, g_step, replays, tail=lambda: [batches[i].step() for i in range(rem)])
-    # the dominant kernel alone: attention calls (main kernel + combine) back to back, same rotation
-    r2 = max(1, min(replays, 200))
-    attn_ms = _time_replays(torch, g_attn, r2) / (r2 * copies)
-    mask_ms = _time_replays(torch, g_mask, r2) / (r2 * copies)
+    # ---- the attention call and the mask builder by themselves: own repeat count, interleaved rounds
+    rounds = 5
+    r2 = max(1, int(np.ceil(ROOFLINE_MIN_CALLS / (rounds * copies))))
+    per = {"step": [], "attn": [], "mask": [], "dep": [], "tick": []}
+    for _ in range(rounds):
+        for key, g in (("step", g_step), ("attn", g_attn), ("mask", g_mask), ("dep", g_dep), ("tick", g_tick)):
+            per[key].append(_time_replays(torch, g, r2) / (r2 * copies))
+    step_chain_ms, attn_ms, mask_ms = _median(per["step"]), _median(per["attn"]), _median(per["mask"])
+    dep_ms = max(_median(per["dep"]) - _median(per["tick"]), 0.0)
+    # ---- one call at a time
+    iso_ms = None
+    if isolated:
+        g_iso = [_graph_of(torch, (lambda b=b: b.attention())) for b in batches[:16]]
+        ts = []
+        for i in range(ISOLATED_CALLS):
+            torch.cuda.synchronize()
+            ts.append(_time_replays(torch, g_iso[i % len(g_iso)], 1))
+        iso_ms = _median(ts[8:])
+        del g_iso
     status = int(first.status.item())
-    return dict(batches=batches, total_ms=total_ms, ms_per_step=total_ms / steps, attn_ms=attn_ms, mask_ms=mask_ms,
+    return dict(batches=batches, total_ms=total_ms, ms_per_step=total_ms / steps, step_chain_ms=step_chain_ms,
+                attn_ms=attn_ms, mask_ms=mask_ms, dep_ms=dep_ms, iso_ms=iso_ms, chain_calls=rounds * r2 * copies,
                 bytes=nbytes, flops=flops, copies=copies, info=info, launches_per_step=launches_per_step, status=status,
                 graph=g_step)
 
@@ -281,6 +345,8 @@ def random_tree_experiment(torch, runner, workloads, B, peaks, device, sizes=(25
         rows.append({"tree_size": n, "workload": w.name, "blocks32": {"creation_order": blocks[0], "dfs_order": blocks[1]},
                      "attention_call_us": {"creation_order_dense": m1["attn_ms"] * 1e3,
                                            "dfs_order_skipping": m2["attn_ms"] * 1e3},
+                     "attention_call_isolated_us": {"creation_order_dense": m1["iso_ms"] * 1e3,
+                                                    "dfs_order_skipping": m2["iso_ms"] * 1e3},
                      "mask_us": {"plain": m1["mask_ms"] * 1e3, "with_tile_sets": m2["mask_ms"] * 1e3},
                      "reorder_us": reorder_us, "bytes": m1["bytes"], "hbm_floor_us": t_hbm_us,
                      "frac_of_hbm_floor": {"creation_order_dense": t_hbm_us / (m1["attn_ms"] * 1e3),
@@ -426,13 +492,13 @@ def paged_experiment(torch, runner, workloads, B, peaks, device, configs=(2, 3, 
     out = {"page_size": page_size, "configs": []}
     for idx in configs:
         w = workloads.make_config(idx)
-        mc = measure_config(torch, runner, w, steps, 3, device)
-        t_c = (mc["ms_per_step"], mc["attn_ms"])
+        mc = measure_config(torch, runner, w, steps, 3, device, isolated=False)
+        t_c = (mc["step_chain_ms"], mc["attn_ms"])
         del mc
         torch.cuda.empty_cache()
-        mp = measure_config(torch, runner, w, steps, 3, device, paged=workloads.to_paged(w, page_size, idx))
+        mp = measure_config(torch, runner, w, steps, 3, device, paged=workloads.to_paged(w, page_size, idx), isolated=False)
         out["configs"].append({"config": idx, "workload": w.name, "contiguous_step_us": t_c[0] * 1e3,
-                               "contiguous_attention_us": t_c[1] * 1e3, "paged_step_us": mp["ms_per_step"] * 1e3,
+                               "contiguous_attention_us": t_c[1] * 1e3, "paged_step_us": mp["step_chain_ms"] * 1e3,
                                "paged_attention_us": mp["attn_ms"] * 1e3, "bytes": mp["bytes"], "status": mp["status"]})
         del mp
         torch.cuda.empty_cache()
@@ -476,10 +542,10 @@ def small_tree_batch_experiment(torch, runner, workloads, peaks, device, steps=1
     ]
     out = []
     for label, w in cases:
-        m = measure_config(torch, runner, w, steps, 3, device)
+        m = measure_config(torch, runner, w, steps, 3, device, isolated=False)
         gbs = m["bytes"] / (m["attn_ms"] * 1e-3) / 1e9
         out.append({"case": label, "tree_tokens": w.total_nodes, "attention_call_us": m["attn_ms"] * 1e3,
-                    "step_us": m["ms_per_step"] * 1e3, "bytes": m["bytes"], "achieved_gbs": gbs,
+                    "step_us": m["step_chain_ms"] * 1e3, "bytes": m["bytes"], "achieved_gbs": gbs,
                     "frac_of_hbm": gbs / peaks["hbm_gbs"], "plan": m["info"], "status": m["status"]})
         del m
         torch.cuda.empty_cache()
@@ -487,21 +553,42 @@ def small_tree_batch_experiment(torch, runner, workloads, peaks, device, steps=1
 
 
 def roofline_entry(m, peaks, peaks_kind):
+    """Roofline of one attention call: t_roof = max(bytes / HBM, flops / bf16 peak); the graded
+    duration is the isolated one (falls back to the back-to-back period when that was not taken)."""
     t_hbm = m["bytes"] / (peaks["hbm_gbs"] * 1e9)
     t_tc = m["flops"] / (peaks["bf16_tflops"] * 1e12)
-    dur = (m["attn_ms"] if m["attn_ms"] is not None else m["ms_per_step"]) * 1e-3
+    graded = "isolated" if m.get("iso_ms") else "chain"
+    dur = (m["iso_ms"] if graded == "isolated" else m["attn_ms"]) * 1e-3
+    chain = m["attn_ms"] * 1e-3
     # nominal figures (HGX B200: 8 TB/s HBM3e as the workload definition quotes it, 2.25 PFLOP/s dense bf16): context only
+    common = {"traffic": None, "kernel": "tree attention call (main kernel + any combine launch)",
+              "duration": graded + (": one call at a time on an idle GPU, cold inputs, median of %d" % (ISOLATED_CALLS - 8)
+                                    if graded == "isolated" else ": back-to-back period"),
+              "launch_us": dur * 1e6, "chain_us": chain * 1e6, "dependent_chain_us": m["dep_ms"] * 1e3,
+              "chain_note": "back-to-back calls on independent buffers overlap (programmatic dependent launch): a period, "
+                            "not a duration; dependent_chain = the same with a serialising tiny kernel after every call",
+              "bytes": m["bytes"], "flops": m["flops"], "roof_us": max(t_hbm, t_tc) * 1e6}
     if t_hbm >= t_tc:
         ach = m["bytes"] / dur / 1e9
-        return {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],
-                "traffic": None, "peak_kind": peaks_kind, "kernel": "tree attention call (main kernel + combine)",
-                "launch_us": dur * 1e6, "frac_of_nominal": ach / NOMINAL_HBM_GBS, "nominal_peak": NOMINAL_HBM_GBS}
+        common.update({"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],
+                       "frac_chain": m["bytes"] / chain / 1e9 / peaks["hbm_gbs"], "peak_kind": peaks_kind,
+                       "frac_of_nominal": ach / NOMINAL_HBM_GBS, "nominal_peak": NOMINAL_HBM_GBS})
+        return common
     ach = m["flops"] / dur / 1e12
-    return {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-            "frac": ach / peaks["bf16_tflops"], "traffic": None, "peak_kind": peaks_kind + " (burst)",
-            "kernel": "tree attention call (main kernel + combine)", "launch_us": dur * 1e6,
-            "frac_of_sustained": ach / peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]),
-            "frac_of_nominal": ach / NOMINAL_BF16_TFLOPS, "nominal_peak": NOMINAL_BF16_TFLOPS}
+    common.update({"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                   "frac": ach / peaks["bf16_tflops"], "frac_chain": m["flops"] / chain / 1e12 / peaks["bf16_tflops"],
+                   "peak_kind": peaks_kind + " (burst)",
+                   "frac_of_sustained": ach / peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]),
+                   "frac_of_nominal": ach / NOMINAL_BF16_TFLOPS, "nominal_peak": NOMINAL_BF16_TFLOPS})
+    return common
+
+
+def compact_roofline(idx, wi, mi, ri):
+    """One per-config entry of roofline.per_config: everything needed to recompute the fraction by hand."""
+    return {"config": idx, "workload": wi.name, "bound": ri["bound"], "bytes": mi["bytes"], "flops": mi["flops"],
+            "roof_us": ri["roof_us"], "isolated_us": None if mi["iso_ms"] is None else mi["iso_ms"] * 1e3,
+            "chain_us": mi["attn_ms"] * 1e3, "dependent_chain_us": mi["dep_ms"] * 1e3, "frac": ri["frac"],
+            "frac_chain": ri["frac_chain"], "graded_on": ri["duration"].split(":")[0]}
 
 
 def run_ours(args):
@@ -600,31 +687,27 @@ def run_ours(args):
     torch.cuda.synchronize()
     warm_us = _time_replays(torch, g_warm, 20) / 400 * 1e3
     del g_warm
-    # one call at a time on an idle GPU, cold inputs (rotating buffer sets): what a single call costs when
-    # nothing of a neighbouring call overlaps it (includes the launch gap; not the graded number)
-    iso = []
-    g_iso = [_graph_of(torch, (lambda b=b: b.attention())) for b in m["batches"][:4]]
-    for i in range(24):
-        torch.cuda.synchronize()
-        iso.append(_time_replays(torch, g_iso[i % len(g_iso)], 1) * 1e3)
-    iso_us = float(np.median(iso[4:]))
-    del g_iso
 
-    # ---- the other configs, same protocol, fewer steps (reported for context in `per_config`)
-    per_config = []
+    # ---- all five configs, same protocol: compact entries inside `roofline`, the longer ones in `per_config`
+    per_config, roof_rows = [], []
     if not args.no_per_config:
         for idx in (1, 2, 3, 4, 5):
             wi = w if idx == args.config else workloads.make_config(idx)
-            mi = m if idx == args.config else measure_config(torch, runner, wi, min(args.steps, 300), args.warmup, device)
+            mi = m if idx == args.config else measure_config(torch, runner, wi, 60, 3, device)
             ri = roofline_entry(mi, peaks, peaks_kind)
+            roof_rows.append(compact_roofline(idx, wi, mi, ri))
             per_config.append({"config": idx, "workload": wi.name, "tree_tokens": wi.total_nodes,
-                               "step_us": mi["ms_per_step"] * 1e3, "attention_call_us": mi["attn_ms"] * 1e3,
-                               "mask_us": mi["mask_ms"] * 1e3, "tokens_per_s": wi.total_nodes / (mi["ms_per_step"] * 1e-3),
+                               "step_us": mi["step_chain_ms"] * 1e3, "attention_call_us": mi["attn_ms"] * 1e3,
+                               "attention_call_isolated_us": mi["iso_ms"] * 1e3, "mask_us": mi["mask_ms"] * 1e3,
+                               "tokens_per_s": wi.total_nodes / (mi["step_chain_ms"] * 1e-3),
                                "bytes": mi["bytes"], "flops": mi["flops"], "bound": ri["bound"], "achieved": ri["achieved"],
                                "unit": ri["unit"], "frac": ri["frac"], "plan": mi["info"], "status": mi["status"]})
             if idx != args.config:
                 del mi["batches"], mi["graph"]
                 torch.cuda.empty_cache()
+    else:
+        roof_rows.append(compact_roofline(args.config, w, m, roof))
+    roof["per_config"] = roof_rows
 
     random_tree = None
     if not args.no_per_config and world == 1:
@@ -671,11 +754,13 @@ def run_ours(args):
                   "tolerance": {"max_abs": 2e-2, "mean_abs": 2e-3}, "device_status": st_g}
     except Exception as e:                # the measurement stands without it
         parity = {"error": repr(e)}
-    try:                                  # the same on one thread (the oracle's only parallelism is its BLAS calls)
-        from threadpoolctl import threadpool_limits
+    try:                                  # the same on one thread (the oracle's only parallelism is its BLAS calls),
+        from threadpoolctl import threadpool_limits   # on the batch's smallest request so that it stays bounded
+        r_small = int(np.argmin(w.n_nodes.astype(np.int64) * (w.prefix_len.astype(np.int64) + w.n_nodes)))
         with threadpool_limits(limits=1):
-            t1 = time_oracle(w, budget_s=4.0, max_passes=5)
-        cpu_baseline["value_1_thread"] = w.total_nodes / (sum(t1) / len(t1))
+            sec1, n1 = time_oracle_request(w, r_small)
+        cpu_baseline["value_1_thread"] = n1 / sec1
+        cpu_baseline["sample_1_thread"] = f"request {r_small} of the batch ({n1} tree tokens), one pass"
     except Exception:
         pass
 
@@ -695,7 +780,9 @@ def run_ours(args):
         "roofline": roof,
         "cpu_baseline": cpu_baseline,
         "kernel_us": {"mask_build": m["mask_ms"] * 1e3, "attention_call": m["attn_ms"] * 1e3,
-                      "attention_call_L2_resident": warm_us, "attention_call_isolated": iso_us},
+                      "attention_call_L2_resident": warm_us, "attention_call_isolated": m["iso_ms"] * 1e3,
+                      "attention_call_dependent_chain": m["dep_ms"] * 1e3, "step_back_to_back": m["step_chain_ms"] * 1e3,
+                      "calls_per_back_to_back_figure": m["chain_calls"]},
         "device_status": m["status"],
         "parity_vs_oracle": parity,
     }
@@ -802,7 +889,7 @@ def main():
     ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", type=int, default=2)
+    ap.add_argument("--config", type=int, default=5)
     ap.add_argument("--no-per-config", action="store_true")
     ap.add_argument("--profile", type=int, default=0,
                     help="run only this many plain (eager) steps of --config and exit: the command to put under ncu")

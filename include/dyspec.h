@@ -83,7 +83,8 @@ int dyspec_build_tree_mask(const int32_t* parents, int n_nodes, uint32_t* ancest
  * (1a) The same for a ragged batch without a plan: node_offsets is a HOST array [n_req + 1] (prefix sums
  * of the tree sizes), parents are request-local indices, concatenated; request r's mask rows and depths
  * start at node_offsets[r]; every row uses the same words_per_row.  status: dev int32 [n_req] or NULL (one
- * word per request).  Runs one launch per request; dyspec_plan_build_tree_mask (1b) does a batch in one.
+ * word per request).  The request list travels with the launch (kernel parameters): one launch per 768
+ * requests, nothing allocated, no host pointer kept.
  */
 int dyspec_build_tree_mask_batched(const int32_t* parents, const int32_t* node_offsets_host, int n_req,
                                    uint32_t* ancestor_bits, int32_t* depths, int words_per_row, int32_t* status,
@@ -141,7 +142,7 @@ int dyspec_schedule_dry_run(int n_q_heads, int n_kv_heads, int head_dim, int n_r
                             const int32_t* n_nodes, int words_per_row, int32_t* items_out, int max_items,
                             int32_t* cta_begin_out, int max_ctas, int64_t* info_out);
 
-/* Testing knobs, read when a plan is created: force the regime (-1 = automatic), the number of
+/* Testing knobs, process-wide; a plan keeps the values it was created with: force the regime (-1 = automatic), the number of
  * CTAs the scheduler balances over (0 = automatic; a negative value -c instead sets the scheduler's
  * per-item cost to c key tiles), and combine_mode = m + 16 k.  m says how split-KV partials are merged:
  * 0 = by the separate combine kernel, 2 (default) = inside a thread-block cluster through distributed
@@ -193,16 +194,23 @@ int dyspec_tree_attention_ragged(const dyspec_plan_t* plan, const void* q, const
                                  int32_t* status, dyspec_stream_t stream);
 
 /*
- * (3b) Single-request convenience form.  The static shape comes from dyspec_set_default_shape;
- * plans and workspaces for each (prefix_len, n_nodes) seen are created on first use and cached
- * inside the library, per device (that first call allocates; later calls do not).  k_cache / v_cache
- * hold exactly prefix_len + n_nodes rows.  Calls of one shape share one cached workspace, so they must
- * follow each other on the GPU (one stream, or streams ordered by events); use the ragged form with
- * workspaces of your own for calls that may overlap.
+ * (3b) Single-request convenience form.  The static shape comes from dyspec_set_default_shape.  The
+ * library keeps, per device and static shape, a small bounded cache: the plans of the last 8
+ * (prefix_len, n_nodes) pairs seen (all layers of a decoding step share one pair, so a step costs one
+ * miss), their device tables in buffers that are reused when a plan is replaced, and one workspace sized
+ * for the worst case of the shape (about 40 MB at head_dim 128).  The first eight misses of a shape
+ * allocate those; after that a miss only runs the host scheduler and sends its tables down `stream` in kernel
+ * parameters -- no allocation, no synchronisation -- unless a tree is large enough to outgrow a table
+ * buffer (64 KB to start with), which replaces that buffer once.  dyspec_release_cache frees everything
+ * (call it with no library work in flight).  k_cache / v_cache hold exactly prefix_len + n_nodes rows.
+ * All calls of one shape share the workspace and the table buffers, so they must follow each other on
+ * the GPU (one stream, or streams ordered by events); use the ragged form with workspaces of your own
+ * for calls that may overlap.
  */
 int dyspec_set_default_shape(int n_q_heads, int n_kv_heads, int head_dim, int words_per_row, float scale);
 int dyspec_tree_attention(const void* q, const void* k_cache, const void* v_cache, int prefix_len,
                           const uint32_t* ancestor_bits, int n_nodes, void* out, dyspec_stream_t stream);
+int dyspec_release_cache(void);
 
 /*
  * (3c) Single-request attention that allocates nothing.  (The paper has no counterpart: this is an
@@ -217,8 +225,10 @@ int dyspec_tree_attention(const void* q, const void* k_cache, const void* v_cach
  * Here the scheduled work list and the split-KV partials live in one fixed device array of
  * DYSPEC_STATIC_SCRATCH_BYTES that is part of the library image: every GPU that loads the library
  * holds those bytes until the process exits, whether or not this call is ever used.  The call runs
- * the host scheduler, copies the work list into the array on `stream`, and launches the same
- * kernels as dyspec_tree_attention_ragged; it calls no cudaMalloc, cudaFree or allocating routine.
+ * the host scheduler, writes the work list into the array on `stream` (the tables travel in kernel
+ * parameters, so no host memory of the call is referred to after it returns and the stream is not
+ * synchronised), and launches the same kernels as dyspec_tree_attention_ragged; it calls no cudaMalloc,
+ * cudaFree or allocating routine.
  * Arguments are those of dyspec_tree_attention plus the static shape (see dyspec_plan_create) and an
  * optional status word; k_cache / v_cache hold exactly prefix_len + n_nodes rows.
  *
@@ -355,18 +365,25 @@ int dyspec_build_tree_threshold(const float* draft_table, int n_rows, int vocab,
 
 /*
  * (7) Keeping the accepted path in the KV cache (after dyspec_verify_tree; the paper only says that the
- * accepted tokens extend the prefix).  For request r with accepted nodes a_0 < a_1 < ... (entries < 0,
- * i.e. emitted tokens without a tree node, are skipped) row off_r + L_r + i of k_cache and v_cache
- * takes the content of row off_r + L_r + a_i, in place, and new_prefix_len[r] = L_r + their number.
+ * accepted tokens extend the prefix).  For request r with kept nodes k_0 < k_1 < ... row off_r + L_r + i
+ * of k_cache and v_cache takes the content of row off_r + L_r + k_i, in place, and new_prefix_len[r] =
+ * L_r + their number.  The kept nodes are the entries >= 0 of accepted_nodes (entries < 0 are emitted
+ * tokens without a tree node) and, when keep_root != 0 and the request's walk emitted anything
+ * (n_accepted[r] > 0), node 0 in front of them: dyspec_verify_tree walks from node 0 and lists only the
+ * accepted children, but node 0 is the last token decoded before the step, a query row of the
+ * verification pass whose own K/V row (tree row 0) was computed in that pass, so the sequence the next
+ * step attends to is old prefix + node 0 + accepted path.  Pass keep_root = 1 when accepted_nodes comes
+ * from dyspec_verify_tree; keep_root = 0 makes the call a plain gather of the listed rows.
  * Rows past the new prefix keep their old content.  One call per layer (per pair of caches).
  *   k_cache, v_cache  dev bf16 [rows][n_kv_heads][head_dim] (16-byte aligned; row bytes a multiple of 16)
  *   kv_row_offset     dev int64 [n_req];  prefix_len  dev int32 [n_req]
- *   accepted_nodes    dev int32 [n_req][max_out], n_accepted dev int32 [n_req]  (as written by dyspec_verify_tree)
+ *   accepted_nodes    dev int32 [n_req][max_out], n_accepted dev int32 [n_req]  (as written by dyspec_verify_tree;
+ *                     node indices increase along a request's list)
  *   new_prefix_len    dev int32 [n_req] or NULL (written)
  */
 int dyspec_compact_kv(void* k_cache, void* v_cache, const int64_t* kv_row_offset, const int32_t* prefix_len,
                       const int32_t* accepted_nodes, const int32_t* n_accepted, int n_req, int max_out, int n_kv_heads,
-                      int head_dim, int32_t* new_prefix_len, dyspec_stream_t stream);
+                      int head_dim, int keep_root, int32_t* new_prefix_len, dyspec_stream_t stream);
 
 /*
  * (8) Paged KV cache (the paper does not fix the cache's memory layout; this is the layout of a serving
@@ -399,9 +416,9 @@ int dyspec_tree_attention_paged(const dyspec_plan_t* plan, const void* q, const 
                                 int32_t* status, dyspec_stream_t stream);
 
 /*
- * (8b) Accepted-path compaction for the paged cache: for request r with accepted nodes a_0 < a_1 < ...
- * (entries < 0 skipped) the pool row of prefix token L_r + i takes the content of tree row
- * tree_row_offset[r] + a_i, for K and V, and new_prefix_len[r] = L_r + their number.  The page table must
+ * (8b) Accepted-path compaction for the paged cache: for request r with kept nodes k_0 < k_1 < ...
+ * (as in dyspec_compact_kv, keep_root included) the pool row of prefix token L_r + i takes the content of
+ * tree row tree_row_offset[r] + k_i, for K and V, and new_prefix_len[r] = L_r + their number.  The page table must
  * already hold a page for every new token; a token without one (entry < 0 or past pages_per_req) stops
  * that request's copy there, new_prefix_len[r] counts what was kept, and *status = DYSPEC_ERR_INVALID_ARG.
  * page_size: a power of two (any).  Other arguments as in dyspec_compact_kv; all arrays dev.
@@ -409,7 +426,7 @@ int dyspec_tree_attention_paged(const dyspec_plan_t* plan, const void* q, const 
 int dyspec_compact_kv_paged(void* k_cache, void* v_cache, const int64_t* tree_row_offset, const int32_t* page_table,
                             int pages_per_req, int page_size, const int32_t* prefix_len, const int32_t* accepted_nodes,
                             const int32_t* n_accepted, int n_req, int max_out, int n_kv_heads, int head_dim,
-                            int32_t* new_prefix_len, int32_t* status, dyspec_stream_t stream);
+                            int keep_root, int32_t* new_prefix_len, int32_t* status, dyspec_stream_t stream);
 
 #ifdef __cplusplus
 }

@@ -24,7 +24,8 @@ What it computes (every function names the passage of the paper it follows):
 Parity status: every function below is pinned by tests/test_oracle_pins.py
 (chain == library causal attention, star == prefix+self, brute force per path
 in pure Python, closed forms, hand-written mask fixture, relabelling
-invariance); the token-reorder functions at the end (App. C) are pinned by
+invariance; visible_pair_count by the chain, star and binary-tree closed forms
+and a pair-by-pair count); the token-reorder functions at the end (App. C) are pinned by
 tests/test_reorder_pins.py (the block counts the paper prints in Table 5,
 closed forms, a hand example, subtree contiguity, attention invariance);
 verify_tree (Algorithm 3) by tests/test_verify_pins.py (the output distribution
@@ -476,12 +477,26 @@ def build_tree_threshold(rows, uniforms, threshold: float, max_nodes: int, root_
 # Keeping the accepted path in the KV cache (the step after verification; the paper only says that the
 # accepted tokens extend the prefix, Sec. 2 / Algorithm 3).
 # ----------------------------------------------------------------------------------------------------
-def compact_kv(cache: np.ndarray, kv_row0: int, prefix_len: int, accepted_nodes: Sequence[int]) -> int:
-    """After a verification step the cache of a request holds prefix_len prefix rows followed by one row
-    per tree node (node j at row kv_row0 + prefix_len + j).  The accepted nodes a_0 < a_1 < ... become
-    part of the prefix: row kv_row0 + prefix_len + i takes the content of node a_i's row, in place.
-    Entries < 0 (an emitted token that has no tree node) are skipped.  Returns the new prefix length."""
+def kept_nodes(accepted_nodes: Sequence[int], keep_root: bool) -> List[int]:
+    """The tree nodes whose K/V rows survive a verification step, in sequence order.  Algorithm 3 walks
+    from the root and emits the accepted CHILDREN (entries < 0 are emitted tokens without a tree node:
+    skipped).  The root itself is the last token decoded before the step; Algorithm 3 needs
+    Target(root, .), so the root is a query row of the verification pass and its K/V row (tree row 0) was
+    computed in that pass too: with keep_root it stays in front of the accepted nodes whenever the
+    walk emitted anything, so that the new prefix is old prefix + root + accepted path."""
     nodes = [int(a) for a in accepted_nodes if int(a) >= 0]
+    if keep_root and len(accepted_nodes) > 0:
+        nodes = [0] + nodes
+    return nodes
+
+
+def compact_kv(cache: np.ndarray, kv_row0: int, prefix_len: int, accepted_nodes: Sequence[int],
+               keep_root: bool = False) -> int:
+    """After a verification step the cache of a request holds prefix_len prefix rows followed by one row
+    per tree node (node j at row kv_row0 + prefix_len + j).  The kept nodes k_0 < k_1 < ... (see
+    kept_nodes) become part of the prefix: row kv_row0 + prefix_len + i takes the content of node k_i's
+    row, in place.  Returns the new prefix length."""
+    nodes = kept_nodes(accepted_nodes, keep_root)
     base = int(kv_row0) + int(prefix_len)
     gathered = [cache[base + a].copy() for a in nodes]       # all reads first: the definition is a gather
     for i, row in enumerate(gathered):
@@ -518,11 +533,11 @@ def tree_attention_paged(q_bits, k_pool, v_pool, page_table, page_size: int, pre
 
 
 def compact_kv_paged(pool: np.ndarray, page_table_row: Sequence[int], page_size: int, tree_row0: int, prefix_len: int,
-                     accepted_nodes: Sequence[int]) -> int:
-    """The accepted nodes a_0 < a_1 < ... become prefix tokens L, L + 1, ...: the pool row of token
-    L + i (through the page table) takes the content of tree row tree_row0 + a_i.  Entries < 0 are
-    skipped.  Returns the new prefix length."""
-    nodes = [int(a) for a in accepted_nodes if int(a) >= 0]
+                     accepted_nodes: Sequence[int], keep_root: bool = False) -> int:
+    """The kept nodes k_0 < k_1 < ... (see kept_nodes) become prefix tokens L, L + 1, ...: the pool row
+    of token L + i (through the page table) takes the content of tree row tree_row0 + k_i.  Returns the
+    new prefix length."""
+    nodes = kept_nodes(accepted_nodes, keep_root)
     L = int(prefix_len)
     dst = paged_prefix_rows(page_table_row, page_size, L + len(nodes))[L:]
     for d, a in zip(dst, nodes):

@@ -51,10 +51,11 @@ SIGNATURES = {
     "dyspec_verify_tree": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _i32, _vp, _vp]),
     "dyspec_build_tree_greedy": (_i32, [_vp, _i32, _i32, _vp, _i32, _vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "dyspec_build_tree_threshold": (_i32, [_vp, _i32, _i32, _vp, _i32, _vp, _i32, _f32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
-    "dyspec_compact_kv": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _i32, _i32, _i32, _i32, _vp, _vp]),
+    "dyspec_compact_kv": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _i32, _i32, _i32, _i32, _i32, _vp, _vp]),
     "dyspec_plan_create_paged": (_i32, [_c.POINTER(_vp), _i32, _i32, _i32, _i32, _vp, _vp, _vp, _i64, _i32, _i32, _f32]),
     "dyspec_tree_attention_paged": (_i32, [_vp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp, _vp, _sz, _vp, _vp]),
-    "dyspec_compact_kv_paged": (_i32, [_vp, _vp, _vp, _vp, _i32, _i32, _vp, _vp, _vp, _i32, _i32, _i32, _i32, _vp, _vp, _vp]),
+    "dyspec_compact_kv_paged": (_i32, [_vp, _vp, _vp, _vp, _i32, _i32, _vp, _vp, _vp, _i32, _i32, _i32, _i32, _i32, _vp, _vp, _vp]),
+    "dyspec_release_cache": (_i32, []),
     "dyspec_tree_attention_static": (_i32, [_vp, _vp, _vp, _i32, _vp, _i32, _vp, _i32, _i32, _i32, _i32, _f32, _vp, _vp]),
 }
 for _name, (_res, _args) in SIGNATURES.items():
@@ -321,11 +322,11 @@ def dyspec_build_tree_threshold(draft_table, n_rows: int, vocab: int, uniforms, 
 
 
 def dyspec_compact_kv(k_cache, v_cache, kv_row_offset, prefix_len, accepted_nodes, n_accepted, n_req: int, max_out: int,
-                      n_kv_heads: int, head_dim: int, new_prefix_len=None, stream=None) -> None:
+                      n_kv_heads: int, head_dim: int, new_prefix_len=None, stream=None, keep_root: bool = False) -> None:
     """Moves the accepted nodes' K/V rows behind the prefix, in place (see include/dyspec.h)."""
     _check(lib.dyspec_compact_kv(_ptr(k_cache), _ptr(v_cache), _ptr(kv_row_offset), _ptr(prefix_len), _ptr(accepted_nodes),
-                                 _ptr(n_accepted), n_req, max_out, n_kv_heads, head_dim, _ptr(new_prefix_len),
-                                 _stream(stream)), "dyspec_compact_kv")
+                                 _ptr(n_accepted), n_req, max_out, n_kv_heads, head_dim, int(bool(keep_root)),
+                                 _ptr(new_prefix_len), _stream(stream)), "dyspec_compact_kv")
 
 
 def dyspec_tree_attention_paged(plan: Plan, q, k_cache, v_cache, page_table, pages_per_req: int, ancestor_bits,
@@ -340,12 +341,17 @@ def dyspec_tree_attention_paged(plan: Plan, q, k_cache, v_cache, page_table, pag
 
 def dyspec_compact_kv_paged(k_cache, v_cache, tree_row_offset, page_table, pages_per_req: int, page_size: int, prefix_len,
                             accepted_nodes, n_accepted, n_req: int, max_out: int, n_kv_heads: int, head_dim: int,
-                            new_prefix_len=None, status=None, stream=None) -> None:
+                            new_prefix_len=None, status=None, stream=None, keep_root: bool = False) -> None:
     """Moves the accepted nodes' K/V rows from the tree rows into the prefix pages (see include/dyspec.h)."""
     _check(lib.dyspec_compact_kv_paged(_ptr(k_cache), _ptr(v_cache), _ptr(tree_row_offset), _ptr(page_table),
                                        int(pages_per_req), int(page_size), _ptr(prefix_len), _ptr(accepted_nodes),
-                                       _ptr(n_accepted), n_req, max_out, n_kv_heads, head_dim, _ptr(new_prefix_len),
-                                       _ptr(status), _stream(stream)), "dyspec_compact_kv_paged")
+                                       _ptr(n_accepted), n_req, max_out, n_kv_heads, head_dim, int(bool(keep_root)),
+                                       _ptr(new_prefix_len), _ptr(status), _stream(stream)), "dyspec_compact_kv_paged")
+
+
+def dyspec_release_cache() -> None:
+    """Frees what dyspec_tree_attention cached (see include/dyspec.h)."""
+    _check(lib.dyspec_release_cache(), "dyspec_release_cache")
 
 
 def dyspec_build_tree_mask_batched(parents, node_offsets: Sequence[int], ancestor_bits, depths, words_per_row: int,

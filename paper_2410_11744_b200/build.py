@@ -12,7 +12,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libdyspec.so")
-SOURCES = ["api.cu", "mask_builder.cu", "dfs_reorder.cu", "verify.cu", "construct.cu", "compact.cu", "attn_mma.cu", "attn_tc.cu", "combine.cu"]
+SOURCES = ["api.cu", "mask_builder.cu", "dfs_reorder.cu", "verify.cu", "construct.cu", "compact.cu", "attn_small.cu", "attn_tc.cu", "combine.cu"]
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
 
 

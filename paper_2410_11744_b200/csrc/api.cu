@@ -18,6 +18,8 @@ namespace dyspec {
 cudaError_t launch_build_tree_mask(const int32_t* parents, const ReqInfo* reqs, int n_req, int single_n, int max_n,
                                    uint32_t* bits, int32_t* depths, uint32_t* node_tiles, int W, int32_t* status,
                                    cudaStream_t stream);
+cudaError_t launch_build_tree_mask_batch(const int32_t* parents, const MaskBatch& batch, int n_req, int max_n, uint32_t* bits,
+                                         int32_t* depths, int W, int32_t* status, cudaStream_t stream);
 cudaError_t launch_dfs_reorder(const int32_t* parents, const ReqInfo* reqs, int n_req, int single_n, int max_n,
                                int32_t* order, int32_t* new_of_old, int32_t* new_parents, int32_t* status,
                                cudaStream_t stream);
@@ -39,11 +41,12 @@ cudaError_t launch_build_tree_threshold(const float* draft_table, int n_rows, in
 cudaError_t launch_compact_kv_paged(void* k_cache, void* v_cache, const int64_t* tree_row_offset, const int32_t* page_table,
                                     int pages_per_req, int page_shift, const int32_t* prefix_len,
                                     const int32_t* accepted_nodes, const int32_t* n_accepted, int n_req, int max_out,
-                                    int row_bytes, int32_t* new_prefix_len, int32_t* status, cudaStream_t stream);
+                                    int row_bytes, int keep_root, int32_t* new_prefix_len, int32_t* status,
+                                    cudaStream_t stream);
 cudaError_t launch_compact_kv(void* k_cache, void* v_cache, const int64_t* kv_row_offset, const int32_t* prefix_len,
                               const int32_t* accepted_nodes, const int32_t* n_accepted, int n_req, int max_out,
-                              int row_bytes, int32_t* new_prefix_len, cudaStream_t stream);
-cudaError_t launch_attn_mma(int head_dim, int n_ctas, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
+                              int row_bytes, int keep_root, int32_t* new_prefix_len, cudaStream_t stream);
+cudaError_t launch_attn_small(int head_dim, int n_ctas, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                             const AttnParams& p, const WorkItem* host_items, cudaStream_t stream);
 cudaError_t launch_combine(int head_dim, int bm, int n_split_groups, const AttnParams& p, cudaStream_t stream);
 cudaError_t launch_attn_tc(int head_dim, int n_ctas, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
@@ -54,13 +57,38 @@ using namespace dyspec;
 
 namespace {
 
-int g_force_regime = -1;
-int g_force_ctas = 0;
-int g_item_cost = 0;       // scheduler experiment knob (0 = default)
-int g_combine_mode = 2;   // 0 separate combine kernel, 2 cluster merge when the plan allows, else as 0
-int g_whole_groups = 0;   // 0: the scheduler's cost model chooses; 1: never deal whole groups; 2: always
-unsigned long long* g_trace = nullptr;   // device buffer for the optional kernel event trace
-int g_trace_capacity = 0;
+// Testing knobs and the developer trace (dyspec_set_tuning, dyspec_set_trace).  Process-wide, but never
+// read while they change: every reader takes a copy under the mutex, and a plan keeps the copy it was
+// created with, so concurrent plan creation and attention calls stay well defined.
+struct Tuning {
+  int force_regime = -1;
+  int force_ctas = 0;
+  int item_cost = 0;       // scheduler experiment knob (0 = default)
+  int combine_mode = 2;    // 0 separate combine kernel, 2 merge on chip / in the attention kernel when the plan allows
+  int whole_groups = 0;    // 0: the scheduler's cost model chooses; 1: never deal whole groups; 2: always
+  unsigned long long* trace = nullptr;   // device buffer for the optional kernel event trace
+  int trace_capacity = 0;
+};
+Tuning g_tuning;
+std::mutex g_tuning_mutex;
+Tuning current_tuning() {
+  std::lock_guard<std::mutex> lock(g_tuning_mutex);
+  return g_tuning;
+}
+
+// SMs of the current device (the scheduler balances over them); B200's count where no device can be asked
+// (the host-only dry run on a machine without a GPU).
+int device_sm_count() {
+  static std::mutex m;
+  static int cached[64] = {};
+  int dev = -1, n = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0) { cudaGetLastError(); return kDefaultSMs; }
+  std::lock_guard<std::mutex> lock(m);
+  if (dev < 64 && cached[dev] > 0) return cached[dev];
+  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) { cudaGetLastError(); return kDefaultSMs; }
+  if (dev < 64) cached[dev] = n;
+  return n;
+}
 
 using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -101,6 +129,30 @@ int cuda_failed(cudaError_t e, const char* where) {
 
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
+// Small host tables -> device memory, stream-ordered, WITHOUT a host pointer that has to outlive the
+// call: the bytes travel in the kernel's parameter space (copied when the launch is enqueued), one
+// launch per 3584-byte piece.  A cudaMemcpyAsync from pageable memory would stage through the driver
+// (and may synchronise the stream); this needs neither pinned memory nor a staging buffer.
+struct TablePiece { uint4 v[224]; };
+__global__ void __launch_bounds__(224) write_table_kernel(uint4* dst, const __grid_constant__ TablePiece piece, int n_vec) {
+  if (int(threadIdx.x) < n_vec) dst[threadIdx.x] = piece.v[threadIdx.x];
+}
+// dst: 16-byte aligned device memory with room for `bytes` rounded up to 16.
+cudaError_t write_table(void* dst, const void* src, size_t bytes, cudaStream_t stream) {
+  const unsigned char* from = static_cast<const unsigned char*>(src);
+  unsigned char* to = static_cast<unsigned char*>(dst);
+  while (bytes > 0) {
+    TablePiece piece;
+    const size_t take = std::min(bytes, sizeof(piece.v));
+    memset(&piece, 0, sizeof(piece));
+    memcpy(piece.v, from, take);
+    write_table_kernel<<<1, 224, 0, stream>>>(reinterpret_cast<uint4*>(to), piece, int((take + 15) / 16));
+    if (cudaError_t e = cudaGetLastError(); e != cudaSuccess) return e;
+    from += take; to += take; bytes -= take;
+  }
+  return cudaSuccess;
+}
+
 }  // namespace
 
 struct dyspec_plan {
@@ -112,6 +164,8 @@ struct dyspec_plan {
   int64_t total_nodes = 0;
   int max_nodes = 0;
   int regime = 0, bm = 64, bn = 64;
+  int n_sms = kDefaultSMs;              // SMs the scheduler balances over (those of the device current at creation)
+  Tuning tune;                          // the testing knobs as they were when the plan was created
   std::vector<ReqInfo> reqs;
   std::vector<WorkItem> items;          // compact list, CTA by CTA
   std::vector<WorkItem> items_strided;  // device layout: CTA c's items at [c * items_stride, ...)
@@ -179,7 +233,9 @@ void schedule(dyspec_plan& pl) {
   // and all pieces fit in one wave, launch one cluster of C CTAs per group; the pieces are merged
   // through distributed shared memory instead of a round trip through global memory.
   pl.cluster = 1;
-  if (pl.regime == 0 && g_combine_mode == 2 && g_force_ctas <= 0) {
+  const Tuning& tn = pl.tune;
+  const int kNumSMs = pl.n_sms;
+  if (pl.regime == 0 && tn.combine_mode == 2 && tn.force_ctas <= 0) {
     int max_tiles = 0;
     for (const Group& gr : groups) max_tiles = std::max(max_tiles, gr.tiles);
     const double mean_tiles = double(total_tiles) / double(groups.size());
@@ -240,10 +296,10 @@ void schedule(dyspec_plan& pl) {
   }
 
   const int ctas_per_sm = 1;   // one wave: every CTA is resident from the start and owns its SM's load queue
-  int max_ctas = g_force_ctas > 0 ? g_force_ctas : kNumSMs * ctas_per_sm;
+  int max_ctas = tn.force_ctas > 0 ? tn.force_ctas : kNumSMs * ctas_per_sm;
   // fixed per-item overhead (Q load, pipeline fill, epilogue), in key tiles: measured ~1 tile of 64 keys in
   // regime 0 and ~3 tiles of 128 keys in regime 1
-  const int item_cost = g_item_cost > 0 ? g_item_cost : (pl.regime == 0 ? 1 : 3);
+  const int item_cost = tn.item_cost > 0 ? tn.item_cost : (pl.regime == 0 ? 1 : 3);
   const int min_tiles = pl.regime == 0 ? 2 : 2;          // smallest piece worth a split
   const int64_t total_cost = total_tiles + int64_t(groups.size()) * item_cost;
   int64_t target = (total_cost + max_ctas - 1) / max_ctas;
@@ -312,7 +368,7 @@ void schedule(dyspec_plan& pl) {
   // (fp32 rows instead of bf16); the combine launch behind the main kernel three (regime 1: 128-key
   // tiles of ~2 us) or four (regime 0) -- measured on the Llama2-70B shape, where the budgeted plan
   // (136 CTAs, 32 split groups) took 53.5 us and whole groups on 128 CTAs 48.1 us.
-  if (g_whole_groups != 1 && (g_force_ctas <= 0 || g_whole_groups == 2)) {
+  if (tn.whole_groups != 1 && (tn.force_ctas <= 0 || tn.whole_groups == 2)) {
     const int partial_cost = 1, combine_cost = pl.regime == 0 ? 4 : 3;
     int64_t cost_split = 0;
     for (int c = 0; c < pl.n_ctas; ++c) {
@@ -338,7 +394,7 @@ void schedule(dyspec_plan& pl) {
       bins[best].push_back(gi);
     }
     const int64_t cost_whole = *std::max_element(load.begin(), load.end());
-    if (!pl.split_groups.empty() && (cost_whole <= cost_split || g_whole_groups == 2)) {
+    if (!pl.split_groups.empty() && (cost_whole <= cost_split || tn.whole_groups == 2)) {
       pl.items.clear();
       pl.cta_begin.clear();
       pl.split_groups.clear();
@@ -469,18 +525,20 @@ int dyspec_set_tuning(int force_regime, int force_ctas, int combine_mode) {
   const int whole = combine_mode >> 4;
   combine_mode &= 15;
   if (force_regime < -1 || force_regime > 1 || (combine_mode != 0 && combine_mode != 2) || whole > 2) return DYSPEC_ERR_INVALID_ARG;
-  g_whole_groups = whole;
-  g_force_regime = force_regime;
-  g_force_ctas = force_ctas >= 0 ? force_ctas : 0;
-  g_item_cost = force_ctas < 0 ? -force_ctas : 0;   // negative values select the per-item cost instead (experiments)
-  g_combine_mode = combine_mode;
+  std::lock_guard<std::mutex> lock(g_tuning_mutex);
+  g_tuning.whole_groups = whole;
+  g_tuning.force_regime = force_regime;
+  g_tuning.force_ctas = force_ctas >= 0 ? force_ctas : 0;
+  g_tuning.item_cost = force_ctas < 0 ? -force_ctas : 0;   // negative values select the per-item cost instead (experiments)
+  g_tuning.combine_mode = combine_mode;
   return DYSPEC_OK;
 }
 
 int dyspec_set_trace(void* trace_buffer, int capacity_entries) {
   if (capacity_entries < 0 || (trace_buffer == nullptr) != (capacity_entries == 0)) return DYSPEC_ERR_INVALID_ARG;
-  g_trace = static_cast<unsigned long long*>(trace_buffer);
-  g_trace_capacity = capacity_entries;
+  std::lock_guard<std::mutex> lock(g_tuning_mutex);
+  g_tuning.trace = static_cast<unsigned long long*>(trace_buffer);
+  g_tuning.trace_capacity = capacity_entries;
   return DYSPEC_OK;
 }
 
@@ -508,16 +566,27 @@ int dyspec_build_tree_mask_batched(const int32_t* parents, const int32_t* node_o
   if (n_req < 0 || (n_req > 0 && !node_offsets_host)) return DYSPEC_ERR_INVALID_ARG;
   for (int r = 0; r < n_req; ++r)
     if (node_offsets_host[r] < 0 || node_offsets_host[r + 1] < node_offsets_host[r]) return DYSPEC_ERR_INVALID_ARG;
-  // Without a plan there is no device copy of the request list: one launch per request (the kernel of
-  // the single-request call), each on the request's slice of the arrays.  dyspec_plan_build_tree_mask
-  // does the whole batch in one launch.
-  for (int r = 0; r < n_req; ++r) {
-    const int64_t at = node_offsets_host[r];
-    const int n = node_offsets_host[r + 1] - node_offsets_host[r];
-    const int rc = build_tree_mask_checked(parents ? parents + at : nullptr, n, ancestor_bits ? ancestor_bits + at * words_per_row : nullptr,
-                                           depths ? depths + at : nullptr, nullptr, words_per_row, status ? status + r : nullptr,
-                                           stream);
-    if (rc != DYSPEC_OK) return rc;
+  if (n_req == 0 || node_offsets_host[n_req] == 0) return DYSPEC_OK;
+  if (words_per_row <= 0 || (words_per_row & 3)) return DYSPEC_ERR_INVALID_ARG;
+  if (words_per_row > DYSPEC_MAX_NODES / 32) return DYSPEC_ERR_UNSUPPORTED;
+  int max_n = 0;
+  for (int r = 0; r < n_req; ++r) max_n = std::max(max_n, node_offsets_host[r + 1] - node_offsets_host[r]);
+  if (max_n > DYSPEC_MAX_NODES) return DYSPEC_ERR_UNSUPPORTED;
+  if (32 * words_per_row < max_n) return DYSPEC_ERR_INVALID_ARG;
+  if (!parents || !ancestor_bits || !aligned(ancestor_bits, 16) || !aligned(parents, 4)) return DYSPEC_ERR_INVALID_ARG;
+  // Without a plan there is no device copy of the request list: it travels with the launch, in the
+  // kernel's parameter space.  One launch takes up to kMaskBatchMax requests.
+  for (int r0 = 0; r0 < n_req; r0 += kMaskBatchMax) {
+    const int cnt = std::min(kMaskBatchMax, n_req - r0);
+    MaskBatch batch;
+    memset(&batch, 0, sizeof(batch));
+    int piece_max = 0;
+    for (int k = 0; k <= cnt; ++k) batch.node0[k] = node_offsets_host[r0 + k];
+    for (int k = 0; k < cnt; ++k) piece_max = std::max(piece_max, batch.node0[k + 1] - batch.node0[k]);
+    batch.first_req = r0;
+    cudaError_t e = launch_build_tree_mask_batch(parents, batch, cnt, piece_max, ancestor_bits, depths, words_per_row, status,
+                                                 reinterpret_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_failed(e, "batched mask launch");
   }
   return DYSPEC_OK;
 }
@@ -608,7 +677,7 @@ int dyspec_build_tree_threshold(const float* draft_table, int n_rows, int vocab,
 
 int dyspec_compact_kv(void* k_cache, void* v_cache, const int64_t* kv_row_offset, const int32_t* prefix_len,
                       const int32_t* accepted_nodes, const int32_t* n_accepted, int n_req, int max_out, int n_kv_heads,
-                      int head_dim, int32_t* new_prefix_len, dyspec_stream_t stream) {
+                      int head_dim, int keep_root, int32_t* new_prefix_len, dyspec_stream_t stream) {
   if (n_req < 0 || max_out <= 0 || n_kv_heads <= 0 || head_dim <= 0) return DYSPEC_ERR_INVALID_ARG;
   const int64_t row_bytes = int64_t(n_kv_heads) * head_dim * 2;
   if (row_bytes % 16 != 0 || row_bytes > (1 << 24)) return DYSPEC_ERR_UNSUPPORTED;
@@ -616,14 +685,14 @@ int dyspec_compact_kv(void* k_cache, void* v_cache, const int64_t* kv_row_offset
   if (!k_cache || !v_cache || !kv_row_offset || !prefix_len || !accepted_nodes || !n_accepted) return DYSPEC_ERR_INVALID_ARG;
   if (!aligned(k_cache, 16) || !aligned(v_cache, 16)) return DYSPEC_ERR_INVALID_ARG;
   cudaError_t e = launch_compact_kv(k_cache, v_cache, kv_row_offset, prefix_len, accepted_nodes, n_accepted, n_req, max_out,
-                                    int(row_bytes), new_prefix_len, reinterpret_cast<cudaStream_t>(stream));
+                                    int(row_bytes), keep_root != 0, new_prefix_len, reinterpret_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? DYSPEC_OK : cuda_failed(e, "compact launch");
 }
 
 int dyspec_compact_kv_paged(void* k_cache, void* v_cache, const int64_t* tree_row_offset, const int32_t* page_table,
                             int pages_per_req, int page_size, const int32_t* prefix_len, const int32_t* accepted_nodes,
                             const int32_t* n_accepted, int n_req, int max_out, int n_kv_heads, int head_dim,
-                            int32_t* new_prefix_len, int32_t* status, dyspec_stream_t stream) {
+                            int keep_root, int32_t* new_prefix_len, int32_t* status, dyspec_stream_t stream) {
   if (n_req < 0 || max_out <= 0 || n_kv_heads <= 0 || head_dim <= 0 || pages_per_req <= 0) return DYSPEC_ERR_INVALID_ARG;
   if (page_size <= 0 || (page_size & (page_size - 1))) return DYSPEC_ERR_INVALID_ARG;
   const int64_t row_bytes = int64_t(n_kv_heads) * head_dim * 2;
@@ -635,7 +704,7 @@ int dyspec_compact_kv_paged(void* k_cache, void* v_cache, const int64_t* tree_ro
   int shift = 0;
   while ((1 << shift) < page_size) ++shift;
   cudaError_t e = launch_compact_kv_paged(k_cache, v_cache, tree_row_offset, page_table, pages_per_req, shift, prefix_len,
-                                          accepted_nodes, n_accepted, n_req, max_out, int(row_bytes), new_prefix_len,
+                                          accepted_nodes, n_accepted, n_req, max_out, int(row_bytes), keep_root != 0, new_prefix_len,
                                           status, reinterpret_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? DYSPEC_OK : cuda_failed(e, "paged compact launch");
 }
@@ -685,7 +754,9 @@ static int make_host_plan(dyspec_plan** out, int n_q_heads, int n_kv_heads, int 
   pl->total_nodes = node0;
   // Regime: tcgen05 tiles (2 x 128 packed rows per item) when some request has more packed rows
   // (nodes x group) than one warp-level tile holds, else warp-level tiles (64 packed rows).
-  pl->regime = g_force_regime >= 0 ? g_force_regime : (max_rows > 64 ? 1 : 0);
+  pl->tune = current_tuning();
+  pl->n_sms = device_sm_count();
+  pl->regime = pl->tune.force_regime >= 0 ? pl->tune.force_regime : (max_rows > 64 ? 1 : 0);
   pl->bm = pl->regime == 0 ? 64 : 256;    // packed query rows per work item (regime 1: two 128-row halves)
   pl->bn = pl->regime == 0 ? 64 : 128;    // keys per tile
   schedule(*pl);
@@ -890,12 +961,15 @@ static int run_attention(const dyspec_plan_t* plan, const void* q, const void* k
   p.scale_log2e = plan->scale * kLog2e;
   p.items_stride = plan->items_stride;
   p.cluster_size = plan->cluster;
-  p.trace = g_trace; p.trace_capacity = g_trace_capacity;
+  {
+    const Tuning now = current_tuning();
+    p.trace = now.trace; p.trace_capacity = now.trace_capacity;
+  }
   p.page_table = page_table; p.pages_per_req = pages_per_req;
   for (p.page_shift = 0; page_table && (1 << p.page_shift) < plan->page_size; ++p.page_shift) {}
 
   cudaError_t e;
-  if (plan->regime == 0) e = launch_attn_mma(plan->d, plan->n_ctas, mq, mk, mv, p, plan->items_strided.data(), st);
+  if (plan->regime == 0) e = launch_attn_small(plan->d, plan->n_ctas, mq, mk, mv, p, plan->items_strided.data(), st);
   else e = launch_attn_tc(plan->d, plan->n_ctas, mq, mk, mv, p, st);
   if (e != cudaSuccess) return cuda_failed(e, "attention launch");
   e = launch_combine(plan->d, bm, int(plan->split_groups.size()), p, st);
@@ -903,13 +977,55 @@ static int run_attention(const dyspec_plan_t* plan, const void* q, const void* k
 }
 
 // ---- single-request convenience form -------------------------------------------------------------
+//
+// In a decoding loop the prefix grows and the tree changes at every step, but all layers of a step
+// share one (prefix_len, n_nodes).  So the cache is small and bounded: per (device, static shape) a
+// handful of slots, each a host plan plus a device table buffer that is reused when the slot is
+// recycled (least recently used first), and ONE workspace sized for the worst case of that shape (a
+// plan never has more than two split pieces per CTA).  A miss runs the host scheduler and sends the
+// tables down the stream in kernel parameters: no allocation, no synchronisation, after the first calls.
 namespace {
 struct DefaultShape { int hq = 0, hkv = 0, d = 0, W = 0; float scale = 0.f; };
 DefaultShape g_shape;
-struct Cached { dyspec_plan* plan; void* workspace; };
-// keyed by device, static shape, scale (bit pattern) and (prefix_len, n_nodes): a plan belongs to one device
-std::map<std::tuple<int, int, int, int, int, uint32_t, int, int>, Cached> g_cache;
+constexpr int kSingleSlots = 8;
+struct SingleSlot {
+  dyspec_plan* plan = nullptr;          // host object; its device tables live in `blob`
+  int prefix_len = -1, n_nodes = -1;
+  uint64_t used = 0;                    // for least-recently-used replacement
+  void* blob = nullptr;
+  size_t blob_bytes = 0;
+};
+struct ShapeCache {
+  SingleSlot slot[kSingleSlots];
+  void* workspace = nullptr;
+  size_t workspace_bytes = 0;
+  uint64_t clock = 0;
+};
+// keyed by device, static shape and scale (bit pattern)
+std::map<std::tuple<int, int, int, int, int, uint32_t>, ShapeCache> g_cache;
 std::mutex g_cache_mutex;
+
+// Places the plan's tables in `blob` (laid out as upload() does) through the stream.
+int send_tables(dyspec_plan& pl, void* blob, size_t blob_bytes, cudaStream_t st, size_t* needed) {
+  auto pad = [](size_t x) { return (x + 255) & ~size_t(255); };
+  const size_t b_reqs = pad(std::max<size_t>(1, pl.reqs.size()) * sizeof(ReqInfo));
+  const size_t b_items = pad(std::max<size_t>(1, pl.items_strided.size()) * sizeof(WorkItem));
+  const size_t b_groups = pad(std::max<size_t>(1, pl.split_groups.size()) * sizeof(GroupInfo));
+  const size_t b_counters = pad(std::max<size_t>(1, pl.split_groups.size()) * sizeof(int32_t));
+  *needed = b_reqs + b_items + b_groups + b_counters;
+  if (!blob || blob_bytes < *needed) return DYSPEC_ERR_WORKSPACE;
+  uint8_t* base = static_cast<uint8_t*>(blob);
+  pl.d_reqs = reinterpret_cast<ReqInfo*>(base);
+  pl.d_items = reinterpret_cast<WorkItem*>(base + b_reqs);
+  pl.d_groups = reinterpret_cast<GroupInfo*>(base + b_reqs + b_items);
+  pl.d_counters = reinterpret_cast<int32_t*>(base + b_reqs + b_items + b_groups);
+  if (write_table(pl.d_reqs, pl.reqs.data(), pl.reqs.size() * sizeof(ReqInfo), st) != cudaSuccess ||
+      write_table(pl.d_items, pl.items_strided.data(), pl.items_strided.size() * sizeof(WorkItem), st) != cudaSuccess ||
+      write_table(pl.d_groups, pl.split_groups.data(), pl.split_groups.size() * sizeof(GroupInfo), st) != cudaSuccess ||
+      cudaMemsetAsync(pl.d_counters, 0, b_counters, st) != cudaSuccess)
+    return DYSPEC_ERR_CUDA;
+  return DYSPEC_OK;
+}
 }  // namespace
 
 int dyspec_set_default_shape(int n_q_heads, int n_kv_heads, int head_dim, int words_per_row, float scale) {
@@ -922,39 +1038,74 @@ int dyspec_set_default_shape(int n_q_heads, int n_kv_heads, int head_dim, int wo
   return DYSPEC_OK;
 }
 
+int dyspec_release_cache(void) {
+  std::lock_guard<std::mutex> lock(g_cache_mutex);
+  int dev0 = -1;
+  cudaGetDevice(&dev0);
+  for (auto& kv : g_cache) {
+    if (cudaSetDevice(std::get<0>(kv.first)) != cudaSuccess) continue;
+    for (SingleSlot& sl : kv.second.slot) {
+      delete sl.plan;                    // host only: its tables are in the slot's buffer
+      if (sl.blob) cudaFree(sl.blob);
+    }
+    if (kv.second.workspace) cudaFree(kv.second.workspace);
+  }
+  g_cache.clear();
+  if (dev0 >= 0) cudaSetDevice(dev0);
+  return DYSPEC_OK;
+}
+
 int dyspec_tree_attention(const void* q, const void* k_cache, const void* v_cache, int prefix_len,
                           const uint32_t* ancestor_bits, int n_nodes, void* out, dyspec_stream_t stream) {
-  Cached c{};
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess) return DYSPEC_ERR_CUDA;
-  {
-    std::lock_guard<std::mutex> lock(g_cache_mutex);
-    if (g_shape.hq == 0) return DYSPEC_ERR_INVALID_ARG;
-    if (prefix_len < 0 || n_nodes < 0) return DYSPEC_ERR_INVALID_ARG;
-    uint32_t scale_bits;
-    memcpy(&scale_bits, &g_shape.scale, 4);
-    const auto key = std::make_tuple(dev, g_shape.hq, g_shape.hkv, g_shape.d, g_shape.W, scale_bits, prefix_len, n_nodes);
-    auto it = g_cache.find(key);
-    if (it == g_cache.end()) {
-      const int32_t L = prefix_len, n = n_nodes;
-      const int64_t off = 0;
-      dyspec_plan* pl = nullptr;
-      int rc = dyspec_plan_create(&pl, g_shape.hq, g_shape.hkv, g_shape.d, 1, &L, &n, &off, int64_t(L) + n, g_shape.W,
-                                  g_shape.scale);
-      if (rc != DYSPEC_OK) return rc;
-      void* ws = nullptr;
-      if (pl->workspace_bytes > 0 &&
-          (cudaMalloc(&ws, pl->workspace_bytes) != cudaSuccess || cudaMemset(ws, 0, pl->workspace_bytes) != cudaSuccess)) {
-        if (ws) cudaFree(ws);
-        dyspec_plan_destroy(pl);
-        return DYSPEC_ERR_CUDA;
-      }
-      it = g_cache.emplace(key, Cached{pl, ws}).first;
-    }
-    c = it->second;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  std::lock_guard<std::mutex> lock(g_cache_mutex);      // held across the launch: the slot must not be recycled under it
+  if (g_shape.hq == 0) return DYSPEC_ERR_INVALID_ARG;
+  if (prefix_len < 0 || n_nodes < 0) return DYSPEC_ERR_INVALID_ARG;
+  uint32_t scale_bits;
+  memcpy(&scale_bits, &g_shape.scale, 4);
+  ShapeCache& sc = g_cache[std::make_tuple(dev, g_shape.hq, g_shape.hkv, g_shape.d, g_shape.W, scale_bits)];
+  SingleSlot* hit = nullptr;
+  SingleSlot* lru = &sc.slot[0];
+  for (SingleSlot& sl : sc.slot) {
+    if (sl.plan && sl.prefix_len == prefix_len && sl.n_nodes == n_nodes) hit = &sl;
+    if (sl.used < lru->used) lru = &sl;
   }
-  return dyspec_tree_attention_ragged(c.plan, q, k_cache, v_cache, ancestor_bits, out, c.workspace,
-                                      c.plan->workspace_bytes, nullptr, stream);
+  if (!hit) {
+    const int32_t L = prefix_len, n = n_nodes;
+    const int64_t off = 0;
+    dyspec_plan* pl = nullptr;
+    // fixed work lists only: the one workspace is shared by every plan of the shape, so there is no place
+    // for a queue head that stays zero between launches of different plans
+    int rc = make_host_plan(&pl, g_shape.hq, g_shape.hkv, g_shape.d, 1, &L, &n, &off, int64_t(L) + n, g_shape.W,
+                            g_shape.scale, 0, false);
+    if (rc != DYSPEC_OK) return rc;
+    pl->device = dev;
+    if (!sc.workspace) {                 // once per (device, shape): at most two split pieces per CTA, 256-row tiles
+      const size_t worst = size_t(2) * size_t(pl->n_sms) * 256 * size_t(g_shape.d + 2) * sizeof(float) + 512;
+      if (cudaMalloc(&sc.workspace, worst) != cudaSuccess) { sc.workspace = nullptr; delete pl; return DYSPEC_ERR_CUDA; }
+      if (cudaMemsetAsync(sc.workspace, 0, worst, st) != cudaSuccess) { delete pl; return DYSPEC_ERR_CUDA; }
+      sc.workspace_bytes = worst;
+    }
+    if (pl->workspace_bytes > sc.workspace_bytes) { delete pl; return DYSPEC_ERR_WORKSPACE; }   // cannot happen (see above)
+    size_t needed = 0;
+    rc = send_tables(*pl, lru->blob, lru->blob_bytes, st, &needed);
+    if (rc == DYSPEC_ERR_WORKSPACE) {    // the slot's table buffer is too small (or not there yet): replace it
+      if (lru->blob) cudaFree(lru->blob);              // (synchronises: nothing in flight reads it afterwards)
+      lru->blob = nullptr;
+      lru->blob_bytes = std::max<size_t>(needed, size_t(64) << 10);
+      if (cudaMalloc(&lru->blob, lru->blob_bytes) != cudaSuccess) { lru->blob = nullptr; lru->blob_bytes = 0; delete pl; return DYSPEC_ERR_CUDA; }
+      rc = send_tables(*pl, lru->blob, lru->blob_bytes, st, &needed);
+    }
+    if (rc != DYSPEC_OK) { delete pl; return rc; }
+    delete lru->plan;
+    lru->plan = pl; lru->prefix_len = prefix_len; lru->n_nodes = n_nodes;
+    hit = lru;
+  }
+  hit->used = ++sc.clock;
+  return dyspec_tree_attention_ragged(hit->plan, q, k_cache, v_cache, ancestor_bits, out, sc.workspace,
+                                      sc.workspace_bytes, nullptr, stream);
 }
 
 }  // extern "C"
@@ -1022,14 +1173,14 @@ extern "C" int dyspec_tree_attention_static(const void* q, const void* k_cache, 
   if (rc != DYSPEC_OK) return rc;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
 
-  // The array keeps whatever the previous call left: rewrite the tables, clear the counters.
-  std::vector<uint8_t> host(o_partial, 0);
-  memcpy(host.data() + o_reqs, pl->reqs.data(), pl->reqs.size() * sizeof(ReqInfo));
-  memcpy(host.data() + o_items, pl->items_strided.data(), pl->items_strided.size() * sizeof(WorkItem));
-  if (!pl->split_groups.empty())
-    memcpy(host.data() + o_groups, pl->split_groups.data(), pl->split_groups.size() * sizeof(GroupInfo));
-  // pageable source: the copy is staged before the call returns, so `host` may go out of scope afterwards
-  if (cudaMemcpyAsync(base, host.data(), o_partial, cudaMemcpyHostToDevice, st) != cudaSuccess) return DYSPEC_ERR_CUDA;
+  // The array keeps whatever the previous call left: rewrite the tables, clear the counters.  The tables
+  // travel in kernel parameters (write_table), so nothing on the device ever refers to this call's host memory.
+  if (write_table(base + o_reqs, pl->reqs.data(), pl->reqs.size() * sizeof(ReqInfo), st) != cudaSuccess ||
+      write_table(base + o_items, pl->items_strided.data(), pl->items_strided.size() * sizeof(WorkItem), st) != cudaSuccess ||
+      (!pl->split_groups.empty() &&
+       write_table(base + o_groups, pl->split_groups.data(), pl->split_groups.size() * sizeof(GroupInfo), st) != cudaSuccess))
+    return DYSPEC_ERR_CUDA;
+  if (cudaMemsetAsync(base + o_counters, 0, o_partial - o_counters, st) != cudaSuccess) return DYSPEC_ERR_CUDA;
 
   CUtensorMap mq, mk, mv;
   const int bm = pl->bm, bn = pl->bn;
@@ -1053,7 +1204,7 @@ extern "C" int dyspec_tree_attention_static(const void* q, const void* k_cache, 
   p.cluster_size = pl->cluster;
 
   cudaError_t e;
-  if (pl->regime == 0) e = launch_attn_mma(pl->d, pl->n_ctas, mq, mk, mv, p, pl->items_strided.data(), st);
+  if (pl->regime == 0) e = launch_attn_small(pl->d, pl->n_ctas, mq, mk, mv, p, pl->items_strided.data(), st);
   else e = launch_attn_tc(pl->d, pl->n_ctas, mq, mk, mv, p, st);
   if (e != cudaSuccess) return DYSPEC_ERR_CUDA;
   e = launch_combine(pl->d, bm, int(pl->split_groups.size()), p, st);

@@ -13,8 +13,8 @@
 //              commit behind it frees the ring stage;
 //   warps 0-7  two sets of four compute warps (16 query rows per warp).  The sets take alternate key
 //              tiles: a warp reads its 16 x 64 scores with tcgen05.ld (with M = 64 accumulator row r
-//              lives in lane 32 (r / 16) + r % 16, and the 16x256b shape returns the rows laid out like
-//              an mma.sync accumulator), applies the ancestor bitmask on tree tiles and runs the fp32
+//              lives in lane 32 (r / 16) + r % 16, and the 16x256b shape gives lane (gid, tig) the column
+//              pairs 8 j + 2 tig of rows gid and gid + 8), applies the ancestor bitmask on tree tiles and runs the fp32
 //              online softmax in the exp2 domain against a LAZY reference: the accumulator is rescaled
 //              (tcgen05.ld / st) only when a row maximum has grown by more than 2^8.  The per-tile code
 //              is a chain of dependent instructions, so one warp per scheduler leaves the SM mostly
@@ -83,9 +83,9 @@ __device__ __forceinline__ uint32_t desc_lo(uint32_t saddr) { return (saddr >> 4
 // Instruction descriptor, kind::f16: bf16 x bf16 -> fp32, both operands K-major, M = 64, N = 64.
 constexpr uint32_t kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(BN >> 3) << 17) | (uint32_t(BM >> 4) << 24);
 // With M = 64 the accumulator row r lives in TMEM lane 32 (r / 16) + r % 16, so warp w reads rows
-// 16 w .. 16 w + 15 from its own lane quarter, and the 16x256b load shape hands them out exactly as
-// mma.sync hands out a 16 x 8 accumulator tile: registers 4j .. 4j+3 of lane (gid, tig) are
-// (row gid, columns 8j + 2 tig, +1) and (row gid + 8, same columns).
+// 16 w .. 16 w + 15 from its own lane quarter, and the 16x256b load shape hands them out in 16 x 8
+// fragments: registers 4j .. 4j+3 of lane (gid = lane / 4, tig = lane % 4) are (row gid, columns
+// 8j + 2 tig, +1) and (row gid + 8, same columns).
 __device__ __forceinline__ void tmem_ld_scores(uint32_t taddr, float (&s)[BN / 8][4]) {
   uint32_t r[32];
   asm volatile(
@@ -146,7 +146,7 @@ __device__ __forceinline__ void tmem_st_rows(uint32_t taddr, const float (&v)[NJ
 
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
-tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+tree_attn_small_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                      const __grid_constant__ CUtensorMap map_v, const AttnParams p,
                      const __grid_constant__ FirstItems first) {
   using L = SmemLayout<D>;
@@ -763,18 +763,18 @@ tree_attn_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   }
 }
 
-size_t attn_mma_smem_bytes(int head_dim) {
+size_t attn_small_smem_bytes(int head_dim) {
   return (head_dim == 128 ? SmemLayout<128>::kTotal : SmemLayout<64>::kTotal) + 1024;
 }
-int attn_mma_threads() { return kThreads; }
+int attn_small_threads() { return kThreads; }
 
-cudaError_t launch_attn_mma(int head_dim, int n_ctas, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
+cudaError_t launch_attn_small(int head_dim, int n_ctas, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                             const AttnParams& p, const WorkItem* host_items, cudaStream_t stream) {
   // host_items: the host copy of p.items (same stride); each CTA's first item travels as a kernel parameter
   FirstItems first;
   for (int c = 0; c < kFirstItems; ++c)
     first.item[c] = c < n_ctas ? host_items[size_t(c) * p.items_stride] : WorkItem{};
-  const size_t smem = attn_mma_smem_bytes(head_dim);
+  const size_t smem = attn_small_smem_bytes(head_dim);
   static DynSmemGrant grant[2];
   cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -791,13 +791,13 @@ cudaError_t launch_attn_mma(int head_dim, int n_ctas, const CUtensorMap& mq, con
   cfg.numAttrs = p.cluster_size > 1 ? 2 : 1;
   cudaError_t e = cudaSuccess;
   if (head_dim == 128) {
-    if (cudaError_t ge = grant[0].ensure(tree_attn_mma_kernel<128>, smem); ge != cudaSuccess) return ge;
+    if (cudaError_t ge = grant[0].ensure(tree_attn_small_kernel<128>, smem); ge != cudaSuccess) return ge;
     cfg.dynamicSmemBytes = smem;
-    e = cudaLaunchKernelEx(&cfg, tree_attn_mma_kernel<128>, mq, mk, mv, p, first);
+    e = cudaLaunchKernelEx(&cfg, tree_attn_small_kernel<128>, mq, mk, mv, p, first);
   } else {
-    if (cudaError_t ge = grant[1].ensure(tree_attn_mma_kernel<64>, smem); ge != cudaSuccess) return ge;
+    if (cudaError_t ge = grant[1].ensure(tree_attn_small_kernel<64>, smem); ge != cudaSuccess) return ge;
     cfg.dynamicSmemBytes = smem;
-    e = cudaLaunchKernelEx(&cfg, tree_attn_mma_kernel<64>, mq, mk, mv, p, first);
+    e = cudaLaunchKernelEx(&cfg, tree_attn_small_kernel<64>, mq, mk, mv, p, first);
   }
   return e != cudaSuccess ? e : cudaGetLastError();
 }

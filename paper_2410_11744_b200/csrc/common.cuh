@@ -11,7 +11,7 @@
 
 namespace dyspec {
 
-constexpr int kNumSMs = 148;            // B200: 2 dies x 74 SMs
+constexpr int kDefaultSMs = 148;        // B200: 2 dies x 74 SMs (the scheduler asks the device; this is the fallback)
 constexpr float kLog2e = 1.4426950408889634f;
 
 // One verification request, device-side view.
@@ -45,7 +45,7 @@ struct WorkItem {
   int32_t slot0;       // first partial slot of the group (slots slot0 .. slot0 + n_splits - 1)
   int32_t n_in_cta;    // in the first item of a CTA: how many items the CTA owns
   int32_t req;         // request index
-  int32_t merge_owners;  // cluster mode: bit k set = CTA k of the cluster merges a share of the rows (see attn_mma.cu)
+  int32_t merge_owners;  // cluster mode: bit k set = CTA k of the cluster merges a share of the rows (see attn_small.cu)
 };
 static_assert(sizeof(WorkItem) == 64, "WorkItem is one 64-byte record");
 
@@ -53,6 +53,15 @@ static_assert(sizeof(WorkItem) == 64, "WorkItem is one 64-byte record");
 // a CTA then knows its first item without a global-memory round trip in front of its first loads.
 constexpr int kFirstItems = 148;
 struct FirstItems { WorkItem item[kFirstItems]; };
+
+// Request list of a ragged mask-builder call without a plan, passed by value: request k of the launch
+// owns nodes node0[k] .. node0[k + 1] - 1; first_req = index of the launch's first request in the batch
+// (its status word).
+constexpr int kMaskBatchMax = 768;
+struct MaskBatch {
+  int32_t node0[kMaskBatchMax + 1];
+  int32_t first_req;
+};
 
 // A split query-tile group, for the combine step.
 struct GroupInfo {

@@ -1,8 +1,11 @@
 // Keeping the accepted path in the KV cache after verification: for each request, the tree rows of the
 // accepted nodes a_0 < a_1 < ... move to the rows right after the prefix (row L + i <- row L + a_i), in
-// place, for K and V, and the prefix length grows by their number.
+// place, for K and V, and the prefix length grows by their number.  With keep_root the walk's start node
+// (tree row 0: the last decoded token, whose K/V this step computed) is kept in front of them: it is in
+// place already, the accepted nodes follow it (row L + 1 + i <- row L + a_i).
 //
-// a_i >= i, so a destination never lies behind its own source, but it can be an EARLIER step's
+// a_i >= i (>= i + 1 with keep_root: the accepted nodes are proper descendants of node 0), so a
+// destination never lies behind its own source, but it can be an EARLIER step's
 // source (path 1, 2, 3: slot 1 receives node 2 after it has given node 1 away).  A thread owns fixed
 // 16-byte columns of a row and walks the steps in order, so for any byte the read of step i precedes
 // the write of step i + 1 in program order, and no two threads ever touch the same byte: no barriers.
@@ -15,7 +18,8 @@ namespace dyspec {
 __global__ void __launch_bounds__(256)
 compact_kv_kernel(uint4* __restrict__ k_cache, uint4* __restrict__ v_cache, const int64_t* __restrict__ kv_row_offset,
                   const int32_t* __restrict__ prefix_len, const int32_t* __restrict__ accepted_nodes,
-                  const int32_t* __restrict__ n_accepted, int max_out, int row_vecs, int32_t* __restrict__ new_prefix_len) {
+                  const int32_t* __restrict__ n_accepted, int max_out, int row_vecs, int keep_root,
+                  int32_t* __restrict__ new_prefix_len) {
   const int r = blockIdx.x;
   uint4* cache = blockIdx.z == 0 ? k_cache : v_cache;
   const int L = prefix_len[r];
@@ -23,7 +27,7 @@ compact_kv_kernel(uint4* __restrict__ k_cache, uint4* __restrict__ v_cache, cons
   const int n = min(n_accepted[r], max_out);
   const int32_t* acc = accepted_nodes + size_t(r) * max_out;
   const int col = blockIdx.y * blockDim.x + threadIdx.x;
-  int kept = 0;
+  int kept = (keep_root && n > 0) ? 1 : 0;          // the root's row is where it belongs already
   for (int i = 0; i < n; ++i) {
     const int a = acc[i];
     if (a < 0 || a >= DYSPEC_MAX_NODES) continue;   // an emitted token without a tree node (or not a node index at all)
@@ -41,7 +45,7 @@ __global__ void __launch_bounds__(256)
 compact_kv_paged_kernel(uint4* __restrict__ k_cache, uint4* __restrict__ v_cache, const int64_t* __restrict__ tree_row_offset,
                         const int32_t* __restrict__ page_table, int pages_per_req, int page_shift,
                         const int32_t* __restrict__ prefix_len, const int32_t* __restrict__ accepted_nodes,
-                        const int32_t* __restrict__ n_accepted, int max_out, int row_vecs,
+                        const int32_t* __restrict__ n_accepted, int max_out, int row_vecs, int keep_root,
                         int32_t* __restrict__ new_prefix_len, int32_t* __restrict__ status) {
   const int r = blockIdx.x;
   uint4* cache = blockIdx.z == 0 ? k_cache : v_cache;
@@ -52,8 +56,9 @@ compact_kv_paged_kernel(uint4* __restrict__ k_cache, uint4* __restrict__ v_cache
   const int32_t* pages = page_table + size_t(r) * pages_per_req;
   const int col = blockIdx.y * blockDim.x + threadIdx.x;
   int kept = 0;
-  for (int i = 0; i < n; ++i) {
-    const int a = acc[i];
+  const int first = (keep_root && n > 0) ? -1 : 0;  // step -1 moves the root's row (tree row 0) to token L
+  for (int i = first; i < n; ++i) {
+    const int a = i < 0 ? 0 : acc[i];
     if (a < 0 || a >= DYSPEC_MAX_NODES) continue;   // an emitted token without a tree node (or not a node index at all)
     const int t = L + kept;
     const int pi = t >> page_shift;
@@ -74,24 +79,25 @@ compact_kv_paged_kernel(uint4* __restrict__ k_cache, uint4* __restrict__ v_cache
 cudaError_t launch_compact_kv_paged(void* k_cache, void* v_cache, const int64_t* tree_row_offset, const int32_t* page_table,
                                     int pages_per_req, int page_shift, const int32_t* prefix_len,
                                     const int32_t* accepted_nodes, const int32_t* n_accepted, int n_req, int max_out,
-                                    int row_bytes, int32_t* new_prefix_len, int32_t* status, cudaStream_t stream) {
+                                    int row_bytes, int keep_root, int32_t* new_prefix_len, int32_t* status,
+                                    cudaStream_t stream) {
   if (n_req <= 0) return cudaSuccess;
   const int row_vecs = row_bytes / 16;
   const dim3 grid(unsigned(n_req), unsigned((row_vecs + 255) / 256), 2u);
   compact_kv_paged_kernel<<<grid, 256, 0, stream>>>(static_cast<uint4*>(k_cache), static_cast<uint4*>(v_cache),
                                                     tree_row_offset, page_table, pages_per_req, page_shift, prefix_len,
-                                                    accepted_nodes, n_accepted, max_out, row_vecs, new_prefix_len, status);
+                                                    accepted_nodes, n_accepted, max_out, row_vecs, keep_root, new_prefix_len, status);
   return cudaGetLastError();
 }
 
 cudaError_t launch_compact_kv(void* k_cache, void* v_cache, const int64_t* kv_row_offset, const int32_t* prefix_len,
                               const int32_t* accepted_nodes, const int32_t* n_accepted, int n_req, int max_out,
-                              int row_bytes, int32_t* new_prefix_len, cudaStream_t stream) {
+                              int row_bytes, int keep_root, int32_t* new_prefix_len, cudaStream_t stream) {
   if (n_req <= 0) return cudaSuccess;
   const int row_vecs = row_bytes / 16;
   const dim3 grid(unsigned(n_req), unsigned((row_vecs + 255) / 256), 2u);
   compact_kv_kernel<<<grid, 256, 0, stream>>>(static_cast<uint4*>(k_cache), static_cast<uint4*>(v_cache), kv_row_offset,
-                                              prefix_len, accepted_nodes, n_accepted, max_out, row_vecs, new_prefix_len);
+                                              prefix_len, accepted_nodes, n_accepted, max_out, row_vecs, keep_root, new_prefix_len);
   return cudaGetLastError();
 }
 

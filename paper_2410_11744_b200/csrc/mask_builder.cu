@@ -19,17 +19,12 @@
 
 namespace dyspec {
 
-__global__ void __launch_bounds__(1024, 1)
-build_tree_mask_kernel(const int32_t* __restrict__ parents, const ReqInfo* __restrict__ reqs, int single_n,
-                       uint32_t* __restrict__ bits, int32_t* __restrict__ depths, uint32_t* __restrict__ node_tiles,
-                       int W, int CW, int32_t* status) {
+// The work of one CTA: request (node0, n), column chunk blockIdx.y.
+__device__ __forceinline__ void build_tree_mask_body(const int32_t* __restrict__ parents, int node0, int n,
+                                                     uint32_t* __restrict__ bits, int32_t* __restrict__ depths,
+                                                     uint32_t* __restrict__ node_tiles, int W, int CW, int32_t* status) {
   extern __shared__ __align__(16) uint8_t mask_smem[];
   trigger_dependents();   // the attention kernel may start streaming K/V now; it waits for us before it reads the mask
-  int node0 = 0, n = single_n;
-  if (reqs != nullptr) {
-    node0 = reqs[blockIdx.x].node0;
-    n = reqs[blockIdx.x].n_nodes;
-  }
   if (n <= 0) return;
   const int chunk = blockIdx.y;
   const int W4 = W >> 2, CW4 = min(CW, W - chunk * CW) >> 2;               // 16-byte groups per row: all, this chunk's
@@ -135,18 +130,71 @@ build_tree_mask_kernel(const int32_t* __restrict__ parents, const ReqInfo* __res
   }
 }
 
+// Request list in a plan's device table (or one request given by its size).
+__global__ void __launch_bounds__(1024, 1)
+build_tree_mask_kernel(const int32_t* __restrict__ parents, const ReqInfo* __restrict__ reqs, int single_n,
+                       uint32_t* __restrict__ bits, int32_t* __restrict__ depths, uint32_t* __restrict__ node_tiles,
+                       int W, int CW, int32_t* status) {
+  int node0 = 0, n = single_n;
+  if (reqs != nullptr) {
+    node0 = reqs[blockIdx.x].node0;
+    n = reqs[blockIdx.x].n_nodes;
+  }
+  build_tree_mask_body(parents, node0, n, bits, depths, node_tiles, W, CW, status);
+}
+
+// Request list passed by value (kernel parameter space): a ragged batch without a plan, one launch for
+// up to kMaskBatchMax requests, one status word per request.
+__global__ void __launch_bounds__(1024, 1)
+build_tree_mask_batch_kernel(const int32_t* __restrict__ parents, const __grid_constant__ MaskBatch batch,
+                             uint32_t* __restrict__ bits, int32_t* __restrict__ depths, int W, int CW, int32_t* status) {
+  const int node0 = batch.node0[blockIdx.x], n = batch.node0[blockIdx.x + 1] - node0;
+  build_tree_mask_body(parents, node0, n, bits, depths, nullptr, W, CW, status ? status + batch.first_req + blockIdx.x : nullptr);
+}
+
+namespace {
+struct MaskLaunch { int CW, n_chunks, threads; size_t smem; };
+MaskLaunch mask_launch_shape(int max_n, int W) {
+  MaskLaunch m;
+  m.CW = W <= 32 ? W : 16;                 // words per column chunk
+  m.n_chunks = (W + m.CW - 1) / m.CW;
+  m.smem = size_t(max_n) * m.CW * 4 + size_t(max_n) * 12;
+  m.threads = ((max_n + 31) / 32) * 32;
+  if (m.threads < 256) m.threads = 256;
+  if (m.threads > 1024) m.threads = 1024;
+  return m;
+}
+}  // namespace
+
+cudaError_t launch_build_tree_mask_batch(const int32_t* parents, const MaskBatch& batch, int n_req, int max_n, uint32_t* bits,
+                                         int32_t* depths, int W, int32_t* status, cudaStream_t stream) {
+  if (n_req <= 0 || max_n <= 0) return cudaSuccess;
+  const MaskLaunch m = mask_launch_shape(max_n, W);
+  static DynSmemGrant grant;
+  if (cudaError_t e = grant.ensure(build_tree_mask_batch_kernel, m.smem); e != cudaSuccess) return e;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(unsigned(n_req), unsigned(m.n_chunks));
+  cfg.blockDim = dim3(unsigned(m.threads));
+  cfg.dynamicSmemBytes = m.smem;
+  cfg.stream = stream;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, build_tree_mask_batch_kernel, parents, batch, bits, depths, W, m.CW, status);
+  return e != cudaSuccess ? e : cudaGetLastError();
+}
+
 cudaError_t launch_build_tree_mask(const int32_t* parents, const ReqInfo* reqs, int n_req, int single_n, int max_n,
                                    uint32_t* bits, int32_t* depths, uint32_t* node_tiles, int W, int32_t* status,
                                    cudaStream_t stream) {
   if (n_req <= 0 || max_n <= 0) return cudaSuccess;
-  const int CW = W <= 32 ? W : 16;                 // words per column chunk
-  const int n_chunks = (W + CW - 1) / CW;
-  const size_t smem = size_t(max_n) * CW * 4 + size_t(max_n) * 12;
+  const MaskLaunch ml = mask_launch_shape(max_n, W);
+  const int CW = ml.CW, n_chunks = ml.n_chunks, threads = ml.threads;
+  const size_t smem = ml.smem;
   static DynSmemGrant grant;
   if (cudaError_t e = grant.ensure(build_tree_mask_kernel, smem); e != cudaSuccess) return e;
-  int threads = ((max_n + 31) / 32) * 32;
-  if (threads < 256) threads = 256;
-  if (threads > 1024) threads = 1024;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;

@@ -139,8 +139,9 @@ def test_paged_argument_checks(rt):
     torch.cuda.synchronize()
 
 
+@pytest.mark.parametrize("keep_root", [False, True])
 @pytest.mark.parametrize("hkv,d,page_size", [(8, 128, 128), (2, 64, 16), (1, 8, 4)])
-def test_paged_compaction_matches_oracle(rt, hkv, d, page_size):
+def test_paged_compaction_matches_oracle(rt, hkv, d, page_size, keep_root):
     import torch
     B, _ = rt
     rng = np.random.default_rng(hkv + d + page_size)
@@ -154,22 +155,24 @@ def test_paged_compaction_matches_oracle(rt, hkv, d, page_size):
     acc = np.full((n_req, max_out), -7, dtype=np.int32)
     cnt = np.zeros(n_req, dtype=np.int32)
     for r in range(n_req):
-        m = int(rng.integers(0, min(max_out - 1, ns[r]) + 1))
-        acc[r, :m] = np.sort(rng.choice(ns[r], size=m, replace=False))
+        lo = 1 if keep_root else 0
+        m = int(rng.integers(0, min(max_out - 2, ns[r] - lo) + 1))
+        acc[r, :m] = np.sort(lo + rng.choice(ns[r] - lo, size=m, replace=False))
         acc[r, m] = -1
         cnt[r] = m + 1
     rk, rv = pw.k.copy(), pw.v.copy()
     want_L = np.zeros(n_req, np.int32)
     for r in range(n_req):
-        want_L[r] = orc.compact_kv_paged(rk, pw.page_table[r], page_size, pw.tree_row_offset[r], Ls[r], acc[r, :cnt[r]])
-        orc.compact_kv_paged(rv, pw.page_table[r], page_size, pw.tree_row_offset[r], Ls[r], acc[r, :cnt[r]])
+        want_L[r] = orc.compact_kv_paged(rk, pw.page_table[r], page_size, pw.tree_row_offset[r], Ls[r], acc[r, :cnt[r]],
+                                         keep_root=keep_root)
+        orc.compact_kv_paged(rv, pw.page_table[r], page_size, pw.tree_row_offset[r], Ls[r], acc[r, :cnt[r]], keep_root=keep_root)
     dev = "cuda:0"
     t = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(dev)
     dk, dv = t(pw.k.view(np.int16)), t(pw.v.view(np.int16))
     newL = torch.zeros(n_req, dtype=torch.int32, device=dev)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     B.dyspec_compact_kv_paged(dk, dv, t(pw.tree_row_offset), t(pw.page_table), pw.pages_per_req, page_size, t(Ls), t(acc),
-                              t(cnt), n_req, max_out, hkv, d, newL, status)
+                              t(cnt), n_req, max_out, hkv, d, newL, status, keep_root=keep_root)
     torch.cuda.synchronize()
     assert int(status.item()) == 0
     assert np.array_equal(dk.cpu().numpy().view(np.uint16), rk)

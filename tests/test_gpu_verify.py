@@ -42,7 +42,7 @@ def run_gpu(B, case, bonus=False, max_out=64, max_nodes=None):
     return out_t.cpu().numpy(), out_n.cpu().numpy(), cnt.cpu().numpy(), int(status.item())
 
 
-def check(B, case, bonus=False, max_excused=0.25):
+def check(B, case, bonus=False, max_excused=2):
     out_t, out_n, cnt, status = run_gpu(B, case, bonus)
     assert status == 0
     excused = 0
@@ -59,7 +59,10 @@ def check(B, case, bonus=False, max_excused=0.25):
         assert out_t[r, :k].tolist() == A
         want_nodes = nodes + [-1] * (len(A) - len(nodes))
         assert out_n[r, :k].tolist() == want_nodes
-    assert excused <= max_excused * max(1, len(case.parents))
+    # a request is excused only when the oracle's own deciding number lies within rounding of its threshold
+    # (1e-4 on a ratio, 3e-6 on a CDF): that must stay rare
+    print(f"verify parity: {excused} of {len(case.parents)} requests excused (oracle margin below rounding)")
+    assert excused <= max_excused, (excused, len(case.parents))
     return excused
 
 
@@ -80,8 +83,8 @@ def test_verify_many_requests_and_rejections(B):
     trees = [wl.greedy_tree(rng, int(rng.integers(2, 60)), 6, 1.0) for _ in range(40)]
     trees.append(np.concatenate([[-1], np.zeros(15, np.int32)]).astype(np.int32))      # 15 branches at the root
     case = wl.make_verify_case(5, 16, trees, sharpness=0.5, disagreement=3.0)
-    check(B, case, bonus=False, max_excused=0.3)
-    check(B, case, bonus=True, max_excused=0.3)
+    check(B, case, bonus=False)
+    check(B, case, bonus=True)
 
 
 def test_verify_draft_equal_to_target_walks_first_branches(B):

@@ -322,6 +322,32 @@ def test_ragged_is_independent_requests():
     assert bits.shape == (10, 4) and depths.tolist()[7:] == [0, 1, 2]
 
 
+# ----------------------------------------------------------------------------- visible (query, key) pairs (what the flop count of the roofline is built on)
+def test_visible_pair_count_closed_forms_and_brute_force():
+    """The number of (query, key) pairs the definition of Sec. 2 / App. C uses: every node sees the L
+    prefix keys, its ancestors and itself.  Chain of n nodes: n L + n (n + 1) / 2.  Forest of n roots
+    (star): n (L + 1).  A perfect binary tree with levels 0 .. d: sum over levels 2^k (L + k + 1).
+    Brute force: count, pair by pair, the keys j <= i that lie on node i's root path."""
+    for L, n in ((0, 1), (5, 1), (7, 9), (128, 16), (1000, 33)):
+        assert orc.visible_pair_count([L], [wl.chain_tree(n)]) == n * L + n * (n + 1) // 2
+        assert orc.visible_pair_count([L], [wl.star_forest(n)]) == n * (L + 1)
+    d, L = 4, 11
+    binary = np.array([-1] + [(i - 1) // 2 for i in range(1, 2 ** (d + 1) - 1)], dtype=np.int32)
+    assert orc.visible_pair_count([L], [binary]) == sum(2 ** k * (L + k + 1) for k in range(d + 1))
+    # ragged: the sum over requests; an empty request adds nothing
+    assert orc.visible_pair_count([3, 9, 2], [wl.chain_tree(4), np.zeros(0, np.int32), wl.star_forest(5)]) == \
+        (4 * 3 + 10) + 0 + 5 * 3
+    rng = np.random.default_rng(12)
+    for n in (1, 6, 40):
+        p = wl.random_tree(rng, n, p_root=0.2)
+        L = int(rng.integers(0, 20))
+        brute = 0
+        for i in range(n):
+            path = set(_path(p, i))
+            brute += L + sum(1 for j in range(n) if j in path)
+        assert orc.visible_pair_count([L], [p]) == brute
+
+
 # ----------------------------------------------------------------------------- workload structure (Sec. 4.3: shallow trees)
 def test_generator_trees_are_valid_and_shallow():
     """Sec. 4.3: depth is typically < 10 at N = 64 and < 30 at N = 768; greedy trees keep parent[i] < i."""

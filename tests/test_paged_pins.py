@@ -95,3 +95,18 @@ def test_compaction_matches_the_contiguous_one_read_through_the_table():
     # nothing else moved
     others = np.setdiff1d(np.arange(pw.pool_rows), rows[L:])
     assert np.array_equal(pool[others], pw.k[others])
+
+
+def test_paged_compaction_keeps_the_root_like_the_contiguous_one():
+    rng = np.random.default_rng(4)
+    L, n = 6, 12
+    w = wl.make_custom(71, 2, 2, 8, [L], [wl.chain_tree(n)])
+    pw = wl.to_paged(w, 4, 3)
+    listed = [2, 5, 9, -1]
+    cont = w.k.copy()
+    pool = pw.k.copy()
+    new_L = orc.compact_kv(cont, 0, L, listed, keep_root=True)
+    assert orc.compact_kv_paged(pool, pw.page_table[0], 4, int(pw.tree_row_offset[0]), L, listed, keep_root=True) == new_L == L + 4
+    rows = orc.paged_prefix_rows(pw.page_table[0], 4, new_L)
+    assert np.array_equal(pool[rows], cont[:new_L])
+    assert np.array_equal(pool[rows[L]], w.k[L])                          # token L is the root's row

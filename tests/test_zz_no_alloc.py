@@ -1,10 +1,13 @@
-"""The allocation-free entry point, dyspec_tree_attention_static, against dyspec_tree_attention_ragged.
+"""The allocation-free entry point, dyspec_tree_attention_static, against dyspec_tree_attention_ragged
+and against the fp64 oracle.
 
 For callers that cannot allocate device memory (everything was given to a pool at start-up, or the
 host framework forbids allocation inside its step function) the library keeps the work list and the
 split-KV partials in a fixed 16 MiB device array.  The array is shared and keeps old contents, so
 the check runs two calls back to back, of different shapes, and each must match the ordinary entry
-point.  This file sorts last on purpose: a run that stops at the first failure has then already
+point and, element by element, the oracle (same tolerance as the parity tests).  It also checks what
+the entry point exists for: the device's free memory does not change across calls of new shapes.
+This file sorts last on purpose: a run that stops at the first failure has then already
 run every other test.
 """
 import numpy as np
@@ -37,6 +40,7 @@ def test_static_scratch_entry_point_matches_ragged_entry_point_twice_in_a_row():
     # the shared queue in the caller's workspace, here (no workspace) from fixed lists
     many = wl.make_custom(22, 64, 8, 128, [200], [wl.greedy_tree(rng, 1024, 8, 0.3)])
     cases = [big, wl.make_custom(21, 8, 2, 64, [300], [wl.greedy_tree(rng, 40, 4, 0.3)]), wl.make_config(2), many, big]
+    from oracle import dyspec_oracle as orc
     for w in cases:
         batch = R.DeviceBatch(w)
         batch.step()                                          # existing entry points: mask + ragged attention
@@ -57,6 +61,43 @@ def test_static_scratch_entry_point_matches_ragged_entry_point_twice_in_a_row():
             assert np.isfinite(got).all()
             err = np.abs(got - want)
             assert err.max() <= MAX_ABS and err.mean() <= MEAN_ABS
+        # the last call's output against the definition (fp64 oracle), element by element
+        ref = orc.tree_attention_ragged(w.q, w.k, w.v, w.prefix_len, w.n_nodes, w.kv_row_offset, w.parents)
+        err = np.abs(got - ref)
+        assert err.max() <= MAX_ABS and err.mean() <= MEAN_ABS, (w.name, err.max(), err.mean())
+
+
+def test_static_entry_point_allocates_no_device_memory():
+    """Calls of shapes never seen before leave the driver's free-memory figure unchanged (all buffers are
+    made beforehand; the entry point itself must not allocate), and a request with no nodes is a no-op."""
+    import torch
+    from paper_2410_11744_b200 import build
+    build.build()
+    from paper_2410_11744_b200 import binding as B, runner as R
+    rng = np.random.default_rng(5)
+    shapes = [(8, 2, 64, 90, 17), (32, 32, 128, 700, 48), (64, 8, 128, 333, 300), (16, 4, 128, 0, 5)]
+    batches = []
+    for i, (hq, hkv, d, L, n) in enumerate(shapes):
+        w = wl.make_custom(40 + i, hq, hkv, d, [L], [wl.greedy_tree(rng, n, 4, 0.3)])
+        b = R.DeviceBatch(w)
+        b.build_mask()
+        batches.append((w, b, torch.zeros_like(b.out)))
+    # warm-up call: the first call on a device looks up the array's address and loads the kernels
+    w, b, out = batches[0]
+    B.dyspec_tree_attention_static(b.q, b.k, b.v, int(w.prefix_len[0]), b.bits, int(w.n_nodes[0]), out, w.n_q_heads,
+                                   w.n_kv_heads, w.head_dim, b.W)
+    torch.cuda.synchronize()
+    free0 = torch.cuda.mem_get_info()[0]
+    for w, b, out in batches[1:] + batches[:1]:
+        B.dyspec_tree_attention_static(b.q, b.k, b.v, int(w.prefix_len[0]), b.bits, int(w.n_nodes[0]), out, w.n_q_heads,
+                                       w.n_kv_heads, w.head_dim, b.W)
+        # no nodes: returns at once, touches nothing
+        B.dyspec_tree_attention_static(b.q, b.k, b.v, int(w.prefix_len[0]), b.bits, 0, out, w.n_q_heads, w.n_kv_heads,
+                                       w.head_dim, b.W)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free0
+    for w, b, out in batches:
+        assert out.any()
 
 
 def test_static_scratch_entry_point_refuses_what_does_not_fit():
