@@ -153,7 +153,7 @@ class Plan:
 
     def describe(self) -> dict:
         names = ["items", "ctas", "groups", "split_groups", "max_splits", "regime", "key_tiles", "rows_per_tile",
-                 "cluster", "dynamic"]
+                 "cluster", "dynamic", "combine_launch"]
         return {k: self.info(i) for i, k in enumerate(names)}
 
     def destroy(self) -> None:

@@ -50,7 +50,7 @@ cudaError_t launch_attn_small(int head_dim, int n_ctas, const CUtensorMap& mq, c
                             const AttnParams& p, const WorkItem* host_items, cudaStream_t stream);
 cudaError_t launch_combine(int head_dim, int bm, int n_split_groups, const AttnParams& p, cudaStream_t stream);
 cudaError_t launch_attn_tc(int head_dim, int n_ctas, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
-                           const AttnParams& p, cudaStream_t stream);
+                           const AttnParams& p, const WorkItem* host_items, cudaStream_t stream);
 }  // namespace dyspec
 
 using namespace dyspec;
@@ -185,6 +185,8 @@ struct dyspec_plan {
   bool dynamic = false;                 // whole groups taken from a shared queue (longest first) instead of fixed lists
   bool allow_queue = true;              // false: fixed lists only (callers that cannot provide zeroed queue words)
   size_t queue_offset = 0;              // dynamic plans: byte offset of the two queue words inside the caller's workspace
+  size_t counters_offset = 0;           // plans with split groups: byte offset of the groups' counter pairs in the workspace
+  bool merge_in_kernel = false;         // tensor-core regime: split groups are merged by their own items, no combine launch
   std::vector<WorkItem> items_queue;    // dynamic plans: all items in queue order
   size_t workspace_bytes = 0;
 };
@@ -369,7 +371,10 @@ void schedule(dyspec_plan& pl) {
   // tiles of ~2 us) or four (regime 0) -- measured on the Llama2-70B shape, where the budgeted plan
   // (136 CTAs, 32 split groups) took 53.5 us and whole groups on 128 CTAs 48.1 us.
   if (tn.whole_groups != 1 && (tn.force_ctas <= 0 || tn.whole_groups == 2)) {
-    const int partial_cost = 1, combine_cost = pl.regime == 0 ? 4 : 3;
+    // (tensor-core regime with the merge inside the kernel: no combine launch; writing the fp32 partial,
+    //  publishing it and merging a share of the rows cost a split item about four tiles: 7 us measured)
+    const bool in_kernel = pl.regime == 1 && tn.combine_mode == 2;
+    const int partial_cost = in_kernel ? 4 : 1, combine_cost = in_kernel ? 0 : (pl.regime == 0 ? 4 : 3);
     int64_t cost_split = 0;
     for (int c = 0; c < pl.n_ctas; ++c) {
       int64_t load = 0;
@@ -434,6 +439,78 @@ void schedule(dyspec_plan& pl) {
           pl.items_queue.push_back(it);
         }
       }
+    }
+  }
+
+  // Few long groups (tensor-core regime, merge inside the kernel): cut every group into pieces of equal
+  // length, ONE piece per CTA, as many pieces as there are SMs to take them.  Against the budgeted plan
+  // this avoids CTAs with two split items (each pays the start-up and the partial epilogue again: on the
+  // Llama2-7B shape with a 4096-key prefix those CTAs finished 8 us after the others).
+  if (pl.regime == 1 && tn.combine_mode == 2 && tn.force_ctas <= 0 && tn.whole_groups != 2 && !pl.dynamic &&
+      int64_t(groups.size()) * 2 <= max_ctas) {
+    const int item_cost_ = item_cost, partial_cost = 4;
+    int64_t cost_now = 0;
+    for (int c = 0; c < pl.n_ctas; ++c) {
+      int64_t load = 0;
+      for (int k = pl.cta_begin[size_t(c)]; k < pl.cta_begin[size_t(c) + 1]; ++k) {
+        const WorkItem& it = pl.items[size_t(k)];
+        load += (it.tile_end - it.tile_begin) + item_cost_ + (it.slot >= 0 ? partial_cost : 0);
+      }
+      cost_now = std::max(cost_now, load);
+    }
+    std::vector<int> pieces(groups.size(), std::max(1, int(max_ctas / int64_t(groups.size()))));
+    int used_ctas = 0;
+    for (size_t gi = 0; gi < groups.size(); ++gi) {
+      pieces[gi] = std::min(pieces[gi], std::max(1, groups[gi].tiles / 2));     // a piece has at least two tiles
+      used_ctas += pieces[gi];
+    }
+    auto piece_len = [&](size_t gi) { return (groups[gi].tiles + pieces[gi] - 1) / pieces[gi]; };
+    while (used_ctas < max_ctas) {            // the spare CTAs go to the groups whose pieces are longest
+      size_t best = 0;
+      for (size_t gi = 1; gi < groups.size(); ++gi)
+        if (piece_len(gi) > piece_len(best)) best = gi;
+      if (pieces[best] + 1 > groups[best].tiles / 2) break;
+      ++pieces[best];
+      ++used_ctas;
+    }
+    int64_t cost_even = 0;
+    for (size_t gi = 0; gi < groups.size(); ++gi)
+      cost_even = std::max<int64_t>(cost_even, piece_len(gi) + item_cost_ + (pieces[gi] > 1 ? partial_cost : 0));
+    if (cost_even < cost_now) {
+      pl.items.clear();
+      pl.cta_begin.clear();
+      pl.split_groups.clear();
+      pl.n_slots = 0;
+      pl.max_splits = 1;
+      pl.cta_begin.push_back(0);
+      for (size_t gi = 0; gi < groups.size(); ++gi) {
+        const Group& gr = groups[gi];
+        const ReqInfo& rq = pl.reqs[size_t(gr.req)];
+        const int C = pieces[gi];
+        for (int c = 0; c < C; ++c) {
+          WorkItem it{};
+          it.kv_row0 = rq.kv_row0; it.prefix_len = rq.prefix_len; it.n_nodes = rq.n_nodes; it.node0 = rq.node0;
+          it.req = gr.req; it.kv_head = gr.kvh; it.row0 = gr.row0;
+          it.tile_begin = int(int64_t(gr.tiles) * c / C);
+          it.tile_end = int(int64_t(gr.tiles) * (c + 1) / C);
+          it.n_in_cta = 0;
+          if (C > 1) {
+            it.slot = pl.n_slots + c; it.slot0 = pl.n_slots; it.n_splits = C; it.group = int(pl.split_groups.size());
+          } else {
+            it.slot = -1; it.slot0 = -1; it.n_splits = 1; it.group = int(gi);
+          }
+          pl.items.push_back(it);
+          pl.cta_begin.push_back(int32_t(pl.items.size()));
+        }
+        if (C > 1) {
+          GroupInfo info{};
+          info.req = gr.req; info.kv_head = gr.kvh; info.row0 = gr.row0; info.slot0 = pl.n_slots; info.n_splits = C;
+          pl.n_slots += C;
+          pl.max_splits = std::max(pl.max_splits, C);
+          pl.split_groups.push_back(info);
+        }
+      }
+      pl.n_ctas = int(pl.items.size());
     }
   }
 
@@ -761,6 +838,11 @@ static int make_host_plan(dyspec_plan** out, int n_q_heads, int n_kv_heads, int 
   pl->bn = pl->regime == 0 ? 64 : 128;    // keys per tile
   schedule(*pl);
   pl->workspace_bytes = size_t(pl->n_slots) * size_t(pl->bm) * (pl->d + 2) * sizeof(float);
+  if (!pl->split_groups.empty()) {      // the groups' counter pairs follow the partials
+    pl->counters_offset = (pl->workspace_bytes + 255) & ~size_t(255);
+    pl->workspace_bytes = pl->counters_offset + ((pl->split_groups.size() * 2 * sizeof(int32_t) + 255) & ~size_t(255));
+    pl->merge_in_kernel = pl->regime == 1 && pl->tune.combine_mode == 2;
+  }
   if (pl->dynamic) {                    // the queue words follow the partials (there are none in such a plan today)
     pl->queue_offset = (pl->workspace_bytes + 255) & ~size_t(255);
     pl->workspace_bytes = pl->queue_offset + 256;
@@ -853,6 +935,7 @@ int64_t dyspec_plan_info(const dyspec_plan_t* plan, int field) {
     case 7: return plan->bm;
     case 8: return plan->cluster;
     case 9: return plan->dynamic ? 1 : 0;
+    case 10: return (!plan->split_groups.empty() && !plan->merge_in_kernel) ? 1 : 0;
     default: return DYSPEC_ERR_INVALID_ARG;
   }
 }
@@ -953,7 +1036,10 @@ static int run_attention(const dyspec_plan_t* plan, const void* q, const void* k
   p.reqs = plan->d_reqs; p.items = plan->d_items; p.groups = plan->d_groups;
   p.bits = ancestor_bits; p.node_tiles = node_tiles; p.out = static_cast<__nv_bfloat16*>(out);
   p.partial = static_cast<float*>(workspace);
-  p.counters = plan->d_counters; p.status = status;
+  p.counters = plan->split_groups.empty() ? nullptr
+                                          : reinterpret_cast<int32_t*>(static_cast<unsigned char*>(workspace) + plan->counters_offset);
+  p.merge_in_kernel = plan->merge_in_kernel ? 1 : 0;
+  p.status = status;
   p.queue = plan->dynamic ? reinterpret_cast<int32_t*>(static_cast<unsigned char*>(workspace) + plan->queue_offset) : nullptr;
   p.n_items_total = int32_t(plan->items_strided.size());
   p.n_q_heads = plan->hq; p.n_kv_heads = plan->hkv; p.group_size = plan->g; p.log2_g = plan->log2g;
@@ -970,8 +1056,9 @@ static int run_attention(const dyspec_plan_t* plan, const void* q, const void* k
 
   cudaError_t e;
   if (plan->regime == 0) e = launch_attn_small(plan->d, plan->n_ctas, mq, mk, mv, p, plan->items_strided.data(), st);
-  else e = launch_attn_tc(plan->d, plan->n_ctas, mq, mk, mv, p, st);
+  else e = launch_attn_tc(plan->d, plan->n_ctas, mq, mk, mv, p, plan->items_strided.data(), st);
   if (e != cudaSuccess) return cuda_failed(e, "attention launch");
+  if (plan->merge_in_kernel) return DYSPEC_OK;
   e = launch_combine(plan->d, bm, int(plan->split_groups.size()), p, st);
   return e == cudaSuccess ? DYSPEC_OK : cuda_failed(e, "combine launch");
 }
@@ -1083,7 +1170,7 @@ int dyspec_tree_attention(const void* q, const void* k_cache, const void* v_cach
     if (rc != DYSPEC_OK) return rc;
     pl->device = dev;
     if (!sc.workspace) {                 // once per (device, shape): at most two split pieces per CTA, 256-row tiles
-      const size_t worst = size_t(2) * size_t(pl->n_sms) * 256 * size_t(g_shape.d + 2) * sizeof(float) + 512;
+      const size_t worst = size_t(2) * size_t(pl->n_sms) * 256 * size_t(g_shape.d + 2) * sizeof(float) + 16 * size_t(pl->n_sms) + 1024;
       if (cudaMalloc(&sc.workspace, worst) != cudaSuccess) { sc.workspace = nullptr; delete pl; return DYSPEC_ERR_CUDA; }
       if (cudaMemsetAsync(sc.workspace, 0, worst, st) != cudaSuccess) { delete pl; return DYSPEC_ERR_CUDA; }
       sc.workspace_bytes = worst;
@@ -1180,7 +1267,10 @@ extern "C" int dyspec_tree_attention_static(const void* q, const void* k_cache, 
       (!pl->split_groups.empty() &&
        write_table(base + o_groups, pl->split_groups.data(), pl->split_groups.size() * sizeof(GroupInfo), st) != cudaSuccess))
     return DYSPEC_ERR_CUDA;
-  if (cudaMemsetAsync(base + o_counters, 0, o_partial - o_counters, st) != cudaSuccess) return DYSPEC_ERR_CUDA;
+  // the split groups' counter pairs sit inside the workspace part, behind the partials: they must start at zero
+  if (!pl->split_groups.empty() &&
+      cudaMemsetAsync(base + o_partial + pl->counters_offset, 0, pl->workspace_bytes - pl->counters_offset, st) != cudaSuccess)
+    return DYSPEC_ERR_CUDA;
 
   CUtensorMap mq, mk, mv;
   const int bm = pl->bm, bn = pl->bn;
@@ -1194,8 +1284,9 @@ extern "C" int dyspec_tree_attention_static(const void* q, const void* k_cache, 
   p.reqs = reinterpret_cast<const ReqInfo*>(base + o_reqs);
   p.items = reinterpret_cast<const WorkItem*>(base + o_items);
   p.groups = reinterpret_cast<const GroupInfo*>(base + o_groups);
-  p.counters = reinterpret_cast<int32_t*>(base + o_counters);
   p.partial = reinterpret_cast<float*>(base + o_partial);
+  p.counters = pl->split_groups.empty() ? nullptr : reinterpret_cast<int32_t*>(base + o_partial + pl->counters_offset);
+  p.merge_in_kernel = pl->merge_in_kernel ? 1 : 0;
   p.bits = ancestor_bits; p.out = static_cast<__nv_bfloat16*>(out); p.status = status;
   p.n_q_heads = pl->hq; p.n_kv_heads = pl->hkv; p.group_size = pl->g; p.log2_g = pl->log2g;
   p.words_per_row = pl->W; p.slot_floats = bm * (pl->d + 2);
@@ -1205,8 +1296,9 @@ extern "C" int dyspec_tree_attention_static(const void* q, const void* k_cache, 
 
   cudaError_t e;
   if (pl->regime == 0) e = launch_attn_small(pl->d, pl->n_ctas, mq, mk, mv, p, pl->items_strided.data(), st);
-  else e = launch_attn_tc(pl->d, pl->n_ctas, mq, mk, mv, p, st);
+  else e = launch_attn_tc(pl->d, pl->n_ctas, mq, mk, mv, p, pl->items_strided.data(), st);
   if (e != cudaSuccess) return DYSPEC_ERR_CUDA;
+  if (pl->merge_in_kernel) return DYSPEC_OK;
   e = launch_combine(pl->d, bm, int(pl->split_groups.size()), p, st);
   return e == cudaSuccess ? DYSPEC_OK : DYSPEC_ERR_CUDA;
 }

@@ -68,6 +68,8 @@ __device__ __forceinline__ void named_arrive(int id, int count) { asm volatile("
 __device__ __forceinline__ void named_sync(int id, int count) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory"); }
 constexpr int kBarPReady = 1;               // named barriers 1, 2: P of half A, B is in TMEM
 constexpr int kPReadyCount = BMH + 32;      // a half's softmax threads + the issuing warp
+constexpr int kBarPartial = 3;              // named barriers 3, 4: a half's partial rows are written (its 128 threads)
+constexpr int kBarMerge = 5;                // all 256 softmax threads, around the split-KV merge
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -213,7 +215,8 @@ __device__ __forceinline__ TileWalk walk_sparse(const AttnParams& p, const WorkI
 template <int D, bool kDyn>
 __global__ void __launch_bounds__(kThreads, 1)
 tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                    const __grid_constant__ CUtensorMap map_v, const AttnParams p) {
+                    const __grid_constant__ CUtensorMap map_v, const AttnParams p,
+                    const __grid_constant__ FirstItems first) {
   using L = TcLayout<D>;
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -268,8 +271,12 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
 
   // Fixed lists: CTA c's items are my_items[0 .. item_end).  Queue: my_items is the whole queue, the
   // CTA's k-th item is my_items[index], the index -1 ends the CTA's work.
+  // Every CTA's first item also travels with the kernel parameters: its first loads then do not wait for
+  // a read of the work list from global memory (about a microsecond when the list is not in L2).
   const WorkItem* my_items = p.items + (kDyn ? size_t(0) : size_t(blockIdx.x) * p.items_stride);
-  const int item_end = kDyn ? 0x7fffffff : my_items[0].n_in_cta;
+  const bool first_here = blockIdx.x < kFirstItems;
+  const int item_end = kDyn ? 0x7fffffff : (first_here ? first.item[blockIdx.x].n_in_cta : my_items[0].n_in_cta);
+  auto item_of = [&](int w, int at) -> WorkItem { return (w == 0 && first_here) ? first.item[blockIdx.x] : my_items[at]; };
   // for the producer warp (all lanes call it): takes the next item off the queue and publishes it
   auto take_index = [&](int k) -> int {
     if (k == 0) return int(blockIdx.x);
@@ -320,7 +327,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           item_at = take_index(w);
           if (item_at < 0) break;
         }
-        const WorkItem item = my_items[item_at];
+        const WorkItem item = item_of(w, item_at);
         const WorkItem& rq = item;
         const int nh = (rq.n_nodes * g - item.row0 > BMH) ? 2 : 1;
         mbar_wait(bar(B_QFREE), (qit & 1) ^ 1, abort_flag, p.status);
@@ -422,7 +429,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           item_at = next_index(w);
           if (item_at < 0) break;
         }
-        const WorkItem item = my_items[item_at];
+        const WorkItem item = item_of(w, item_at);
         const WorkItem& rq = item;
         const bool two = rq.n_nodes * g - item.row0 > BMH;        // both query halves live
         const int n_prefix_tiles = (rq.prefix_len + BN - 1) / BN;
@@ -531,7 +538,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     const uint32_t t_o = tmem_base + 256u + uint32_t(h) * 128u + lane_sel;
     TraceCursor tc_cur = trace_open(p, 1 + h, 3);
     // wall-clock stamps of every CTA (last 2048 entries of the trace buffer, 8 per CTA, first 256 CTAs), by
-    // row 0 of half A: 0 start, 1 first scores seen, 2 .. 6 end of the CTA's items 0 .. 4, 7 exit
+    // row 0 of half A: 0 start, 1 first scores seen, 2 / 4 last PV of item 0 / 1 seen, 3 / 5 epilogue of item 0 / 1
+    // done, 6 first split-KV merge may start (all partials of its group have arrived), 7 exit
     auto stamp = [&](int k) {
 #ifdef DYSPEC_CTA_STAMPS
       if (p.trace != nullptr && h == 0 && r == 0 && blockIdx.x < 256 && p.trace_capacity > 4096)
@@ -551,7 +559,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         item_at = next_index(w);
         if (item_at < 0) break;
       }
-      const WorkItem item = my_items[item_at];
+      const WorkItem item = item_of(w, item_at);
       const WorkItem& rq = item;
       const int n_rows = rq.n_nodes * g;
       const int nh = (n_rows - item.row0 > BMH) ? 2 : 1;
@@ -559,7 +567,14 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       if (p.node_tiles != nullptr) need_dep();           // the tile walk reads the per-node tile sets
       const TileWalk wk = walk_sparse(p, item, n_prefix_tiles, lane);
       const int T = wk.T;
-      if (h >= nh) { sc += 2u * uint32_t(T); continue; }
+      if (h >= nh) {
+        sc += 2u * uint32_t(T);
+        if (item.slot >= 0 && p.merge_in_kernel) {         // this half has no rows: nothing to write, but the group counts halves
+          need_dep();
+          if (r == 0) red_release_gpu_add(p.counters + 2 * item.group, 1);
+        }
+        continue;
+      }
       uint32_t rem = wk.need;
       const int row = item.row0 + h * BMH + r;
       const bool ok = row < n_rows;
@@ -699,24 +714,29 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       // ---- epilogue: wait for the last PV, read O, normalise (or emit the partial)
       mbar_wait(bar(B_ODONE + h), n_o & 1, abort_flag, p.status);
       ++n_o;
+      if (w < (kDyn ? 1 : 2)) stamp(2 + 2 * w);
       if (r == 0) trace_event(tc_cur, DYSPEC_TAG(1 + h, 6, 0));
       tc_fence_after();
       need_dep();                                          // global writes from here on
       const int head = item.kv_head * g + (row & (g - 1));
+      // the whole O row (D fp32) in registers: all loads in flight together, one wait
+      uint32_t ov[D];
+#pragma unroll
+      for (int c = 0; c < D / 32; ++c) tmem_ld32(t_o + uint32_t(c) * 32u, ov + 32 * c);
+      tmem_wait_ld();
+      tc_fence_before();
+      mbar_arrive(bar(B_OFREE + h));                       // the accumulator may take the next item's products already
       if (item.slot < 0) {
         const float inv = l > 0.f ? 1.f / l : 0.f;
         __nv_bfloat16* out = p.out + (size_t(rq.node0 + node) * p.n_q_heads + head) * D;
         const bool out_aligned32 = (reinterpret_cast<uintptr_t>(p.out) & 31) == 0;   // rows are multiples of 128 bytes
+        if (ok) {
 #pragma unroll
-        for (int c = 0; c < D / 32; ++c) {
-          uint32_t v[32];
-          tmem_ld32(t_o + uint32_t(c) * 32u, v);
-          tmem_wait_ld();
-          if (ok) {
+          for (int c = 0; c < D / 32; ++c) {
             uint32_t pk[16];
 #pragma unroll
             for (int i = 0; i < 16; ++i)
-              pk[i] = pack_bf16x2(__uint_as_float(v[2 * i]) * inv, __uint_as_float(v[2 * i + 1]) * inv);
+              pk[i] = pack_bf16x2(__uint_as_float(ov[32 * c + 2 * i]) * inv, __uint_as_float(ov[32 * c + 2 * i + 1]) * inv);
             if (out_aligned32) {
               st_global_v8(out + c * 32, pk);
               st_global_v8(out + c * 32 + 16, pk + 8);
@@ -731,25 +751,150 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         // partial slot: O [256][D] fp32, then m [256], then l [256]
         float* slot = p.partial + size_t(item.slot) * p.slot_floats;
         const int pr = h * BMH + r;
+        if (ok) {   // the workspace is 256-byte aligned and slots / rows are multiples of 32 bytes
 #pragma unroll
-        for (int c = 0; c < D / 32; ++c) {
-          uint32_t v[32];
-          tmem_ld32(t_o + uint32_t(c) * 32u, v);
-          tmem_wait_ld();
-          if (ok) {   // the workspace is 256-byte aligned and slots / rows are multiples of 32 bytes
-#pragma unroll
-            for (int i = 0; i < 4; ++i) st_global_v8(slot + pr * D + c * 32 + i * 8, v + 8 * i);
-          }
+          for (int i = 0; i < D / 8; ++i) st_global_v8(slot + pr * D + i * 8, ov + 8 * i);
         }
         if (ok) {
           slot[2 * BMH * D + pr] = m_used;
           slot[2 * BMH * D + 2 * BMH + pr] = l;
         }
+        if (p.merge_in_kernel) {
+          // the group's items merge the rows themselves once every half of every item has arrived
+          named_sync(kBarPartial + h, BMH);             // the half's rows are written (CTA scope) ...
+          if (r == 0) {
+            __threadfence();                            // ... one cumulative fence makes them visible GPU-wide
+            red_release_gpu_add(p.counters + 2 * item.group, 1);
+          }
+        }
       }
-      tc_fence_before();
-      mbar_arrive(bar(B_OFREE + h));
       if (r == 0) trace_event(tc_cur, DYSPEC_TAG(1 + h, 7, 0));
-      if (w < 5) stamp(2 + w);
+      if (w < (kDyn ? 1 : 2)) stamp(3 + 2 * w);
+#ifdef DYSPEC_CTA_STAMPS
+      // developer statistics for the queue plans (which stamp item 0 only): slot 4 = items, slot 5 = key tiles of this CTA
+      if (kDyn && p.trace != nullptr && h == 0 && r == 0 && blockIdx.x < 256 && p.trace_capacity > 4096) {
+        p.trace[p.trace_capacity - 2048 + 8 * blockIdx.x + 4] = (unsigned long long)(w + 1);
+        p.trace[p.trace_capacity - 2048 + 8 * blockIdx.x + 5] += (unsigned long long)T;
+      }
+#endif
+    }
+    // ---- split-KV merge (no combine launch): every item of a split group merges a share of the group's
+    // rows once all of the group's partials are in the workspace.  Done after ALL of the CTA's items, so
+    // that no CTA waits for a partial while it still owes one (arrivals never depend on a wait).  All CTAs
+    // of the launch are resident (one wave), so the waits end; they are bounded all the same.
+    if constexpr (!kDyn) {
+      if (p.merge_in_kernel) {
+        const int tid = h * BMH + r;                     // 0 .. 255
+        const int mw = tid >> 5;                         // merge warp 0 .. 7
+        for (int w = 0; w < item_end; ++w) {
+          const WorkItem item = item_of(w, w);
+          if (item.slot < 0) continue;
+          int32_t* ctr = p.counters + 2 * item.group;
+          const int ns = item.n_splits;
+          if (tid == 0) {
+            const uint64_t t0 = global_timer_ns();
+            uint32_t spins = 0;
+            while (ld_acquire_gpu(ctr) < 2 * ns) {
+              if ((++spins & 0x3f) == 0 && (*abort_flag || global_timer_ns() - t0 > kWaitLimitNs)) {
+                *abort_flag = 1;
+                if (p.status) atomicCAS(p.status, 0, DYSPEC_ERR_TIMEOUT);
+                break;
+              }
+            }
+          }
+          named_sync(kBarMerge, 2 * BMH);
+          stamp(6);
+          const int n_rows = item.n_nodes * g;
+          const int share = ((2 * BMH + ns - 1) / ns + 7) & ~7;                 // rows per item, a multiple of the 8 merge warps
+          const int s_idx = item.slot - item.slot0;
+          const int row_lo = s_idx * share, row_hi = min(2 * BMH, row_lo + share);
+          const float* base = p.partial + size_t(item.slot0) * p.slot_floats;
+          const float* base_m = base + 2 * BMH * D;                             // a slot: O [256][D], m [256], l [256]
+          constexpr int V = D / 32;                                             // floats per lane
+          constexpr int KR = 4, KS = 4;                                         // rows per warp and pass; partials in flight per row
+          // A pass: KR rows per warp.  Lane 8 k + u fetches (m, l) of row k from partials u, u + 8, ...; every lane
+          // fetches its V columns of KS partial rows per row at a time, so a pass is one or two round trips
+          // to L2 whatever the number of splits (a loop that uses each value as it arrives is a chain of them).
+          for (int pr0 = row_lo + KR * mw; pr0 < row_hi; pr0 += 8 * KR) {
+            const int lk = lane >> 3, lu = lane & 7;
+            const int lrow = min(pr0 + lk, 2 * BMH - 1);
+            float m_l = -INFINITY;
+            for (int s_ = lu; s_ < ns; s_ += 8) m_l = fmaxf(m_l, ld_cg_f32(base_m + size_t(s_) * p.slot_floats + lrow));
+            m_l = fmaxf(m_l, __shfl_xor_sync(0xffffffffu, m_l, 1));
+            m_l = fmaxf(m_l, __shfl_xor_sync(0xffffffffu, m_l, 2));
+            m_l = fmaxf(m_l, __shfl_xor_sync(0xffffffffu, m_l, 4));
+            const float ref_l = m_l == -INFINITY ? 0.f : m_l;                   // the row's reference, known to its 8 lanes
+            float acc[KR][V], lsum = 0.f;
+#pragma unroll
+            for (int k = 0; k < KR; ++k)
+#pragma unroll
+              for (int e = 0; e < V; ++e) acc[k][e] = 0.f;
+            for (int s0 = 0; s0 < ns; s0 += 8) {
+              // weights of partials s0 .. s0 + 7 for this lane's row
+              float f_l = 0.f;
+              if (s0 + lu < ns) {
+                const float* sl = base_m + size_t(s0 + lu) * p.slot_floats;
+                const float mv = ld_cg_f32(sl + lrow), lv = ld_cg_f32(sl + 2 * BMH + lrow);
+                f_l = fast_exp2(mv - ref_l);
+                lsum += f_l * lv;
+              }
+              for (int s1 = s0; s1 < min(ns, s0 + 8); s1 += KS) {
+                float vv[KR][KS][V];
+#pragma unroll
+                for (int k = 0; k < KR; ++k)
+#pragma unroll
+                  for (int u = 0; u < KS; ++u) {
+                    const int pr = min(pr0 + k, 2 * BMH - 1);
+                    const float* sl = base + size_t(min(s1 + u, ns - 1)) * p.slot_floats + pr * D;
+                    if constexpr (V == 4) {
+                      const float4 x = ld_cg_f32x4(sl + lane * 4);
+                      vv[k][u][0] = x.x; vv[k][u][1] = x.y; vv[k][u][2] = x.z; vv[k][u][3] = x.w;
+                    } else {
+                      const float2 x = ld_cg_f32x2(sl + lane * 2);
+                      vv[k][u][0] = x.x; vv[k][u][1] = x.y;
+                    }
+                  }
+#pragma unroll
+                for (int k = 0; k < KR; ++k)
+#pragma unroll
+                  for (int u = 0; u < KS; ++u) {
+                    float f = __shfl_sync(0xffffffffu, f_l, 8 * k + ((s1 - s0 + u) & 7));
+                    if (s1 + u >= ns) f = 0.f;
+#pragma unroll
+                    for (int e = 0; e < V; ++e) acc[k][e] += f * vv[k][u][e];
+                  }
+              }
+            }
+            lsum += __shfl_xor_sync(0xffffffffu, lsum, 1);
+            lsum += __shfl_xor_sync(0xffffffffu, lsum, 2);
+            lsum += __shfl_xor_sync(0xffffffffu, lsum, 4);
+#pragma unroll
+            for (int k = 0; k < KR; ++k) {
+              const float lk_sum = __shfl_sync(0xffffffffu, lsum, 8 * k);
+              const int pr = pr0 + k, row = item.row0 + pr;
+              if (pr < row_hi && row < n_rows) {
+                const float inv = lk_sum > 0.f ? 1.f / lk_sum : 0.f;
+                const int node = row >> p.log2_g;
+                const int head = item.kv_head * g + (row & (g - 1));
+                __nv_bfloat16* out = p.out + (size_t(item.node0 + node) * p.n_q_heads + head) * D;
+                if constexpr (V == 4) {
+                  uint2 o;
+                  o.x = pack_bf16x2(acc[k][0] * inv, acc[k][1] * inv);
+                  o.y = pack_bf16x2(acc[k][2] * inv, acc[k][3] * inv);
+                  *reinterpret_cast<uint2*>(out + lane * 4) = o;
+                } else {
+                  *reinterpret_cast<uint32_t*>(out + lane * 2) = pack_bf16x2(acc[k][0] * inv, acc[k][1] * inv);
+                }
+              }
+            }
+          }
+          // the group's last merger leaves the counter pair at zero for the next launch
+          if (tid == 0 && atomicAdd(ctr + 1, 1) == ns - 1) {
+            ctr[0] = 0;
+            ctr[1] = 0;
+          }
+        }
+      }
     }
     stamp(7);
   }
@@ -765,16 +910,20 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
 namespace {
 template <int D, bool kDyn>
 cudaError_t launch_one(cudaLaunchConfig_t& cfg, size_t smem, const CUtensorMap& mq, const CUtensorMap& mk,
-                       const CUtensorMap& mv, const AttnParams& p) {
+                       const CUtensorMap& mv, const AttnParams& p, const FirstItems& first) {
   static DynSmemGrant grant;           // one per instantiation
   if (cudaError_t e = grant.ensure(tree_attn_tc_kernel<D, kDyn>, smem); e != cudaSuccess) return e;
   cfg.dynamicSmemBytes = smem;
-  return cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<D, kDyn>, mq, mk, mv, p);
+  return cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<D, kDyn>, mq, mk, mv, p, first);
 }
 }  // namespace
 
 cudaError_t launch_attn_tc(int head_dim, int n_ctas, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
-                           const AttnParams& p, cudaStream_t stream) {
+                           const AttnParams& p, const WorkItem* host_items, cudaStream_t stream) {
+  // host_items: the host copy of p.items (same layout); each CTA's first item travels as a kernel parameter
+  FirstItems first;
+  const size_t stride = p.queue != nullptr ? 1 : size_t(p.items_stride);
+  for (int c = 0; c < kFirstItems; ++c) first.item[c] = c < n_ctas ? host_items[size_t(c) * stride] : WorkItem{};
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
@@ -788,12 +937,12 @@ cudaError_t launch_attn_tc(int head_dim, int n_ctas, const CUtensorMap& mq, cons
   cudaError_t le = cudaSuccess;
   if (head_dim == 128) {
     const size_t smem = TcLayout<128>::kTotal + 1024;
-    le = dyn ? launch_one<128, true>(cfg, smem, mq, mk, mv, p) : launch_one<128, false>(cfg, smem, mq, mk, mv, p);
+    le = dyn ? launch_one<128, true>(cfg, smem, mq, mk, mv, p, first) : launch_one<128, false>(cfg, smem, mq, mk, mv, p, first);
   } else {
     // padded past half of an SM's shared memory: one CTA per SM, since each CTA takes all 512 TMEM columns
     const size_t smem = 120 * 1024;
     static_assert(TcLayout<64>::kTotal + 1024 <= 120 * 1024, "smem layout");
-    le = dyn ? launch_one<64, true>(cfg, smem, mq, mk, mv, p) : launch_one<64, false>(cfg, smem, mq, mk, mv, p);
+    le = dyn ? launch_one<64, true>(cfg, smem, mq, mk, mv, p, first) : launch_one<64, false>(cfg, smem, mq, mk, mv, p, first);
   }
   return le != cudaSuccess ? le : cudaGetLastError();
 }

@@ -82,7 +82,9 @@ struct AttnParams {
   const uint32_t* node_tiles;      // optional [sum n]: bit t = the node's row touches tree columns [64 t, 64 t + 64)
   __nv_bfloat16* out;              // [sum n][H_q][D]
   float* partial;                  // split-KV partials: slot s at partial + s * slot_floats
-  int32_t* counters;               // per-group arrival counters (zero between calls)
+  int32_t* counters;               // two words per split group, in the caller's workspace, zero between calls:
+                                   // [2 g] = halves of the group's items whose partial is written, [2 g + 1] = items that have merged their share
+  int32_t merge_in_kernel;         // tensor-core regime: the items of a split group merge the group's rows themselves (no combine launch)
   int32_t* status;                 // may be null
   int32_t n_q_heads;
   int32_t n_kv_heads;
@@ -288,6 +290,31 @@ __device__ __forceinline__ uint2 ld_after_dependency_v2(const void* ptr) {
 __device__ __forceinline__ uint32_t ld_after_dependency_u32(const void* ptr) {
   uint32_t v;
   asm volatile("ld.global.u32 %0, [%1];" : "=r"(v) : "l"(ptr) : "memory");
+  return v;
+}
+// Cross-CTA hand-off through global memory (split-KV merge inside the attention kernel).
+__device__ __forceinline__ void red_release_gpu_add(int32_t* addr, int32_t v) {
+  asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(addr), "r"(v) : "memory");
+}
+__device__ __forceinline__ int32_t ld_acquire_gpu(const int32_t* addr) {
+  int32_t v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(addr) : "memory");
+  return v;
+}
+// Data another SM wrote during this launch: read from L2 (this SM's L1 may hold a stale line).
+__device__ __forceinline__ float4 ld_cg_f32x4(const float* ptr) {
+  float4 v;
+  asm volatile("ld.global.cg.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(ptr) : "memory");
+  return v;
+}
+__device__ __forceinline__ float2 ld_cg_f32x2(const float* ptr) {
+  float2 v;
+  asm volatile("ld.global.cg.v2.f32 {%0,%1}, [%2];" : "=f"(v.x), "=f"(v.y) : "l"(ptr) : "memory");
+  return v;
+}
+__device__ __forceinline__ float ld_cg_f32(const float* ptr) {
+  float v;
+  asm volatile("ld.global.cg.f32 %0, [%1];" : "=f"(v) : "l"(ptr) : "memory");
   return v;
 }
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
