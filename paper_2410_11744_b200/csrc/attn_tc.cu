@@ -185,10 +185,16 @@ __device__ __forceinline__ TileWalk walk_dense(const WorkItem& item, int n_prefi
   wk.T = wk.P + __popc(wk.need);
   return wk;
 }
+// Can the tile sets shorten this walk at all?  With one or two tree tiles they cannot pay: the query tile's
+// own columns are always visible, and reading the tile sets means waiting for the mask kernel before the
+// first tree tile is even requested.
+__device__ __forceinline__ bool walk_may_skip(const AttnParams& p, const TileWalk& dense) {
+  return p.node_tiles != nullptr && __popc(dense.need) > 2;
+}
 // Whole warp.  The mask kernel must have completed (grid_dependency_wait) before this reads node_tiles.
 __device__ __forceinline__ TileWalk walk_sparse(const AttnParams& p, const WorkItem& item, int n_prefix_tiles, int lane) {
   TileWalk wk = walk_dense(item, n_prefix_tiles);
-  if (p.node_tiles == nullptr || wk.need == 0u) return wk;
+  if (!walk_may_skip(p, wk)) return wk;
   const int node_lo = item.row0 >> p.log2_g;
   const int node_hi = min(item.n_nodes, ((item.row0 + 2 * BMH - 1) >> p.log2_g) + 1);
   uint32_t occ = 0u;
@@ -342,7 +348,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         // Prefix tiles stream at once; the set of tree tiles may depend on the mask kernel's output,
         // so it is settled (after waiting for that kernel) only when the walk reaches the tree.
         TileWalk wk = walk_dense(item, n_prefix_tiles);
-        bool exact = p.node_tiles == nullptr || wk.need == 0u;
+        bool exact = !walk_may_skip(p, wk);
         uint32_t rem = wk.need;
         for (int j = 0;; ++j) {
           if (!exact && j >= wk.P) {
@@ -434,7 +440,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         const bool two = rq.n_nodes * g - item.row0 > BMH;        // both query halves live
         const int n_prefix_tiles = (rq.prefix_len + BN - 1) / BN;
         TileWalk wk = walk_dense(item, n_prefix_tiles);
-        bool exact = p.node_tiles == nullptr || wk.need == 0u;
+        bool exact = !walk_may_skip(p, wk);
         int T = exact ? wk.T : 0x7fffffff;
         auto settle = [&](int j) {
           if (!exact && j + 2 >= wk.P) {
@@ -564,7 +570,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       const int n_rows = rq.n_nodes * g;
       const int nh = (n_rows - item.row0 > BMH) ? 2 : 1;
       const int n_prefix_tiles = (rq.prefix_len + BN - 1) / BN;
-      if (p.node_tiles != nullptr) need_dep();           // the tile walk reads the per-node tile sets
+      if (walk_may_skip(p, walk_dense(item, n_prefix_tiles))) need_dep();   // the tile walk reads the per-node tile sets
       const TileWalk wk = walk_sparse(p, item, n_prefix_tiles, lane);
       const int T = wk.T;
       if (h >= nh) {

@@ -12,7 +12,13 @@
 //     is an array scanned by the whole block (<= 4096 slots: one pass).
 //   threshold (Algorithm 2): layer by layer, each position keeps drawing while v >= t.
 // The residual lives in registers (thread t owns float4 chunks t, t + 1024, ...); a draw is an
-// inverse-CDF search in token order (row totals, then one block scan).
+// inverse-CDF search in token order (row totals, then one block scan).  The tokens a position has
+// already used are struck out in constant time whatever their number: every thread looks at one or two
+// nodes of the tree, and where a node is a child of the position it sets the token's bit in the word of
+// the thread that owns the token (32 tokens per thread, one shared-memory word each); after a barrier a
+// thread zeroes what its word marks.  (Walking the position's child list instead costs a dependent
+// shared-memory hop per earlier sibling in all 32 warps: quadratic in the width of a position, and
+// language-model rows give the root hundreds of children.)
 #include "vocab_ops.cuh"
 
 namespace dyspec {
@@ -43,26 +49,25 @@ build_tree_greedy_kernel(const float* __restrict__ draft_table, int n_rows, int 
                          int n_uniforms, const int32_t* __restrict__ root_row, int m, TreeOut out,
                          int32_t* __restrict__ n_nodes_out) {
   extern __shared__ __align__(16) uint8_t csm[];
-  // slots: value, position, attempt; per node: row id, first / last child, next sibling, token
+  // slots: value, position, attempt; per node: row id, token, the position it was drawn at
   const int max_slots = 2 * m + 2;
   double* s_v = reinterpret_cast<double*>(csm);                     // [max_slots]   (-1 = taken); fp64 like the draws
   int16_t* s_pos = reinterpret_cast<int16_t*>(s_v + max_slots);     // [max_slots]
   int16_t* s_att = s_pos + max_slots;                               // [max_slots]
   int32_t* s_row = reinterpret_cast<int32_t*>(s_att + max_slots + (max_slots & 1));   // [m + 1]
   int32_t* s_tok = s_row + (m + 1);                                 // [m + 1]
-  int16_t* s_first = reinterpret_cast<int16_t*>(s_tok + (m + 1));   // [m + 1]
-  int16_t* s_next = s_first + (m + 1);                              // [m + 1]
-  int16_t* s_last = s_next + (m + 1);                               // [m + 1]
+  int16_t* s_ppos = reinterpret_cast<int16_t*>(s_tok + (m + 1));    // [m + 1] the position (parent) a node was drawn at
+  __shared__ uint32_t s_kill[kVThreads];                            // bit 4 k + e of word t: element e of thread t's chunk k is used up
   __shared__ VocabScratch s_vs;
   __shared__ double s_bv[33];
   __shared__ int s_bi[33];
 
   const int r = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const size_t base = size_t(r) * (m + 1);
-  for (int i = tid; i <= m; i += kVThreads) { s_first[i] = -1; s_next[i] = -1; s_last[i] = -1; }
   if (tid == 0) {
     s_row[0] = ((root_row[r] % n_rows) + n_rows) % n_rows;        // non-negative remainder: any int32 maps to a row
     s_tok[0] = 0;
+    s_ppos[0] = -1;
     s_v[0] = 1.0; s_pos[0] = 0; s_att[0] = 0;
     write_node(out, base, 0, -1, 0, 1.f, 1.f, s_row[0]);
   }
@@ -109,15 +114,24 @@ build_tree_greedy_kernel(const float* __restrict__ draft_table, int n_rows, int 
     // ---- residual of the position: its row with the tokens of its existing children zeroed
     float4 R[kMaxChunks];
     load_row(R, draft_table + size_t(prow) * vocab, vocab);
-    for (int c = s_first[pos]; c >= 0; c = s_next[c]) {
-      const int y = s_tok[c];
-      const int y4 = y >> 2, yk = y4 / kVThreads, yt = y4 - yk * kVThreads, ye = y & 3;
-      if (tid == yt) {
+    if (attempt > 0) {                                           // (a first sampling has nothing to strike out)
+      s_kill[tid] = 0u;
+      __syncthreads();
+      for (int c = 1 + tid; c <= n_created; c += kVThreads)
+        if (s_ppos[c] == pos) {
+          const int yc = s_tok[c], y4 = yc >> 2;
+          atomicOr(&s_kill[y4 % kVThreads], 1u << ((y4 / kVThreads) * 4 + (yc & 3)));
+        }
+      __syncthreads();
+      const uint32_t kill = s_kill[tid];
+      if (kill) {
 #pragma unroll
-        for (int k = 0; k < kMaxChunks; ++k)
-          if (k == yk) {
-            if (ye == 0) R[k].x = 0.f; else if (ye == 1) R[k].y = 0.f; else if (ye == 2) R[k].z = 0.f; else R[k].w = 0.f;
-          }
+        for (int k = 0; k < kMaxChunks; ++k) {
+          if ((kill >> (4 * k)) & 1u) R[k].x = 0.f;
+          if ((kill >> (4 * k + 1)) & 1u) R[k].y = 0.f;
+          if ((kill >> (4 * k + 2)) & 1u) R[k].z = 0.f;
+          if ((kill >> (4 * k + 3)) & 1u) R[k].w = 0.f;
+        }
       }
     }
     double total;
@@ -132,8 +146,7 @@ build_tree_greedy_kernel(const float* __restrict__ draft_table, int n_rows, int 
       const int krow = int(draft_row_of_child(uint32_t(prow), uint32_t(y), uint32_t(n_rows)));
       s_row[k] = krow;
       s_tok[k] = y;
-      if (s_first[pos] < 0) s_first[pos] = int16_t(k); else s_next[s_last[pos]] = int16_t(k);
-      s_last[pos] = int16_t(k);
+      s_ppos[k] = int16_t(pos);
       write_node(out, base, k, pos, y, float(v), float(v * rr), krow);
       int ns = n_slots;
       if (1.0 - rr > 0.0) { s_v[ns] = v * (1.0 - rr); s_pos[ns] = int16_t(pos); s_att[ns] = int16_t(attempt + 1); ++ns; }
@@ -199,7 +212,7 @@ build_tree_threshold_kernel(const float* __restrict__ draft_table, int n_rows, i
 
 size_t build_tree_greedy_smem(int m) {
   const size_t max_slots = 2 * size_t(m) + 2;          // value (8 bytes) + position and attempt (2 + 2) per slot
-  return 12 * max_slots + 14 * size_t(m + 1) + 64;     // row and token (4 + 4) + three 2-byte links per node
+  return 12 * max_slots + 10 * size_t(m + 1) + 64;     // row and token (4 + 4) + the 2-byte position per node
 }
 
 cudaError_t launch_build_tree_greedy(const float* draft_table, int n_rows, int vocab, const float* uniforms, int n_uniforms,

@@ -2,7 +2,13 @@
 // sampling along the tree), on the device, so that the step after the tree attention needs no host
 // round trip.
 //
-// One CTA of 1024 threads per request walks the tree from node 0.  At a node it loads the target row
+// One CTA of 1024 threads per request walks the tree from node 0.  As long as the FIRST branch of the
+// current node is accepted the walk needs two numbers per node, Target(node, y) and Draft(node, y), not the
+// rows: one warp does it alone (first child by ballots over the parent array in shared memory, two scalar
+// loads, the test), about a microsecond per node, while the other warps wait at a block barrier.  Only at
+// a first rejection -- or where a token has to be drawn -- the whole block takes the node over, from
+// its first branch again (the test is repeated with the same numbers, so the decision is the same):
+// it loads the target row
 // into registers (the residual R; thread t owns the float4 chunks t, t + 1024, ... of the vocabulary)
 // and the draft row D into shared memory in the same interleaved order (coalesced global loads,
 // conflict-free shared accesses).  Both carry a scalar scale instead of being renormalised in place:
@@ -29,6 +35,9 @@ verify_tree_kernel(const int32_t* __restrict__ parents, const int32_t* __restric
   extern __shared__ __align__(16) uint8_t vsm[];
   float4* s_d = reinterpret_cast<float4*>(vsm);                                   // draft row, [chunk][thread]
   int32_t* s_par = reinterpret_cast<int32_t*>(vsm + size_t(kMaxChunks) * kVThreads * 16);   // [n] parents of the request
+  int32_t* s_tok = s_par + max_nodes;                                             // [n] tokens of the nodes
+  float* s_acc = reinterpret_cast<float*>(s_tok + max_nodes);                     // [n] acceptance numbers
+  __shared__ int s_walk[3];                                                       // fast path -> block: node, tokens emitted, what next
   // small scalars
   __shared__ VocabScratch s_vs;
   __shared__ int s_cnt[64];
@@ -54,13 +63,45 @@ verify_tree_kernel(const int32_t* __restrict__ parents, const int32_t* __restric
     int p_ = parents[node0 + i];
     if (p_ < -1 || p_ >= i) { p_ = -1; bad = true; }
     s_par[i] = p_;
+    s_tok[i] = tokens[node0 + i];
+    s_acc[i] = accept_u[node0 + i];
   }
   if (bad && status) atomicCAS(status, 0, DYSPEC_ERR_BAD_TREE);
   __syncthreads();
 
   int cur = 0;
   for (int step = 0; step <= n; ++step) {                        // at most n moves; bounded in any case
-    // ---- branches of `cur`, in index order
+    // ---- fast path: warp 0 follows first branches for as long as they are accepted
+    if (warp == 0) {
+      int what = 0;                                              // 1: the block must take over at `cur`; 2: a leaf
+      for (int hop = 0; hop <= n; ++hop) {
+        int first = 0x7fffffff;
+        for (int c0 = 0; c0 < n && first == 0x7fffffff; c0 += 32) {
+          const int i = c0 + lane;
+          const uint32_t m = __ballot_sync(0xffffffffu, i > 0 && i < n && s_par[i] == cur);
+          if (m) first = c0 + __ffs(m) - 1;
+        }
+        if (first == 0x7fffffff) { what = 2; break; }
+        const int y = s_tok[first];
+        if (y < 0 || y >= vocab) { what = 1; break; }            // not a token: the block path reports it
+        float ry = 0.f, dy = 0.f;
+        if (lane == 0) ry = __ldg(target_probs + size_t(node0 + cur) * vocab + y);
+        if (lane == 1) dy = __ldg(draft_probs + size_t(node0 + cur) * vocab + y);
+        ry = __shfl_sync(0xffffffffu, ry, 0);
+        dy = __shfl_sync(0xffffffffu, dy, 1);
+        const float ratio = dy > 0.f ? ry / dy : (ry > 0.f ? INFINITY : 0.f);
+        if (!(s_acc[first] <= ratio)) { what = 1; break; }
+        if (lane == 0 && n_out < max_out) { out_tokens[size_t(r) * max_out + n_out] = y; out_nodes[size_t(r) * max_out + n_out] = first; }
+        ++n_out;
+        cur = first;
+      }
+      if (lane == 0) { s_walk[0] = cur; s_walk[1] = n_out; s_walk[2] = what; }
+    }
+    __syncthreads();
+    cur = s_walk[0];
+    n_out = s_walk[1];
+    if (s_walk[2] == 2 && !bonus_at_leaf) break;                 // as printed: the loop runs while there are branches
+    // ---- the block takes the node over: branches of `cur`, in index order
     if (tid < 64) s_cnt[tid] = 0;
     __syncthreads();
     for (int c0 = warp * 32; c0 < n; c0 += kVThreads) {          // chunk of 32 nodes per warp per round
@@ -118,12 +159,12 @@ verify_tree_kernel(const int32_t* __restrict__ parents, const int32_t* __restric
     bool moved = false;
     for (int b = 0; b < n_child; ++b) {
       const int child = s_child[b];
-      int y = tokens[node0 + child];
+      int y = s_tok[child];
       if (y < 0 || y >= vocab) {                                 // not a token: report it, carry on with a legal index
         if (tid == 0 && status) atomicCAS(status, 0, DYSPEC_ERR_INVALID_ARG);
         y = min(max(y, 0), vocab - 1);
       }
-      const float c = accept_u[node0 + child];
+      const float c = s_acc[child];
       // the owner of token y publishes R[y] and D[y]
       const int y4 = y >> 2, yk = y4 / kVThreads, yt = y4 - yk * kVThreads, ye = y & 3;
       if (tid == yt) {
@@ -194,7 +235,7 @@ cudaError_t launch_verify_tree(const int32_t* parents, const int32_t* tokens, co
                                int32_t* out_tokens, int32_t* out_nodes, int32_t* out_count, int max_out, int32_t* status,
                                cudaStream_t stream) {
   if (n_req <= 0) return cudaSuccess;
-  const size_t smem = size_t(kMaxChunks) * kVThreads * 16 + size_t(max_nodes) * 4;
+  const size_t smem = size_t(kMaxChunks) * kVThreads * 16 + size_t(max_nodes) * 12;
   static DynSmemGrant grant;
   if (cudaError_t e = grant.ensure(verify_tree_kernel, smem); e != cudaSuccess) return e;
   verify_tree_kernel<<<n_req, kVThreads, smem, stream>>>(parents, tokens, draft_probs, target_probs, accept_u, sample_u,
