@@ -42,7 +42,8 @@ struct TcLayout {
   static constexpr int kQBytes = 2 * kTileBytes;
   static constexpr int kRingOffset = kQBytes;
   static constexpr int kBarOffset = kRingOffset + kSlots * kTileBytes;
-  static constexpr int kTotal = kBarOffset + 512;
+  static constexpr int kItemRingOffset = kBarOffset + 512;   // queue plans: the CTA's next work items, 8 entries of 64 bytes
+  static constexpr int kTotal = kItemRingOffset + 512;
 };
 
 // Trace tags (see dyspec_set_trace): tag = role << 14 | event << 10 | key-tile index j.
@@ -282,7 +283,22 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   const WorkItem* my_items = p.items + (kDyn ? size_t(0) : size_t(blockIdx.x) * p.items_stride);
   const bool first_here = blockIdx.x < kFirstItems;
   const int item_end = kDyn ? 0x7fffffff : (first_here ? first.item[blockIdx.x].n_in_cta : my_items[0].n_in_cta);
-  auto item_of = [&](int w, int at) -> WorkItem { return (w == 0 && first_here) ? first.item[blockIdx.x] : my_items[at]; };
+  // Queue plans: the producer warp, which runs ahead of the other roles, also copies each item it takes into
+  // a ring in shared memory, so that the issuing and softmax warps do not pay a global-memory round trip
+  // (about a microsecond, on their critical path) at every item boundary.
+  uint4* q_item = reinterpret_cast<uint4*>(smem + L::kItemRingOffset);
+  auto item_of = [&](int w, int at) -> WorkItem {
+    if (w == 0 && first_here) return first.item[blockIdx.x];
+    if constexpr (kDyn) {
+      if (w > 0) {
+        union { WorkItem it; uint4 v[4]; } u;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) u.v[i] = q_item[((w - 1) & 7) * 4 + i];
+        return u.it;
+      }
+    }
+    return my_items[at];
+  };
   // for the producer warp (all lanes call it): takes the next item off the queue and publishes it
   auto take_index = [&](int k) -> int {
     if (k == 0) return int(blockIdx.x);
@@ -294,12 +310,18 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       const int t = atomicAdd(p.queue, 1) + int(gridDim.x);
       idx = t < p.n_items_total ? t : -1;
       q_idx[(k - 1) & 7] = idx;
-      mbar_arrive(q_full + 8u * uint32_t((k - 1) & 7));
+      if (idx >= 0) {
+        const uint4* src = reinterpret_cast<const uint4*>(p.items + idx);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) q_item[((k - 1) & 7) * 4 + i] = __ldg(src + i);
+      }
+      mbar_arrive(q_full + 8u * uint32_t((k - 1) & 7));      // (release: the entry is written)
       if (idx < 0 && atomicAdd(p.queue + 1, 1) == int(gridDim.x) - 1) {   // every CTA has drained the queue
         p.queue[0] = 0;
         p.queue[1] = 0;
       }
     }
+    __syncwarp();                                            // the other lanes of the producer read the entry too
     return __shfl_sync(0xffffffffu, idx, 0);
   };
   // for every other role
@@ -725,38 +747,34 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       tc_fence_after();
       need_dep();                                          // global writes from here on
       const int head = item.kv_head * g + (row & (g - 1));
-      // the whole O row (D fp32) in registers: all loads in flight together, one wait
-      uint32_t ov[D];
-#pragma unroll
-      for (int c = 0; c < D / 32; ++c) tmem_ld32(t_o + uint32_t(c) * 32u, ov + 32 * c);
-      tmem_wait_ld();
-      tc_fence_before();
-      mbar_arrive(bar(B_OFREE + h));                       // the accumulator may take the next item's products already
       if (item.slot < 0) {
         const float inv = l > 0.f ? 1.f / l : 0.f;
         __nv_bfloat16* out = p.out + (size_t(rq.node0 + node) * p.n_q_heads + head) * D;
-        const bool out_aligned32 = (reinterpret_cast<uintptr_t>(p.out) & 31) == 0;   // rows are multiples of 128 bytes
-        if (ok) {
 #pragma unroll
-          for (int c = 0; c < D / 32; ++c) {
+        for (int c = 0; c < D / 32; ++c) {
+          uint32_t v[32];
+          tmem_ld32(t_o + uint32_t(c) * 32u, v);
+          tmem_wait_ld();
+          if (c == D / 32 - 1) { tc_fence_before(); mbar_arrive(bar(B_OFREE + h)); }
+          if (ok) {
             uint32_t pk[16];
 #pragma unroll
             for (int i = 0; i < 16; ++i)
-              pk[i] = pack_bf16x2(__uint_as_float(ov[32 * c + 2 * i]) * inv, __uint_as_float(ov[32 * c + 2 * i + 1]) * inv);
-            if (out_aligned32) {
-              st_global_v8(out + c * 32, pk);
-              st_global_v8(out + c * 32 + 16, pk + 8);
-            } else {
-#pragma unroll
-              for (int i = 0; i < 4; ++i)
-                *reinterpret_cast<uint4*>(out + c * 32 + i * 8) = make_uint4(pk[4 * i], pk[4 * i + 1], pk[4 * i + 2], pk[4 * i + 3]);
-            }
+              pk[i] = pack_bf16x2(__uint_as_float(v[2 * i]) * inv, __uint_as_float(v[2 * i + 1]) * inv);
+            st_global_v8(out + c * 32, pk);
+            st_global_v8(out + c * 32 + 16, pk + 8);
           }
         }
       } else {
         // partial slot: O [256][D] fp32, then m [256], then l [256]
         float* slot = p.partial + size_t(item.slot) * p.slot_floats;
         const int pr = h * BMH + r;
+        uint32_t ov[D];
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) tmem_ld32(t_o + uint32_t(c) * 32u, ov + 32 * c);
+        tmem_wait_ld();
+        tc_fence_before();
+        mbar_arrive(bar(B_OFREE + h));
         if (ok) {   // the workspace is 256-byte aligned and slots / rows are multiples of 32 bytes
 #pragma unroll
           for (int i = 0; i < D / 8; ++i) st_global_v8(slot + pr * D + i * 8, ov + 8 * i);
