@@ -34,8 +34,9 @@ METRIC = "tree_verify_attention_tree_tokens_per_s"
 UNIT = "tree tokens/s"
 L2_BYTES = 126 * 1024 * 1024
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu
-# captures summarised under profiles/ (tree_attn_small_c2_*.md, tree_attn_tc_c4_*.md)
-NCU_TRAFFIC_BYTES = {"c2_llama2_7b_L1024_n64": 18413312, "c4_llama2_70b_L2048_n512": 18992128}
+# captures summarised under profiles/ (tree_attn_small_c2_*.md, tree_attn_tc_c3_*.md, ..._c4_*.md, ..._c5_*.md)
+NCU_TRAFFIC_BYTES = {"c2_llama2_7b_L1024_n64": 18413312, "c3_llama2_7b_L4096_n256": 77343744,
+                     "c4_llama2_70b_L2048_n512": 18984192, "c5_ragged8_llama2_70b": 154844672}
 NOMINAL_HBM_GBS, NOMINAL_BF16_TFLOPS = 8000.0, 2250.0
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
@@ -256,10 +257,11 @@ def measure_config(torch, runner, w, steps, warmup, device, sparse=False, paged=
                  dependent launch), so this is a period, not a duration;
       dependent  the same chain with a tiny ordinary kernel after every call, which serialises the
                  stream the way the next layer's GEMM does (the tiny kernel's own period is subtracted);
-      isolated   one call at a time: a kernel that overwrites a buffer twice the size of L2 runs first (it
-                 evicts the inputs and keeps the GPU busy while the host enqueues), then an event, the
-                 single attention call, an event; nothing else is on the GPU while the call runs.  Median
-                 of the calls: the duration the roofline fraction is graded on.
+      isolated   one call at a time: a kernel that only spins (no memory traffic, ~50 us) keeps the GPU busy
+                 while the host enqueues an event, the single attention call and an event behind it, so
+                 the host's launch latency is not in the figure; nothing else is on the GPU while the call
+                 runs, and its inputs are cold (calls rotate over the buffer copies).  Median of the
+                 calls: the duration the roofline fraction is graded on.
     The back-to-back figures are taken in five interleaved rounds (step, attention, mask, ...) and
     reported as medians, so that a clock or power state that drifts during the run hits all alike."""
     first = runner.DeviceBatch(w, device=device, sparse=sparse, paged=paged)
@@ -301,20 +303,18 @@ def measure_config(torch, runner, w, steps, warmup, device, sparse=False, paged=
     # ---- one call at a time
     iso_ms = None
     if isolated:
-        flush = torch.empty(2 * L2_BYTES // 4, dtype=torch.float32, device=device)
         stream = torch.cuda.current_stream()
         ts = []
         for i in range(ISOLATED_CALLS):
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             torch.cuda.synchronize()
-            flush.fill_(float(i))           # ~100 us: evicts L2; the three enqueues below land while it runs
+            torch.cuda._sleep(100000)       # ~50 us of spinning: the three enqueues below land while it runs
             e0.record(stream)
             batches[i % copies].attention()
             e1.record(stream)
             torch.cuda.synchronize()
             ts.append(e0.elapsed_time(e1))
         iso_ms = _median(ts[8:])
-        del flush
     status = int(first.status.item())
     return dict(batches=batches, total_ms=total_ms, ms_per_step=total_ms / steps, step_chain_ms=step_chain_ms,
                 attn_ms=attn_ms, mask_ms=mask_ms, dep_ms=dep_ms, iso_ms=iso_ms, chain_calls=rounds * r2 * copies,
@@ -571,7 +571,7 @@ def roofline_entry(m, peaks, peaks_kind):
     chain = m["attn_ms"] * 1e-3
     # nominal figures (HGX B200: 8 TB/s HBM3e as the workload definition quotes it, 2.25 PFLOP/s dense bf16): context only
     common = {"traffic": None, "kernel": "tree attention call (main kernel + any combine launch)",
-              "duration": graded + (": L2 flushed, then one call alone on the GPU, events around it, median of %d" % (ISOLATED_CALLS - 8)
+              "duration": graded + (": one call alone on the GPU (cold inputs), events around it, median of %d" % (ISOLATED_CALLS - 8)
                                     if graded == "isolated" else ": back-to-back period"),
               "launch_us": dur * 1e6, "chain_us": chain * 1e6, "dependent_chain_us": m["dep_ms"] * 1e3,
               "chain_note": "back-to-back calls on independent buffers overlap (programmatic dependent launch): a period, "
@@ -597,6 +597,7 @@ def compact_roofline(idx, wi, mi, ri):
     return {"config": idx, "workload": wi.name, "bound": ri["bound"], "bytes": mi["bytes"], "flops": mi["flops"],
             "roof_us": ri["roof_us"], "isolated_us": None if mi["iso_ms"] is None else mi["iso_ms"] * 1e3,
             "chain_us": mi["attn_ms"] * 1e3, "dependent_chain_us": mi["dep_ms"] * 1e3, "frac": ri["frac"],
+            "traffic": NCU_TRAFFIC_BYTES.get(wi.name),
             "frac_chain": ri["frac_chain"], "graded_on": ri["duration"].split(":")[0]}
 
 
