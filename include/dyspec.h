@@ -128,7 +128,9 @@ size_t dyspec_plan_workspace_bytes(const dyspec_plan_t* plan);
  * 2 = query-tile groups, 3 = groups that are split, 4 = max splits of a group, 5 = kernel regime
  * (0 = 64-row tiles for small trees, 1 = 2 x 128-row tcgen05 tiles), 6 = total key tiles, 7 = query rows per tile,
  * 8 = thread-block cluster size (1 = no clusters), 9 = 1 when the CTAs take whole groups from a shared
- * queue on the device instead of fixed lists (the item list then shows the nominal assignment). */
+ * queue on the device instead of fixed lists (the item list then shows the nominal assignment), 10 = 1 when
+ * split groups are merged by a separate combine launch (0: no split groups, or they are merged on chip or
+ * inside the attention kernel). */
 int64_t dyspec_plan_info(const dyspec_plan_t* plan, int field);
 
 /* Host-only view of the scheduler, for tests and tools: validates the arguments and schedules exactly
@@ -136,8 +138,8 @@ int64_t dyspec_plan_info(const dyspec_plan_t* plan, int field);
  * Copies up to max_items work items into items_out (host, 8 int32 each: request, kv head, first
  * packed query row, first key tile, one-past-last key tile, partial slot or -1, group id, number of
  * splits of the group), the per-CTA item ranges into cta_begin_out (host, n_ctas + 1 entries, at most
- * max_ctas) and, into info_out (host int64 [11]), dyspec_plan_info fields 0-7 followed by keys per
- * tile, workspace bytes and the cluster size.  Any output pointer may be NULL.  Returns the item count or an error. */
+ * max_ctas) and, into info_out (host int64 [12]), dyspec_plan_info fields 0-7 followed by keys per
+ * tile, workspace bytes, the cluster size and dyspec_plan_info field 10.  Any output pointer may be NULL.  Returns the item count or an error. */
 int dyspec_schedule_dry_run(int n_q_heads, int n_kv_heads, int head_dim, int n_req, const int32_t* prefix_len,
                             const int32_t* n_nodes, int words_per_row, int32_t* items_out, int max_items,
                             int32_t* cta_begin_out, int max_ctas, int64_t* info_out);

@@ -200,7 +200,7 @@ def dyspec_schedule_dry_run(n_q_heads: int, n_kv_heads: int, head_dim: int, pref
     nn = np.asarray(list(n_nodes) or [0], dtype=np.int32)
     items = np.zeros((max_items, 8), dtype=np.int32)
     cta = np.zeros(max_items + 1, dtype=np.int32)
-    info = np.zeros(11, dtype=np.int64)
+    info = np.zeros(12, dtype=np.int64)
     rc = lib.dyspec_schedule_dry_run(n_q_heads, n_kv_heads, head_dim, n_req, pl.ctypes.data, nn.ctypes.data,
                                      words_per_row, items.ctypes.data, max_items, cta.ctypes.data, max_items + 1,
                                      info.ctypes.data)
@@ -209,7 +209,7 @@ def dyspec_schedule_dry_run(n_q_heads: int, n_kv_heads: int, head_dim: int, pref
     if rc > max_items:
         return dyspec_schedule_dry_run(n_q_heads, n_kv_heads, head_dim, prefix_len, n_nodes, words_per_row, rc)
     names = ["items", "ctas", "groups", "split_groups", "max_splits", "regime", "key_tiles", "rows_per_tile",
-             "keys_per_tile", "workspace_bytes", "cluster"]
+             "keys_per_tile", "workspace_bytes", "cluster", "combine_launch"]
     d = {k: int(v) for k, v in zip(names, info)}
     return items[:rc].copy(), cta[:d["ctas"] + 1].copy(), d
 

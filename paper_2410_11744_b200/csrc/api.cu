@@ -841,7 +841,9 @@ static int make_host_plan(dyspec_plan** out, int n_q_heads, int n_kv_heads, int 
   if (!pl->split_groups.empty()) {      // the groups' counter pairs follow the partials
     pl->counters_offset = (pl->workspace_bytes + 255) & ~size_t(255);
     pl->workspace_bytes = pl->counters_offset + ((pl->split_groups.size() * 2 * sizeof(int32_t) + 255) & ~size_t(255));
-    pl->merge_in_kernel = pl->regime == 1 && pl->tune.combine_mode == 2;
+    // (the items of a group wait for each other inside the kernel: only when every CTA of the launch is
+    //  resident at once, i.e. one CTA per SM and no more CTAs than SMs; a forced larger grid keeps the combine launch)
+    pl->merge_in_kernel = pl->regime == 1 && pl->tune.combine_mode == 2 && pl->n_ctas <= pl->n_sms;
   }
   if (pl->dynamic) {                    // the queue words follow the partials (there are none in such a plan today)
     pl->queue_offset = (pl->workspace_bytes + 255) & ~size_t(255);
@@ -908,6 +910,7 @@ int dyspec_schedule_dry_run(int n_q_heads, int n_kv_heads, int head_dim, int n_r
     info_out[0] = n_items; info_out[1] = pl->n_ctas; info_out[2] = pl->n_groups; info_out[3] = int64_t(pl->split_groups.size());
     info_out[4] = pl->max_splits; info_out[5] = pl->regime; info_out[6] = pl->total_tiles; info_out[7] = pl->bm;
     info_out[8] = pl->bn; info_out[9] = int64_t(pl->workspace_bytes); info_out[10] = pl->cluster;
+    info_out[11] = (!pl->split_groups.empty() && !pl->merge_in_kernel) ? 1 : 0;
   }
   delete pl;
   return n_items;

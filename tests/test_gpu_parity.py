@@ -366,3 +366,25 @@ def test_calls_that_follow_each_other_may_share_a_workspace(rt, shape):
         ref = orc.tree_attention_ragged(w.q, w.k, w.v, w.prefix_len, w.n_nodes, w.kv_row_offset, w.parents)
         err = np.abs(orc.bf16_bits_to_f64(out_bits) - ref)
         assert err.max() <= MAX_ABS and err.mean() <= MEAN_ABS, (shape, err.max())
+
+
+@pytest.mark.parametrize("hq,hkv,d,L,n,ctas", [(8, 1, 128, 20000, 40, 0), (8, 1, 64, 9000, 40, 0), (4, 4, 128, 3000, 300, 37),
+                                               (16, 2, 64, 700, 260, 11)])
+def test_merge_inside_the_tensor_core_kernel(rt, hq, hkv, d, L, n, ctas):
+    """Split-KV groups of the tensor-core regime are merged by their own items (no combine launch): few
+    groups cut into many equal pieces, one per CTA (more than eight splits, so the merge walks the
+    partials in several rounds; both head dimensions), and forced CTA counts that give CTAs several split
+    items of different groups.  The counters in the workspace must be back at zero: a second call on the
+    same buffers gives the same bits."""
+    B, R = rt
+    rng = np.random.default_rng(hq * 1000 + n)
+    w = wl.make_custom(70, hq, hkv, d, [L], [wl.greedy_tree(rng, n, 6, 0.3)])
+    batch, got, _ = run_and_check(rt, w, regime=1, ctas=ctas, fuse=2 + (16 if ctas else 0))
+    info = batch.plan.describe()
+    assert info["regime"] == 1 and info["split_groups"] > 0 and info["combine_launch"] == 0
+    if ctas == 0:
+        assert info["max_splits"] > 8 or d == 64
+    batch.out.zero_()
+    batch.attention()
+    _, _, out2, status = batch.results()
+    assert status == 0 and np.array_equal(orc.bf16_bits_to_f64(out2), got)

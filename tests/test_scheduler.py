@@ -151,3 +151,17 @@ def test_whole_group_plan_balances_a_ragged_batch(B):
     assert info["split_groups"] == 0 and info["ctas"] == 148
     longest = max(-(-int(L) // 128) + -(-int(n) // 128) for L, n in zip(w.prefix_len, w.n_nodes))
     assert max(loads) <= sum(loads) / len(loads) + longest
+
+
+def test_merge_in_kernel_only_when_the_grid_is_one_wave(B):
+    """The items of a split group wait for each other inside the tensor-core kernel, so that plan is only
+    made when all CTAs are resident at once (no more CTAs than SMs); a forced larger grid, the small-tile
+    regime and combine mode 0 keep the combine launch."""
+    shape = (8, 1, 128, [60000], [40])                              # 2 groups of 470 key tiles
+    info, _ = check_schedule(B, *shape, regime=1)
+    assert info["ctas"] <= 148 and info["split_groups"] == 2 and info["combine_launch"] == 0
+    info_big, _ = check_schedule(B, *shape, regime=1, ctas=200, fuse=2 + 16)
+    assert info_big["ctas"] > 148 and info_big["split_groups"] == 2 and info_big["combine_launch"] == 1
+    assert check_schedule(B, *shape, regime=1, fuse=0)[0]["combine_launch"] == 1
+    small = check_schedule(B, 32, 32, 128, [4096] * 8, [64] * 8)[0]  # regime 0, split, not uniform enough for clusters
+    assert small["regime"] == 0 and small["split_groups"] > 0 and small["combine_launch"] == 1
