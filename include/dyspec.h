@@ -153,15 +153,17 @@ int dyspec_schedule_dry_run(int n_q_heads, int n_kv_heads, int head_dim, int n_r
  * model says that is quicker (and force_ctas is 0), 1 = never, 2 = always. */
 int dyspec_set_tuning(int force_regime, int force_ctas, int combine_mode);
 
-/* Developer aid: event trace of the attention kernels.  trace_buffer is a dev uint64 array of
- * capacity_entries entries that the caller zeroes; while set, CTA 0 of every tensor-core attention
- * launch writes (tag << 44 | SM clock) entries into three equal regions (MMA issuer, softmax half A,
- * softmax half B; tags are listed in csrc/attn_tc.cu; zero entries are unused).  When capacity_entries
- * > 4096 the last 2048 entries are not part of those regions: there each of the first 256 CTAs of an
- * attention launch leaves 8 wall-clock stamps (globaltimer, ns) of its phases, listed where the kernels
- * take them (the tensor-core kernel only in a library built with -DDYSPEC_CTA_STAMPS: its softmax threads
- * sit at the register limit and the stamps cost it ~2 us per launch).  Pass (NULL, 0) to switch it off
- * (the default). */
+/* Developer aid: event trace of the attention kernels.  The hooks are compiled out of the ordinary
+ * library (even never-taken checks in the MMA-issuing and softmax loops cost the tensor-core kernel
+ * 8 - 10 %): build with DYSPEC_NVCC_FLAGS="-DDYSPEC_TRACE" (event trace) and / or "-DDYSPEC_CTA_STAMPS"
+ * (per-CTA wall-clock stamps); in an ordinary build a non-NULL buffer is refused with
+ * DYSPEC_ERR_UNSUPPORTED.  trace_buffer is a dev uint64 array of capacity_entries entries that the
+ * caller zeroes; while set, CTA 0 of every tensor-core attention launch writes (tag << 44 | SM clock)
+ * entries into three equal regions (MMA issuer, softmax half A, softmax half B; tags are listed in
+ * csrc/attn_tc.cu; zero entries are unused).  When capacity_entries > 4096 the last 2048 entries are
+ * not part of those regions: there each of the first 256 CTAs of an attention launch leaves 8
+ * wall-clock stamps (globaltimer, ns) of its phases, listed where the kernels take them.  Pass
+ * (NULL, 0) to switch it off (the default). */
 int dyspec_set_trace(void* trace_buffer, int capacity_entries);
 
 /*

@@ -613,6 +613,9 @@ int dyspec_set_tuning(int force_regime, int force_ctas, int combine_mode) {
 
 int dyspec_set_trace(void* trace_buffer, int capacity_entries) {
   if (capacity_entries < 0 || (trace_buffer == nullptr) != (capacity_entries == 0)) return DYSPEC_ERR_INVALID_ARG;
+#if !defined(DYSPEC_TRACE) && !defined(DYSPEC_CTA_STAMPS)
+  if (trace_buffer != nullptr) return DYSPEC_ERR_UNSUPPORTED;      // the hooks are compiled out of this build
+#endif
   std::lock_guard<std::mutex> lock(g_tuning_mutex);
   g_tuning.trace = static_cast<unsigned long long*>(trace_buffer);
   g_tuning.trace_capacity = capacity_entries;

@@ -177,8 +177,12 @@ tree_attn_small_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
   // taken by thread 0 for the CTA's first item: 0 entry, 3 first scores read, 5 key loop done, 1 set 1's
   // partial folded in, 6 partial parked, 2 pushes issued, 4 (owners) last fold done, 7 exit
   auto stamp = [&](int k) {
+#ifdef DYSPEC_CTA_STAMPS
     if (p.trace != nullptr && blockIdx.x < 256 && p.trace_capacity > 4096)
       p.trace[p.trace_capacity - 2048 + 8 * blockIdx.x + k] = global_timer_ns();
+#else
+    (void)k;
+#endif
   };
   if (threadIdx.x == 0) stamp(0);
   if (threadIdx.x == kProducerWarp * 32) {      // the descriptors' fetch overlaps the set-up below
