@@ -373,9 +373,14 @@ def verification_experiment(torch, workloads, B, peaks, device):
     visited nodes."""
     rows = []
     rng = np.random.default_rng(workloads.MASTER_SEED + 7000)
-    for label, trees in (("1 request, 64 nodes", [workloads.greedy_tree(rng, 64, 8, 0.3)]),
-                         ("8 requests, 256 nodes", [workloads.greedy_tree(rng, 256, 8, 0.1) for _ in range(8)])):
-        case = workloads.make_verify_case(workloads.MASTER_SEED + 7001, 32000, trees, sharpness=3.0, disagreement=1.0)
+    tree64 = [workloads.greedy_tree(rng, 64, 8, 0.3)]
+    for label, trees, disagreement in (
+            ("1 request, 64 nodes", tree64, 1.0),
+            ("8 requests, 256 nodes", [workloads.greedy_tree(rng, 256, 8, 0.1) for _ in range(8)], 1.0),
+            # a draft close to the target (the regime speculative decoding is run in): first branches are accepted
+            # and the walk needs two numbers per node instead of two rows
+            ("1 request, 64 nodes, draft close to target", tree64, 0.05)):
+        case = workloads.make_verify_case(workloads.MASTER_SEED + 7001, 32000, trees, sharpness=3.0, disagreement=disagreement)
         n_req = len(trees)
         N = int(case.node_offsets[-1])
         row_bytes = 2 * N * case.vocab * 4
@@ -401,10 +406,12 @@ def verification_experiment(torch, workloads, B, peaks, device):
         torch.cuda.synchronize()
         us = _time_replays(torch, g, 20) / (20 * copies) * 1e3
         emitted = cnt.cpu().numpy()
-        visited = int(emitted.sum())                       # nodes whose rows were read: accepted ones + the start node - ... = tokens emitted
+        visited = int(emitted.sum())                       # an upper bound of the nodes whose rows were read (a node whose first branch
+                                                           # is accepted reads two numbers, not its rows)
         nbytes = visited * 2 * case.vocab * 4
-        rows.append({"case": label, "vocab": case.vocab, "call_us": us, "tokens_emitted": emitted.tolist(),
-                     "rows_read": visited, "bytes": nbytes, "achieved_gbs": nbytes / (us * 1e-6) / 1e9,
+        rows.append({"case": label, "vocab": case.vocab, "call_us": us, "us_per_token": us / max(1, int(emitted.max())),
+                     "tokens_emitted": emitted.tolist(),
+                     "rows_read_at_most": visited, "bytes_at_most": nbytes, "achieved_gbs": nbytes / (us * 1e-6) / 1e9,
                      "frac_of_hbm": nbytes / (us * 1e-6) / 1e9 / peaks["hbm_gbs"], "copies": copies,
                      "status": int(status.item())})
         del bufs
