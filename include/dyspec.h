@@ -147,8 +147,10 @@ int dyspec_schedule_dry_run(int n_q_heads, int n_kv_heads, int head_dim, int n_r
 /* Testing knobs, process-wide; a plan keeps the values it was created with: force the regime (-1 = automatic), the number of
  * CTAs the scheduler balances over (0 = automatic; a negative value -c instead sets the scheduler's
  * per-item cost to c key tiles), and combine_mode = m + 16 k.  m says how split-KV partials are merged:
- * 0 = by the separate combine kernel, 2 (default) = inside a thread-block cluster through distributed
- * shared memory when the plan is uniform enough, else as 0.  k says whether the scheduler may deal whole
+ * 0 = by the separate combine kernel, 2 (default) = without a combine launch where the plan allows: in the
+ * small-tile regime inside a thread-block cluster through distributed shared memory when the plan is
+ * uniform enough, in the tcgen05 regime by the split items themselves inside the attention kernel when the
+ * grid is one wave; else as 0.  k says whether the scheduler may deal whole
  * (unsplit) groups to the CTAs instead of cutting them to equal budgets: 0 (default) = when its cost
  * model says that is quicker (and force_ctas is 0), 1 = never, 2 = always. */
 int dyspec_set_tuning(int force_regime, int force_ctas, int combine_mode);
@@ -185,11 +187,11 @@ int dyspec_plan_build_tree_mask(const dyspec_plan_t* plan, const int32_t* parent
  *   k_cache,v_cache dev bf16 [kv_total_rows][H_kv][D]    (16-byte aligned)
  *   ancestor_bits  dev uint32 [sum n_r][W]               (from the mask builder)
  *   out            dev bf16 [sum n_r][H_q][D]            (written)
- *   workspace      dev, >= dyspec_plan_workspace_bytes(plan), 256-byte aligned; its arrival counters
- *                  must be zero before the first call (dyspec_plan_create's caller zeroes it once;
- *                  the kernels leave them zero).  Two calls that overlap on the GPU need two workspaces
- *                  (a workspace holds words that a launch uses and clears: the head of the plan's
- *                  shared work queue); calls that follow each other on one stream may share one, and a
+ *   workspace      dev, >= dyspec_plan_workspace_bytes(plan), 256-byte aligned; it must be zero before the
+ *                  first call (the caller zeroes it once; the kernels leave its counters zero).  Two
+ *                  calls that overlap on the GPU need two workspaces (a workspace holds the split-KV
+ *                  partials and words that a launch uses and clears: the arrival counters of the split
+ *                  groups, the head of the plan's shared work queue); calls that follow each other on one stream may share one, and a
  *                  plan may be shared by any number of calls.
  *   status         dev int32 [1] or NULL
  */

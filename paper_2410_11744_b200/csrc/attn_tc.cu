@@ -20,6 +20,9 @@
 //   warps 8-11    the same for query half B.  The two halves alternate on the tensor pipe, so one
 //                 half's softmax overlaps the other half's MMAs, and each K/V tile is loaded once
 //                 for 256 query rows.
+// An item whose group was cut along the keys writes an fp32 partial (O, m, l); after all of its items a CTA
+// merges, for each of its split items, a share of the group's rows (no combine launch; see the end of the
+// softmax branch).
 // Every wait is bounded (see mbar_wait); every TMA load goes to this CTA alone, and the kernel is never launched in clusters.
 #include "common.cuh"
 
@@ -335,7 +338,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   const int g = p.group_size;
 
   // Register budget: the softmax threads hold a whole S row; the control warps need few registers.
-  trigger_dependents();     // the combine kernel may be scheduled; it waits for this grid before reading partials
+  trigger_dependents();     // the next kernel of the stream may be scheduled; it waits for this grid before it touches what this one writes
   if (warp < 4) {
   asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
   if (warp == 0) {
