@@ -750,7 +750,46 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       tc_fence_after();
       need_dep();                                          // global writes from here on
       const int head = item.kv_head * g + (row & (g - 1));
-      if (item.slot < 0) {
+      // The CTA's LAST item (fixed lists) leaves through shared memory: this half's region of the Q tile is
+      // dead by now (only this half's score products read it, and they have all completed), so the rows
+      // are parked there, 16-byte chunks XOR-swizzled by the row, and copied out with whole rows per warp
+      // instruction instead of one 32-byte piece of 32 different rows.
+      bool staged = false;
+      if constexpr (!kDyn) staged = w == item_end - 1;
+      constexpr int RB = 2 * D;                            // bytes of a row in the staging region (128 rows of them = one Q half)
+      constexpr int CH = RB / 16;                          // 16-byte chunks per row
+      uint8_t* stage = smem + h * L::kTileBytes;
+      auto stage_at = [&](int srow, int ch) -> uint4* {
+        return reinterpret_cast<uint4*>(stage + (ch >> 3) * L::kPanelBytes + srow * 128 + (((ch & 7) ^ (srow & 7)) << 4));
+      };
+      if (item.slot < 0 && staged) {
+        const float inv = l > 0.f ? 1.f / l : 0.f;
+        uint32_t ov[D];
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) tmem_ld32(t_o + uint32_t(c) * 32u, ov + 32 * c);
+        tmem_wait_ld();
+        tc_fence_before();
+        mbar_arrive(bar(B_OFREE + h));
+#pragma unroll
+        for (int ch = 0; ch < CH; ++ch) {                  // bf16 row: D / 2 words = CH chunks
+          uint4 v;
+          v.x = pack_bf16x2(__uint_as_float(ov[8 * ch + 0]) * inv, __uint_as_float(ov[8 * ch + 1]) * inv);
+          v.y = pack_bf16x2(__uint_as_float(ov[8 * ch + 2]) * inv, __uint_as_float(ov[8 * ch + 3]) * inv);
+          v.z = pack_bf16x2(__uint_as_float(ov[8 * ch + 4]) * inv, __uint_as_float(ov[8 * ch + 5]) * inv);
+          v.w = pack_bf16x2(__uint_as_float(ov[8 * ch + 6]) * inv, __uint_as_float(ov[8 * ch + 7]) * inv);
+          *stage_at(r, ch) = v;
+        }
+        named_sync(kBarPartial + h, BMH);
+#pragma unroll 4
+        for (int id = r; id < BMH * CH; id += BMH) {
+          const int srow = id / CH, ch = id % CH;
+          const int grow = item.row0 + h * BMH + srow;
+          if (grow < n_rows) {
+            __nv_bfloat16* dst = p.out + (size_t(rq.node0 + (grow >> p.log2_g)) * p.n_q_heads + item.kv_head * g + (grow & (g - 1))) * D;
+            *reinterpret_cast<uint4*>(dst + ch * 8) = *stage_at(srow, ch);
+          }
+        }
+      } else if (item.slot < 0) {
         const float inv = l > 0.f ? 1.f / l : 0.f;
         __nv_bfloat16* out = p.out + (size_t(rq.node0 + node) * p.n_q_heads + head) * D;
 #pragma unroll
@@ -778,7 +817,24 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         tmem_wait_ld();
         tc_fence_before();
         mbar_arrive(bar(B_OFREE + h));
-        if (ok) {   // the workspace is 256-byte aligned and slots / rows are multiples of 32 bytes
+        if (staged) {
+          // an fp32 row is twice the staging row: two passes of D / 2 columns
+#pragma unroll
+          for (int pass = 0; pass < 2; ++pass) {
+#pragma unroll
+            for (int ch = 0; ch < CH; ++ch)
+              *stage_at(r, ch) = make_uint4(ov[pass * (D / 2) + 4 * ch], ov[pass * (D / 2) + 4 * ch + 1],
+                                            ov[pass * (D / 2) + 4 * ch + 2], ov[pass * (D / 2) + 4 * ch + 3]);
+            named_sync(kBarPartial + h, BMH);
+#pragma unroll 4
+            for (int id = r; id < BMH * CH; id += BMH) {
+              const int srow = id / CH, ch = id % CH;
+              if (item.row0 + h * BMH + srow < n_rows)
+                *reinterpret_cast<uint4*>(slot + (h * BMH + srow) * D + pass * (D / 2) + 4 * ch) = *stage_at(srow, ch);
+            }
+            if (pass == 0) named_sync(kBarPartial + h, BMH);   // all of pass 0 is read before the region is written again
+          }
+        } else if (ok) {   // the workspace is 256-byte aligned and slots / rows are multiples of 32 bytes
 #pragma unroll
           for (int i = 0; i < D / 8; ++i) st_global_v8(slot + pr * D + i * 8, ov + 8 * i);
         }
