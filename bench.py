@@ -790,7 +790,7 @@ def run_ours(args):
         "config": {"workload": w.name, "n_q_heads": w.n_q_heads, "n_kv_heads": w.n_kv_heads, "head_dim": w.head_dim,
                    "prefix_len": w.prefix_len.tolist(), "n_nodes": w.n_nodes.tolist(), "parallelism": "replicas only",
                    "l2": f"inputs rotate over {m['copies']} independent copies ({m['copies'] * m['bytes'] / 1e6:.0f} MB > 2x L2)",
-                   "step": "mask build + tree attention + split-KV combine", "plan": m["info"]},
+                   "step": "mask build + tree attention (split-KV merge included)", "plan": m["info"]},
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
         "gpu_launches": m["launches_per_step"] * args.steps,
