@@ -901,6 +901,78 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           for (int pr0 = row_lo + KR * mw; pr0 < row_hi; pr0 += 8 * KR) {
             const int lk = lane >> 3, lu = lane & 7;
             const int lrow = min(pr0 + lk, 2 * BMH - 1);
+            if (ns <= 8) {
+              // Up to eight splits (the usual case): the row's scalars AND the first four partial rows are
+              // requested together, before anything is used: one round trip for up to four splits, two beyond.
+              float mv = -INFINITY, lv = 0.f;
+              if (lu < ns) {
+                const float* sl = base_m + size_t(lu) * p.slot_floats;
+                mv = ld_cg_f32(sl + lrow);
+                lv = ld_cg_f32(sl + 2 * BMH + lrow);
+              }
+              float acc[KR][V];
+#pragma unroll
+              for (int k = 0; k < KR; ++k)
+#pragma unroll
+                for (int e = 0; e < V; ++e) acc[k][e] = 0.f;
+              float f_l = 0.f, lsum = 0.f;
+#pragma unroll
+              for (int s1 = 0; s1 < 8; s1 += KS) {
+                if (s1 >= ns) break;
+                float vv[KR][KS][V];
+#pragma unroll
+                for (int k = 0; k < KR; ++k)
+#pragma unroll
+                  for (int u = 0; u < KS; ++u) {
+                    const int pr = min(pr0 + k, 2 * BMH - 1);
+                    const float* sl = base + size_t(min(s1 + u, ns - 1)) * p.slot_floats + pr * D;
+                    if constexpr (V == 4) {
+                      const float4 x = ld_cg_f32x4(sl + lane * 4);
+                      vv[k][u][0] = x.x; vv[k][u][1] = x.y; vv[k][u][2] = x.z; vv[k][u][3] = x.w;
+                    } else {
+                      const float2 x = ld_cg_f32x2(sl + lane * 2);
+                      vv[k][u][0] = x.x; vv[k][u][1] = x.y;
+                    }
+                  }
+                if (s1 == 0) {                                 // the row's reference and this lane's weight
+                  float m_r = mv;
+                  m_r = fmaxf(m_r, __shfl_xor_sync(0xffffffffu, m_r, 1));
+                  m_r = fmaxf(m_r, __shfl_xor_sync(0xffffffffu, m_r, 2));
+                  m_r = fmaxf(m_r, __shfl_xor_sync(0xffffffffu, m_r, 4));
+                  f_l = lu < ns ? fast_exp2(mv - (m_r == -INFINITY ? 0.f : m_r)) : 0.f;
+                  lsum = f_l * lv;
+                  lsum += __shfl_xor_sync(0xffffffffu, lsum, 1);
+                  lsum += __shfl_xor_sync(0xffffffffu, lsum, 2);
+                  lsum += __shfl_xor_sync(0xffffffffu, lsum, 4);
+                }
+#pragma unroll
+                for (int k = 0; k < KR; ++k)
+#pragma unroll
+                  for (int u = 0; u < KS; ++u) {
+                    const float f = __shfl_sync(0xffffffffu, f_l, 8 * k + s1 + u);     // 0 for a split that does not exist
+#pragma unroll
+                    for (int e = 0; e < V; ++e) acc[k][e] += f * vv[k][u][e];
+                  }
+              }
+#pragma unroll
+              for (int k = 0; k < KR; ++k) {
+                const float lk_sum = __shfl_sync(0xffffffffu, lsum, 8 * k);
+                const int pr = pr0 + k, row = item.row0 + pr;
+                if (pr < row_hi && row < n_rows) {
+                  const float inv = lk_sum > 0.f ? 1.f / lk_sum : 0.f;
+                  __nv_bfloat16* out = p.out + (size_t(item.node0 + (row >> p.log2_g)) * p.n_q_heads + item.kv_head * g + (row & (g - 1))) * D;
+                  if constexpr (V == 4) {
+                    uint2 o;
+                    o.x = pack_bf16x2(acc[k][0] * inv, acc[k][1] * inv);
+                    o.y = pack_bf16x2(acc[k][2] * inv, acc[k][3] * inv);
+                    *reinterpret_cast<uint2*>(out + lane * 4) = o;
+                  } else {
+                    *reinterpret_cast<uint32_t*>(out + lane * 2) = pack_bf16x2(acc[k][0] * inv, acc[k][1] * inv);
+                  }
+                }
+              }
+              continue;
+            }
             float m_l = -INFINITY;
             for (int s_ = lu; s_ < ns; s_ += 8) m_l = fmaxf(m_l, ld_cg_f32(base_m + size_t(s_) * p.slot_floats + lrow));
             m_l = fmaxf(m_l, __shfl_xor_sync(0xffffffffu, m_l, 1));
