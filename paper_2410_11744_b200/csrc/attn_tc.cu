@@ -59,7 +59,7 @@ struct TcLayout {
 // barrier indices (8 bytes each)
 enum { B_QFULL = 0, B_QFREE = 1, B_SLOT_FULL = 2, B_SLOT_EMPTY = B_SLOT_FULL + kSlots,
        B_SREADY = B_SLOT_EMPTY + kSlots, B_PREADY = B_SREADY + 2, B_ODONE = B_PREADY + 2, B_OFREE = B_ODONE + 2,
-       B_PVDONE = B_OFREE + 2, B_COUNT = B_PVDONE + 2 };
+       B_PVDONE = B_OFREE + 2, B_QFULLB = B_PVDONE + 2, B_COUNT = B_QFULLB + 1 };
 
 // Hardware named barriers for thread-to-thread hand-offs inside the CTA (P ready: 128 softmax threads
 // -> the MMA-issuing warp): an order of magnitude quicker to notice than an mbarrier in shared memory
@@ -251,6 +251,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
 
   if (threadIdx.x == 0) {
     mbar_init(bar(B_QFULL), 1);
+    mbar_init(bar(B_QFULLB), 1);
     mbar_init(bar(B_QFREE), 2);
     for (int s = 0; s < kSlots; ++s) {
       mbar_init(bar(B_SLOT_FULL + s), 1);
@@ -362,13 +363,17 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         const WorkItem& rq = item;
         const int nh = (rq.n_nodes * g - item.row0 > BMH) ? 2 : 1;
         mbar_wait(bar(B_QFREE), (qit & 1) ^ 1, abort_flag, p.status);
-        if (elected) {
-          mbar_expect_tx(bar(B_QFULL), uint32_t(nh) * L::kTileBytes);
-          for (int h = 0; h < nh; ++h)
+        // Half A's rows first, then (below) the first K tile, then half B's rows: the item's first score
+        // product needs only the first two, and at a launch's start every CTA is waiting for exactly that.
+        auto load_q_half = [&](int h, int b) {
+          if (elected) {
+            mbar_expect_tx(bar(b), L::kTileBytes);
             for (int pn = 0; pn < L::kPanels; ++pn)
-              tma_load_3d(s_q + h * L::kTileBytes + pn * L::kPanelBytes, &map_q, bar(B_QFULL), pn * 64, item.kv_head * g,
+              tma_load_3d(s_q + h * L::kTileBytes + pn * L::kPanelBytes, &map_q, bar(b), pn * 64, item.kv_head * g,
                           rq.node0 + ((item.row0 + h * BMH) >> p.log2_g));
-        }
+          }
+        };
+        load_q_half(0, B_QFULL);
         const int n_prefix_tiles = (rq.prefix_len + BN - 1) / BN;
         // Prefix tiles stream at once; the set of tree tiles may depend on the mask kernel's output,
         // so it is settled (after waiting for that kernel) only when the walk reaches the tree.
@@ -399,6 +404,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 tma_load_3d(s_ring + slot * L::kTileBytes + pn * L::kPanelBytes, kv == 0 ? &map_k : &map_v,
                             bar(B_SLOT_FULL + slot), pn * 64, item.kv_head, int(row));
             }
+            if (j == 0 && kv == 0 && nh == 2) load_q_half(1, B_QFULLB);
           }
         }
       }
@@ -483,7 +489,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           if (!two && elected) tc_commit(bar(b));                 // no half B in this item: warp 1 gives both
         };
         const bool mine = h == 0 || two;
-        if (mine) mbar_wait(bar(B_QFULL), qit & 1, abort_flag, p.status);
+        if (mine) mbar_wait(bar(h == 0 ? B_QFULL : B_QFULLB), (h == 0 ? qit : n_it) & 1, abort_flag, p.status);
         {
           const uint32_t kslot = sc % kSlots, kph = (sc / kSlots) & 1;
           ++sc;
