@@ -508,7 +508,8 @@ def compact_kv(cache: np.ndarray, kv_row0: int, prefix_len: int, accepted_nodes:
 # Paged KV cache (the paper is silent on the cache's memory layout; this is the layout a serving stack
 # keeps its caches in).  The cache is a pool of pages of page_size rows.  Prefix token t of a request
 # lies in the request's page number t // page_size, at row t % page_size of that page; the request's
-# tree rows (one per node, in node order) are a contiguous run of pool rows of their own.
+# tree rows (one per node, in node order) are either a contiguous run of pool rows of their own, or
+# (tree_row_offset / tree_row0 = None) tokens L, L + 1, ... of the same paged sequence.
 # ----------------------------------------------------------------------------------------------------
 def paged_prefix_rows(page_table_row: Sequence[int], page_size: int, length: int) -> List[int]:
     """Pool row of each of the first `length` tokens of a request whose pages are page_table_row."""
@@ -518,13 +519,17 @@ def paged_prefix_rows(page_table_row: Sequence[int], page_size: int, length: int
 def tree_attention_paged(q_bits, k_pool, v_pool, page_table, page_size: int, prefix_len, n_nodes, tree_row_offset,
                          parents_list, scale: float | None = None):
     """Tree-verify attention (same definition as tree_attention) with the prefix keys read through the
-    page table and the tree keys from rows tree_row_offset[r] ..  Returns float64 [sum n][H_q][D]."""
+    page table and the tree keys from rows tree_row_offset[r] .. (tree_row_offset None: node j is token
+    L + j of the paged sequence).  Returns float64 [sum n][H_q][D]."""
     outs = []
     qo = 0
     for r in range(len(prefix_len)):
         n, L = int(n_nodes[r]), int(prefix_len[r])
         if n:
-            rows = paged_prefix_rows(page_table[r], page_size, L) + [int(tree_row_offset[r]) + j for j in range(n)]
+            if tree_row_offset is None:
+                rows = paged_prefix_rows(page_table[r], page_size, L + n)
+            else:
+                rows = paged_prefix_rows(page_table[r], page_size, L) + [int(tree_row_offset[r]) + j for j in range(n)]
             outs.append(tree_attention(q_bits[qo:qo + n], k_pool[rows], v_pool[rows], L, parents_list[r], scale))
         qo += n
     if not outs:
@@ -535,11 +540,16 @@ def tree_attention_paged(q_bits, k_pool, v_pool, page_table, page_size: int, pre
 def compact_kv_paged(pool: np.ndarray, page_table_row: Sequence[int], page_size: int, tree_row0: int, prefix_len: int,
                      accepted_nodes: Sequence[int], keep_root: bool = False) -> int:
     """The kept nodes k_0 < k_1 < ... (see kept_nodes) become prefix tokens L, L + 1, ...: the pool row
-    of token L + i (through the page table) takes the content of tree row tree_row0 + k_i.  Returns the
-    new prefix length."""
+    of token L + i (through the page table) takes the content of tree row tree_row0 + k_i (tree_row0 None:
+    of token L + k_i, the node's row inside the paged sequence).  Returns the new prefix length."""
     nodes = kept_nodes(accepted_nodes, keep_root)
     L = int(prefix_len)
     dst = paged_prefix_rows(page_table_row, page_size, L + len(nodes))[L:]
-    for d, a in zip(dst, nodes):
-        pool[d] = pool[int(tree_row0) + a]
+    if tree_row0 is None:
+        src = [int(page_table_row[(L + a) // page_size]) * page_size + (L + a) % page_size for a in nodes]
+    else:
+        src = [int(tree_row0) + a for a in nodes]
+    gathered = [pool[s_].copy() for s_ in src]               # all reads first: the definition is a gather
+    for d, row in zip(dst, gathered):
+        pool[d] = row
     return L + len(nodes)

@@ -309,14 +309,17 @@ class PagedWorkload:
         return int(self.k.shape[0])
 
 
-def to_paged(w: Workload, page_size: int, seed: int = 0, room_for_accepted: bool = True) -> PagedWorkload:
+def to_paged(w: Workload, page_size: int, seed: int = 0, room_for_accepted: bool = True,
+             tree_in_pages: bool = False) -> PagedWorkload:
     """Scatters w's contiguous cache into a paged pool.  Every request gets enough pages for its prefix
     (plus its tree size when room_for_accepted, so that accepted tokens have somewhere to go), the page
     numbers of all requests are shuffled together, rows of a page past the prefix hold finite filler
     (large values, so that a key that leaks through a mask shows), and the tree rows follow the pages
-    with odd gaps between requests."""
+    with odd gaps between requests.  With tree_in_pages the tree rows are tokens L .. L + n - 1 of the
+    paged sequence instead (tree_row_offset is then None)."""
     rng = np.random.default_rng(seed + 99173)
     n_req = w.n_req
+    room_for_accepted = room_for_accepted or tree_in_pages
     need = [-(-(int(w.prefix_len[r]) + (int(w.n_nodes[r]) if room_for_accepted else 0)) // page_size) for r in range(n_req)]
     pages_per_req = max(need + [1])
     n_pages = sum(need) + 2                                   # two pages nobody owns
@@ -344,7 +347,13 @@ def to_paged(w: Workload, page_size: int, seed: int = 0, room_for_accepted: bool
             dst = int(page_table[r, t0 // page_size]) * page_size
             k[dst:dst + cnt] = w.k[o + t0:o + t0 + cnt]
             v[dst:dst + cnt] = w.v[o + t0:o + t0 + cnt]
+        if tree_in_pages:
+            for t in range(L, L + n):
+                dst = int(page_table[r, t // page_size]) * page_size + t % page_size
+                k[dst] = w.k[o + t]
+                v[dst] = w.v[o + t]
+            continue
         t = int(tree_row_offset[r])
         k[t:t + n] = w.k[o + L:o + L + n]
         v[t:t + n] = w.v[o + L:o + L + n]
-    return PagedWorkload(w, int(page_size), page_table, tree_row_offset, k, v)
+    return PagedWorkload(w, int(page_size), page_table, None if tree_in_pages else tree_row_offset, k, v)

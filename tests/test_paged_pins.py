@@ -110,3 +110,51 @@ def test_paged_compaction_keeps_the_root_like_the_contiguous_one():
     rows = orc.paged_prefix_rows(pw.page_table[0], 4, new_L)
     assert np.array_equal(pool[rows], cont[:new_L])
     assert np.array_equal(pool[rows[L]], w.k[L])                          # token L is the root's row
+
+
+# ---- tree rows inside the paged sequence (tokens L .. L + n - 1 of the request's pages) ----------------
+def test_tree_rows_inside_the_pages_change_nothing():
+    """The same keys in the same order, whatever pages the tree rows lie in: bit-identical to the
+    contiguous form, also when a tree crosses page boundaries at an odd offset."""
+    for w in _cases():
+        ref = orc.tree_attention_ragged(w.q, w.k, w.v, w.prefix_len, w.n_nodes, w.kv_row_offset, w.parents)
+        for page_size, seed in ((4, 0), (8, 1), (16, 2)):
+            pw = wl.to_paged(w, page_size, seed, tree_in_pages=True)
+            assert pw.tree_row_offset is None
+            got = orc.tree_attention_paged(w.q, pw.k, pw.v, pw.page_table, page_size, w.prefix_len, w.n_nodes,
+                                           None, w.parents)
+            assert np.array_equal(got, ref)
+
+
+def test_tree_rows_inside_the_pages_hand_example():
+    """Pages of 4 rows, the request owns pages 2 then 0; prefix 3 tokens, 3 nodes: node 0 is token 3
+    (pool row 11), nodes 1 and 2 are tokens 4, 5 (pool rows 0, 1).  A star forest sees prefix + self only:
+    V of the node's own row leaks into its output and nobody else's."""
+    w = wl.make_custom(5, 1, 1, 8, [3], [wl.star_forest(3)])
+    pw = wl.to_paged(w, 4, 0, tree_in_pages=True)
+    table = pw.page_table[0]
+    rows = [int(table[t // 4]) * 4 + t % 4 for t in range(6)]
+    assert np.array_equal(pw.k[rows], w.k[:6]) and np.array_equal(pw.v[rows], w.v[:6])
+    base = orc.tree_attention_paged(w.q, pw.k, pw.v, pw.page_table, 4, w.prefix_len, w.n_nodes, None, w.parents)
+    v2 = pw.v.copy()
+    v2[rows[4]] ^= 0x0040                                    # node 1's own V row
+    moved = orc.tree_attention_paged(w.q, pw.k, v2, pw.page_table, 4, w.prefix_len, w.n_nodes, None, w.parents)
+    assert not np.array_equal(moved[1], base[1])
+    assert np.array_equal(moved[0], base[0]) and np.array_equal(moved[2], base[2])
+
+
+def test_in_sequence_compaction_is_the_contiguous_one_read_through_the_table():
+    """Source and destination rows overlap here (token L + 1 receives node 2 after node 1 ... was read):
+    the definition is a gather, as in the contiguous form."""
+    L, n = 6, 12
+    w = wl.make_custom(72, 2, 2, 8, [L], [wl.chain_tree(n)])
+    for listed, keep_root in (([1, 2, 3, -1], False), ([1, 2, 3, -1], True), ([2, 5, 9], True), ([0, 1, 2], False), ([], True)):
+        cont = w.k.copy()
+        new_L = orc.compact_kv(cont, 0, L, listed, keep_root=keep_root)
+        pw = wl.to_paged(w, 4, 3, tree_in_pages=True)
+        pool = pw.k.copy()
+        assert orc.compact_kv_paged(pool, pw.page_table[0], 4, None, L, listed, keep_root=keep_root) == new_L
+        rows = orc.paged_prefix_rows(pw.page_table[0], 4, L + n)
+        assert np.array_equal(pool[rows], cont[:L + n])       # kept rows moved, everything behind them as it was
+        others = np.setdiff1d(np.arange(pw.pool_rows), rows)
+        assert np.array_equal(pool[others], pw.k[others])
