@@ -401,15 +401,23 @@ int dyspec_compact_kv(void* k_cache, void* v_cache, const int64_t* kv_row_offset
  * and the request's tree rows (one per node, in node order) are the contiguous pool rows
  * tree_row_offset[r] .. tree_row_offset[r] + n_r - 1, outside the prefix pages (scratch rows of the
  * speculation step; dyspec_compact_kv_paged moves the accepted ones into the prefix pages).
- * Rows of a mapped page past the prefix are read and masked: they must hold finite values (zero a page
- * when it is allocated).  A page number that is negative or beyond the pool reads as zeros, it does not
- * fault; the result for that request is then meaningless.
+ * Alternatively (tree_row_offset == NULL) the tree rows are part of the paged sequence: node j of
+ * request r is token L_r + j, addressed by the rule above like a prefix token (the draft tokens' K/V were
+ * appended to the sequence's pages).  Key tiles then follow the sequence, whatever L_r modulo the tile
+ * size is: a row's mask slice for a tile is its bit row shifted by that remainder.  The per-node tile sets
+ * (node_tiles) are ignored by such a plan.
+ * Rows of a mapped page past the request's last token are read and masked: they must hold finite values
+ * (zero a page when it is allocated).  A page number that is negative or beyond the pool reads as zeros,
+ * it does not fault; the result for that request is then meaningless.
  *
- * dyspec_plan_create_paged: as dyspec_plan_create, with tree_row_offset (host int64 [n_req]) in place of
- * kv_row_offset, kv_total_rows = rows of the pool, and the page size.  The plan works with
+ * dyspec_plan_create_paged: as dyspec_plan_create, with tree_row_offset (host int64 [n_req], or NULL: tree
+ * rows inside the pages) in place of kv_row_offset, kv_total_rows = rows of the pool, and the page size.
+ * The plan works with
  * dyspec_tree_attention_paged only (the contiguous calls return DYSPEC_ERR_INVALID_ARG for it, and this
  * call for a contiguous plan); the mask builder and reorder calls take either kind.
- *   page_table   dev int32 [n_req][pages_per_req]; entries past a request's last prefix page are not read.
+ *   page_table   dev int32 [n_req][pages_per_req]; entries past a request's last prefix page (last page of
+ *                prefix + tree when the tree rows are inside the pages, which pages_per_req must cover:
+ *                DYSPEC_ERR_INVALID_ARG otherwise) are not read.
  *                Like q and the caches it is read before the preceding kernel of the stream is known to
  *                have finished, so it must not be written by the kernel launched just before this call.
  *   node_tiles   as in dyspec_tree_attention_ragged_sparse, or NULL
@@ -429,6 +437,9 @@ int dyspec_tree_attention_paged(const dyspec_plan_t* plan, const void* q, const 
  * tree row tree_row_offset[r] + k_i, for K and V, and new_prefix_len[r] = L_r + their number.  The page table must
  * already hold a page for every new token; a token without one (entry < 0 or past pages_per_req) stops
  * that request's copy there, new_prefix_len[r] counts what was kept, and *status = DYSPEC_ERR_INVALID_ARG.
+ * tree_row_offset == NULL: the tree rows are tokens L_r .. of the paged sequence (node k = token L_r + k);
+ * the rows then move in place, inside the request's pages (a kept node whose token has no page stops the
+ * copy in the same way).
  * page_size: a power of two (any).  Other arguments as in dyspec_compact_kv; all arrays dev.
  */
 int dyspec_compact_kv_paged(void* k_cache, void* v_cache, const int64_t* tree_row_offset, const int32_t* page_table,

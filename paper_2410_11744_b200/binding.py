@@ -130,11 +130,13 @@ class Plan:
         n_req = len(prefix_len)
         pl = (_c.c_int32 * max(1, n_req))(*[int(x) for x in prefix_len])
         nn = (_c.c_int32 * max(1, n_req))(*[int(x) for x in n_nodes])
-        off = (_c.c_int64 * max(1, n_req))(*[int(x) for x in kv_row_offset])
+        off = None if kv_row_offset is None else (_c.c_int64 * max(1, n_req))(*[int(x) for x in kv_row_offset])
         handle = _vp()
         if page_size is not None:
+            # kv_row_offset None: the tree rows are tokens L .. L + n - 1 of the paged sequence (NULL in the C call)
             _check(lib.dyspec_plan_create_paged(_c.byref(handle), n_q_heads, n_kv_heads, head_dim, n_req,
-                                                _c.cast(pl, _vp), _c.cast(nn, _vp), _c.cast(off, _vp), int(kv_total_rows),
+                                                _c.cast(pl, _vp), _c.cast(nn, _vp),
+                                                _vp() if off is None else _c.cast(off, _vp), int(kv_total_rows),
                                                 int(page_size), words_per_row, float(scale)), "dyspec_plan_create_paged")
         else:
             _check(lib.dyspec_plan_create(_c.byref(handle), n_q_heads, n_kv_heads, head_dim, n_req,

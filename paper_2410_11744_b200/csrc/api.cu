@@ -161,6 +161,7 @@ struct dyspec_plan {
   int n_req = 0;
   int64_t kv_total_rows = 0;
   int page_size = 0;                    // > 0: paged cache (prefix through a page table, kv_row0 = first tree row)
+  bool tree_in_pages = false;           // paged cache whose tree rows are tokens L .. L + n - 1 of the paged sequence
   int64_t total_nodes = 0;
   int max_nodes = 0;
   int regime = 0, bm = 64, bn = 64;
@@ -206,14 +207,17 @@ void schedule(dyspec_plan& pl) {
   for (int r = 0; r < pl.n_req; ++r) {
     const ReqInfo& rq = pl.reqs[r];
     if (rq.n_nodes == 0) continue;
-    const int prefix_tiles = (rq.prefix_len + bn - 1) / bn;
+    // (tree rows inside the paged sequence: the tiles follow the sequence, and the tree's column 0 sits
+    //  L % bn keys inside the first tile that needs the mask)
+    const int prefix_tiles = prefix_tile_count(rq.prefix_len, bn, pl.tree_in_pages);
+    const int shift = tree_tile_shift(rq.prefix_len, bn, pl.tree_in_pages);
     const int q_tiles = (rq.n_nodes + nodes_per_tile - 1) / nodes_per_tile;
     for (int kvh = 0; kvh < pl.hkv; ++kvh)
       for (int qt = 0; qt < q_tiles; ++qt) {
         // parents[i] < i: a node only sees tree columns <= its own index, so tree tiles past the
         // tile's last node are never needed.
         const int last_node = std::min(rq.n_nodes, (qt + 1) * nodes_per_tile);
-        const int tiles = prefix_tiles + (last_node + bn - 1) / bn;
+        const int tiles = prefix_tiles + (shift + last_node + bn - 1) / bn;
         groups.push_back({r, kvh, qt * bm, tiles});
         total_tiles += tiles;
       }
@@ -526,7 +530,7 @@ void schedule(dyspec_plan& pl) {
   {
     const int bn = pl.bn;
     auto ungated_tiles = [&](const WorkItem& it) {
-      const int npt = (it.prefix_len + bn - 1) / bn;
+      const int npt = prefix_tile_count(it.prefix_len, bn, pl.tree_in_pages);
       const int prefix_part = std::max(0, std::min(int(it.tile_end), npt) - int(it.tile_begin));
       return it.tile_end > npt ? prefix_part : int(it.tile_end - it.tile_begin);
     };
@@ -778,7 +782,7 @@ int dyspec_compact_kv_paged(void* k_cache, void* v_cache, const int64_t* tree_ro
   const int64_t row_bytes = int64_t(n_kv_heads) * head_dim * 2;
   if (row_bytes % 16 != 0 || row_bytes > (1 << 24)) return DYSPEC_ERR_UNSUPPORTED;
   if (n_req == 0) return DYSPEC_OK;
-  if (!k_cache || !v_cache || !tree_row_offset || !page_table || !prefix_len || !accepted_nodes || !n_accepted)
+  if (!k_cache || !v_cache || !page_table || !prefix_len || !accepted_nodes || !n_accepted)   // (tree_row_offset may be NULL)
     return DYSPEC_ERR_INVALID_ARG;
   if (!aligned(k_cache, 16) || !aligned(v_cache, 16)) return DYSPEC_ERR_INVALID_ARG;
   int shift = 0;
@@ -793,7 +797,7 @@ int dyspec_compact_kv_paged(void* k_cache, void* v_cache, const int64_t* tree_ro
 static int make_host_plan(dyspec_plan** out, int n_q_heads, int n_kv_heads, int head_dim, int n_req,
                           const int32_t* prefix_len, const int32_t* n_nodes, const int64_t* kv_row_offset,
                           int64_t kv_total_rows, int words_per_row, float scale, int page_size = 0,
-                          bool allow_queue = true) {
+                          bool allow_queue = true, bool tree_in_pages = false) {
   *out = nullptr;
   if (n_q_heads <= 0 || n_kv_heads <= 0 || n_req < 0 || kv_total_rows < 0) return DYSPEC_ERR_INVALID_ARG;
   if (page_size < 0 || (page_size & (page_size - 1))) return DYSPEC_ERR_INVALID_ARG;
@@ -815,6 +819,7 @@ static int make_host_plan(dyspec_plan** out, int n_q_heads, int n_kv_heads, int 
   pl->n_req = n_req;
   pl->kv_total_rows = kv_total_rows;
   pl->page_size = page_size;
+  pl->tree_in_pages = tree_in_pages && page_size != 0;
   pl->allow_queue = allow_queue;
   int64_t node0 = 0;
   int max_rows = 0;
@@ -822,7 +827,7 @@ static int make_host_plan(dyspec_plan** out, int n_q_heads, int n_kv_heads, int 
     if (prefix_len[r] < 0 || n_nodes[r] < 0 || kv_row_offset[r] < 0) { delete pl; return DYSPEC_ERR_INVALID_ARG; }
     if (n_nodes[r] > DYSPEC_MAX_NODES) { delete pl; return DYSPEC_ERR_UNSUPPORTED; }
     if (32 * words_per_row < n_nodes[r]) { delete pl; return DYSPEC_ERR_INVALID_ARG; }
-    if (kv_row_offset[r] + (page_size ? 0 : prefix_len[r]) + n_nodes[r] > kv_total_rows) { delete pl; return DYSPEC_ERR_INVALID_ARG; }
+    if (!pl->tree_in_pages && kv_row_offset[r] + (page_size ? 0 : prefix_len[r]) + n_nodes[r] > kv_total_rows) { delete pl; return DYSPEC_ERR_INVALID_ARG; }
     ReqInfo rq{};
     rq.kv_row0 = kv_row_offset[r]; rq.prefix_len = prefix_len[r]; rq.n_nodes = n_nodes[r]; rq.node0 = int32_t(node0);
     pl->reqs.push_back(rq);
@@ -878,8 +883,11 @@ int dyspec_plan_create_paged(dyspec_plan_t** plan, int n_q_heads, int n_kv_heads
   *plan = nullptr;
   if (page_size <= 0) return DYSPEC_ERR_INVALID_ARG;
   dyspec_plan* pl = nullptr;
-  int rc = make_host_plan(&pl, n_q_heads, n_kv_heads, head_dim, n_req, prefix_len, n_nodes, tree_row_offset,
-                          kv_total_rows, words_per_row, scale, page_size);
+  // no tree rows of their own: node j of request r is token L_r + j of its paged sequence
+  const bool in_pages = tree_row_offset == nullptr;
+  const std::vector<int64_t> zeros(size_t(std::max(n_req, 1)), 0);
+  int rc = make_host_plan(&pl, n_q_heads, n_kv_heads, head_dim, n_req, prefix_len, n_nodes,
+                          in_pages ? zeros.data() : tree_row_offset, kv_total_rows, words_per_row, scale, page_size, true, in_pages);
   if (rc != DYSPEC_OK) return rc;
   rc = upload(*pl);
   if (rc != DYSPEC_OK) { dyspec_plan_destroy(pl); return rc; }
@@ -1008,7 +1016,8 @@ int dyspec_tree_attention_paged(const dyspec_plan_t* plan, const void* q, const 
   if (plan->n_ctas == 0) return DYSPEC_OK;
   if (!page_table || !aligned(page_table, 4) || pages_per_req <= 0) return DYSPEC_ERR_INVALID_ARG;
   for (const ReqInfo& rq : plan->reqs)                                   // every prefix token has a table entry
-    if ((int64_t(rq.prefix_len) + plan->page_size - 1) / plan->page_size > pages_per_req) return DYSPEC_ERR_INVALID_ARG;
+    if ((int64_t(rq.prefix_len) + (plan->tree_in_pages ? rq.n_nodes : 0) + plan->page_size - 1) / plan->page_size > pages_per_req)
+      return DYSPEC_ERR_INVALID_ARG;
   return run_attention(plan, q, k_cache, v_cache, page_table, pages_per_req, ancestor_bits, node_tiles, out, workspace,
                        workspace_bytes, status, stream);
 }
@@ -1040,7 +1049,8 @@ static int run_attention(const dyspec_plan_t* plan, const void* q, const void* k
 
   AttnParams p{};
   p.reqs = plan->d_reqs; p.items = plan->d_items; p.groups = plan->d_groups;
-  p.bits = ancestor_bits; p.node_tiles = node_tiles; p.out = static_cast<__nv_bfloat16*>(out);
+  p.bits = ancestor_bits; p.out = static_cast<__nv_bfloat16*>(out);
+  p.node_tiles = plan->tree_in_pages ? nullptr : node_tiles;   // the tile sets count unshifted tree tiles
   p.partial = static_cast<float*>(workspace);
   p.counters = plan->split_groups.empty() ? nullptr
                                           : reinterpret_cast<int32_t*>(static_cast<unsigned char*>(workspace) + plan->counters_offset);
@@ -1058,6 +1068,7 @@ static int run_attention(const dyspec_plan_t* plan, const void* q, const void* k
     p.trace = now.trace; p.trace_capacity = now.trace_capacity;
   }
   p.page_table = page_table; p.pages_per_req = pages_per_req;
+  p.tree_in_pages = plan->tree_in_pages ? 1 : 0;
   for (p.page_shift = 0; page_table && (1 << p.page_shift) < plan->page_size; ++p.page_shift) {}
 
   cudaError_t e;

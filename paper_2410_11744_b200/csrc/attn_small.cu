@@ -254,7 +254,7 @@ tree_attn_small_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
         for (int h = 0; h < L::kHalves; ++h)
           tma_load_3d(s_q + h * (BM * 128), &map_q, bar_qfull, h * 64, item.kv_head * g,
                       rq.node0 + (item.row0 >> p.log2_g));
-        const int n_prefix_tiles = (rq.prefix_len + BN - 1) / BN;
+        const int n_prefix_tiles = prefix_tile_count(rq.prefix_len, BN, p.tree_in_pages);
         for (int t = item.tile_begin; t < item.tile_end; ++t) {
           const int stage = ring_stage;
           const uint32_t ph = ring_phase;
@@ -383,7 +383,7 @@ tree_attn_small_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
   for (int w = item_begin; w < item_end; ++w, ++qit) {
     const WorkItem item = item_of(w);
     const WorkItem& rq = item;
-    const int n_prefix_tiles = (rq.prefix_len + BN - 1) / BN;
+    const int n_prefix_tiles = prefix_tile_count(rq.prefix_len, BN, p.tree_in_pages);
     const int n_rows = rq.n_nodes * g;                     // packed rows of this (request, kv head)
     const int row_lo = item.row0 + wrow + gid;             // the two packed rows this thread owns
     const int row_hi = row_lo + 8;
@@ -411,12 +411,23 @@ tree_attn_small_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
       //      tile visible to this thread.
       // A tree tile's mask words are fetched first (after the preceding kernels are known to be done:
       // the mask builder is one of them), so that the loads are in flight during the waits below.
+      // (Tree rows inside the paged sequence: the tile's 64 columns start shift = L % 64 bits before the
+      //  64-bit group u of the row, so the group in front of it is fetched as well.)
       uint2 w_lo = make_uint2(0u, 0u), w_hi = make_uint2(0u, 0u);
+      uint2 x_lo = make_uint2(0u, 0u), x_hi = make_uint2(0u, 0u);       // the group in front (shifted tiles only)
+      const int shift = tree_tile_shift(rq.prefix_len, BN, p.tree_in_pages);
       if (t >= n_prefix_tiles) {
         need_dep();
         const int u = t - n_prefix_tiles;
-        if (ok_lo) w_lo = ld_after_dependency_v2(reinterpret_cast<const uint2*>(p.bits + size_t(rq.node0 + node_lo) * p.words_per_row) + u);
-        if (ok_hi) w_hi = ld_after_dependency_v2(reinterpret_cast<const uint2*>(p.bits + size_t(rq.node0 + node_hi) * p.words_per_row) + u);
+        const uint2* bits_lo = reinterpret_cast<const uint2*>(p.bits + size_t(rq.node0 + node_lo) * p.words_per_row);
+        const uint2* bits_hi = reinterpret_cast<const uint2*>(p.bits + size_t(rq.node0 + node_hi) * p.words_per_row);
+        const bool cur = 2 * u < p.words_per_row;                        // a shifted tile may start in the row's last group
+        if (ok_lo && cur) w_lo = ld_after_dependency_v2(bits_lo + u);
+        if (ok_hi && cur) w_hi = ld_after_dependency_v2(bits_hi + u);
+        if (shift != 0 && u > 0) {
+          if (ok_lo) x_lo = ld_after_dependency_v2(bits_lo + u - 1);
+          if (ok_hi) x_hi = ld_after_dependency_v2(bits_hi + u - 1);
+        }
       }
       mbar_wait(bar_sfull + 8 * sb, uint32_t(pos / kSBufs) & 1u, abort_flag, p.status);
       mbar_wait(bar_full + 8 * stage, ph, abort_flag, p.status);
@@ -438,9 +449,16 @@ tree_attn_small_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
         vis_lo = vis_hi = m;
       } else {
         const int u = t - n_prefix_tiles;
-        own = min(BN, rq.n_nodes - u * BN);
+        own = min(BN, rq.n_nodes + shift - u * BN);
         vis_lo = (uint64_t(w_lo.y) << 32) | w_lo.x;
         vis_hi = (uint64_t(w_hi.y) << 32) | w_hi.x;
+        if (shift != 0) {
+          // tile column c is tree column u * 64 + c - shift: the row's bits from 64 u - shift onwards; in
+          // front of the tree's column 0 (u = 0) are the prefix's last `shift` keys, visible to every row
+          const uint64_t head = u > 0 ? 0ull : ((1ull << shift) - 1ull);
+          vis_lo = (vis_lo << shift) | (((uint64_t(x_lo.y) << 32) | x_lo.x) >> (64 - shift)) | head;
+          vis_hi = (vis_hi << shift) | (((uint64_t(x_hi.y) << 32) | x_hi.x) >> (64 - shift)) | head;
+        }
       }
 
       // ---- online softmax (exp2 domain) against a LAZY reference: the accumulator lives in tensor memory, so

@@ -222,7 +222,10 @@ __device__ __forceinline__ TileWalk walk_sparse(const AttnParams& p, const WorkI
 // kDyn: the CTAs take their items from the shared queue (AttnParams::queue) instead of fixed lists.  A
 // template parameter, not a run-time flag: the softmax threads sit right at the register limit and the
 // fixed-list kernel should compile exactly as it would without the queue.
-template <int D, bool kDyn>
+// kInPages: the tree rows are part of the paged sequence (AttnParams::tree_in_pages): key tiles follow the
+// sequence and a row's mask slice is shifted.  A template parameter for the same reason (the shift code as
+// a run-time branch cost the ordinary layouts 2 % on the ragged batch of 8).
+template <int D, bool kDyn, bool kInPages>
 __global__ void __launch_bounds__(kThreads, 1)
 tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                     const __grid_constant__ CUtensorMap map_v, const AttnParams p,
@@ -374,7 +377,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           }
         };
         load_q_half(0, B_QFULL);
-        const int n_prefix_tiles = (rq.prefix_len + BN - 1) / BN;
+        const int n_prefix_tiles = prefix_tile_count(rq.prefix_len, BN, kInPages ? 1 : 0);
         // Prefix tiles stream at once; the set of tree tiles may depend on the mask kernel's output,
         // so it is settled (after waiting for that kernel) only when the walk reaches the tree.
         TileWalk wk = walk_dense(item, n_prefix_tiles);
@@ -469,7 +472,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         const WorkItem item = item_of(w, item_at);
         const WorkItem& rq = item;
         const bool two = rq.n_nodes * g - item.row0 > BMH;        // both query halves live
-        const int n_prefix_tiles = (rq.prefix_len + BN - 1) / BN;
+        const int n_prefix_tiles = prefix_tile_count(rq.prefix_len, BN, kInPages ? 1 : 0);
         TileWalk wk = walk_dense(item, n_prefix_tiles);
         bool exact = !walk_may_skip(p, wk);
         int T = exact ? wk.T : 0x7fffffff;
@@ -600,7 +603,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       const WorkItem& rq = item;
       const int n_rows = rq.n_nodes * g;
       const int nh = (n_rows - item.row0 > BMH) ? 2 : 1;
-      const int n_prefix_tiles = (rq.prefix_len + BN - 1) / BN;
+      const int n_prefix_tiles = prefix_tile_count(rq.prefix_len, BN, kInPages ? 1 : 0);
       if (walk_may_skip(p, walk_dense(item, n_prefix_tiles))) need_dep();   // the tile walk reads the per-node tile sets
       const TileWalk wk = walk_sparse(p, item, n_prefix_tiles, lane);
       const int T = wk.T;
@@ -642,11 +645,29 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           }
         } else {
           const int u = t - n_prefix_tiles;
-          own = min(BN, rq.n_nodes - u * BN);
+          const int shift = tree_tile_shift(rq.prefix_len, BN, kInPages ? 1 : 0);
+          own = min(BN, rq.n_nodes + shift - u * BN);
           uint4 mv = make_uint4(0u, 0u, 0u, 0u);
           need_dep();
-          if (ok) mv = ld_after_dependency_v4(mask_row + u);
+          if (ok && (!kInPages || 4 * u < p.words_per_row)) mv = ld_after_dependency_v4(mask_row + u);   // (a shifted tile may start past the row's last group)
           vis[0] = mv.x; vis[1] = mv.y; vis[2] = mv.z; vis[3] = mv.w;
+          if (kInPages && shift != 0) {
+            // Tree rows inside the paged sequence: tile column c is tree column u * 128 + c - shift, i.e. the
+            // 128 bits that start `shift` bits before group u of the row; in front of the tree's column 0
+            // (u = 0) are the prefix's last `shift` keys, visible to every row.
+            uint4 pv = make_uint4(0u, 0u, 0u, 0u);
+            if (ok && u > 0) pv = ld_after_dependency_v4(mask_row + u - 1);
+            const int o = BN - shift, ws = o >> 5, bs = o & 31;          // window = bits o .. o + 127 of (pv, mv)
+            const uint32_t x[8] = {pv.x, pv.y, pv.z, pv.w, mv.x, mv.y, mv.z, mv.w};
+            uint32_t a[5];
+#pragma unroll
+            for (int q4 = 0; q4 < 5; ++q4) a[q4] = ws == 0 ? x[q4] : ws == 1 ? x[q4 + 1] : ws == 2 ? x[q4 + 2] : x[q4 + 3];
+#pragma unroll
+            for (int q4 = 0; q4 < 4; ++q4) {
+              const int head = u > 0 ? 0 : shift - 32 * q4;
+              vis[q4] = __funnelshift_r(a[q4], a[q4 + 1], bs) | (head >= 32 ? 0xffffffffu : (head <= 0 ? 0u : ((1u << head) - 1u)));
+            }
+          }
         }
 
         mbar_wait(bar(B_SREADY + h), n_s & 1, abort_flag, p.status);
@@ -1069,13 +1090,13 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
 }
 
 namespace {
-template <int D, bool kDyn>
+template <int D, bool kDyn, bool kInPages>
 cudaError_t launch_one(cudaLaunchConfig_t& cfg, size_t smem, const CUtensorMap& mq, const CUtensorMap& mk,
                        const CUtensorMap& mv, const AttnParams& p, const FirstItems& first) {
   static DynSmemGrant grant;           // one per instantiation
-  if (cudaError_t e = grant.ensure(tree_attn_tc_kernel<D, kDyn>, smem); e != cudaSuccess) return e;
+  if (cudaError_t e = grant.ensure(tree_attn_tc_kernel<D, kDyn, kInPages>, smem); e != cudaSuccess) return e;
   cfg.dynamicSmemBytes = smem;
-  return cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<D, kDyn>, mq, mk, mv, p, first);
+  return cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<D, kDyn, kInPages>, mq, mk, mv, p, first);
 }
 }  // namespace
 
@@ -1098,12 +1119,18 @@ cudaError_t launch_attn_tc(int head_dim, int n_ctas, const CUtensorMap& mq, cons
   cudaError_t le = cudaSuccess;
   if (head_dim == 128) {
     const size_t smem = TcLayout<128>::kTotal + 1024;
-    le = dyn ? launch_one<128, true>(cfg, smem, mq, mk, mv, p, first) : launch_one<128, false>(cfg, smem, mq, mk, mv, p, first);
+    if (p.tree_in_pages)
+      le = dyn ? launch_one<128, true, true>(cfg, smem, mq, mk, mv, p, first) : launch_one<128, false, true>(cfg, smem, mq, mk, mv, p, first);
+    else
+      le = dyn ? launch_one<128, true, false>(cfg, smem, mq, mk, mv, p, first) : launch_one<128, false, false>(cfg, smem, mq, mk, mv, p, first);
   } else {
     // padded past half of an SM's shared memory: one CTA per SM, since each CTA takes all 512 TMEM columns
     const size_t smem = 120 * 1024;
     static_assert(TcLayout<64>::kTotal + 1024 <= 120 * 1024, "smem layout");
-    le = dyn ? launch_one<64, true>(cfg, smem, mq, mk, mv, p, first) : launch_one<64, false>(cfg, smem, mq, mk, mv, p, first);
+    if (p.tree_in_pages)
+      le = dyn ? launch_one<64, true, true>(cfg, smem, mq, mk, mv, p, first) : launch_one<64, false, true>(cfg, smem, mq, mk, mv, p, first);
+    else
+      le = dyn ? launch_one<64, true, false>(cfg, smem, mq, mk, mv, p, first) : launch_one<64, false, false>(cfg, smem, mq, mk, mv, p, first);
   }
   return le != cudaSuccess ? le : cudaGetLastError();
 }

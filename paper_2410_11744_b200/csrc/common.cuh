@@ -104,6 +104,11 @@ struct AttnParams {
   const int32_t* page_table;
   int32_t pages_per_req;
   int32_t page_shift;
+  // Paged cache with the tree rows INSIDE the paged sequence (node j = token L + j): key tiles then follow
+  // the sequence, not the tree: the first L / BN tiles are full prefix tiles, tile L / BN + u covers tokens
+  // [(L / BN + u) BN, ...), i.e. tree columns u BN - L % BN onwards (its leading L % BN keys, for u = 0, are
+  // the prefix's last ones), and a row's mask slice for the tile is its bit row shifted by L % BN.
+  int32_t tree_in_pages;
   // Shared work queue (null = every CTA has a fixed list): `items` then holds all n_items_total items in
   // queue order, CTA c starts with item c and takes further ones with an atomic add on queue[0];
   // queue[1] counts the CTAs that found the queue empty, and the last of them clears both words.
@@ -132,10 +137,20 @@ struct DynSmemGrant {
   }
 };
 
+// Key tiles of a (request, query tile) group, host and device: the tiles in front of the first one that
+// needs the mask, and how far the tree's column 0 sits inside that one (0 unless the tree rows are
+// part of the paged sequence).
+__host__ __device__ inline int prefix_tile_count(int prefix_len, int bn, int tree_in_pages) {
+  return tree_in_pages ? prefix_len / bn : (prefix_len + bn - 1) / bn;
+}
+__host__ __device__ inline int tree_tile_shift(int prefix_len, int bn, int tree_in_pages) {
+  return tree_in_pages ? prefix_len % bn : 0;
+}
+
 #ifdef __CUDACC__
 // First cache row of key tile t of a work item's group (tiles of BN keys: prefix tiles, then tree tiles).
 __device__ __forceinline__ int64_t kv_tile_row(const AttnParams& p, const WorkItem& it, int t, int n_prefix_tiles, int BN) {
-  if (t >= n_prefix_tiles)
+  if (t >= n_prefix_tiles && !p.tree_in_pages)
     return it.kv_row0 + (p.page_table ? 0 : int64_t(it.prefix_len)) + int64_t(t - n_prefix_tiles) * BN;
   const int64_t s = int64_t(t) * BN;
   if (!p.page_table) return it.kv_row0 + s;

@@ -39,8 +39,10 @@ compact_kv_kernel(uint4* __restrict__ k_cache, uint4* __restrict__ v_cache, cons
 
 // Paged cache: the accepted nodes' rows leave the request's tree rows (tree_row_offset[r] + a_i) for the
 // pages of the prefix: token L + i lies in page (L + i) / page_size of the request, at row (L + i) %
-// page_size of it.  Source and destination never overlap (the tree rows are outside the prefix pages),
-// so the steps are independent.
+// page_size of it.  With the tree rows outside the prefix pages source and destination never overlap.
+// With tree_row_offset == nullptr the tree rows are tokens L .. of the paged sequence themselves (node a
+// = token L + a): an in-place move again, safe for the reason given above (a thread walks the steps in
+// order over its own columns; the accepted nodes increase along their path).
 __global__ void __launch_bounds__(256)
 compact_kv_paged_kernel(uint4* __restrict__ k_cache, uint4* __restrict__ v_cache, const int64_t* __restrict__ tree_row_offset,
                         const int32_t* __restrict__ page_table, int pages_per_req, int page_shift,
@@ -50,7 +52,8 @@ compact_kv_paged_kernel(uint4* __restrict__ k_cache, uint4* __restrict__ v_cache
   const int r = blockIdx.x;
   uint4* cache = blockIdx.z == 0 ? k_cache : v_cache;
   const int L = prefix_len[r];
-  const int64_t src0 = tree_row_offset[r];
+  const bool in_pages = tree_row_offset == nullptr;
+  const int64_t src0 = in_pages ? 0 : tree_row_offset[r];
   const int n = min(n_accepted[r], max_out);
   const int32_t* acc = accepted_nodes + size_t(r) * max_out;
   const int32_t* pages = page_table + size_t(r) * pages_per_req;
@@ -67,9 +70,19 @@ compact_kv_paged_kernel(uint4* __restrict__ k_cache, uint4* __restrict__ v_cache
       if (status && col == 0 && blockIdx.z == 0) atomicCAS(status, 0, DYSPEC_ERR_INVALID_ARG);
       break;
     }
+    int64_t src = src0 + a;
+    if (in_pages) {
+      const int ts = L + a, ps = ts >> page_shift;
+      const int spage = ps < pages_per_req ? pages[ps] : -1;
+      if (spage < 0) {                         // the node's row has no page: nothing to move from
+        if (status && col == 0 && blockIdx.z == 0) atomicCAS(status, 0, DYSPEC_ERR_INVALID_ARG);
+        break;
+      }
+      src = (int64_t(spage) << page_shift) + (ts & ((1 << page_shift) - 1));
+    }
     if (col < row_vecs) {
       const int64_t dst = (int64_t(page) << page_shift) + (t & ((1 << page_shift) - 1));
-      cache[dst * row_vecs + col] = cache[(src0 + a) * int64_t(row_vecs) + col];
+      if (dst != src) cache[dst * row_vecs + col] = cache[src * int64_t(row_vecs) + col];
     }
     ++kept;
   }
