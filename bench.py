@@ -501,9 +501,11 @@ def compaction_experiment(torch, B, peaks, device):
     return out
 
 
-def paged_experiment(torch, runner, workloads, B, peaks, device, configs=(2, 3, 4), page_size=256, steps=400):
-    """The same step with the cache in shuffled pages of page_size rows (prefix through a page table,
-    tree rows in a run of their own) beside the contiguous layout: same algorithmic bytes, so the two
+def paged_experiment(torch, runner, workloads, B, peaks, device, configs=(2, 3, 4, 5), page_size=256, steps=400):
+    """The same step with the cache in shuffled pages of page_size rows beside the contiguous layout: prefix
+    through a page table and tree rows in a run of their own ("paged"), and prefix and tree rows both in the
+    pages ("in_sequence": key tiles follow the sequence, mask slices are shifted by L modulo the tile size;
+    configs 2 - 4 have L on a tile boundary, the ragged batch does not).  Same algorithmic bytes, so the
     times should agree.  After it, the paged accepted-path compaction (8 accepted nodes, 64 requests)."""
     out = {"page_size": page_size, "configs": []}
     for idx in configs:
@@ -513,10 +515,17 @@ def paged_experiment(torch, runner, workloads, B, peaks, device, configs=(2, 3, 
         del mc
         torch.cuda.empty_cache()
         mp = measure_config(torch, runner, w, steps, 3, device, paged=workloads.to_paged(w, page_size, idx), isolated=False)
-        out["configs"].append({"config": idx, "workload": w.name, "contiguous_step_us": t_c[0] * 1e3,
-                               "contiguous_attention_us": t_c[1] * 1e3, "paged_step_us": mp["step_chain_ms"] * 1e3,
-                               "paged_attention_us": mp["attn_ms"] * 1e3, "bytes": mp["bytes"], "status": mp["status"]})
+        entry = {"config": idx, "workload": w.name, "contiguous_step_us": t_c[0] * 1e3,
+                 "contiguous_attention_us": t_c[1] * 1e3, "paged_step_us": mp["step_chain_ms"] * 1e3,
+                 "paged_attention_us": mp["attn_ms"] * 1e3, "bytes": mp["bytes"], "status": mp["status"]}
         del mp
+        torch.cuda.empty_cache()
+        ms = measure_config(torch, runner, w, steps, 3, device,
+                            paged=workloads.to_paged(w, page_size, idx, tree_in_pages=True), isolated=False)
+        entry.update({"in_sequence_step_us": ms["step_chain_ms"] * 1e3, "in_sequence_attention_us": ms["attn_ms"] * 1e3,
+                      "in_sequence_status": ms["status"]})
+        out["configs"].append(entry)
+        del ms
         torch.cuda.empty_cache()
     n_req, hkv, d, L, n, max_out = 64, 8, 128, 1024, 64, 16
     pages_per_req = (L + n + page_size - 1) // page_size
@@ -541,6 +550,15 @@ def paged_experiment(torch, runner, workloads, B, peaks, device, configs=(2, 3, 
     nbytes = n_req * 8 * hkv * d * 2 * 2 * 2
     out["compaction"] = {"case": "64 requests, 8 kv heads, 8 accepted nodes", "call_us": us, "bytes": nbytes,
                          "achieved_gbs": nbytes / (us * 1e-6) / 1e9}
+    # the same move with the tree rows inside the pages (node a = token L + a): in place
+    call = lambda: B.dyspec_compact_kv_paged(k, v, None, table, pages_per_req, page_size, Ls, acc, cnt, n_req, max_out,
+                                             hkv, d, newL)
+    call()
+    torch.cuda.synchronize()
+    g = _graph_of(torch, lambda: [call() for _ in range(20)])
+    g.replay()
+    torch.cuda.synchronize()
+    out["compaction"]["in_place_call_us"] = _time_replays(torch, g, 20) / 400 * 1e3
     return out
 
 
