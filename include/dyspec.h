@@ -279,8 +279,10 @@ int dyspec_tree_attention_static(const void* q, const void* k_cache, const void*
  * dyspec_tree_attention_ragged_sparse: dyspec_tree_attention_ragged that skips the tree key tiles no
  * row of a query tile touches (node_tiles must come from the same parents as ancestor_bits; NULL
  * gives dyspec_tree_attention_ragged).  Results are those of the dense call up to the order of the
- * fp32 additions.  Only the tcgen05 regime skips tiles; the small-tree regime, whose tree part is one
- * or two key tiles, ignores node_tiles.
+ * fp32 additions.  Only the tcgen05 regime skips tiles, and only for a query tile with at least three
+ * tree key tiles besides the ones that hold its own nodes (those, which every row sees, run first, before
+ * the tile sets are read); the small-tree regime, whose tree part is one or two key tiles, ignores
+ * node_tiles.
  */
 int dyspec_dfs_reorder(const int32_t* parents, int n_nodes, int32_t* order, int32_t* new_of_old, int32_t* new_parents,
                        int32_t* status, dyspec_stream_t stream);

@@ -180,6 +180,7 @@ struct TileWalk {
   int P;            // prefix tiles in the range: tiles tile_begin .. tile_begin + P - 1
   int T;            // tiles processed in all
   uint32_t need;    // tree tiles processed: bit u = tree columns [u * BN, (u + 1) * BN)
+  uint32_t first;   // those of them that are processed first (see walk_first); 0 = plain ascending order
 };
 __device__ __forceinline__ TileWalk walk_dense(const WorkItem& item, int n_prefix_tiles) {
   TileWalk wk;
@@ -187,18 +188,36 @@ __device__ __forceinline__ TileWalk walk_dense(const WorkItem& item, int n_prefi
   const int u0 = max(item.tile_begin, n_prefix_tiles) - n_prefix_tiles, u1 = item.tile_end - n_prefix_tiles;
   wk.need = u1 > u0 ? (((1u << u1) - 1u) & ~((1u << u0) - 1u)) : 0u;
   wk.T = wk.P + __popc(wk.need);
+  wk.first = 0u;
   return wk;
 }
-// Can the tile sets shorten this walk at all?  With one or two tree tiles they cannot pay: the query tile's
-// own columns are always visible, and reading the tile sets means waiting for the mask kernel before the
-// first tree tile is even requested.
-__device__ __forceinline__ bool walk_may_skip(const AttnParams& p, const TileWalk& dense) {
-  return p.node_tiles != nullptr && __popc(dense.need) > 2;
+// Next tree tile of a walk: the `first` ones in ascending order, then the others in ascending order.
+__device__ __forceinline__ int pop_tree_tile(uint32_t& rem, uint32_t first) {
+  const uint32_t a = rem & first;
+  const int u = __ffs(a ? a : rem) - 1;
+  rem &= ~(1u << u);
+  return u;
+}
+// The tree tiles that hold the query tile's own columns: every row sees its own key, so these are needed
+// whatever the tile sets say, and a walk that may skip tiles runs them before it has to read the sets
+// (i.e. before it has to wait for the mask kernel, or for whatever precedes the call in the stream).
+__device__ __forceinline__ uint32_t walk_first(const AttnParams& p, const WorkItem& item, const TileWalk& dense) {
+  const int node_lo = item.row0 >> p.log2_g;
+  const int node_hi = min(item.n_nodes, ((item.row0 + 2 * BMH - 1) >> p.log2_g) + 1);   // one past the tile's last node
+  const int u_lo = node_lo / BN, u_hi = (node_hi - 1) / BN;
+  return dense.need & ((2u << u_hi) - 1u) & ~((1u << u_lo) - 1u);
+}
+// Can the tile sets shorten this walk at all?  Only tiles other than the query tile's own can be skipped, and
+// the tile with the root never is; reading the sets costs a round trip to global memory in every role, after
+// waiting for the mask kernel.  With fewer than three candidates that has not paid (512-token random trees:
+// 16.0 us with the sets read against 14.6 without).
+__device__ __forceinline__ bool walk_may_skip(const AttnParams& p, const WorkItem& item, const TileWalk& dense) {
+  return p.node_tiles != nullptr && __popc(dense.need & ~walk_first(p, item, dense)) > 2;
 }
 // Whole warp.  The mask kernel must have completed (grid_dependency_wait) before this reads node_tiles.
 __device__ __forceinline__ TileWalk walk_sparse(const AttnParams& p, const WorkItem& item, int n_prefix_tiles, int lane) {
   TileWalk wk = walk_dense(item, n_prefix_tiles);
-  if (!walk_may_skip(p, wk)) return wk;
+  if (!walk_may_skip(p, item, wk)) return wk;
   const int node_lo = item.row0 >> p.log2_g;
   const int node_hi = min(item.n_nodes, ((item.row0 + 2 * BMH - 1) >> p.log2_g) + 1);
   uint32_t occ = 0u;
@@ -210,9 +229,10 @@ __device__ __forceinline__ TileWalk walk_sparse(const AttnParams& p, const WorkI
   x = (x | (x >> 2)) & 0x0f0f0f0fu;
   x = (x | (x >> 4)) & 0x00ff00ffu;
   x = (x | (x >> 8)) & 0x0000ffffu;
-  const uint32_t first = wk.need & (0u - wk.need);
-  wk.need &= x;
-  if (wk.P == 0 && wk.need == 0u) wk.need = first;     // an item always runs at least one (fully masked) tile
+  const uint32_t lowest = wk.need & (0u - wk.need);
+  wk.first = walk_first(p, item, wk);
+  wk.need = (wk.need & x) | wk.first;
+  if (wk.P == 0 && wk.need == 0u) wk.need = lowest;    // an item always runs at least one (fully masked) tile
   wk.T = wk.P + __popc(wk.need);
   return wk;
 }
@@ -381,21 +401,19 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         // Prefix tiles stream at once; the set of tree tiles may depend on the mask kernel's output,
         // so it is settled (after waiting for that kernel) only when the walk reaches the tree.
         TileWalk wk = walk_dense(item, n_prefix_tiles);
-        bool exact = !walk_may_skip(p, wk);
+        bool exact = !walk_may_skip(p, item, wk);
+        if (!exact) wk.first = walk_first(p, item, wk);
         uint32_t rem = wk.need;
         for (int j = 0;; ++j) {
-          if (!exact && j >= wk.P) {
+          if (!exact && j >= wk.P + __popc(wk.first)) {
             grid_dependency_wait();
             wk = walk_sparse(p, item, n_prefix_tiles, lane);
-            rem = wk.need;
+            rem = wk.need & ~wk.first;                   // (the first ones are behind us)
             exact = true;
           }
           if (j >= wk.T) break;
           int t = item.tile_begin + j;
-          if (j >= wk.P) {
-            t = n_prefix_tiles + __ffs(rem) - 1;
-            rem &= rem - 1u;
-          }
+          if (j >= wk.P) t = n_prefix_tiles + pop_tree_tile(rem, wk.first);
           const int64_t row = kv_tile_row(p, item, t, n_prefix_tiles, BN);
           for (int kv = 0; kv < 2; ++kv, ++sc) {
             const int slot = sc % kSlots;
@@ -474,10 +492,11 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         const bool two = rq.n_nodes * g - item.row0 > BMH;        // both query halves live
         const int n_prefix_tiles = prefix_tile_count(rq.prefix_len, BN, kInPages ? 1 : 0);
         TileWalk wk = walk_dense(item, n_prefix_tiles);
-        bool exact = !walk_may_skip(p, wk);
+        bool exact = !walk_may_skip(p, item, wk);
         int T = exact ? wk.T : 0x7fffffff;
+        const int n_sure = exact ? 0 : wk.P + __popc(walk_first(p, item, wk));   // tiles that run whatever the tile sets say
         auto settle = [&](int j) {
-          if (!exact && j + 2 >= wk.P) {
+          if (!exact && j + 2 >= n_sure) {
             grid_dependency_wait();
             wk = walk_sparse(p, item, n_prefix_tiles, lane);
             T = wk.T;
@@ -604,7 +623,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       const int n_rows = rq.n_nodes * g;
       const int nh = (n_rows - item.row0 > BMH) ? 2 : 1;
       const int n_prefix_tiles = prefix_tile_count(rq.prefix_len, BN, kInPages ? 1 : 0);
-      if (walk_may_skip(p, walk_dense(item, n_prefix_tiles))) need_dep();   // the tile walk reads the per-node tile sets
+      if (walk_may_skip(p, item, walk_dense(item, n_prefix_tiles))) need_dep();   // the tile walk reads the per-node tile sets
       const TileWalk wk = walk_sparse(p, item, n_prefix_tiles, lane);
       const int T = wk.T;
       if (h >= nh) {
@@ -624,10 +643,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       float m_used = -INFINITY, l = 0.f;
       for (int j = 0; j < T; ++j) {
         int t = item.tile_begin + j;
-        if (j >= wk.P) {
-          t = n_prefix_tiles + __ffs(rem) - 1;
-          rem &= rem - 1u;
-        }
+        if (j >= wk.P) t = n_prefix_tiles + pop_tree_tile(rem, wk.first);
         const uint32_t vslot = sc + 1u;
         sc += 2u;
         // visibility of the 128 key columns of this tile for this row
