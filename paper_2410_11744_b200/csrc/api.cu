@@ -64,7 +64,8 @@ struct Tuning {
   int force_regime = -1;
   int force_ctas = 0;
   int item_cost = 0;       // scheduler experiment knob (0 = default)
-  int combine_mode = 2;    // 0 separate combine kernel, 2 merge on chip / in the attention kernel when the plan allows
+  int combine_mode = 2;    // 0 separate combine kernel; 2 merge on chip (clusters) / in the attention kernel when the plan
+                           // allows; 1 as 2 but the tensor-core regime never uses clusters (merge through the workspace)
   int whole_groups = 0;    // 0: the scheduler's cost model chooses; 1: never deal whole groups; 2: always
   unsigned long long* trace = nullptr;   // device buffer for the optional kernel event trace
   int trace_capacity = 0;
@@ -377,7 +378,7 @@ void schedule(dyspec_plan& pl) {
   if (tn.whole_groups != 1 && (tn.force_ctas <= 0 || tn.whole_groups == 2)) {
     // (tensor-core regime with the merge inside the kernel: no combine launch; writing the fp32 partial,
     //  publishing it and merging a share of the rows cost a split item about four tiles: 7 us measured)
-    const bool in_kernel = pl.regime == 1 && tn.combine_mode == 2;
+    const bool in_kernel = pl.regime == 1 && tn.combine_mode != 0;
     const int partial_cost = in_kernel ? 4 : 1, combine_cost = in_kernel ? 0 : (pl.regime == 0 ? 4 : 3);
     int64_t cost_split = 0;
     for (int c = 0; c < pl.n_ctas; ++c) {
@@ -450,7 +451,7 @@ void schedule(dyspec_plan& pl) {
   // length, ONE piece per CTA, as many pieces as there are SMs to take them.  Against the budgeted plan
   // this avoids CTAs with two split items (each pays the start-up and the partial epilogue again: on the
   // Llama2-7B shape with a 4096-key prefix those CTAs finished 8 us after the others).
-  if (pl.regime == 1 && tn.combine_mode == 2 && tn.force_ctas <= 0 && tn.whole_groups != 2 && !pl.dynamic &&
+  if (pl.regime == 1 && tn.combine_mode != 0 && tn.force_ctas <= 0 && tn.whole_groups != 2 && !pl.dynamic &&
       int64_t(groups.size()) * 2 <= max_ctas) {
     const int item_cost_ = item_cost, partial_cost = 4;
     int64_t cost_now = 0;
@@ -515,6 +516,55 @@ void schedule(dyspec_plan& pl) {
         }
       }
       pl.n_ctas = int(pl.items.size());
+    }
+    // The same idea with one thread-block cluster per group (C pieces each, C the same for all groups): the
+    // pieces' partials then stay in shared memory (each CTA fetches its share of the rows from its peers),
+    // which costs a piece about one tile instead of four (the fp32 partials of all CTAs at once go through
+    // L2 at its bandwidth, twice).  Needs groups of similar length and at least two tiles per piece.
+    if (tn.combine_mode == 2) {
+      int max_tiles = 0, min_tiles_g = INT32_MAX;
+      for (const Group& gr : groups) { max_tiles = std::max(max_tiles, gr.tiles); min_tiles_g = std::min(min_tiles_g, gr.tiles); }
+      int64_t cost_plan = 0;                             // of the plan chosen so far
+      for (int c = 0; c < pl.n_ctas; ++c) {
+        int64_t load = 0;
+        for (int k = pl.cta_begin[size_t(c)]; k < pl.cta_begin[size_t(c) + 1]; ++k) {
+          const WorkItem& it = pl.items[size_t(k)];
+          load += (it.tile_end - it.tile_begin) + item_cost_ + (it.slot >= 0 ? partial_cost : 0);
+        }
+        cost_plan = std::max(cost_plan, load);
+      }
+      int best_c = 0;
+      int64_t best_cost = cost_plan;
+      for (int C : {8, 4, 2}) {
+        if (int64_t(groups.size()) * C > max_ctas || min_tiles_g < 2 * C) continue;
+        const int64_t cost = (max_tiles + C - 1) / C + item_cost_ + 1;
+        if (cost < best_cost) { best_cost = cost; best_c = C; }
+      }
+      if (best_c > 0) {
+        const int C = best_c;
+        pl.cluster = C;
+        pl.items.clear();
+        pl.cta_begin.clear();
+        pl.split_groups.clear();
+        pl.n_slots = 0;
+        pl.cta_begin.push_back(0);
+        for (size_t gi = 0; gi < groups.size(); ++gi) {
+          const Group& gr = groups[gi];
+          const ReqInfo& rq = pl.reqs[size_t(gr.req)];
+          for (int c = 0; c < C; ++c) {
+            WorkItem it{};
+            it.kv_row0 = rq.kv_row0; it.prefix_len = rq.prefix_len; it.n_nodes = rq.n_nodes; it.node0 = rq.node0;
+            it.req = gr.req; it.kv_head = gr.kvh; it.row0 = gr.row0;
+            it.tile_begin = int(int64_t(gr.tiles) * c / C);
+            it.tile_end = int(int64_t(gr.tiles) * (c + 1) / C);
+            it.slot = -1; it.slot0 = -1; it.group = int(gi); it.n_splits = C; it.n_in_cta = 1;
+            pl.items.push_back(it);
+            pl.cta_begin.push_back(int32_t(pl.items.size()));
+          }
+        }
+        pl.max_splits = C;
+        pl.n_ctas = int(pl.items.size());
+      }
     }
   }
 
@@ -605,7 +655,7 @@ int dyspec_set_tuning(int force_regime, int force_ctas, int combine_mode) {
   if (combine_mode < 0) return DYSPEC_ERR_INVALID_ARG;
   const int whole = combine_mode >> 4;
   combine_mode &= 15;
-  if (force_regime < -1 || force_regime > 1 || (combine_mode != 0 && combine_mode != 2) || whole > 2) return DYSPEC_ERR_INVALID_ARG;
+  if (force_regime < -1 || force_regime > 1 || combine_mode > 2 || whole > 2) return DYSPEC_ERR_INVALID_ARG;
   std::lock_guard<std::mutex> lock(g_tuning_mutex);
   g_tuning.whole_groups = whole;
   g_tuning.force_regime = force_regime;
@@ -851,7 +901,7 @@ static int make_host_plan(dyspec_plan** out, int n_q_heads, int n_kv_heads, int 
     pl->workspace_bytes = pl->counters_offset + ((pl->split_groups.size() * 2 * sizeof(int32_t) + 255) & ~size_t(255));
     // (the items of a group wait for each other inside the kernel: only when every CTA of the launch is
     //  resident at once, i.e. one CTA per SM and no more CTAs than SMs; a forced larger grid keeps the combine launch)
-    pl->merge_in_kernel = pl->regime == 1 && pl->tune.combine_mode == 2 && pl->n_ctas <= pl->n_sms;
+    pl->merge_in_kernel = pl->regime == 1 && pl->tune.combine_mode != 0 && pl->n_ctas <= pl->n_sms;
   }
   if (pl->dynamic) {                    // the queue words follow the partials (there are none in such a plan today)
     pl->queue_offset = (pl->workspace_bytes + 255) & ~size_t(255);

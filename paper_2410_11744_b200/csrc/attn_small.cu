@@ -79,7 +79,7 @@ __device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint32_t a_lo, uint32_t
 // (8-row groups 1024 bytes apart): low word = address >> 4 | (16 >> 4) << 16; high word = 1024 >> 4 |
 // version 1 | swizzle mode 2.
 constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
-__device__ __forceinline__ uint32_t desc_lo(uint32_t saddr) { return (saddr >> 4) | (1u << 16); }
+__device__ __forceinline__ uint32_t desc_lo(uint32_t saddr) { return ((saddr & 0x3ffffu) >> 4) | (1u << 16); }   // 14-bit address field (a CTA in a cluster has address bits above it)
 // Instruction descriptor, kind::f16: bf16 x bf16 -> fp32, both operands K-major, M = 64, N = 64.
 constexpr uint32_t kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(BN >> 3) << 17) | (uint32_t(BM >> 4) << 24);
 // With M = 64 the accumulator row r lives in TMEM lane 32 (r / 16) + r % 16, so warp w reads rows

@@ -23,8 +23,14 @@
 // An item whose group was cut along the keys writes an fp32 partial (O, m, l); after all of its items a CTA
 // merges, for each of its split items, a share of the group's rows (no combine launch; see the end of the
 // softmax branch).
-// Every wait is bounded (see mbar_wait); every TMA load goes to this CTA alone, and the kernel is never launched in clusters.
+// Plans with few long groups of equal length run one thread-block cluster per group instead: every CTA parks
+// its partial in its own shared memory and fetches its share of the rows from its peers' (distributed shared
+// memory; nothing goes through global memory).
+// Every wait on a flag or an mbarrier is bounded (see mbar_wait); every TMA load goes to this CTA alone, also
+// when the kernel is launched in clusters (the cluster is used for plain loads of peers' shared memory and
+// for its hardware barrier only).
 #include "common.cuh"
+#include <type_traits>
 
 namespace dyspec {
 
@@ -47,6 +53,12 @@ struct TcLayout {
   static constexpr int kBarOffset = kRingOffset + kSlots * kTileBytes;
   static constexpr int kItemRingOffset = kBarOffset + 512;   // queue plans: the CTA's next work items, 8 entries of 64 bytes
   static constexpr int kTotal = kItemRingOffset + 512;
+  // Cluster plans: when its products are done a CTA parks its partial over the (idle) Q tile and ring:
+  // 256 rows of D + 4 floats (the padding keeps 16-byte row accesses of a warp off each other's banks),
+  // then the rows' maxima and sums.
+  static constexpr int kParkRow = D + 4;
+  static constexpr int kParkScalars = 2 * BMH * kParkRow * 4;
+  static_assert(kParkScalars + 2 * 2 * BMH * 4 <= kBarOffset, "the parked partial fits in front of the barriers");
 };
 
 // Trace tags (see dyspec_set_trace): tag = role << 14 | event << 10 | key-tile index j.
@@ -102,7 +114,9 @@ __device__ __forceinline__ void umma_ts_lohi(uint32_t d_tmem, uint32_t a_tmem, u
 // Descriptor words: low = address >> 4 | (leading byte offset >> 4) << 16; high = stride byte offset >> 4 |
 // version 1 (bit 46) | 128-byte swizzle (bits 61-63).
 __host__ __device__ constexpr uint32_t desc_hi(uint32_t sbo_bytes) { return (sbo_bytes >> 4) | (1u << 14) | (2u << 29); }
-__device__ __forceinline__ uint32_t desc_lo(uint32_t saddr, uint32_t lbo_bytes) { return (saddr >> 4) | ((lbo_bytes >> 4) << 16); }
+// (The address field is 14 bits: an address in the shared window of a CTA that runs in a cluster has bits
+//  above them, which must not leak into the leading-offset field.)
+__device__ __forceinline__ uint32_t desc_lo(uint32_t saddr, uint32_t lbo_bytes) { return ((saddr & 0x3ffffu) >> 4) | ((lbo_bytes >> 4) << 16); }
 
 // Instruction descriptor, kind::f16: bf16 x bf16 -> fp32, A K-major, M = 128.
 __host__ __device__ constexpr uint32_t make_idesc(int n, int b_mn_major) {
@@ -575,6 +589,12 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       }
     }
   }
+  // cluster plans: "every CTA has parked its partial" (the softmax threads arrive once theirs is written)
+  if (p.cluster_size > 1) {
+    __syncwarp();
+    cluster_arrive();
+    cluster_wait();
+  }
   } else {
     asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");
     // ------------------------------------------------------------------ softmax + epilogue warps
@@ -631,6 +651,16 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         if (item.slot >= 0 && p.merge_in_kernel) {         // this half has no rows: nothing to write, but the group counts halves
           need_dep();
           if (r == 0) red_release_gpu_add(p.counters + 2 * item.group, 1);
+        }
+        if (p.cluster_size > 1) {                          // cluster plan: the peers read this half's rows all the same
+          named_sync(kBarMerge, 2 * BMH);                  // (the other half's products no longer read the Q tile and the ring)
+          float* park = reinterpret_cast<float*>(smem);
+          const int pr = h * BMH + r;
+#pragma unroll
+          for (int i = 0; i < D / 4; ++i) *reinterpret_cast<float4*>(park + pr * L::kParkRow + 4 * i) = make_float4(0.f, 0.f, 0.f, 0.f);
+          float* park_m = reinterpret_cast<float*>(smem + L::kParkScalars);
+          park_m[pr] = -INFINITY;
+          park_m[2 * BMH + pr] = 0.f;
         }
         continue;
       }
@@ -805,7 +835,26 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       auto stage_at = [&](int srow, int ch) -> uint4* {
         return reinterpret_cast<uint4*>(stage + (ch >> 3) * L::kPanelBytes + srow * 128 + (((ch & 7) ^ (srow & 7)) << 4));
       };
-      if (item.slot < 0 && staged) {
+      if (p.cluster_size > 1) {
+        // Cluster plan: the item is one piece of its group's keys, the other pieces are with the other CTAs
+        // of the cluster.  The row's unnormalised output, maximum and sum are parked in this CTA's shared
+        // memory, where the peers fetch them (see the merge behind the item loop).
+        uint32_t ov[D];
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) tmem_ld32(t_o + uint32_t(c) * 32u, ov + 32 * c);
+        tmem_wait_ld();
+        tc_fence_before();
+        mbar_arrive(bar(B_OFREE + h));
+        named_sync(kBarMerge, 2 * BMH);                    // both halves' products are done: Q tile and ring are idle
+        float* park = reinterpret_cast<float*>(smem);
+        const int pr = h * BMH + r;
+#pragma unroll
+        for (int i = 0; i < D / 4; ++i)
+          *reinterpret_cast<uint4*>(park + pr * L::kParkRow + 4 * i) = make_uint4(ov[4 * i], ov[4 * i + 1], ov[4 * i + 2], ov[4 * i + 3]);
+        float* park_m = reinterpret_cast<float*>(smem + L::kParkScalars);
+        park_m[pr] = m_used;
+        park_m[2 * BMH + pr] = l;
+      } else if (item.slot < 0 && staged) {
         const float inv = l > 0.f ? 1.f / l : 0.f;
         uint32_t ov[D];
 #pragma unroll
@@ -1094,9 +1143,108 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         }
       }
     }
+    // ---- split-KV merge of a cluster plan: the CTAs of a cluster hold the pieces of one (request, kv head,
+    // query tile) group, one item each.  Once every CTA has parked its partial (cluster barrier), CTA k
+    // fetches rows [k * 256 / C, (k + 1) * 256 / C) of all C partials from the peers' shared memory (its own
+    // included), merges and stores them: nothing goes through global memory, and there is no counter to wait
+    // on.  A second cluster barrier (below, all threads) keeps every CTA's shared memory alive until its
+    // peers have read it.
+    if constexpr (!kDyn) {
+      if (p.cluster_size > 1) {
+        __syncwarp();
+        cluster_arrive_release();                          // this thread's parked values are written
+        cluster_wait();
+        stamp(6);
+        const WorkItem item = item_of(0, 0);
+        const int n_rows = item.n_nodes * g;
+        const int tid = h * BMH + r;
+        const uint32_t park_u32 = smem_u32(smem);
+        const uint32_t rank = cluster_ctarank();
+        need_dep();                                        // global writes below
+        auto merge = [&](auto c_tag) {
+          constexpr int C = decltype(c_tag)::value;
+          constexpr int kRows = 2 * BMH / C;               // rows per CTA
+          constexpr int V = D / 32;                        // floats per lane: a warp reads one whole parked row per load
+          constexpr int KR = 4;                            // rows per warp and pass
+          const int mw = tid >> 5, lk = lane >> 3, lu = lane & 7;
+          uint32_t base[C];
+#pragma unroll
+          for (int s_ = 0; s_ < C; ++s_) base[s_] = map_to_cta(park_u32, uint32_t(s_));
+          // A pass: KR rows per warp.  Lane 8 k + u fetches (m, l) of row k from CTA u; every lane fetches its V
+          // columns of the KR rows from all C CTAs, all requested before anything is used.  (Loads of a peer's
+          // shared memory are slow when a warp's lanes ask for 32 different rows; one row per request is not.)
+          for (int pr0 = int(rank) * kRows + KR * mw; pr0 < (int(rank) + 1) * kRows; pr0 += 8 * KR) {
+            float mv = -INFINITY, lv = 0.f;
+            if (lu < C) {
+              const uint32_t sc_base = map_to_cta(park_u32, uint32_t(lu)) + uint32_t(L::kParkScalars);
+              mv = ld_dsmem_f32(sc_base + 4u * uint32_t(pr0 + lk));
+              lv = ld_dsmem_f32(sc_base + 4u * uint32_t(2 * BMH + pr0 + lk));
+            }
+            float vv[KR][C][V];
+#pragma unroll
+            for (int k = 0; k < KR; ++k)
+#pragma unroll
+              for (int s_ = 0; s_ < C; ++s_) {
+                const uint32_t at = base[s_] + 4u * uint32_t((pr0 + k) * L::kParkRow + lane * V);
+                if constexpr (V == 4) {
+                  const float4 x = ld_dsmem_f32x4(at);
+                  vv[k][s_][0] = x.x; vv[k][s_][1] = x.y; vv[k][s_][2] = x.z; vv[k][s_][3] = x.w;
+                } else {
+                  const float2 x = ld_dsmem_f32x2(at);
+                  vv[k][s_][0] = x.x; vv[k][s_][1] = x.y;
+                }
+              }
+            float m_r = mv;
+            m_r = fmaxf(m_r, __shfl_xor_sync(0xffffffffu, m_r, 1));
+            m_r = fmaxf(m_r, __shfl_xor_sync(0xffffffffu, m_r, 2));
+            m_r = fmaxf(m_r, __shfl_xor_sync(0xffffffffu, m_r, 4));
+            const float f_l = lu < C ? fast_exp2(mv - (m_r == -INFINITY ? 0.f : m_r)) : 0.f;
+            float lsum = f_l * lv;
+            lsum += __shfl_xor_sync(0xffffffffu, lsum, 1);
+            lsum += __shfl_xor_sync(0xffffffffu, lsum, 2);
+            lsum += __shfl_xor_sync(0xffffffffu, lsum, 4);
+#pragma unroll
+            for (int k = 0; k < KR; ++k) {
+              float acc[V];
+#pragma unroll
+              for (int e = 0; e < V; ++e) acc[e] = 0.f;
+#pragma unroll
+              for (int s_ = 0; s_ < C; ++s_) {
+                const float f = __shfl_sync(0xffffffffu, f_l, 8 * k + s_);
+#pragma unroll
+                for (int e = 0; e < V; ++e) acc[e] += f * vv[k][s_][e];
+              }
+              const float lk_sum = __shfl_sync(0xffffffffu, lsum, 8 * k);
+              const int row = item.row0 + pr0 + k;
+              if (row < n_rows) {
+                const float inv = lk_sum > 0.f ? 1.f / lk_sum : 0.f;
+                __nv_bfloat16* out = p.out + (size_t(item.node0 + (row >> p.log2_g)) * p.n_q_heads + item.kv_head * g + (row & (g - 1))) * D;
+                if constexpr (V == 4) {
+                  uint2 o;
+                  o.x = pack_bf16x2(acc[0] * inv, acc[1] * inv);
+                  o.y = pack_bf16x2(acc[2] * inv, acc[3] * inv);
+                  *reinterpret_cast<uint2*>(out + lane * 4) = o;
+                } else {
+                  *reinterpret_cast<uint32_t*>(out + lane * 2) = pack_bf16x2(acc[0] * inv, acc[1] * inv);
+                }
+              }
+            }
+          }
+        };
+        if (p.cluster_size == 2) merge(std::integral_constant<int, 2>{});
+        else if (p.cluster_size == 4) merge(std::integral_constant<int, 4>{});
+        else merge(std::integral_constant<int, 8>{});
+      }
+    }
     stamp(7);
   }
 
+  // cluster plans: no CTA leaves (its shared memory with it) before its peers have fetched what they need
+  if (p.cluster_size > 1) {
+    __syncwarp();
+    cluster_arrive_release();
+    cluster_wait();
+  }
   tc_fence_before();
   __syncthreads();
   if (warp == 2) {
@@ -1122,15 +1270,19 @@ cudaError_t launch_attn_tc(int head_dim, int n_ctas, const CUtensorMap& mq, cons
   FirstItems first;
   const size_t stride = p.queue != nullptr ? 1 : size_t(p.items_stride);
   for (int c = 0; c < kFirstItems; ++c) first.item[c] = c < n_ctas ? host_items[size_t(c) * stride] : WorkItem{};
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[1].id = cudaLaunchAttributeClusterDimension;      // cluster plans: one cluster per split group
+  attr[1].val.clusterDim.x = unsigned(p.cluster_size > 1 ? p.cluster_size : 1);
+  attr[1].val.clusterDim.y = 1;
+  attr[1].val.clusterDim.z = 1;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(unsigned(n_ctas));
   cfg.blockDim = dim3(unsigned(kThreads));
   cfg.stream = stream;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = p.cluster_size > 1 ? 2 : 1;
   const bool dyn = p.queue != nullptr;
   cudaError_t le = cudaSuccess;
   if (head_dim == 128) {

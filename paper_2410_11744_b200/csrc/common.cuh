@@ -348,6 +348,7 @@ __device__ __forceinline__ void cluster_sync_all() {
 // thread arrives early and waits only when it needs the peers to have arrived.
 // (relaxed: what the peers must see -- the initialised mbarriers -- was published by fence.mbarrier_init)
 __device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_arrive_release() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
 // Asynchronous copy of `bytes` (a multiple of 16; both addresses 16-byte aligned) from this CTA's
 // shared memory into a peer CTA's; the peer's mbarrier receives the byte count when the data has

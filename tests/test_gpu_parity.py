@@ -347,7 +347,8 @@ def test_calls_that_follow_each_other_may_share_a_workspace(rt, shape):
         tuning = (-1, 0, 0)          # separate combine kernel instead of the cluster merge
     else:
         mk = lambda seed: wl.make_custom(seed, 4, 4, 128, [2500], [wl.random_tree(np.random.default_rng(6), 256)])
-        tuning = (-1, 0, 2)
+        tuning = (-1, 0, 1)          # merged inside the kernel through the workspace (the default plan for this shape
+                                     # is a cluster plan, which has no workspace)
     wa, wb = mk(301), mk(302)
     B.dyspec_set_tuning(*tuning)
     try:
@@ -379,12 +380,35 @@ def test_merge_inside_the_tensor_core_kernel(rt, hq, hkv, d, L, n, ctas):
     B, R = rt
     rng = np.random.default_rng(hq * 1000 + n)
     w = wl.make_custom(70, hq, hkv, d, [L], [wl.greedy_tree(rng, n, 6, 0.3)])
-    batch, got, _ = run_and_check(rt, w, regime=1, ctas=ctas, fuse=2 + (16 if ctas else 0))
+    batch, got, _ = run_and_check(rt, w, regime=1, ctas=ctas, fuse=1 + (16 if ctas else 0))     # 1: never clusters
     info = batch.plan.describe()
-    assert info["regime"] == 1 and info["split_groups"] > 0 and info["combine_launch"] == 0
+    assert info["regime"] == 1 and info["split_groups"] > 0 and info["combine_launch"] == 0 and info["cluster"] == 1
     if ctas == 0:
         assert info["max_splits"] > 8 or d == 64
     batch.out.zero_()
     batch.attention()
     _, _, out2, status = batch.results()
     assert status == 0 and np.array_equal(orc.bf16_bits_to_f64(out2), got)
+
+
+@pytest.mark.parametrize("hq,hkv,d,L,n,want_c", [(8, 8, 128, 2000, 256, 8), (16, 16, 128, 1500, 200, 4), (64, 64, 64, 700, 130, 2),
+                                                 (8, 1, 128, 3000, 12, 8), (32, 4, 64, 1000, 64, 4)])
+def test_cluster_merge_in_the_tensor_core_regime(rt, hq, hkv, d, L, n, want_c):
+    """Few groups of equal length: one thread-block cluster per group, every CTA parks its partial in shared
+    memory and fetches its share of the rows from its peers.  Cluster sizes 2, 4 and 8, both head dimensions,
+    a ragged second half, a group with one half only (the other half parks neutral rows), GQA.  No workspace,
+    no second launch; a second call on the same buffers gives the same bits."""
+    B, R = rt
+    rng = np.random.default_rng(hq * 100 + n)
+    w = wl.make_custom(75, hq, hkv, d, [L], [wl.greedy_tree(rng, n, 6, 0.3)])
+    batch, got, _ = run_and_check(rt, w, regime=1)
+    info = batch.plan.describe()
+    assert info["regime"] == 1 and info["cluster"] == want_c and info["combine_launch"] == 0, info
+    assert batch.plan.workspace_bytes() == 0
+    batch.out.zero_()
+    batch.attention()
+    _, _, out2, status = batch.results()
+    assert status == 0 and np.array_equal(orc.bf16_bits_to_f64(out2), got)
+    # the same request merged through the workspace instead: the same result up to the order of the additions
+    _, got_l2, _ = run_and_check(rt, w, regime=1, fuse=1)
+    assert np.abs(got_l2 - got).max() <= 2e-2

@@ -136,8 +136,14 @@ def test_whole_group_plan_is_chosen_when_cheaper(B):
     w3 = wl.make_config(3)
     args3 = (w3.n_q_heads, w3.n_kv_heads, w3.head_dim, w3.prefix_len.tolist(), w3.n_nodes.tolist())
     info3, loads3 = check_schedule(B, *args3)
-    # few long groups: even pieces, one per CTA, on as many CTAs as there are SMs (20 groups in 5, 12 in 4)
-    assert info3["split_groups"] == 32 and info3["ctas"] == 148 == info3["items"] and max(loads3) == 9
+    # few long groups of equal length: one cluster of 4 CTAs per group, merged through distributed shared memory
+    assert info3["cluster"] == 4 and info3["split_groups"] == 0 and info3["ctas"] == 128 == info3["items"]
+    assert max(loads3) == 9 and info3["workspace_bytes"] == 0 and info3["combine_launch"] == 0
+    # without clusters: even pieces, one per CTA, on as many CTAs as there are SMs (20 groups in 5, 12 in 4),
+    # merged inside the kernel through the workspace
+    info3e, loads3e = check_schedule(B, *args3, fuse=1)
+    assert info3e["cluster"] == 1 and info3e["split_groups"] == 32 and info3e["ctas"] == 148 == info3e["items"]
+    assert max(loads3e) == 9 and info3e["combine_launch"] == 0
     info3_always, loads3 = check_schedule(B, *args3, fuse=2 + 32)   # forced: 32 CTAs with 34 tiles each
     assert info3_always["split_groups"] == 0 and info3_always["ctas"] == 32 and set(loads3) == {34}
 

@@ -105,13 +105,20 @@ def test_static_scratch_entry_point_refuses_what_does_not_fit():
     from paper_2410_11744_b200 import build
     build.build()
     from paper_2410_11744_b200 import binding as B, runner as R
-    w = wl.make_config(3)                                     # 32 heads x 5 splits: ~21 MiB of partials, over the 16 MiB array
+    # 32 heads x 5 splits merged through the workspace: ~21 MiB of partials, over the 16 MiB array.  (The plan the
+    # scheduler would choose by itself for this shape is a cluster plan, which needs no workspace at all: the
+    # workspace merge is asked for here.)
+    w = wl.make_config(3)
     batch = R.DeviceBatch(w)
     batch.build_mask()
     out = torch.zeros_like(batch.out)
-    with pytest.raises(B.DyspecError) as e:
-        B.dyspec_tree_attention_static(batch.q, batch.k, batch.v, int(w.prefix_len[0]), batch.bits, int(w.n_nodes[0]),
-                                       out, w.n_q_heads, w.n_kv_heads, w.head_dim, batch.W)
+    B.dyspec_set_tuning(-1, 0, 1)
+    try:
+        with pytest.raises(B.DyspecError) as e:
+            B.dyspec_tree_attention_static(batch.q, batch.k, batch.v, int(w.prefix_len[0]), batch.bits, int(w.n_nodes[0]),
+                                           out, w.n_q_heads, w.n_kv_heads, w.head_dim, batch.W)
+    finally:
+        B.dyspec_set_tuning(-1, 0, 2)
     assert e.value.code == -3
     torch.cuda.synchronize()
     assert not out.any()
