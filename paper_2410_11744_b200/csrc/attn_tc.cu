@@ -53,12 +53,21 @@ struct TcLayout {
   static constexpr int kBarOffset = kRingOffset + kSlots * kTileBytes;
   static constexpr int kItemRingOffset = kBarOffset + 512;   // queue plans: the CTA's next work items, 8 entries of 64 bytes
   static constexpr int kTotal = kItemRingOffset + 512;
-  // Cluster plans: when its products are done a CTA parks its partial over the (idle) Q tile and ring:
-  // 256 rows of D + 4 floats (the padding keeps 16-byte row accesses of a warp off each other's banks),
-  // then the rows' maxima and sums.
+  // Cluster plans (C CTAs per group): when its products are done a CTA parks its partial over the (idle) Q
+  // tile and ring, as C shares of 256 / C rows, one per CTA of the cluster: a share is its rows (D + 4 floats
+  // each: the padding keeps 16-byte row accesses of a warp off each other's banks), then their maxima, then
+  // their sums.  Behind the parked partial is room for some of the peers' shares of THIS CTA's rows, which they
+  // push there with bulk copies; the rest is fetched from the peers with plain loads.
   static constexpr int kParkRow = D + 4;
-  static constexpr int kParkScalars = 2 * BMH * kParkRow * 4;
-  static_assert(kParkScalars + 2 * 2 * BMH * 4 <= kBarOffset, "the parked partial fits in front of the barriers");
+  static constexpr int kParkRowBytes = kParkRow * 4 + 8;       // a row and its two scalars
+  static constexpr int kParkTotal = 2 * BMH * kParkRowBytes;
+  static constexpr int kRecvOffset = kParkTotal;
+  static_assert(kParkTotal % 16 == 0 && kParkTotal + BMH * kParkRowBytes <= kBarOffset, "parked partial + one share of 128 rows");
+  // shares of 256 / C rows that fit behind the parked partial, at most C - 1
+  __host__ __device__ static constexpr int pushed_shares(int c) {
+    const int fit = (kBarOffset - kRecvOffset) / ((2 * BMH / c) * kParkRowBytes);
+    return fit < c - 1 ? fit : c - 1;
+  }
 };
 
 // Trace tags (see dyspec_set_trace): tag = role << 14 | event << 10 | key-tile index j.
@@ -71,7 +80,7 @@ struct TcLayout {
 // barrier indices (8 bytes each)
 enum { B_QFULL = 0, B_QFREE = 1, B_SLOT_FULL = 2, B_SLOT_EMPTY = B_SLOT_FULL + kSlots,
        B_SREADY = B_SLOT_EMPTY + kSlots, B_PREADY = B_SREADY + 2, B_ODONE = B_PREADY + 2, B_OFREE = B_ODONE + 2,
-       B_PVDONE = B_OFREE + 2, B_QFULLB = B_PVDONE + 2, B_COUNT = B_QFULLB + 1 };
+       B_PVDONE = B_OFREE + 2, B_QFULLB = B_PVDONE + 2, B_RECV = B_QFULLB + 1, B_COUNT = B_RECV + 1 };
 
 // Hardware named barriers for thread-to-thread hand-offs inside the CTA (P ready: 128 softmax threads
 // -> the MMA-issuing warp): an order of magnitude quicker to notice than an mbarrier in shared memory
@@ -289,6 +298,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   if (threadIdx.x == 0) {
     mbar_init(bar(B_QFULL), 1);
     mbar_init(bar(B_QFULLB), 1);
+    mbar_init(bar(B_RECV), 1);             // cluster plans: the peers' shares pushed into this CTA have landed
     mbar_init(bar(B_QFREE), 2);
     for (int s = 0; s < kSlots; ++s) {
       mbar_init(bar(B_SLOT_FULL + s), 1);
@@ -374,6 +384,17 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     return idx < p.n_items_total ? idx : -1;
   };
   const int g = p.group_size;
+  // Cluster plans: where packed row pr of the parked partial lies (share pr / rows, rows = 256 / C), in bytes
+  // from the start of shared memory: the row itself, and its maximum (its sum is 4 * rows bytes further).
+  const int park_log2rows = 8 - (p.cluster_size >= 8 ? 3 : p.cluster_size >= 4 ? 2 : 1);
+  auto park_row_at = [&](int pr) -> int {
+    const int rows = 1 << park_log2rows;
+    return (pr >> park_log2rows) * rows * L::kParkRowBytes + (pr & (rows - 1)) * (L::kParkRow * 4);
+  };
+  auto park_max_at = [&](int pr) -> int {
+    const int rows = 1 << park_log2rows;
+    return (pr >> park_log2rows) * rows * L::kParkRowBytes + rows * (L::kParkRow * 4) + (pr & (rows - 1)) * 4;
+  };
 
   // Register budget: the softmax threads hold a whole S row; the control warps need few registers.
   trigger_dependents();     // the next kernel of the stream may be scheduled; it waits for this grid before it touches what this one writes
@@ -654,13 +675,13 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         }
         if (p.cluster_size > 1) {                          // cluster plan: the peers read this half's rows all the same
           named_sync(kBarMerge, 2 * BMH);                  // (the other half's products no longer read the Q tile and the ring)
-          float* park = reinterpret_cast<float*>(smem);
           const int pr = h * BMH + r;
+          uint8_t* row_at = smem + park_row_at(pr);
 #pragma unroll
-          for (int i = 0; i < D / 4; ++i) *reinterpret_cast<float4*>(park + pr * L::kParkRow + 4 * i) = make_float4(0.f, 0.f, 0.f, 0.f);
-          float* park_m = reinterpret_cast<float*>(smem + L::kParkScalars);
-          park_m[pr] = -INFINITY;
-          park_m[2 * BMH + pr] = 0.f;
+          for (int i = 0; i < D / 4; ++i) *reinterpret_cast<float4*>(row_at + 16 * i) = make_float4(0.f, 0.f, 0.f, 0.f);
+          *reinterpret_cast<float*>(smem + park_max_at(pr)) = -INFINITY;
+          *reinterpret_cast<float*>(smem + park_max_at(pr) + (4 << park_log2rows)) = 0.f;
+          fence_proxy_async();                             // (bulk copies read the parked rows)
         }
         continue;
       }
@@ -846,14 +867,14 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         tc_fence_before();
         mbar_arrive(bar(B_OFREE + h));
         named_sync(kBarMerge, 2 * BMH);                    // both halves' products are done: Q tile and ring are idle
-        float* park = reinterpret_cast<float*>(smem);
         const int pr = h * BMH + r;
+        uint8_t* row_at = smem + park_row_at(pr);
 #pragma unroll
         for (int i = 0; i < D / 4; ++i)
-          *reinterpret_cast<uint4*>(park + pr * L::kParkRow + 4 * i) = make_uint4(ov[4 * i], ov[4 * i + 1], ov[4 * i + 2], ov[4 * i + 3]);
-        float* park_m = reinterpret_cast<float*>(smem + L::kParkScalars);
-        park_m[pr] = m_used;
-        park_m[2 * BMH + pr] = l;
+          *reinterpret_cast<uint4*>(row_at + 16 * i) = make_uint4(ov[4 * i], ov[4 * i + 1], ov[4 * i + 2], ov[4 * i + 3]);
+        *reinterpret_cast<float*>(smem + park_max_at(pr)) = m_used;
+        *reinterpret_cast<float*>(smem + park_max_at(pr) + (4 << park_log2rows)) = l;
+        fence_proxy_async();                               // (bulk copies read the parked rows)
       } else if (item.slot < 0 && staged) {
         const float inv = l > 0.f ? 1.f / l : 0.f;
         uint32_t ov[D];
@@ -1144,54 +1165,91 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       }
     }
     // ---- split-KV merge of a cluster plan: the CTAs of a cluster hold the pieces of one (request, kv head,
-    // query tile) group, one item each.  Once every CTA has parked its partial (cluster barrier), CTA k
-    // fetches rows [k * 256 / C, (k + 1) * 256 / C) of all C partials from the peers' shared memory (its own
-    // included), merges and stores them: nothing goes through global memory, and there is no counter to wait
-    // on.  A second cluster barrier (below, all threads) keeps every CTA's shared memory alive until its
-    // peers have read it.
+    // query tile) group, one item each, and CTA k merges rows [k * 256 / C, (k + 1) * 256 / C) of the C
+    // partials.  Once every CTA has parked its partial (cluster barrier: every CTA's products are done, so
+    // its shared memory can also take what the peers send), each CTA pushes its shares of some peers' rows
+    // into those peers with bulk copies (as many as fit behind a parked partial) and fetches the remaining
+    // peers' shares of its own rows with plain loads of their shared memory, which are far slower per byte
+    // but need no room.  Nothing goes through global memory, and there is no counter to wait on.  A second
+    // cluster barrier (below, all threads) keeps every CTA's shared memory alive until its peers are done.
     if constexpr (!kDyn) {
       if (p.cluster_size > 1) {
+        const int tid = h * BMH + r;
+        const uint32_t rank = cluster_ctarank();
+        const uint32_t park_u32 = smem_u32(smem);
         __syncwarp();
         cluster_arrive_release();                          // this thread's parked values are written
         cluster_wait();
         stamp(6);
         const WorkItem item = item_of(0, 0);
         const int n_rows = item.n_nodes * g;
-        const int tid = h * BMH + r;
-        const uint32_t park_u32 = smem_u32(smem);
-        const uint32_t rank = cluster_ctarank();
         need_dep();                                        // global writes below
         auto merge = [&](auto c_tag) {
           constexpr int C = decltype(c_tag)::value;
           constexpr int kRows = 2 * BMH / C;               // rows per CTA
+          constexpr int kShare = kRows * L::kParkRowBytes; // bytes of a share
+          constexpr int NP = L::pushed_shares(C);          // peers whose shares of my rows are pushed to me
           constexpr int V = D / 32;                        // floats per lane: a warp reads one whole parked row per load
           constexpr int KR = 4;                            // rows per warp and pass
+          // Slot j of this CTA's receive area is filled by CTA (rank + 1 + j) % C, i.e. this CTA sends its share
+          // of CTA d's rows to slot j of d = (rank - 1 - j) mod C.  Four lanes per copy, so that the copies overlap.
+          if (tid == 0) mbar_expect_tx(bar(B_RECV), uint32_t(NP * kShare));
+          if (tid < 4 * NP) {
+            const uint32_t j = uint32_t(tid) >> 2, piece = uint32_t(tid) & 3u;
+            const uint32_t d = (rank + uint32_t(2 * C - 1) - j) % uint32_t(C);
+            constexpr uint32_t part = uint32_t(kShare / 4);          // a multiple of 16 bytes for every C and D
+            dsmem_push(map_to_cta(park_u32 + uint32_t(L::kRecvOffset) + j * uint32_t(kShare) + piece * part, d),
+                       park_u32 + d * uint32_t(kShare) + piece * part, part, map_to_cta(bar(B_RECV), d));
+          }
           const int mw = tid >> 5, lk = lane >> 3, lu = lane & 7;
-          uint32_t base[C];
+          // the sources of my rows: 0 = my own parked share, 1 .. NP = the receive slots, above = peers' shared memory
+          const uint8_t* own_share = smem + int(rank) * kShare;
+          const uint8_t* recv = smem + L::kRecvOffset;
+          uint32_t remote[C];                              // (entries up to NP are unused)
 #pragma unroll
-          for (int s_ = 0; s_ < C; ++s_) base[s_] = map_to_cta(park_u32, uint32_t(s_));
-          // A pass: KR rows per warp.  Lane 8 k + u fetches (m, l) of row k from CTA u; every lane fetches its V
-          // columns of the KR rows from all C CTAs, all requested before anything is used.  (Loads of a peer's
+          for (int s_ = NP + 1; s_ < C; ++s_)
+            remote[s_] = map_to_cta(park_u32 + rank * uint32_t(kShare), (rank + uint32_t(s_)) % uint32_t(C));
+          if (NP > 0) mbar_wait(bar(B_RECV), 0, abort_flag, p.status);
+          // A pass: KR rows per warp.  Lane 8 k + u fetches (m, l) of row k from source u; every lane fetches its V
+          // columns of the KR rows from all C sources, all requested before anything is used.  (Loads of a peer's
           // shared memory are slow when a warp's lanes ask for 32 different rows; one row per request is not.)
-          for (int pr0 = int(rank) * kRows + KR * mw; pr0 < (int(rank) + 1) * kRows; pr0 += 8 * KR) {
+          for (int r0 = KR * mw; r0 < kRows; r0 += 8 * KR) {
             float mv = -INFINITY, lv = 0.f;
             if (lu < C) {
-              const uint32_t sc_base = map_to_cta(park_u32, uint32_t(lu)) + uint32_t(L::kParkScalars);
-              mv = ld_dsmem_f32(sc_base + 4u * uint32_t(pr0 + lk));
-              lv = ld_dsmem_f32(sc_base + 4u * uint32_t(2 * BMH + pr0 + lk));
+              const int at = kRows * (L::kParkRow * 4) + 4 * (r0 + lk);
+              if (lu <= NP) {
+                const uint8_t* src = lu == 0 ? own_share : recv + (lu - 1) * kShare;
+                mv = *reinterpret_cast<const float*>(src + at);
+                lv = *reinterpret_cast<const float*>(src + at + 4 * kRows);
+              } else {
+                const uint32_t src = map_to_cta(park_u32 + rank * uint32_t(kShare), (rank + uint32_t(lu)) % uint32_t(C));
+                mv = ld_dsmem_f32(src + uint32_t(at));
+                lv = ld_dsmem_f32(src + uint32_t(at + 4 * kRows));
+              }
             }
             float vv[KR][C][V];
 #pragma unroll
             for (int k = 0; k < KR; ++k)
 #pragma unroll
               for (int s_ = 0; s_ < C; ++s_) {
-                const uint32_t at = base[s_] + 4u * uint32_t((pr0 + k) * L::kParkRow + lane * V);
-                if constexpr (V == 4) {
-                  const float4 x = ld_dsmem_f32x4(at);
-                  vv[k][s_][0] = x.x; vv[k][s_][1] = x.y; vv[k][s_][2] = x.z; vv[k][s_][3] = x.w;
+                const int at = (r0 + k) * (L::kParkRow * 4) + lane * (4 * V);
+                if (s_ <= NP) {
+                  const uint8_t* src = (s_ == 0 ? own_share : recv + (s_ - 1) * kShare) + at;
+                  if constexpr (V == 4) {
+                    const float4 x = *reinterpret_cast<const float4*>(src);
+                    vv[k][s_][0] = x.x; vv[k][s_][1] = x.y; vv[k][s_][2] = x.z; vv[k][s_][3] = x.w;
+                  } else {
+                    const float2 x = *reinterpret_cast<const float2*>(src);
+                    vv[k][s_][0] = x.x; vv[k][s_][1] = x.y;
+                  }
                 } else {
-                  const float2 x = ld_dsmem_f32x2(at);
-                  vv[k][s_][0] = x.x; vv[k][s_][1] = x.y;
+                  if constexpr (V == 4) {
+                    const float4 x = ld_dsmem_f32x4(remote[s_] + uint32_t(at));
+                    vv[k][s_][0] = x.x; vv[k][s_][1] = x.y; vv[k][s_][2] = x.z; vv[k][s_][3] = x.w;
+                  } else {
+                    const float2 x = ld_dsmem_f32x2(remote[s_] + uint32_t(at));
+                    vv[k][s_][0] = x.x; vv[k][s_][1] = x.y;
+                  }
                 }
               }
             float m_r = mv;
@@ -1215,7 +1273,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 for (int e = 0; e < V; ++e) acc[e] += f * vv[k][s_][e];
               }
               const float lk_sum = __shfl_sync(0xffffffffu, lsum, 8 * k);
-              const int row = item.row0 + pr0 + k;
+              const int row = item.row0 + int(rank) * kRows + r0 + k;
               if (row < n_rows) {
                 const float inv = lk_sum > 0.f ? 1.f / lk_sum : 0.f;
                 __nv_bfloat16* out = p.out + (size_t(item.node0 + (row >> p.log2_g)) * p.n_q_heads + item.kv_head * g + (row & (g - 1))) * D;
@@ -1230,6 +1288,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
               }
             }
           }
+          if (tid < 4 * NP) dsmem_push_wait_source_read();    // the parked rows must outlive the copies that read them
         };
         if (p.cluster_size == 2) merge(std::integral_constant<int, 2>{});
         else if (p.cluster_size == 4) merge(std::integral_constant<int, 4>{});
