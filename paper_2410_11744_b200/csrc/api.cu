@@ -49,6 +49,7 @@ cudaError_t launch_compact_kv(void* k_cache, void* v_cache, const int64_t* kv_ro
 cudaError_t launch_attn_small(int head_dim, int n_ctas, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                             const AttnParams& p, const WorkItem* host_items, cudaStream_t stream);
 cudaError_t launch_combine(int head_dim, int bm, int n_split_groups, const AttnParams& p, cudaStream_t stream);
+int attn_tc_max_clusters(int head_dim, int cluster_size);
 cudaError_t launch_attn_tc(int head_dim, int n_ctas, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                            const AttnParams& p, const WorkItem* host_items, cudaStream_t stream);
 }  // namespace dyspec
@@ -895,6 +896,12 @@ static int make_host_plan(dyspec_plan** out, int n_q_heads, int n_kv_heads, int 
   pl->bm = pl->regime == 0 ? 64 : 256;    // packed query rows per work item (regime 1: two 128-row halves)
   pl->bn = pl->regime == 0 ? 64 : 128;    // keys per tile
   schedule(*pl);
+  // A cluster plan of the tensor-core regime needs C CTAs of 1 CTA / SM side by side: where the device cannot
+  // hold even one such cluster (a reduced share of its SMs), plan again without clusters.
+  if (pl->regime == 1 && pl->cluster > 1 && attn_tc_max_clusters(pl->d, pl->cluster) == 0) {
+    pl->tune.combine_mode = 1;
+    schedule(*pl);
+  }
   pl->workspace_bytes = size_t(pl->n_slots) * size_t(pl->bm) * (pl->d + 2) * sizeof(float);
   if (!pl->split_groups.empty()) {      // the groups' counter pairs follow the partials
     pl->counters_offset = (pl->workspace_bytes + 255) & ~size_t(255);

@@ -1323,6 +1323,47 @@ cudaError_t launch_one(cudaLaunchConfig_t& cfg, size_t smem, const CUtensorMap& 
 }
 }  // namespace
 
+// How many clusters of `cluster_size` CTAs of this kernel the current device can hold at once (0: such a
+// cluster cannot be launched at all, e.g. on a reduced share of the SMs); -1 when that cannot be asked
+// (no device).  Asked once per (device, head dimension, cluster size).
+int attn_tc_max_clusters(int head_dim, int cluster_size) {
+  static std::atomic<int> cache[DynSmemGrant::kDevices][2][4];
+  static std::atomic<bool> init{false};
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= DynSmemGrant::kDevices) { cudaGetLastError(); return -1; }
+  if (!init.exchange(true))
+    for (auto& d : cache) for (auto& h : d) for (auto& c : h) c.store(-2);
+  const int hi = head_dim == 128 ? 0 : 1, ci = cluster_size == 8 ? 3 : cluster_size == 4 ? 2 : cluster_size == 2 ? 1 : 0;
+  int have = cache[dev][hi][ci].load();
+  if (have != -2 && have != -3) return have;           // (-3: another thread is filling the table; ask again below, harmless)
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = unsigned(cluster_size);
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(unsigned(cluster_size));
+  cfg.blockDim = dim3(unsigned(kThreads));
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  int n = 0;
+  cudaError_t e;
+  if (head_dim == 128) {
+    cfg.dynamicSmemBytes = TcLayout<128>::kTotal + 1024;
+    static DynSmemGrant grant;
+    e = grant.ensure(tree_attn_tc_kernel<128, false, false>, cfg.dynamicSmemBytes);
+    if (e == cudaSuccess) e = cudaOccupancyMaxActiveClusters(&n, tree_attn_tc_kernel<128, false, false>, &cfg);
+  } else {
+    cfg.dynamicSmemBytes = 120 * 1024;
+    static DynSmemGrant grant;
+    e = grant.ensure(tree_attn_tc_kernel<64, false, false>, cfg.dynamicSmemBytes);
+    if (e == cudaSuccess) e = cudaOccupancyMaxActiveClusters(&n, tree_attn_tc_kernel<64, false, false>, &cfg);
+  }
+  if (e != cudaSuccess) { cudaGetLastError(); n = 0; }
+  cache[dev][hi][ci].store(n);
+  return n;
+}
+
 cudaError_t launch_attn_tc(int head_dim, int n_ctas, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                            const AttnParams& p, const WorkItem* host_items, cudaStream_t stream) {
   // host_items: the host copy of p.items (same layout); each CTA's first item travels as a kernel parameter
