@@ -322,6 +322,28 @@ def measure_config(torch, runner, w, steps, warmup, device, sparse=False, paged=
                 graph=g_step)
 
 
+def isolated_floor(torch):
+    """What the isolated protocol reads for a kernel that does nothing, and for no kernel at all: the same
+    spin kernel, events and median as in measure_config, around torch's one-cycle spin kernel and around
+    nothing.  Context for the isolated durations (every one of them contains this much launch and event
+    latency); the graded figures are not corrected by it."""
+    stream = torch.cuda.current_stream()
+    out = {}
+    for label, fn in (("empty_kernel_us", lambda: torch.cuda._sleep(1)), ("event_pair_us", lambda: None)):
+        ts = []
+        for _ in range(ISOLATED_CALLS):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            torch.cuda._sleep(100000)
+            e0.record(stream)
+            fn()
+            e1.record(stream)
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1))
+        out[label] = _median(ts[8:]) * 1e3
+    return out
+
+
 def random_tree_experiment(torch, runner, workloads, B, peaks, device, sizes=(256, 512, 1024, 2048), steps=200):
     """The paper's random-tree attention experiment (App. C.1, Table 5: one request, 64 heads x 128,
     no prefix, uniform random recursive trees): block counts and attention time in creation order
@@ -743,6 +765,7 @@ def run_ours(args):
     else:
         roof_rows.append(compact_roofline(args.config, w, m, roof))
     roof["per_config"] = roof_rows
+    roof["isolated_floor"] = isolated_floor(torch)
 
     random_tree = None
     if not args.no_per_config and world == 1:

@@ -154,7 +154,8 @@ int dyspec_schedule_dry_run(int n_q_heads, int n_kv_heads, int head_dim, int n_r
  * 1 = as 2, but the tcgen05 regime never uses clusters.  (Items that merge through the workspace wait for
  * each other inside the kernel, bounded to one second: this assumes that the process may use every SM of the
  * device it counted.  Where it may not -- a reduced SM share under MPS, a green context -- create the plans
- * with m = 0.  The CTAs of a cluster are scheduled together by the hardware: no such assumption there.)  k says whether the scheduler may deal whole
+ * with m = 0.  The CTAs of a cluster are scheduled together by the hardware: no such assumption there; where
+ * the device cannot hold even one cluster of the planned size, the plan falls back to the workspace merge.)  k says whether the scheduler may deal whole
  * (unsplit) groups to the CTAs instead of cutting them to equal budgets: 0 (default) = when its cost
  * model says that is quicker (and force_ctas is 0), 1 = never, 2 = always. */
 int dyspec_set_tuning(int force_regime, int force_ctas, int combine_mode);
