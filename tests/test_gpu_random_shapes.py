@@ -127,3 +127,56 @@ def test_random_large_ragged_batches_on_sampled_rows(rt, seed):
             err = np.abs(got[qo:qo + n][nodes] - ref)
             assert err.max() <= MAX_ABS and err.mean() <= MEAN_ABS, (what, r, err.max(), err.mean())
             qo += n
+
+
+def _draw_few_long(rng, index):
+    """One to three requests with long prefixes: the shapes that get cluster plans, even pieces merged through
+    the workspace, or the combine launch, depending on the merge mode."""
+    g = int(rng.choice([1, 2, 4, 8]))
+    hkv = int(rng.choice([1, 2, 4, 8, 16]))
+    d = int(rng.choice([64, 128]))
+    n_req = int(rng.choice([1, 1, 1, 2, 3]))
+    Ls = [int(np.exp(rng.uniform(np.log(100.0), np.log(7000.0)))) for _ in range(n_req)]
+    ns = [int(rng.choice([5, 12, 33, 64, 100, 129, 256, 300, 512])) for _ in range(n_req)]
+    trees = [wl.greedy_tree(rng, k, 6, 0.3) if rng.random() < 0.7 else wl.random_tree(rng, k) for k in ns]
+    return wl.make_custom(30000 + index, hkv * g, hkv, d, Ls, trees)
+
+
+def test_random_plans_merge_modes_and_cache_layouts(rt):
+    """Few long requests under every merge mode (0 combine launch, 1 through the workspace inside the kernel,
+    2 clusters where the plan allows), either regime, and the three cache layouts (contiguous, paged with the
+    tree rows outside the pages, paged with the tree rows inside); sampled rows against the oracle."""
+    B, R = rt
+    seen = set()
+    for seed, index in [(s_, i) for s_ in (31, 32) for i in range(24)]:
+        if index == 0:
+            rng = np.random.default_rng(seed)
+        w = _draw_few_long(rng, 100 * seed + index)
+        layout = int(rng.integers(0, 3))
+        page = int(rng.choice([128, 256, 1024]))
+        paged = None if layout == 0 else wl.to_paged(w, page, seed=seed, tree_in_pages=(layout == 2))
+        combine, regime = int(rng.choice([2, 2, 2, 1, 0])), int(rng.choice([-1, -1, 1]))
+        B.dyspec_set_tuning(regime, 0, combine)
+        try:
+            batch = R.DeviceBatch(w, paged=paged)
+        finally:
+            B.dyspec_set_tuning(-1, 0, 2)
+        for _ in range(2):
+            batch.step()
+        _, _, out_bits, status = batch.results()
+        info = batch.plan.describe()
+        what = dict(heads=(w.n_q_heads, w.n_kv_heads), d=w.head_dim, L=w.prefix_len.tolist(), n=w.n_nodes.tolist(),
+                    layout=layout, page=page, combine=combine, regime=regime, plan=info)
+        seen.add((info["regime"], info["cluster"] > 1, info["split_groups"] > 0))
+        assert status == 0, what
+        got = orc.bf16_bits_to_f64(out_bits)
+        assert np.isfinite(got).all(), what
+        qo = 0
+        for r in range(w.n_req):
+            n, o, L = int(w.n_nodes[r]), int(w.kv_row_offset[r]), int(w.prefix_len[r])
+            nodes = sorted(set(rng.integers(0, n, size=min(n, 6)).tolist() + [0, n - 1]))
+            ref = orc.tree_attention_nodes(w.q[qo:qo + n], w.k[o:o + L + n], w.v[o:o + L + n], L, w.parents[r], nodes)
+            err = np.abs(got[qo:qo + n][nodes] - ref)
+            assert err.max() <= MAX_ABS and err.mean() <= MEAN_ABS, (what, r, err.max(), err.mean())
+            qo += n
+    assert (1, True, False) in seen and (1, False, True) in seen, seen      # cluster plans and workspace merges both ran
