@@ -171,3 +171,22 @@ def test_merge_in_kernel_only_when_the_grid_is_one_wave(B):
     assert check_schedule(B, *shape, regime=1, fuse=0)[0]["combine_launch"] == 1
     small = check_schedule(B, 32, 32, 128, [4096] * 8, [64] * 8)[0]  # regime 0, split, not uniform enough for clusters
     assert small["regime"] == 0 and small["split_groups"] > 0 and small["combine_launch"] == 1
+
+
+def test_cluster_plans_of_the_tensor_core_regime(B):
+    """Few groups of similar length in the tensor-core regime: one cluster of C CTAs per group (C the same
+    for all groups, at least two tiles per piece, all CTAs in one wave), no workspace; merge mode 1 keeps the
+    merge through the workspace; too many groups, or groups too short, get no clusters."""
+    for shape, want in (((8, 8, 128, [2000], [256]), 8), ((16, 16, 128, [1500], [200]), 4), ((64, 64, 64, [700], [130]), 2),
+                        ((8, 1, 128, [3000], [12]), 8)):
+        info, loads = check_schedule(B, *shape, regime=1)
+        assert info["cluster"] == want and info["workspace_bytes"] == 0 and info["combine_launch"] == 0, (shape, info)
+        assert info["ctas"] == info["groups"] * want and min(loads) >= 2 and max(loads) - min(loads) <= 1
+        never = check_schedule(B, *shape, regime=1, fuse=1)[0]
+        assert never["cluster"] == 1 and never["combine_launch"] == 0
+    # 128 groups: two CTAs each would not fit in one wave
+    assert check_schedule(B, 64, 8, 128, [2048], [512], regime=1)[0]["cluster"] == 1
+    # one group of three tiles: a piece would have fewer than two
+    assert check_schedule(B, 8, 1, 128, [200], [16], regime=1)[0]["cluster"] == 1
+    # two requests of very different length: the cost model decides, every tile is still covered once (check_schedule)
+    check_schedule(B, 16, 16, 128, [6000, 300], [200, 200], regime=1)
