@@ -148,14 +148,16 @@ int dyspec_schedule_dry_run(int n_q_heads, int n_kv_heads, int head_dim, int n_r
  * CTAs the scheduler balances over (0 = automatic; a negative value -c instead sets the scheduler's
  * per-item cost to c key tiles), and combine_mode = m + 16 k.  m says how split-KV partials are merged:
  * 0 = by the separate combine kernel, 2 (default) = without a combine launch where the plan allows: inside a
- * thread-block cluster through distributed shared memory when the plan is uniform enough (few groups of
- * similar length: one cluster per group, no workspace; both regimes), else in the tcgen05 regime by the split
- * items themselves inside the attention kernel, through the workspace, when the grid is one wave; else as 0.
- * 1 = as 2, but the tcgen05 regime never uses clusters.  (Items that merge through the workspace wait for
- * each other inside the kernel, bounded to one second: this assumes that the process may use every SM of the
- * device it counted.  Where it may not -- a reduced SM share under MPS, a green context -- create the plans
- * with m = 0.  The CTAs of a cluster are scheduled together by the hardware: no such assumption there; where
- * the device cannot hold even one cluster of the planned size, the plan falls back to the workspace merge.)  k says whether the scheduler may deal whole
+ * thread-block cluster per group when the plan is uniform enough (few groups of similar length; small-tile
+ * regime: through distributed shared memory, no workspace; tcgen05 regime: the partials travel through the
+ * workspace and the cluster's hardware barrier stands in for counters and polling), else in the tcgen05
+ * regime by the split items themselves inside the attention kernel, with arrival counters in the workspace,
+ * when the grid is one wave; else as 0.  1 = as 2, but the tcgen05 regime never uses clusters.  (Items that
+ * wait for arrival counters do so inside the kernel, bounded to one second: this assumes that the process may
+ * use every SM of the device it counted.  Where it may not -- a reduced SM share under MPS, a green context --
+ * create the plans with m = 0.  The CTAs of a cluster are scheduled together by the hardware: no such
+ * assumption there; where the device cannot hold even one cluster of the planned size, the plan falls back
+ * to the counters.)  k says whether the scheduler may deal whole
  * (unsplit) groups to the CTAs instead of cutting them to equal budgets: 0 (default) = when its cost
  * model says that is quicker (and force_ctas is 0), 1 = never, 2 = always. */
 int dyspec_set_tuning(int force_regime, int force_ctas, int combine_mode);

@@ -50,6 +50,7 @@ cudaError_t launch_attn_small(int head_dim, int n_ctas, const CUtensorMap& mq, c
                             const AttnParams& p, const WorkItem* host_items, cudaStream_t stream);
 cudaError_t launch_combine(int head_dim, int bm, int n_split_groups, const AttnParams& p, cudaStream_t stream);
 int attn_tc_max_clusters(int head_dim, int cluster_size);
+size_t attn_tc_cluster_workspace_per_cta(int head_dim, int cluster_size);
 cudaError_t launch_attn_tc(int head_dim, int n_ctas, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                            const AttnParams& p, const WorkItem* host_items, cudaStream_t stream);
 }  // namespace dyspec
@@ -903,6 +904,8 @@ static int make_host_plan(dyspec_plan** out, int n_q_heads, int n_kv_heads, int 
     schedule(*pl);
   }
   pl->workspace_bytes = size_t(pl->n_slots) * size_t(pl->bm) * (pl->d + 2) * sizeof(float);
+  if (pl->regime == 1 && pl->cluster > 1)   // cluster plan: the shares a CTA's peers cannot push into its shared memory
+    pl->workspace_bytes = size_t(pl->n_ctas) * attn_tc_cluster_workspace_per_cta(pl->d, pl->cluster);
   if (!pl->split_groups.empty()) {      // the groups' counter pairs follow the partials
     pl->counters_offset = (pl->workspace_bytes + 255) & ~size_t(255);
     pl->workspace_bytes = pl->counters_offset + ((pl->split_groups.size() * 2 * sizeof(int32_t) + 255) & ~size_t(255));

@@ -23,12 +23,11 @@
 // An item whose group was cut along the keys writes an fp32 partial (O, m, l); after all of its items a CTA
 // merges, for each of its split items, a share of the group's rows (no combine launch; see the end of the
 // softmax branch).
-// Plans with few long groups of equal length run one thread-block cluster per group instead: every CTA parks
-// its partial in its own shared memory and fetches its share of the rows from its peers' (distributed shared
-// memory; nothing goes through global memory).
+// Plans with few long groups of equal length run one thread-block cluster per group instead: the cluster's
+// hardware barrier stands in for the arrival counters, fences and polling (the partials still travel
+// through L2: moving them between the CTAs' shared memories was measured and is no quicker).
 // Every wait on a flag or an mbarrier is bounded (see mbar_wait); every TMA load goes to this CTA alone, also
-// when the kernel is launched in clusters (the cluster is used for plain loads of peers' shared memory and
-// for its hardware barrier only).
+// when the kernel is launched in clusters (the cluster is used for its hardware barrier only).
 #include "common.cuh"
 #include <type_traits>
 
@@ -53,21 +52,14 @@ struct TcLayout {
   static constexpr int kBarOffset = kRingOffset + kSlots * kTileBytes;
   static constexpr int kItemRingOffset = kBarOffset + 512;   // queue plans: the CTA's next work items, 8 entries of 64 bytes
   static constexpr int kTotal = kItemRingOffset + 512;
-  // Cluster plans (C CTAs per group): when its products are done a CTA parks its partial over the (idle) Q
-  // tile and ring, as C shares of 256 / C rows, one per CTA of the cluster: a share is its rows (D + 4 floats
-  // each: the padding keeps 16-byte row accesses of a warp off each other's banks), then their maxima, then
-  // their sums.  Behind the parked partial is room for some of the peers' shares of THIS CTA's rows, which they
-  // push there with bulk copies; the rest is fetched from the peers with plain loads.
+  // Cluster plans (C CTAs per group): CTA k of a cluster merges rows [256 k / C, 256 (k + 1) / C) of the group.
+  // When its products are done a CTA keeps its own share of its partial in shared memory, over the (idle) Q
+  // tile: the rows (D + 4 floats each: the padding keeps 16-byte row accesses of a warp off each other's
+  // banks), then their maxima, then their sums.  The other shares go to their owners' slots in the workspace.
   static constexpr int kParkRow = D + 4;
   static constexpr int kParkRowBytes = kParkRow * 4 + 8;       // a row and its two scalars
-  static constexpr int kParkTotal = 2 * BMH * kParkRowBytes;
-  static constexpr int kRecvOffset = kParkTotal;
-  static_assert(kParkTotal % 16 == 0 && kParkTotal + BMH * kParkRowBytes <= kBarOffset, "parked partial + one share of 128 rows");
-  // shares of 256 / C rows that fit behind the parked partial, at most C - 1
-  __host__ __device__ static constexpr int pushed_shares(int c) {
-    const int fit = (kBarOffset - kRecvOffset) / ((2 * BMH / c) * kParkRowBytes);
-    return fit < c - 1 ? fit : c - 1;
-  }
+  static constexpr int kSpillRowBytes = D * 4 + 8;             // the same in the workspace: rows of D floats (whole 32-byte sectors)
+  static_assert(BMH * kParkRowBytes <= kBarOffset, "a share of 128 rows fits in front of the barriers");
 };
 
 // Trace tags (see dyspec_set_trace): tag = role << 14 | event << 10 | key-tile index j.
@@ -80,7 +72,7 @@ struct TcLayout {
 // barrier indices (8 bytes each)
 enum { B_QFULL = 0, B_QFREE = 1, B_SLOT_FULL = 2, B_SLOT_EMPTY = B_SLOT_FULL + kSlots,
        B_SREADY = B_SLOT_EMPTY + kSlots, B_PREADY = B_SREADY + 2, B_ODONE = B_PREADY + 2, B_OFREE = B_ODONE + 2,
-       B_PVDONE = B_OFREE + 2, B_QFULLB = B_PVDONE + 2, B_RECV = B_QFULLB + 1, B_COUNT = B_RECV + 1 };
+       B_PVDONE = B_OFREE + 2, B_QFULLB = B_PVDONE + 2, B_COUNT = B_QFULLB + 1 };
 
 // Hardware named barriers for thread-to-thread hand-offs inside the CTA (P ready: 128 softmax threads
 // -> the MMA-issuing warp): an order of magnitude quicker to notice than an mbarrier in shared memory
@@ -298,7 +290,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   if (threadIdx.x == 0) {
     mbar_init(bar(B_QFULL), 1);
     mbar_init(bar(B_QFULLB), 1);
-    mbar_init(bar(B_RECV), 1);             // cluster plans: the peers' shares pushed into this CTA have landed
     mbar_init(bar(B_QFREE), 2);
     for (int s = 0; s < kSlots; ++s) {
       mbar_init(bar(B_SLOT_FULL + s), 1);
@@ -386,14 +377,35 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   const int g = p.group_size;
   // Cluster plans: where packed row pr of the parked partial lies (share pr / rows, rows = 256 / C), in bytes
   // from the start of shared memory: the row itself, and its maximum (its sum is 4 * rows bytes further).
+  // Cluster plans: share d of this CTA's partial (the rows CTA d of the cluster merges) stays in shared memory
+  // when d is this CTA, else it goes to slot (rank - d) mod C - 1 of CTA d's C - 1 slots in the workspace
+  // (p.partial), from where d reads it through L2.
   const int park_log2rows = 8 - (p.cluster_size >= 8 ? 3 : p.cluster_size >= 4 ? 2 : 1);
-  auto park_row_at = [&](int pr) -> int {
-    const int rows = 1 << park_log2rows;
-    return (pr >> park_log2rows) * rows * L::kParkRowBytes + (pr & (rows - 1)) * (L::kParkRow * 4);
-  };
-  auto park_max_at = [&](int pr) -> int {
-    const int rows = 1 << park_log2rows;
-    return (pr >> park_log2rows) * rows * L::kParkRowBytes + rows * (L::kParkRow * 4) + (pr & (rows - 1)) * 4;
+  const uint32_t cl_rank = p.cluster_size > 1 ? cluster_ctarank() : 0u;
+  // Writes packed row pr (D fp32 values as bit patterns), its maximum and its sum where they belong.  Rows in the
+  // workspace are D floats apart and written with 32-byte stores: whole sectors, which L2 takes without
+  // first fetching them from memory.
+  auto park_row = [&](int pr, const uint32_t* vals, float m_row, float l_row) {
+    const int rows = 1 << park_log2rows, d = pr >> park_log2rows, lr = pr & (rows - 1);
+    const int src_no = (int(cl_rank) - d) & (p.cluster_size - 1);
+    if (src_no > 0) {
+      uint8_t* base = reinterpret_cast<uint8_t*>(p.partial) +
+                      (size_t(blockIdx.x - cl_rank + uint32_t(d)) * size_t(p.cluster_size - 1) + size_t(src_no - 1)) * size_t(rows * L::kSpillRowBytes);
+      float* row_at = reinterpret_cast<float*>(base) + lr * D;
+#pragma unroll
+      for (int i = 0; i < D / 8; ++i) st_global_v8(row_at + 8 * i, vals + 8 * i);
+      float* max_at = reinterpret_cast<float*>(base) + rows * D + lr;
+      max_at[0] = m_row;
+      max_at[rows] = l_row;
+    } else {
+      const uint32_t base = s_q;                           // (ld.shared / st.shared by 32-bit address: the compiler cannot tell that `smem` is shared)
+      const uint32_t row_at = base + uint32_t(lr * (L::kParkRow * 4));
+#pragma unroll
+      for (int i = 0; i < D / 4; ++i) st_shared_v4(row_at + 16u * uint32_t(i), vals[4 * i], vals[4 * i + 1], vals[4 * i + 2], vals[4 * i + 3]);
+      const uint32_t max_at = base + uint32_t(rows * (L::kParkRow * 4) + 4 * lr);
+      st_shared_f32(max_at, m_row);
+      st_shared_f32(max_at + uint32_t(4 * rows), l_row);
+    }
   };
 
   // Register budget: the softmax threads hold a whole S row; the control warps need few registers.
@@ -610,7 +622,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       }
     }
   }
-  // cluster plans: "every CTA has parked its partial" (the softmax threads arrive once theirs is written)
+  // cluster plans: "every CTA has written its partial" (the softmax threads arrive once theirs is out; the
+  // hardware barrier counts every thread of the cluster, these warps included)
   if (p.cluster_size > 1) {
     __syncwarp();
     cluster_arrive();
@@ -676,12 +689,11 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         if (p.cluster_size > 1) {                          // cluster plan: the peers read this half's rows all the same
           named_sync(kBarMerge, 2 * BMH);                  // (the other half's products no longer read the Q tile and the ring)
           const int pr = h * BMH + r;
-          uint8_t* row_at = smem + park_row_at(pr);
+          need_dep();                                      // (shares go to the workspace)
+          uint32_t zeros[D];
 #pragma unroll
-          for (int i = 0; i < D / 4; ++i) *reinterpret_cast<float4*>(row_at + 16 * i) = make_float4(0.f, 0.f, 0.f, 0.f);
-          *reinterpret_cast<float*>(smem + park_max_at(pr)) = -INFINITY;
-          *reinterpret_cast<float*>(smem + park_max_at(pr) + (4 << park_log2rows)) = 0.f;
-          fence_proxy_async();                             // (bulk copies read the parked rows)
+          for (int i = 0; i < D; ++i) zeros[i] = 0u;
+          park_row(pr, zeros, -INFINITY, 0.f);
         }
         continue;
       }
@@ -868,13 +880,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         mbar_arrive(bar(B_OFREE + h));
         named_sync(kBarMerge, 2 * BMH);                    // both halves' products are done: Q tile and ring are idle
         const int pr = h * BMH + r;
-        uint8_t* row_at = smem + park_row_at(pr);
-#pragma unroll
-        for (int i = 0; i < D / 4; ++i)
-          *reinterpret_cast<uint4*>(row_at + 16 * i) = make_uint4(ov[4 * i], ov[4 * i + 1], ov[4 * i + 2], ov[4 * i + 3]);
-        *reinterpret_cast<float*>(smem + park_max_at(pr)) = m_used;
-        *reinterpret_cast<float*>(smem + park_max_at(pr) + (4 << park_log2rows)) = l;
-        fence_proxy_async();                               // (bulk copies read the parked rows)
+        park_row(pr, ov, m_used, l);                       // shared memory, or the owner's slot in the workspace
       } else if (item.slot < 0 && staged) {
         const float inv = l > 0.f ? 1.f / l : 0.f;
         uint32_t ov[D];
@@ -1166,19 +1172,18 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     }
     // ---- split-KV merge of a cluster plan: the CTAs of a cluster hold the pieces of one (request, kv head,
     // query tile) group, one item each, and CTA k merges rows [k * 256 / C, (k + 1) * 256 / C) of the C
-    // partials.  Once every CTA has parked its partial (cluster barrier: every CTA's products are done, so
-    // its shared memory can also take what the peers send), each CTA pushes its shares of some peers' rows
-    // into those peers with bulk copies (as many as fit behind a parked partial) and fetches the remaining
-    // peers' shares of its own rows with plain loads of their shared memory, which are far slower per byte
-    // but need no room.  Nothing goes through global memory, and there is no counter to wait on.  A second
-    // cluster barrier (below, all threads) keeps every CTA's shared memory alive until its peers are done.
+    // partials.  Every CTA has kept its own share of those rows in shared memory and written its shares of the
+    // peers' rows to their slots in the workspace; the cluster barrier (release / acquire) makes all of it
+    // visible, so there are no arrival counters, no fences and no polling, and the slowest CTA of the cluster
+    // is the only thing anybody waits for.  The peers' shares come back through L2: shared-to-shared copies
+    // between the CTAs (bulk pushes, or loads of a peer's shared memory) were built and measured first and
+    // were no quicker -- a CTA moves about 27 GB/s that way, and loads with one row per lane far less.
     if constexpr (!kDyn) {
       if (p.cluster_size > 1) {
         const int tid = h * BMH + r;
-        const uint32_t rank = cluster_ctarank();
-        const uint32_t park_u32 = smem_u32(smem);
+        const uint32_t rank = cl_rank;
         __syncwarp();
-        cluster_arrive_release();                          // this thread's parked values are written
+        cluster_arrive_release();                          // this thread's parked and spilled values are written
         cluster_wait();
         stamp(6);
         const WorkItem item = item_of(0, 0);
@@ -1187,71 +1192,70 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         auto merge = [&](auto c_tag) {
           constexpr int C = decltype(c_tag)::value;
           constexpr int kRows = 2 * BMH / C;               // rows per CTA
-          constexpr int kShare = kRows * L::kParkRowBytes; // bytes of a share
-          constexpr int NP = L::pushed_shares(C);          // peers whose shares of my rows are pushed to me
-          constexpr int V = D / 32;                        // floats per lane: a warp reads one whole parked row per load
+          constexpr int V = D / 32;                        // floats per lane: a warp reads one whole row per load
           constexpr int KR = 4;                            // rows per warp and pass
-          // Slot j of this CTA's receive area is filled by CTA (rank + 1 + j) % C, i.e. this CTA sends its share
-          // of CTA d's rows to slot j of d = (rank - 1 - j) mod C.  Four lanes per copy, so that the copies overlap.
-          if (tid == 0) mbar_expect_tx(bar(B_RECV), uint32_t(NP * kShare));
-          if (tid < 4 * NP) {
-            const uint32_t j = uint32_t(tid) >> 2, piece = uint32_t(tid) & 3u;
-            const uint32_t d = (rank + uint32_t(2 * C - 1) - j) % uint32_t(C);
-            constexpr uint32_t part = uint32_t(kShare / 4);          // a multiple of 16 bytes for every C and D
-            dsmem_push(map_to_cta(park_u32 + uint32_t(L::kRecvOffset) + j * uint32_t(kShare) + piece * part, d),
-                       park_u32 + d * uint32_t(kShare) + piece * part, part, map_to_cta(bar(B_RECV), d));
-          }
+          constexpr int NR = C - 1;                        // sources in the workspace (source 0 is this CTA's own share)
+          constexpr int kSpill = kRows * L::kSpillRowBytes;   // bytes of a share in the workspace
           const int mw = tid >> 5, lk = lane >> 3, lu = lane & 7;
-          // the sources of my rows: 0 = my own parked share, 1 .. NP = the receive slots, above = peers' shared memory
-          const uint8_t* own_share = smem + int(rank) * kShare;
-          const uint8_t* recv = smem + L::kRecvOffset;
-          uint32_t remote[C];                              // (entries up to NP are unused)
-#pragma unroll
-          for (int s_ = NP + 1; s_ < C; ++s_)
-            remote[s_] = map_to_cta(park_u32 + rank * uint32_t(kShare), (rank + uint32_t(s_)) % uint32_t(C));
-          if (NP > 0) mbar_wait(bar(B_RECV), 0, abort_flag, p.status);
-          // A pass: KR rows per warp.  Lane 8 k + u fetches (m, l) of row k from source u; every lane fetches its V
-          // columns of the KR rows from all C sources, all requested before anything is used.  (Loads of a peer's
-          // shared memory are slow when a warp's lanes ask for 32 different rows; one row per request is not.)
-          for (int r0 = KR * mw; r0 < kRows; r0 += 8 * KR) {
-            float mv = -INFINITY, lv = 0.f;
-            if (lu < C) {
-              const int at = kRows * (L::kParkRow * 4) + 4 * (r0 + lk);
-              if (lu <= NP) {
-                const uint8_t* src = lu == 0 ? own_share : recv + (lu - 1) * kShare;
-                mv = *reinterpret_cast<const float*>(src + at);
-                lv = *reinterpret_cast<const float*>(src + at + 4 * kRows);
-              } else {
-                const uint32_t src = map_to_cta(park_u32 + rank * uint32_t(kShare), (rank + uint32_t(lu)) % uint32_t(C));
-                mv = ld_dsmem_f32(src + uint32_t(at));
-                lv = ld_dsmem_f32(src + uint32_t(at + 4 * kRows));
-              }
+          const float* spilled = reinterpret_cast<const float*>(reinterpret_cast<const uint8_t*>(p.partial) +
+                                                               size_t(blockIdx.x) * size_t(NR) * size_t(kSpill));
+          // This code runs once per CTA, so the loop over the passes stays rolled.  A pass: KR rows per warp; lane
+          // 8 k + u holds (m, l) of row k from source u; every lane its V columns of the KR rows from all C
+          // sources, all requested before anything is used, the workspace's one pass ahead.
+          constexpr int kPasses = kRows / (8 * KR);
+          static_assert(kRows % (8 * KR) == 0, "whole passes");
+          float nvv[KR][NR][V], nmv = -INFINITY, nlv = 0.f;           // the next pass's values from the workspace
+          auto fetch_spilled = [&](int r0) {
+            nmv = -INFINITY;
+            nlv = 0.f;
+            if (lu > 0 && lu < C) {
+              const float* sc_ = spilled + (lu - 1) * (kSpill / 4) + kRows * D + r0 + lk;
+              nmv = ld_cg_f32(sc_);
+              nlv = ld_cg_f32(sc_ + kRows);
             }
+#pragma unroll
+            for (int k = 0; k < KR; ++k)
+#pragma unroll
+              for (int q = 0; q < NR; ++q) {
+                const float* at = spilled + q * (kSpill / 4) + (r0 + k) * D + lane * V;
+                if constexpr (V == 4) {
+                  const float4 x = ld_cg_f32x4(at);
+                  nvv[k][q][0] = x.x; nvv[k][q][1] = x.y; nvv[k][q][2] = x.z; nvv[k][q][3] = x.w;
+                } else {
+                  const float2 x = ld_cg_f32x2(at);
+                  nvv[k][q][0] = x.x; nvv[k][q][1] = x.y;
+                }
+              }
+          };
+          fetch_spilled(KR * mw);
+#pragma unroll 1
+          for (int ps = 0; ps < kPasses; ++ps) {
+            const int r0 = KR * mw + ps * 8 * KR;
+            float mv = nmv, lv = nlv;
             float vv[KR][C][V];
 #pragma unroll
             for (int k = 0; k < KR; ++k)
 #pragma unroll
-              for (int s_ = 0; s_ < C; ++s_) {
-                const int at = (r0 + k) * (L::kParkRow * 4) + lane * (4 * V);
-                if (s_ <= NP) {
-                  const uint8_t* src = (s_ == 0 ? own_share : recv + (s_ - 1) * kShare) + at;
-                  if constexpr (V == 4) {
-                    const float4 x = *reinterpret_cast<const float4*>(src);
-                    vv[k][s_][0] = x.x; vv[k][s_][1] = x.y; vv[k][s_][2] = x.z; vv[k][s_][3] = x.w;
-                  } else {
-                    const float2 x = *reinterpret_cast<const float2*>(src);
-                    vv[k][s_][0] = x.x; vv[k][s_][1] = x.y;
-                  }
-                } else {
-                  if constexpr (V == 4) {
-                    const float4 x = ld_dsmem_f32x4(remote[s_] + uint32_t(at));
-                    vv[k][s_][0] = x.x; vv[k][s_][1] = x.y; vv[k][s_][2] = x.z; vv[k][s_][3] = x.w;
-                  } else {
-                    const float2 x = ld_dsmem_f32x2(remote[s_] + uint32_t(at));
-                    vv[k][s_][0] = x.x; vv[k][s_][1] = x.y;
-                  }
-                }
+              for (int q = 0; q < NR; ++q)
+#pragma unroll
+                for (int e = 0; e < V; ++e) vv[k][1 + q][e] = nvv[k][q][e];
+            if (ps + 1 < kPasses) fetch_spilled(r0 + 8 * KR);
+            if (lu == 0) {                                 // this CTA's own share: shared memory
+              const uint32_t at = s_q + uint32_t(kRows * (L::kParkRow * 4) + 4 * (r0 + lk));
+              mv = ld_shared_f32(at);
+              lv = ld_shared_f32(at + uint32_t(4 * kRows));
+            }
+#pragma unroll
+            for (int k = 0; k < KR; ++k) {
+              const uint32_t src = s_q + uint32_t((r0 + k) * (L::kParkRow * 4) + lane * (4 * V));
+              if constexpr (V == 4) {
+                const float4 x = ld_shared_f32x4(src);
+                vv[k][0][0] = x.x; vv[k][0][1] = x.y; vv[k][0][2] = x.z; vv[k][0][3] = x.w;
+              } else {
+                const float2 x = ld_shared_f32x2(src);
+                vv[k][0][0] = x.x; vv[k][0][1] = x.y;
               }
+            }
             float m_r = mv;
             m_r = fmaxf(m_r, __shfl_xor_sync(0xffffffffu, m_r, 1));
             m_r = fmaxf(m_r, __shfl_xor_sync(0xffffffffu, m_r, 2));
@@ -1288,7 +1292,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
               }
             }
           }
-          if (tid < 4 * NP) dsmem_push_wait_source_read();    // the parked rows must outlive the copies that read them
         };
         if (p.cluster_size == 2) merge(std::integral_constant<int, 2>{});
         else if (p.cluster_size == 4) merge(std::integral_constant<int, 4>{});
@@ -1298,12 +1301,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     stamp(7);
   }
 
-  // cluster plans: no CTA leaves (its shared memory with it) before its peers have fetched what they need
-  if (p.cluster_size > 1) {
-    __syncwarp();
-    cluster_arrive_release();
-    cluster_wait();
-  }
   tc_fence_before();
   __syncthreads();
   if (warp == 2) {
@@ -1322,6 +1319,13 @@ cudaError_t launch_one(cudaLaunchConfig_t& cfg, size_t smem, const CUtensorMap& 
   return cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<D, kDyn, kInPages>, mq, mk, mv, p, first);
 }
 }  // namespace
+
+// Workspace bytes per CTA of a cluster plan: its peers' shares of the rows it merges.
+size_t attn_tc_cluster_workspace_per_cta(int head_dim, int cluster_size) {
+  if (cluster_size < 2) return 0;
+  const int row_bytes = head_dim == 128 ? TcLayout<128>::kSpillRowBytes : TcLayout<64>::kSpillRowBytes;
+  return size_t(cluster_size - 1) * size_t(2 * BMH / cluster_size) * size_t(row_bytes);
+}
 
 // How many clusters of `cluster_size` CTAs of this kernel the current device can hold at once (0: such a
 // cluster cannot be launched at all, e.g. on a reduced share of the SMs); -1 when that cannot be asked

@@ -394,17 +394,17 @@ def test_merge_inside_the_tensor_core_kernel(rt, hq, hkv, d, L, n, ctas):
 @pytest.mark.parametrize("hq,hkv,d,L,n,want_c", [(8, 8, 128, 2000, 256, 8), (16, 16, 128, 1500, 200, 4), (64, 64, 64, 700, 130, 2),
                                                  (8, 1, 128, 3000, 12, 8), (32, 4, 64, 1000, 64, 4)])
 def test_cluster_merge_in_the_tensor_core_regime(rt, hq, hkv, d, L, n, want_c):
-    """Few groups of equal length: one thread-block cluster per group, every CTA parks its partial in shared
-    memory and fetches its share of the rows from its peers.  Cluster sizes 2, 4 and 8, both head dimensions,
-    a ragged second half, a group with one half only (the other half parks neutral rows), GQA.  No workspace,
-    no second launch; a second call on the same buffers gives the same bits."""
+    """Few groups of equal length: one thread-block cluster per group, every CTA merges its share of the rows
+    once the cluster's barrier says that all partials are written.  Cluster sizes 2, 4 and 8, both head dimensions,
+    a ragged second half, a group with one half only (the other half parks neutral rows), GQA.  No second
+    launch, no counters; a second call on the same buffers gives the same bits."""
     B, R = rt
     rng = np.random.default_rng(hq * 100 + n)
     w = wl.make_custom(75, hq, hkv, d, [L], [wl.greedy_tree(rng, n, 6, 0.3)])
     batch, got, _ = run_and_check(rt, w, regime=1)
     info = batch.plan.describe()
     assert info["regime"] == 1 and info["cluster"] == want_c and info["combine_launch"] == 0, info
-    assert batch.plan.workspace_bytes() == 0
+    assert batch.plan.workspace_bytes() > 0                          # the peers' shares travel through the workspace
     batch.out.zero_()
     batch.attention()
     _, _, out2, status = batch.results()

@@ -15,6 +15,12 @@ def B():
     return binding
 
 
+def cluster_workspace_per_cta(d, c):
+    """Tensor-core regime, cluster of c CTAs: a CTA merges 256 / c rows and gets its c - 1 peers' shares of them
+    through the workspace (a row: d floats and two scalars)."""
+    return (c - 1) * (256 // c) * (d * 4 + 8)
+
+
 def check_schedule(B, hq, hkv, d, Ls, ns, regime=-1, ctas=0, fuse=2):
     B.dyspec_set_tuning(regime, ctas, fuse)
     try:
@@ -62,6 +68,8 @@ def check_schedule(B, hq, hkv, d, Ls, ns, regime=-1, ctas=0, fuse=2):
     pad = lambda x: (x + 255) & ~255
     n_split = len([1 for pieces in covered.values() if len(pieces) > 1]) if info["cluster"] == 1 else 0
     want = len(slots) * bm * (d + 2) * 4
+    if info["cluster"] > 1 and info["regime"] == 1:
+        want = info["ctas"] * cluster_workspace_per_cta(d, info["cluster"])
     if n_split:
         want = pad(want) + pad(8 * n_split)
     if queue:
@@ -138,7 +146,7 @@ def test_whole_group_plan_is_chosen_when_cheaper(B):
     info3, loads3 = check_schedule(B, *args3)
     # few long groups of equal length: one cluster of 4 CTAs per group, merged through distributed shared memory
     assert info3["cluster"] == 4 and info3["split_groups"] == 0 and info3["ctas"] == 128 == info3["items"]
-    assert max(loads3) == 9 and info3["workspace_bytes"] == 0 and info3["combine_launch"] == 0
+    assert max(loads3) == 9 and info3["workspace_bytes"] == 128 * 3 * 64 * 520 and info3["combine_launch"] == 0   # three peers' shares per CTA
     # without clusters: even pieces, one per CTA, on as many CTAs as there are SMs (20 groups in 5, 12 in 4),
     # merged inside the kernel through the workspace
     info3e, loads3e = check_schedule(B, *args3, fuse=1)
@@ -175,12 +183,14 @@ def test_merge_in_kernel_only_when_the_grid_is_one_wave(B):
 
 def test_cluster_plans_of_the_tensor_core_regime(B):
     """Few groups of similar length in the tensor-core regime: one cluster of C CTAs per group (C the same
-    for all groups, at least two tiles per piece, all CTAs in one wave), no workspace; merge mode 1 keeps the
+    for all groups, at least two tiles per piece, all CTAs in one wave), a workspace for the peers' shares but no
+    counters; merge mode 1 keeps the
     merge through the workspace; too many groups, or groups too short, get no clusters."""
     for shape, want in (((8, 8, 128, [2000], [256]), 8), ((16, 16, 128, [1500], [200]), 4), ((64, 64, 64, [700], [130]), 2),
                         ((8, 1, 128, [3000], [12]), 8)):
         info, loads = check_schedule(B, *shape, regime=1)
-        assert info["cluster"] == want and info["workspace_bytes"] == 0 and info["combine_launch"] == 0, (shape, info)
+        assert info["cluster"] == want and info["combine_launch"] == 0, (shape, info)
+        assert info["workspace_bytes"] == info["ctas"] * cluster_workspace_per_cta(shape[2], want)
         assert info["ctas"] == info["groups"] * want and min(loads) >= 2 and max(loads) - min(loads) <= 1
         never = check_schedule(B, *shape, regime=1, fuse=1)[0]
         assert never["cluster"] == 1 and never["combine_launch"] == 0
