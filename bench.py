@@ -35,7 +35,7 @@ UNIT = "tree tokens/s"
 L2_BYTES = 126 * 1024 * 1024
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu
 # captures summarised under profiles/ (tree_attn_small_c2_*.md, tree_attn_tc_c3_*.md, ..._c4_*.md, ..._c5_*.md)
-NCU_TRAFFIC_BYTES = {"c2_llama2_7b_L1024_n64": 18411264, "c3_llama2_7b_L4096_n256": 74971136,
+NCU_TRAFFIC_BYTES = {"c2_llama2_7b_L1024_n64": 18411264, "c3_llama2_7b_L4096_n256": 77289216,
                      "c4_llama2_70b_L2048_n512": 18981120, "c5_ragged8_llama2_70b": 154391040}
 NOMINAL_HBM_GBS, NOMINAL_BF16_TFLOPS = 8000.0, 2250.0
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
