@@ -50,6 +50,7 @@ cudaError_t launch_attn_small(int head_dim, int n_ctas, const CUtensorMap& mq, c
                             const AttnParams& p, const WorkItem* host_items, cudaStream_t stream);
 cudaError_t launch_combine(int head_dim, int bm, int n_split_groups, const AttnParams& p, cudaStream_t stream);
 int attn_tc_max_clusters(int head_dim, int cluster_size);
+int attn_small_max_clusters(int head_dim, int cluster_size);
 size_t attn_tc_cluster_workspace_per_cta(int head_dim, int cluster_size);
 cudaError_t launch_attn_tc(int head_dim, int n_ctas, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                            const AttnParams& p, const WorkItem* host_items, cudaStream_t stream);
@@ -191,6 +192,7 @@ struct dyspec_plan {
   size_t queue_offset = 0;              // dynamic plans: byte offset of the two queue words inside the caller's workspace
   size_t counters_offset = 0;           // plans with split groups: byte offset of the groups' counter pairs in the workspace
   bool merge_in_kernel = false;         // tensor-core regime: split groups are merged by their own items, no combine launch
+  int cluster_fit[9] = {-1, -1, -1, -1, -1, -1, -1, -1, -1};   // clusters of C CTAs of the regime's kernel the device holds at once (-1: not known)
   std::vector<WorkItem> items_queue;    // dynamic plans: all items in queue order
   size_t workspace_bytes = 0;
 };
@@ -250,6 +252,7 @@ void schedule(dyspec_plan& pl) {
     const double mean_tiles = double(total_tiles) / double(groups.size());
     for (int C : {8, 4, 2}) {
       if (int64_t(groups.size()) * C > kNumSMs) continue;
+      if (pl.cluster_fit[C] >= 0 && int64_t(groups.size()) > pl.cluster_fit[C]) continue;   // all clusters at once, or none
       if (mean_tiles / C < 2.0 || double(max_tiles) > 1.3 * mean_tiles) continue;
       bool ok = true;
       for (const Group& gr : groups) ok = ok && gr.tiles >= C;
@@ -539,6 +542,9 @@ void schedule(dyspec_plan& pl) {
       int64_t best_cost = cost_plan;
       for (int C : {8, 4, 2}) {
         if (int64_t(groups.size()) * C > max_ctas || min_tiles_g < 2 * C) continue;
+        // all clusters at once (the SMs of a cluster come from one GPC, so fewer fit than SMs / C): the ones
+        // left over would run as a second wave
+        if (pl.cluster_fit[C] >= 0 && int64_t(groups.size()) > pl.cluster_fit[C]) continue;
         const int64_t cost = (max_tiles + C - 1) / C + item_cost_ + 1;
         if (cost < best_cost) { best_cost = cost; best_c = C; }
       }
@@ -896,12 +902,20 @@ static int make_host_plan(dyspec_plan** out, int n_q_heads, int n_kv_heads, int 
   pl->regime = pl->tune.force_regime >= 0 ? pl->tune.force_regime : (max_rows > 64 ? 1 : 0);
   pl->bm = pl->regime == 0 ? 64 : 256;    // packed query rows per work item (regime 1: two 128-row halves)
   pl->bn = pl->regime == 0 ? 64 : 128;    // keys per tile
+  if (pl->tune.combine_mode == 2)
+    for (int C : {2, 4, 8})
+      pl->cluster_fit[C] = pl->regime == 1 ? attn_tc_max_clusters(pl->d, C) : attn_small_max_clusters(pl->d, C);
   schedule(*pl);
   // A cluster plan of the tensor-core regime needs C CTAs of 1 CTA / SM side by side: where the device cannot
   // hold even one such cluster (a reduced share of its SMs), plan again without clusters.
-  if (pl->regime == 1 && pl->cluster > 1 && attn_tc_max_clusters(pl->d, pl->cluster) == 0) {
-    pl->tune.combine_mode = 1;
-    schedule(*pl);
+  // (The same when the device cannot hold all of the plan's clusters at once -- the SMs of a cluster have to
+  //  come from one GPC -- since the clusters left over would run as a second wave.)
+  if (pl->regime == 1 && pl->cluster > 1) {
+    const int fit = attn_tc_max_clusters(pl->d, pl->cluster);
+    if (fit >= 0 && fit < pl->n_ctas / pl->cluster) {
+      pl->tune.combine_mode = 1;
+      schedule(*pl);
+    }
   }
   pl->workspace_bytes = size_t(pl->n_slots) * size_t(pl->bm) * (pl->d + 2) * sizeof(float);
   if (pl->regime == 1 && pl->cluster > 1)   // cluster plan: the shares a CTA's peers cannot push into its shared memory

@@ -790,6 +790,45 @@ size_t attn_small_smem_bytes(int head_dim) {
 }
 int attn_small_threads() { return kThreads; }
 
+// How many clusters of `cluster_size` CTAs of this kernel the current device can hold at once (the SMs of a
+// cluster come from one GPC, so fewer than SMs / cluster_size); -1 when that cannot be asked (no device).
+// Asked once per (device, head dimension, cluster size).
+int attn_small_max_clusters(int head_dim, int cluster_size) {
+  static std::atomic<int> cache[DynSmemGrant::kDevices][2][4];
+  static std::atomic<bool> init{false};
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= DynSmemGrant::kDevices) { cudaGetLastError(); return -1; }
+  if (!init.exchange(true))
+    for (auto& d : cache) for (auto& h : d) for (auto& c : h) c.store(-2);
+  const int hi = head_dim == 128 ? 0 : 1, ci = cluster_size == 8 ? 3 : cluster_size == 4 ? 2 : cluster_size == 2 ? 1 : 0;
+  const int have = cache[dev][hi][ci].load();
+  if (have != -2) return have;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = unsigned(cluster_size);
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(unsigned(cluster_size));
+  cfg.blockDim = dim3(unsigned(kThreads));
+  cfg.dynamicSmemBytes = attn_small_smem_bytes(head_dim);
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  int n = 0;
+  static DynSmemGrant grant[2];
+  cudaError_t e;
+  if (head_dim == 128) {
+    e = grant[0].ensure(tree_attn_small_kernel<128>, cfg.dynamicSmemBytes);
+    if (e == cudaSuccess) e = cudaOccupancyMaxActiveClusters(&n, tree_attn_small_kernel<128>, &cfg);
+  } else {
+    e = grant[1].ensure(tree_attn_small_kernel<64>, cfg.dynamicSmemBytes);
+    if (e == cudaSuccess) e = cudaOccupancyMaxActiveClusters(&n, tree_attn_small_kernel<64>, &cfg);
+  }
+  if (e != cudaSuccess) { cudaGetLastError(); n = 0; }
+  cache[dev][hi][ci].store(n);
+  return n;
+}
+
 cudaError_t launch_attn_small(int head_dim, int n_ctas, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                             const AttnParams& p, const WorkItem* host_items, cudaStream_t stream) {
   // host_items: the host copy of p.items (same stride); each CTA's first item travels as a kernel parameter
