@@ -248,8 +248,8 @@ int dyspec_release_cache(void);
  *   - A batch whose work list plus partials exceed the array is refused with DYSPEC_ERR_WORKSPACE
  *     before anything is launched (as a guide: Llama2-70B shape, prefix 1500, 40 nodes needs 12.2 MiB;
  *     small uniform batches that merge their splits on chip need only a few KiB).
- *   - The first call on each device looks up the array's device address (with that device current);
- *     make that first call outside any stream capture.
+ *   - The first call on each device looks up the array's device address (with that device current), a
+ *     synchronous call of the CUDA runtime; later calls on that device do not.
  *   - All calls share the one array, which keeps the previous call's contents; each call rewrites the
  *     tables and clears the counters it needs.  Calls on the same stream are ordered and safe.  Two
  *     calls that overlap on the GPU (different streams, or different host threads without ordering)
