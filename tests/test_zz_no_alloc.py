@@ -39,7 +39,11 @@ def test_static_scratch_entry_point_matches_ragged_entry_point_twice_in_a_row():
     # ... and one request with more (kv head, query tile) groups than CTAs: through a plan it runs from
     # the shared queue in the caller's workspace, here (no workspace) from fixed lists
     many = wl.make_custom(22, 64, 8, 128, [200], [wl.greedy_tree(rng, 1024, 8, 0.3)])
-    cases = [big, wl.make_custom(21, 8, 2, 64, [300], [wl.greedy_tree(rng, 40, 4, 0.3)]), wl.make_config(2), many, big]
+    # ... and a shape that runs as one thread-block cluster per group in the tensor-core regime (its CTAs' shares
+    # of the partials go through the scratch array, 7.5 MiB here)
+    clustered = wl.make_custom(23, 8, 8, 128, [2000], [wl.greedy_tree(rng, 256, 8, 0.3)])
+    cases = [big, wl.make_custom(21, 8, 2, 64, [300], [wl.greedy_tree(rng, 40, 4, 0.3)]), wl.make_config(2), many,
+             clustered, big]
     from oracle import dyspec_oracle as orc
     for w in cases:
         batch = R.DeviceBatch(w)
@@ -47,6 +51,8 @@ def test_static_scratch_entry_point_matches_ragged_entry_point_twice_in_a_row():
         bits, _, want_bits, status = batch.results()
         assert status == 0
         assert batch.plan.describe()["dynamic"] == (1 if w is many else 0)
+        if w is clustered:
+            assert batch.plan.describe()["regime"] == 1 and batch.plan.describe()["cluster"] == 8
         L, n = int(w.prefix_len[0]), int(w.n_nodes[0])
         out = torch.zeros_like(batch.out)
         st = torch.zeros((1,), dtype=torch.int32, device=out.device)
